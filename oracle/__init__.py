@@ -1,0 +1,159 @@
+"""CPU oracle for Dynamic Mask Attention: thin ctypes access to ``dma_oracle.cpp``.
+
+TEST INFRASTRUCTURE ONLY: imported by the tests, by the smoke check and by the benchmark's
+CPU-baseline leg. The product package never imports it and it never imports the product package.
+Arrays are numpy, contiguous, in the layouts documented at the top of ``dma_oracle.cpp``.
+"""
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_DIR = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_DIR, "dma_oracle.cpp")
+_LIB = os.path.join(_DIR, "libdma_oracle.so")
+_lib = None
+
+
+def build(force=False):
+    """Compile the oracle with g++ (no fast-math, no fp contraction: delta-v1 needs exact IEEE ops)."""
+    if not force and os.path.exists(_LIB) and os.path.getmtime(_LIB) >= os.path.getmtime(_SRC):
+        return _LIB
+    cmd = ["g++", "-std=c++17", "-O2", "-fopenmp", "-ffp-contract=off", "-fno-fast-math", "-shared", "-fPIC",
+           _SRC, "-o", _LIB + ".tmp"]
+    subprocess.check_call(cmd)
+    os.replace(_LIB + ".tmp", _LIB)
+    return _LIB
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        _lib = ctypes.CDLL(build())
+        for n in ("dmao_exp_spec", "dmao_log1p_spec", "dmao_softplus_spec"):
+            getattr(_lib, n).restype = ctypes.c_float
+            getattr(_lib, n).argtypes = [ctypes.c_float]
+    return _lib
+
+
+def threads():
+    """Number of OpenMP threads the oracle uses (OMP_NUM_THREADS, else all cores)."""
+    v = os.environ.get("OMP_NUM_THREADS")
+    return int(v) if v else os.cpu_count()
+
+
+def _p(a):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _c(a, dt):
+    return None if a is None else np.ascontiguousarray(a, dtype=dt)
+
+
+def exp_spec(x):
+    return lib().dmao_exp_spec(float(np.float32(x)))
+
+
+def log1p_spec(t):
+    return lib().dmao_log1p_spec(float(np.float32(t)))
+
+
+def softplus_spec(z):
+    return lib().dmao_softplus_spec(float(np.float32(z)))
+
+
+def delta(V, W, A, Hq):
+    """V [B,L,Hkv,d], W [Hq,d], A [Hq] (values exactly representable in fp32) -> (z, delta) [B,Hq,L] fp32."""
+    V = _c(V, np.float32); W = _c(W, np.float32); A = _c(A, np.float32)
+    B, L, Hkv, d = V.shape
+    z = np.empty((B, Hq, L), np.float32)
+    dl = np.empty((B, Hq, L), np.float32)
+    rc = lib().dmao_delta(_p(V), _p(W), _p(A), B, L, Hq, Hkv, d, _p(z), _p(dl))
+    assert rc == 0, rc
+    return z, dl
+
+
+def select_definition(dl, w):
+    """delta [..., L] -> keep [..., L, L] uint8 by the per-row sort definition."""
+    dl = _c(dl, np.float32)
+    L = dl.shape[-1]
+    BH = dl.size // L
+    keep = np.empty(dl.shape + (L,), np.uint8)
+    assert lib().dmao_select_definition(_p(dl), BH, L, int(w), _p(keep)) == 0
+    return keep
+
+
+def select_expiry(dl, w):
+    """delta [..., L] -> expiry [..., L] int32: key j is kept by rows j <= i < expiry[j]."""
+    dl = _c(dl, np.float32)
+    L = dl.shape[-1]
+    e = np.empty(dl.shape, np.int32)
+    assert lib().dmao_select_expiry(_p(dl), dl.size // L, L, int(w), _p(e)) == 0
+    return e
+
+
+def keep_from_expiry(e):
+    e = _c(e, np.int32)
+    L = e.shape[-1]
+    keep = np.empty(e.shape + (L,), np.uint8)
+    assert lib().dmao_keep_from_expiry(_p(e), e.size // L, L, _p(keep)) == 0
+    return keep
+
+
+def _bitmap_shape(lead, L, bm, bn):
+    return lead + ((L + bm - 1) // bm, ((L + bn - 1) // bn + 31) // 32)
+
+
+def bitmap_definition(keep, bm=128, bn=128):
+    keep = _c(keep, np.uint8)
+    L = keep.shape[-1]
+    bmp = np.empty(_bitmap_shape(keep.shape[:-2], L, bm, bn), np.uint32)
+    assert lib().dmao_bitmap_definition(_p(keep), keep.size // (L * L), L, bm, bn, _p(bmp)) == 0
+    return bmp
+
+
+def bitmap_from_expiry(e, bm=128, bn=128):
+    e = _c(e, np.int32)
+    L = e.shape[-1]
+    bmp = np.empty(_bitmap_shape(e.shape[:-1], L, bm, bn), np.uint32)
+    assert lib().dmao_bitmap_from_expiry(_p(e), e.size // L, L, bm, bn, _p(bmp)) == 0
+    return bmp
+
+
+def forward(Q, K, V, bias, expiry=None, keep=None, scale=None, rows=None, dtype=np.float64):
+    """Eq. (attention_output). Returns (O, LSE). With ``rows`` only those query rows are evaluated and the
+    outputs are compact: O [B,len(rows),Hq,d], LSE [B,Hq,len(rows)]."""
+    Q = _c(Q, dtype); K = _c(K, dtype); V = _c(V, dtype); bias = _c(bias, dtype)
+    expiry = _c(expiry, np.int32); keep = _c(keep, np.uint8); rows = _c(rows, np.int32)
+    B, L, Hq, d = Q.shape
+    Hkv = K.shape[2]
+    scale = d ** -0.5 if scale is None else scale
+    R = L if rows is None else len(rows)
+    O = np.empty((B, R, Hq, d), dtype)
+    LSE = np.empty((B, Hq, R), dtype)
+    f = lib().dmao_fwd_f64 if dtype == np.float64 else lib().dmao_fwd_f32
+    rc = f(_p(Q), _p(K), _p(V), _p(bias), _p(expiry), _p(keep), B, L, Hq, Hkv, d, ctypes.c_double(scale),
+           _p(rows), 0 if rows is None else len(rows), _p(O), _p(LSE))
+    assert rc == 0, rc
+    return O, LSE
+
+
+def backward(Q, K, V, dO, bias, expiry=None, keep=None, scale=None, keys=None, want_dq=True, dtype=np.float64):
+    """Sec. 4.3 gradients with the mask and bias values held fixed. Returns (dQ, dK, dV, dM). With ``keys`` only
+    those keys are evaluated: dK,dV [B,len(keys),Hkv,d], dM [B,Hq,len(keys)] (dQ stays full, or None)."""
+    Q = _c(Q, dtype); K = _c(K, dtype); V = _c(V, dtype); dO = _c(dO, dtype); bias = _c(bias, dtype)
+    expiry = _c(expiry, np.int32); keep = _c(keep, np.uint8); keys = _c(keys, np.int32)
+    B, L, Hq, d = Q.shape
+    Hkv = K.shape[2]
+    scale = d ** -0.5 if scale is None else scale
+    NK = L if keys is None else len(keys)
+    dQ = np.empty((B, L, Hq, d), dtype) if want_dq else None
+    dK = np.empty((B, NK, Hkv, d), dtype)
+    dV = np.empty((B, NK, Hkv, d), dtype)
+    dM = np.empty((B, Hq, NK), dtype)
+    f = lib().dmao_bwd_f64 if dtype == np.float64 else lib().dmao_bwd_f32
+    rc = f(_p(Q), _p(K), _p(V), _p(dO), _p(bias), _p(expiry), _p(keep), B, L, Hq, Hkv, d,
+           ctypes.c_double(scale), _p(keys), 0 if keys is None else len(keys), _p(dQ), _p(dK), _p(dV), _p(dM))
+    assert rc == 0, rc
+    return dQ, dK, dV, dM
