@@ -1,0 +1,290 @@
+#!/usr/bin/env python
+"""Benchmark of the DMA hot path (mask build + forward + backward) on synthetic data.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 3] [--impl reference]
+
+One step = dma_mask_build + dma_attn_fwd (+ dma_attn_bwd) on one batch of the workload (default: the 16K training
+configuration the headline metric is quoted on). Prints one JSON line. With N > 1 (under torchrun) every rank
+runs its own replica of the batch (the path has no exchange step), the step time is the max over ranks and the
+value is the whole-job aggregate. `--impl reference` times the CPU oracle on a bounded sample instead.
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+import torch  # noqa: E402
+
+from paper_2508_02124_b200 import workloads as wl  # noqa: E402
+
+METRIC = "dma_fwd_bwd_executed_tile_tflops"
+NOMINAL_BF16_TFLOPS = 2250.0
+
+
+def tile_flops(active_tiles, d, backward, bm=128, bn=128):
+    """Executed-tile FLOPs: 2 GEMMs forward, 5 backward, each 2*bm*bn*d per active tile."""
+    return active_tiles * (4 + (10 if backward else 0)) * bm * bn * d
+
+
+def causal_tiles(case):
+    T = -(-case.L // 128)
+    return case.B * case.Hq * T * (T + 1) // 2
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        m = json.load(open(path))
+        return {"bf16_burst": m["bf16_tflops"], "bf16_sustained": m.get("bf16_tflops_sustained", m["bf16_tflops"]),
+                "hbm_gbs": m["hbm_gbs"], "source": "measured"}
+    return {"bf16_burst": 1590.0, "bf16_sustained": 1400.0, "hbm_gbs": 6650.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """nvidia-smi clock/throttle samples during the timed region (read-only query)."""
+    Q = "clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown," \
+        "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap"
+
+    def __init__(self, index):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.p = None
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
+                                       "-i", str(index)], stdout=self.f, stderr=subprocess.DEVNULL)
+        except OSError:
+            pass
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.p is None:
+            return out
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.p.kill()
+        self.f.flush()
+        rows = [r.split(",") for r in open(self.f.name).read().strip().splitlines() if r.count(",") >= 6]
+        os.unlink(self.f.name)
+        if not rows:
+            return out
+        sm = sorted(float(r[0]) for r in rows)
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = [n for k, n in enumerate(names) if any("Active" in r[3 + k] and "Not" not in r[3 + k] for r in rows)]
+        out.update(sm_mhz=sm[len(sm) // 2], sm_max_mhz=float(rows[0][1]), reasons=reasons, samples=len(rows),
+                   power_w_max=max(float(r[2]) for r in rows))
+        return out
+
+
+def oracle_sample_run(case, inp, Ls):
+    """The CPU oracle (fp32 instantiation, as it stands) on a bounded sample: the first KV-head group, first Ls
+    rows (a causal prefix is a self-contained problem). Returns (seconds, executed-tile FLOPs of the sample)."""
+    import oracle
+    G = case.Hq // case.Hkv
+    f = lambda t, n: np.ascontiguousarray(t[:1, :Ls, :n].float().numpy())
+    Q, K, V, dO = f(inp["Q"], G), f(inp["K"], 1), f(inp["V"], 1), f(inp["dO"], G)
+    W, A = inp["W_delta"][:G].numpy(), inp["A"][:G].numpy()
+    t0 = time.perf_counter()
+    _, dl = oracle.delta(V, W, A, G)
+    e = oracle.select_expiry(dl, min(case.w, Ls))
+    bmp = oracle.bitmap_from_expiry(e)
+    oracle.forward(Q, K, V, dl, expiry=e, dtype=np.float32)
+    if case.backward:
+        oracle.backward(Q, K, V, dO, dl, expiry=e, dtype=np.float32)
+    sec = time.perf_counter() - t0
+    active = int(sum(bin(int(x)).count("1") for x in bmp.ravel()))
+    return sec, tile_flops(active, case.d, case.backward), oracle.threads()
+
+
+def run_reference(args, case):
+    """--impl reference: the oracle on the host cores, each step one bounded sample."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    inp = wl.make_inputs(case)
+    Ls = min(case.L, args.ref_rows)
+    for _ in range(args.warmup):
+        oracle_sample_run(case, inp, Ls)
+    secs = []
+    for _ in range(args.steps):
+        s, flops, cores = oracle_sample_run(case, inp, Ls)
+        secs.append(s)
+    ms = 1e3 * sum(secs) / len(secs)
+    val = flops / (ms * 1e-3) / 1e12
+    sample = f"first KV-head group ({case.Hq // case.Hkv} query heads), first {Ls} rows of {case.name}, fp32 oracle, mask+fwd" + ("+bwd" if case.backward else "")
+    print(json.dumps({"impl": "reference", "metric": METRIC, "value": val, "unit": "TFLOP/s", "n_gpus": args.gpus,
+                      "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+                      "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+                      "config": {"workload": case.name, "sample": sample},
+                      "cpu_baseline": {"value": val, "unit": "TFLOP/s", "cores": cores, "kind": "oracle", "sample": sample},
+                      "e2e": {"value": val, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="3", help="key of workloads.CONFIGS (3 = 16K training step, the headline)")
+    ap.add_argument("--impl", default="dma", choices=["dma", "reference"])
+    ap.add_argument("--ref-rows", type=int, default=4096, help="rows of the oracle sample per step (--impl reference)")
+    ap.add_argument("--cpu-rows", type=int, default=8192, help="rows of the oracle sample for cpu_baseline (0 = skip)")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--flags", type=int, default=0)
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "dma" else args.warmup
+    case = wl.CONFIGS[args.workload]
+    if args.impl == "reference":
+        return run_reference(args, case)
+
+    from paper_2508_02124_b200 import binding as dma
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the DMA path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    inp = wl.make_inputs(case)
+    p = dma.problem(case.B, case.Hq, case.Hkv, case.L, case.d, case.w, dtype=case.torch_dtype, flags=args.flags)
+    Q, K, V, dO, W, A = (inp[k].to(dev) for k in ("Q", "K", "V", "dO", "W_delta", "A"))
+    m_ws, f_ws, b_ws = dma.dma_query_workspace(p)
+    ws_m, ws_f, ws_b = (torch.empty(n, dtype=torch.uint8, device=dev) for n in (m_ws, f_ws, b_ws))
+    bias = torch.empty(case.B, case.Hq, case.L, dtype=torch.float32, device=dev)
+    expiry = torch.empty(case.B, case.Hq, case.L, dtype=torch.int32, device=dev)
+    bitmap = torch.empty(dma.dma_bitmap_words(p), dtype=torch.int32, device=dev)
+    O, lse = torch.empty_like(Q), torch.empty(case.B, case.Hq, case.L, dtype=torch.float32, device=dev)
+    dQ, dK, dV = torch.empty_like(Q), torch.empty_like(K), torch.empty_like(V)
+    dM = torch.empty_like(lse)
+
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    stage_ms = {"mask": 0.0, "fwd": 0.0, "bwd": 0.0}
+
+    def step(timed=False):
+        e = [ev() for _ in range(4)] if timed else None
+        if timed: e[0].record()
+        dma.dma_mask_build(p, V, W, A, bias, expiry, bitmap, ws_m)
+        if timed: e[1].record()
+        dma.dma_attn_fwd(p, Q, K, V, bias, expiry, bitmap, O, lse, ws_f)
+        if timed: e[2].record()
+        if case.backward:
+            dma.dma_attn_bwd(p, Q, K, V, O, dO, lse, bias, expiry, bitmap, dQ, dK, dV, dM, ws_b)
+        if timed: e[3].record()
+        return e
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    assert dma.dma_read_status(ws_f) == 0 and (not case.backward or dma.dma_read_status(ws_b) == 0), "device status"
+    active = int(sum(bin(int(x) & 0xFFFFFFFF).count("1") for x in bitmap.cpu().numpy().ravel()))
+
+    sampler = ClockSampler(torch.cuda.current_device() if "CUDA_VISIBLE_DEVICES" not in os.environ else
+                           os.environ["CUDA_VISIBLE_DEVICES"].split(",")[local]) if rank == 0 else None
+    launches0 = dma.dma_launch_count()
+    t0, t1 = ev(), ev()
+    barrier()
+    t0.record()
+    evs = [step(timed=True) for _ in range(args.steps)]
+    t1.record()
+    barrier()
+    launches = dma.dma_launch_count() - launches0
+    clocks = sampler.stop() if sampler else None
+    total_ms = t0.elapsed_time(t1)
+    for e in evs:
+        stage_ms["mask"] += e[0].elapsed_time(e[1]); stage_ms["fwd"] += e[1].elapsed_time(e[2]); stage_ms["bwd"] += e[2].elapsed_time(e[3])
+    stage_ms = {k: v / args.steps for k, v in stage_ms.items()}
+    ms = total_ms / args.steps
+    if dist is not None:
+        t = torch.tensor([ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+
+    # ---- end to end through the host-buffer entry point: pinned host tensors in, results back on the host
+    e2e = None
+    if not args.no_e2e:
+        arena = torch.empty(dma.dma_step_host_arena(p, case.backward), dtype=torch.uint8, device=dev)
+        pin = lambda t: t.contiguous().pin_memory()
+        hin = [pin(inp[k]) for k in ("Q", "K", "V", "dO", "W_delta", "A")]
+        hO, hlse = pin(torch.empty_like(inp["Q"])), pin(torch.empty(case.B, case.Hq, case.L))
+        hdQ, hdK, hdV, hdM = pin(torch.empty_like(inp["Q"])), pin(torch.empty_like(inp["K"])), pin(torch.empty_like(inp["V"])), pin(torch.empty(case.B, case.Hq, case.L))
+        call = lambda: dma.dma_step_host(p, case.backward, hin[0], hin[1], hin[2], hin[3], hin[4], hin[5], hO, hlse, hdQ, hdK, hdV, hdM, arena)
+        n_e2e = max(3, min(args.steps, 10))
+        call(); call()
+        barrier()
+        t2, t3 = ev(), ev()
+        t2.record()
+        for _ in range(n_e2e):
+            call()
+        t3.record()
+        barrier()
+        e2e_ms = t2.elapsed_time(t3) / n_e2e
+        if dist is not None:
+            t = torch.tensor([e2e_ms], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e2e_ms = float(t.item())
+        nb = lambda *ts: int(sum(t.numel() * t.element_size() for t in ts))
+        h2d = nb(*hin) if case.backward else nb(hin[0], hin[1], hin[2], hin[4], hin[5])
+        d2h = nb(hO, hlse) + (nb(hdQ, hdK, hdV, hdM) if case.backward else 0)
+        assert torch.equal(hO, O.cpu()), "host-buffer path disagrees with the device path"
+        e2e = {"value": world * tile_flops(active, case.d, case.backward) / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s",
+               "ms_per_step": e2e_ms, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+    pk = peaks()
+    flops = tile_flops(active, case.d, case.backward)
+    value = world * flops / (ms * 1e-3) / 1e12
+    dom = "bwd" if case.backward else "fwd"
+    dom_flops = tile_flops(active, case.d, False) * (2.5 if case.backward else 1.0)
+    achieved = dom_flops / (stage_ms[dom] * 1e-3) / 1e12
+    tensor_path = case.dtype == "bf16" and case.d == 128 and not (args.flags & dma.DMA_FLAG_SIMT)
+    out = {
+        "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16" if case.dtype == "bf16" else "f32", "data": "synthetic",
+        "config": {"workload": case.name, "B": case.B, "Hq": case.Hq, "Hkv": case.Hkv, "L": case.L, "d": case.d, "w": case.w,
+                   "passes": "mask+fwd+bwd" if case.backward else "mask+fwd", "parallelism": f"replicas x{world}",
+                   "l2": "inputs larger than L2 (no flush needed)" if (Q.numel() + 2 * K.numel()) * Q.element_size() > 126e6 else "inputs smaller than L2"},
+        "stage_ms": stage_ms, "active_tiles": active, "causal_tiles": causal_tiles(case),
+        "executed_tile_tflop_per_step": flops / 1e12,
+        "frac_of_nominal_bf16_peak": value / world / NOMINAL_BF16_TFLOPS,
+        "frac_of_measured_bf16_peak": value / world / pk["bf16_sustained"],
+        "fwd_tflops": tile_flops(active, case.d, False) / (stage_ms["fwd"] * 1e-3) / 1e12,
+        "bwd_tflops": (dom_flops / (stage_ms["bwd"] * 1e-3) / 1e12) if case.backward else None,
+        "dense_causal_equivalent_speedup": causal_tiles(case) / max(active, 1),
+        "roofline": {"bound": "tensor" if tensor_path else "alu", "kernel": f"dma_attn_{dom} (stage time, includes its pre/post kernels)",
+                     "achieved": achieved, "peak": pk["bf16_sustained"], "peak_source": pk["source"] + " sustained cuBLAS bf16",
+                     "unit": "TFLOP/s", "frac": achieved / pk["bf16_sustained"], "traffic": None},
+        "gpu_launches": launches, "clocks": clocks, "e2e": e2e,
+    }
+    if args.cpu_rows:
+        Ls = min(case.L, args.cpu_rows)
+        sec, fl, cores = oracle_sample_run(case, inp, Ls)
+        out["cpu_baseline"] = {"value": fl / sec / 1e12, "unit": "TFLOP/s", "cores": cores, "kind": "oracle", "seconds": sec,
+                               "sample": f"first KV-head group ({case.Hq // case.Hkv} query heads), first {Ls} rows of {case.name}, fp32 oracle"}
+    print(json.dumps(out))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

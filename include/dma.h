@@ -1,0 +1,129 @@
+/* dma.h - C ABI of the B200 (sm_100a) Dynamic Mask Attention hot path.
+ *
+ * Three stages, each one entry point:
+ *   dma_mask_build   value vectors -> per-key dynamic weight (the additive bias), per-key expiry row
+ *                    (compact form of the per-row top-w mask) and a (query tile, key tile) activity bitmap
+ *   dma_attn_fwd     block-sparse attention forward: O and the row log-sum-exp
+ *   dma_attn_bwd     backward: dQ, dK, dV and dM (gradient of the mask bias)
+ *
+ * Conventions
+ *   - Unless a parameter is marked HOST, every pointer is a DEVICE pointer owned by the caller, 16-byte
+ *     aligned. The library allocates no device memory, keeps no state between calls, enqueues work only
+ *     on the caller's stream (a cudaStream_t passed as void*; NULL = default stream) and does not
+ *     synchronise, except in dma_read_status and dma_step_host.
+ *   - Element type of Q,K,V,O,dO,dQ,dK,dV is `dtype` (bf16 or fp32). bias, lse, dM, W_delta, A are fp32.
+ *   - Q,O,dO,dQ are [B, L, Hq, d]; K,V,dK,dV are [B, L, Hkv, d]; d is contiguous; the batch, sequence and
+ *     head strides are given in elements in the problem descriptor (0 = contiguous default). bias, expiry,
+ *     lse, dM are contiguous [B, Hq, L]. Query head h reads KV head h / (Hq / Hkv).
+ *   - Every entry point returns 0 (DMA_OK) or a negative dma_status code; nothing is thrown across the ABI.
+ *     On an error return no kernel has been launched. Outputs are fully overwritten (no pre-zeroing needed).
+ *   - There is no CPU path: without a CUDA device of compute capability 10.x the calls return DMA_ERR_CUDA.
+ */
+#ifndef DMA_B200_H
+#define DMA_B200_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    DMA_OK = 0,
+    DMA_ERR_NULL = -1,           /* a required pointer is NULL                                      */
+    DMA_ERR_SHAPE = -2,          /* non-positive size, Hq % Hkv != 0, w < 1, bad tile size          */
+    DMA_ERR_ALIGN = -3,          /* pointer not 16-byte aligned or stride not a multiple of 8       */
+    DMA_ERR_UNSUPPORTED = -4,    /* valid request outside what is implemented (see each call)       */
+    DMA_ERR_WORKSPACE = -5,      /* workspace NULL or smaller than dma_query_workspace reports      */
+    DMA_ERR_CUDA = -6,           /* a CUDA runtime / driver call failed (launch, descriptor, device)*/
+    DMA_ERR_DEVICE_TIMEOUT = -7  /* a bounded device-side wait gave up (read via dma_read_status)    */
+} dma_status;
+
+enum { DMA_BF16 = 0, DMA_FP32 = 1 };
+
+/* flags */
+enum {
+    DMA_FLAG_IGNORE_BITMAP = 1,  /* visit every causal tile regardless of the bitmap (result must not change:
+                                    block skipping is an optimisation only, Sec. 4.2 last paragraph)           */
+    DMA_FLAG_SIMT = 2            /* run the CUDA-core kernels also for bf16 (they always serve fp32)            */
+};
+
+typedef struct {
+    int32_t B, Hq, Hkv, L, d;    /* d in {64, 128}; Hq % Hkv == 0; L >= 1 (query and key length are equal)      */
+    int32_t w;                   /* keep window of Eq. (mask_combine), >= 1; values above L act as L            */
+    int32_t causal;              /* must be 1: key j is visible to row i iff j <= i                             */
+    int32_t dtype;               /* DMA_BF16 | DMA_FP32                                                         */
+    int32_t tile_m, tile_n;      /* bitmap granularity (query rows x keys per bit); 0,0 = 128,128               */
+    int32_t flags;               /* DMA_FLAG_*                                                                  */
+    float softmax_scale;         /* 0 -> 1/sqrt(d)  (Alg. 1: S = Q K^T d^-1/2 + M)                              */
+    int64_t q_stride[3];         /* batch, sequence, head strides of Q (also dQ) in elements; all 0 = contiguous*/
+    int64_t k_stride[3];         /* same for K (also dK)                                                        */
+    int64_t v_stride[3];         /* same for V (also dV)                                                        */
+    int64_t o_stride[3];         /* same for O (also dO)                                                        */
+} dma_problem_t;
+
+/* Bytes of device workspace each stage needs for this problem (any pointer may be NULL to skip it).
+ * Each workspace begins with a 256-byte header whose first int32 is the device status word. */
+int dma_query_workspace(const dma_problem_t* p, size_t* mask_ws, size_t* fwd_ws, size_t* bwd_ws);
+
+/* Number of uint32 words of the bitmap, [B, Hq, Tr, ceil(Tc/32)] with Tr = ceil(L/tile_m), Tc = ceil(L/tile_n). */
+int dma_bitmap_words(const dma_problem_t* p, size_t* words);
+
+/* Mask generation (Sec. 4.1).
+ *   z[b,h,j]     = V[b,j,h/G,:] . W_delta[h,:]                        value projection, Eq. (delta_calc)
+ *   bias[b,h,j]  = exp(A[h] * softplus(z))                             the dynamic weight delta; it is the additive
+ *                                                                      mask value wherever the key is kept
+ *   expiry[b,h,j]                                                      row i keeps key j iff j <= i < expiry[j]. This
+ *        is the exact compact form of Eq. (mask_combine) read per query row over the causally visible keys:
+ *        row i keeps the min(w, i+1) best keys under the order (delta descending, index ascending).
+ *   bitmap       bit (kt % 32) of word [b,h,qt,kt/32] is 1 iff some (i in tile qt, j in tile kt) is kept: the
+ *                block-level Judge test of Alg. 1 / Alg. 2.
+ * delta is computed in fp32 in a fixed operation order so that its bit pattern, and therefore the selection,
+ * is reproducible. W_delta is [Hq, d] fp32, A is [Hq] fp32. Supports both dtypes, d in {64,128}. */
+int dma_mask_build(const dma_problem_t* p, const void* V, const float* W_delta, const float* A,
+                   float* bias, int32_t* expiry, uint32_t* bitmap,
+                   void* ws, size_t ws_bytes, void* cuda_stream);
+
+/* Forward (Sec. 4.2, Eq. (attention_output), Alg. 1): for each row i of head h
+ *   s_j = q_i . k_j * scale + bias[j]   over keys with j <= i < expiry[j];   p = softmax(s);   O_i = sum p_j v_j
+ *   lse_i = log sum_j exp(s_j)   (natural log; replaces Alg. 1's (l, m) pair)
+ * Key tiles whose bitmap bit is 0 are neither loaded nor computed. Any self-consistent (bias, expiry, bitmap)
+ * triple is accepted. bf16: tcgen05/TMA kernel, d = 128 (d = 64 runs the CUDA-core kernel); fp32: CUDA-core kernel. */
+int dma_attn_fwd(const dma_problem_t* p, const void* Q, const void* K, const void* V,
+                 const float* bias, const int32_t* expiry, const uint32_t* bitmap,
+                 void* O, float* lse, void* ws, size_t ws_bytes, void* cuda_stream);
+
+/* Backward (Sec. 4.3, Alg. 2, Eqs. (grad_v), (grad_s), (grad_m), (grad_qk)), mask and bias values held fixed:
+ *   D_i = dO_i . O_i;  p_ij = exp(s_ij - lse_i);  dP_ij = dO_i . v_j;  dS_ij = p_ij (dP_ij - D_i)
+ *   dV_j = sum_i p_ij dO_i;  dK_j = scale sum_i dS_ij q_i;  dQ_i = scale sum_j dS_ij k_j;  dM[b,h,j] = sum_i dS_ij
+ * dK and dV are summed over the Hq/Hkv query heads that share a KV head; dM is per query head.
+ * dQ is accumulated with floating-point atomics: its rounding depends on execution order. */
+int dma_attn_bwd(const dma_problem_t* p, const void* Q, const void* K, const void* V,
+                 const void* O, const void* dO, const float* lse,
+                 const float* bias, const int32_t* expiry, const uint32_t* bitmap,
+                 void* dQ, void* dK, void* dV, float* dM,
+                 void* ws, size_t ws_bytes, void* cuda_stream);
+
+/* The whole hot path on HOST buffers (all contiguous, default strides only): copies Q,K,V,(dO),W_delta,A into the
+ * caller's device arena, runs dma_mask_build, dma_attn_fwd and, if `backward` != 0, dma_attn_bwd on the stream,
+ * copies O, lse (and dQ,dK,dV,dM) back and synchronises the stream before returning. h* pointers are HOST memory
+ * (pinned memory makes the copies asynchronous and faster); dev_arena is DEVICE memory, 256-byte aligned, of at
+ * least dma_step_host_arena() bytes; hdO, hdQ, hdK, hdV, hdM may be NULL when `backward` is 0. */
+int dma_step_host_arena(const dma_problem_t* p, int backward, size_t* bytes);
+int dma_step_host(const dma_problem_t* p, int backward, const void* hQ, const void* hK, const void* hV, const void* hdO,
+                  const float* hW_delta, const float* hA, void* hO, float* hlse, void* hdQ, void* hdK, void* hdV,
+                  float* hdM, void* dev_arena, size_t arena_bytes, void* cuda_stream);
+
+/* Synchronises the stream and returns the device status word of a workspace (0 or DMA_ERR_DEVICE_TIMEOUT). */
+int dma_read_status(const void* ws, void* cuda_stream);
+
+/* Number of kernels the library has launched in this process (all entry points), for accounting. */
+long long dma_launch_count(void);
+
+const char* dma_strerror(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DMA_B200_H */

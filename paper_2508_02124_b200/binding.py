@@ -1,0 +1,159 @@
+"""ctypes binding of ``libdma_b200.so`` (declared in ``include/dma.h``): argument marshalling only.
+
+Every function here has the name of the C entry point it calls. Tensors are torch CUDA tensors used as
+device memory; the current torch stream is passed as the CUDA stream. There is no fallback: if the library is
+not built, or a call returns an error status, a ``DmaError`` is raised.
+"""
+import ctypes
+import os
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libdma_b200.so")
+_lib = None
+
+DMA_BF16, DMA_FP32 = 0, 1
+DMA_FLAG_IGNORE_BITMAP, DMA_FLAG_SIMT = 1, 2
+
+ENTRY_POINTS = ("dma_query_workspace", "dma_bitmap_words", "dma_mask_build", "dma_attn_fwd", "dma_attn_bwd",
+                "dma_read_status", "dma_launch_count", "dma_strerror", "dma_step_host_arena", "dma_step_host")
+
+
+class DmaError(RuntimeError):
+    def __init__(self, status, what):
+        self.status = status
+        super().__init__(f"{what}: status {status} ({dma_strerror(status)})")
+
+
+class dma_problem_t(ctypes.Structure):
+    _fields_ = [("B", ctypes.c_int32), ("Hq", ctypes.c_int32), ("Hkv", ctypes.c_int32), ("L", ctypes.c_int32),
+                ("d", ctypes.c_int32), ("w", ctypes.c_int32), ("causal", ctypes.c_int32), ("dtype", ctypes.c_int32),
+                ("tile_m", ctypes.c_int32), ("tile_n", ctypes.c_int32), ("flags", ctypes.c_int32),
+                ("softmax_scale", ctypes.c_float),
+                ("q_stride", ctypes.c_int64 * 3), ("k_stride", ctypes.c_int64 * 3),
+                ("v_stride", ctypes.c_int64 * 3), ("o_stride", ctypes.c_int64 * 3)]
+
+
+def lib():
+    """Loads the shared library; raises if it has not been built (``python -m paper_2508_02124_b200.build``)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise DmaError(-6, f"{LIB_PATH} is missing: build it with `python -m paper_2508_02124_b200.build`")
+        L = ctypes.CDLL(LIB_PATH)
+        L.dma_strerror.restype = ctypes.c_char_p
+        L.dma_launch_count.restype = ctypes.c_longlong
+        _lib = L
+    return _lib
+
+
+def dma_strerror(status):
+    try:
+        return lib().dma_strerror(int(status)).decode()
+    except Exception:
+        return "?"
+
+
+def problem(B, Hq, Hkv, L, d, w, dtype=torch.bfloat16, causal=1, tile_m=0, tile_n=0, flags=0, softmax_scale=0.0):
+    p = dma_problem_t()
+    p.B, p.Hq, p.Hkv, p.L, p.d, p.w, p.causal = B, Hq, Hkv, L, d, w, causal
+    p.dtype = DMA_BF16 if dtype == torch.bfloat16 else DMA_FP32
+    p.tile_m, p.tile_n, p.flags, p.softmax_scale = tile_m, tile_n, flags, softmax_scale
+    return p
+
+
+def _ptr(t):
+    return ctypes.c_void_p(0 if t is None else t.data_ptr())
+
+
+def _stream():
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _check(rc, what):
+    if rc != 0:
+        raise DmaError(rc, what)
+
+
+def dma_query_workspace(p):
+    m, f, b = ctypes.c_size_t(), ctypes.c_size_t(), ctypes.c_size_t()
+    _check(lib().dma_query_workspace(ctypes.byref(p), ctypes.byref(m), ctypes.byref(f), ctypes.byref(b)), "dma_query_workspace")
+    return m.value, f.value, b.value
+
+
+def dma_bitmap_words(p):
+    n = ctypes.c_size_t()
+    _check(lib().dma_bitmap_words(ctypes.byref(p), ctypes.byref(n)), "dma_bitmap_words")
+    return n.value
+
+
+def _ws(nbytes, device):
+    return torch.empty((nbytes + 255) // 256 * 256, dtype=torch.uint8, device=device)
+
+
+def dma_mask_build(p, V, W_delta, A, bias=None, expiry=None, bitmap=None, ws=None):
+    """Returns (bias [B,Hq,L] fp32, expiry [B,Hq,L] int32, bitmap [B,Hq,Tr,ceil(Tc/32)] int32-typed uint32 words)."""
+    dev = V.device
+    if bias is None:
+        bias = torch.empty(p.B, p.Hq, p.L, dtype=torch.float32, device=dev)
+    if expiry is None:
+        expiry = torch.empty(p.B, p.Hq, p.L, dtype=torch.int32, device=dev)
+    if bitmap is None:
+        tm, tn = (p.tile_m or 128), (p.tile_n or 128)
+        Tr, Tc = -(-p.L // tm), -(-p.L // tn)
+        bitmap = torch.empty(p.B, p.Hq, Tr, (Tc + 31) // 32, dtype=torch.int32, device=dev)
+    if ws is None:
+        ws = _ws(dma_query_workspace(p)[0], dev)
+    _check(lib().dma_mask_build(ctypes.byref(p), _ptr(V), _ptr(W_delta), _ptr(A), _ptr(bias), _ptr(expiry), _ptr(bitmap),
+                                _ptr(ws), ctypes.c_size_t(ws.numel()), _stream()), "dma_mask_build")
+    return bias, expiry, bitmap
+
+
+def dma_attn_fwd(p, Q, K, V, bias, expiry, bitmap, O=None, lse=None, ws=None):
+    """Returns (O like Q, lse [B,Hq,L] fp32)."""
+    if O is None:
+        O = torch.empty_like(Q)
+    if lse is None:
+        lse = torch.empty(p.B, p.Hq, p.L, dtype=torch.float32, device=Q.device)
+    if ws is None:
+        ws = _ws(dma_query_workspace(p)[1], Q.device)
+    _check(lib().dma_attn_fwd(ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(bias), _ptr(expiry), _ptr(bitmap), _ptr(O),
+                              _ptr(lse), _ptr(ws), ctypes.c_size_t(ws.numel()), _stream()), "dma_attn_fwd")
+    return O, lse
+
+
+def dma_attn_bwd(p, Q, K, V, O, dO, lse, bias, expiry, bitmap, dQ=None, dK=None, dV=None, dM=None, ws=None):
+    """Returns (dQ like Q, dK like K, dV like V, dM [B,Hq,L] fp32)."""
+    dQ = torch.empty_like(Q) if dQ is None else dQ
+    dK = torch.empty_like(K) if dK is None else dK
+    dV = torch.empty_like(V) if dV is None else dV
+    if dM is None:
+        dM = torch.empty(p.B, p.Hq, p.L, dtype=torch.float32, device=Q.device)
+    if ws is None:
+        ws = _ws(dma_query_workspace(p)[2], Q.device)
+    _check(lib().dma_attn_bwd(ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(O), _ptr(dO), _ptr(lse), _ptr(bias),
+                              _ptr(expiry), _ptr(bitmap), _ptr(dQ), _ptr(dK), _ptr(dV), _ptr(dM), _ptr(ws),
+                              ctypes.c_size_t(ws.numel()), _stream()), "dma_attn_bwd")
+    return dQ, dK, dV, dM
+
+
+def dma_read_status(ws):
+    return lib().dma_read_status(_ptr(ws), _stream())
+
+
+def dma_launch_count():
+    return lib().dma_launch_count()
+
+
+def dma_step_host_arena(p, backward):
+    n = ctypes.c_size_t()
+    _check(lib().dma_step_host_arena(ctypes.byref(p), int(backward), ctypes.byref(n)), "dma_step_host_arena")
+    return n.value
+
+
+def dma_step_host(p, backward, hQ, hK, hV, hdO, hW, hA, hO, hlse, hdQ, hdK, hdV, hdM, arena):
+    """All h* are CPU tensors (ideally pinned); `arena` is a CUDA uint8 tensor of dma_step_host_arena() bytes."""
+    _check(lib().dma_step_host(ctypes.byref(p), int(backward), _ptr(hQ), _ptr(hK), _ptr(hV), _ptr(hdO), _ptr(hW), _ptr(hA),
+                               _ptr(hO), _ptr(hlse), _ptr(hdQ), _ptr(hdK), _ptr(hdV), _ptr(hdM), _ptr(arena),
+                               ctypes.c_size_t(arena.numel()), _stream()), "dma_step_host")

@@ -1,0 +1,164 @@
+// C-ABI entry points (include/dma.h): argument validation, defaults, dispatch to the stage launchers.
+#include <atomic>
+#include <cmath>
+
+#include "common.cuh"
+
+namespace dma {
+
+static std::atomic<long long> g_launches{0};
+void count_launch(int n) { g_launches += n; }
+int check_launch() { return cudaGetLastError() == cudaSuccess ? DMA_OK : DMA_ERR_CUDA; }
+
+static bool fill_strides(const int64_t in[3], int64_t out[3], int L, int H, int d) {
+    if (in[0] == 0 && in[1] == 0 && in[2] == 0) {
+        out[0] = (int64_t)L * H * d; out[1] = (int64_t)H * d; out[2] = d;
+        return true;
+    }
+    for (int i = 0; i < 3; ++i) {
+        if (in[i] <= 0 || in[i] % 8) return false;
+        out[i] = in[i];
+    }
+    return true;
+}
+
+int resolve(const dma_problem_t* p, Prob* o) {
+    if (!p) return DMA_ERR_NULL;
+    if (p->B < 1 || p->Hq < 1 || p->Hkv < 1 || p->L < 1 || p->w < 1 || p->Hq % p->Hkv) return DMA_ERR_SHAPE;
+    if (p->d != 64 && p->d != 128) return DMA_ERR_UNSUPPORTED;
+    if (p->causal != 1) return DMA_ERR_UNSUPPORTED;
+    if (p->dtype != DMA_BF16 && p->dtype != DMA_FP32) return DMA_ERR_UNSUPPORTED;
+    if ((p->tile_m == 0) != (p->tile_n == 0) || p->tile_m < 0 || p->tile_n < 0) return DMA_ERR_SHAPE;
+    if (!(p->softmax_scale >= 0.0f) || std::isinf(p->softmax_scale)) return DMA_ERR_SHAPE;
+    o->B = p->B; o->Hq = p->Hq; o->Hkv = p->Hkv; o->L = p->L; o->d = p->d; o->G = p->Hq / p->Hkv;
+    o->w = p->w < p->L ? p->w : p->L;
+    o->dtype = p->dtype; o->flags = p->flags;
+    o->bm = p->tile_m ? p->tile_m : 128;
+    o->bn = p->tile_n ? p->tile_n : 128;
+    o->Tr = (p->L + o->bm - 1) / o->bm;
+    o->Tc = (p->L + o->bn - 1) / o->bn;
+    o->Wd = (o->Tc + 31) / 32;
+    o->scale = p->softmax_scale > 0.0f ? p->softmax_scale : 1.0f / sqrtf((float)p->d);
+    if (!fill_strides(p->q_stride, o->qs, p->L, p->Hq, p->d) || !fill_strides(p->k_stride, o->ks, p->L, p->Hkv, p->d) ||
+        !fill_strides(p->v_stride, o->vs, p->L, p->Hkv, p->d) || !fill_strides(p->o_stride, o->os, p->L, p->Hq, p->d))
+        return DMA_ERR_ALIGN;
+    return DMA_OK;
+}
+
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+static bool use_tensor_cores(const Prob& P) {
+    return P.dtype == DMA_BF16 && P.d == 128 && P.bm == 128 && P.bn == 128 && !(P.flags & DMA_FLAG_SIMT);
+}
+
+static int device_ok() {
+    int dev = 0, major = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return DMA_ERR_CUDA;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return DMA_ERR_CUDA;
+    return major == 10 ? DMA_OK : DMA_ERR_CUDA;
+}
+
+}  // namespace dma
+
+using namespace dma;
+
+extern "C" {
+
+int dma_query_workspace(const dma_problem_t* p, size_t* mask_ws, size_t* fwd_ws, size_t* bwd_ws) {
+    Prob P;
+    int rc = resolve(p, &P);
+    if (rc) return rc;
+    if (mask_ws) *mask_ws = mask_ws_bytes(P);
+    if (fwd_ws) *fwd_ws = use_tensor_cores(P) ? tc_fwd_ws_bytes(P) : (size_t)kWsHeaderBytes;
+    if (bwd_ws) *bwd_ws = use_tensor_cores(P) ? tc_bwd_ws_bytes(P) : simt_bwd_ws_bytes(P);
+    return DMA_OK;
+}
+
+int dma_bitmap_words(const dma_problem_t* p, size_t* words) {
+    Prob P;
+    int rc = resolve(p, &P);
+    if (rc) return rc;
+    if (!words) return DMA_ERR_NULL;
+    *words = (size_t)P.B * P.Hq * P.Tr * P.Wd;
+    return DMA_OK;
+}
+
+int dma_mask_build(const dma_problem_t* p, const void* V, const float* W_delta, const float* A, float* bias,
+                   int32_t* expiry, uint32_t* bitmap, void* ws, size_t ws_bytes, void* cuda_stream) {
+    Prob P;
+    int rc = resolve(p, &P);
+    if (rc) return rc;
+    if (!V || !W_delta || !A || !bias || !expiry || !bitmap) return DMA_ERR_NULL;
+    if (!aligned16(V) || !aligned16(W_delta) || !aligned16(bias) || !aligned16(expiry) || !aligned16(bitmap))
+        return DMA_ERR_ALIGN;
+    if (!ws || ws_bytes < mask_ws_bytes(P) || !aligned16(ws)) return DMA_ERR_WORKSPACE;
+    if ((rc = device_ok())) return rc;
+    return launch_mask_build(P, V, W_delta, A, bias, expiry, bitmap, ws, (cudaStream_t)cuda_stream);
+}
+
+int dma_attn_fwd(const dma_problem_t* p, const void* Q, const void* K, const void* V, const float* bias,
+                 const int32_t* expiry, const uint32_t* bitmap, void* O, float* lse, void* ws, size_t ws_bytes,
+                 void* cuda_stream) {
+    Prob P;
+    int rc = resolve(p, &P);
+    if (rc) return rc;
+    if (!Q || !K || !V || !bias || !expiry || !bitmap || !O || !lse) return DMA_ERR_NULL;
+    if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || !aligned16(bias) || !aligned16(expiry) ||
+        !aligned16(lse))
+        return DMA_ERR_ALIGN;
+    const bool tc = use_tensor_cores(P);
+    const size_t need = tc ? tc_fwd_ws_bytes(P) : (size_t)kWsHeaderBytes;
+    if (!ws || ws_bytes < need || !aligned16(ws)) return DMA_ERR_WORKSPACE;
+    if ((rc = device_ok())) return rc;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    if (cudaMemsetAsync(ws, 0, kWsHeaderBytes, st) != cudaSuccess) return DMA_ERR_CUDA;
+    if (tc) return launch_tc_fwd(P, Q, K, V, bias, expiry, bitmap, O, lse, ws, st);
+    return launch_simt_fwd(P, Q, K, V, bias, expiry, bitmap, O, lse, st);
+}
+
+int dma_attn_bwd(const dma_problem_t* p, const void* Q, const void* K, const void* V, const void* O, const void* dO,
+                 const float* lse, const float* bias, const int32_t* expiry, const uint32_t* bitmap, void* dQ, void* dK,
+                 void* dV, float* dM, void* ws, size_t ws_bytes, void* cuda_stream) {
+    Prob P;
+    int rc = resolve(p, &P);
+    if (rc) return rc;
+    if (!Q || !K || !V || !O || !dO || !lse || !bias || !expiry || !bitmap || !dQ || !dK || !dV || !dM) return DMA_ERR_NULL;
+    if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || !aligned16(dO) || !aligned16(dQ) ||
+        !aligned16(dK) || !aligned16(dV) || !aligned16(dM) || !aligned16(lse))
+        return DMA_ERR_ALIGN;
+    const bool tc = use_tensor_cores(P);
+    const size_t need = tc ? tc_bwd_ws_bytes(P) : simt_bwd_ws_bytes(P);
+    if (!ws || ws_bytes < need || !aligned16(ws)) return DMA_ERR_WORKSPACE;
+    if ((rc = device_ok())) return rc;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    if (cudaMemsetAsync(ws, 0, kWsHeaderBytes, st) != cudaSuccess) return DMA_ERR_CUDA;
+    if (tc) return launch_tc_bwd(P, Q, K, V, O, dO, lse, bias, expiry, bitmap, dQ, dK, dV, dM, ws, st);
+    return launch_simt_bwd(P, Q, K, V, O, dO, lse, bias, expiry, bitmap, dQ, dK, dV, dM, ws, st);
+}
+
+int dma_read_status(const void* ws, void* cuda_stream) {
+    if (!ws) return DMA_ERR_NULL;
+    int32_t word = 0;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    if (cudaMemcpyAsync(&word, ws, sizeof(word), cudaMemcpyDeviceToHost, st) != cudaSuccess) return DMA_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return DMA_ERR_CUDA;
+    return word == 0 ? DMA_OK : DMA_ERR_DEVICE_TIMEOUT;
+}
+
+long long dma_launch_count(void) { return g_launches.load(); }
+
+const char* dma_strerror(int status) {
+    switch (status) {
+        case DMA_OK: return "ok";
+        case DMA_ERR_NULL: return "a required pointer is NULL";
+        case DMA_ERR_SHAPE: return "invalid shape, window, tile size or scale";
+        case DMA_ERR_ALIGN: return "pointer not 16-byte aligned or stride not a positive multiple of 8 elements";
+        case DMA_ERR_UNSUPPORTED: return "request outside the implemented range (d in {64,128}, causal=1, bf16/fp32)";
+        case DMA_ERR_WORKSPACE: return "workspace missing, misaligned or smaller than dma_query_workspace reports";
+        case DMA_ERR_CUDA: return "CUDA call failed or no sm_100 device";
+        case DMA_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait expired";
+        default: return "unknown status";
+    }
+}
+
+}  // extern "C"

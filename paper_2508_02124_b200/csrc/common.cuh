@@ -1,0 +1,61 @@
+// Shared declarations of the DMA CUDA library: resolved problem view, launch accounting, small device helpers.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "dma.h"
+
+namespace dma {
+
+constexpr int kWsHeaderBytes = 256;   // every workspace starts with this header; int32 word 0 = status
+
+// dma_problem_t with defaults resolved and derived sizes filled in.
+struct Prob {
+    int B, Hq, Hkv, L, d, G;
+    int w;                 // min(w, L)
+    int dtype, flags;
+    int bm, bn, Tr, Tc, Wd;   // bitmap tile sizes, tile counts, uint32 words per bitmap row
+    float scale;
+    int64_t qs[3], ks[3], vs[3], os[3];   // batch, seq, head strides in elements
+};
+
+int resolve(const dma_problem_t* p, Prob* out);          // validation + defaults; returns dma_status
+void count_launch(int n = 1);
+int check_launch();                                       // cudaGetLastError -> dma_status
+
+// stage launchers (each returns a dma_status); defined in the stage's .cu file
+size_t mask_ws_bytes(const Prob& P);
+int launch_mask_build(const Prob& P, const void* V, const float* W, const float* A, float* bias, int32_t* expiry,
+                      uint32_t* bitmap, void* ws, cudaStream_t st);
+
+size_t simt_bwd_ws_bytes(const Prob& P);
+int launch_simt_fwd(const Prob& P, const void* Q, const void* K, const void* V, const float* bias,
+                    const int32_t* expiry, const uint32_t* bitmap, void* O, float* lse, cudaStream_t st);
+int launch_simt_bwd(const Prob& P, const void* Q, const void* K, const void* V, const void* O, const void* dO,
+                    const float* lse, const float* bias, const int32_t* expiry, const uint32_t* bitmap, void* dQ,
+                    void* dK, void* dV, float* dM, void* ws, cudaStream_t st);
+
+size_t tc_fwd_ws_bytes(const Prob& P);
+int launch_tc_fwd(const Prob& P, const void* Q, const void* K, const void* V, const float* bias,
+                  const int32_t* expiry, const uint32_t* bitmap, void* O, float* lse, void* ws, cudaStream_t st);
+size_t tc_bwd_ws_bytes(const Prob& P);
+int launch_tc_bwd(const Prob& P, const void* Q, const void* K, const void* V, const void* O, const void* dO,
+                  const float* lse, const float* bias, const int32_t* expiry, const uint32_t* bitmap, void* dQ,
+                  void* dK, void* dV, float* dM, void* ws, cudaStream_t st);
+
+// ---------------------------------------------------------------------------------------------
+// device helpers
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ float to_f32(float x) { return x; }
+__device__ __forceinline__ float to_f32(__nv_bfloat16 x) { return __bfloat162float(x); }
+__device__ __forceinline__ void store_as(float* p, float x) { *p = x; }
+__device__ __forceinline__ void store_as(__nv_bfloat16* p, float x) { *p = __float2bfloat16_rn(x); }
+
+// bit (kt % 32) of word [bh, qt, kt / 32]
+__device__ __forceinline__ bool bitmap_test(const uint32_t* bitmap, int Tr, int Wd, int bh, int qt, int kt) {
+    return (bitmap[((size_t)bh * Tr + qt) * Wd + (kt >> 5)] >> (kt & 31)) & 1u;
+}
+
+}  // namespace dma

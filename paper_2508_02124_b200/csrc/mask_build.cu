@@ -1,0 +1,256 @@
+// Mask generation (Sec. 4.1): value projection + gating (Eq. delta_calc), exact per-row top-w selection in
+// compact "expiry" form (Eq. mask_combine read per query row over the causally visible keys), and the
+// (query tile, key tile) activity bitmap (the Judge test of Alg. 1 / Alg. 2).
+//
+// Kernels
+//   delta_kernel        V read once (HBM-bound); z, softplus, exp in a fixed fp32 operation order
+//   chunk_sort_kernel   256-key chunks of (delta bits, ~index) keys sorted in shared memory
+//   expiry_kernel       per key: the index of the w-th key (in index order) that beats it, by counting beaters
+//                       chunk by chunk with a binary search in each sorted chunk
+//   bitmap_kernel       per key tile: union of the query-tile intervals its keys are kept in
+#include "common.cuh"
+
+namespace dma {
+namespace {
+
+constexpr int kChunk = 256;   // keys per sorted chunk (= threads of the sort and expiry kernels)
+
+// ---- fixed-order fp32 routines: every step is one correctly rounded IEEE operation -----------------------
+
+__device__ __forceinline__ float exp_fixed(float x) {
+    x = fminf(fmaxf(x, -87.0f), 88.0f);
+    const float magic = 12582912.0f;
+    float t = __fmul_rn(x, 0x1.715476p+0f);
+    float n = __fadd_rn(__fadd_rn(t, magic), -magic);
+    float r = __fmaf_rn(n, -0x1.62e4p-1f, x);
+    r = __fmaf_rn(n, -0x1.7f7d1cp-20f, r);
+    float q = 0x1.a01a02p-13f;
+    q = __fmaf_rn(q, r, 0x1.6c16c2p-10f);
+    q = __fmaf_rn(q, r, 0x1.111112p-7f);
+    q = __fmaf_rn(q, r, 0x1.555556p-5f);
+    q = __fmaf_rn(q, r, 0x1.555556p-3f);
+    q = __fmaf_rn(q, r, 0.5f);
+    q = __fmaf_rn(q, r, 1.0f);
+    q = __fmaf_rn(q, r, 1.0f);
+    return __fmul_rn(q, __int_as_float(((int)n + 127) << 23));
+}
+
+__device__ __forceinline__ float log1p_fixed(float t) {
+    float s = __fdiv_rn(t, __fadd_rn(2.0f, t));
+    float u = __fmul_rn(s, s);
+    float q = 0x1.111112p-4f;
+    q = __fmaf_rn(q, u, 0x1.3b13b2p-4f);
+    q = __fmaf_rn(q, u, 0x1.745d18p-4f);
+    q = __fmaf_rn(q, u, 0x1.c71c72p-4f);
+    q = __fmaf_rn(q, u, 0x1.24924ap-3f);
+    q = __fmaf_rn(q, u, 0x1.99999ap-3f);
+    q = __fmaf_rn(q, u, 0x1.555556p-2f);
+    q = __fmaf_rn(q, u, 1.0f);
+    return __fmul_rn(__fmul_rn(2.0f, s), q);
+}
+
+__device__ __forceinline__ float delta_fixed(float z, float a) {
+    float sp = __fadd_rn(fmaxf(z, 0.0f), log1p_fixed(exp_fixed(-fabsf(z))));
+    return exp_fixed(__fmul_rn(a, sp));
+}
+
+// eight consecutive channels of one value row as fp32
+__device__ __forceinline__ void load8(const float* p, float (&v)[8]) {
+    float4 a = *reinterpret_cast<const float4*>(p), b = *reinterpret_cast<const float4*>(p + 4);
+    v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+}
+__device__ __forceinline__ void load8(const __nv_bfloat16* p, float (&v)[8]) {
+    uint4 a = *reinterpret_cast<const uint4*>(p);
+    uint32_t u[4] = {a.x, a.y, a.z, a.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        v[2 * i] = __uint_as_float(u[i] << 16);
+        v[2 * i + 1] = __uint_as_float(u[i] & 0xffff0000u);
+    }
+}
+
+// One CTA: kRows consecutive keys of one (batch, KV head); writes delta for the G query heads of the group.
+// A group of D/8 lanes owns a row: each lane forms the fma chain over its 8 channels, an xor butterfly adds
+// adjacent partials pairwise (IEEE addition commutes, so every lane of the group holds the same sum).
+template <typename T, int D>
+__global__ void __launch_bounds__(256) delta_kernel(const T* __restrict__ V, const float* __restrict__ W,
+                                                    const float* __restrict__ A, float* __restrict__ delta,
+                                                    int L, int Hq, int G, int64_t vs_b, int64_t vs_l, int64_t vs_h) {
+    constexpr int LPR = D / 8;            // lanes per row
+    constexpr int RPW = 32 / LPR;         // rows per warp and pass
+    constexpr int kRows = 128;
+    extern __shared__ float smem[];
+    float* sW = smem;                     // [G][D]
+    float* sOut = smem + G * D;           // [G][kRows]
+    const int hk = blockIdx.y, b = blockIdx.z, j0 = blockIdx.x * kRows;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int sub = lane % LPR, grp = lane / LPR;
+    for (int i = tid; i < G * D; i += 256) sW[i] = W[(size_t)hk * G * D + i];
+    __syncthreads();
+    for (int r0 = warp * RPW; r0 < kRows; r0 += 8 * RPW) {
+        const int r = r0 + grp, j = j0 + r;
+        float v[8];
+        if (j < L) {
+            load8(V + b * vs_b + (int64_t)j * vs_l + hk * vs_h + sub * 8, v);
+        } else {
+#pragma unroll
+            for (int c = 0; c < 8; ++c) v[c] = 0.0f;
+        }
+        for (int g = 0; g < G; ++g) {
+            const float* w = sW + g * D + sub * 8;
+            float p = 0.0f;
+#pragma unroll
+            for (int c = 0; c < 8; ++c) p = __fmaf_rn(v[c], w[c], p);
+#pragma unroll
+            for (int m = 1; m < LPR; m <<= 1) p = __fadd_rn(p, __shfl_xor_sync(0xffffffffu, p, m));
+            if (sub == g % LPR) sOut[g * kRows + r] = delta_fixed(p, A[hk * G + g]);
+        }
+    }
+    __syncthreads();
+    for (int i = tid; i < G * kRows; i += 256) {
+        const int g = i / kRows, r = i % kRows;
+        if (j0 + r < L) delta[((size_t)b * Hq + hk * G + g) * L + j0 + r] = sOut[i];
+    }
+}
+
+// ---- selection --------------------------------------------------------------------------------------------
+// Order: key a beats key b iff (delta_a, -a) > (delta_b, -b). delta > 0, so its bit pattern orders like the
+// value and one unsigned 64-bit compare decides.
+__device__ __forceinline__ unsigned long long sort_key(float dl, int j) {
+    return ((unsigned long long)__float_as_uint(dl) << 32) | (unsigned long long)(0xFFFFFFFFu - (unsigned)j);
+}
+
+__global__ void __launch_bounds__(kChunk) chunk_sort_kernel(const float* __restrict__ delta,
+                                                            unsigned long long* __restrict__ sorted, int L, int nchunk) {
+    __shared__ unsigned long long s[kChunk];
+    const int bh = blockIdx.y, c = blockIdx.x, t = threadIdx.x, j = c * kChunk + t;
+    s[t] = j < L ? sort_key(delta[(size_t)bh * L + j], j) : 0ull;   // padding sorts below every real key
+    __syncthreads();
+    for (int k = 2; k <= kChunk; k <<= 1)
+        for (int m = k >> 1; m > 0; m >>= 1) {
+            int o = t ^ m;
+            if (o > t) {
+                unsigned long long a = s[t], b = s[o];
+                bool up = (t & k) == 0;
+                if ((a > b) == up) { s[t] = b; s[o] = a; }
+            }
+            __syncthreads();
+        }
+    sorted[((size_t)bh * nchunk + c) * kChunk + t] = s[t];   // ascending
+}
+
+// expiry[j] = max(j, index of the w-th key in index order that beats j), or L if fewer than w keys beat it.
+__global__ void __launch_bounds__(kChunk) expiry_kernel(const float* __restrict__ delta,
+                                                        const unsigned long long* __restrict__ sorted,
+                                                        int32_t* __restrict__ expiry, int L, int w, int nchunk) {
+    __shared__ unsigned long long s[kChunk];
+    const int bh = blockIdx.y, t = threadIdx.x, j = blockIdx.x * kChunk + t;
+    const float* dl = delta + (size_t)bh * L;
+    const bool valid = j < L;
+    const unsigned long long key = valid ? sort_key(dl[j], j) : ~0ull;
+    int cnt = 0, e = L;
+    bool done = !valid;
+    for (int c = 0; c < nchunk; ++c) {
+        s[t] = sorted[((size_t)bh * nchunk + c) * kChunk + t];
+        __syncthreads();
+        if (!done) {
+            int lo = 0, hi = kChunk;              // first position whose key is greater than ours
+            while (lo < hi) {
+                int mid = (lo + hi) >> 1;
+                if (s[mid] > key) hi = mid; else lo = mid + 1;
+            }
+            const int n = kChunk - lo;
+            if (cnt + n >= w) {
+                int need = w - cnt;
+                for (int k = c * kChunk;; ++k)    // the need-th beater lies in this chunk: walk it in index order
+                    if (sort_key(dl[k], k) > key && --need == 0) { e = max(j, k); break; }
+                done = true;
+            }
+            cnt += n;
+        }
+        if (__syncthreads_and(done)) break;
+    }
+    if (valid) expiry[(size_t)bh * L + j] = e;
+}
+
+__global__ void fill_i32_kernel(int32_t* p, size_t n, int32_t v) {
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) p[i] = v;
+}
+
+// One CTA per (key tile, head): key j is kept by rows [j, expiry[j]), i.e. by query tiles j/bm .. (expiry[j]-1)/bm.
+// A difference array over query tiles forms the union; bits are OR-ed into the (pre-zeroed) bitmap.
+__global__ void __launch_bounds__(128) bitmap_kernel(const int32_t* __restrict__ expiry, uint32_t* __restrict__ bitmap,
+                                                     int L, int bm, int bn, int Tr, int Wd) {
+    extern __shared__ int diff[];                 // [Tr + 1]
+    const int kt = blockIdx.x, bh = blockIdx.y, t = threadIdx.x;
+    for (int i = t; i <= Tr; i += blockDim.x) diff[i] = 0;
+    __syncthreads();
+    const int jend = min(L, (kt + 1) * bn);
+    for (int j = kt * bn + t; j < jend; j += blockDim.x) {
+        const int e = expiry[(size_t)bh * L + j];
+        if (e > j) {
+            atomicAdd(&diff[j / bm], 1);
+            atomicAdd(&diff[(e - 1) / bm + 1], -1);
+        }
+    }
+    __syncthreads();
+    if (t == 0) {
+        int run = 0;
+        for (int q = 0; q < Tr; ++q) { run += diff[q]; diff[q] = run > 0; }
+    }
+    __syncthreads();
+    for (int q = t; q < Tr; q += blockDim.x)
+        if (diff[q]) atomicOr(&bitmap[((size_t)bh * Tr + q) * Wd + (kt >> 5)], 1u << (kt & 31));
+}
+
+}  // namespace
+
+size_t mask_ws_bytes(const Prob& P) {
+    const size_t nchunk = (P.L + kChunk - 1) / kChunk;
+    return kWsHeaderBytes + (size_t)P.B * P.Hq * nchunk * kChunk * sizeof(unsigned long long);
+}
+
+template <typename T, int D>
+static int launch_delta(const Prob& P, const void* V, const float* W, const float* A, float* bias, cudaStream_t st) {
+    dim3 grid((P.L + 127) / 128, P.Hkv, P.B);
+    size_t smem = (size_t)P.G * (D + 128) * sizeof(float);
+    if (smem > 48 * 1024) return DMA_ERR_UNSUPPORTED;
+    delta_kernel<T, D><<<grid, 256, smem, st>>>((const T*)V, W, A, bias, P.L, P.Hq, P.G, P.vs[0], P.vs[1], P.vs[2]);
+    count_launch();
+    return check_launch();
+}
+
+int launch_mask_build(const Prob& P, const void* V, const float* W, const float* A, float* bias, int32_t* expiry,
+                      uint32_t* bitmap, void* ws, cudaStream_t st) {
+    int rc;
+    if (P.dtype == DMA_BF16)
+        rc = P.d == 128 ? launch_delta<__nv_bfloat16, 128>(P, V, W, A, bias, st)
+                        : launch_delta<__nv_bfloat16, 64>(P, V, W, A, bias, st);
+    else
+        rc = P.d == 128 ? launch_delta<float, 128>(P, V, W, A, bias, st) : launch_delta<float, 64>(P, V, W, A, bias, st);
+    if (rc) return rc;
+
+    const int BH = P.B * P.Hq;
+    const int nchunk = (P.L + kChunk - 1) / kChunk;
+    if (P.w >= P.L) {   // every visible key is kept
+        size_t n = (size_t)BH * P.L;
+        fill_i32_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(expiry, n, P.L);
+        count_launch();
+    } else {
+        auto* sorted = reinterpret_cast<unsigned long long*>((char*)ws + kWsHeaderBytes);
+        chunk_sort_kernel<<<dim3(nchunk, BH), kChunk, 0, st>>>(bias, sorted, P.L, nchunk);
+        expiry_kernel<<<dim3(nchunk, BH), kChunk, 0, st>>>(bias, sorted, expiry, P.L, P.w, nchunk);
+        count_launch(2);
+    }
+    if ((rc = check_launch())) return rc;
+
+    if (cudaMemsetAsync(bitmap, 0, (size_t)BH * P.Tr * P.Wd * sizeof(uint32_t), st) != cudaSuccess) return DMA_ERR_CUDA;
+    size_t smem = (size_t)(P.Tr + 1) * sizeof(int);
+    if (smem > 48 * 1024) return DMA_ERR_UNSUPPORTED;
+    bitmap_kernel<<<dim3(P.Tc, BH), 128, smem, st>>>(expiry, bitmap, P.L, P.bm, P.bn, P.Tr, P.Wd);
+    count_launch();
+    return check_launch();
+}
+
+}  // namespace dma

@@ -1,0 +1,74 @@
+"""Shared test plumbing: run a workload through the C-ABI on the GPU, and through the CPU oracle."""
+import numpy as np
+import torch
+
+import oracle
+from paper_2508_02124_b200 import binding as dma
+
+# Tolerances of the parity gate: max-abs and whole-tensor relative L2, by element type.
+TOL = {"bf16": (2e-2, 5e-3), "fp32": (1e-4, 1e-4)}
+
+
+def f64(t):
+    return t.detach().cpu().to(torch.float64).numpy()
+
+
+def problem_of(case, **kw):
+    return dma.problem(case.B, case.Hq, case.Hkv, case.L, case.d, case.w, dtype=case.torch_dtype, **kw)
+
+
+def gpu_mask(case, inp, **kw):
+    p = problem_of(case, **kw)
+    dev = torch.device("cuda:0")
+    V = inp["V"].to(dev)
+    bias, expiry, bitmap = dma.dma_mask_build(p, V, inp["W_delta"].to(dev), inp["A"].to(dev))
+    torch.cuda.synchronize()
+    return p, bias, expiry, bitmap
+
+
+def gpu_run(case, inp, backward=True, mask=None, **kw):
+    """Full path on the GPU. `mask` = (bias, expiry, bitmap) CPU/GPU tensors to inject instead of building one."""
+    dev = torch.device("cuda:0")
+    p = problem_of(case, **kw)
+    Q, K, V, dO = (inp[k].to(dev) for k in ("Q", "K", "V", "dO"))
+    if mask is None:
+        bias, expiry, bitmap = dma.dma_mask_build(p, V, inp["W_delta"].to(dev), inp["A"].to(dev))
+    else:
+        bias, expiry, bitmap = (torch.as_tensor(m).to(dev) for m in mask)
+    O, lse = dma.dma_attn_fwd(p, Q, K, V, bias, expiry, bitmap)
+    out = {"bias": bias, "expiry": expiry, "bitmap": bitmap, "O": O, "lse": lse}
+    if backward:
+        dQ, dK, dV, dM = dma.dma_attn_bwd(p, Q, K, V, O, dO, lse, bias, expiry, bitmap)
+        out.update(dQ=dQ, dK=dK, dV=dV, dM=dM)
+    torch.cuda.synchronize()
+    return out
+
+
+def oracle_mask(case, inp, tile=(128, 128)):
+    """(delta fp32, expiry int32, bitmap uint32) from the oracle; V is passed as its exact fp32 image."""
+    z, dl = oracle.delta(inp["V"].float().numpy(), inp["W_delta"].numpy(), inp["A"].numpy(), case.Hq)
+    e = oracle.select_expiry(dl, min(case.w, case.L))
+    return dl, e, oracle.bitmap_from_expiry(e, *tile)
+
+
+def bits_equal(gpu_f32, ref_f32):
+    return np.array_equal(gpu_f32.detach().cpu().numpy().view(np.uint32), np.asarray(ref_f32, np.float32).view(np.uint32))
+
+
+def errors(got, ref):
+    """(max-abs, relative L2 over the whole tensor) of a GPU tensor against an fp64 numpy reference."""
+    g = f64(got) if isinstance(got, torch.Tensor) else np.asarray(got, np.float64)
+    diff = g - ref
+    den = np.sqrt((ref * ref).sum())
+    return float(np.abs(diff).max()), float(np.sqrt((diff * diff).sum()) / den) if den > 0 else float(np.abs(diff).max())
+
+
+def assert_close(got, ref, dtype, what, lse_like=False):
+    amax, rel = errors(got, ref)
+    tol_abs, tol_rel = TOL[dtype]
+    if lse_like:
+        # log-sum-exp carries the bias magnitude (delta can reach 1e2..1e4): an absolute error of one fp32 ulp
+        # at that magnitude already exceeds 1e-4, so the absolute bound scales with the reference magnitude.
+        tol_abs = max(tol_abs, tol_abs * float(np.abs(ref).max()) / 16.0)
+    assert amax <= tol_abs and rel <= tol_rel, f"{what}: max-abs {amax:.3e} (tol {tol_abs:.1e}), rel-L2 {rel:.3e} (tol {tol_rel:.1e})"
+    return amax, rel

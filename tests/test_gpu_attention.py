@@ -1,0 +1,144 @@
+"""GPU parity of the attention forward (Sec. 4.2) and backward (Sec. 4.3) against the CPU oracle (fp64
+instantiation, fed the same rounded inputs), through the C-ABI."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2508_02124_b200 import binding as dma
+from paper_2508_02124_b200 import workloads as wl
+
+from helpers import assert_close, f64, gpu_run, oracle_mask
+
+pytestmark = pytest.mark.gpu
+
+C1, C2 = wl.CONFIGS["1"], wl.CONFIGS["2"]
+CASES = [
+    C1,
+    wl.small(C1, L=1, w=1, name="fp32 L1"),
+    wl.small(C1, L=77, w=200, name="fp32 w>=L ragged"),
+    wl.small(C1, B=2, d=128, Hq=4, Hkv=2, L=321, w=50, name="fp32 d128 gqa ragged"),
+    wl.small(C2, B=2, Hq=4, Hkv=2, L=1000, w=129, backward=True, name="bf16 ragged gqa"),
+    wl.small(C2, B=1, Hq=8, Hkv=2, L=1024, w=256, backward=True, name="bf16 L1024"),
+    wl.small(C2, B=1, Hq=2, Hkv=1, L=640, w=1, backward=True, name="bf16 w=1"),
+    wl.small(C2, B=1, Hq=2, Hkv=2, L=130, w=999, backward=True, name="bf16 dense-causal"),
+    wl.small(C2, B=1, Hq=4, Hkv=4, L=512, w=64, d=64, backward=True, name="bf16 d64"),
+    wl.small(C2, B=1, Hq=4, Hkv=1, L=1536, w=200, backward=True, qk_scale=3.0, name="bf16 peaked"),
+]
+
+
+def oracle_all(case, inp, bias, e, backward=True):
+    Q, K, V, dO = (f64(inp[k]) for k in ("Q", "K", "V", "dO"))
+    O, lse = oracle.forward(Q, K, V, bias.astype(np.float64), expiry=e)
+    out = {"O": O, "lse": lse}
+    if backward:
+        dQ, dK, dV, dM = oracle.backward(Q, K, V, dO, bias.astype(np.float64), expiry=e)
+        out.update(dQ=dQ, dK=dK, dV=dV, dM=dM)
+    return out
+
+
+def compare(case, got, ref, backward=True):
+    assert_close(got["O"], ref["O"], case.dtype, "O")
+    assert_close(got["lse"], ref["lse"], case.dtype, "lse", lse_like=True)
+    if backward:
+        for k in ("dQ", "dK", "dV", "dM"):
+            assert_close(got[k], ref[k], case.dtype, k)
+
+
+@pytest.mark.parametrize("case", CASES, ids=lambda c: c.name)
+def test_forward_backward_small(case):
+    inp = wl.make_inputs(case)
+    dl, e, bmp = oracle_mask(case, inp)
+    got = gpu_run(case, inp)
+    assert np.array_equal(got["expiry"].cpu().numpy(), e)
+    ref = oracle_all(case, inp, dl, e)
+    compare(case, got, ref)
+    # block skipping is an optimisation only: ignoring the bitmap must give the same result
+    again = gpu_run(case, inp, flags=dma.DMA_FLAG_IGNORE_BITMAP)
+    compare(case, again, ref)
+
+
+@pytest.mark.parametrize("case", [c for c in CASES if c.dtype == "bf16"], ids=lambda c: c.name)
+def test_cuda_core_kernels_on_bf16(case):
+    inp = wl.make_inputs(case)
+    dl, e, bmp = oracle_mask(case, inp)
+    compare(case, gpu_run(case, inp, flags=dma.DMA_FLAG_SIMT), oracle_all(case, inp, dl, e))
+
+
+def test_injected_mask_zero_bias_is_dense_causal_attention():
+    # any self-consistent (bias, expiry, bitmap) is accepted: zero bias + everything kept = textbook causal attention
+    case = wl.small(C2, B=1, Hq=4, Hkv=2, L=700, w=700, backward=True, name="inject")
+    inp = wl.make_inputs(case)
+    B, Hq, L = case.B, case.Hq, case.L
+    bias = np.zeros((B, Hq, L), np.float32)
+    e = np.full((B, Hq, L), L, np.int32)
+    bmp = oracle.bitmap_from_expiry(e).view(np.int32)
+    got = gpu_run(case, inp, mask=(bias, e, bmp))
+    q, k, v = (inp[n].double().permute(0, 2, 1, 3) for n in ("Q", "K", "V"))
+    G = Hq // case.Hkv
+    ref = torch.nn.functional.scaled_dot_product_attention(q, k.repeat_interleave(G, 1), v.repeat_interleave(G, 1), is_causal=True)
+    assert_close(got["O"], ref.permute(0, 2, 1, 3).numpy(), "bf16", "O vs SDPA")
+    compare(case, got, oracle_all(case, inp, bias, e))
+
+
+def test_skipped_tiles_do_not_change_the_result_on_a_banded_mask():
+    # structured workload at reduced length: many inactive tiles
+    case = wl.small(wl.CONFIGS["S"], L=2048, w=256, Hq=6, Hkv=2, name="S-small")
+    inp = wl.make_inputs(case)
+    dl, e, bmp = oracle_mask(case, inp)
+    T = case.L // 128
+    t = np.arange(T)
+    active = ((bmp[..., t // 32] >> (t % 32)) & 1).sum()
+    assert active < 0.8 * case.B * case.Hq * T * (T + 1) / 2           # the mask really has holes
+    ref = oracle_all(case, inp, dl, e)
+    compare(case, gpu_run(case, inp), ref)
+    compare(case, gpu_run(case, inp, flags=dma.DMA_FLAG_IGNORE_BITMAP), ref)
+
+
+def sampled_check(case, inp, got, nrows=24, nkeys=6, seed=0):
+    """Full-size parity on sampled outputs: query rows (O, lse, dQ) and keys (dK, dV, dM) that the oracle
+    evaluates one by one. Keys are sampled near the end of the sequence (few rows keep them) plus the
+    globally strongest key of a head (kept by every later row)."""
+    rng = np.random.default_rng(seed)
+    dl, e, _ = oracle_mask(case, inp)
+    Q, K, V, dO = (f64(inp[k]) for k in ("Q", "K", "V", "dO"))
+    L = case.L
+    rows = np.unique(np.concatenate([[0, 1, 127, 128, L - 1], rng.integers(0, L, nrows)])).astype(np.int32)
+    O, lse = oracle.forward(Q, K, V, dl.astype(np.float64), expiry=e, rows=rows)
+    assert_close(got["O"][:, rows], O, case.dtype, "O rows")
+    assert_close(got["lse"][:, :, rows], lse, case.dtype, "lse rows", lse_like=True)
+    if not case.backward:
+        return
+    keys = np.unique(np.concatenate([[L - 1, L - 130], rng.integers(L - 600, L, nkeys)])).astype(np.int32)
+    _, dK, dV, dM = oracle.backward(Q, K, V, dO, dl.astype(np.float64), expiry=e, keys=keys, want_dq=False)
+    assert_close(got["dK"][:, keys], dK, case.dtype, "dK keys")
+    assert_close(got["dV"][:, keys], dV, case.dtype, "dV keys")
+    assert_close(got["dM"][:, :, keys], dM, case.dtype, "dM keys")
+    # properties that hold at any size (Sec. 4.3): rows of dS sum to zero; q.dQ and k.dK balance per KV group
+    dMs = f64(got["dM"]).sum(-1)
+    assert np.abs(dMs).max() < 0.5, dMs
+    G = case.Hq // case.Hkv
+    lhs = (Q * f64(got["dQ"])).sum(-1).reshape(case.B, L, case.Hkv, G).sum((1, 3))
+    rhs = (K * f64(got["dK"])).sum(-1).sum(1)
+    assert np.abs(lhs - rhs).max() <= 2e-2 * max(1.0, np.abs(rhs).max())
+
+
+def dq_rows_check(case, inp, got, rows):
+    """dQ on sampled rows: a one-head-group slice of the problem keeps the oracle's cost bounded."""
+    dl, e, _ = oracle_mask(case, inp)
+    G = case.Hq // case.Hkv
+    Q, K, V, dO = (f64(inp[k][:, :, :n]) for k, n in (("Q", G), ("K", 1), ("V", 1), ("dO", G)))
+    Lr = int(rows.max()) + 1                       # causal: rows < Lr only see keys < Lr
+    dQ, _, _, _ = oracle.backward(Q[:, :Lr], K[:, :Lr], V[:, :Lr], dO[:, :Lr], dl[:, :G, :Lr].astype(np.float64),
+                                  expiry=np.minimum(e[:, :G, :Lr], Lr), keys=np.array([0], np.int32))
+    assert_close(got["dQ"][:, rows, :G], dQ[:, rows], case.dtype, "dQ rows")
+
+
+@pytest.mark.parametrize("key", ["2", "3", "3x3", "4w256", "4w8192", "5", "S"])
+def test_full_size_configs_sampled(key):
+    case = wl.CONFIGS[key]
+    inp = wl.make_inputs(case)
+    got = gpu_run(case, inp, backward=case.backward)
+    sampled_check(case, inp, got)
+    if case.backward:
+        dq_rows_check(case, inp, got, np.array([0, 5, 130, 700, 1500]))
