@@ -139,10 +139,11 @@ def forward(Q, K, V, bias, expiry=None, keep=None, scale=None, rows=None, dtype=
     return O, LSE
 
 
-def backward(Q, K, V, dO, bias, expiry=None, keep=None, scale=None, keys=None, want_dq=True, dtype=np.float64):
+def backward(Q, K, V, dO, bias, expiry=None, keep=None, scale=None, keys=None, want_dq=True, dtype=np.float64, O=None):
     """Sec. 4.3 gradients with the mask and bias values held fixed. Returns (dQ, dK, dV, dM). With ``keys`` only
-    those keys are evaluated: dK,dV [B,len(keys),Hkv,d], dM [B,Hq,len(keys)] (dQ stays full, or None)."""
-    Q = _c(Q, dtype); K = _c(K, dtype); V = _c(V, dtype); dO = _c(dO, dtype); bias = _c(bias, dtype)
+    those keys are evaluated: dK,dV [B,len(keys),Hkv,d], dM [B,Hq,len(keys)] (dQ stays full, or None).
+    ``O`` is the stored forward output that Alg. 2 reads for D = rowsum(dO o O); None = the exact output."""
+    Q = _c(Q, dtype); K = _c(K, dtype); V = _c(V, dtype); dO = _c(dO, dtype); bias = _c(bias, dtype); O = _c(O, dtype)
     expiry = _c(expiry, np.int32); keep = _c(keep, np.uint8); keys = _c(keys, np.int32)
     B, L, Hq, d = Q.shape
     Hkv = K.shape[2]
@@ -153,7 +154,7 @@ def backward(Q, K, V, dO, bias, expiry=None, keep=None, scale=None, keys=None, w
     dV = np.empty((B, NK, Hkv, d), dtype)
     dM = np.empty((B, Hq, NK), dtype)
     f = lib().dmao_bwd_f64 if dtype == np.float64 else lib().dmao_bwd_f32
-    rc = f(_p(Q), _p(K), _p(V), _p(dO), _p(bias), _p(expiry), _p(keep), B, L, Hq, Hkv, d,
+    rc = f(_p(Q), _p(K), _p(V), _p(O), _p(dO), _p(bias), _p(expiry), _p(keep), B, L, Hq, Hkv, d,
            ctypes.c_double(scale), _p(keys), 0 if keys is None else len(keys), _p(dQ), _p(dK), _p(dV), _p(dM))
     assert rc == 0, rc
     return dQ, dK, dV, dM

@@ -187,13 +187,15 @@ int forward(const Problem<T>& P, const int32_t* rows, int nrows, T* O, T* LSE) {
     return 0;
 }
 
-// Backward of Sec. 4.3. Pass 1 (per query row): forward quantities, D_i = dO_i . o_i, and dQ_i.
+// Backward of Sec. 4.3. Pass 1 (per query row): forward quantities, D_i = dO_i . o_i, and dQ_i. Alg. 2 takes O
+// as an input read back from memory (D_i = rowsum(dO_i o O_i)), so when Ostored is given (the forward output as
+// it was stored, i.e. rounded to the element type) D uses it; when it is null D uses the exact o of this pass.
 // Pass 2 (per key): dV_j, dK_j (summed over the query heads sharing the KV head) and dM_j, each a
 // sum over the query rows that keep key j. keys == null: all keys; else only the listed keys, with
 // compact outputs dK,dV [B,nkeys,Hkv,d], dM [B,Hq,nkeys]; dQ may be null to skip it.
 template <class T>
-int backward(const Problem<T>& P, const T* dO, const int32_t* keys, int nkeys, T* dQ, T* dK, T* dV,
-             T* dM) {
+int backward(const Problem<T>& P, const T* Ostored, const T* dO, const int32_t* keys, int nkeys, T* dQ, T* dK,
+             T* dV, T* dM) {
     const int L = P.L, d = P.d, Hq = P.Hq, Hkv = P.Hkv, G = P.G();
     std::vector<T> LSE((size_t)P.B * Hq * L), D((size_t)P.B * Hq * L);
     std::vector<uint8_t> need((size_t)P.B * Hq * L, keys ? 0 : 1);
@@ -222,8 +224,9 @@ int backward(const Problem<T>& P, const T* dO, const int32_t* keys, int nkeys, T
             T lse;
             row_forward(P, b, h, i, idx, p, o.data(), &lse);
             const T* doi = dO + (((size_t)b * L + i) * Hq + h) * d;
+            const T* oi = Ostored ? Ostored + (((size_t)b * L + i) * Hq + h) * d : o.data();
             T Di = 0;
-            for (int c = 0; c < d; ++c) Di += doi[c] * o[c];
+            for (int c = 0; c < d; ++c) Di += doi[c] * oi[c];
             LSE[bhi] = lse;
             D[bhi] = Di;
             if (dQ) {
@@ -410,12 +413,12 @@ DMAO_FWD(dmao_fwd_f32, float)
 DMAO_FWD(dmao_fwd_f64, double)
 
 #define DMAO_BWD(NAME, T)                                                                            \
-    int NAME(const T* Q, const T* K, const T* V, const T* dO, const T* bias, const int32_t* expiry,  \
-             const uint8_t* keep, int B, int L, int Hq, int Hkv, int d, double scale,                \
+    int NAME(const T* Q, const T* K, const T* V, const T* Ostored, const T* dO, const T* bias,       \
+             const int32_t* expiry, const uint8_t* keep, int B, int L, int Hq, int Hkv, int d, double scale, \
              const int32_t* keys, int nkeys, T* dQ, T* dK, T* dV, T* dM) {                           \
         if (Hq % Hkv || (!expiry && !keep)) return -1;                                               \
         return backward<T>(make_problem<T>(B, L, Hq, Hkv, d, scale, Q, K, V, bias, expiry, keep),   \
-                           dO, keys, nkeys, dQ, dK, dV, dM);                                         \
+                           Ostored, dO, keys, nkeys, dQ, dK, dV, dM);                                         \
     }
 DMAO_BWD(dmao_bwd_f32, float)
 DMAO_BWD(dmao_bwd_f64, double)

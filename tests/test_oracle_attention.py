@@ -211,3 +211,25 @@ def test_backward_key_subset_equals_full():
     dQs, dKs, dVs, dMs = oracle.backward(Q, K, V, dO, bias, expiry=e, keys=keys, want_dq=False)
     assert dQs is None
     assert (dKs == dK[:, keys]).all() and (dVs == dV[:, keys]).all() and (dMs == dM[:, :, keys]).all()
+
+
+def test_backward_with_stored_output():
+    # Alg. 2 reads O back from memory for D = rowsum(dO o O): passing the exact O changes nothing; passing a
+    # perturbed O moves D by dO.(O' - O) and hence dS by -p * that, which for dM (column sums of dS) is checkable.
+    Q, K, V, dO, bias, e = rand_case(11, B=1, L=40, Hq=2, Hkv=1, d=8, w=6)
+    O, _ = oracle.forward(Q, K, V, bias, expiry=e)
+    base = oracle.backward(Q, K, V, dO, bias, expiry=e)
+    same = oracle.backward(Q, K, V, dO, bias, expiry=e, O=O)
+    for a, b in zip(base, same):
+        assert np.abs(a - b).max() < 1e-13
+    O2 = O + 0.01
+    pert = oracle.backward(Q, K, V, dO, bias, expiry=e, O=O2)
+    shift = (dO * (O2 - O)).sum(-1)                                    # [B, L, Hq] change of D_i
+    keep = oracle.keep_from_expiry(e).astype(np.float64)
+    s = np.einsum("blhc,bmhc->bhlm", Q, np.repeat(K, 2, axis=2)) / math.sqrt(8) + bias[:, :, None, :]
+    s = np.where(keep > 0, s, -np.inf)
+    p = np.exp(s - s.max(-1, keepdims=True))
+    p /= p.sum(-1, keepdims=True)
+    expect_dM = base[3] - np.einsum("bhlm,blh->bhm", p, shift)
+    assert np.abs(pert[3] - expect_dM).max() < 1e-12
+    assert np.abs(pert[2] - base[2]).max() < 1e-13                     # dV does not depend on D
