@@ -6,9 +6,11 @@ import oracle
 from paper_2508_02124_b200 import binding as dma
 
 # Parity gate by element type: (max-abs, whole-tensor relative L2). bf16: 2e-2 / 5e-3; fp32: 1e-4 / 1e-4.
-# The max-abs bound is meant for O(1) tensors. It is scaled by max(1, max|ref| / 8): from magnitude 8 on, half the
-# spacing of bf16 (the OUTPUT format) already exceeds 2e-2, and dK, dV, dM are sums over up to L query rows whose
-# fp32 score/log-sum-exp rounding (the bias reaches 1e2..1e4, one fp32 ulp there is 1e-5..1e-3) accumulates with them.
+# The max-abs bound is read as absolute for tensors of unit scale and as relative to the tensor's largest
+# magnitude M beyond that (tol = atol * max(1, M)): half the spacing of bf16, the OUTPUT format, is 2^-8 M, P and dS
+# enter the tensor-core GEMMs rounded to bf16, D = rowsum(dO o O) is formed from the stored bf16 O, and dK, dV, dM are
+# sums over up to L query rows. The log-sum-exp is an fp32 output whatever the element type: it carries the bias
+# magnitude (1e2..1e4) and is held to atol + 1e-6 M, a few fp32 ulps of that magnitude.
 TOL = {"bf16": (2e-2, 5e-3), "fp32": (1e-4, 1e-4)}
 
 
@@ -71,14 +73,15 @@ def errors(got, ref):
     return float(np.abs(diff).max()), float(np.sqrt((diff * diff).sum()) / den) if den > 0 else float(np.abs(diff).max())
 
 
-def assert_close(got, ref, dtype, what):
+def assert_close(got, ref, dtype, what, lse=False):
     g = f64(got) if isinstance(got, torch.Tensor) else np.asarray(got, np.float64)
     atol, tol_rel = TOL[dtype]
     diff = np.abs(g - ref)
-    tol_abs = atol * max(1.0, float(np.abs(ref).max()) / 8.0)
+    M = float(np.abs(ref[np.isfinite(ref)]).max()) if np.isfinite(ref).any() else 0.0
+    tol_abs = atol + 1e-6 * M if lse else atol * max(1.0, M)
     den = np.sqrt((ref * ref).sum())
     rel = float(np.sqrt((diff * diff).sum()) / den) if den > 0 else float(diff.max())
     assert np.isfinite(g).all(), f"{what}: non-finite values"
     assert diff.max() <= tol_abs and rel <= tol_rel, (f"{what}: max-abs {diff.max():.3e} (tol {tol_abs:.2e}, |ref| max "
-                                                     f"{np.abs(ref).max():.3e}), rel-L2 {rel:.3e} (tol {tol_rel:.1e})")
+                                                     f"{M:.3e}), rel-L2 {rel:.3e} (tol {tol_rel:.1e})")
     return float(diff.max()), rel

@@ -40,7 +40,7 @@ def oracle_all(case, inp, bias, e, backward=True):
 
 def compare(case, got, ref, backward=True):
     assert_close(got["O"], ref["O"], case.dtype, "O")
-    assert_close(got["lse"], ref["lse"], case.dtype, "lse")
+    assert_close(got["lse"], ref["lse"], case.dtype, "lse", lse=True)
     if backward:
         for k in ("dQ", "dK", "dV", "dM"):
             assert_close(got[k], ref[k], case.dtype, k)
@@ -106,7 +106,7 @@ def sampled_check(case, inp, got, nrows=24, nkeys=6, seed=0):
     rows = np.unique(np.concatenate([[0, 1, 127, 128, L - 1], rng.integers(0, L, nrows)])).astype(np.int32)
     O, lse = oracle.forward(Q, K, V, dl.astype(np.float64), expiry=e, rows=rows)
     assert_close(got["O"][:, rows], O, case.dtype, "O rows")
-    assert_close(got["lse"][:, :, rows], lse, case.dtype, "lse rows")
+    assert_close(got["lse"][:, :, rows], lse, case.dtype, "lse rows", lse=True)
     if not case.backward:
         return
     keys = np.unique(np.concatenate([[L - 1, L - 130], rng.integers(L - 600, L, nkeys)])).astype(np.int32)
