@@ -1,10 +1,447 @@
-// placeholder until the tcgen05 backward lands
+// Tensor-core backward (Sec. 4.3, Alg. 2) for bf16, d = 128, on sm_100a.
+//
+// One CTA owns one 128-key tile of one KV head and, as in Alg. 2's outer loop, keeps dK, dV (fp32, tensor memory)
+// and dM (registers) for it while walking the query heads of the group and their active query tiles in steps of
+// 64 query rows. Everything is computed transposed, keys on the 128 TMEM lanes, so that dM is a per-thread row sum
+// and P^T, dS^T feed the dV / dK GEMMs straight from tensor memory:
+//   S^T  = K Q^T            dP^T = V dO^T                      (smem x smem  -> TMEM, 64 columns each)
+//   P^T  = exp2(S^T c + log2e (bias_j - lse_i)) where j <= i < expiry[j], else 0;   dS^T = P^T o (dP^T - D_i)
+//   dV  += P^T dO           dK  += dS^T Q                      (TMEM x smem  -> TMEM, 128 columns each)
+//   dQ^T = K^T dS^T                                            (smem x smem  -> TMEM, 64 columns), then added to the
+//                                                              fp32 dQ accumulator in global memory with red.add
+// Warp roles: warps 0-3 compute group (thread = key), warps 4-7 dQ drain group (thread = channel), warp 8 TMA
+// producer + schedule, warp 9 MMA issuer, warps 10-11 idle (register donors).
+// TMEM columns: dK [0,128) dV [128,256) S^T [256,320) dP^T [320,384) P^T [384,416) dS^T [416,448) dQ^T [448,512).
 #include "common.cuh"
+#include "sm100_ptx.cuh"
+
 namespace dma {
-size_t tc_bwd_ws_bytes(const Prob& P) { return simt_bwd_ws_bytes(P); }
+namespace {
+
+using namespace ptx;
+
+constexpr int kStages = 3;
+constexpr int kMaxSteps = 4096;
+constexpr int kThreads = 384;
+constexpr uint32_t kKVBytes = 128 * 128 * 2;   // K or V tile: two 16 KB halves (channels 0-63 | 64-127)
+constexpr uint32_t kQBytes = 64 * 128 * 2;     // Q or dO step tile (64 rows): two 8 KB halves
+constexpr int cDK = 0, cDV = 128, cS = 256, cDP = 320, cP = 384, cDS = 416, cDQ = 448;
+
+struct SharedStorage {
+    alignas(1024) uint8_t k[kKVBytes];
+    alignas(1024) uint8_t v[kKVBytes];
+    alignas(1024) uint8_t q[kStages][kQBytes];
+    alignas(1024) uint8_t g[kStages][kQBytes];       // dO
+    alignas(1024) uint8_t ds[128 * 128];             // dS^T as bf16: [128 keys][64 queries], 128-byte swizzled rows
+    alignas(16) float nlse[kStages][64];             // -log2(e) * lse_i
+    alignas(16) float dvec[kStages][64];             // D_i
+    uint32_t sched[kMaxSteps];                       // head-in-group << 24 | query tile << 1 | half
+    uint64_t kv_full, qd_full[kStages], qd_empty[kStages];
+    uint64_t sdp_full, sdp_free, pds_ready, pds_free, dq_full, dq_free;
+    uint32_t tmem_base;
+    int n_steps;
+    int abort_flag;
+};
+
+struct BwdParams {
+    const float* lse;
+    const float* Dv;
+    const float* bias;
+    const int32_t* expiry;
+    const uint32_t* bitmap;
+    float* dQacc;               // [B, L, Hq, 128] fp32, zeroed
+    __nv_bfloat16* dK;
+    __nv_bfloat16* dV;
+    float* dM;
+    int32_t* status;
+    int B, Hq, Hkv, G, L, Tr, Tc, Wd, ignore_bitmap;
+    float scale, scale_log2;
+    int64_t ks_b, ks_l, ks_h, vs_b, vs_l, vs_h;
+};
+
+__device__ __forceinline__ void red_add_f32(float* addr, float v) {
+    asm volatile("red.global.add.f32 [%0], %1;" ::"l"(addr), "f"(v) : "memory");
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+           const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmG, const BwdParams P) {
+    extern __shared__ uint8_t smem_raw[];
+    SharedStorage& S = *reinterpret_cast<SharedStorage*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int b = blockIdx.x / P.Hkv, hk = blockIdx.x % P.Hkv;
+    const int kt = blockIdx.y;                         // key tile 0 has the most query tiles: heaviest first
+    const int j0 = kt * 128;
+    volatile int* abort_flag = &S.abort_flag;
+
+    if (tid == 0) {
+        mbar_init(&S.kv_full, 1);
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(&S.qd_full[s], 1);
+            mbar_init(&S.qd_empty[s], 1);
+        }
+        mbar_init(&S.sdp_full, 1);
+        mbar_init(&S.sdp_free, 128);
+        mbar_init(&S.pds_ready, 128);
+        mbar_init(&S.pds_free, 1);
+        mbar_init(&S.dq_full, 1);
+        mbar_init(&S.dq_free, 128);
+        S.abort_flag = 0;
+        S.n_steps = 0;
+        fence_barrier_init();
+    }
+    if (warp == 9) {
+        tmem_alloc(&S.tmem_base, 512);
+        tmem_relinquish();
+    }
+    if (warp == 8) {
+        // schedule: for each query head of the group, the active query tiles (ascending), two 64-row steps each
+        if (lane == 0) { prefetch_tmap(&tmQ); prefetch_tmap(&tmK); prefetch_tmap(&tmV); prefetch_tmap(&tmG); }
+        int n = 0;
+        for (int g = 0; g < P.G; ++g) {
+            const int bh = b * P.Hq + hk * P.G + g;
+            for (int base = kt; base < P.Tr; base += 32) {
+                const int qt = base + lane;
+                const bool act = qt < P.Tr && (P.ignore_bitmap || bitmap_test(P.bitmap, P.Tr, P.Wd, bh, qt, kt));
+                const int halves = act ? ((qt * 128 + 64 < P.L) ? 2 : 1) : 0;
+                // exclusive prefix sum of `halves` over the warp
+                int incl = halves;
+                for (int o = 1; o < 32; o <<= 1) {
+                    int t = __shfl_up_sync(0xffffffffu, incl, o);
+                    if (lane >= o) incl += t;
+                }
+                const int pos = n + incl - halves;
+                for (int hf = 0; hf < halves; ++hf)
+                    if (pos + hf < kMaxSteps) S.sched[pos + hf] = ((uint32_t)g << 24) | ((uint32_t)qt << 1) | (uint32_t)hf;
+                n += __shfl_sync(0xffffffffu, incl, 31);
+            }
+        }
+        if (lane == 0) S.n_steps = min(n, kMaxSteps);
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = S.tmem_base;
+    const int n_steps = S.n_steps;
+
+    if (warp < 4) {
+        // ============================ compute group: thread = key j, columns = query rows ============================
+        setmaxnreg_inc<216>();
+        const int r = tid;                                  // key within the tile = TMEM lane
+        const int j = j0 + r;
+        const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+        float dm = 0.0f, bj = 0.0f;
+        int len = 0, cur_g = -1;
+        bool ok = true;
+        for (int n = 0; n < n_steps && ok; ++n) {
+            const uint32_t e = S.sched[n];
+            const int g = (int)(e >> 24), i0 = (int)((e >> 1) & 0x7FFFFF) * 128 + (int)(e & 1) * 64;
+            const int st = n % kStages;
+            if (g != cur_g) {
+                const int bh = b * P.Hq + hk * P.G + g;
+                if (cur_g >= 0 && j < P.L) P.dM[(size_t)(bh - (g - cur_g)) * P.L + j] = dm;
+                dm = 0.0f;
+                bj = j < P.L ? P.bias[(size_t)bh * P.L + j] * 1.4426950408889634f : 0.0f;
+                len = j < P.L ? P.expiry[(size_t)bh * P.L + j] - j : 0;
+                cur_g = g;
+            }
+            ok = mbar_wait_warp(&S.sdp_full, n & 1, abort_flag) && mbar_wait_warp(&S.qd_full[st], (n / kStages) & 1, abort_flag);
+            if (!ok) break;
+            tc_fence_after();
+            uint32_t sr[64], pr[64];
+#pragma unroll
+            for (int c = 0; c < 2; ++c) {
+                tmem_ld32(tmem + lane_base + cS + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&sr[c * 32]));
+                tmem_ld32(tmem + lane_base + cDP + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&pr[c * 32]));
+            }
+            tc_wait_ld();
+            tc_fence_before();
+            mbar_arrive(&S.sdp_free);
+            // valid columns of this thread: col in [lo, lo + width)
+            const int lo = max(0, j - i0);
+            const int width = max(0, min(64, j - i0 + len) - lo);
+            uint32_t pp[32], dd[32];
+#pragma unroll
+            for (int c = 0; c < 64; c += 4) {
+                const float4 nl = *reinterpret_cast<const float4*>(&S.nlse[st][c]);
+                const float4 dv = *reinterpret_cast<const float4*>(&S.dvec[st][c]);
+                const float nlv[4] = {nl.x, nl.y, nl.z, nl.w};
+                const float dvv[4] = {dv.x, dv.y, dv.z, dv.w};
+                float p[4], ds[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const float x = fmaf(__uint_as_float(sr[c + u]), P.scale_log2, bj + nlv[u]);
+                    const bool valid = (unsigned)(c + u - lo) < (unsigned)width;
+                    p[u] = valid ? ex2(x) : 0.0f;
+                    ds[u] = p[u] * (__uint_as_float(pr[c + u]) - dvv[u]);
+                    dm += ds[u];
+                }
+                pp[(c >> 1)] = pack_bf16(p[0], p[1]);
+                pp[(c >> 1) + 1] = pack_bf16(p[2], p[3]);
+                dd[(c >> 1)] = pack_bf16(ds[0], ds[1]);
+                dd[(c >> 1) + 1] = pack_bf16(ds[2], ds[3]);
+            }
+            // the previous step's dV / dK / dQ GEMMs must have finished reading P^T, dS^T (TMEM) and dS^T (smem)
+            if (n > 0) ok = mbar_wait_warp(&S.pds_free, (n - 1) & 1, abort_flag);
+            if (!ok) break;
+            tc_fence_after();
+            tmem_st32(tmem + lane_base + cP, pp);
+            tmem_st32(tmem + lane_base + cDS, dd);
+            {   // dS^T row r -> shared memory, eight 16-byte chunks, chunk index XOR (row % 8) (128-byte swizzle)
+                uint8_t* row = S.ds + r * 128;
+#pragma unroll
+                for (int c = 0; c < 8; ++c)
+                    *reinterpret_cast<uint4*>(row + ((c ^ (r & 7)) << 4)) = make_uint4(dd[4 * c], dd[4 * c + 1], dd[4 * c + 2], dd[4 * c + 3]);
+            }
+            fence_proxy_async();
+            tc_wait_st();
+            tc_fence_before();
+            mbar_arrive(&S.pds_ready);
+        }
+        if (cur_g >= 0 && j < P.L) P.dM[(size_t)(b * P.Hq + hk * P.G + cur_g) * P.L + j] = dm;
+        // heads of the group that had no active tile for this key tile: dM = 0
+        if (ok && j < P.L) {
+            uint32_t seen = 0;
+            for (int n = 0; n < n_steps; ++n) seen |= 1u << (S.sched[n] >> 24);
+            for (int g = 0; g < P.G; ++g)
+                if (!((seen >> g) & 1u)) P.dM[(size_t)(b * P.Hq + hk * P.G + g) * P.L + j] = 0.0f;
+        }
+        // epilogue: dK (scaled) and dV rows to global memory
+        if (ok && n_steps > 0) ok = mbar_wait_warp(&S.pds_free, (n_steps - 1) & 1, abort_flag);
+        if (ok) {
+            tc_fence_after();
+            __nv_bfloat16* dk = P.dK + b * P.ks_b + (int64_t)j * P.ks_l + hk * P.ks_h;
+            __nv_bfloat16* dv = P.dV + b * P.vs_b + (int64_t)j * P.vs_l + hk * P.vs_h;
+#pragma unroll
+            for (int which = 0; which < 2; ++which) {
+                const float mul = which == 0 ? P.scale : 1.0f;
+                __nv_bfloat16* out = which == 0 ? dk : dv;
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t o[32];
+                    if (n_steps > 0) {
+                        tmem_ld32(tmem + lane_base + (which == 0 ? cDK : cDV) + c * 32, o);
+                        tc_wait_ld();
+                    } else {
+#pragma unroll
+                        for (int u = 0; u < 32; ++u) o[u] = 0;
+                    }
+                    if (j < P.L) {
+#pragma unroll
+                        for (int u = 0; u < 32; u += 8) {
+                            uint4 pkt;
+                            pkt.x = pack_bf16(__uint_as_float(o[u]) * mul, __uint_as_float(o[u + 1]) * mul);
+                            pkt.y = pack_bf16(__uint_as_float(o[u + 2]) * mul, __uint_as_float(o[u + 3]) * mul);
+                            pkt.z = pack_bf16(__uint_as_float(o[u + 4]) * mul, __uint_as_float(o[u + 5]) * mul);
+                            pkt.w = pack_bf16(__uint_as_float(o[u + 6]) * mul, __uint_as_float(o[u + 7]) * mul);
+                            *reinterpret_cast<uint4*>(out + c * 32 + u) = pkt;
+                        }
+                    }
+                }
+            }
+        }
+    } else if (warp < 8) {
+        // ============================ dQ drain group: thread = channel c, columns = query rows ============================
+        setmaxnreg_inc<216>();
+        const int c = tid - 128;
+        const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+        bool ok = true;
+        for (int n = 0; n < n_steps && ok; ++n) {
+            const uint32_t e = S.sched[n];
+            const int g = (int)(e >> 24), i0 = (int)((e >> 1) & 0x7FFFFF) * 128 + (int)(e & 1) * 64;
+            ok = mbar_wait_warp(&S.dq_full, n & 1, abort_flag);
+            if (!ok) break;
+            tc_fence_after();
+            uint32_t v[64];
+            tmem_ld32(tmem + lane_base + cDQ, *reinterpret_cast<uint32_t(*)[32]>(&v[0]));
+            tmem_ld32(tmem + lane_base + cDQ + 32, *reinterpret_cast<uint32_t(*)[32]>(&v[32]));
+            tc_wait_ld();
+            tc_fence_before();
+            mbar_arrive(&S.dq_free);
+            float* base = P.dQacc + (((size_t)b * P.L + i0) * P.Hq + hk * P.G + g) * 128 + c;
+            const int rows = min(64, P.L - i0);
+#pragma unroll
+            for (int u = 0; u < 64; ++u)
+                if (u < rows) red_add_f32(base + (size_t)u * P.Hq * 128, __uint_as_float(v[u]) * P.scale);
+        }
+    } else {
+        setmaxnreg_dec<72>();      // 4 warps x 96 registers released = 8 warps x 48 acquired above
+        if (warp == 8) {
+            // ============================ producer ============================
+            if (lane == 0) {
+                mbar_arrive_expect_tx(&S.kv_full, 2 * kKVBytes);
+                for (int hf = 0; hf < 2; ++hf) {
+                    tma_load_4d(&S.k[hf * (kKVBytes / 2)], &tmK, &S.kv_full, hf * 64, j0, hk, b);
+                    tma_load_4d(&S.v[hf * (kKVBytes / 2)], &tmV, &S.kv_full, hf * 64, j0, hk, b);
+                }
+            }
+            bool ok = true;
+            for (int n = 0; n < n_steps && ok; ++n) {
+                const uint32_t e = S.sched[n];
+                const int h = hk * P.G + (int)(e >> 24), i0 = (int)((e >> 1) & 0x7FFFFF) * 128 + (int)(e & 1) * 64;
+                const int st = n % kStages;
+                if (n >= kStages) ok = mbar_wait_warp(&S.qd_empty[st], ((n / kStages) - 1) & 1, abort_flag);
+                if (!ok) break;
+                const size_t rowbase = (size_t)(b * P.Hq + h) * P.L;
+#pragma unroll
+                for (int c = lane; c < 64; c += 32) {
+                    const int i = i0 + c;
+                    S.nlse[st][c] = i < P.L ? -1.4426950408889634f * P.lse[rowbase + i] : 0.0f;
+                    S.dvec[st][c] = i < P.L ? P.Dv[rowbase + i] : 0.0f;
+                }
+                __syncwarp();
+                if (lane == 0) {
+                    mbar_arrive_expect_tx(&S.qd_full[st], 2 * kQBytes);
+                    for (int hf = 0; hf < 2; ++hf) {
+                        tma_load_4d(&S.q[st][hf * (kQBytes / 2)], &tmQ, &S.qd_full[st], hf * 64, i0, h, b);
+                        tma_load_4d(&S.g[st][hf * (kQBytes / 2)], &tmG, &S.qd_full[st], hf * 64, i0, h, b);
+                    }
+                }
+            }
+            for (int n = max(0, n_steps - kStages); n < n_steps && ok; ++n)
+                ok = mbar_wait_warp(&S.qd_empty[n % kStages], (n / kStages) & 1, abort_flag);
+        } else if (warp == 9 && lane == 0) {
+            // ============================ MMA issuer ============================
+            constexpr uint32_t id_sdp = idesc_bf16(128, 64, 0, 0);     // K|V (K-major) x Q|dO (K-major)       -> 128 x 64
+            constexpr uint32_t id_dkv = idesc_bf16(128, 128, 0, 1);    // P^T|dS^T (TMEM) x dO|Q (MN-major)    -> 128 x 128
+            constexpr uint32_t id_dq = idesc_bf16(128, 64, 1, 1);      // K^T (MN-major) x dS^T (MN-major)     -> 128 x 64
+            auto issue_sdp = [&](int st) {
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk) {
+                    const uint32_t offa = (kk >> 2) * (kKVBytes / 2) + (kk & 3) * 32, offb = (kk >> 2) * (kQBytes / 2) + (kk & 3) * 32;
+                    mma_ss(tmem + cS, smem_desc_sw128(smem_u32(&S.k[offa]), 16, 1024),
+                           smem_desc_sw128(smem_u32(&S.q[st][offb]), 16, 1024), id_sdp, kk > 0);
+                }
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk) {
+                    const uint32_t offa = (kk >> 2) * (kKVBytes / 2) + (kk & 3) * 32, offb = (kk >> 2) * (kQBytes / 2) + (kk & 3) * 32;
+                    mma_ss(tmem + cDP, smem_desc_sw128(smem_u32(&S.v[offa]), 16, 1024),
+                           smem_desc_sw128(smem_u32(&S.g[st][offb]), 16, 1024), id_sdp, kk > 0);
+                }
+                tc_commit(&S.sdp_full);
+            };
+            bool ok = mbar_wait(&S.kv_full, 0, abort_flag);
+            if (ok && n_steps > 0) {
+                ok = mbar_wait(&S.qd_full[0], 0, abort_flag);
+                if (ok) {
+                    tc_fence_after();
+                    issue_sdp(0);
+                }
+            }
+            for (int n = 0; n < n_steps && ok; ++n) {
+                const int st = n % kStages;
+                if (n + 1 < n_steps) {
+                    const int nst = (n + 1) % kStages;
+                    ok = mbar_wait(&S.qd_full[nst], ((n + 1) / kStages) & 1, abort_flag) && mbar_wait(&S.sdp_free, n & 1, abort_flag);
+                    if (!ok) break;
+                    tc_fence_after();
+                    issue_sdp(nst);
+                }
+                ok = mbar_wait(&S.pds_ready, n & 1, abort_flag);
+                if (ok && n > 0) ok = mbar_wait(&S.dq_free, (n - 1) & 1, abort_flag);
+                if (!ok) break;
+                tc_fence_after();
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk) {       // 64 query rows = 4 k-steps of 16
+                    mma_ts(tmem + cDV, tmem + cP + kk * 8, smem_desc_sw128(smem_u32(&S.g[st][kk * 2048]), kQBytes / 2, 1024),
+                           id_dkv, (n > 0 || kk > 0) ? 1u : 0u);
+                }
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk) {
+                    mma_ts(tmem + cDK, tmem + cDS + kk * 8, smem_desc_sw128(smem_u32(&S.q[st][kk * 2048]), kQBytes / 2, 1024),
+                           id_dkv, (n > 0 || kk > 0) ? 1u : 0u);
+                }
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk) {       // 128 keys = 8 k-steps of 16
+                    mma_ss(tmem + cDQ, smem_desc_sw128(smem_u32(&S.k[kk * 2048]), kKVBytes / 2, 1024),
+                           smem_desc_sw128(smem_u32(&S.ds[kk * 2048]), 16, 1024), id_dq, kk > 0);
+                }
+                tc_commit(&S.pds_free);
+                tc_commit(&S.dq_full);
+                tc_commit(&S.qd_empty[st]);
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 9) {
+        tc_fence_after();
+        tmem_dealloc(tmem, 512);
+    }
+    if (tid == 0 && S.abort_flag) atomicExch(P.status, (int32_t)DMA_ERR_DEVICE_TIMEOUT);
+}
+
+// D_i = dO_i . O_i  (Alg. 2): one warp per (b, h, i), 16-byte loads
+__global__ void rowdot_bf16_kernel(const __nv_bfloat16* __restrict__ O, const __nv_bfloat16* __restrict__ dO,
+                                   float* __restrict__ Dv, int B, int L, int Hq, int64_t os_b, int64_t os_l, int64_t os_h) {
+    const long row = (long)blockIdx.x * (blockDim.x / 32) + threadIdx.x / 32;
+    const int lane = threadIdx.x % 32;
+    if (row >= (long)B * Hq * L) return;
+    const int i = row % L, h = (row / L) % Hq, b = row / ((long)L * Hq);
+    const int64_t off = b * os_b + (int64_t)i * os_l + h * os_h + (lane & 15) * 8;
+    float s = 0.0f;
+    if (lane < 16) {
+        const uint4 a = *reinterpret_cast<const uint4*>(O + off), g = *reinterpret_cast<const uint4*>(dO + off);
+        const uint32_t au[4] = {a.x, a.y, a.z, a.w}, gu[4] = {g.x, g.y, g.z, g.w};
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+            s = fmaf(__uint_as_float(au[t] << 16), __uint_as_float(gu[t] << 16), s);
+            s = fmaf(__uint_as_float(au[t] & 0xffff0000u), __uint_as_float(gu[t] & 0xffff0000u), s);
+        }
+    }
+    for (int m = 8; m; m >>= 1) s += __shfl_xor_sync(0xffffffffu, s, m);
+    if (lane == 0) Dv[row] = s;
+}
+
+// fp32 accumulator [B, L, Hq, 128] -> bf16 dQ in the caller's layout; 8 elements per thread
+__global__ void dq_convert_bf16_kernel(const float* __restrict__ acc, __nv_bfloat16* __restrict__ dQ, size_t n8, int L, int Hq,
+                                       int64_t qs_b, int64_t qs_l, int64_t qs_h) {
+    const size_t t = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= n8) return;
+    const size_t e = t * 8;
+    const int c = e % 128, h = (e / 128) % Hq, i = (e / ((size_t)128 * Hq)) % L, b = e / ((size_t)128 * Hq * L);
+    const float4 a = *reinterpret_cast<const float4*>(acc + e), bb = *reinterpret_cast<const float4*>(acc + e + 4);
+    uint4 o;
+    o.x = ptx::pack_bf16(a.x, a.y); o.y = ptx::pack_bf16(a.z, a.w); o.z = ptx::pack_bf16(bb.x, bb.y); o.w = ptx::pack_bf16(bb.z, bb.w);
+    *reinterpret_cast<uint4*>(dQ + b * qs_b + (int64_t)i * qs_l + h * qs_h + c) = o;
+}
+
+}  // namespace
+
+size_t tc_bwd_ws_bytes(const Prob& P) {
+    const size_t rows = (size_t)P.B * P.Hq * P.L;
+    return kWsHeaderBytes + (((rows + 63) / 64) * 64 + rows * P.d) * sizeof(float);
+}
+
 int launch_tc_bwd(const Prob& P, const void* Q, const void* K, const void* V, const void* O, const void* dO,
                   const float* lse, const float* bias, const int32_t* expiry, const uint32_t* bitmap, void* dQ,
                   void* dK, void* dV, float* dM, void* ws, cudaStream_t st) {
-    return launch_simt_bwd(P, Q, K, V, O, dO, lse, bias, expiry, bitmap, dQ, dK, dV, dM, ws, st);
+    if ((size_t)P.G * P.Tr * 2 > (size_t)kMaxSteps) return DMA_ERR_UNSUPPORTED;
+    const size_t rows = (size_t)P.B * P.Hq * P.L, nq = rows * P.d;
+    float* Dv = reinterpret_cast<float*>((char*)ws + kWsHeaderBytes);
+    float* acc = Dv + ((rows + 63) / 64) * 64;
+    CUtensorMap tmQ, tmK, tmV, tmG;
+    int rc;
+    if ((rc = make_tmap_bf16(&tmQ, Q, P.B, P.L, P.Hq, P.d, P.qs, 64))) return rc;
+    if ((rc = make_tmap_bf16(&tmG, dO, P.B, P.L, P.Hq, P.d, P.os, 64))) return rc;
+    if ((rc = make_tmap_bf16(&tmK, K, P.B, P.L, P.Hkv, P.d, P.ks, 128))) return rc;
+    if ((rc = make_tmap_bf16(&tmV, V, P.B, P.L, P.Hkv, P.d, P.vs, 128))) return rc;
+    rowdot_bf16_kernel<<<(unsigned)((rows + 7) / 8), 256, 0, st>>>((const __nv_bfloat16*)O, (const __nv_bfloat16*)dO, Dv, P.B, P.L, P.Hq,
+                                                                    P.os[0], P.os[1], P.os[2]);
+    if (cudaMemsetAsync(acc, 0, nq * sizeof(float), st) != cudaSuccess) return DMA_ERR_CUDA;
+    BwdParams bp;
+    bp.lse = lse; bp.Dv = Dv; bp.bias = bias; bp.expiry = expiry; bp.bitmap = bitmap; bp.dQacc = acc;
+    bp.dK = (__nv_bfloat16*)dK; bp.dV = (__nv_bfloat16*)dV; bp.dM = dM; bp.status = (int32_t*)ws;
+    bp.B = P.B; bp.Hq = P.Hq; bp.Hkv = P.Hkv; bp.G = P.G; bp.L = P.L; bp.Tr = P.Tr; bp.Tc = P.Tc; bp.Wd = P.Wd;
+    bp.ignore_bitmap = (P.flags & DMA_FLAG_IGNORE_BITMAP) ? 1 : 0;
+    bp.scale = P.scale; bp.scale_log2 = P.scale * 1.4426950408889634f;
+    bp.ks_b = P.ks[0]; bp.ks_l = P.ks[1]; bp.ks_h = P.ks[2]; bp.vs_b = P.vs[0]; bp.vs_l = P.vs[1]; bp.vs_h = P.vs[2];
+    const size_t smem = sizeof(SharedStorage) + 1024;
+    if (cudaFuncSetAttribute(bwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return DMA_ERR_CUDA;
+    bwd_kernel<<<dim3(P.B * P.Hkv, P.Tc), kThreads, smem, st>>>(tmQ, tmK, tmV, tmG, bp);
+    dq_convert_bf16_kernel<<<(unsigned)((nq / 8 + 255) / 256), 256, 0, st>>>(acc, (__nv_bfloat16*)dQ, nq / 8, P.L, P.Hq, P.qs[0], P.qs[1], P.qs[2]);
+    count_launch(3);
+    return check_launch();
 }
-}
+
+}  // namespace dma
