@@ -85,6 +85,23 @@ int dma_mask_build(const dma_problem_t* p, const void* V, const float* W_delta, 
                    float* bias, int32_t* expiry, uint32_t* bitmap,
                    void* ws, size_t ws_bytes, void* cuda_stream);
 
+/* Same computation and outputs as dma_mask_build, for callers that cannot supply a workspace. (The paper has no
+ * counterpart: this is a property of the library, not of the method.) Some hosts forbid device allocation
+ * at the point where the mask is built: an inference server that has handed all device memory to its own arena
+ * and treats any later cudaMalloc as an error, or a plug-in that runs inside another framework's step and has no
+ * allocator of its own to ask. This entry point allocates nothing and calls no allocating routine: its scratch is
+ * a fixed 8 MiB array inside the library's device image, present on every GPU that loads the library until the
+ * process exits.
+ *   Limit: B * Hq * roundup(L, 256) <= 1,048,576 sort keys; beyond that it returns DMA_ERR_WORKSPACE and launches
+ *   nothing (use dma_mask_build with a caller-provided workspace instead).
+ *   The first call on each device looks up the array's device address (that device must be current, as for
+ *   every call); make that first call before starting any stream capture.
+ *   All calls on a device share the one array. Nothing in it has to start at zero (each call rewrites what it
+ *   reads), but two calls whose kernels overlap on the GPU, from different streams or threads, race on it:
+ *   serialise them. */
+int dma_mask_build_static(const dma_problem_t* p, const void* V, const float* W_delta, const float* A,
+                          float* bias, int32_t* expiry, uint32_t* bitmap, void* cuda_stream);
+
 /* Forward (Sec. 4.2, Eq. (attention_output), Alg. 1): for each row i of head h
  *   s_j = q_i . k_j * scale + bias[j]   over keys with j <= i < expiry[j];   p = softmax(s);   O_i = sum p_j v_j
  *   lse_i = log sum_j exp(s_j)   (natural log; replaces Alg. 1's (l, m) pair)

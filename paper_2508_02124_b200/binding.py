@@ -17,7 +17,7 @@ DMA_BF16, DMA_FP32 = 0, 1
 DMA_FLAG_IGNORE_BITMAP, DMA_FLAG_SIMT = 1, 2
 
 ENTRY_POINTS = ("dma_query_workspace", "dma_bitmap_words", "dma_mask_build", "dma_attn_fwd", "dma_attn_bwd",
-                "dma_read_status", "dma_launch_count", "dma_strerror", "dma_step_host_arena", "dma_step_host")
+                "dma_read_status", "dma_launch_count", "dma_strerror", "dma_step_host_arena", "dma_step_host", "dma_mask_build_static")
 
 
 class DmaError(RuntimeError):
@@ -157,3 +157,11 @@ def dma_step_host(p, backward, hQ, hK, hV, hdO, hW, hA, hO, hlse, hdQ, hdK, hdV,
     _check(lib().dma_step_host(ctypes.byref(p), int(backward), _ptr(hQ), _ptr(hK), _ptr(hV), _ptr(hdO), _ptr(hW), _ptr(hA),
                                _ptr(hO), _ptr(hlse), _ptr(hdQ), _ptr(hdK), _ptr(hdV), _ptr(hdM), _ptr(arena),
                                ctypes.c_size_t(arena.numel()), _stream()), "dma_step_host")
+
+
+def dma_mask_build_static(p, V, W_delta, A, bias, expiry, bitmap):
+    """dma_mask_build without a workspace: the scratch is a fixed array inside the library (see include/dma.h for
+    the size limit and the sharing rules). Outputs must be preallocated by the caller; nothing is allocated here."""
+    _check(lib().dma_mask_build_static(ctypes.byref(p), _ptr(V), _ptr(W_delta), _ptr(A), _ptr(bias), _ptr(expiry),
+                                       _ptr(bitmap), _stream()), "dma_mask_build_static")
+    return bias, expiry, bitmap

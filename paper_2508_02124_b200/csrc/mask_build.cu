@@ -8,6 +8,8 @@
 //   expiry_kernel       per key: the index of the w-th key (in index order) that beats it, by counting beaters
 //                       chunk by chunk with a binary search in each sorted chunk
 //   bitmap_kernel       per key tile: union of the query-tile intervals its keys are kept in
+#include <mutex>
+
 #include "common.cuh"
 
 namespace dma {
@@ -254,3 +256,42 @@ int launch_mask_build(const Prob& P, const void* V, const float* W, const float*
 }
 
 }  // namespace dma
+
+// ---------------------------------------------------------------------------------------------------------------
+// dma_mask_build_static: mask generation for callers that cannot hand over a workspace.
+// The sorted-chunk scratch lives in this file-scope device array, which every GPU that loads the library keeps
+// until the process exits. In host code the array's name is only a stand-in; its device address is looked up
+// once per device with cudaGetSymbolAddress and that pointer is what the kernels receive.
+// ---------------------------------------------------------------------------------------------------------------
+namespace {
+constexpr size_t kStaticKeys = 1u << 20;   // 1 Mi sort keys = 8 MiB: B * Hq * roundup(L, 256) must not exceed this
+static __device__ __align__(256) unsigned long long g_static_scratch[dma::kWsHeaderBytes / 8 + kStaticKeys];
+constexpr int kMaxDevices = 64;
+void* g_static_ptr[kMaxDevices];            // per-device address of g_static_scratch (0 = not looked up yet)
+std::mutex g_static_mutex;
+}  // namespace
+
+extern "C" int dma_mask_build_static(const dma_problem_t* p, const void* V, const float* W_delta, const float* A,
+                                     float* bias, int32_t* expiry, uint32_t* bitmap, void* cuda_stream) {
+    dma::Prob P;
+    int rc = dma::resolve(p, &P);
+    if (rc) return rc;
+    if (!V || !W_delta || !A || !bias || !expiry || !bitmap) return DMA_ERR_NULL;
+    const uintptr_t bits = (uintptr_t)V | (uintptr_t)W_delta | (uintptr_t)bias | (uintptr_t)expiry | (uintptr_t)bitmap;
+    if (bits & 15) return DMA_ERR_ALIGN;
+    const size_t keys = (size_t)P.B * P.Hq * ((P.L + 255) / 256) * 256;
+    if (keys > kStaticKeys) return DMA_ERR_WORKSPACE;          // larger problems must use dma_mask_build
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return DMA_ERR_CUDA;
+    void* scratch;
+    {
+        std::lock_guard<std::mutex> lock(g_static_mutex);
+        if (!g_static_ptr[dev]) {       // first call on this device (which is current): resolve the symbol's address
+            void* ptr = nullptr;
+            if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || !ptr) return DMA_ERR_CUDA;
+            g_static_ptr[dev] = ptr;
+        }
+        scratch = g_static_ptr[dev];
+    }
+    return dma::launch_mask_build(P, V, W_delta, A, bias, expiry, bitmap, scratch, (cudaStream_t)cuda_stream);
+}
