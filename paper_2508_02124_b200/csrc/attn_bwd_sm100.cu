@@ -9,8 +9,9 @@
 //   dV  += P^T dO           dK  += dS^T Q                      (TMEM x smem  -> TMEM, 128 columns each)
 //   dQ^T = K^T dS^T                                            (smem x smem  -> TMEM, 64 columns), then added to the
 //                                                              fp32 dQ accumulator in global memory with red.add
-// Warp roles: warps 0-3 compute group (thread = key), warps 4-7 dQ drain group (thread = channel), warp 8 TMA
-// producer + schedule, warp 9 MMA issuer, warps 10-11 idle (register donors).
+// Warp roles (16 warps): warps 0-7 compute (thread = key; warps w and w+4 share the 32 TMEM lanes of quadrant w%4 and
+// split the 64 query columns of a step), warps 8-11 dQ drain (thread = channel), warp 12 TMA producer + schedule,
+// warps 13 and 14 MMA issuers (S^T, dP^T | dV, dK, dQ^T), warp 15 idle.
 // TMEM columns: dK [0,128) dV [128,256) S^T [256,320) dP^T [320,384) P^T [384,416) dS^T [416,448) dQ^T [448,512).
 #include "common.cuh"
 #include "sm100_ptx.cuh"
@@ -22,7 +23,7 @@ using namespace ptx;
 
 constexpr int kStages = 3;
 constexpr int kMaxSteps = 4096;
-constexpr int kThreads = 384;
+constexpr int kThreads = 512;
 constexpr uint32_t kKVBytes = 128 * 128 * 2;   // K or V tile: two 16 KB halves (channels 0-63 | 64-127)
 constexpr uint32_t kQBytes = 64 * 128 * 2;     // Q or dO step tile (64 rows): two 8 KB halves
 constexpr int cDK = 0, cDV = 128, cS = 256, cDP = 320, cP = 384, cDS = 416, cDQ = 448;
@@ -34,7 +35,7 @@ struct SharedStorage {
     alignas(1024) uint8_t g[kStages][kQBytes];       // dO
     alignas(1024) uint8_t ds[128 * 128];             // dS^T as bf16: [128 keys][64 queries], 128-byte swizzled rows
     alignas(16) float nlse[kStages][64];             // -log2(e) * lse_i
-    alignas(16) float dvec[kStages][64];             // D_i
+    alignas(16) float dvec[kStages][64];             // -D_i
     uint32_t sched[kMaxSteps];                       // head-in-group << 24 | query tile << 1 | half
     uint64_t kv_full, qd_full[kStages], qd_empty[kStages];
     uint64_t sdp_full, sdp_free, pds_ready, pds_free, dq_full, dq_free;
@@ -81,8 +82,8 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             mbar_init(&S.qd_empty[s], 1);
         }
         mbar_init(&S.sdp_full, 1);
-        mbar_init(&S.sdp_free, 128);
-        mbar_init(&S.pds_ready, 128);
+        mbar_init(&S.sdp_free, 256);
+        mbar_init(&S.pds_ready, 256);
         mbar_init(&S.pds_free, 1);
         mbar_init(&S.dq_full, 1);
         mbar_init(&S.dq_free, 128);
@@ -90,11 +91,11 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
         S.n_steps = 0;
         fence_barrier_init();
     }
-    if (warp == 9) {
+    if (warp == 13) {
         tmem_alloc(&S.tmem_base, 512);
         tmem_relinquish();
     }
-    if (warp == 8) {
+    if (warp == 12) {
         // schedule: for each query head of the group, the active query tiles (ascending), two 64-row steps each
         if (lane == 0) { prefetch_tmap(&tmQ); prefetch_tmap(&tmK); prefetch_tmap(&tmV); prefetch_tmap(&tmG); }
         int n = 0;
@@ -124,13 +125,14 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
     const uint32_t tmem = S.tmem_base;
     const int n_steps = S.n_steps;
 
-    if (warp < 4) {
-        // ============================ compute group: thread = key j, columns = query rows ============================
-        setmaxnreg_inc<216>();
-        const int r = tid;                                  // key within the tile = TMEM lane
+    if (warp < 8) {
+        // ============================ compute group: thread = key j, 32 of the step's 64 query columns ============================
+        const int quad = warp & 3, hsel = warp >> 2;
+        const int r = quad * 32 + lane;                     // key within the tile = TMEM lane
         const int j = j0 + r;
-        const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
-        float dm = 0.0f, bj = 0.0f;
+        const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
+        float bj = 0.0f;
+        float2 dm2 = make_float2(0.0f, 0.0f);
         int len = 0, cur_g = -1;
         bool ok = true;
         for (int n = 0; n < n_steps && ok; ++n) {
@@ -139,8 +141,8 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             const int st = n % kStages;
             if (g != cur_g) {
                 const int bh = b * P.Hq + hk * P.G + g;
-                if (cur_g >= 0 && j < P.L) P.dM[(size_t)(bh - (g - cur_g)) * P.L + j] = dm;
-                dm = 0.0f;
+                if (cur_g >= 0 && j < P.L) atomicAdd(&P.dM[(size_t)(bh - (g - cur_g)) * P.L + j], dm2.x + dm2.y);
+                dm2 = make_float2(0.0f, 0.0f);
                 bj = j < P.L ? P.bias[(size_t)bh * P.L + j] * 1.4426950408889634f : 0.0f;
                 len = j < P.L ? P.expiry[(size_t)bh * P.L + j] - j : 0;
                 cur_g = g;
@@ -148,65 +150,60 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             ok = mbar_wait_warp(&S.sdp_full, n & 1, abort_flag) && mbar_wait_warp(&S.qd_full[st], (n / kStages) & 1, abort_flag);
             if (!ok) break;
             tc_fence_after();
-            uint32_t sr[64], pr[64];
-#pragma unroll
-            for (int c = 0; c < 2; ++c) {
-                tmem_ld32(tmem + lane_base + cS + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&sr[c * 32]));
-                tmem_ld32(tmem + lane_base + cDP + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&pr[c * 32]));
-            }
+            uint32_t sr[32], pr[32];
+            tmem_ld32(tmem + lane_base + cS + hsel * 32, sr);
+            tmem_ld32(tmem + lane_base + cDP + hsel * 32, pr);
             tc_wait_ld();
             tc_fence_before();
             mbar_arrive(&S.sdp_free);
-            // valid columns of this thread: col in [lo, lo + width)
-            const int lo = max(0, j - i0);
-            const int width = max(0, min(64, j - i0 + len) - lo);
-            uint32_t pp[32], dd[32];
+            // valid columns of this thread within its 32: col in [lo, lo + width)
+            const int c0 = hsel * 32;
+            const int lo = max(0, j - i0 - c0);
+            const int width = max(0, min(32, j - i0 - c0 + len) - lo);
+            const bool plain = __all_sync(0xffffffffu, lo == 0);      // off the diagonal only the upper bound matters
+            uint32_t pp[16], dd[16];
+            const float2 bj2 = make_float2(bj, bj), sc2 = make_float2(P.scale_log2, P.scale_log2);
 #pragma unroll
-            for (int c = 0; c < 64; c += 4) {
-                const float4 nl = *reinterpret_cast<const float4*>(&S.nlse[st][c]);
-                const float4 dv = *reinterpret_cast<const float4*>(&S.dvec[st][c]);
-                const float nlv[4] = {nl.x, nl.y, nl.z, nl.w};
-                const float dvv[4] = {dv.x, dv.y, dv.z, dv.w};
-                float p[4], ds[4];
+            for (int c = 0; c < 32; c += 4) {
+                const float4 nl = *reinterpret_cast<const float4*>(&S.nlse[st][c0 + c]);
+                const float4 nd = *reinterpret_cast<const float4*>(&S.dvec[st][c0 + c]);   // holds -D_i
+                float2 x[2], t[2];
+                x[0] = fma2(make_float2(__uint_as_float(sr[c]), __uint_as_float(sr[c + 1])), sc2, add2(make_float2(nl.x, nl.y), bj2));
+                x[1] = fma2(make_float2(__uint_as_float(sr[c + 2]), __uint_as_float(sr[c + 3])), sc2, add2(make_float2(nl.z, nl.w), bj2));
+                t[0] = add2(make_float2(__uint_as_float(pr[c]), __uint_as_float(pr[c + 1])), make_float2(nd.x, nd.y));
+                t[1] = add2(make_float2(__uint_as_float(pr[c + 2]), __uint_as_float(pr[c + 3])), make_float2(nd.z, nd.w));
+                float p[4] = {ex2(x[0].x), ex2(x[0].y), ex2(x[1].x), ex2(x[1].y)};
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
-                    const float x = fmaf(__uint_as_float(sr[c + u]), P.scale_log2, bj + nlv[u]);
-                    const bool valid = (unsigned)(c + u - lo) < (unsigned)width;
-                    p[u] = valid ? ex2(x) : 0.0f;
-                    ds[u] = p[u] * (__uint_as_float(pr[c + u]) - dvv[u]);
-                    dm += ds[u];
+                    const bool valid = plain ? (c + u < width) : ((unsigned)(c + u - lo) < (unsigned)width);
+                    p[u] = valid ? p[u] : 0.0f;
                 }
+                const float2 d0 = mul2(make_float2(p[0], p[1]), t[0]), d1 = mul2(make_float2(p[2], p[3]), t[1]);
+                dm2 = add2(dm2, add2(d0, d1));
                 pp[(c >> 1)] = pack_bf16(p[0], p[1]);
                 pp[(c >> 1) + 1] = pack_bf16(p[2], p[3]);
-                dd[(c >> 1)] = pack_bf16(ds[0], ds[1]);
-                dd[(c >> 1) + 1] = pack_bf16(ds[2], ds[3]);
+                dd[(c >> 1)] = pack_bf16(d0.x, d0.y);
+                dd[(c >> 1) + 1] = pack_bf16(d1.x, d1.y);
             }
             // the previous step's dV / dK / dQ GEMMs must have finished reading P^T, dS^T (TMEM) and dS^T (smem)
             if (n > 0) ok = mbar_wait_warp(&S.pds_free, (n - 1) & 1, abort_flag);
             if (!ok) break;
             tc_fence_after();
-            tmem_st32(tmem + lane_base + cP, pp);
-            tmem_st32(tmem + lane_base + cDS, dd);
-            {   // dS^T row r -> shared memory, eight 16-byte chunks, chunk index XOR (row % 8) (128-byte swizzle)
+            tmem_st16(tmem + lane_base + cP + hsel * 16, pp);
+            tmem_st16(tmem + lane_base + cDS + hsel * 16, dd);
+            {   // dS^T row r -> shared memory: 16-byte chunk q of the row sits at q XOR (row % 8) (128-byte swizzle)
                 uint8_t* row = S.ds + r * 128;
 #pragma unroll
-                for (int c = 0; c < 8; ++c)
-                    *reinterpret_cast<uint4*>(row + ((c ^ (r & 7)) << 4)) = make_uint4(dd[4 * c], dd[4 * c + 1], dd[4 * c + 2], dd[4 * c + 3]);
+                for (int q = 0; q < 4; ++q)
+                    *reinterpret_cast<uint4*>(row + (((hsel * 4 + q) ^ (r & 7)) << 4)) = make_uint4(dd[4 * q], dd[4 * q + 1], dd[4 * q + 2], dd[4 * q + 3]);
             }
             fence_proxy_async();
             tc_wait_st();
             tc_fence_before();
             mbar_arrive(&S.pds_ready);
         }
-        if (cur_g >= 0 && j < P.L) P.dM[(size_t)(b * P.Hq + hk * P.G + cur_g) * P.L + j] = dm;
-        // heads of the group that had no active tile for this key tile: dM = 0
-        if (ok && j < P.L) {
-            uint32_t seen = 0;
-            for (int n = 0; n < n_steps; ++n) seen |= 1u << (S.sched[n] >> 24);
-            for (int g = 0; g < P.G; ++g)
-                if (!((seen >> g) & 1u)) P.dM[(size_t)(b * P.Hq + hk * P.G + g) * P.L + j] = 0.0f;
-        }
-        // epilogue: dK (scaled) and dV rows to global memory
+        if (cur_g >= 0 && j < P.L) atomicAdd(&P.dM[(size_t)(b * P.Hq + hk * P.G + cur_g) * P.L + j], dm2.x + dm2.y);
+        // epilogue: dK (scaled) and dV rows to global memory; warps w and w+4 each write one half of the channels
         if (ok && n_steps > 0) ok = mbar_wait_warp(&S.pds_free, (n_steps - 1) & 1, abort_flag);
         if (ok) {
             tc_fence_after();
@@ -217,7 +214,8 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                 const float mul = which == 0 ? P.scale : 1.0f;
                 __nv_bfloat16* out = which == 0 ? dk : dv;
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
+                for (int cc = 0; cc < 2; ++cc) {
+                    const int c = hsel * 2 + cc;
                     uint32_t o[32];
                     if (n_steps > 0) {
                         tmem_ld32(tmem + lane_base + (which == 0 ? cDK : cDV) + c * 32, o);
@@ -240,10 +238,9 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                 }
             }
         }
-    } else if (warp < 8) {
+    } else if (warp < 12) {
         // ============================ dQ drain group: thread = channel c, columns = query rows ============================
-        setmaxnreg_inc<216>();
-        const int c = tid - 128;
+        const int c = tid - 256;
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
         bool ok = true;
         for (int n = 0; n < n_steps && ok; ++n) {
@@ -265,8 +262,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                 if (u < rows) red_add_f32(base + (size_t)u * P.Hq * 128, __uint_as_float(v[u]) * P.scale);
         }
     } else {
-        setmaxnreg_dec<72>();      // 4 warps x 96 registers released = 8 warps x 48 acquired above
-        if (warp == 8) {
+        if (warp == 12) {
             // ============================ producer ============================
             if (lane == 0) {
                 mbar_arrive_expect_tx(&S.kv_full, 2 * kKVBytes);
@@ -287,7 +283,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                 for (int c = lane; c < 64; c += 32) {
                     const int i = i0 + c;
                     S.nlse[st][c] = i < P.L ? -1.4426950408889634f * P.lse[rowbase + i] : 0.0f;
-                    S.dvec[st][c] = i < P.L ? P.Dv[rowbase + i] : 0.0f;
+                    S.dvec[st][c] = i < P.L ? -P.Dv[rowbase + i] : 0.0f;
                 }
                 __syncwarp();
                 if (lane == 0) {
@@ -300,62 +296,52 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             }
             for (int n = max(0, n_steps - kStages); n < n_steps && ok; ++n)
                 ok = mbar_wait_warp(&S.qd_empty[n % kStages], (n / kStages) & 1, abort_flag);
-        } else if (warp == 9 && lane == 0) {
-            // ============================ MMA issuer ============================
+        } else if (warp == 13 && lane == 0) {
+            // ============================ MMA issuer 1: S^T = K Q^T, dP^T = V dO^T ============================
+            // (two issuing threads: every hand-over between them and the other groups is an explicit mbarrier,
+            //  nothing relies on the order of the two threads' MMAs)
             constexpr uint32_t id_sdp = idesc_bf16(128, 64, 0, 0);     // K|V (K-major) x Q|dO (K-major)       -> 128 x 64
-            constexpr uint32_t id_dkv = idesc_bf16(128, 128, 0, 1);    // P^T|dS^T (TMEM) x dO|Q (MN-major)    -> 128 x 128
-            constexpr uint32_t id_dq = idesc_bf16(128, 64, 1, 1);      // K^T (MN-major) x dS^T (MN-major)     -> 128 x 64
-            auto issue_sdp = [&](int st) {
-#pragma unroll
-                for (int kk = 0; kk < 8; ++kk) {
-                    const uint32_t offa = (kk >> 2) * (kKVBytes / 2) + (kk & 3) * 32, offb = (kk >> 2) * (kQBytes / 2) + (kk & 3) * 32;
-                    mma_ss(tmem + cS, smem_desc_sw128(smem_u32(&S.k[offa]), 16, 1024),
-                           smem_desc_sw128(smem_u32(&S.q[st][offb]), 16, 1024), id_sdp, kk > 0);
-                }
-#pragma unroll
-                for (int kk = 0; kk < 8; ++kk) {
-                    const uint32_t offa = (kk >> 2) * (kKVBytes / 2) + (kk & 3) * 32, offb = (kk >> 2) * (kQBytes / 2) + (kk & 3) * 32;
-                    mma_ss(tmem + cDP, smem_desc_sw128(smem_u32(&S.v[offa]), 16, 1024),
-                           smem_desc_sw128(smem_u32(&S.g[st][offb]), 16, 1024), id_sdp, kk > 0);
-                }
-                tc_commit(&S.sdp_full);
-            };
+            const uint64_t dK = smem_desc_sw128(smem_u32(S.k), 16, 1024), dV = smem_desc_sw128(smem_u32(S.v), 16, 1024);
             bool ok = mbar_wait(&S.kv_full, 0, abort_flag);
-            if (ok && n_steps > 0) {
-                ok = mbar_wait(&S.qd_full[0], 0, abort_flag);
-                if (ok) {
-                    tc_fence_after();
-                    issue_sdp(0);
-                }
-            }
             for (int n = 0; n < n_steps && ok; ++n) {
                 const int st = n % kStages;
-                if (n + 1 < n_steps) {
-                    const int nst = (n + 1) % kStages;
-                    ok = mbar_wait(&S.qd_full[nst], ((n + 1) / kStages) & 1, abort_flag) && mbar_wait(&S.sdp_free, n & 1, abort_flag);
-                    if (!ok) break;
-                    tc_fence_after();
-                    issue_sdp(nst);
-                }
+                ok = mbar_wait(&S.qd_full[st], (n / kStages) & 1, abort_flag);
+                if (ok && n > 0) ok = mbar_wait(&S.sdp_free, (n - 1) & 1, abort_flag);
+                if (!ok) break;
+                tc_fence_after();
+                const uint64_t dQ = smem_desc_sw128(smem_u32(S.q[st]), 16, 1024), dG = smem_desc_sw128(smem_u32(S.g[st]), 16, 1024);
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk)
+                    mma_ss(tmem + cS, dK + (uint64_t)(((kk >> 2) * (kKVBytes / 2) + (kk & 3) * 32) >> 4),
+                           dQ + (uint64_t)(((kk >> 2) * (kQBytes / 2) + (kk & 3) * 32) >> 4), id_sdp, kk > 0);
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk)
+                    mma_ss(tmem + cDP, dV + (uint64_t)(((kk >> 2) * (kKVBytes / 2) + (kk & 3) * 32) >> 4),
+                           dG + (uint64_t)(((kk >> 2) * (kQBytes / 2) + (kk & 3) * 32) >> 4), id_sdp, kk > 0);
+                tc_commit(&S.sdp_full);
+            }
+        } else if (warp == 14 && lane == 0) {
+            // ============================ MMA issuer 2: dV += P^T dO, dK += dS^T Q, dQ^T = K^T dS^T ============================
+            constexpr uint32_t id_dkv = idesc_bf16(128, 128, 0, 1);    // P^T|dS^T (TMEM) x dO|Q (MN-major)    -> 128 x 128
+            constexpr uint32_t id_dq = idesc_bf16(128, 64, 1, 1);      // K^T (MN-major) x dS^T (MN-major)     -> 128 x 64
+            const uint64_t dKt = smem_desc_sw128(smem_u32(S.k), kKVBytes / 2, 1024), dDs = smem_desc_sw128(smem_u32(S.ds), 16, 1024);
+            bool ok = true;
+            for (int n = 0; n < n_steps && ok; ++n) {
+                const int st = n % kStages;
                 ok = mbar_wait(&S.pds_ready, n & 1, abort_flag);
                 if (ok && n > 0) ok = mbar_wait(&S.dq_free, (n - 1) & 1, abort_flag);
                 if (!ok) break;
                 tc_fence_after();
+                const uint64_t dGm = smem_desc_sw128(smem_u32(S.g[st]), kQBytes / 2, 1024), dQm = smem_desc_sw128(smem_u32(S.q[st]), kQBytes / 2, 1024);
 #pragma unroll
-                for (int kk = 0; kk < 4; ++kk) {       // 64 query rows = 4 k-steps of 16
-                    mma_ts(tmem + cDV, tmem + cP + kk * 8, smem_desc_sw128(smem_u32(&S.g[st][kk * 2048]), kQBytes / 2, 1024),
-                           id_dkv, (n > 0 || kk > 0) ? 1u : 0u);
-                }
+                for (int kk = 0; kk < 4; ++kk)         // 64 query rows = 4 k-steps of 16
+                    mma_ts(tmem + cDV, tmem + cP + kk * 8, dGm + (uint64_t)((kk * 2048) >> 4), id_dkv, (n > 0 || kk > 0) ? 1u : 0u);
 #pragma unroll
-                for (int kk = 0; kk < 4; ++kk) {
-                    mma_ts(tmem + cDK, tmem + cDS + kk * 8, smem_desc_sw128(smem_u32(&S.q[st][kk * 2048]), kQBytes / 2, 1024),
-                           id_dkv, (n > 0 || kk > 0) ? 1u : 0u);
-                }
+                for (int kk = 0; kk < 4; ++kk)
+                    mma_ts(tmem + cDK, tmem + cDS + kk * 8, dQm + (uint64_t)((kk * 2048) >> 4), id_dkv, (n > 0 || kk > 0) ? 1u : 0u);
 #pragma unroll
-                for (int kk = 0; kk < 8; ++kk) {       // 128 keys = 8 k-steps of 16
-                    mma_ss(tmem + cDQ, smem_desc_sw128(smem_u32(&S.k[kk * 2048]), kKVBytes / 2, 1024),
-                           smem_desc_sw128(smem_u32(&S.ds[kk * 2048]), 16, 1024), id_dq, kk > 0);
-                }
+                for (int kk = 0; kk < 8; ++kk)         // 128 keys = 8 k-steps of 16
+                    mma_ss(tmem + cDQ, dKt + (uint64_t)((kk * 2048) >> 4), dDs + (uint64_t)((kk * 2048) >> 4), id_dq, kk > 0);
                 tc_commit(&S.pds_free);
                 tc_commit(&S.dq_full);
                 tc_commit(&S.qd_empty[st]);
@@ -364,7 +350,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 9) {
+    if (warp == 13) {
         tc_fence_after();
         tmem_dealloc(tmem, 512);
     }
@@ -429,6 +415,7 @@ int launch_tc_bwd(const Prob& P, const void* Q, const void* K, const void* V, co
     rowdot_bf16_kernel<<<(unsigned)((rows + 7) / 8), 256, 0, st>>>((const __nv_bfloat16*)O, (const __nv_bfloat16*)dO, Dv, P.B, P.L, P.Hq,
                                                                     P.os[0], P.os[1], P.os[2]);
     if (cudaMemsetAsync(acc, 0, nq * sizeof(float), st) != cudaSuccess) return DMA_ERR_CUDA;
+    if (cudaMemsetAsync(dM, 0, rows * sizeof(float), st) != cudaSuccess) return DMA_ERR_CUDA;   // two partial sums are added per key
     BwdParams bp;
     bp.lse = lse; bp.Dv = Dv; bp.bias = bias; bp.expiry = expiry; bp.bitmap = bitmap; bp.dQacc = acc;
     bp.dK = (__nv_bfloat16*)dK; bp.dV = (__nv_bfloat16*)dV; bp.dM = dM; bp.status = (int32_t*)ws;

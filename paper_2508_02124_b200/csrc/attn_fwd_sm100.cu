@@ -6,12 +6,14 @@
 //   warps 0-3 / 4-7  softmax group 0 / 1: thread r owns query row r of its tile (TMEM lane r): reads S, adds the
 //                    bias, applies the validity test j <= i < expiry[j], keeps the running max / sum, writes P (bf16)
 //                    back to tensor memory over S, rescales O when the max has grown, and finally normalises O
-//   warp 8           producer: builds the tile schedule from the bitmap, then per key tile stages bias / validity
-//                    lengths in shared memory and issues the TMA loads of K and V (inactive tiles are never loaded)
+//   warp 8           producer: builds the tile schedule from the bitmap, then issues the TMA loads of K and V per
+//                    active key tile (inactive tiles are never loaded); warp 10 stages bias / expiry vectors
 //   warp 9           MMA issuer: S_w = Q_w K^T, O_w += P_w V, ping-ponging between the two query tiles so that the
 //                    tensor cores run one tile's GEMMs while the other tile's softmax is in flight
 // Tensor memory (512 columns): S0 [0,128) S1 [128,256) O0 [256,384) O1 [384,512); P_w aliases columns [0,64) of S_w.
 // The log-sum-exp replaces Alg. 1's (l, m) pair. Scores are kept in the log2 domain: x = log2(e) (s scale + bias).
+#include <type_traits>
+
 #include "common.cuh"
 #include "sm100_ptx.cuh"
 
@@ -31,9 +33,9 @@ struct SharedStorage {
     alignas(1024) uint8_t k[kStages][kTileBytes];
     alignas(1024) uint8_t v[kStages][kTileBytes];
     alignas(16) float bias[kStages][128];     // log2(e) * bias of the staged key tile
-    alignas(16) int len[kStages][128];        // expiry[j] - j (0 beyond L): row i keeps key j iff 0 <= i - j < len
+    alignas(16) int len[kStages][128];        // expiry[j] (0 beyond L): row i keeps key j iff j <= i < expiry[j]
     uint32_t sched[kMaxSched];                // key tile | use by tile 0 << 30 | use by tile 1 << 31
-    uint64_t q_full, k_full[kStages], v_full[kStages], kv_empty[kStages];
+    uint64_t q_full, k_full[kStages], v_full[kStages], k_empty[kStages], v_empty[kStages];
     uint64_t s_full[2], p_ready[2], o_done[2];
     uint32_t tmem_base;
     int n_iters;
@@ -70,9 +72,10 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
     if (tid == 0) {
         mbar_init(&S.q_full, 1);
         for (int s = 0; s < kStages; ++s) {
-            mbar_init(&S.k_full[s], 1);
+            mbar_init(&S.k_full[s], 2);      // TMA bytes of K + the staged bias / expiry vectors
             mbar_init(&S.v_full[s], 1);
-            mbar_init(&S.kv_empty[s], 1);
+            mbar_init(&S.k_empty[s], 1);
+            mbar_init(&S.v_empty[s], 1);
         }
         for (int w = 0; w < 2; ++w) {
             mbar_init(&S.s_full[w], 1);
@@ -140,21 +143,29 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
 #pragma unroll
                 for (int u = 0; u < 32; ++u) x[c * 32 + u] = __uint_as_float(raw[u]);
             }
-            const int rel = i - j0;
-            float mx = -INFINITY;
+            // x = log2e (s scale + bias) where row i keeps key j (j <= i < expiry[j]), else -inf. Off the diagonal
+            // j <= i always holds and one compare against the staged expiry decides; the two cases are separate
+            // loops so that neither pays for the other's test. Four independent max chains.
+            float mxa[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+            auto score_pass = [&](auto diag) {
+                constexpr bool kDiag = decltype(diag)::value;
 #pragma unroll
-            for (int c = 0; c < 128; c += 4) {
-                const float4 bb = *reinterpret_cast<const float4*>(&S.bias[st][c]);
-                const int4 ll = *reinterpret_cast<const int4*>(&S.len[st][c]);
-                const float bv[4] = {bb.x, bb.y, bb.z, bb.w};
-                const int lv[4] = {ll.x, ll.y, ll.z, ll.w};
+                for (int c = 0; c < 128; c += 4) {
+                    const float4 bb = *reinterpret_cast<const float4*>(&S.bias[st][c]);
+                    const int4 ee = *reinterpret_cast<const int4*>(&S.len[st][c]);
+                    const float bv[4] = {bb.x, bb.y, bb.z, bb.w};
+                    const int ev[4] = {ee.x, ee.y, ee.z, ee.w};
 #pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const float xv = fmaf(x[c + u], P.scale_log2, bv[u]);
-                    x[c + u] = ((unsigned)(rel - (c + u)) < (unsigned)lv[u]) ? xv : -INFINITY;
-                    mx = fmaxf(mx, x[c + u]);
+                    for (int u = 0; u < 4; ++u) {
+                        const float xv = fmaf(x[c + u], P.scale_log2, bv[u]);
+                        const bool valid = kDiag ? (j0 + c + u <= i && i < ev[u]) : (i < ev[u]);
+                        x[c + u] = valid ? xv : -INFINITY;
+                        mxa[u] = fmaxf(mxa[u], x[c + u]);
+                    }
                 }
-            }
+            };
+            if (j0 + 127 > qt * 128) score_pass(std::true_type{}); else score_pass(std::false_type{});
+            const float mx = fmaxf(fmaxf(mxa[0], mxa[1]), fmaxf(mxa[2], mxa[3]));
             const float m_new = fmaxf(m_ref, mx);
             if (n_used == 0) {
                 m_ref = m_new;
@@ -178,19 +189,19 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                 m_ref = m_new;
             }
             const float m_use = (m_ref == -INFINITY) ? 0.0f : m_ref;
-            float sum = 0.0f;
+            float sa[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
             for (int half = 0; half < 2; ++half) {
                 uint32_t pk[32];
 #pragma unroll
                 for (int c = 0; c < 64; c += 2) {
                     const float p0 = ex2(x[half * 64 + c] - m_use), p1 = ex2(x[half * 64 + c + 1] - m_use);
-                    sum += p0 + p1;
+                    sa[(c >> 1) & 3] += p0 + p1;
                     pk[c >> 1] = pack_bf16(p0, p1);
                 }
                 tmem_st32(tS + half * 32, pk);
             }
-            l += sum;
+            l += (sa[0] + sa[1]) + (sa[2] + sa[3]);
             tc_wait_st();
             tc_fence_before();
             mbar_arrive(&S.p_ready[w]);
@@ -237,22 +248,21 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                     for (int hf = 0; hf < 2; ++hf)
                         tma_load_4d(&S.q[w][hf * (kTileBytes / 2)], &tmQ, &S.q_full, hf * 64, (qt0 + w) * 128, h, b);
             }
+            // K and V of a stage are released separately (K once its S = Q K^T products are done, V after P V), so
+            // the next K tile is in flight about two key tiles ahead of its use
             bool ok = true;
             for (int it = 0; it < n_iters && ok; ++it) {
-                const int st = it % kStages, kt = (int)(S.sched[it] & 0xFFFFF), j0 = kt * 128;
-                if (it >= kStages) ok = mbar_wait_warp(&S.kv_empty[st], ((it / kStages) - 1) & 1, abort_flag);
+                const int st = it % kStages, j0 = (int)(S.sched[it] & 0xFFFFF) * 128;
+                if (it >= kStages) ok = mbar_wait_warp(&S.k_empty[st], ((it / kStages) - 1) & 1, abort_flag);
                 if (!ok) break;
-#pragma unroll
-                for (int c = lane; c < 128; c += 32) {
-                    const int j = j0 + c;
-                    S.bias[st][c] = j < P.L ? P.bias[(size_t)bh * P.L + j] * 1.4426950408889634f : 0.0f;
-                    S.len[st][c] = j < P.L ? P.expiry[(size_t)bh * P.L + j] - j : 0;
-                }
-                __syncwarp();
                 if (lane == 0) {
                     mbar_arrive_expect_tx(&S.k_full[st], kTileBytes);
                     tma_load_4d(&S.k[st][0], &tmK, &S.k_full[st], 0, j0, hk, b);
                     tma_load_4d(&S.k[st][kTileBytes / 2], &tmK, &S.k_full[st], 64, j0, hk, b);
+                }
+                if (it >= kStages) ok = mbar_wait_warp(&S.v_empty[st], ((it / kStages) - 1) & 1, abort_flag);
+                if (!ok) break;
+                if (lane == 0) {
                     mbar_arrive_expect_tx(&S.v_full[st], kTileBytes);
                     tma_load_4d(&S.v[st][0], &tmV, &S.v_full[st], 0, j0, hk, b);
                     tma_load_4d(&S.v[st][kTileBytes / 2], &tmV, &S.v_full[st], 64, j0, hk, b);
@@ -260,7 +270,42 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             }
             // tail: the last stages' release arrivals must land before the CTA's shared memory is given up
             for (int it = max(0, n_iters - kStages); it < n_iters && ok; ++it)
-                ok = mbar_wait_warp(&S.kv_empty[it % kStages], (it / kStages) & 1, abort_flag);
+                ok = mbar_wait_warp(&S.k_empty[it % kStages], (it / kStages) & 1, abort_flag) &&
+                     mbar_wait_warp(&S.v_empty[it % kStages], (it / kStages) & 1, abort_flag);
+        } else if (warp == 10) {
+            // =========================================== stager ===========================================
+            // bias (log2 domain) and expiry of each key tile -> shared memory; the global loads run one tile ahead
+            auto fetch = [&](int it, float (&bv)[4], int (&ev)[4]) {
+                const int j0 = (int)(S.sched[it] & 0xFFFFF) * 128;
+#pragma unroll
+                for (int t = 0; t < 4; ++t) {
+                    const int j = j0 + lane + 32 * t;
+                    bv[t] = j < P.L ? P.bias[(size_t)bh * P.L + j] : 0.0f;
+                    ev[t] = j < P.L ? P.expiry[(size_t)bh * P.L + j] : 0;
+                }
+            };
+            float bv[4] = {0.f, 0.f, 0.f, 0.f};
+            int ev[4] = {0, 0, 0, 0};
+            if (n_iters > 0) fetch(0, bv, ev);
+            bool ok = true;
+            for (int it = 0; it < n_iters && ok; ++it) {
+                const int st = it % kStages;
+                float bn[4] = {0.f, 0.f, 0.f, 0.f};
+                int en[4] = {0, 0, 0, 0};
+                if (it + 1 < n_iters) fetch(it + 1, bn, en);
+                // the vectors of this stage were last read by the softmax groups before they released P (hence before P V)
+                if (it >= kStages) ok = mbar_wait_warp(&S.v_empty[st], ((it / kStages) - 1) & 1, abort_flag);
+                if (!ok) break;
+#pragma unroll
+                for (int t = 0; t < 4; ++t) {
+                    S.bias[st][lane + 32 * t] = bv[t] * 1.4426950408889634f;
+                    S.len[st][lane + 32 * t] = ev[t];
+                    bv[t] = bn[t];
+                    ev[t] = en[t];
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&S.k_full[st]);
+            }
         } else if (warp == 9 && lane == 0) {
             // =========================================== MMA issuer ===========================================
             constexpr uint32_t idesc_s = idesc_bf16(128, 128, 0, 0);     // Q (K-major) x K (K-major)
@@ -282,14 +327,14 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                     tc_fence_after();
                     for (int w = 0; w < 2; ++w)
                         if (use_bit(S.sched[0], w)) issue_s(w, 0);
+                    tc_commit(&S.k_empty[0]);
                 }
             }
             for (int it = 0; it < n_iters && ok; ++it) {
                 const int st = it % kStages, nst = (it + 1) % kStages;
                 const uint32_t entry = S.sched[it], next = it + 1 < n_iters ? S.sched[it + 1] : 0u;
                 ok = mbar_wait(&S.v_full[st], (it / kStages) & 1, abort_flag);
-                if (ok && it + 1 < n_iters) ok = mbar_wait(&S.k_full[nst], ((it + 1) / kStages) & 1, abort_flag);
-                tc_fence_after();
+                bool k_ready = false;
                 for (int w = 0; w < 2 && ok; ++w) {
                     if (use_bit(entry, w)) {
                         ok = mbar_wait(&S.p_ready[w], n_p[w] & 1, abort_flag);
@@ -303,9 +348,20 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                         tc_commit(&S.o_done[w]);
                         ++n_p[w];
                     }
-                    if (use_bit(next, w)) issue_s(w, nst);
+                    if (use_bit(next, w)) {
+                        if (!k_ready) {
+                            ok = mbar_wait(&S.k_full[nst], ((it + 1) / kStages) & 1, abort_flag);
+                            if (!ok) break;
+                            tc_fence_after();
+                            k_ready = true;
+                        }
+                        issue_s(w, nst);
+                    }
                 }
-                if (ok) tc_commit(&S.kv_empty[st]);
+                if (ok) {
+                    tc_commit(&S.v_empty[st]);
+                    if (it + 1 < n_iters) tc_commit(&S.k_empty[nst]);
+                }
             }
         }
     }

@@ -142,10 +142,13 @@ __global__ void __launch_bounds__(kChunk) chunk_sort_kernel(const float* __restr
 }
 
 // expiry[j] = max(j, index of the w-th key in index order that beats j), or L if fewer than w keys beat it.
+// The CTA walks the chunks together: each chunk's sorted keys (for the count) and keys in index order (for the
+// final walk) are staged in shared memory once for all 256 threads.
 __global__ void __launch_bounds__(kChunk) expiry_kernel(const float* __restrict__ delta,
                                                         const unsigned long long* __restrict__ sorted,
                                                         int32_t* __restrict__ expiry, int L, int w, int nchunk) {
-    __shared__ unsigned long long s[kChunk];
+    __shared__ unsigned long long s[kChunk];      // chunk c, ascending
+    __shared__ unsigned long long u[kChunk];      // chunk c, index order
     const int bh = blockIdx.y, t = threadIdx.x, j = blockIdx.x * kChunk + t;
     const float* dl = delta + (size_t)bh * L;
     const bool valid = j < L;
@@ -153,7 +156,9 @@ __global__ void __launch_bounds__(kChunk) expiry_kernel(const float* __restrict_
     int cnt = 0, e = L;
     bool done = !valid;
     for (int c = 0; c < nchunk; ++c) {
+        const int k = c * kChunk + t;
         s[t] = sorted[((size_t)bh * nchunk + c) * kChunk + t];
+        u[t] = k < L ? sort_key(dl[k], k) : 0ull;
         __syncthreads();
         if (!done) {
             int lo = 0, hi = kChunk;              // first position whose key is greater than ours
@@ -163,9 +168,11 @@ __global__ void __launch_bounds__(kChunk) expiry_kernel(const float* __restrict_
             }
             const int n = kChunk - lo;
             if (cnt + n >= w) {
-                int need = w - cnt;
-                for (int k = c * kChunk;; ++k)    // the need-th beater lies in this chunk: walk it in index order
-                    if (sort_key(dl[k], k) > key && --need == 0) { e = max(j, k); break; }
+                int need = w - cnt;               // the need-th beater lies in this chunk: walk it in index order
+                int q = 0;
+                for (; q < kChunk; ++q)
+                    if (u[q] > key && --need == 0) break;
+                e = max(j, c * kChunk + q);
                 done = true;
             }
             cnt += n;
