@@ -7,11 +7,11 @@
 //   S^T  = K Q^T            dP^T = V dO^T                      (smem x smem  -> TMEM, 64 columns each)
 //   P^T  = exp2(S^T c + log2e (bias_j - lse_i)) where j <= i < expiry[j], else 0;   dS^T = P^T o (dP^T - D_i)
 //   dV  += P^T dO           dK  += dS^T Q                      (TMEM x smem  -> TMEM, 128 columns each)
-//   dQ^T = K^T dS^T                                            (smem x smem  -> TMEM, 64 columns), then added to the
-//                                                              fp32 dQ accumulator in global memory with red.add
+//   dQ^T = K^T dS^T                                            (smem x smem  -> TMEM, 64 columns), staged in shared memory
+//                                                              and added to the fp32 dQ accumulator by a TMA reduce-add
 // Warp roles (16 warps): warps 0-7 compute (thread = key; warps w and w+4 share the 32 TMEM lanes of quadrant w%4 and
 // split the 64 query columns of a step), warps 8-11 dQ drain (thread = channel), warp 12 TMA producer + schedule,
-// warps 13 and 14 MMA issuers (S^T, dP^T | dV, dK, dQ^T), warp 15 idle.
+// warps 13 and 14 MMA issuers (S^T, dP^T | dV, dK, dQ^T), warp 15 stages -lse and -D of each step's query rows.
 // TMEM columns: dK [0,128) dV [128,256) S^T [256,320) dP^T [320,384) P^T [384,416) dS^T [416,448) dQ^T [448,512).
 #include "common.cuh"
 #include "sm100_ptx.cuh"
@@ -34,11 +34,12 @@ struct SharedStorage {
     alignas(1024) uint8_t q[kStages][kQBytes];
     alignas(1024) uint8_t g[kStages][kQBytes];       // dO
     alignas(1024) uint8_t ds[128 * 128];             // dS^T as bf16: [128 keys][64 queries], 128-byte swizzled rows
+    alignas(1024) float dq_stage[64][128];           // dQ of one step, [query row][channel], source of the TMA reduce-add
     alignas(16) float nlse[kStages][64];             // -log2(e) * lse_i
     alignas(16) float dvec[kStages][64];             // -D_i
-    uint32_t sched[kMaxSteps];                       // head-in-group << 24 | query tile << 1 | half
+    uint16_t sched[kMaxSteps];                       // head-in-group << 11 | query tile << 1 | half
     uint64_t kv_full, qd_full[kStages], qd_empty[kStages];
-    uint64_t sdp_full, sdp_free, pds_ready, pds_free, dq_full, dq_free;
+    uint64_t sdp_full, sdp_free, pds_ready, pds_free, dq_full, dq_free, drain_bar;
     uint32_t tmem_base;
     int n_steps;
     int abort_flag;
@@ -60,13 +61,10 @@ struct BwdParams {
     int64_t ks_b, ks_l, ks_h, vs_b, vs_l, vs_h;
 };
 
-__device__ __forceinline__ void red_add_f32(float* addr, float v) {
-    asm volatile("red.global.add.f32 [%0], %1;" ::"l"(addr), "f"(v) : "memory");
-}
-
 __global__ void __launch_bounds__(kThreads, 1)
 bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
-           const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmG, const BwdParams P) {
+           const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmG,
+           const __grid_constant__ CUtensorMap tmDQ, const BwdParams P) {
     extern __shared__ uint8_t smem_raw[];
     SharedStorage& S = *reinterpret_cast<SharedStorage*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -78,7 +76,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
     if (tid == 0) {
         mbar_init(&S.kv_full, 1);
         for (int s = 0; s < kStages; ++s) {
-            mbar_init(&S.qd_full[s], 1);
+            mbar_init(&S.qd_full[s], 2);      // TMA bytes + the staged vectors
             mbar_init(&S.qd_empty[s], 1);
         }
         mbar_init(&S.sdp_full, 1);
@@ -87,6 +85,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
         mbar_init(&S.pds_free, 1);
         mbar_init(&S.dq_full, 1);
         mbar_init(&S.dq_free, 128);
+        mbar_init(&S.drain_bar, 128);
         S.abort_flag = 0;
         S.n_steps = 0;
         fence_barrier_init();
@@ -113,7 +112,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                 }
                 const int pos = n + incl - halves;
                 for (int hf = 0; hf < halves; ++hf)
-                    if (pos + hf < kMaxSteps) S.sched[pos + hf] = ((uint32_t)g << 24) | ((uint32_t)qt << 1) | (uint32_t)hf;
+                    if (pos + hf < kMaxSteps) S.sched[pos + hf] = (uint16_t)((g << 11) | (qt << 1) | hf);
                 n += __shfl_sync(0xffffffffu, incl, 31);
             }
         }
@@ -137,7 +136,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
         bool ok = true;
         for (int n = 0; n < n_steps && ok; ++n) {
             const uint32_t e = S.sched[n];
-            const int g = (int)(e >> 24), i0 = (int)((e >> 1) & 0x7FFFFF) * 128 + (int)(e & 1) * 64;
+            const int g = (int)(e >> 11), i0 = (int)((e >> 1) & 0x3FF) * 128 + (int)(e & 1) * 64;
             const int st = n % kStages;
             if (g != cur_g) {
                 const int bh = b * P.Hq + hk * P.G + g;
@@ -245,7 +244,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
         bool ok = true;
         for (int n = 0; n < n_steps && ok; ++n) {
             const uint32_t e = S.sched[n];
-            const int g = (int)(e >> 24), i0 = (int)((e >> 1) & 0x7FFFFF) * 128 + (int)(e & 1) * 64;
+            const int g = (int)(e >> 11), i0 = (int)((e >> 1) & 0x3FF) * 128 + (int)(e & 1) * 64;
             ok = mbar_wait_warp(&S.dq_full, n & 1, abort_flag);
             if (!ok) break;
             tc_fence_after();
@@ -255,12 +254,23 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             tc_wait_ld();
             tc_fence_before();
             mbar_arrive(&S.dq_free);
-            float* base = P.dQacc + (((size_t)b * P.L + i0) * P.Hq + hk * P.G + g) * 128 + c;
-            const int rows = min(64, P.L - i0);
+            // hand the step's dQ (scaled) to the TMA: staging buffer free -> write [row][channel] -> one reduce-add
+            if (tid == 256) bulk_wait_read_all();
+            mbar_arrive(&S.drain_bar);
+            ok = mbar_wait_warp(&S.drain_bar, (2 * n) & 1, abort_flag);
+            if (!ok) break;
 #pragma unroll
-            for (int u = 0; u < 64; ++u)
-                if (u < rows) red_add_f32(base + (size_t)u * P.Hq * 128, __uint_as_float(v[u]) * P.scale);
+            for (int u = 0; u < 64; ++u) S.dq_stage[u][c] = __uint_as_float(v[u]) * P.scale;
+            fence_proxy_async();
+            mbar_arrive(&S.drain_bar);
+            ok = mbar_wait_warp(&S.drain_bar, (2 * n + 1) & 1, abort_flag);
+            if (!ok) break;
+            if (tid == 256) {
+                tma_reduce_add_4d(&tmDQ, &S.dq_stage[0][0], 0, hk * P.G + g, i0, b);     // rows beyond L are clipped
+                bulk_commit();
+            }
         }
+        if (tid == 256) bulk_wait_all();
     } else {
         if (warp == 12) {
             // ============================ producer ============================
@@ -274,18 +284,10 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             bool ok = true;
             for (int n = 0; n < n_steps && ok; ++n) {
                 const uint32_t e = S.sched[n];
-                const int h = hk * P.G + (int)(e >> 24), i0 = (int)((e >> 1) & 0x7FFFFF) * 128 + (int)(e & 1) * 64;
+                const int h = hk * P.G + (int)(e >> 11), i0 = (int)((e >> 1) & 0x3FF) * 128 + (int)(e & 1) * 64;
                 const int st = n % kStages;
                 if (n >= kStages) ok = mbar_wait_warp(&S.qd_empty[st], ((n / kStages) - 1) & 1, abort_flag);
                 if (!ok) break;
-                const size_t rowbase = (size_t)(b * P.Hq + h) * P.L;
-#pragma unroll
-                for (int c = lane; c < 64; c += 32) {
-                    const int i = i0 + c;
-                    S.nlse[st][c] = i < P.L ? -1.4426950408889634f * P.lse[rowbase + i] : 0.0f;
-                    S.dvec[st][c] = i < P.L ? -P.Dv[rowbase + i] : 0.0f;
-                }
-                __syncwarp();
                 if (lane == 0) {
                     mbar_arrive_expect_tx(&S.qd_full[st], 2 * kQBytes);
                     for (int hf = 0; hf < 2; ++hf) {
@@ -296,6 +298,38 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             }
             for (int n = max(0, n_steps - kStages); n < n_steps && ok; ++n)
                 ok = mbar_wait_warp(&S.qd_empty[n % kStages], (n / kStages) & 1, abort_flag);
+        } else if (warp == 15) {
+            // ============================ stager: -log2e*lse and -D of each step's query rows, loaded one step ahead ============================
+            auto fetch = [&](int n, float (&lv)[2], float (&dv)[2]) {
+                const uint32_t e = S.sched[n];
+                const int h = hk * P.G + (int)(e >> 11), i0 = (int)((e >> 1) & 0x3FF) * 128 + (int)(e & 1) * 64;
+                const size_t rowbase = (size_t)(b * P.Hq + h) * P.L;
+#pragma unroll
+                for (int t = 0; t < 2; ++t) {
+                    const int i = i0 + lane + 32 * t;
+                    lv[t] = i < P.L ? P.lse[rowbase + i] : 0.0f;
+                    dv[t] = i < P.L ? P.Dv[rowbase + i] : 0.0f;
+                }
+            };
+            float lv[2] = {0.f, 0.f}, dv[2] = {0.f, 0.f};
+            if (n_steps > 0) fetch(0, lv, dv);
+            bool ok = true;
+            for (int n = 0; n < n_steps && ok; ++n) {
+                const int st = n % kStages;
+                float ln[2] = {0.f, 0.f}, dn[2] = {0.f, 0.f};
+                if (n + 1 < n_steps) fetch(n + 1, ln, dn);
+                if (n >= kStages) ok = mbar_wait_warp(&S.qd_empty[st], ((n / kStages) - 1) & 1, abort_flag);
+                if (!ok) break;
+#pragma unroll
+                for (int t = 0; t < 2; ++t) {
+                    S.nlse[st][lane + 32 * t] = -1.4426950408889634f * lv[t];
+                    S.dvec[st][lane + 32 * t] = -dv[t];
+                    lv[t] = ln[t];
+                    dv[t] = dn[t];
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&S.qd_full[st]);
+            }
         } else if (warp == 13 && lane == 0) {
             // ============================ MMA issuer 1: S^T = K Q^T, dP^T = V dO^T ============================
             // (two issuing threads: every hand-over between them and the other groups is an explicit mbarrier,
@@ -402,7 +436,7 @@ size_t tc_bwd_ws_bytes(const Prob& P) {
 int launch_tc_bwd(const Prob& P, const void* Q, const void* K, const void* V, const void* O, const void* dO,
                   const float* lse, const float* bias, const int32_t* expiry, const uint32_t* bitmap, void* dQ,
                   void* dK, void* dV, float* dM, void* ws, cudaStream_t st) {
-    if ((size_t)P.G * P.Tr * 2 > (size_t)kMaxSteps) return DMA_ERR_UNSUPPORTED;
+    if ((size_t)P.G * P.Tr * 2 > (size_t)kMaxSteps || P.G > 16 || P.Tr > 1024) return DMA_ERR_UNSUPPORTED;
     const size_t rows = (size_t)P.B * P.Hq * P.L, nq = rows * P.d;
     float* Dv = reinterpret_cast<float*>((char*)ws + kWsHeaderBytes);
     float* acc = Dv + ((rows + 63) / 64) * 64;
@@ -412,6 +446,8 @@ int launch_tc_bwd(const Prob& P, const void* Q, const void* K, const void* V, co
     if ((rc = make_tmap_bf16(&tmG, dO, P.B, P.L, P.Hq, P.d, P.os, 64))) return rc;
     if ((rc = make_tmap_bf16(&tmK, K, P.B, P.L, P.Hkv, P.d, P.ks, 128))) return rc;
     if ((rc = make_tmap_bf16(&tmV, V, P.B, P.L, P.Hkv, P.d, P.vs, 128))) return rc;
+    CUtensorMap tmDQ;
+    if ((rc = make_tmap_f32_rows(&tmDQ, acc, P.B, P.L, P.Hq, 64))) return rc;
     rowdot_bf16_kernel<<<(unsigned)((rows + 7) / 8), 256, 0, st>>>((const __nv_bfloat16*)O, (const __nv_bfloat16*)dO, Dv, P.B, P.L, P.Hq,
                                                                     P.os[0], P.os[1], P.os[2]);
     if (cudaMemsetAsync(acc, 0, nq * sizeof(float), st) != cudaSuccess) return DMA_ERR_CUDA;
@@ -425,7 +461,7 @@ int launch_tc_bwd(const Prob& P, const void* Q, const void* K, const void* V, co
     bp.ks_b = P.ks[0]; bp.ks_l = P.ks[1]; bp.ks_h = P.ks[2]; bp.vs_b = P.vs[0]; bp.vs_l = P.vs[1]; bp.vs_h = P.vs[2];
     const size_t smem = sizeof(SharedStorage) + 1024;
     if (cudaFuncSetAttribute(bwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return DMA_ERR_CUDA;
-    bwd_kernel<<<dim3(P.B * P.Hkv, P.Tc), kThreads, smem, st>>>(tmQ, tmK, tmV, tmG, bp);
+    bwd_kernel<<<dim3(P.B * P.Hkv, P.Tc), kThreads, smem, st>>>(tmQ, tmK, tmV, tmG, tmDQ, bp);
     dq_convert_bf16_kernel<<<(unsigned)((nq / 8 + 255) / 256), 256, 0, st>>>(acc, (__nv_bfloat16*)dQ, nq / 8, P.L, P.Hq, P.qs[0], P.qs[1], P.qs[2]);
     count_launch(3);
     return check_launch();

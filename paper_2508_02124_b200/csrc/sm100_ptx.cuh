@@ -83,6 +83,17 @@ __device__ __forceinline__ void tma_load_4d(void* dst, const CUtensorMap* m, uin
         : "memory");
 }
 
+// 4-D tiled reduce-add from shared memory into global memory (element type from the tensor map); bulk-group tracked
+__device__ __forceinline__ void tma_reduce_add_4d(const CUtensorMap* m, const void* src, int c0, int c1, int c2, int c3) {
+    asm volatile(
+        "cp.reduce.async.bulk.tensor.4d.global.shared::cta.add.tile.bulk_group [%0, {%2, %3, %4, %5}], [%1];"
+        ::"l"(reinterpret_cast<uint64_t>(m)), "r"(smem_u32(src)), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+        : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read_all() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+
 // ---- tcgen05 / TMEM -----------------------------------------------------------------------------------------------
 __device__ __forceinline__ void tmem_alloc(uint32_t* dst_smem, uint32_t ncols) {   // whole warp
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)), "r"(ncols) : "memory");
@@ -237,5 +248,9 @@ EncodeTiledFn get_encode_tiled();
 // bf16 tensor [B, L, H, 128] with element strides (batch, seq, head): box = 64 channels x `rows` sequence positions,
 // 128-byte swizzle, out-of-range rows read as zero. Coordinates: (channel, seq, head, batch).
 int make_tmap_bf16(CUtensorMap* m, const void* base, int B, int L, int H, int d, const int64_t strides[3], int rows);
+
+// fp32 tensor [B, L, H, 128] contiguous: box = 128 channels x `rows` sequence positions of one head, no swizzle.
+// Coordinates: (channel, head, seq, batch). Used as the destination of the dQ reduce-add.
+int make_tmap_f32_rows(CUtensorMap* m, const void* base, int B, int L, int H, int rows);
 
 }  // namespace dma
