@@ -15,7 +15,8 @@
 namespace dma {
 namespace {
 
-constexpr int kChunk = 256;   // keys per sorted chunk (= threads of the sort and expiry kernels)
+constexpr int kChunk = 256;   // keys per sorted chunk (= threads of the sort kernel)
+constexpr int kExpThreads = 256;
 
 // ---- fixed-order fp32 routines: every step is one correctly rounded IEEE operation -----------------------
 
@@ -142,42 +143,76 @@ __global__ void __launch_bounds__(kChunk) chunk_sort_kernel(const float* __restr
 }
 
 // expiry[j] = max(j, index of the w-th key in index order that beats j), or L if fewer than w keys beat it.
-// The CTA walks the chunks together: each chunk's sorted keys (for the count) and keys in index order (for the
-// final walk) are staged in shared memory once for all 256 threads.
-__global__ void __launch_bounds__(kChunk) expiry_kernel(const float* __restrict__ delta,
-                                                        const unsigned long long* __restrict__ sorted,
-                                                        int32_t* __restrict__ expiry, int L, int w, int nchunk) {
-    __shared__ unsigned long long s[kChunk];      // chunk c, ascending
-    __shared__ unsigned long long u[kChunk];      // chunk c, index order
-    const int bh = blockIdx.y, t = threadIdx.x, j = blockIdx.x * kChunk + t;
+// Phase 1: the CTA walks the sorted chunks together (each staged once in shared memory as separate high / low
+// words, the next one already in flight) and every thread counts its beaters chunk by chunk with a binary search
+// until the count reaches w. Phase 2: the warp locates, lane by lane, the remaining need-th beater inside that
+// lane's final chunk with coalesced 32-key loads and a ballot.
+__global__ void __launch_bounds__(kExpThreads) expiry_kernel(const float* __restrict__ delta,
+                                                             const unsigned long long* __restrict__ sorted,
+                                                             int32_t* __restrict__ expiry, int L, int w, int nchunk) {
+    constexpr int kPer = kChunk / kExpThreads;
+    __shared__ uint32_t shi[2][kChunk], slo[2][kChunk];
+    const int bh = blockIdx.y, t = threadIdx.x, lane = t & 31, j = blockIdx.x * kExpThreads + t;
     const float* dl = delta + (size_t)bh * L;
+    const unsigned long long* srt = sorted + (size_t)bh * nchunk * kChunk;
     const bool valid = j < L;
     const unsigned long long key = valid ? sort_key(dl[j], j) : ~0ull;
-    int cnt = 0, e = L;
+    const uint32_t khi = (uint32_t)(key >> 32), klo = (uint32_t)key;
+    int cnt = 0, fin = -1, need = 0;
     bool done = !valid;
+    unsigned long long nxt[kPer];
+#pragma unroll
+    for (int u = 0; u < kPer; ++u) nxt[u] = srt[u * kExpThreads + t];
     for (int c = 0; c < nchunk; ++c) {
-        const int k = c * kChunk + t;
-        s[t] = sorted[((size_t)bh * nchunk + c) * kChunk + t];
-        u[t] = k < L ? sort_key(dl[k], k) : 0ull;
+        uint32_t* hi = shi[c & 1];
+        uint32_t* lo = slo[c & 1];
+#pragma unroll
+        for (int u = 0; u < kPer; ++u) {
+            hi[u * kExpThreads + t] = (uint32_t)(nxt[u] >> 32);
+            lo[u * kExpThreads + t] = (uint32_t)nxt[u];
+        }
+        if (c + 1 < nchunk) {
+#pragma unroll
+            for (int u = 0; u < kPer; ++u) nxt[u] = srt[(size_t)(c + 1) * kChunk + u * kExpThreads + t];
+        }
         __syncthreads();
         if (!done) {
-            int lo = 0, hi = kChunk;              // first position whose key is greater than ours
-            while (lo < hi) {
-                int mid = (lo + hi) >> 1;
-                if (s[mid] > key) hi = mid; else lo = mid + 1;
+            int a = 0, z = kChunk;                // first position whose 64-bit key is greater than ours
+            while (a < z) {
+                const int mid = (a + z) >> 1;
+                const uint32_t h = hi[mid];
+                const bool greater = h > khi || (h == khi && lo[mid] > klo);
+                if (greater) z = mid; else a = mid + 1;
             }
-            const int n = kChunk - lo;
-            if (cnt + n >= w) {
-                int need = w - cnt;               // the need-th beater lies in this chunk: walk it in index order
-                int q = 0;
-                for (; q < kChunk; ++q)
-                    if (u[q] > key && --need == 0) break;
-                e = max(j, c * kChunk + q);
-                done = true;
-            }
+            const int n = kChunk - a;
+            if (cnt + n >= w) { need = w - cnt; fin = c; done = true; }
             cnt += n;
         }
         if (__syncthreads_and(done)) break;
+    }
+    // phase 2, warp-cooperative: lane `src` broadcasts (chunk, key, need); the warp scans that chunk 32 keys at a time
+    int e = L;
+    const uint32_t pending = __ballot_sync(0xffffffffu, fin >= 0);
+    for (uint32_t rest = pending; rest; rest &= rest - 1) {
+        const int src = __ffs(rest) - 1;
+        const int base = __shfl_sync(0xffffffffu, fin, src) * kChunk;
+        const uint32_t bhi = __shfl_sync(0xffffffffu, khi, src), blo = __shfl_sync(0xffffffffu, klo, src);
+        int nd = __shfl_sync(0xffffffffu, need, src);
+        const unsigned long long bkey = ((unsigned long long)bhi << 32) | blo;
+        int found = L;
+        for (int g = 0; g < kChunk; g += 32) {
+            const int k = base + g + lane;
+            const bool beat = k < L && sort_key(dl[k], k) > bkey;
+            uint32_t m = __ballot_sync(0xffffffffu, beat);
+            const int pc = __popc(m);
+            if (nd <= pc) {
+                for (int r = 1; r < nd; ++r) m &= m - 1;          // drop the nd-1 lowest beaters
+                found = base + g + __ffs(m) - 1;
+                break;
+            }
+            nd -= pc;
+        }
+        if (lane == src) e = max(j, found);
     }
     if (valid) expiry[(size_t)bh * L + j] = e;
 }
@@ -215,6 +250,8 @@ __global__ void __launch_bounds__(128) bitmap_kernel(const int32_t* __restrict__
 
 }  // namespace
 
+constexpr int kStaticChunk = kChunk;
+
 size_t mask_ws_bytes(const Prob& P) {
     const size_t nchunk = (P.L + kChunk - 1) / kChunk;
     return kWsHeaderBytes + (size_t)P.B * P.Hq * nchunk * kChunk * sizeof(unsigned long long);
@@ -249,7 +286,7 @@ int launch_mask_build(const Prob& P, const void* V, const float* W, const float*
     } else {
         auto* sorted = reinterpret_cast<unsigned long long*>((char*)ws + kWsHeaderBytes);
         chunk_sort_kernel<<<dim3(nchunk, BH), kChunk, 0, st>>>(bias, sorted, P.L, nchunk);
-        expiry_kernel<<<dim3(nchunk, BH), kChunk, 0, st>>>(bias, sorted, expiry, P.L, P.w, nchunk);
+        expiry_kernel<<<dim3((P.L + kExpThreads - 1) / kExpThreads, BH), kExpThreads, 0, st>>>(bias, sorted, expiry, P.L, P.w, nchunk);
         count_launch(2);
     }
     if ((rc = check_launch())) return rc;
@@ -286,7 +323,7 @@ extern "C" int dma_mask_build_static(const dma_problem_t* p, const void* V, cons
     if (!V || !W_delta || !A || !bias || !expiry || !bitmap) return DMA_ERR_NULL;
     const uintptr_t bits = (uintptr_t)V | (uintptr_t)W_delta | (uintptr_t)bias | (uintptr_t)expiry | (uintptr_t)bitmap;
     if (bits & 15) return DMA_ERR_ALIGN;
-    const size_t keys = (size_t)P.B * P.Hq * ((P.L + 255) / 256) * 256;
+    const size_t keys = (size_t)P.B * P.Hq * ((P.L + dma::kStaticChunk - 1) / dma::kStaticChunk) * dma::kStaticChunk;
     if (keys > kStaticKeys) return DMA_ERR_WORKSPACE;          // larger problems must use dma_mask_build
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return DMA_ERR_CUDA;
