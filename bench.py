@@ -137,10 +137,13 @@ def main():
     ap.add_argument("--ref-rows", type=int, default=4096, help="rows of the oracle sample per step (--impl reference)")
     ap.add_argument("--cpu-rows", type=int, default=8192, help="rows of the oracle sample for cpu_baseline (0 = skip)")
     ap.add_argument("--no-e2e", action="store_true")
-    ap.add_argument("--flags", type=int, default=0)
+    ap.add_argument("--flags", type=int, default=0, help="dma_problem_t.flags (1 = ignore the bitmap, 2 = CUDA-core kernels)")
+    ap.add_argument("--seq-len", type=int, default=0, help="override the workload's sequence length (profiling of a smaller case)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "dma" else args.warmup
     case = wl.CONFIGS[args.workload]
+    if args.seq_len:
+        case = wl.small(case, L=args.seq_len, w=min(case.w, args.seq_len), name=f"{case.name}-L{args.seq_len}")
     if args.impl == "reference":
         return run_reference(args, case)
 
