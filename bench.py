@@ -26,6 +26,9 @@ from paper_2508_02124_b200 import workloads as wl  # noqa: E402
 
 METRIC = "dma_fwd_bwd_executed_tile_tflops"
 NOMINAL_BF16_TFLOPS = 2250.0
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from one ncu capture of this
+# command at full size (profiles/dram_traffic_cfg3_train16k.md); other workloads: not captured.
+NCU_TRAFFIC_BYTES = {"cfg3-train-16k": {"bwd": 3.65e9, "fwd": 0.514e9}}
 
 
 def tile_flops(active_tiles, d, backward, bm=128, bn=128):
@@ -130,7 +133,7 @@ def run_reference(args, case):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", default="3", help="key of workloads.CONFIGS (3 = 16K training step, the headline)")
     ap.add_argument("--impl", default="dma", choices=["dma", "reference"])
@@ -276,7 +279,8 @@ def main():
         "dense_causal_equivalent_speedup": causal_tiles(case) / max(active, 1),
         "roofline": {"bound": "tensor" if tensor_path else "alu", "kernel": f"dma_attn_{dom} (stage time, includes its pre/post kernels)",
                      "achieved": achieved, "peak": pk["bf16_sustained"], "peak_source": pk["source"] + " sustained cuBLAS bf16",
-                     "unit": "TFLOP/s", "frac": achieved / pk["bf16_sustained"], "traffic": None},
+                     "unit": "TFLOP/s", "frac": achieved / pk["bf16_sustained"],
+                     "traffic": NCU_TRAFFIC_BYTES.get(case.name, {}).get(dom) if tensor_path else None},
         "gpu_launches": launches, "clocks": clocks, "e2e": e2e,
     }
     if args.cpu_rows:

@@ -1,4 +1,7 @@
 """Shared test plumbing: run a workload through the C-ABI on the GPU, and through the CPU oracle."""
+import json
+import os
+
 import numpy as np
 import torch
 
@@ -81,6 +84,10 @@ def assert_close(got, ref, dtype, what, lse=False):
     tol_abs = atol + 1e-6 * M if lse else atol * max(1.0, M)
     den = np.sqrt((ref * ref).sum())
     rel = float(np.sqrt((diff * diff).sum()) / den) if den > 0 else float(diff.max())
+    if os.environ.get("DMA_PARITY_LOG"):          # optional record of the measured errors (one JSON line per check)
+        with open(os.environ["DMA_PARITY_LOG"], "a") as f:
+            f.write(json.dumps({"test": os.environ.get("PYTEST_CURRENT_TEST", ""), "what": what, "dtype": dtype,
+                                "max_abs": float(diff.max()), "tol_abs": tol_abs, "rel_l2": rel, "ref_max": M}) + "\n")
     assert np.isfinite(g).all(), f"{what}: non-finite values"
     assert diff.max() <= tol_abs and rel <= tol_rel, (f"{what}: max-abs {diff.max():.3e} (tol {tol_abs:.2e}, |ref| max "
                                                      f"{M:.3e}), rel-L2 {rel:.3e} (tol {tol_rel:.1e})")
