@@ -151,6 +151,7 @@ def main():
         return run_reference(args, case)
 
     from paper_2508_02124_b200 import binding as dma
+    from paper_2508_02124_b200 import replicas
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
@@ -216,11 +217,7 @@ def main():
     for e in evs:
         stage_ms["mask"] += e[0].elapsed_time(e[1]); stage_ms["fwd"] += e[1].elapsed_time(e[2]); stage_ms["bwd"] += e[2].elapsed_time(e[3])
     stage_ms = {k: v / args.steps for k, v in stage_ms.items()}
-    ms = total_ms / args.steps
-    if dist is not None:
-        t = torch.tensor([ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = replicas.max_over_ranks(total_ms / args.steps, dev)
 
     # ---- end to end through the host-buffer entry point: pinned host tensors in, results back on the host
     e2e = None
@@ -240,11 +237,7 @@ def main():
             call()
         t3.record()
         barrier()
-        e2e_ms = t2.elapsed_time(t3) / n_e2e
-        if dist is not None:
-            t = torch.tensor([e2e_ms], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e2e_ms = float(t.item())
+        e2e_ms = replicas.max_over_ranks(t2.elapsed_time(t3) / n_e2e, dev)
         nb = lambda *ts: int(sum(t.numel() * t.element_size() for t in ts))
         h2d = nb(*hin) if case.backward else nb(hin[0], hin[1], hin[2], hin[4], hin[5])
         d2h = nb(hO, hlse) + (nb(hdQ, hdK, hdV, hdM) if case.backward else 0)

@@ -135,6 +135,12 @@ int dma_step_host(const dma_problem_t* p, int backward, const void* hQ, const vo
 /* Synchronises the stream and returns the device status word of a workspace (0 or DMA_ERR_DEVICE_TIMEOUT). */
 int dma_read_status(const void* ws, void* cuda_stream);
 
+/* Self-test of the bounded device-side waits (every mbarrier wait in the kernels gives up after a cycle limit, raises
+ * the CTA's abort flag and leaves DMA_ERR_DEVICE_TIMEOUT in the workspace status word instead of hanging): launches
+ * one small CTA that waits, with a ~2 ms limit, on a barrier nothing arrives at. Afterwards dma_read_status(ws) must
+ * return DMA_ERR_DEVICE_TIMEOUT and the context stays usable. ws: any workspace of at least 256 bytes. */
+int dma_selftest_wait_timeout(void* ws, size_t ws_bytes, void* cuda_stream);
+
 /* Number of kernels the library has launched in this process (all entry points), for accounting. */
 long long dma_launch_count(void);
 

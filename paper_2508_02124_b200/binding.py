@@ -17,7 +17,7 @@ DMA_BF16, DMA_FP32 = 0, 1
 DMA_FLAG_IGNORE_BITMAP, DMA_FLAG_SIMT = 1, 2
 
 ENTRY_POINTS = ("dma_query_workspace", "dma_bitmap_words", "dma_mask_build", "dma_attn_fwd", "dma_attn_bwd",
-                "dma_read_status", "dma_launch_count", "dma_strerror", "dma_step_host_arena", "dma_step_host", "dma_mask_build_static")
+                "dma_read_status", "dma_launch_count", "dma_strerror", "dma_step_host_arena", "dma_step_host", "dma_mask_build_static", "dma_selftest_wait_timeout")
 
 
 class DmaError(RuntimeError):
@@ -165,3 +165,8 @@ def dma_mask_build_static(p, V, W_delta, A, bias, expiry, bitmap):
     _check(lib().dma_mask_build_static(ctypes.byref(p), _ptr(V), _ptr(W_delta), _ptr(A), _ptr(bias), _ptr(expiry),
                                        _ptr(bitmap), _stream()), "dma_mask_build_static")
     return bias, expiry, bitmap
+
+
+def dma_selftest_wait_timeout(ws):
+    """Launches the bounded-wait self test; afterwards dma_read_status(ws) reports DMA_ERR_DEVICE_TIMEOUT (-7)."""
+    _check(lib().dma_selftest_wait_timeout(_ptr(ws), ctypes.c_size_t(ws.numel()), _stream()), "dma_selftest_wait_timeout")

@@ -3,6 +3,7 @@
 #include <cmath>
 
 #include "common.cuh"
+#include "sm100_ptx.cuh"
 
 namespace dma {
 
@@ -56,6 +57,22 @@ static int device_ok() {
     if (cudaGetDevice(&dev) != cudaSuccess) return DMA_ERR_CUDA;
     if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return DMA_ERR_CUDA;
     return major == 10 ? DMA_OK : DMA_ERR_CUDA;
+}
+
+// One CTA waits on an mbarrier that nothing ever arrives at, with a limit of about two milliseconds: the wait gives
+// up, the abort flag is raised and the status word is written, exactly as in the attention kernels.
+__global__ void selftest_wait_kernel(int32_t* status) {
+    __shared__ uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        ptx::mbar_init(&bar, 1);
+        abort_flag = 0;
+        ptx::fence_barrier_init();
+    }
+    __syncthreads();
+    const bool ok = ptx::mbar_wait(&bar, 0, &abort_flag, 1ll << 22);
+    __syncthreads();
+    if (threadIdx.x == 0 && (!ok || abort_flag)) atomicExch(status, (int32_t)DMA_ERR_DEVICE_TIMEOUT);
 }
 
 }  // namespace dma
@@ -143,6 +160,17 @@ int dma_read_status(const void* ws, void* cuda_stream) {
     if (cudaMemcpyAsync(&word, ws, sizeof(word), cudaMemcpyDeviceToHost, st) != cudaSuccess) return DMA_ERR_CUDA;
     if (cudaStreamSynchronize(st) != cudaSuccess) return DMA_ERR_CUDA;
     return word == 0 ? DMA_OK : DMA_ERR_DEVICE_TIMEOUT;
+}
+
+int dma_selftest_wait_timeout(void* ws, size_t ws_bytes, void* cuda_stream) {
+    if (!ws || ws_bytes < (size_t)kWsHeaderBytes || !aligned16(ws)) return DMA_ERR_WORKSPACE;
+    int rc = device_ok();
+    if (rc) return rc;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    if (cudaMemsetAsync(ws, 0, kWsHeaderBytes, st) != cudaSuccess) return DMA_ERR_CUDA;
+    selftest_wait_kernel<<<1, 64, 0, st>>>((int32_t*)ws);
+    count_launch();
+    return check_launch();
 }
 
 long long dma_launch_count(void) { return g_launches.load(); }

@@ -52,13 +52,14 @@ __device__ __forceinline__ bool mbar_try_wait_hint(uint64_t* bar, uint32_t parit
 
 // Bounded wait: gives up after ~2^31 clock cycles (about a second) or when another thread of the CTA has already
 // given up; on expiry raises the CTA's abort flag so that every other wait of the CTA returns at once.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                          long long limit_cycles = (1ll << 31)) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     while (true) {
         if (mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
-        if (clock64() - t0 > (1ll << 31)) {
+        if (clock64() - t0 > limit_cycles) {
             *abort_flag = 1;
             return false;
         }

@@ -152,3 +152,16 @@ def test_full_size_configs_sampled(key):
     sampled_check(case, inp, got)
     if case.backward:
         dq_rows_check(case, inp, got, np.array([0, 5, 130, 700, 1500]))
+
+
+def test_bounded_wait_reports_timeout_and_context_survives():
+    # a wait that nothing satisfies gives up after its limit and leaves a status, instead of hanging the GPU
+    dev = torch.device("cuda:0")
+    ws = torch.zeros(256, dtype=torch.uint8, device=dev)
+    dma.dma_selftest_wait_timeout(ws)
+    assert dma.dma_read_status(ws) == -7
+    # the context is still usable and a normal call leaves a clean status
+    case = wl.small(C2, B=1, Hq=2, Hkv=1, L=256, w=64, backward=False, name="after-timeout")
+    inp = wl.make_inputs(case)
+    got = gpu_run(case, inp, backward=False)
+    assert torch.isfinite(got["O"].float()).all()
