@@ -14,7 +14,7 @@ OBJ = os.path.join(PKG, "build")
 LIB = os.path.join(PKG, "libdma_b200.so")
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 FLAGS = ["-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-Xcompiler", "-fPIC",
-         "-I", os.path.join(ROOT, "include"), "-I", CSRC]
+         "-I", os.path.join(ROOT, "include"), "-I", CSRC] + os.environ.get("DMA_NVCC_FLAGS", "").split()
 
 
 def sources():

@@ -13,6 +13,8 @@
 // split the 64 query columns of a step), warps 8-11 dQ drain (thread = channel), warp 12 TMA producer + schedule,
 // warps 13 and 14 MMA issuers (S^T, dP^T | dV, dK, dQ^T), warp 15 stages -lse and -D of each step's query rows.
 // TMEM columns: dK [0,128) dV [128,256) S^T [256,320) dP^T [320,384) P^T [384,416) dS^T [416,448) dQ^T [448,512).
+#include <cstdlib>
+
 #include "common.cuh"
 #include "sm100_ptx.cuh"
 
@@ -34,12 +36,12 @@ struct SharedStorage {
     alignas(1024) uint8_t q[kStages][kQBytes];
     alignas(1024) uint8_t g[kStages][kQBytes];       // dO
     alignas(1024) uint8_t ds[128 * 128];             // dS^T as bf16: [128 keys][64 queries], 128-byte swizzled rows
-    alignas(1024) float dq_stage[64][128];           // dQ of one step, [query row][channel], source of the TMA reduce-add
+    alignas(1024) float dq_stage[4][2][32][32];      // dQ per drain warp (32 channels) and half step: [query row][channel], sources of the TMA reduce-adds
     alignas(16) float nlse[kStages][64];             // -log2(e) * lse_i
     alignas(16) float dvec[kStages][64];             // -D_i
     uint16_t sched[kMaxSteps];                       // head-in-group << 11 | query tile << 1 | half
     uint64_t kv_full, qd_full[kStages], qd_empty[kStages];
-    uint64_t sdp_full, sdp_free, pds_ready, pds_free, dq_full, dq_free, drain_bar;
+    uint64_t sdp_full, sdp_free, pds_ready, pds_free, dq_full, dq_free;
     uint32_t tmem_base;
     int n_steps;
     int abort_flag;
@@ -59,7 +61,22 @@ struct BwdParams {
     int B, Hq, Hkv, G, L, Tr, Tc, Wd, ignore_bitmap;
     float scale, scale_log2;
     int64_t ks_b, ks_l, ks_h, vs_b, vs_l, vs_h;
+#ifdef DMA_PROF
+    long long* prof;            // role timing (development builds only): cycles per phase of CTA (0, 0)
+#endif
 };
+
+// PROF_WAIT(slot, expr): evaluates expr (a wait) and, in development builds, adds its duration to a per-role counter
+#ifdef DMA_PROF
+#define PROF_DECL(role) const bool prof_on = P.prof && blockIdx.x == 0 && blockIdx.y == 0 && lane == 0; \
+    long long prof_acc[8] = {0, 0, 0, 0, 0, 0, 0, 0}; const long long prof_start = clock64(); const int prof_role = role
+#define PROF_WAIT(slot, expr) do { const long long t0_ = clock64(); expr; prof_acc[slot] += clock64() - t0_; } while (0)
+#define PROF_END() do { if (prof_on) { prof_acc[7] = clock64() - prof_start; for (int k_ = 0; k_ < 8; ++k_) P.prof[prof_role * 8 + k_] = prof_acc[k_]; } } while (0)
+#else
+#define PROF_DECL(role)
+#define PROF_WAIT(slot, expr) do { expr; } while (0)
+#define PROF_END()
+#endif
 
 __global__ void __launch_bounds__(kThreads, 1)
 bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
@@ -85,7 +102,6 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
         mbar_init(&S.pds_free, 1);
         mbar_init(&S.dq_full, 1);
         mbar_init(&S.dq_free, 128);
-        mbar_init(&S.drain_bar, 128);
         S.abort_flag = 0;
         S.n_steps = 0;
         fence_barrier_init();
@@ -134,6 +150,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
         float2 dm2 = make_float2(0.0f, 0.0f);
         int len = 0, cur_g = -1;
         bool ok = true;
+        PROF_DECL(warp == 0 ? 0 : 7);
         for (int n = 0; n < n_steps && ok; ++n) {
             const uint32_t e = S.sched[n];
             const int g = (int)(e >> 11), i0 = (int)((e >> 1) & 0x3FF) * 128 + (int)(e & 1) * 64;
@@ -146,46 +163,82 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                 len = j < P.L ? P.expiry[(size_t)bh * P.L + j] - j : 0;
                 cur_g = g;
             }
-            ok = mbar_wait_warp(&S.sdp_full, n & 1, abort_flag) && mbar_wait_warp(&S.qd_full[st], (n / kStages) & 1, abort_flag);
+            PROF_WAIT(0, ok = mbar_wait_warp(&S.sdp_full, n & 1, abort_flag) && mbar_wait_warp(&S.qd_full[st], (n / kStages) & 1, abort_flag));
             if (!ok) break;
             tc_fence_after();
             uint32_t sr[32], pr[32];
+#ifdef DMA_PROF
+            const long long tp0 = clock64();
+#endif
             tmem_ld32(tmem + lane_base + cS + hsel * 32, sr);
             tmem_ld32(tmem + lane_base + cDP + hsel * 32, pr);
             tc_wait_ld();
             tc_fence_before();
             mbar_arrive(&S.sdp_free);
+#ifdef DMA_PROF
+            const long long tp1 = clock64();
+            prof_acc[2] += tp1 - tp0;
+#endif
             // valid columns of this thread within its 32: col in [lo, lo + width)
             const int c0 = hsel * 32;
             const int lo = max(0, j - i0 - c0);
             const int width = max(0, min(32, j - i0 - c0 + len) - lo);
-            const bool plain = __all_sync(0xffffffffu, lo == 0);      // off the diagonal only the upper bound matters
+            // Almost every (key, 32-row group) pair is all-or-nothing: then the mask is one additive term per thread
+            // (0 or -inf) and the per-element test is skipped. Warps with a partly kept key take the general loop.
+            const bool uniform = __all_sync(0xffffffffu, lo == 0 && (width == 0 || width == 32));
             uint32_t pp[16], dd[16];
-            const float2 bj2 = make_float2(bj, bj), sc2 = make_float2(P.scale_log2, P.scale_log2);
+            const float2 sc2 = make_float2(P.scale_log2, P.scale_log2);
+            if (uniform) {
+                const float be = width ? bj : -INFINITY;
+                const float2 bj2 = make_float2(be, be);
 #pragma unroll
-            for (int c = 0; c < 32; c += 4) {
-                const float4 nl = *reinterpret_cast<const float4*>(&S.nlse[st][c0 + c]);
-                const float4 nd = *reinterpret_cast<const float4*>(&S.dvec[st][c0 + c]);   // holds -D_i
-                float2 x[2], t[2];
-                x[0] = fma2(make_float2(__uint_as_float(sr[c]), __uint_as_float(sr[c + 1])), sc2, add2(make_float2(nl.x, nl.y), bj2));
-                x[1] = fma2(make_float2(__uint_as_float(sr[c + 2]), __uint_as_float(sr[c + 3])), sc2, add2(make_float2(nl.z, nl.w), bj2));
-                t[0] = add2(make_float2(__uint_as_float(pr[c]), __uint_as_float(pr[c + 1])), make_float2(nd.x, nd.y));
-                t[1] = add2(make_float2(__uint_as_float(pr[c + 2]), __uint_as_float(pr[c + 3])), make_float2(nd.z, nd.w));
-                float p[4] = {ex2(x[0].x), ex2(x[0].y), ex2(x[1].x), ex2(x[1].y)};
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const bool valid = plain ? (c + u < width) : ((unsigned)(c + u - lo) < (unsigned)width);
-                    p[u] = valid ? p[u] : 0.0f;
+                for (int c = 0; c < 32; c += 4) {
+                    const float4 nl = *reinterpret_cast<const float4*>(&S.nlse[st][c0 + c]);
+                    const float4 nd = *reinterpret_cast<const float4*>(&S.dvec[st][c0 + c]);   // holds -D_i
+                    float2 x[2], t[2];
+                    x[0] = fma2(make_float2(__uint_as_float(sr[c]), __uint_as_float(sr[c + 1])), sc2, add2(make_float2(nl.x, nl.y), bj2));
+                    x[1] = fma2(make_float2(__uint_as_float(sr[c + 2]), __uint_as_float(sr[c + 3])), sc2, add2(make_float2(nl.z, nl.w), bj2));
+                    t[0] = add2(make_float2(__uint_as_float(pr[c]), __uint_as_float(pr[c + 1])), make_float2(nd.x, nd.y));
+                    t[1] = add2(make_float2(__uint_as_float(pr[c + 2]), __uint_as_float(pr[c + 3])), make_float2(nd.z, nd.w));
+                    const float2 p0 = make_float2(ex2(x[0].x), ex2(x[0].y)), p1 = make_float2(ex2(x[1].x), ex2(x[1].y));
+                    const float2 d0 = mul2(p0, t[0]), d1 = mul2(p1, t[1]);
+                    dm2 = add2(dm2, add2(d0, d1));
+                    pp[(c >> 1)] = pack_bf16(p0.x, p0.y);
+                    pp[(c >> 1) + 1] = pack_bf16(p1.x, p1.y);
+                    dd[(c >> 1)] = pack_bf16(d0.x, d0.y);
+                    dd[(c >> 1) + 1] = pack_bf16(d1.x, d1.y);
                 }
-                const float2 d0 = mul2(make_float2(p[0], p[1]), t[0]), d1 = mul2(make_float2(p[2], p[3]), t[1]);
-                dm2 = add2(dm2, add2(d0, d1));
-                pp[(c >> 1)] = pack_bf16(p[0], p[1]);
-                pp[(c >> 1) + 1] = pack_bf16(p[2], p[3]);
-                dd[(c >> 1)] = pack_bf16(d0.x, d0.y);
-                dd[(c >> 1) + 1] = pack_bf16(d1.x, d1.y);
+            } else {
+                const float2 bj2 = make_float2(bj, bj);
+#pragma unroll
+                for (int c = 0; c < 32; c += 4) {
+                    const float4 nl = *reinterpret_cast<const float4*>(&S.nlse[st][c0 + c]);
+                    const float4 nd = *reinterpret_cast<const float4*>(&S.dvec[st][c0 + c]);   // holds -D_i
+                    float2 x[2], t[2];
+                    x[0] = fma2(make_float2(__uint_as_float(sr[c]), __uint_as_float(sr[c + 1])), sc2, add2(make_float2(nl.x, nl.y), bj2));
+                    x[1] = fma2(make_float2(__uint_as_float(sr[c + 2]), __uint_as_float(sr[c + 3])), sc2, add2(make_float2(nl.z, nl.w), bj2));
+                    t[0] = add2(make_float2(__uint_as_float(pr[c]), __uint_as_float(pr[c + 1])), make_float2(nd.x, nd.y));
+                    t[1] = add2(make_float2(__uint_as_float(pr[c + 2]), __uint_as_float(pr[c + 3])), make_float2(nd.z, nd.w));
+                    float p[4] = {ex2(x[0].x), ex2(x[0].y), ex2(x[1].x), ex2(x[1].y)};
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const bool valid = (unsigned)(c + u - lo) < (unsigned)width;
+                        p[u] = valid ? p[u] : 0.0f;
+                    }
+                    const float2 d0 = mul2(make_float2(p[0], p[1]), t[0]), d1 = mul2(make_float2(p[2], p[3]), t[1]);
+                    dm2 = add2(dm2, add2(d0, d1));
+                    pp[(c >> 1)] = pack_bf16(p[0], p[1]);
+                    pp[(c >> 1) + 1] = pack_bf16(p[2], p[3]);
+                    dd[(c >> 1)] = pack_bf16(d0.x, d0.y);
+                    dd[(c >> 1) + 1] = pack_bf16(d1.x, d1.y);
+                }
             }
+#ifdef DMA_PROF
+            const long long tp2 = clock64();
+            prof_acc[3] += tp2 - tp1 + (long long)(pp[3] == 0x12345u && dd[7] == 0x54321u);
+#endif
             // the previous step's dV / dK / dQ GEMMs must have finished reading P^T, dS^T (TMEM) and dS^T (smem)
-            if (n > 0) ok = mbar_wait_warp(&S.pds_free, (n - 1) & 1, abort_flag);
+            if (n > 0) PROF_WAIT(1, ok = mbar_wait_warp(&S.pds_free, (n - 1) & 1, abort_flag));
             if (!ok) break;
             tc_fence_after();
             tmem_st16(tmem + lane_base + cP + hsel * 16, pp);
@@ -200,7 +253,11 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             tc_wait_st();
             tc_fence_before();
             mbar_arrive(&S.pds_ready);
+#ifdef DMA_PROF
+            prof_acc[4] += clock64() - tp2;
+#endif
         }
+        if (warp == 0) PROF_END();
         if (cur_g >= 0 && j < P.L) atomicAdd(&P.dM[(size_t)(b * P.Hq + hk * P.G + cur_g) * P.L + j], dm2.x + dm2.y);
         // epilogue: dK (scaled) and dV rows to global memory; warps w and w+4 each write one half of the channels
         if (ok && n_steps > 0) ok = mbar_wait_warp(&S.pds_free, (n_steps - 1) & 1, abort_flag);
@@ -239,13 +296,17 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
         }
     } else if (warp < 12) {
         // ============================ dQ drain group: thread = channel c, columns = query rows ============================
-        const int c = tid - 256;
-        const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+        // Each warp owns 32 channels and its own pair of staging buffers (one per 32-row half step), so the warps
+        // never wait for each other: a half is rewritten once the reduce-add issued from it two groups ago has
+        // finished reading it.
+        const int dw = warp & 3;
+        const uint32_t lane_base = (uint32_t)(dw * 32) << 16;
         bool ok = true;
+        PROF_DECL(warp == 8 ? 1 : 7);
         for (int n = 0; n < n_steps && ok; ++n) {
             const uint32_t e = S.sched[n];
             const int g = (int)(e >> 11), i0 = (int)((e >> 1) & 0x3FF) * 128 + (int)(e & 1) * 64;
-            ok = mbar_wait_warp(&S.dq_full, n & 1, abort_flag);
+            PROF_WAIT(0, ok = mbar_wait_warp(&S.dq_full, n & 1, abort_flag));
             if (!ok) break;
             tc_fence_after();
             uint32_t v[64];
@@ -254,23 +315,21 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             tc_wait_ld();
             tc_fence_before();
             mbar_arrive(&S.dq_free);
-            // hand the step's dQ (scaled) to the TMA: staging buffer free -> write [row][channel] -> one reduce-add
-            if (tid == 256) bulk_wait_read_all();
-            mbar_arrive(&S.drain_bar);
-            ok = mbar_wait_warp(&S.drain_bar, (2 * n) & 1, abort_flag);
-            if (!ok) break;
 #pragma unroll
-            for (int u = 0; u < 64; ++u) S.dq_stage[u][c] = __uint_as_float(v[u]) * P.scale;
-            fence_proxy_async();
-            mbar_arrive(&S.drain_bar);
-            ok = mbar_wait_warp(&S.drain_bar, (2 * n + 1) & 1, abort_flag);
-            if (!ok) break;
-            if (tid == 256) {
-                tma_reduce_add_4d(&tmDQ, &S.dq_stage[0][0], 0, hk * P.G + g, i0, b);     // rows beyond L are clipped
-                bulk_commit();
+            for (int hf = 0; hf < 2; ++hf) {
+                PROF_WAIT(1 + hf, if (lane == 0) bulk_wait_read_1(); __syncwarp());
+#pragma unroll
+                for (int u = 0; u < 32; ++u) S.dq_stage[dw][hf][u][lane] = __uint_as_float(v[hf * 32 + u]);
+                fence_proxy_async();
+                __syncwarp();
+                if (lane == 0 && i0 + hf * 32 < P.L) {
+                    tma_reduce_add_4d(&tmDQ, &S.dq_stage[dw][hf][0][0], dw * 32, hk * P.G + g, i0 + hf * 32, b);   // rows beyond L are clipped
+                }
+                if (lane == 0) bulk_commit();
             }
         }
-        if (tid == 256) bulk_wait_all();
+        if (warp == 8) PROF_END();
+        if (lane == 0) bulk_wait_all();
     } else {
         if (warp == 12) {
             // ============================ producer ============================
@@ -337,10 +396,11 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             constexpr uint32_t id_sdp = idesc_bf16(128, 64, 0, 0);     // K|V (K-major) x Q|dO (K-major)       -> 128 x 64
             const uint64_t dK = smem_desc_sw128(smem_u32(S.k), 16, 1024), dV = smem_desc_sw128(smem_u32(S.v), 16, 1024);
             bool ok = mbar_wait(&S.kv_full, 0, abort_flag);
+            PROF_DECL(2);
             for (int n = 0; n < n_steps && ok; ++n) {
                 const int st = n % kStages;
-                ok = mbar_wait(&S.qd_full[st], (n / kStages) & 1, abort_flag);
-                if (ok && n > 0) ok = mbar_wait(&S.sdp_free, (n - 1) & 1, abort_flag);
+                PROF_WAIT(0, ok = mbar_wait(&S.qd_full[st], (n / kStages) & 1, abort_flag));
+                if (ok && n > 0) PROF_WAIT(1, ok = mbar_wait(&S.sdp_free, (n - 1) & 1, abort_flag));
                 if (!ok) break;
                 tc_fence_after();
                 const uint64_t dQ = smem_desc_sw128(smem_u32(S.q[st]), 16, 1024), dG = smem_desc_sw128(smem_u32(S.g[st]), 16, 1024);
@@ -354,16 +414,18 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                            dG + (uint64_t)(((kk >> 2) * (kQBytes / 2) + (kk & 3) * 32) >> 4), id_sdp, kk > 0);
                 tc_commit(&S.sdp_full);
             }
+            PROF_END();
         } else if (warp == 14 && lane == 0) {
             // ============================ MMA issuer 2: dV += P^T dO, dK += dS^T Q, dQ^T = K^T dS^T ============================
             constexpr uint32_t id_dkv = idesc_bf16(128, 128, 0, 1);    // P^T|dS^T (TMEM) x dO|Q (MN-major)    -> 128 x 128
             constexpr uint32_t id_dq = idesc_bf16(128, 64, 1, 1);      // K^T (MN-major) x dS^T (MN-major)     -> 128 x 64
             const uint64_t dKt = smem_desc_sw128(smem_u32(S.k), kKVBytes / 2, 1024), dDs = smem_desc_sw128(smem_u32(S.ds), 16, 1024);
             bool ok = true;
+            PROF_DECL(3);
             for (int n = 0; n < n_steps && ok; ++n) {
                 const int st = n % kStages;
-                ok = mbar_wait(&S.pds_ready, n & 1, abort_flag);
-                if (ok && n > 0) ok = mbar_wait(&S.dq_free, (n - 1) & 1, abort_flag);
+                PROF_WAIT(0, ok = mbar_wait(&S.pds_ready, n & 1, abort_flag));
+                if (ok && n > 0) PROF_WAIT(1, ok = mbar_wait(&S.dq_free, (n - 1) & 1, abort_flag));
                 if (!ok) break;
                 tc_fence_after();
                 const uint64_t dGm = smem_desc_sw128(smem_u32(S.g[st]), kQBytes / 2, 1024), dQm = smem_desc_sw128(smem_u32(S.q[st]), kQBytes / 2, 1024);
@@ -373,13 +435,14 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
 #pragma unroll
                 for (int kk = 0; kk < 4; ++kk)
                     mma_ts(tmem + cDK, tmem + cDS + kk * 8, dQm + (uint64_t)((kk * 2048) >> 4), id_dkv, (n > 0 || kk > 0) ? 1u : 0u);
+                tc_commit(&S.qd_empty[st]);            // the dQ GEMM reads K and dS^T only: Q / dO of this stage are free here
 #pragma unroll
                 for (int kk = 0; kk < 8; ++kk)         // 128 keys = 8 k-steps of 16
                     mma_ss(tmem + cDQ, dKt + (uint64_t)((kk * 2048) >> 4), dDs + (uint64_t)((kk * 2048) >> 4), id_dq, kk > 0);
                 tc_commit(&S.pds_free);
                 tc_commit(&S.dq_full);
-                tc_commit(&S.qd_empty[st]);
             }
+            PROF_END();
         }
     }
     tc_fence_before();
@@ -413,16 +476,17 @@ __global__ void rowdot_bf16_kernel(const __nv_bfloat16* __restrict__ O, const __
     if (lane == 0) Dv[row] = s;
 }
 
-// fp32 accumulator [B, L, Hq, 128] -> bf16 dQ in the caller's layout; 8 elements per thread
+// fp32 accumulator [B, L, Hq, 128] (unscaled dS K sums) -> softmax scale applied -> bf16 dQ in the caller's layout; 8 elements per thread
 __global__ void dq_convert_bf16_kernel(const float* __restrict__ acc, __nv_bfloat16* __restrict__ dQ, size_t n8, int L, int Hq,
-                                       int64_t qs_b, int64_t qs_l, int64_t qs_h) {
+                                       int64_t qs_b, int64_t qs_l, int64_t qs_h, float scale) {
     const size_t t = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (t >= n8) return;
     const size_t e = t * 8;
     const int c = e % 128, h = (e / 128) % Hq, i = (e / ((size_t)128 * Hq)) % L, b = e / ((size_t)128 * Hq * L);
     const float4 a = *reinterpret_cast<const float4*>(acc + e), bb = *reinterpret_cast<const float4*>(acc + e + 4);
     uint4 o;
-    o.x = ptx::pack_bf16(a.x, a.y); o.y = ptx::pack_bf16(a.z, a.w); o.z = ptx::pack_bf16(bb.x, bb.y); o.w = ptx::pack_bf16(bb.z, bb.w);
+    o.x = ptx::pack_bf16(a.x * scale, a.y * scale); o.y = ptx::pack_bf16(a.z * scale, a.w * scale);
+    o.z = ptx::pack_bf16(bb.x * scale, bb.y * scale); o.w = ptx::pack_bf16(bb.z * scale, bb.w * scale);
     *reinterpret_cast<uint4*>(dQ + b * qs_b + (int64_t)i * qs_l + h * qs_h + c) = o;
 }
 
@@ -447,7 +511,7 @@ int launch_tc_bwd(const Prob& P, const void* Q, const void* K, const void* V, co
     if ((rc = make_tmap_bf16(&tmK, K, P.B, P.L, P.Hkv, P.d, P.ks, 128))) return rc;
     if ((rc = make_tmap_bf16(&tmV, V, P.B, P.L, P.Hkv, P.d, P.vs, 128))) return rc;
     CUtensorMap tmDQ;
-    if ((rc = make_tmap_f32_rows(&tmDQ, acc, P.B, P.L, P.Hq, 64))) return rc;
+    if ((rc = make_tmap_f32_rows(&tmDQ, acc, P.B, P.L, P.Hq, 32, 32))) return rc;
     rowdot_bf16_kernel<<<(unsigned)((rows + 7) / 8), 256, 0, st>>>((const __nv_bfloat16*)O, (const __nv_bfloat16*)dO, Dv, P.B, P.L, P.Hq,
                                                                     P.os[0], P.os[1], P.os[2]);
     if (cudaMemsetAsync(acc, 0, nq * sizeof(float), st) != cudaSuccess) return DMA_ERR_CUDA;
@@ -459,10 +523,14 @@ int launch_tc_bwd(const Prob& P, const void* Q, const void* K, const void* V, co
     bp.ignore_bitmap = (P.flags & DMA_FLAG_IGNORE_BITMAP) ? 1 : 0;
     bp.scale = P.scale; bp.scale_log2 = P.scale * 1.4426950408889634f;
     bp.ks_b = P.ks[0]; bp.ks_l = P.ks[1]; bp.ks_h = P.ks[2]; bp.vs_b = P.vs[0]; bp.vs_l = P.vs[1]; bp.vs_h = P.vs[2];
+#ifdef DMA_PROF
+    const char* prof_env = getenv("DMA_PROF_PTR");
+    bp.prof = prof_env ? (long long*)strtoull(prof_env, nullptr, 10) : nullptr;
+#endif
     const size_t smem = sizeof(SharedStorage) + 1024;
     if (cudaFuncSetAttribute(bwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return DMA_ERR_CUDA;
     bwd_kernel<<<dim3(P.B * P.Hkv, P.Tc), kThreads, smem, st>>>(tmQ, tmK, tmV, tmG, tmDQ, bp);
-    dq_convert_bf16_kernel<<<(unsigned)((nq / 8 + 255) / 256), 256, 0, st>>>(acc, (__nv_bfloat16*)dQ, nq / 8, P.L, P.Hq, P.qs[0], P.qs[1], P.qs[2]);
+    dq_convert_bf16_kernel<<<(unsigned)((nq / 8 + 255) / 256), 256, 0, st>>>(acc, (__nv_bfloat16*)dQ, nq / 8, P.L, P.Hq, P.qs[0], P.qs[1], P.qs[2], P.scale);
     count_launch(3);
     return check_launch();
 }

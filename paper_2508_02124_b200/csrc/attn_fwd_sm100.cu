@@ -401,12 +401,12 @@ int make_tmap_bf16(CUtensorMap* m, const void* base, int B, int L, int H, int d,
     return r == CUDA_SUCCESS ? DMA_OK : DMA_ERR_CUDA;
 }
 
-int make_tmap_f32_rows(CUtensorMap* m, const void* base, int B, int L, int H, int rows) {
+int make_tmap_f32_rows(CUtensorMap* m, const void* base, int B, int L, int H, int rows, int channels) {
     EncodeTiledFn enc = get_encode_tiled();
     if (!enc) return DMA_ERR_CUDA;
     cuuint64_t dims[4] = {128, (cuuint64_t)H, (cuuint64_t)L, (cuuint64_t)B};
     cuuint64_t str[3] = {128 * 4, (cuuint64_t)H * 128 * 4, (cuuint64_t)L * H * 128 * 4};
-    cuuint32_t box[4] = {128, 1, (cuuint32_t)rows, 1};
+    cuuint32_t box[4] = {(cuuint32_t)channels, 1, (cuuint32_t)rows, 1};
     cuuint32_t estr[4] = {1, 1, 1, 1};
     CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, const_cast<void*>(base), dims, str, box, estr,
                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
