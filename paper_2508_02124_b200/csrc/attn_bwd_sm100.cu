@@ -84,7 +84,8 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
            const __grid_constant__ CUtensorMap tmDQ, const BwdParams P) {
     extern __shared__ uint8_t smem_raw[];
     SharedStorage& S = *reinterpret_cast<SharedStorage*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int tid = threadIdx.x, lane = tid & 31;
+    const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);      // warp-uniform to the compiler: role branches stay uniform
     const int b = blockIdx.x / P.Hkv, hk = blockIdx.x % P.Hkv;
     const int kt = blockIdx.y;                         // key tile 0 has the most query tiles: heaviest first
     const int j0 = kt * 128;
@@ -97,11 +98,11 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             mbar_init(&S.qd_empty[s], 1);
         }
         mbar_init(&S.sdp_full, 1);
-        mbar_init(&S.sdp_free, 256);
-        mbar_init(&S.pds_ready, 256);
+        mbar_init(&S.sdp_free, 8);        // one arrival per compute warp (256 serialised arrivals would cost hundreds of cycles)
+        mbar_init(&S.pds_ready, 8);
         mbar_init(&S.pds_free, 1);
         mbar_init(&S.dq_full, 1);
-        mbar_init(&S.dq_free, 128);
+        mbar_init(&S.dq_free, 4);         // one arrival per drain warp
         S.abort_flag = 0;
         S.n_steps = 0;
         fence_barrier_init();
@@ -174,7 +175,8 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             tmem_ld32(tmem + lane_base + cDP + hsel * 32, pr);
             tc_wait_ld();
             tc_fence_before();
-            mbar_arrive(&S.sdp_free);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&S.sdp_free);
 #ifdef DMA_PROF
             const long long tp1 = clock64();
             prof_acc[2] += tp1 - tp0;
@@ -252,7 +254,8 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             fence_proxy_async();
             tc_wait_st();
             tc_fence_before();
-            mbar_arrive(&S.pds_ready);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&S.pds_ready);
 #ifdef DMA_PROF
             prof_acc[4] += clock64() - tp2;
 #endif
@@ -314,7 +317,8 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             tmem_ld32(tmem + lane_base + cDQ + 32, *reinterpret_cast<uint32_t(*)[32]>(&v[32]));
             tc_wait_ld();
             tc_fence_before();
-            mbar_arrive(&S.dq_free);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&S.dq_free);
 #pragma unroll
             for (int hf = 0; hf < 2; ++hf) {
                 PROF_WAIT(1 + hf, if (lane == 0) bulk_wait_read_1(); __syncwarp());
@@ -389,58 +393,72 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&S.qd_full[st]);
             }
-        } else if (warp == 13 && lane == 0) {
+        } else if (warp == 13) {
             // ============================ MMA issuer 1: S^T = K Q^T, dP^T = V dO^T ============================
-            // (two issuing threads: every hand-over between them and the other groups is an explicit mbarrier,
-            //  nothing relies on the order of the two threads' MMAs)
+            // (two issuing warps: every hand-over between them and the other groups is an explicit mbarrier, nothing
+            //  relies on the order of their MMAs. Each walks the schedule as a whole warp with warp-uniform values, so
+            //  that descriptors and counters stay in the uniform datapath; one elected lane issues.)
             constexpr uint32_t id_sdp = idesc_bf16(128, 64, 0, 0);     // K|V (K-major) x Q|dO (K-major)       -> 128 x 64
             const uint64_t dK = smem_desc_sw128(smem_u32(S.k), 16, 1024), dV = smem_desc_sw128(smem_u32(S.v), 16, 1024);
-            bool ok = mbar_wait(&S.kv_full, 0, abort_flag);
+            const uint64_t dQ0 = smem_desc_sw128(smem_u32(S.q[0]), 16, 1024), dG0 = smem_desc_sw128(smem_u32(S.g[0]), 16, 1024);
+            const uint32_t tmem_u = __shfl_sync(0xffffffffu, tmem, 0);
+            const int n_steps_u = __shfl_sync(0xffffffffu, n_steps, 0);
+            bool ok = mbar_wait_warp(&S.kv_full, 0, abort_flag);
             PROF_DECL(2);
-            for (int n = 0; n < n_steps && ok; ++n) {
+            for (int n = 0; n < n_steps_u && ok; ++n) {
                 const int st = n % kStages;
-                PROF_WAIT(0, ok = mbar_wait(&S.qd_full[st], (n / kStages) & 1, abort_flag));
-                if (ok && n > 0) PROF_WAIT(1, ok = mbar_wait(&S.sdp_free, (n - 1) & 1, abort_flag));
+                PROF_WAIT(0, ok = mbar_wait_warp(&S.qd_full[st], (n / kStages) & 1, abort_flag));
+                if (ok && n > 0) PROF_WAIT(1, ok = mbar_wait_warp(&S.sdp_free, (n - 1) & 1, abort_flag));
                 if (!ok) break;
                 tc_fence_after();
-                const uint64_t dQ = smem_desc_sw128(smem_u32(S.q[st]), 16, 1024), dG = smem_desc_sw128(smem_u32(S.g[st]), 16, 1024);
+                const uint64_t dQ = dQ0 + (uint64_t)(st * (kQBytes >> 4)), dG = dG0 + (uint64_t)(st * (kQBytes >> 4));
+                if (elect_one()) {
 #pragma unroll
-                for (int kk = 0; kk < 8; ++kk)
-                    mma_ss(tmem + cS, dK + (uint64_t)(((kk >> 2) * (kKVBytes / 2) + (kk & 3) * 32) >> 4),
-                           dQ + (uint64_t)(((kk >> 2) * (kQBytes / 2) + (kk & 3) * 32) >> 4), id_sdp, kk > 0);
+                    for (int kk = 0; kk < 8; ++kk)
+                        mma_ss(tmem_u + cS, dK + (uint64_t)(((kk >> 2) * (kKVBytes / 2) + (kk & 3) * 32) >> 4),
+                               dQ + (uint64_t)(((kk >> 2) * (kQBytes / 2) + (kk & 3) * 32) >> 4), id_sdp, kk > 0);
 #pragma unroll
-                for (int kk = 0; kk < 8; ++kk)
-                    mma_ss(tmem + cDP, dV + (uint64_t)(((kk >> 2) * (kKVBytes / 2) + (kk & 3) * 32) >> 4),
-                           dG + (uint64_t)(((kk >> 2) * (kQBytes / 2) + (kk & 3) * 32) >> 4), id_sdp, kk > 0);
-                tc_commit(&S.sdp_full);
+                    for (int kk = 0; kk < 8; ++kk)
+                        mma_ss(tmem_u + cDP, dV + (uint64_t)(((kk >> 2) * (kKVBytes / 2) + (kk & 3) * 32) >> 4),
+                               dG + (uint64_t)(((kk >> 2) * (kQBytes / 2) + (kk & 3) * 32) >> 4), id_sdp, kk > 0);
+                    tc_commit(&S.sdp_full);
+                }
+                __syncwarp();
             }
             PROF_END();
-        } else if (warp == 14 && lane == 0) {
+        } else if (warp == 14) {
             // ============================ MMA issuer 2: dV += P^T dO, dK += dS^T Q, dQ^T = K^T dS^T ============================
             constexpr uint32_t id_dkv = idesc_bf16(128, 128, 0, 1);    // P^T|dS^T (TMEM) x dO|Q (MN-major)    -> 128 x 128
             constexpr uint32_t id_dq = idesc_bf16(128, 64, 1, 1);      // K^T (MN-major) x dS^T (MN-major)     -> 128 x 64
             const uint64_t dKt = smem_desc_sw128(smem_u32(S.k), kKVBytes / 2, 1024), dDs = smem_desc_sw128(smem_u32(S.ds), 16, 1024);
+            const uint64_t dGm0 = smem_desc_sw128(smem_u32(S.g[0]), kQBytes / 2, 1024), dQm0 = smem_desc_sw128(smem_u32(S.q[0]), kQBytes / 2, 1024);
+            const uint32_t tmem_u = __shfl_sync(0xffffffffu, tmem, 0);
+            const int n_steps_u = __shfl_sync(0xffffffffu, n_steps, 0);
             bool ok = true;
             PROF_DECL(3);
-            for (int n = 0; n < n_steps && ok; ++n) {
+            for (int n = 0; n < n_steps_u && ok; ++n) {
                 const int st = n % kStages;
-                PROF_WAIT(0, ok = mbar_wait(&S.pds_ready, n & 1, abort_flag));
-                if (ok && n > 0) PROF_WAIT(1, ok = mbar_wait(&S.dq_free, (n - 1) & 1, abort_flag));
+                PROF_WAIT(0, ok = mbar_wait_warp(&S.pds_ready, n & 1, abort_flag));
+                if (ok && n > 0) PROF_WAIT(1, ok = mbar_wait_warp(&S.dq_free, (n - 1) & 1, abort_flag));
                 if (!ok) break;
                 tc_fence_after();
-                const uint64_t dGm = smem_desc_sw128(smem_u32(S.g[st]), kQBytes / 2, 1024), dQm = smem_desc_sw128(smem_u32(S.q[st]), kQBytes / 2, 1024);
+                const uint64_t dGm = dGm0 + (uint64_t)(st * (kQBytes >> 4)), dQm = dQm0 + (uint64_t)(st * (kQBytes >> 4));
+                const uint32_t acc0 = n > 0 ? 1u : 0u;
+                if (elect_one()) {
 #pragma unroll
-                for (int kk = 0; kk < 4; ++kk)         // 64 query rows = 4 k-steps of 16
-                    mma_ts(tmem + cDV, tmem + cP + kk * 8, dGm + (uint64_t)((kk * 2048) >> 4), id_dkv, (n > 0 || kk > 0) ? 1u : 0u);
+                    for (int kk = 0; kk < 4; ++kk)         // 64 query rows = 4 k-steps of 16
+                        mma_ts(tmem_u + cDV, tmem_u + cP + kk * 8, dGm + (uint64_t)((kk * 2048) >> 4), id_dkv, kk > 0 ? 1u : acc0);
 #pragma unroll
-                for (int kk = 0; kk < 4; ++kk)
-                    mma_ts(tmem + cDK, tmem + cDS + kk * 8, dQm + (uint64_t)((kk * 2048) >> 4), id_dkv, (n > 0 || kk > 0) ? 1u : 0u);
-                tc_commit(&S.qd_empty[st]);            // the dQ GEMM reads K and dS^T only: Q / dO of this stage are free here
+                    for (int kk = 0; kk < 4; ++kk)
+                        mma_ts(tmem_u + cDK, tmem_u + cDS + kk * 8, dQm + (uint64_t)((kk * 2048) >> 4), id_dkv, kk > 0 ? 1u : acc0);
+                    tc_commit(&S.qd_empty[st]);            // the dQ GEMM reads K and dS^T only: Q / dO of this stage are free here
 #pragma unroll
-                for (int kk = 0; kk < 8; ++kk)         // 128 keys = 8 k-steps of 16
-                    mma_ss(tmem + cDQ, dKt + (uint64_t)((kk * 2048) >> 4), dDs + (uint64_t)((kk * 2048) >> 4), id_dq, kk > 0);
-                tc_commit(&S.pds_free);
-                tc_commit(&S.dq_full);
+                    for (int kk = 0; kk < 8; ++kk)         // 128 keys = 8 k-steps of 16
+                        mma_ss(tmem_u + cDQ, dKt + (uint64_t)((kk * 2048) >> 4), dDs + (uint64_t)((kk * 2048) >> 4), id_dq, kk > 0);
+                    tc_commit(&S.pds_free);
+                    tc_commit(&S.dq_full);
+                }
+                __syncwarp();
             }
             PROF_END();
         }

@@ -2,17 +2,22 @@
 // accumulators in tensor memory, online softmax in registers, bitmap-driven tile skipping.
 //
 // One CTA owns two consecutive 128-row query tiles of one (batch, head) and walks the union of their active key
-// tiles. Warp roles (12 warps):
-//   warps 0-3 / 4-7  softmax group 0 / 1: thread r owns query row r of its tile (TMEM lane r): reads S, adds the
-//                    bias, applies the validity test j <= i < expiry[j], keeps the running max / sum, writes P (bf16)
-//                    back to tensor memory over S, rescales O when the max has grown, and finally normalises O
+// tiles. Bias and mask are folded into the score GEMM: S_w = Q_w K^T gets a ninth k-step whose operands the stager
+// warps build per (key tile, query tile) - it adds bias / scale, -BIG for keys that expired before the tile's rows
+// and a step function per key that expires inside them - so that the softmax warps read finished scores from tensor
+// memory and touch no shared memory per element. Diagonal tiles, and tiles in which more than 13 keys expire inside
+// the query tile's rows, take the general path with the explicit test j <= i < expiry[j].
+// Warp roles (12 warps):
+//   warps 0-3 / 4-7  softmax group 0 / 1: thread r owns query row r of its tile (TMEM lane r): row max, lazy rescale of
+//                    O, p = 2^(x c - stab), row sum, P (bf16) written back to tensor memory over S, final normalisation
 //   warp 8           producer: builds the tile schedule from the bitmap, then issues the TMA loads of K and V per
-//                    active key tile (inactive tiles are never loaded); warp 10 stages bias / expiry vectors
-//   warp 9           MMA issuer: S_w = Q_w K^T, O_w += P_w V, ping-ponging between the two query tiles so that the
-//                    tensor cores run one tile's GEMMs while the other tile's softmax is in flight
+//                    active key tile (inactive tiles are never loaded); K and V stages are released separately
+//   warp 9           MMA issuer (whole warp, warp-uniform values, one elected lane issues): S_w = Q_w K^T (+ ninth
+//                    k-step), O_w += P_w V, ping-ponging between the two query tiles
+//   warps 10, 11     stagers for query tile 0 / 1: ninth k-step operands, expiry vector, fast / general flag
 // Tensor memory (512 columns): S0 [0,128) S1 [128,256) O0 [256,384) O1 [384,512); P_w aliases columns [0,64) of S_w.
-// The log-sum-exp replaces Alg. 1's (l, m) pair. Scores are kept in the log2 domain: x = log2(e) (s scale + bias).
-#include <type_traits>
+// The log-sum-exp replaces Alg. 1's (l, m) pair.
+#include <cstdlib>
 
 #include "common.cuh"
 #include "sm100_ptx.cuh"
@@ -26,14 +31,23 @@ constexpr int kStages = 2;
 constexpr int kMaxSched = 1024;               // key tiles per CTA schedule (L <= 131072)
 constexpr int kThreads = 384;
 constexpr uint32_t kTileBytes = 128 * 128 * 2;   // one 128 x 128 bf16 tile = two 16 KB swizzled half tiles
+constexpr int kMaskSlots = 13;                 // keys expiring inside a tile's rows that the ninth k-step can mask
+constexpr float kSmallStab = 1048576.0f;        // 2^20: below it the stabiliser is fl(m_ref c), see the softmax groups
 constexpr float kRescaleThreshold = 8.0f;     // log2 units: P stays below 2^8, O is rescaled only on larger jumps
 
 struct SharedStorage {
     alignas(1024) uint8_t q[2][kTileBytes];
     alignas(1024) uint8_t k[kStages][kTileBytes];
     alignas(1024) uint8_t v[kStages][kTileBytes];
-    alignas(16) float bias[kStages][128];     // log2(e) * bias of the staged key tile
+    // Ninth k-step of S = Q K^T, per query tile: A rows [1, 1, 1, t_0(r) .. t_12(r)], B rows [b_hi, b_mid, b_lo, -BIG [j = j_0] ..],
+    // unswizzled K-major core matrices (row r, element e at (r/8) 256 + (e/8) 128 + (r%8) 16 + (e%8) 2 bytes). The
+    // product adds bias / scale to the score, -BIG for keys that expired before the tile's rows, and -BIG from row
+    // expiry[j_k] on for the up to 13 keys j_k that expire inside the tile's rows (t_k(r) = 1 from that row on).
+    alignas(128) uint8_t aext[2][4096];
+    alignas(128) uint8_t bext[2][4096];
     alignas(16) int len[kStages][128];        // expiry[j] (0 beyond L): row i keeps key j iff j <= i < expiry[j]
+    int thr[2][16];                           // stager scratch: row thresholds of the keys that expire inside the tile
+    uint32_t fast[kStages][2];                // 1: the extra k-step carries the whole mask of this (key tile, query tile)
     uint32_t sched[kMaxSched];                // key tile | use by tile 0 << 30 | use by tile 1 << 31
     uint64_t q_full, k_full[kStages], v_full[kStages], k_empty[kStages], v_empty[kStages];
     uint64_t s_full[2], p_ready[2], o_done[2];
@@ -51,8 +65,23 @@ struct FwdParams {
     int32_t* status;
     int B, Hq, G, L, Tr, Tc, Wd, ignore_bitmap;
     float scale_log2;                          // softmax scale * log2(e)
+    float inv_scale;                           // 1 / softmax scale
+    float rescale_gap;                         // growth of a row max (score units) beyond which O is rescaled
     int64_t os_b, os_l, os_h;
+#ifdef DMA_PROF
+    long long* prof;                           // role timing (development builds only): cycles per phase of CTA (0, 0)
+#endif
 };
+
+#ifdef DMA_PROF
+#define TRACE(it, ev) do { if (P.prof && blockIdx.x == 0 && blockIdx.y == 0 && (it) >= 60 && (it) < 64) P.prof[64 + ((it) - 60) * 16 + (ev)] = clock64(); } while (0)
+#define PROF_T(var) const long long var = clock64()
+#define PROF_ADD(slot, expr) do { if (prof_on) prof_acc[slot] += (expr); } while (0)
+#else
+#define TRACE(it, ev)
+#define PROF_T(var)
+#define PROF_ADD(slot, expr)
+#endif
 
 __device__ __forceinline__ uint32_t use_bit(uint32_t entry, int w) { return (entry >> (30 + w)) & 1u; }
 
@@ -61,7 +90,8 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
            const __grid_constant__ CUtensorMap tmV, const FwdParams P) {
     extern __shared__ uint8_t smem_raw[];
     SharedStorage& S = *reinterpret_cast<SharedStorage*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int tid = threadIdx.x, lane = tid & 31;
+    const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);      // warp-uniform to the compiler: role branches stay uniform
     const int bh = blockIdx.x, b = bh / P.Hq, h = bh % P.Hq, hk = h / P.G;
     const int npairs = (P.Tr + 1) / 2;
     const int pair = npairs - 1 - (int)blockIdx.y;          // heaviest query tiles first
@@ -72,14 +102,14 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
     if (tid == 0) {
         mbar_init(&S.q_full, 1);
         for (int s = 0; s < kStages; ++s) {
-            mbar_init(&S.k_full[s], 2);      // TMA bytes of K + the staged bias / expiry vectors
+            mbar_init(&S.k_full[s], 3);      // TMA bytes of K + the two stager warps
             mbar_init(&S.v_full[s], 1);
             mbar_init(&S.k_empty[s], 1);
             mbar_init(&S.v_empty[s], 1);
         }
         for (int w = 0; w < 2; ++w) {
             mbar_init(&S.s_full[w], 1);
-            mbar_init(&S.p_ready[w], 128);
+            mbar_init(&S.p_ready[w], 4);         // one arrival per softmax warp
             mbar_init(&S.o_done[w], 1);
         }
         S.abort_flag = 0;
@@ -116,7 +146,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
 
     if (warp < 8) {
         // =========================================== softmax groups ===========================================
-        setmaxnreg_inc<216>();
+        setmaxnreg_inc<208>();
         const int w = warp >> 2;
         const int r = tid & 127;
         const int qt = w ? qt1 : qt0;
@@ -124,16 +154,28 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
         const uint32_t tS = tmem + lane_base + w * 128;
         const uint32_t tO = tmem + lane_base + 256 + w * 128;
-        float m_ref = -INFINITY, l = 0.0f;
+        float m_ref = -INFINITY, r_ref = 0.0f, l = 0.0f;
         int n_used = 0;
         bool ok = true;
+#ifdef DMA_PROF
+        const bool prof_on = P.prof && blockIdx.x == 0 && blockIdx.y == 0 && lane == 0;
+        long long prof_acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+        const long long prof_start = clock64();
+#endif
         for (int it = 0; it < n_iters && ok; ++it) {
             const uint32_t entry = S.sched[it];
             if (!use_bit(entry, w)) continue;
+            PROF_T(t_a);
             const int st = it % kStages, j0 = (int)(entry & 0xFFFFF) * 128;
             ok = mbar_wait_warp(&S.s_full[w], n_used & 1, abort_flag) && mbar_wait_warp(&S.k_full[st], (it / kStages) & 1, abort_flag);
             if (!ok) break;
             tc_fence_after();
+            PROF_T(t_b);
+            PROF_ADD(0, t_b - t_a);
+            if ((warp & 3) == 0 && lane == 0) TRACE(it, w * 4 + 0);
+            // The accumulator holds q.k + bias / scale (+ -BIG where the ninth k-step masks). On the fast path that
+            // is the whole masked score; otherwise (diagonal tile, or more than 13 keys expiring inside the tile's
+            // rows) the validity test j <= i < expiry[j] is applied here. x = log2e * scale * score, -inf if masked.
             float x[128];
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
@@ -143,38 +185,51 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
 #pragma unroll
                 for (int u = 0; u < 32; ++u) x[c * 32 + u] = __uint_as_float(raw[u]);
             }
-            // x = log2e (s scale + bias) where row i keeps key j (j <= i < expiry[j]), else -inf. Off the diagonal
-            // j <= i always holds and one compare against the staged expiry decides; the two cases are separate
-            // loops so that neither pays for the other's test. Four independent max chains.
+            PROF_T(t_c);
+            PROF_ADD(1, t_c - t_b);
+            if ((warp & 3) == 0 && lane == 0) TRACE(it, w * 4 + 1);
             float mxa[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-            auto score_pass = [&](auto diag) {
-                constexpr bool kDiag = decltype(diag)::value;
+            if (S.fast[st][w]) {
+                PROF_ADD(6, 1);
 #pragma unroll
                 for (int c = 0; c < 128; c += 4) {
-                    const float4 bb = *reinterpret_cast<const float4*>(&S.bias[st][c]);
+                    mxa[(c >> 2) & 1] = max3(mxa[(c >> 2) & 1], x[c], x[c + 1]);
+                    mxa[2 + ((c >> 2) & 1)] = max3(mxa[2 + ((c >> 2) & 1)], x[c + 2], x[c + 3]);
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u) mxa[u] = mxa[u] < -1e20f ? -INFINITY : mxa[u];
+            } else {
+#pragma unroll
+                for (int c = 0; c < 128; c += 4) {
                     const int4 ee = *reinterpret_cast<const int4*>(&S.len[st][c]);
-                    const float bv[4] = {bb.x, bb.y, bb.z, bb.w};
                     const int ev[4] = {ee.x, ee.y, ee.z, ee.w};
 #pragma unroll
                     for (int u = 0; u < 4; ++u) {
-                        const float xv = fmaf(x[c + u], P.scale_log2, bv[u]);
-                        const bool valid = kDiag ? (j0 + c + u <= i && i < ev[u]) : (i < ev[u]);
-                        x[c + u] = valid ? xv : -INFINITY;
+                        const bool valid = j0 + c + u <= i && i < ev[u];
+                        x[c + u] = valid ? x[c + u] : -INFINITY;
                         mxa[u] = fmaxf(mxa[u], x[c + u]);
                     }
                 }
-            };
-            if (j0 + 127 > qt * 128) score_pass(std::true_type{}); else score_pass(std::false_type{});
+            }
+            // The running max m_ref stays in score units and the exponent is formed as (x - m_ref) * c: the difference
+            // is exact for the entries that matter, whatever the magnitude of the bias.
             const float mx = fmaxf(fmaxf(mxa[0], mxa[1]), fmaxf(mxa[2], mxa[3]));
             const float m_new = fmaxf(m_ref, mx);
+            auto stab_resid = [&](float m) {           // m c - stab(m); 0 for m = -inf
+                const float mm = (m == -INFINITY) ? 0.0f : m;
+                const float Mm = mm * P.scale_log2;
+                return fabsf(Mm) < kSmallStab ? fmaf(mm, P.scale_log2, -Mm) : 0.0f;
+            };
             if (n_used == 0) {
                 m_ref = m_new;
-            } else if (__any_sync(0xffffffffu, m_new > m_ref + kRescaleThreshold)) {
-                // O_w *= 2^(m_ref - m_new): the previous P V product must have landed first
+                r_ref = stab_resid(m_ref);
+            } else if (__any_sync(0xffffffffu, m_new > m_ref + P.rescale_gap)) {
+                // O_w *= 2^(stab(m_ref) - stab(m_new)): the previous P V product must have landed first
                 ok = mbar_wait_warp(&S.o_done[w], (n_used - 1) & 1, abort_flag);
                 if (!ok) break;
                 tc_fence_after();
-                const float f = (m_new == -INFINITY) ? 1.0f : ex2(m_ref - m_new);
+                const float r_new = stab_resid(m_new);
+                const float f = (m_new == -INFINITY) ? 1.0f : (m_ref == -INFINITY) ? 0.0f : ex2(fmaf(m_ref - m_new, P.scale_log2, r_new - r_ref));
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
                     uint32_t o[32];
@@ -187,26 +242,65 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                 tc_wait_st();
                 l *= f;
                 m_ref = m_new;
+                r_ref = r_new;
             }
+            // p = 2^(x c - stab(m_ref)). The stabiliser is a function of the row's m_ref alone: fl(m_ref c) while that
+            // is below 2^20 in magnitude (then x c - stab is one FMA per element and fl() is off by < 0.07), else the
+            // exact product m_ref c, reached by taking the exact difference x - m_ref first (bias magnitudes up to the
+            // fp32 range stay safe). r_ref = m_ref c - stab(m_ref) travels with m_ref.
             const float m_use = (m_ref == -INFINITY) ? 0.0f : m_ref;
+            const float M = m_use * P.scale_log2, nM = -M;
+            const float resid = r_ref;
+            const bool small = __all_sync(0xffffffffu, fabsf(M) < kSmallStab);
+            PROF_T(t_d);
+            PROF_ADD(2, t_d - t_c + (long long)(m_use == 1.2345f));
+            if ((warp & 3) == 0 && lane == 0) TRACE(it, w * 4 + 2);
             float sa[4] = {0.f, 0.f, 0.f, 0.f};
+            if (small) {
 #pragma unroll
-            for (int half = 0; half < 2; ++half) {
-                uint32_t pk[32];
+                for (int half = 0; half < 2; ++half) {
+                    uint32_t pk[32];
 #pragma unroll
-                for (int c = 0; c < 64; c += 2) {
-                    const float p0 = ex2(x[half * 64 + c] - m_use), p1 = ex2(x[half * 64 + c + 1] - m_use);
-                    sa[(c >> 1) & 3] += p0 + p1;
-                    pk[c >> 1] = pack_bf16(p0, p1);
+                    for (int c = 0; c < 64; c += 2) {
+                        const float p0 = ex2(fmaf(x[half * 64 + c], P.scale_log2, nM)), p1 = ex2(fmaf(x[half * 64 + c + 1], P.scale_log2, nM));
+                        sa[(c >> 1) & 3] += p0 + p1;
+                        pk[c >> 1] = pack_bf16(p0, p1);
+                    }
+                    tmem_st32(tS + half * 32, pk);
                 }
-                tmem_st32(tS + half * 32, pk);
+            } else {
+#pragma unroll
+                for (int half = 0; half < 2; ++half) {
+                    uint32_t pk[32];
+#pragma unroll
+                    for (int c = 0; c < 64; c += 2) {
+                        const float p0 = ex2(fmaf(x[half * 64 + c] - m_use, P.scale_log2, resid));
+                        const float p1 = ex2(fmaf(x[half * 64 + c + 1] - m_use, P.scale_log2, resid));
+                        sa[(c >> 1) & 3] += p0 + p1;
+                        pk[c >> 1] = pack_bf16(p0, p1);
+                    }
+                    tmem_st32(tS + half * 32, pk);
+                }
             }
             l += (sa[0] + sa[1]) + (sa[2] + sa[3]);
             tc_wait_st();
             tc_fence_before();
-            mbar_arrive(&S.p_ready[w]);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&S.p_ready[w]);      // one arrival per warp: 128 serialised arrivals cost ~400 cycles
             ++n_used;
+            PROF_T(t_e);
+            PROF_ADD(3, t_e - t_d);
+            if ((warp & 3) == 0 && lane == 0) TRACE(it, w * 4 + 3);
+            PROF_ADD(4, 1);
         }
+#ifdef DMA_PROF
+        if (prof_on) {
+            prof_acc[5] = clock64() - prof_start;
+            if ((warp & 3) == 0) for (int k = 0; k < 8; ++k) P.prof[w * 8 + k] = prof_acc[k];
+            P.prof[32 + warp * 2] = prof_acc[0];
+            P.prof[33 + warp * 2] = prof_acc[5];
+        }
+#endif
         // epilogue: O_w / l -> bf16 rows, log-sum-exp in natural log
         const bool exists = w == 0 || has1;
         if (ok && exists && n_used > 0) ok = mbar_wait_warp(&S.o_done[w], (n_used - 1) & 1, abort_flag);
@@ -236,10 +330,10 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                     }
                 }
             }
-            if (i < P.L) P.lse[(size_t)bh * P.L + i] = l > 0.0f ? 0.6931471805599453f * (m_ref + log2f(l)) : -INFINITY;
+            if (i < P.L) P.lse[(size_t)bh * P.L + i] = l > 0.0f ? 0.6931471805599453f * ((m_ref * P.scale_log2 - r_ref) + log2f(l)) : -INFINITY;
         }
     } else {
-        setmaxnreg_dec<72>();   // 4 warps x 96 registers released = 8 warps x 48 acquired below
+        setmaxnreg_dec<88>();   // 4 warps x 80 registers released = 8 warps x 40 acquired above
         if (warp == 8) {
             // =========================================== producer ===========================================
             if (lane == 0) {
@@ -272,9 +366,14 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             for (int it = max(0, n_iters - kStages); it < n_iters && ok; ++it)
                 ok = mbar_wait_warp(&S.k_empty[it % kStages], (it / kStages) & 1, abort_flag) &&
                      mbar_wait_warp(&S.v_empty[it % kStages], (it / kStages) & 1, abort_flag);
-        } else if (warp == 10) {
-            // =========================================== stager ===========================================
-            // bias (log2 domain) and expiry of each key tile -> shared memory; the global loads run one tile ahead
+        } else if (warp >= 10) {
+            // =========================================== stagers ===========================================
+            // Warp 10 + w serves query tile w: per key tile it builds the ninth k-step operands described at
+            // SharedStorage (warp 10 also stages the expiry vector for the general softmax path). The global loads run
+            // one tile ahead and the rows are formed in registers before the wait for the blocks to be free, so that
+            // only the stores are left between the previous S product and the next one.
+            const int w = warp - 10;
+            const int i0 = (w ? qt1 : qt0) * 128;
             auto fetch = [&](int it, float (&bv)[4], int (&ev)[4]) {
                 const int j0 = (int)(S.sched[it] & 0xFFFFF) * 128;
 #pragma unroll
@@ -284,83 +383,187 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                     ev[t] = j < P.L ? P.expiry[(size_t)bh * P.L + j] : 0;
                 }
             };
+            constexpr uint32_t kOne = 0x3F80u, kNegBig = 0xF14Au;     // bf16 1.0 and about -1e30
             float bv[4] = {0.f, 0.f, 0.f, 0.f};
             int ev[4] = {0, 0, 0, 0};
             if (n_iters > 0) fetch(0, bv, ev);
             bool ok = true;
             for (int it = 0; it < n_iters && ok; ++it) {
                 const int st = it % kStages;
+                const uint32_t entry = S.sched[it];
+                const bool use = use_bit(entry, w);
                 float bn[4] = {0.f, 0.f, 0.f, 0.f};
                 int en[4] = {0, 0, 0, 0};
                 if (it + 1 < n_iters) fetch(it + 1, bn, en);
-                // the vectors of this stage were last read by the softmax groups before they released P (hence before P V)
+                uint32_t b0[4], b1[4], aw[4][7];
+                int hot[4];
+                bool fast = false;
+                if (use) {
+                    const bool diag = (int)(entry & 0xFFFFF) == (w ? qt1 : qt0);
+                    uint32_t bal[4];
+                    bool mixed[4];
+#pragma unroll
+                    for (int t = 0; t < 4; ++t) {
+                        mixed[t] = ev[t] > i0 && ev[t] < i0 + 128;
+                        bal[t] = __ballot_sync(0xffffffffu, mixed[t]);
+                    }
+                    const int cnt = __popc(bal[0]) + __popc(bal[1]) + __popc(bal[2]) + __popc(bal[3]);
+                    fast = !diag && cnt <= kMaskSlots;
+                    if (lane < kMaskSlots) S.thr[w][lane] = 1 << 20;
+                    __syncwarp();
+                    int before = 0;
+#pragma unroll
+                    for (int t = 0; t < 4; ++t) {
+                        const int slot = before + __popc(bal[t] & ((1u << lane) - 1));
+                        before += __popc(bal[t]);
+                        hot[t] = (fast && mixed[t]) ? 3 + slot : -1;          // element that holds this key's -BIG
+                        if (hot[t] >= 0) S.thr[w][slot] = ev[t] - i0;
+                    }
+                    __syncwarp();
+                    // B rows (keys): bias / scale as three bf16 terms (24 significant bits, as many as the fp32 bias
+                    // has), or -BIG for a key that is gone for the whole tile
+#pragma unroll
+                    for (int t = 0; t < 4; ++t) {
+                        const float bs = bv[t] * P.inv_scale;
+                        const __nv_bfloat16 hi = __float2bfloat16_rn(bs);
+                        const float r1 = bs - __bfloat162float(hi);
+                        const __nv_bfloat16 mid = __float2bfloat16_rn(r1);
+                        const __nv_bfloat16 lo = __float2bfloat16_rn(r1 - __bfloat162float(mid));
+                        const bool dead = ev[t] <= i0;
+                        b0[t] = dead ? kNegBig : ((uint32_t)__bfloat16_as_ushort(hi) | ((uint32_t)__bfloat16_as_ushort(mid) << 16));
+                        b1[t] = (dead ? 0u : (uint32_t)__bfloat16_as_ushort(lo)) | (hot[t] == 3 ? (kNegBig << 16) : 0u);
+                    }
+                    // A rows (queries): ones for the bias terms, then one step function per expiring key
+                    int th[kMaskSlots];
+#pragma unroll
+                    for (int k = 0; k < kMaskSlots; ++k) th[k] = S.thr[w][k];
+#pragma unroll
+                    for (int t = 0; t < 4; ++t) {
+                        const int r = lane + 32 * t;
+                        aw[t][0] = kOne | (r >= th[0] ? (kOne << 16) : 0u);
+#pragma unroll
+                        for (int m = 2; m < 8; ++m)
+                            aw[t][m - 1] = (r >= th[2 * m - 3] ? kOne : 0u) | (r >= th[2 * m - 2] ? (kOne << 16) : 0u);
+                    }
+                }
+                // fast[st] / len[st] were last read by the softmax groups before they released P of tile it - kStages
+                // (hence before its P V); the operand blocks were last read by the S products of tile it - 1
                 if (it >= kStages) ok = mbar_wait_warp(&S.v_empty[st], ((it / kStages) - 1) & 1, abort_flag);
+                if (ok && it >= 1) ok = mbar_wait_warp(&S.k_empty[(it - 1) % kStages], ((it - 1) / kStages) & 1, abort_flag);
                 if (!ok) break;
+                if (w == 0) {
+#pragma unroll
+                    for (int t = 0; t < 4; ++t) S.len[st][lane + 32 * t] = ev[t];
+                }
+                if (use) {
+#pragma unroll
+                    for (int t = 0; t < 4; ++t) {
+                        const int c = lane + 32 * t;
+                        uint32_t wd[8];
+                        wd[0] = b0[t];
+                        wd[1] = b1[t];
+#pragma unroll
+                        for (int m = 2; m < 8; ++m) wd[m] = (hot[t] >> 1) == m ? (kNegBig << ((hot[t] & 1) * 16)) : 0u;
+                        uint8_t* brow = S.bext[w] + (c >> 3) * 256 + (c & 7) * 16;
+                        *reinterpret_cast<uint4*>(brow) = make_uint4(wd[0], wd[1], wd[2], wd[3]);
+                        *reinterpret_cast<uint4*>(brow + 128) = make_uint4(wd[4], wd[5], wd[6], wd[7]);
+                        uint8_t* arow = S.aext[w] + (c >> 3) * 256 + (c & 7) * 16;
+                        *reinterpret_cast<uint4*>(arow) = make_uint4(kOne | (kOne << 16), aw[t][0], aw[t][1], aw[t][2]);
+                        *reinterpret_cast<uint4*>(arow + 128) = make_uint4(aw[t][3], aw[t][4], aw[t][5], aw[t][6]);
+                    }
+                    if (lane == 0) S.fast[st][w] = fast ? 1u : 0u;
+                }
 #pragma unroll
                 for (int t = 0; t < 4; ++t) {
-                    S.bias[st][lane + 32 * t] = bv[t] * 1.4426950408889634f;
-                    S.len[st][lane + 32 * t] = ev[t];
                     bv[t] = bn[t];
                     ev[t] = en[t];
                 }
+                fence_proxy_async();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&S.k_full[st]);
             }
-        } else if (warp == 9 && lane == 0) {
+        } else if (warp == 9) {
             // =========================================== MMA issuer ===========================================
+            // The whole warp walks the schedule with warp-uniform values (descriptors, stage and tile indices stay in
+            // the uniform datapath); one elected lane issues the tcgen05 instructions.
             constexpr uint32_t idesc_s = idesc_bf16(128, 128, 0, 0);     // Q (K-major) x K (K-major)
             constexpr uint32_t idesc_pv = idesc_bf16(128, 128, 0, 1);    // P (TMEM)    x V (MN-major)
+            // operand descriptors are formed once; a stage, query tile or k-step only moves the 16-byte address field
+            const uint64_t dQ0 = smem_desc_sw128(smem_u32(S.q[0]), 16, 1024), dK0 = smem_desc_sw128(smem_u32(S.k[0]), 16, 1024);
+            const uint64_t dV0 = smem_desc_sw128(smem_u32(S.v[0]), kTileBytes / 2, 1024);
+            const uint64_t dA0 = smem_desc_plain(smem_u32(S.aext[0]), 128, 256), dB0 = smem_desc_plain(smem_u32(S.bext[0]), 128, 256);
+            const uint32_t tmem_u = __shfl_sync(0xffffffffu, tmem, 0);
+            const int n_iters_u = __shfl_sync(0xffffffffu, n_iters, 0);
             auto issue_s = [&](int w, int st) {
+                const uint64_t dq = dQ0 + (uint64_t)(w * (kTileBytes >> 4)), dk = dK0 + (uint64_t)(st * (kTileBytes >> 4));
+                const uint32_t d_tmem = tmem_u + w * 128;
+                if (elect_one()) {
 #pragma unroll
-                for (int kk = 0; kk < 8; ++kk) {
-                    const uint32_t off = (kk >> 2) * (kTileBytes / 2) + (kk & 3) * 32;
-                    mma_ss(tmem + w * 128, smem_desc_sw128(smem_u32(&S.q[w][off]), 16, 1024),
-                           smem_desc_sw128(smem_u32(&S.k[st][off]), 16, 1024), idesc_s, kk > 0);
+                    for (int kk = 0; kk < 8; ++kk) {
+                        const uint32_t off = ((kk >> 2) * (kTileBytes / 2) + (kk & 3) * 32) >> 4;
+                        mma_ss(d_tmem, dq + off, dk + off, idesc_s, kk > 0);
+                    }
+                    mma_ss(d_tmem, dA0 + (uint64_t)(w * (4096 >> 4)), dB0 + (uint64_t)(w * (4096 >> 4)), idesc_s, 1u);
+                    tc_commit(&S.s_full[w]);
                 }
-                tc_commit(&S.s_full[w]);
+                __syncwarp();
             };
             int n_p[2] = {0, 0};
-            bool ok = mbar_wait(&S.q_full, 0, abort_flag);
-            if (ok && n_iters > 0) {
-                ok = mbar_wait(&S.k_full[0], 0, abort_flag);
+            bool ok = mbar_wait_warp(&S.q_full, 0, abort_flag);
+            if (ok && n_iters_u > 0) {
+                ok = mbar_wait_warp(&S.k_full[0], 0, abort_flag);
                 if (ok) {
                     tc_fence_after();
+                    const uint32_t e0 = __shfl_sync(0xffffffffu, S.sched[0], 0);
+#pragma unroll
                     for (int w = 0; w < 2; ++w)
-                        if (use_bit(S.sched[0], w)) issue_s(w, 0);
-                    tc_commit(&S.k_empty[0]);
+                        if (use_bit(e0, w)) issue_s(w, 0);
+                    if (elect_one()) tc_commit(&S.k_empty[0]);
+                    __syncwarp();
                 }
             }
-            for (int it = 0; it < n_iters && ok; ++it) {
+            for (int it = 0; it < n_iters_u && ok; ++it) {
                 const int st = it % kStages, nst = (it + 1) % kStages;
-                const uint32_t entry = S.sched[it], next = it + 1 < n_iters ? S.sched[it + 1] : 0u;
-                ok = mbar_wait(&S.v_full[st], (it / kStages) & 1, abort_flag);
+                const uint32_t entry = __shfl_sync(0xffffffffu, S.sched[it], 0);
+                const uint32_t next = it + 1 < n_iters_u ? __shfl_sync(0xffffffffu, S.sched[it + 1], 0) : 0u;
+                ok = mbar_wait_warp(&S.v_full[st], (it / kStages) & 1, abort_flag);
                 bool k_ready = false;
-                for (int w = 0; w < 2 && ok; ++w) {
-                    if (use_bit(entry, w)) {
-                        ok = mbar_wait(&S.p_ready[w], n_p[w] & 1, abort_flag);
-                        if (!ok) break;
-                        tc_fence_after();
 #pragma unroll
-                        for (int kk = 0; kk < 8; ++kk)
-                            mma_ts(tmem + 256 + w * 128, tmem + w * 128 + kk * 8,
-                                   smem_desc_sw128(smem_u32(&S.v[st][kk * 2048]), kTileBytes / 2, 1024), idesc_pv,
-                                   (n_p[w] > 0 || kk > 0) ? 1u : 0u);
-                        tc_commit(&S.o_done[w]);
-                        ++n_p[w];
-                    }
-                    if (use_bit(next, w)) {
-                        if (!k_ready) {
-                            ok = mbar_wait(&S.k_full[nst], ((it + 1) / kStages) & 1, abort_flag);
-                            if (!ok) break;
+                for (int w = 0; w < 2; ++w) {          // unrolled: n_p[] stays in registers
+                    if (ok && use_bit(entry, w)) {
+                        ok = mbar_wait_warp(&S.p_ready[w], n_p[w] & 1, abort_flag);
+                        if (lane == 0) TRACE(it, 8 + w * 2);
+                        if (ok) {
                             tc_fence_after();
+                            const uint64_t dv = dV0 + (uint64_t)(st * (kTileBytes >> 4));
+                            const uint32_t d_tmem = tmem_u + 256 + w * 128, a_tmem = tmem_u + w * 128;
+                            const uint32_t acc0 = n_p[w] > 0 ? 1u : 0u;
+                            if (elect_one()) {
+#pragma unroll
+                                for (int kk = 0; kk < 8; ++kk)
+                                    mma_ts(d_tmem, a_tmem + kk * 8, dv + (uint64_t)((kk * 2048) >> 4), idesc_pv, kk > 0 ? 1u : acc0);
+                                tc_commit(&S.o_done[w]);
+                            }
+                            __syncwarp();
+                            ++n_p[w];
+                        }
+                    }
+                    if (ok && use_bit(next, w)) {
+                        if (!k_ready) {
+                            ok = mbar_wait_warp(&S.k_full[nst], ((it + 1) / kStages) & 1, abort_flag);
+                            if (ok) tc_fence_after();
                             k_ready = true;
                         }
-                        issue_s(w, nst);
+                        if (ok) issue_s(w, nst);
                     }
+                    if (lane == 0) TRACE(it, 9 + w * 2);
                 }
                 if (ok) {
-                    tc_commit(&S.v_empty[st]);
-                    if (it + 1 < n_iters) tc_commit(&S.k_empty[nst]);
+                    if (elect_one()) {
+                        tc_commit(&S.v_empty[st]);
+                        if (it + 1 < n_iters_u) tc_commit(&S.k_empty[nst]);
+                    }
+                    __syncwarp();
                 }
             }
         }
@@ -430,7 +633,13 @@ int launch_tc_fwd(const Prob& P, const void* Q, const void* K, const void* V, co
     fp.B = P.B; fp.Hq = P.Hq; fp.G = P.G; fp.L = P.L; fp.Tr = P.Tr; fp.Tc = P.Tc; fp.Wd = P.Wd;
     fp.ignore_bitmap = (P.flags & DMA_FLAG_IGNORE_BITMAP) ? 1 : 0;
     fp.scale_log2 = P.scale * 1.4426950408889634f;
+    fp.inv_scale = 1.0f / P.scale;
+    fp.rescale_gap = kRescaleThreshold / fp.scale_log2;
     fp.os_b = P.os[0]; fp.os_l = P.os[1]; fp.os_h = P.os[2];
+#ifdef DMA_PROF
+    const char* prof_env = getenv("DMA_PROF_PTR");
+    fp.prof = prof_env ? (long long*)strtoull(prof_env, nullptr, 10) : nullptr;
+#endif
     const size_t smem = sizeof(SharedStorage) + 1024;
     if (cudaFuncSetAttribute(fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return DMA_ERR_CUDA;
     dim3 grid(P.B * P.Hq, (P.Tr + 1) / 2);

@@ -245,6 +245,13 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr, uint32_t lbo
     return (uint64_t)((saddr & 0x3FFFF) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) | ((uint64_t)(sbo_bytes >> 4) << 32) |
            (1ull << 46) | (2ull << 61);
 }
+// The same descriptor without swizzle (layout type 0): 8-row x 16-byte core matrices; for a K-major operand the leading
+// byte offset is the distance between the core matrices of one 8-row group along K, the stride byte offset the
+// distance between 8-row groups.
+__device__ __forceinline__ uint64_t smem_desc_plain(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+    return (uint64_t)((saddr & 0x3FFFF) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) | ((uint64_t)(sbo_bytes >> 4) << 32) |
+           (1ull << 46);
+}
 // Instruction descriptor for kind::f16 with bf16 inputs and fp32 accumulation.
 //   bits 4-5 D format (1 = f32), 7-9 A format (1 = bf16), 10-12 B format, 15 A major (1 = MN), 16 B major,
 //   17-22 N >> 3, 24-28 M >> 4
