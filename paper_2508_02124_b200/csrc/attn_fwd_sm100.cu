@@ -50,7 +50,7 @@ struct SharedStorage {
     uint32_t fast[kStages][2];                // 1: the extra k-step carries the whole mask of this (key tile, query tile)
     uint32_t sched[kMaxSched];                // key tile | use by tile 0 << 30 | use by tile 1 << 31
     uint64_t q_full, k_full[kStages], v_full[kStages], k_empty[kStages], v_empty[kStages];
-    uint64_t s_full[2], p_ready[2], o_done[2];
+    uint64_t s_full[2], p_half[2], p_ready[2], o_done[2];
     uint32_t tmem_base;
     int n_iters;
     int abort_flag;
@@ -109,7 +109,8 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
         }
         for (int w = 0; w < 2; ++w) {
             mbar_init(&S.s_full[w], 1);
-            mbar_init(&S.p_ready[w], 4);         // one arrival per softmax warp
+            mbar_init(&S.p_half[w], 4);          // one arrival per softmax warp
+            mbar_init(&S.p_ready[w], 4);
             mbar_init(&S.o_done[w], 1);
         }
         S.abort_flag = 0;
@@ -167,7 +168,11 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             if (!use_bit(entry, w)) continue;
             PROF_T(t_a);
             const int st = it % kStages, j0 = (int)(entry & 0xFFFFF) * 128;
-            ok = mbar_wait_warp(&S.s_full[w], n_used & 1, abort_flag) && mbar_wait_warp(&S.k_full[st], (it / kStages) & 1, abort_flag);
+            // the stagers' flag is there long before the S product: read it while waiting for S
+            ok = mbar_wait_warp(&S.k_full[st], (it / kStages) & 1, abort_flag);
+            if (!ok) break;
+            const bool fast_tile = S.fast[st][w] != 0;
+            ok = mbar_wait_warp(&S.s_full[w], n_used & 1, abort_flag);
             if (!ok) break;
             tc_fence_after();
             PROF_T(t_b);
@@ -177,19 +182,19 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             // is the whole masked score; otherwise (diagonal tile, or more than 13 keys expiring inside the tile's
             // rows) the validity test j <= i < expiry[j] is applied here. x = log2e * scale * score, -inf if masked.
             float x[128];
+            {
+                uint32_t raw[128];                 // the four loads are in flight together, one wait
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                uint32_t raw[32];
-                tmem_ld32(tS + c * 32, raw);
+                for (int c = 0; c < 4; ++c) tmem_ld32p(tS + c * 32, &raw[c * 32]);
                 tc_wait_ld();
 #pragma unroll
-                for (int u = 0; u < 32; ++u) x[c * 32 + u] = __uint_as_float(raw[u]);
+                for (int u = 0; u < 128; ++u) x[u] = __uint_as_float(raw[u]);
             }
             PROF_T(t_c);
             PROF_ADD(1, t_c - t_b);
             if ((warp & 3) == 0 && lane == 0) TRACE(it, w * 4 + 1);
             float mxa[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-            if (S.fast[st][w]) {
+            if (fast_tile) {
                 PROF_ADD(6, 1);
 #pragma unroll
                 for (int c = 0; c < 128; c += 4) {
@@ -267,6 +272,12 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                         pk[c >> 1] = pack_bf16(p0, p1);
                     }
                     tmem_st32(tS + half * 32, pk);
+                    if (half == 0) {          // keys 0-63 of P are complete: their half of P V can start now
+                        tc_wait_st();
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(&S.p_half[w]);
+                    }
                 }
             } else {
 #pragma unroll
@@ -280,6 +291,12 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                         pk[c >> 1] = pack_bf16(p0, p1);
                     }
                     tmem_st32(tS + half * 32, pk);
+                    if (half == 0) {
+                        tc_wait_st();
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(&S.p_half[w]);
+                    }
                 }
             }
             l += (sa[0] + sa[1]) + (sa[2] + sa[3]);
@@ -531,17 +548,28 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
 #pragma unroll
                 for (int w = 0; w < 2; ++w) {          // unrolled: n_p[] stays in registers
                     if (ok && use_bit(entry, w)) {
-                        ok = mbar_wait_warp(&S.p_ready[w], n_p[w] & 1, abort_flag);
+                        // P V in two halves of 64 keys: the first runs while the softmax group still forms the second
+                        const uint64_t dv = dV0 + (uint64_t)(st * (kTileBytes >> 4));
+                        const uint32_t d_tmem = tmem_u + 256 + w * 128, a_tmem = tmem_u + w * 128;
+                        const uint32_t acc0 = n_p[w] > 0 ? 1u : 0u;
+                        ok = mbar_wait_warp(&S.p_half[w], n_p[w] & 1, abort_flag);
+                        if (ok) {
+                            tc_fence_after();
+                            if (elect_one()) {
+#pragma unroll
+                                for (int kk = 0; kk < 4; ++kk)
+                                    mma_ts(d_tmem, a_tmem + kk * 8, dv + (uint64_t)((kk * 2048) >> 4), idesc_pv, kk > 0 ? 1u : acc0);
+                            }
+                            __syncwarp();
+                            ok = mbar_wait_warp(&S.p_ready[w], n_p[w] & 1, abort_flag);
+                        }
                         if (lane == 0) TRACE(it, 8 + w * 2);
                         if (ok) {
                             tc_fence_after();
-                            const uint64_t dv = dV0 + (uint64_t)(st * (kTileBytes >> 4));
-                            const uint32_t d_tmem = tmem_u + 256 + w * 128, a_tmem = tmem_u + w * 128;
-                            const uint32_t acc0 = n_p[w] > 0 ? 1u : 0u;
                             if (elect_one()) {
 #pragma unroll
-                                for (int kk = 0; kk < 8; ++kk)
-                                    mma_ts(d_tmem, a_tmem + kk * 8, dv + (uint64_t)((kk * 2048) >> 4), idesc_pv, kk > 0 ? 1u : acc0);
+                                for (int kk = 4; kk < 8; ++kk)
+                                    mma_ts(d_tmem, a_tmem + kk * 8, dv + (uint64_t)((kk * 2048) >> 4), idesc_pv, 1u);
                                 tc_commit(&S.o_done[w]);
                             }
                             __syncwarp();
