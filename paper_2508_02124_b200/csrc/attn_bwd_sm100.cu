@@ -4,14 +4,18 @@
 // and dM (registers) for it while walking the query heads of the group and their active query tiles in steps of
 // 64 query rows. Everything is computed transposed, keys on the 128 TMEM lanes, so that dM is a per-thread row sum
 // and P^T, dS^T feed the dV / dK GEMMs straight from tensor memory:
-//   S^T  = K Q^T            dP^T = V dO^T                      (smem x smem  -> TMEM, 64 columns each)
-//   P^T  = exp2(S^T c + log2e (bias_j - lse_i)) where j <= i < expiry[j], else 0;   dS^T = P^T o (dP^T - D_i)
+//   S^T  = K Q^T - lse_i / scale     dP^T = V dO^T - D_i      (smem x smem -> TMEM, 64 columns each; the per-row terms
+//                                                              come from a ninth k-step: ones (x) three bf16 terms)
+//   P^T  = exp2(c S^T + log2e bias_j) where j <= i < expiry[j], else 0;   dS^T = P^T o dP^T
 //   dV  += P^T dO           dK  += dS^T Q                      (TMEM x smem  -> TMEM, 128 columns each)
 //   dQ^T = K^T dS^T                                            (smem x smem  -> TMEM, 64 columns), staged in shared memory
-//                                                              and added to the fp32 dQ accumulator by a TMA reduce-add
+//                                                              and added to the fp32 dQ accumulator by TMA reduce-adds
+// Shared-memory bandwidth is the scarce resource (operand reads of the smem x smem MMAs alone take ~1400 of a step's
+// ~2250 cycles), so the compute warps read nothing from shared memory per element.
 // Warp roles (16 warps): warps 0-7 compute (thread = key; warps w and w+4 share the 32 TMEM lanes of quadrant w%4 and
 // split the 64 query columns of a step), warps 8-11 dQ drain (thread = channel), warp 12 TMA producer + schedule,
-// warps 13 and 14 MMA issuers (S^T, dP^T | dV, dK, dQ^T), warp 15 stages -lse and -D of each step's query rows.
+// warps 13 and 14 MMA issuers (S^T, dP^T | dV, dK, dQ^T; whole warps with warp-uniform values, one elected lane
+// issues), warp 15 stages the ninth k-step operand of each step's query rows.
 // TMEM columns: dK [0,128) dV [128,256) S^T [256,320) dP^T [320,384) P^T [384,416) dS^T [416,448) dQ^T [448,512).
 #include <cstdlib>
 
@@ -36,9 +40,14 @@ struct SharedStorage {
     alignas(1024) uint8_t q[kStages][kQBytes];
     alignas(1024) uint8_t g[kStages][kQBytes];       // dO
     alignas(1024) uint8_t ds[128 * 128];             // dS^T as bf16: [128 keys][64 queries], 128-byte swizzled rows
-    alignas(1024) float dq_stage[4][2][32][32];      // dQ per drain warp (32 channels) and half step: [query row][channel], sources of the TMA reduce-adds
-    alignas(16) float nlse[kStages][64];             // -log2(e) * lse_i
-    alignas(16) float dvec[kStages][64];             // -D_i
+    alignas(1024) float dq_stage[4][2][16][32];      // dQ per drain warp (32 channels), two buffers of 16 query rows: sources of the TMA reduce-adds
+    // Ninth k-step of S^T = K Q^T and dP^T = V dO^T (unswizzled K-major core matrices of 8 rows x 16 bytes): it adds
+    // -lse_i / scale to S^T and -D_i to dP^T, each as three bf16 terms, so that the compute warps read finished values
+    // from tensor memory and need no per-column vector. `ones` = [zero | rows (1,1,1,0..) | zero] blocks of 128 rows:
+    // A operand with the ones in elements 0-2 (block 1, then block 2) or in elements 8-10 (block 0, then block 1).
+    // `qext[stage]` = B operand, 64 query rows: elements 0-2 = -lse / scale, elements 8-10 = -D.
+    alignas(128) uint8_t ones[3][2048];
+    alignas(128) uint8_t qext[kStages][2048];
     uint16_t sched[kMaxSteps];                       // head-in-group << 11 | query tile << 1 | half
     uint64_t kv_full, qd_full[kStages], qd_empty[kStages];
     uint64_t sdp_full, sdp_free, pds_ready, pds_free, dq_full, dq_free;
@@ -59,7 +68,7 @@ struct BwdParams {
     float* dM;
     int32_t* status;
     int B, Hq, Hkv, G, L, Tr, Tc, Wd, ignore_bitmap;
-    float scale, scale_log2;
+    float scale, scale_log2, inv_scale;
     int64_t ks_b, ks_l, ks_h, vs_b, vs_l, vs_h;
 #ifdef DMA_PROF
     long long* prof;            // role timing (development builds only): cycles per phase of CTA (0, 0)
@@ -77,6 +86,15 @@ struct BwdParams {
 #define PROF_WAIT(slot, expr) do { expr; } while (0)
 #define PROF_END()
 #endif
+
+// x as three bf16 terms (hi, mid, lo: 24 significant bits) in elements 0-2 of a 16-byte core-matrix row
+__device__ __forceinline__ uint4 split3(float x) {
+    const __nv_bfloat16 hi = __float2bfloat16_rn(x);
+    const float r1 = x - __bfloat162float(hi);
+    const __nv_bfloat16 mid = __float2bfloat16_rn(r1);
+    const __nv_bfloat16 lo = __float2bfloat16_rn(r1 - __bfloat162float(mid));
+    return make_uint4((uint32_t)__bfloat16_as_ushort(hi) | ((uint32_t)__bfloat16_as_ushort(mid) << 16), (uint32_t)__bfloat16_as_ushort(lo), 0u, 0u);
+}
 
 __global__ void __launch_bounds__(kThreads, 1)
 bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
@@ -134,6 +152,15 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             }
         }
         if (lane == 0) S.n_steps = min(n, kMaxSteps);
+    }
+    if (warp == 15) {
+        // constant A operand of the ninth k-step: zero block | rows (1, 1, 1, 0, ...) | zero block
+        for (int r = lane; r < 128; r += 32) {
+            *reinterpret_cast<uint4*>(S.ones[0] + r * 16) = make_uint4(0u, 0u, 0u, 0u);
+            *reinterpret_cast<uint4*>(S.ones[1] + r * 16) = make_uint4(0x3F803F80u, 0x00003F80u, 0u, 0u);
+            *reinterpret_cast<uint4*>(S.ones[2] + r * 16) = make_uint4(0u, 0u, 0u, 0u);
+        }
+        fence_proxy_async();
     }
     tc_fence_before();
     __syncthreads();
@@ -195,15 +222,12 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                 const float2 bj2 = make_float2(be, be);
 #pragma unroll
                 for (int c = 0; c < 32; c += 4) {
-                    const float4 nl = *reinterpret_cast<const float4*>(&S.nlse[st][c0 + c]);
-                    const float4 nd = *reinterpret_cast<const float4*>(&S.dvec[st][c0 + c]);   // holds -D_i
-                    float2 x[2], t[2];
-                    x[0] = fma2(make_float2(__uint_as_float(sr[c]), __uint_as_float(sr[c + 1])), sc2, add2(make_float2(nl.x, nl.y), bj2));
-                    x[1] = fma2(make_float2(__uint_as_float(sr[c + 2]), __uint_as_float(sr[c + 3])), sc2, add2(make_float2(nl.z, nl.w), bj2));
-                    t[0] = add2(make_float2(__uint_as_float(pr[c]), __uint_as_float(pr[c + 1])), make_float2(nd.x, nd.y));
-                    t[1] = add2(make_float2(__uint_as_float(pr[c + 2]), __uint_as_float(pr[c + 3])), make_float2(nd.z, nd.w));
-                    const float2 p0 = make_float2(ex2(x[0].x), ex2(x[0].y)), p1 = make_float2(ex2(x[1].x), ex2(x[1].y));
-                    const float2 d0 = mul2(p0, t[0]), d1 = mul2(p1, t[1]);
+                    const float2 x0 = fma2(make_float2(__uint_as_float(sr[c]), __uint_as_float(sr[c + 1])), sc2, bj2);
+                    const float2 x1 = fma2(make_float2(__uint_as_float(sr[c + 2]), __uint_as_float(sr[c + 3])), sc2, bj2);
+                    const float2 t0 = make_float2(__uint_as_float(pr[c]), __uint_as_float(pr[c + 1]));
+                    const float2 t1 = make_float2(__uint_as_float(pr[c + 2]), __uint_as_float(pr[c + 3]));
+                    const float2 p0 = make_float2(ex2(x0.x), ex2(x0.y)), p1 = make_float2(ex2(x1.x), ex2(x1.y));
+                    const float2 d0 = mul2(p0, t0), d1 = mul2(p1, t1);
                     dm2 = add2(dm2, add2(d0, d1));
                     pp[(c >> 1)] = pack_bf16(p0.x, p0.y);
                     pp[(c >> 1) + 1] = pack_bf16(p1.x, p1.y);
@@ -214,20 +238,17 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                 const float2 bj2 = make_float2(bj, bj);
 #pragma unroll
                 for (int c = 0; c < 32; c += 4) {
-                    const float4 nl = *reinterpret_cast<const float4*>(&S.nlse[st][c0 + c]);
-                    const float4 nd = *reinterpret_cast<const float4*>(&S.dvec[st][c0 + c]);   // holds -D_i
-                    float2 x[2], t[2];
-                    x[0] = fma2(make_float2(__uint_as_float(sr[c]), __uint_as_float(sr[c + 1])), sc2, add2(make_float2(nl.x, nl.y), bj2));
-                    x[1] = fma2(make_float2(__uint_as_float(sr[c + 2]), __uint_as_float(sr[c + 3])), sc2, add2(make_float2(nl.z, nl.w), bj2));
-                    t[0] = add2(make_float2(__uint_as_float(pr[c]), __uint_as_float(pr[c + 1])), make_float2(nd.x, nd.y));
-                    t[1] = add2(make_float2(__uint_as_float(pr[c + 2]), __uint_as_float(pr[c + 3])), make_float2(nd.z, nd.w));
-                    float p[4] = {ex2(x[0].x), ex2(x[0].y), ex2(x[1].x), ex2(x[1].y)};
+                    const float2 x0 = fma2(make_float2(__uint_as_float(sr[c]), __uint_as_float(sr[c + 1])), sc2, bj2);
+                    const float2 x1 = fma2(make_float2(__uint_as_float(sr[c + 2]), __uint_as_float(sr[c + 3])), sc2, bj2);
+                    const float2 t0 = make_float2(__uint_as_float(pr[c]), __uint_as_float(pr[c + 1]));
+                    const float2 t1 = make_float2(__uint_as_float(pr[c + 2]), __uint_as_float(pr[c + 3]));
+                    float p[4] = {ex2(x0.x), ex2(x0.y), ex2(x1.x), ex2(x1.y)};
 #pragma unroll
                     for (int u = 0; u < 4; ++u) {
                         const bool valid = (unsigned)(c + u - lo) < (unsigned)width;
                         p[u] = valid ? p[u] : 0.0f;
                     }
-                    const float2 d0 = mul2(make_float2(p[0], p[1]), t[0]), d1 = mul2(make_float2(p[2], p[3]), t[1]);
+                    const float2 d0 = mul2(make_float2(p[0], p[1]), t0), d1 = mul2(make_float2(p[2], p[3]), t1);
                     dm2 = add2(dm2, add2(d0, d1));
                     pp[(c >> 1)] = pack_bf16(p[0], p[1]);
                     pp[(c >> 1) + 1] = pack_bf16(p[2], p[3]);
@@ -299,8 +320,8 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
         }
     } else if (warp < 12) {
         // ============================ dQ drain group: thread = channel c, columns = query rows ============================
-        // Each warp owns 32 channels and its own pair of staging buffers (one per 32-row half step), so the warps
-        // never wait for each other: a half is rewritten once the reduce-add issued from it two groups ago has
+        // Each warp owns 32 channels and its own pair of staging buffers (16 query rows each, used in turn), so the
+        // warps never wait for each other: a buffer is rewritten once the reduce-add issued from it two groups ago has
         // finished reading it.
         const int dw = warp & 3;
         const uint32_t lane_base = (uint32_t)(dw * 32) << 16;
@@ -320,14 +341,14 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             __syncwarp();
             if (lane == 0) mbar_arrive(&S.dq_free);
 #pragma unroll
-            for (int hf = 0; hf < 2; ++hf) {
-                PROF_WAIT(1 + hf, if (lane == 0) bulk_wait_read_1(); __syncwarp());
+            for (int qr = 0; qr < 4; ++qr) {           // quarter steps of 16 query rows, two staging buffers in turn
+                PROF_WAIT(1 + (qr & 1), if (lane == 0) bulk_wait_read_1(); __syncwarp());
 #pragma unroll
-                for (int u = 0; u < 32; ++u) S.dq_stage[dw][hf][u][lane] = __uint_as_float(v[hf * 32 + u]);
+                for (int u = 0; u < 16; ++u) S.dq_stage[dw][qr & 1][u][lane] = __uint_as_float(v[qr * 16 + u]);
                 fence_proxy_async();
                 __syncwarp();
-                if (lane == 0 && i0 + hf * 32 < P.L) {
-                    tma_reduce_add_4d(&tmDQ, &S.dq_stage[dw][hf][0][0], dw * 32, hk * P.G + g, i0 + hf * 32, b);   // rows beyond L are clipped
+                if (lane == 0 && i0 + qr * 16 < P.L) {
+                    tma_reduce_add_4d(&tmDQ, &S.dq_stage[dw][qr & 1][0][0], dw * 32, hk * P.G + g, i0 + qr * 16, b);   // rows beyond L are clipped
                 }
                 if (lane == 0) bulk_commit();
             }
@@ -362,7 +383,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             for (int n = max(0, n_steps - kStages); n < n_steps && ok; ++n)
                 ok = mbar_wait_warp(&S.qd_empty[n % kStages], (n / kStages) & 1, abort_flag);
         } else if (warp == 15) {
-            // ============================ stager: -log2e*lse and -D of each step's query rows, loaded one step ahead ============================
+            // ============================ stager: ninth k-step B operand (-lse / scale, -D) of each step's query rows, loaded one step ahead ============================
             auto fetch = [&](int n, float (&lv)[2], float (&dv)[2]) {
                 const uint32_t e = S.sched[n];
                 const int h = hk * P.G + (int)(e >> 11), i0 = (int)((e >> 1) & 0x3FF) * 128 + (int)(e & 1) * 64;
@@ -385,11 +406,14 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                 if (!ok) break;
 #pragma unroll
                 for (int t = 0; t < 2; ++t) {
-                    S.nlse[st][lane + 32 * t] = -1.4426950408889634f * lv[t];
-                    S.dvec[st][lane + 32 * t] = -dv[t];
+                    const int r = lane + 32 * t;
+                    uint8_t* row = S.qext[st] + (r >> 3) * 256 + (r & 7) * 16;
+                    *reinterpret_cast<uint4*>(row) = split3(-lv[t] * P.inv_scale);        // elements 0-2: -lse_i / scale
+                    *reinterpret_cast<uint4*>(row + 128) = split3(-dv[t]);                // elements 8-10: -D_i
                     lv[t] = ln[t];
                     dv[t] = dn[t];
                 }
+                fence_proxy_async();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&S.qd_full[st]);
             }
@@ -401,6 +425,9 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             constexpr uint32_t id_sdp = idesc_bf16(128, 64, 0, 0);     // K|V (K-major) x Q|dO (K-major)       -> 128 x 64
             const uint64_t dK = smem_desc_sw128(smem_u32(S.k), 16, 1024), dV = smem_desc_sw128(smem_u32(S.v), 16, 1024);
             const uint64_t dQ0 = smem_desc_sw128(smem_u32(S.q[0]), 16, 1024), dG0 = smem_desc_sw128(smem_u32(S.g[0]), 16, 1024);
+            // ninth k-step: 8-row groups 128 bytes apart, second K core matrix one 2 KB block further (A) / 128 bytes further (B)
+            const uint64_t dOnesLo = smem_desc_plain(smem_u32(S.ones[1]), 2048, 128), dOnesHi = smem_desc_plain(smem_u32(S.ones[0]), 2048, 128);
+            const uint64_t dX0 = smem_desc_plain(smem_u32(S.qext[0]), 128, 256);
             const uint32_t tmem_u = __shfl_sync(0xffffffffu, tmem, 0);
             const int n_steps_u = __shfl_sync(0xffffffffu, n_steps, 0);
             bool ok = mbar_wait_warp(&S.kv_full, 0, abort_flag);
@@ -412,15 +439,18 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                 if (!ok) break;
                 tc_fence_after();
                 const uint64_t dQ = dQ0 + (uint64_t)(st * (kQBytes >> 4)), dG = dG0 + (uint64_t)(st * (kQBytes >> 4));
+                const uint64_t dX = dX0 + (uint64_t)(st * (2048 >> 4));
                 if (elect_one()) {
 #pragma unroll
                     for (int kk = 0; kk < 8; ++kk)
                         mma_ss(tmem_u + cS, dK + (uint64_t)(((kk >> 2) * (kKVBytes / 2) + (kk & 3) * 32) >> 4),
                                dQ + (uint64_t)(((kk >> 2) * (kQBytes / 2) + (kk & 3) * 32) >> 4), id_sdp, kk > 0);
+                    mma_ss(tmem_u + cS, dOnesLo, dX, id_sdp, 1u);          // S^T  += 1 (x) (-lse / scale)
 #pragma unroll
                     for (int kk = 0; kk < 8; ++kk)
                         mma_ss(tmem_u + cDP, dV + (uint64_t)(((kk >> 2) * (kKVBytes / 2) + (kk & 3) * 32) >> 4),
                                dG + (uint64_t)(((kk >> 2) * (kQBytes / 2) + (kk & 3) * 32) >> 4), id_sdp, kk > 0);
+                    mma_ss(tmem_u + cDP, dOnesHi, dX, id_sdp, 1u);         // dP^T += 1 (x) (-D)
                     tc_commit(&S.sdp_full);
                 }
                 __syncwarp();
@@ -529,7 +559,7 @@ int launch_tc_bwd(const Prob& P, const void* Q, const void* K, const void* V, co
     if ((rc = make_tmap_bf16(&tmK, K, P.B, P.L, P.Hkv, P.d, P.ks, 128))) return rc;
     if ((rc = make_tmap_bf16(&tmV, V, P.B, P.L, P.Hkv, P.d, P.vs, 128))) return rc;
     CUtensorMap tmDQ;
-    if ((rc = make_tmap_f32_rows(&tmDQ, acc, P.B, P.L, P.Hq, 32, 32))) return rc;
+    if ((rc = make_tmap_f32_rows(&tmDQ, acc, P.B, P.L, P.Hq, 16, 32))) return rc;
     rowdot_bf16_kernel<<<(unsigned)((rows + 7) / 8), 256, 0, st>>>((const __nv_bfloat16*)O, (const __nv_bfloat16*)dO, Dv, P.B, P.L, P.Hq,
                                                                     P.os[0], P.os[1], P.os[2]);
     if (cudaMemsetAsync(acc, 0, nq * sizeof(float), st) != cudaSuccess) return DMA_ERR_CUDA;
@@ -539,7 +569,7 @@ int launch_tc_bwd(const Prob& P, const void* Q, const void* K, const void* V, co
     bp.dK = (__nv_bfloat16*)dK; bp.dV = (__nv_bfloat16*)dV; bp.dM = dM; bp.status = (int32_t*)ws;
     bp.B = P.B; bp.Hq = P.Hq; bp.Hkv = P.Hkv; bp.G = P.G; bp.L = P.L; bp.Tr = P.Tr; bp.Tc = P.Tc; bp.Wd = P.Wd;
     bp.ignore_bitmap = (P.flags & DMA_FLAG_IGNORE_BITMAP) ? 1 : 0;
-    bp.scale = P.scale; bp.scale_log2 = P.scale * 1.4426950408889634f;
+    bp.scale = P.scale; bp.scale_log2 = P.scale * 1.4426950408889634f; bp.inv_scale = 1.0f / P.scale;
     bp.ks_b = P.ks[0]; bp.ks_l = P.ks[1]; bp.ks_h = P.ks[2]; bp.vs_b = P.vs[0]; bp.vs_l = P.vs[1]; bp.vs_h = P.vs[2];
 #ifdef DMA_PROF
     const char* prof_env = getenv("DMA_PROF_PTR");
