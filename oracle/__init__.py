@@ -158,3 +158,32 @@ def backward(Q, K, V, dO, bias, expiry=None, keep=None, scale=None, keys=None, w
            ctypes.c_double(scale), _p(keys), 0 if keys is None else len(keys), _p(dQ), _p(dK), _p(dV), _p(dM))
     assert rc == 0, rc
     return dQ, dK, dV, dM
+
+
+def mask_backward(V, W, A, dM, Hq):
+    """Gradient of the mask-generation bias path (Sec. 4.3: the bias gradient dM reaches the sampling weights and
+    the gate; Eq. delta_calc differentiated with the top-w selection held fixed). Plain numpy, fp64:
+
+        z = v . W_h,  sp = softplus(z),  delta = exp(A_h sp)          (forward, per query head h and key j)
+        g = dM delta;  dA_h = sum g sp;  dz = g A_h sigmoid(z);  dW_h = sum dz v;  dV[j, kv head] = sum_h dz W_h
+
+    V [B,L,Hkv,d], W [Hq,d], A [Hq], dM [B,Hq,L] -> (dV [B,L,Hkv,d], dW [Hq,d], dA [Hq]); query head h reads KV
+    head h // (Hq // Hkv)."""
+    V = np.asarray(V, np.float64); W = np.asarray(W, np.float64); A = np.asarray(A, np.float64)
+    dM = np.asarray(dM, np.float64)
+    B, L, Hkv, d = V.shape
+    G = Hq // Hkv
+    dV = np.zeros_like(V); dW = np.zeros_like(W); dA = np.zeros_like(A)
+    for h in range(Hq):
+        hk = h // G
+        v = V[:, :, hk, :]                                   # [B, L, d]
+        z = v @ W[h]                                         # [B, L]
+        sp = np.maximum(z, 0.0) + np.log1p(np.exp(-np.abs(z)))
+        delta = np.exp(A[h] * sp)
+        g = dM[:, h, :] * delta
+        dA[h] = (g * sp).sum()
+        sig = np.where(z >= 0, 1.0 / (1.0 + np.exp(-np.abs(z))), np.exp(-np.abs(z)) / (1.0 + np.exp(-np.abs(z))))
+        dz = g * A[h] * sig
+        dW[h] = np.einsum("bl,bld->d", dz, v)
+        dV[:, :, hk, :] += dz[..., None] * W[h]
+    return dV, dW, dA
