@@ -219,6 +219,25 @@ def main():
     stage_ms = {k: v / args.steps for k, v in stage_ms.items()}
     ms = replicas.max_over_ranks(total_ms / args.steps, dev)
 
+    # ---- mask-generation backward (bias gradient on to W_delta, A and V), timed on its own after the step: it is
+    # not part of the headline metric. HBM-bound: V read once, dV read and written once, bias and dM read once.
+    mask_bwd = None
+    if case.backward:
+        ws_g = torch.empty(dma.dma_mask_bwd_workspace(p), dtype=torch.uint8, device=dev)
+        dWd, dAg = torch.empty_like(W), torch.empty_like(A)
+        for _ in range(3):
+            dma.dma_mask_bwd(p, V, W, A, bias, dM, dV, dWd, dAg, ws_g)
+        g0, g1 = ev(), ev()
+        barrier()
+        g0.record()
+        for _ in range(10):
+            dma.dma_mask_bwd(p, V, W, A, bias, dM, dV, dWd, dAg, ws_g)
+        g1.record()
+        barrier()
+        g_ms = g0.elapsed_time(g1) / 10
+        g_bytes = 3 * V.numel() * V.element_size() + 2 * bias.numel() * 4
+        mask_bwd = {"ms": g_ms, "algorithmic_bytes": g_bytes, "gbs": g_bytes / (g_ms * 1e-3) / 1e9}
+
     # ---- end to end through the host-buffer entry point: pinned host tensors in, results back on the host
     e2e = None
     if not args.no_e2e:
@@ -276,6 +295,9 @@ def main():
                      "traffic": NCU_TRAFFIC_BYTES.get(case.name, {}).get(dom) if tensor_path else None},
         "gpu_launches": launches, "clocks": clocks, "e2e": e2e,
     }
+    if mask_bwd is not None:
+        mask_bwd["frac_of_measured_hbm"] = mask_bwd["gbs"] / pk["hbm_gbs"]
+        out["mask_bwd"] = mask_bwd
     if args.cpu_rows:
         Ls = min(case.L, args.cpu_rows)
         sec, fl, cores = oracle_sample_run(case, inp, Ls)

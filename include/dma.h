@@ -122,6 +122,19 @@ int dma_attn_bwd(const dma_problem_t* p, const void* Q, const void* K, const voi
                  void* dQ, void* dK, void* dV, float* dM,
                  void* ws, size_t ws_bytes, void* cuda_stream);
 
+/* Mask-generation backward (Sec. 4.3: the bias gradient dM produced by dma_attn_bwd flows on to the sampling weights
+ * and the gate; Eq. (delta_calc) differentiated with the top-w selection held fixed). With z = v_j . W_delta[h],
+ * sp = softplus(z) and delta = exp(A[h] sp) = bias[b,h,j]:
+ *   g = dM[b,h,j] delta;   dA[h] = sum_{b,j} g sp;   dz = g A[h] sigmoid(z);
+ *   dW_delta[h,:] = sum_{b,j} dz v_j;      dV[b,j,h / (Hq/Hkv),:] += sum_{h in group} dz W_delta[h,:]
+ * V, bias (the delta written by dma_mask_build), dM: inputs. dV [B,L,Hkv,d] (layout and strides of V, element type of
+ * the problem) is IN/OUT: the contribution is added to what it holds (the attention backward's dV), in fp32, and
+ * rounded once. dW_delta [Hq,d] and dA [Hq] fp32 are overwritten; their sums are formed in a fixed order (no
+ * floating-point atomics). ws: dma_mask_bwd_workspace() bytes. All pointers device memory, 16-byte aligned. */
+int dma_mask_bwd_workspace(const dma_problem_t* p, size_t* bytes);
+int dma_mask_bwd(const dma_problem_t* p, const void* V, const float* W_delta, const float* A, const float* bias,
+                 const float* dM, void* dV, float* dW_delta, float* dA, void* ws, size_t ws_bytes, void* cuda_stream);
+
 /* The whole hot path on HOST buffers (all contiguous, default strides only): copies Q,K,V,(dO),W_delta,A into the
  * caller's device arena, runs dma_mask_build, dma_attn_fwd and, if `backward` != 0, dma_attn_bwd on the stream,
  * copies O, lse (and dQ,dK,dV,dM) back and synchronises the stream before returning. h* pointers are HOST memory

@@ -17,7 +17,8 @@ DMA_BF16, DMA_FP32 = 0, 1
 DMA_FLAG_IGNORE_BITMAP, DMA_FLAG_SIMT = 1, 2
 
 ENTRY_POINTS = ("dma_query_workspace", "dma_bitmap_words", "dma_mask_build", "dma_attn_fwd", "dma_attn_bwd",
-                "dma_read_status", "dma_launch_count", "dma_strerror", "dma_step_host_arena", "dma_step_host", "dma_mask_build_static", "dma_selftest_wait_timeout")
+                "dma_read_status", "dma_launch_count", "dma_strerror", "dma_step_host_arena", "dma_step_host", "dma_mask_build_static", "dma_selftest_wait_timeout",
+                "dma_mask_bwd_workspace", "dma_mask_bwd")
 
 
 class DmaError(RuntimeError):
@@ -108,6 +109,26 @@ def dma_mask_build(p, V, W_delta, A, bias=None, expiry=None, bitmap=None, ws=Non
     _check(lib().dma_mask_build(ctypes.byref(p), _ptr(V), _ptr(W_delta), _ptr(A), _ptr(bias), _ptr(expiry), _ptr(bitmap),
                                 _ptr(ws), ctypes.c_size_t(ws.numel()), _stream()), "dma_mask_build")
     return bias, expiry, bitmap
+
+
+def dma_mask_bwd_workspace(p):
+    n = ctypes.c_size_t()
+    _check(lib().dma_mask_bwd_workspace(ctypes.byref(p), ctypes.byref(n)), "dma_mask_bwd_workspace")
+    return n.value
+
+
+def dma_mask_bwd(p, V, W_delta, A, bias, dM, dV, dW_delta=None, dA=None, ws=None):
+    """Adds the mask path's contribution to dV in place; returns (dV, dW_delta [Hq,d] fp32, dA [Hq] fp32)."""
+    dev = V.device
+    if dW_delta is None:
+        dW_delta = torch.empty(p.Hq, p.d, dtype=torch.float32, device=dev)
+    if dA is None:
+        dA = torch.empty(p.Hq, dtype=torch.float32, device=dev)
+    if ws is None:
+        ws = _ws(dma_mask_bwd_workspace(p), dev)
+    _check(lib().dma_mask_bwd(ctypes.byref(p), _ptr(V), _ptr(W_delta), _ptr(A), _ptr(bias), _ptr(dM), _ptr(dV), _ptr(dW_delta),
+                              _ptr(dA), _ptr(ws), ctypes.c_size_t(ws.numel()), _stream()), "dma_mask_bwd")
+    return dV, dW_delta, dA
 
 
 def dma_attn_fwd(p, Q, K, V, bias, expiry, bitmap, O=None, lse=None, ws=None):

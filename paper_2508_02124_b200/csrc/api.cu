@@ -113,6 +113,28 @@ int dma_mask_build(const dma_problem_t* p, const void* V, const float* W_delta, 
     return launch_mask_build(P, V, W_delta, A, bias, expiry, bitmap, ws, (cudaStream_t)cuda_stream);
 }
 
+int dma_mask_bwd_workspace(const dma_problem_t* p, size_t* bytes) {
+    Prob P;
+    int rc = resolve(p, &P);
+    if (rc) return rc;
+    if (!bytes) return DMA_ERR_NULL;
+    *bytes = mask_bwd_ws_bytes(P);
+    return DMA_OK;
+}
+
+int dma_mask_bwd(const dma_problem_t* p, const void* V, const float* W_delta, const float* A, const float* bias,
+                 const float* dM, void* dV, float* dW_delta, float* dA, void* ws, size_t ws_bytes, void* cuda_stream) {
+    Prob P;
+    int rc = resolve(p, &P);
+    if (rc) return rc;
+    if (!V || !W_delta || !A || !bias || !dM || !dV || !dW_delta || !dA) return DMA_ERR_NULL;
+    if (!aligned16(V) || !aligned16(W_delta) || !aligned16(bias) || !aligned16(dM) || !aligned16(dV) || !aligned16(dW_delta))
+        return DMA_ERR_ALIGN;
+    if (!ws || ws_bytes < mask_bwd_ws_bytes(P) || !aligned16(ws)) return DMA_ERR_WORKSPACE;
+    if ((rc = device_ok())) return rc;
+    return launch_mask_bwd(P, V, W_delta, A, bias, dM, dV, dW_delta, dA, ws, (cudaStream_t)cuda_stream);
+}
+
 int dma_attn_fwd(const dma_problem_t* p, const void* Q, const void* K, const void* V, const float* bias,
                  const int32_t* expiry, const uint32_t* bitmap, void* O, float* lse, void* ws, size_t ws_bytes,
                  void* cuda_stream) {

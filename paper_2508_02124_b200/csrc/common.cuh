@@ -27,6 +27,9 @@ int check_launch();                                       // cudaGetLastError ->
 
 // stage launchers (each returns a dma_status); defined in the stage's .cu file
 size_t mask_ws_bytes(const Prob& P);
+size_t mask_bwd_ws_bytes(const Prob& P);
+int launch_mask_bwd(const Prob& P, const void* V, const float* W, const float* A, const float* delta, const float* dM,
+                    void* dV, float* dW, float* dA, void* ws, cudaStream_t st);
 int launch_mask_build(const Prob& P, const void* V, const float* W, const float* A, float* bias, int32_t* expiry,
                       uint32_t* bitmap, void* ws, cudaStream_t st);
 
