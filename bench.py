@@ -238,6 +238,27 @@ def main():
         g_bytes = 3 * V.numel() * V.element_size() + 2 * bias.numel() * 4
         mask_bwd = {"ms": g_ms, "algorithmic_bytes": g_bytes, "gbs": g_bytes / (g_ms * 1e-3) / 1e9}
 
+    # ---- token-compacted forward (DMA_FLAG_COMPACT_KV), timed on its own: same outputs, O(L w d) work
+    compact = None
+    if case.dtype == "bf16" and case.d == 128 and not (args.flags & dma.DMA_FLAG_SIMT):
+        pc = dma.problem(case.B, case.Hq, case.Hkv, case.L, case.d, case.w, dtype=case.torch_dtype,
+                         flags=args.flags | dma.DMA_FLAG_COMPACT_KV)
+        ws_c = torch.empty(dma.dma_query_workspace(pc)[1], dtype=torch.uint8, device=dev)
+        Oc, lsec = torch.empty_like(O), torch.empty_like(lse)
+        for _ in range(3):
+            dma.dma_attn_fwd(pc, Q, K, V, bias, expiry, bitmap, Oc, lsec, ws_c)
+        c0, c1 = ev(), ev()
+        barrier()
+        c0.record()
+        for _ in range(10):
+            dma.dma_attn_fwd(pc, Q, K, V, bias, expiry, bitmap, Oc, lsec, ws_c)
+        c1.record()
+        barrier()
+        assert dma.dma_read_status(ws_c) == 0, "device status (compact forward)"
+        c_ms = c0.elapsed_time(c1) / 10
+        compact = {"fwd_ms": c_ms, "tile_fwd_ms": stage_ms["fwd"], "speedup_over_tile_skipping": stage_ms["fwd"] / c_ms,
+                   "max_abs_diff_vs_tile_path": float((Oc.float() - O.float()).abs().max())}
+
     # ---- end to end through the host-buffer entry point: pinned host tensors in, results back on the host
     e2e = None
     if not args.no_e2e:
@@ -295,6 +316,8 @@ def main():
                      "traffic": NCU_TRAFFIC_BYTES.get(case.name, {}).get(dom) if tensor_path else None},
         "gpu_launches": launches, "clocks": clocks, "e2e": e2e,
     }
+    if compact is not None:
+        out["compact_fwd"] = compact
     if mask_bwd is not None:
         mask_bwd["frac_of_measured_hbm"] = mask_bwd["gbs"] / pk["hbm_gbs"]
         out["mask_bwd"] = mask_bwd

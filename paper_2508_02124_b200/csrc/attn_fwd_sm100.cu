@@ -46,8 +46,10 @@ struct SharedStorage {
     alignas(128) uint8_t aext[2][4096];
     alignas(128) uint8_t bext[2][4096];
     alignas(16) int len[kStages][128];        // expiry[j] (0 beyond L): row i keeps key j iff j <= i < expiry[j]
+    alignas(16) int jidx[kStages][128];       // token-compacted mode: the key index of each gathered column
     int thr[2][16];                           // stager scratch: row thresholds of the keys that expire inside the tile
-    uint32_t fast[kStages][2];                // 1: the extra k-step carries the whole mask of this (key tile, query tile)
+    uint32_t fast[kStages][2];                // 1: the extra k-step carries the whole mask of this (key tile, query tile);
+                                              // token-compacted mode: bit q = 32-column chunk q needs the per-element test
     uint32_t sched[kMaxSched];                // key tile | use by tile 0 << 30 | use by tile 1 << 31
     uint64_t q_full, k_full[kStages], v_full[kStages], k_empty[kStages], v_empty[kStages];
     uint64_t s_full[2], p_half[2], p_ready[2], o_done[2];
@@ -67,6 +69,13 @@ struct FwdParams {
     float scale_log2;                          // softmax scale * log2(e)
     float inv_scale;                           // 1 / softmax scale
     float rescale_gap;                         // growth of a row max (score units) beyond which O is rescaled
+    // token-compacted mode: per (batch, head, pair of query tiles) the ascending list of keys that some row of the
+    // pair keeps, padded with -1 to a multiple of 128 (ccap entries per list), and its length
+    const int* cidx;
+    const int* ccnt;
+    const __nv_bfloat16* Kg;                   // K and V as contiguous [B, L, Hkv, 128] row arrays
+    const __nv_bfloat16* Vg;
+    int ccap, Hkv;
     int64_t os_b, os_l, os_h;
 #ifdef DMA_PROF
     long long* prof;                           // role timing (development builds only): cycles per phase of CTA (0, 0)
@@ -85,6 +94,12 @@ struct FwdParams {
 
 __device__ __forceinline__ uint32_t use_bit(uint32_t entry, int w) { return (entry >> (30 + w)) & 1u; }
 
+// kCompact: instead of walking the active 128-key tiles of the bitmap, the CTA walks its gathered key list (keys that
+// at least one of its 256 query rows keeps, at most w + 256 of them). Warps 8 and 11 fetch the K and V rows with 16-byte
+// asynchronous copies into the swizzled tile layout (TMA row gathers of four rows were measured at ~70 cycles per
+// request: too slow), warp 10 builds the B rows of the ninth k-step (bias, and -BIG for columns no row of the tile keeps; the A
+// rows are constant) and flags the 32-column chunks that still need the per-element test.
+template <bool kCompact>
 __global__ void __launch_bounds__(kThreads, 1)
 fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
            const __grid_constant__ CUtensorMap tmV, const FwdParams P) {
@@ -102,8 +117,8 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
     if (tid == 0) {
         mbar_init(&S.q_full, 1);
         for (int s = 0; s < kStages; ++s) {
-            mbar_init(&S.k_full[s], 3);      // TMA bytes of K + the two stager warps
-            mbar_init(&S.v_full[s], 1);
+            mbar_init(&S.k_full[s], kCompact ? 33 : 3);   // K: TMA bytes + the two stager warps | 32 gathering lanes + the stager warp
+            mbar_init(&S.v_full[s], kCompact ? 32 : 1);
             mbar_init(&S.k_empty[s], 1);
             mbar_init(&S.v_empty[s], 1);
         }
@@ -124,18 +139,24 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
     if (warp == 8) {
         // schedule: ascending key tiles that at least one of the two query tiles uses
         if (lane == 0) { prefetch_tmap(&tmQ); prefetch_tmap(&tmK); prefetch_tmap(&tmV); }
-        const int kt_last = min(has1 ? qt1 : qt0, P.Tc - 1);
         int n = 0;
-        for (int base = 0; base <= kt_last; base += 32) {
-            const int kt = base + lane;
-            uint32_t u0 = 0, u1 = 0;
-            if (kt <= kt_last) {
-                u0 = kt <= qt0 && (P.ignore_bitmap || bitmap_test(P.bitmap, P.Tr, P.Wd, bh, qt0, kt));
-                u1 = has1 && kt <= qt1 && (P.ignore_bitmap || bitmap_test(P.bitmap, P.Tr, P.Wd, bh, qt1, kt));
+        if constexpr (kCompact) {
+            // every 128-key slice of the gathered list, used by both query tiles
+            n = min((P.ccnt[(size_t)bh * npairs + pair] + 127) / 128, kMaxSched);
+            for (int t = lane; t < n; t += 32) S.sched[t] = (uint32_t)t | (1u << 30) | (has1 ? (1u << 31) : 0u);
+        } else {
+            const int kt_last = min(has1 ? qt1 : qt0, P.Tc - 1);
+            for (int base = 0; base <= kt_last; base += 32) {
+                const int kt = base + lane;
+                uint32_t u0 = 0, u1 = 0;
+                if (kt <= kt_last) {
+                    u0 = kt <= qt0 && (P.ignore_bitmap || bitmap_test(P.bitmap, P.Tr, P.Wd, bh, qt0, kt));
+                    u1 = has1 && kt <= qt1 && (P.ignore_bitmap || bitmap_test(P.bitmap, P.Tr, P.Wd, bh, qt1, kt));
+                }
+                const uint32_t act = __ballot_sync(0xffffffffu, u0 | u1);
+                if (u0 | u1) S.sched[n + __popc(act & ((1u << lane) - 1))] = (uint32_t)kt | (u0 << 30) | (u1 << 31);
+                n += __popc(act);
             }
-            const uint32_t act = __ballot_sync(0xffffffffu, u0 | u1);
-            if (u0 | u1) S.sched[n + __popc(act & ((1u << lane) - 1))] = (uint32_t)kt | (u0 << 30) | (u1 << 31);
-            n += __popc(act);
         }
         if (lane == 0) S.n_iters = n;
     }
@@ -171,7 +192,8 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             // the stagers' flag is there long before the S product: read it while waiting for S
             ok = mbar_wait_warp(&S.k_full[st], (it / kStages) & 1, abort_flag);
             if (!ok) break;
-            const bool fast_tile = S.fast[st][w] != 0;
+            const uint32_t tile_flags = S.fast[st][w];
+            const bool fast_tile = kCompact || tile_flags != 0;      // token-compacted mode: the flags are a chunk mask instead
             ok = mbar_wait_warp(&S.s_full[w], n_used & 1, abort_flag);
             if (!ok) break;
             tc_fence_after();
@@ -194,6 +216,24 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             PROF_ADD(1, t_c - t_b);
             if ((warp & 3) == 0 && lane == 0) TRACE(it, w * 4 + 1);
             float mxa[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+            if constexpr (kCompact) {
+                // gathered columns: bias and the keys that are gone for the whole tile are already in the score; the
+                // per-element test is needed only in the 32-column chunks the stager flagged (a key expiring or
+                // entering inside the tile's rows)
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    if ((tile_flags >> q) & 1u) {
+#pragma unroll
+                        for (int c = 32 * q; c < 32 * q + 32; c += 4) {
+                            const int4 ee = *reinterpret_cast<const int4*>(&S.len[st][c]);
+                            const int4 jj = *reinterpret_cast<const int4*>(&S.jidx[st][c]);
+                            const int ev[4] = {ee.x, ee.y, ee.z, ee.w}, jv[4] = {jj.x, jj.y, jj.z, jj.w};
+#pragma unroll
+                            for (int u = 0; u < 4; ++u) x[c + u] = (jv[u] <= i && i < ev[u]) ? x[c + u] : -INFINITY;
+                        }
+                    }
+                }
+            }
             if (fast_tile) {
                 PROF_ADD(6, 1);
 #pragma unroll
@@ -351,7 +391,138 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
         }
     } else {
         setmaxnreg_dec<88>();   // 4 warps x 80 registers released = 8 warps x 40 acquired above
-        if (warp == 8) {
+        if (kCompact && (warp == 8 || warp == 11)) {
+            // ================================ token-compacted mode: gather warps ================================
+            // Warp 8 fetches the K rows of each 128-key slice of the gathered list, warp 11 the V rows: 16-byte
+            // asynchronous copies into the 128-byte-swizzled tile layout (8 lanes per 128-byte half row, 4 rows per
+            // instruction; padding entries (-1) are zero-filled). Each lane's copies report to the stage's barrier.
+            const bool isK = warp == 8;
+            if (isK && lane == 0) {
+                mbar_arrive_expect_tx(&S.q_full, has1 ? 2 * kTileBytes : kTileBytes);
+                for (int w = 0; w < (has1 ? 2 : 1); ++w)
+                    for (int hf = 0; hf < 2; ++hf)
+                        tma_load_4d(&S.q[w][hf * (kTileBytes / 2)], &tmQ, &S.q_full, hf * 64, (qt0 + w) * 128, h, b);
+            }
+            const int* list = P.cidx + ((size_t)bh * npairs + pair) * P.ccap;
+            const __nv_bfloat16* src = (isK ? P.Kg : P.Vg) + (size_t)hk * 128 + (lane & 7) * 8;
+            const int rsub = lane >> 3;
+            const uint32_t sw0 = (uint32_t)(((lane & 7) ^ rsub) << 4), sw1 = (uint32_t)(((lane & 7) ^ (rsub + 4)) << 4);
+            int jrow[32];
+            if (n_iters > 0) {
+#pragma unroll
+                for (int q = 0; q < 32; ++q) jrow[q] = list[4 * q + rsub];
+            }
+            bool ok = true;
+            for (int it = 0; it < n_iters && ok; ++it) {
+                const int st = it % kStages;
+                uint64_t* empty = isK ? &S.k_empty[st] : &S.v_empty[st];
+                uint64_t* full = isK ? &S.k_full[st] : &S.v_full[st];
+                uint8_t* dst = (isK ? S.k[st] : S.v[st]) + rsub * 128;
+                if (it >= kStages) ok = mbar_wait_warp(empty, ((it / kStages) - 1) & 1, abort_flag);
+                if (!ok) break;
+#pragma unroll
+                for (int q = 0; q < 32; ++q) {
+                    const int j = jrow[q];
+                    const __nv_bfloat16* row = src + (size_t)(b * P.L + max(j, 0)) * P.Hkv * 128;
+                    uint8_t* d = dst + q * 512 + ((q & 1) ? sw1 : sw0);          // row r = 4q + rsub, chunk c ^ (r & 7)
+                    cp_async16(d, row, j >= 0 ? 16 : 0);
+                    cp_async16(d + kTileBytes / 2, row + 64, j >= 0 ? 16 : 0);
+                }
+                cp_async_arrive(full);
+                if (it + 1 < n_iters) {
+#pragma unroll
+                    for (int q = 0; q < 32; ++q) jrow[q] = list[(it + 1) * 128 + 4 * q + rsub];
+                }
+            }
+            for (int it = max(0, n_iters - kStages); it < n_iters && ok; ++it)
+                ok = mbar_wait_warp(isK ? &S.k_empty[it % kStages] : &S.v_empty[it % kStages], (it / kStages) & 1, abort_flag);
+        } else if (kCompact && warp == 10) {
+            // ================================ token-compacted mode: stager ================================
+            // Per 128-key slice and query tile: the B rows of the ninth k-step (bias / scale as three bf16 terms, or
+            // -BIG for a column that no row of the tile keeps; the A rows are constant ones), the key index and expiry
+            // vectors, and the mask of 32-column chunks that hold a key expiring or entering inside the tile's rows (only
+            // those need the per-element test). Two dependent levels of global loads, each issued a tile ahead.
+            constexpr uint32_t kOne = 0x3F80u, kNegBig = 0xF14Au;     // bf16 1.0 and about -1e30
+            for (int r = lane; r < 128; r += 32) {
+#pragma unroll
+                for (int w = 0; w < 2; ++w) {
+                    uint8_t* arow = S.aext[w] + (r >> 3) * 256 + (r & 7) * 16;
+                    *reinterpret_cast<uint4*>(arow) = make_uint4(kOne | (kOne << 16), kOne, 0u, 0u);
+                    *reinterpret_cast<uint4*>(arow + 128) = make_uint4(0u, 0u, 0u, 0u);
+                    *reinterpret_cast<uint4*>(S.bext[w] + (r >> 3) * 256 + (r & 7) * 16 + 128) = make_uint4(0u, 0u, 0u, 0u);
+                }
+            }
+            const int* list = P.cidx + ((size_t)bh * npairs + pair) * P.ccap;
+            auto vals = [&](const int (&jv)[4], float (&bv)[4], int (&ev)[4]) {
+#pragma unroll
+                for (int t = 0; t < 4; ++t) {
+                    bv[t] = jv[t] >= 0 ? P.bias[(size_t)bh * P.L + jv[t]] : 0.0f;
+                    ev[t] = jv[t] >= 0 ? P.expiry[(size_t)bh * P.L + jv[t]] : 0;
+                }
+            };
+            int jv[4] = {-1, -1, -1, -1}, jn[4] = {-1, -1, -1, -1}, ev[4] = {0, 0, 0, 0};
+            float bv[4] = {0.f, 0.f, 0.f, 0.f};
+            if (n_iters > 0) {
+#pragma unroll
+                for (int t = 0; t < 4; ++t) jv[t] = list[lane + 32 * t];
+                vals(jv, bv, ev);
+            }
+            if (n_iters > 1) {
+#pragma unroll
+                for (int t = 0; t < 4; ++t) jn[t] = list[128 + lane + 32 * t];
+            }
+            bool ok = true;
+            for (int it = 0; it < n_iters && ok; ++it) {
+                const int st = it % kStages;
+                float bn[4] = {0.f, 0.f, 0.f, 0.f};
+                int en[4] = {0, 0, 0, 0}, jnn[4] = {-1, -1, -1, -1};
+                if (it + 1 < n_iters) vals(jn, bn, en);
+                if (it + 2 < n_iters) {
+#pragma unroll
+                    for (int t = 0; t < 4; ++t) jnn[t] = list[(it + 2) * 128 + lane + 32 * t];
+                }
+                // rows and flags are formed in registers before the waits
+                uint32_t b0[2][4], b1[4], flags[2] = {0u, 0u};
+#pragma unroll
+                for (int t = 0; t < 4; ++t) {
+                    const float bsc = bv[t] * P.inv_scale;
+                    const __nv_bfloat16 hi = __float2bfloat16_rn(bsc);
+                    const float r1 = bsc - __bfloat162float(hi);
+                    const __nv_bfloat16 mid = __float2bfloat16_rn(r1);
+                    const __nv_bfloat16 lo = __float2bfloat16_rn(r1 - __bfloat162float(mid));
+                    const uint32_t w0 = (uint32_t)__bfloat16_as_ushort(hi) | ((uint32_t)__bfloat16_as_ushort(mid) << 16);
+                    b1[t] = (uint32_t)__bfloat16_as_ushort(lo);
+#pragma unroll
+                    for (int w = 0; w < 2; ++w) {
+                        const int i0 = (w ? qt1 : qt0) * 128;
+                        const bool dead = jv[t] < 0 || ev[t] <= i0 || jv[t] > i0 + 127;
+                        const bool mixed = !dead && (ev[t] < i0 + 128 || jv[t] > i0);
+                        b0[w][t] = dead ? kNegBig : w0;
+                        flags[w] |= __ballot_sync(0xffffffffu, mixed) ? (1u << t) : 0u;
+                    }
+                }
+                // the vectors of this stage were last read by the softmax groups before they released P of tile
+                // it - kStages (hence before its P V); the B rows were last read by the S products of tile it - 1
+                if (it >= kStages) ok = mbar_wait_warp(&S.v_empty[st], ((it / kStages) - 1) & 1, abort_flag);
+                if (ok && it >= 1) ok = mbar_wait_warp(&S.k_empty[(it - 1) % kStages], ((it - 1) / kStages) & 1, abort_flag);
+                if (!ok) break;
+#pragma unroll
+                for (int t = 0; t < 4; ++t) {
+                    const int c = lane + 32 * t;
+                    S.jidx[st][c] = jv[t] >= 0 ? jv[t] : 0x7fffffff;                   // padding: never <= a row index
+                    S.len[st][c] = ev[t];
+#pragma unroll
+                    for (int w = 0; w < 2; ++w)
+                        *reinterpret_cast<uint4*>(S.bext[w] + (c >> 3) * 256 + (c & 7) * 16) =
+                            make_uint4(b0[w][t], b0[w][t] == kNegBig ? 0u : b1[t], 0u, 0u);
+                    jv[t] = jn[t]; bv[t] = bn[t]; ev[t] = en[t]; jn[t] = jnn[t];
+                }
+                if (lane < 2) S.fast[st][lane] = lane ? flags[1] : flags[0];
+                fence_proxy_async();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&S.k_full[st]);
+            }
+        } else if (warp == 8) {
             // =========================================== producer ===========================================
             if (lane == 0) {
                 mbar_arrive_expect_tx(&S.q_full, has1 ? 2 * kTileBytes : kTileBytes);
@@ -391,37 +562,51 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             // only the stores are left between the previous S product and the next one.
             const int w = warp - 10;
             const int i0 = (w ? qt1 : qt0) * 128;
-            auto fetch = [&](int it, float (&bv)[4], int (&ev)[4]) {
+            // key indices of a tile's columns, then their bias and expiry, loaded one tile before they are needed
+            auto fetch_idx = [&](int it, int (&jv)[4]) {
                 const int j0 = (int)(S.sched[it] & 0xFFFFF) * 128;
 #pragma unroll
                 for (int t = 0; t < 4; ++t) {
-                    const int j = j0 + lane + 32 * t;
-                    bv[t] = j < P.L ? P.bias[(size_t)bh * P.L + j] : 0.0f;
-                    ev[t] = j < P.L ? P.expiry[(size_t)bh * P.L + j] : 0;
+                    jv[t] = j0 + lane + 32 * t;
+                }
+            };
+            auto fetch_vals = [&](const int (&jv)[4], float (&bv)[4], int (&ev)[4]) {
+#pragma unroll
+                for (int t = 0; t < 4; ++t) {
+                    const bool real = jv[t] >= 0 && jv[t] < P.L;
+                    bv[t] = real ? P.bias[(size_t)bh * P.L + jv[t]] : 0.0f;
+                    ev[t] = real ? P.expiry[(size_t)bh * P.L + jv[t]] : 0;
                 }
             };
             constexpr uint32_t kOne = 0x3F80u, kNegBig = 0xF14Au;     // bf16 1.0 and about -1e30
             float bv[4] = {0.f, 0.f, 0.f, 0.f};
-            int ev[4] = {0, 0, 0, 0};
-            if (n_iters > 0) fetch(0, bv, ev);
+            int ev[4] = {0, 0, 0, 0}, jv[4] = {0, 0, 0, 0}, jn[4] = {0, 0, 0, 0};
+            if (n_iters > 0) { fetch_idx(0, jv); fetch_vals(jv, bv, ev); }
+            if (n_iters > 1) fetch_idx(1, jn);
             bool ok = true;
             for (int it = 0; it < n_iters && ok; ++it) {
                 const int st = it % kStages;
                 const uint32_t entry = S.sched[it];
                 const bool use = use_bit(entry, w);
+#ifdef DMA_PROF
+                const long long ts_loop = clock64();
+#endif
                 float bn[4] = {0.f, 0.f, 0.f, 0.f};
-                int en[4] = {0, 0, 0, 0};
-                if (it + 1 < n_iters) fetch(it + 1, bn, en);
+                int en[4] = {0, 0, 0, 0}, jnn[4] = {0, 0, 0, 0};
+                if (it + 1 < n_iters) fetch_vals(jn, bn, en);
+                if (it + 2 < n_iters) fetch_idx(it + 2, jnn);
                 uint32_t b0[4], b1[4], aw[4][7];
                 int hot[4];
                 bool fast = false;
                 if (use) {
+                    // general path needed: the tile holds keys that enter inside the query tile's rows (the diagonal tile)
                     const bool diag = (int)(entry & 0xFFFFF) == (w ? qt1 : qt0);
                     uint32_t bal[4];
-                    bool mixed[4];
+                    bool mixed[4], dead[4];
 #pragma unroll
                     for (int t = 0; t < 4; ++t) {
-                        mixed[t] = ev[t] > i0 && ev[t] < i0 + 128;
+                        dead[t] = ev[t] <= i0;
+                        mixed[t] = !dead[t] && ev[t] < i0 + 128;
                         bal[t] = __ballot_sync(0xffffffffu, mixed[t]);
                     }
                     const int cnt = __popc(bal[0]) + __popc(bal[1]) + __popc(bal[2]) + __popc(bal[3]);
@@ -446,9 +631,8 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                         const float r1 = bs - __bfloat162float(hi);
                         const __nv_bfloat16 mid = __float2bfloat16_rn(r1);
                         const __nv_bfloat16 lo = __float2bfloat16_rn(r1 - __bfloat162float(mid));
-                        const bool dead = ev[t] <= i0;
-                        b0[t] = dead ? kNegBig : ((uint32_t)__bfloat16_as_ushort(hi) | ((uint32_t)__bfloat16_as_ushort(mid) << 16));
-                        b1[t] = (dead ? 0u : (uint32_t)__bfloat16_as_ushort(lo)) | (hot[t] == 3 ? (kNegBig << 16) : 0u);
+                        b0[t] = dead[t] ? kNegBig : ((uint32_t)__bfloat16_as_ushort(hi) | ((uint32_t)__bfloat16_as_ushort(mid) << 16));
+                        b1[t] = (dead[t] ? 0u : (uint32_t)__bfloat16_as_ushort(lo)) | (hot[t] == 3 ? (kNegBig << 16) : 0u);
                     }
                     // A rows (queries): ones for the bias terms, then one step function per expiring key
                     int th[kMaskSlots];
@@ -465,12 +649,21 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                 }
                 // fast[st] / len[st] were last read by the softmax groups before they released P of tile it - kStages
                 // (hence before its P V); the operand blocks were last read by the S products of tile it - 1
+#ifdef DMA_PROF
+                const long long ts0 = clock64();
+#endif
                 if (it >= kStages) ok = mbar_wait_warp(&S.v_empty[st], ((it / kStages) - 1) & 1, abort_flag);
                 if (ok && it >= 1) ok = mbar_wait_warp(&S.k_empty[(it - 1) % kStages], ((it - 1) / kStages) & 1, abort_flag);
+#ifdef DMA_PROF
+                const long long ts1 = clock64();
+                if (P.prof && blockIdx.x == 0 && blockIdx.y == 0 && lane == 0 && w == 0) { P.prof[24] += ts1 - ts0; P.prof[25] += ts0 - ts_loop; }
+#endif
                 if (!ok) break;
                 if (w == 0) {
 #pragma unroll
-                    for (int t = 0; t < 4; ++t) S.len[st][lane + 32 * t] = ev[t];
+                    for (int t = 0; t < 4; ++t) {
+                        S.len[st][lane + 32 * t] = ev[t];
+                    }
                 }
                 if (use) {
 #pragma unroll
@@ -494,10 +687,15 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                 for (int t = 0; t < 4; ++t) {
                     bv[t] = bn[t];
                     ev[t] = en[t];
+                    jv[t] = jn[t];
+                    jn[t] = jnn[t];
                 }
                 fence_proxy_async();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&S.k_full[st]);
+#ifdef DMA_PROF
+                if (P.prof && blockIdx.x == 0 && blockIdx.y == 0 && lane == 0 && w == 0) P.prof[26] += clock64() - ts1;
+#endif
             }
         } else if (warp == 9) {
             // =========================================== MMA issuer ===========================================
@@ -526,10 +724,17 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                 __syncwarp();
             };
             int n_p[2] = {0, 0};
+#ifdef DMA_PROF
+            long long iss_acc[4] = {0, 0, 0, 0};
+#define PROF_W(slot, expr) do { const long long t0_ = clock64(); expr; iss_acc[slot] += clock64() - t0_; } while (0)
+#else
+#define PROF_W(slot, expr) do { expr; } while (0)
+#endif
             bool ok = mbar_wait_warp(&S.q_full, 0, abort_flag);
             if (ok && n_iters_u > 0) {
                 ok = mbar_wait_warp(&S.k_full[0], 0, abort_flag);
                 if (ok) {
+                    if constexpr (kCompact) fence_proxy_async();
                     tc_fence_after();
                     const uint32_t e0 = __shfl_sync(0xffffffffu, S.sched[0], 0);
 #pragma unroll
@@ -543,7 +748,8 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                 const int st = it % kStages, nst = (it + 1) % kStages;
                 const uint32_t entry = __shfl_sync(0xffffffffu, S.sched[it], 0);
                 const uint32_t next = it + 1 < n_iters_u ? __shfl_sync(0xffffffffu, S.sched[it + 1], 0) : 0u;
-                ok = mbar_wait_warp(&S.v_full[st], (it / kStages) & 1, abort_flag);
+                PROF_W(0, ok = mbar_wait_warp(&S.v_full[st], (it / kStages) & 1, abort_flag));
+                if constexpr (kCompact) fence_proxy_async();     // the gathered tiles were written through the generic proxy
                 bool k_ready = false;
 #pragma unroll
                 for (int w = 0; w < 2; ++w) {          // unrolled: n_p[] stays in registers
@@ -552,7 +758,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                         const uint64_t dv = dV0 + (uint64_t)(st * (kTileBytes >> 4));
                         const uint32_t d_tmem = tmem_u + 256 + w * 128, a_tmem = tmem_u + w * 128;
                         const uint32_t acc0 = n_p[w] > 0 ? 1u : 0u;
-                        ok = mbar_wait_warp(&S.p_half[w], n_p[w] & 1, abort_flag);
+                        PROF_W(2 + w, ok = mbar_wait_warp(&S.p_half[w], n_p[w] & 1, abort_flag));
                         if (ok) {
                             tc_fence_after();
                             if (elect_one()) {
@@ -578,7 +784,8 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                     }
                     if (ok && use_bit(next, w)) {
                         if (!k_ready) {
-                            ok = mbar_wait_warp(&S.k_full[nst], ((it + 1) / kStages) & 1, abort_flag);
+                            PROF_W(1, ok = mbar_wait_warp(&S.k_full[nst], ((it + 1) / kStages) & 1, abort_flag));
+                            if constexpr (kCompact) fence_proxy_async();
                             if (ok) tc_fence_after();
                             k_ready = true;
                         }
@@ -594,6 +801,9 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                     __syncwarp();
                 }
             }
+#ifdef DMA_PROF
+            if (P.prof && blockIdx.x == 0 && blockIdx.y == 0 && lane == 0) for (int k = 0; k < 4; ++k) P.prof[16 + k] = iss_acc[k];
+#endif
         }
     }
     // teardown: every role falls through to here, also after a timed-out wait
@@ -645,17 +855,66 @@ int make_tmap_f32_rows(CUtensorMap* m, const void* base, int B, int L, int H, in
     return r == CUDA_SUCCESS ? DMA_OK : DMA_ERR_CUDA;
 }
 
-size_t tc_fwd_ws_bytes(const Prob&) { return kWsHeaderBytes; }
+// Token-compacted mode, per (batch, head, pair of query tiles): the ascending list of keys j that some row i of the
+// pair's 256 rows keeps, i.e. j <= i < expiry[j] for some i in [i0, i0 + 255]  <=>  j <= i0 + 255 and expiry[j] > max(i0, j).
+// At most w + 256 keys qualify. One warp per list: 32 keys per pass, ballot + popcount keep the order; the list is
+// padded with -1 to the next multiple of 128.
+__global__ void compact_lists_kernel(const int32_t* __restrict__ expiry, int* __restrict__ cidx, int* __restrict__ ccnt,
+                                     int L, int npairs, int cap, int nlists) {
+    const int list = blockIdx.x * (blockDim.x / 32) + threadIdx.x / 32, lane = threadIdx.x % 32;
+    if (list >= nlists) return;
+    const int bh = list / npairs, pair = list % npairs, i0 = pair * 256;
+    const int32_t* e = expiry + (size_t)bh * L;
+    int* out = cidx + (size_t)list * cap;
+    const int jend = min(L, i0 + 256);
+    int n = 0;
+    for (int base = 0; base < jend; base += 32) {
+        const int j = base + lane;
+        const bool keep = j < jend && e[j] > max(i0, j);
+        const uint32_t bal = __ballot_sync(0xffffffffu, keep);
+        const int pos = n + __popc(bal & ((1u << lane) - 1));
+        if (keep && pos < cap) out[pos] = j;
+        n += __popc(bal);
+    }
+    n = min(n, cap);
+    for (int t = n + lane; t < ((n + 127) / 128) * 128 && t < cap; t += 32) out[t] = -1;
+    if (lane == 0) ccnt[list] = n;
+}
+
+static int compact_cap(const Prob& P) { return ((P.w + 256 + 127) / 128) * 128; }
+static size_t compact_lists(const Prob& P) { return (size_t)P.B * P.Hq * ((P.Tr + 1) / 2); }
+
+size_t tc_fwd_ws_bytes(const Prob& P) {
+    if (!(P.flags & DMA_FLAG_COMPACT_KV)) return kWsHeaderBytes;
+    const size_t cnt_bytes = ((compact_lists(P) * sizeof(int) + 255) / 256) * 256;
+    return kWsHeaderBytes + cnt_bytes + compact_lists(P) * compact_cap(P) * sizeof(int);
+}
 
 int launch_tc_fwd(const Prob& P, const void* Q, const void* K, const void* V, const float* bias,
                   const int32_t* expiry, const uint32_t* bitmap, void* O, float* lse, void* ws, cudaStream_t st) {
+    const bool compact = (P.flags & DMA_FLAG_COMPACT_KV) != 0;
     if (P.Tc > kMaxSched) return DMA_ERR_UNSUPPORTED;
     CUtensorMap tmQ, tmK, tmV;
     int rc;
     if ((rc = make_tmap_bf16(&tmQ, Q, P.B, P.L, P.Hq, P.d, P.qs, 128))) return rc;
+    FwdParams fp;
+    fp.cidx = nullptr; fp.ccnt = nullptr; fp.ccap = 0; fp.Hkv = P.Hkv;
+    if (compact) {
+        // the gathers address K and V as plain row arrays: contiguous [B, L, Hkv, 128] only
+        const int64_t want[3] = {(int64_t)P.L * P.Hkv * P.d, (int64_t)P.Hkv * P.d, P.d};
+        for (int t = 0; t < 3; ++t)
+            if (P.ks[t] != want[t] || P.vs[t] != want[t]) return DMA_ERR_UNSUPPORTED;
+        if (compact_cap(P) / 128 > kMaxSched) return DMA_ERR_UNSUPPORTED;
+        const size_t nl = compact_lists(P);
+        int* ccnt = reinterpret_cast<int*>((char*)ws + kWsHeaderBytes);
+        int* cidx = reinterpret_cast<int*>((char*)ws + kWsHeaderBytes + ((nl * sizeof(int) + 255) / 256) * 256);
+        compact_lists_kernel<<<(unsigned)((nl + 3) / 4), 128, 0, st>>>(expiry, cidx, ccnt, P.L, (P.Tr + 1) / 2, compact_cap(P), (int)nl);
+        count_launch();
+        fp.cidx = cidx; fp.ccnt = ccnt; fp.ccap = compact_cap(P);
+    }
+    fp.Kg = (const __nv_bfloat16*)K; fp.Vg = (const __nv_bfloat16*)V;
     if ((rc = make_tmap_bf16(&tmK, K, P.B, P.L, P.Hkv, P.d, P.ks, 128))) return rc;
     if ((rc = make_tmap_bf16(&tmV, V, P.B, P.L, P.Hkv, P.d, P.vs, 128))) return rc;
-    FwdParams fp;
     fp.bias = bias; fp.expiry = expiry; fp.bitmap = bitmap; fp.O = (__nv_bfloat16*)O; fp.lse = lse;
     fp.status = (int32_t*)ws;
     fp.B = P.B; fp.Hq = P.Hq; fp.G = P.G; fp.L = P.L; fp.Tr = P.Tr; fp.Tc = P.Tc; fp.Wd = P.Wd;
@@ -669,9 +928,14 @@ int launch_tc_fwd(const Prob& P, const void* Q, const void* K, const void* V, co
     fp.prof = prof_env ? (long long*)strtoull(prof_env, nullptr, 10) : nullptr;
 #endif
     const size_t smem = sizeof(SharedStorage) + 1024;
-    if (cudaFuncSetAttribute(fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return DMA_ERR_CUDA;
     dim3 grid(P.B * P.Hq, (P.Tr + 1) / 2);
-    fwd_kernel<<<grid, kThreads, smem, st>>>(tmQ, tmK, tmV, fp);
+    if (compact) {
+        if (cudaFuncSetAttribute(fwd_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return DMA_ERR_CUDA;
+        fwd_kernel<true><<<grid, kThreads, smem, st>>>(tmQ, tmK, tmV, fp);
+    } else {
+        if (cudaFuncSetAttribute(fwd_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return DMA_ERR_CUDA;
+        fwd_kernel<false><<<grid, kThreads, smem, st>>>(tmQ, tmK, tmV, fp);
+    }
     count_launch();
     return check_launch();
 }

@@ -8,7 +8,7 @@ import oracle
 from paper_2508_02124_b200 import binding as dma
 from paper_2508_02124_b200 import workloads as wl
 
-from helpers import assert_close, f64, gpu_run, oracle_mask, round_to
+from helpers import assert_close, f64, gpu_run, oracle_mask, problem_of, round_to
 
 pytestmark = pytest.mark.gpu
 
@@ -96,7 +96,7 @@ def test_skipped_tiles_do_not_change_the_result_on_a_banded_mask():
     compare(case, gpu_run(case, inp, flags=dma.DMA_FLAG_IGNORE_BITMAP), ref)
 
 
-def sampled_check(case, inp, got, nrows=24, nkeys=6, seed=0):
+def sampled_check(case, inp, got, nrows=24, nkeys=6, seed=0, forward_only=False):
     """Full-size parity on sampled outputs: query rows (O, lse, dQ) and keys (dK, dV, dM) that the oracle
     evaluates one by one. Keys are sampled near the end of the sequence, where few rows can keep them."""
     rng = np.random.default_rng(seed)
@@ -107,7 +107,7 @@ def sampled_check(case, inp, got, nrows=24, nkeys=6, seed=0):
     O, lse = oracle.forward(Q, K, V, dl.astype(np.float64), expiry=e, rows=rows)
     assert_close(got["O"][:, rows], O, case.dtype, "O rows")
     assert_close(got["lse"][:, :, rows], lse, case.dtype, "lse rows", lse=True)
-    if not case.backward:
+    if forward_only or not case.backward:
         return
     keys = np.unique(np.concatenate([[L - 1, L - 130], rng.integers(L - 600, L, nkeys)])).astype(np.int32)
     tail = np.arange(L - 600, L, dtype=np.int32)               # the only rows that can keep those keys
@@ -165,3 +165,53 @@ def test_bounded_wait_reports_timeout_and_context_survives():
     inp = wl.make_inputs(case)
     got = gpu_run(case, inp, backward=False)
     assert torch.isfinite(got["O"].float()).all()
+
+
+# ---- token-compacted forward (DMA_FLAG_COMPACT_KV): same results as the oracle, from the gathered key lists ----------
+
+def _compact_run(case, inp):
+    dev = torch.device("cuda:0")
+    p = problem_of(case)
+    pc = problem_of(case, flags=dma.DMA_FLAG_COMPACT_KV)
+    Q, K, V = (inp[k].to(dev) for k in ("Q", "K", "V"))
+    bias, expiry, bitmap = dma.dma_mask_build(p, V, inp["W_delta"].to(dev), inp["A"].to(dev))
+    ws = torch.empty(dma.dma_query_workspace(pc)[1], dtype=torch.uint8, device=dev)
+    O, lse = dma.dma_attn_fwd(pc, Q, K, V, bias, expiry, bitmap, ws=ws)
+    torch.cuda.synchronize()
+    assert dma.dma_read_status(ws) == 0
+    return {"bias": bias, "expiry": expiry, "bitmap": bitmap, "O": O, "lse": lse}
+
+
+@pytest.mark.parametrize("kw", [
+    dict(B=1, Hq=2, Hkv=1, L=384, w=64),            # ragged pair count (3 query tiles), small window
+    dict(B=2, Hq=4, Hkv=2, L=1000, w=200),          # ragged tail rows, GQA
+    dict(B=1, Hq=2, Hkv=2, L=1536, w=2000),         # w >= L: every causal key is gathered (dense causal attention)
+    dict(B=1, Hq=4, Hkv=1, L=2048, w=1),            # w = 1: one key per row
+])
+def test_compact_forward_small_cases(kw):
+    case = wl.small(C2, name="compact-small", backward=False, **kw)
+    inp = wl.make_inputs(case)
+    got = _compact_run(case, inp)
+    e = got["expiry"].cpu().numpy()
+    ref = oracle.forward(inp["Q"].double().numpy(), inp["K"].double().numpy(), inp["V"].double().numpy(),
+                         got["bias"].double().cpu().numpy(), expiry=e, scale=case.d ** -0.5)
+    assert_close(got["O"], round_to(case, ref[0]), case.dtype, "compact O")
+    assert_close(got["lse"], ref[1], case.dtype, "compact lse", lse=True)
+
+
+@pytest.mark.parametrize("key", ["3", "S", "5"])
+def test_compact_forward_full_size_sampled(key):
+    case = wl.CONFIGS[key]
+    inp = wl.make_inputs(case)
+    got = _compact_run(case, inp)
+    sampled_check(case, inp, got, forward_only=True)
+
+
+def test_compact_flag_is_rejected_where_unsupported():
+    dev = torch.device("cuda:0")
+    case = wl.small(C2, B=1, Hq=2, Hkv=1, L=256, w=64, d=64, name="compact-d64")
+    inp = wl.make_inputs(case)
+    p = problem_of(case, flags=dma.DMA_FLAG_COMPACT_KV)
+    with pytest.raises(dma.DmaError) as e:
+        gpu_run(case, inp, backward=False, flags=dma.DMA_FLAG_COMPACT_KV)
+    assert e.value.status == -4
