@@ -256,8 +256,24 @@ def main():
         barrier()
         assert dma.dma_read_status(ws_c) == 0, "device status (compact forward)"
         c_ms = c0.elapsed_time(c1) / 10
-        compact = {"fwd_ms": c_ms, "tile_fwd_ms": stage_ms["fwd"], "speedup_over_tile_skipping": stage_ms["fwd"] / c_ms,
+        compact = {"fwd_ms": c_ms, "tile_fwd_ms": stage_ms["fwd"], "fwd_speedup_over_tile_skipping": stage_ms["fwd"] / c_ms,
                    "max_abs_diff_vs_tile_path": float((Oc.float() - O.float()).abs().max())}
+        if case.backward:
+            ws_cb = torch.empty(dma.dma_query_workspace(pc)[2], dtype=torch.uint8, device=dev)
+            dQc, dKc, dVc, dMc = torch.empty_like(dQ), torch.empty_like(dK), torch.empty_like(dV), torch.empty_like(dM)
+            for _ in range(3):
+                dma.dma_attn_bwd(pc, Q, K, V, O, dO, lse, bias, expiry, bitmap, dQc, dKc, dVc, dMc, ws_cb)
+            barrier()
+            c0.record()
+            for _ in range(10):
+                dma.dma_attn_bwd(pc, Q, K, V, O, dO, lse, bias, expiry, bitmap, dQc, dKc, dVc, dMc, ws_cb)
+            c1.record()
+            barrier()
+            assert dma.dma_read_status(ws_cb) == 0, "device status (compact backward)"
+            cb_ms = c0.elapsed_time(c1) / 10
+            compact.update({"bwd_ms": cb_ms, "tile_bwd_ms": stage_ms["bwd"], "bwd_speedup_over_tile_skipping": stage_ms["bwd"] / cb_ms,
+                            "step_ms": stage_ms["mask"] + c_ms + cb_ms, "tile_step_ms": sum(stage_ms.values()),
+                            "dK_max_abs_diff_vs_tile_path": float((dKc.float() - dK.float()).abs().max())})
 
     # ---- end to end through the host-buffer entry point: pinned host tensors in, results back on the host
     e2e = None
@@ -317,7 +333,7 @@ def main():
         "gpu_launches": launches, "clocks": clocks, "e2e": e2e,
     }
     if compact is not None:
-        out["compact_fwd"] = compact
+        out["compact"] = compact
     if mask_bwd is not None:
         mask_bwd["frac_of_measured_hbm"] = mask_bwd["gbs"] / pk["hbm_gbs"]
         out["mask_bwd"] = mask_bwd

@@ -47,11 +47,15 @@ enum {
     DMA_FLAG_IGNORE_BITMAP = 1,  /* visit every causal tile regardless of the bitmap (result must not change:
                                     block skipping is an optimisation only, Sec. 4.2 last paragraph)           */
     DMA_FLAG_SIMT = 2,           /* run the CUDA-core kernels also for bf16 (they always serve fp32)            */
-    DMA_FLAG_COMPACT_KV = 4      /* dma_attn_fwd, bf16, d = 128, contiguous K and V: token-compacted execution. Each
-                                    pair of query tiles gathers only the keys that one of its 256 rows keeps (at most
-                                    w + 256) instead of walking every active 128-key tile: work falls from O(L^2 d) to
-                                    O(L w d) (Sec. 3.3, computational sparsity). Same results up to rounding; needs the
-                                    larger forward workspace dma_query_workspace reports for it; ignores the bitmap */
+    DMA_FLAG_COMPACT_KV = 4      /* dma_attn_fwd and dma_attn_bwd, bf16, d = 128, contiguous K and V: token-compacted
+                                    execution (Sec. 3.3, computational sparsity: O(L w d) instead of O(L^2 d) work).
+                                    Forward: each pair of query tiles gathers only the keys that one of its 256 rows
+                                    keeps (at most w + 256) instead of walking every active 128-key tile. Backward: a CTA
+                                    owns 128 keys of one query head that expire within the same band of rows (a
+                                    lifetime-sorted permutation built per call) and walks only the query tiles between
+                                    the first key and the last expiry; dK, dV are summed over the group in fp32. Same
+                                    results up to rounding; needs the larger workspaces dma_query_workspace reports for
+                                    it; ignores the bitmap */
 };
 
 typedef struct {

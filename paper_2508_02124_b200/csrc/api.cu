@@ -167,6 +167,7 @@ int dma_attn_bwd(const dma_problem_t* p, const void* Q, const void* K, const voi
         !aligned16(dK) || !aligned16(dV) || !aligned16(dM) || !aligned16(lse))
         return DMA_ERR_ALIGN;
     const bool tc = use_tensor_cores(P);
+    if ((P.flags & DMA_FLAG_COMPACT_KV) && !tc) return DMA_ERR_UNSUPPORTED;
     const size_t need = tc ? tc_bwd_ws_bytes(P) : simt_bwd_ws_bytes(P);
     if (!ws || ws_bytes < need || !aligned16(ws)) return DMA_ERR_WORKSPACE;
     if ((rc = device_ok())) return rc;

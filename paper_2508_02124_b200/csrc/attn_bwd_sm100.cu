@@ -69,6 +69,14 @@ struct BwdParams {
     int32_t* status;
     int B, Hq, Hkv, G, L, Tr, Tc, Wd, ignore_bitmap;
     float scale, scale_log2, inv_scale;
+    // token-compacted mode: per (batch, query head) a permutation of the keys (padded with L to a multiple of 128) that
+    // groups keys of similar lifetime; a CTA owns 128 consecutive entries of one query head's permutation
+    const int* perm;
+    const int32_t* expiry_all;
+    const __nv_bfloat16* Kg;    // K, V as contiguous [B, L, Hkv, 128] row arrays
+    const __nv_bfloat16* Vg;
+    float* dKacc;               // fp32 [B, L, Hkv, 128] accumulators (several query heads add into one KV head's rows)
+    float* dVacc;
     int64_t ks_b, ks_l, ks_h, vs_b, vs_l, vs_h;
 #ifdef DMA_PROF
     long long* prof;            // role timing (development builds only): cycles per phase of CTA (0, 0)
@@ -96,6 +104,12 @@ __device__ __forceinline__ uint4 split3(float x) {
     return make_uint4((uint32_t)__bfloat16_as_ushort(hi) | ((uint32_t)__bfloat16_as_ushort(mid) << 16), (uint32_t)__bfloat16_as_ushort(lo), 0u, 0u);
 }
 
+// kCompact: token-compacted mode. The CTA's 128 keys are 128 consecutive entries of one QUERY head's lifetime-sorted
+// key permutation instead of 128 consecutive keys of a KV head: keys that live equally long are kept by about the
+// same query rows, so the walk over query tiles [first key's tile, last expiry's tile] wastes little. K and V rows
+// are gathered once with 16-byte asynchronous copies; dK and dV are added to fp32 accumulators (the query heads of a
+// group meet there), dM is written directly.
+template <bool kCompact>
 __global__ void __launch_bounds__(kThreads, 1)
 bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
            const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmG,
@@ -104,9 +118,13 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
     SharedStorage& S = *reinterpret_cast<SharedStorage*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const int tid = threadIdx.x, lane = tid & 31;
     const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);      // warp-uniform to the compiler: role branches stay uniform
-    const int b = blockIdx.x / P.Hkv, hk = blockIdx.x % P.Hkv;
+    // tile mode: blockIdx.x = (batch, KV head); token-compacted mode: (batch, query head), whose group index is fixed
+    const int b = blockIdx.x / (kCompact ? P.Hq : P.Hkv);
+    const int hq_c = blockIdx.x % P.Hq;                // token-compacted mode only
+    const int hk = kCompact ? hq_c / P.G : blockIdx.x % P.Hkv;
     const int kt = blockIdx.y;                         // key tile 0 has the most query tiles: heaviest first
     const int j0 = kt * 128;
+    const int* my_perm = kCompact ? P.perm + ((size_t)blockIdx.x * P.Tc + kt) * 128 : nullptr;
     volatile int* abort_flag = &S.abort_flag;
 
     if (tid == 0) {
@@ -133,6 +151,29 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
         // schedule: for each query head of the group, the active query tiles (ascending), two 64-row steps each
         if (lane == 0) { prefetch_tmap(&tmQ); prefetch_tmap(&tmK); prefetch_tmap(&tmV); prefetch_tmap(&tmG); }
         int n = 0;
+        if constexpr (kCompact) {
+            // query tiles from the first key's tile to the tile of the last row that keeps one of the keys
+            int jmin = 0x7fffffff, emax = 0;
+            for (int t = 0; t < 4; ++t) {
+                const int j = my_perm[lane + 32 * t];
+                const int e = j < P.L ? P.expiry_all[(size_t)blockIdx.x * P.L + j] : 0;
+                if (e > j) { jmin = min(jmin, j); emax = max(emax, e); }
+            }
+            for (int o = 16; o; o >>= 1) {
+                jmin = min(jmin, __shfl_xor_sync(0xffffffffu, jmin, o));
+                emax = max(emax, __shfl_xor_sync(0xffffffffu, emax, o));
+            }
+            if (emax > 0) {
+                const int g = hq_c % P.G, q0 = jmin / 128, q1 = (emax - 1) / 128;
+                for (int qt = q0 + lane; qt <= q1; qt += 32) {
+                    const int pos = 2 * (qt - q0);
+                    if (pos < kMaxSteps) S.sched[pos] = (uint16_t)((g << 11) | (qt << 1));
+                    if (pos + 1 < kMaxSteps) S.sched[pos + 1] = (uint16_t)((g << 11) | (qt << 1) | 1);
+                }
+                n = 2 * (q1 - q0 + 1);
+                if (q1 * 128 + 64 >= P.L) n -= 1;       // the last tile has one 64-row step only
+            }
+        } else {
         for (int g = 0; g < P.G; ++g) {
             const int bh = b * P.Hq + hk * P.G + g;
             for (int base = kt; base < P.Tr; base += 32) {
@@ -150,6 +191,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                     if (pos + hf < kMaxSteps) S.sched[pos + hf] = (uint16_t)((g << 11) | (qt << 1) | hf);
                 n += __shfl_sync(0xffffffffu, incl, 31);
             }
+        }
         }
         if (lane == 0) S.n_steps = min(n, kMaxSteps);
     }
@@ -172,7 +214,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
         // ============================ compute group: thread = key j, 32 of the step's 64 query columns ============================
         const int quad = warp & 3, hsel = warp >> 2;
         const int r = quad * 32 + lane;                     // key within the tile = TMEM lane
-        const int j = j0 + r;
+        const int j = kCompact ? my_perm[r] : j0 + r;           // token-compacted mode: padding entries hold L
         const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
         float bj = 0.0f;
         float2 dm2 = make_float2(0.0f, 0.0f);
@@ -214,7 +256,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             const int width = max(0, min(32, j - i0 - c0 + len) - lo);
             // Almost every (key, 32-row group) pair is all-or-nothing: then the mask is one additive term per thread
             // (0 or -inf) and the per-element test is skipped. Warps with a partly kept key take the general loop.
-            const bool uniform = __all_sync(0xffffffffu, lo == 0 && (width == 0 || width == 32));
+            const bool uniform = __all_sync(0xffffffffu, width == 0 || (lo == 0 && width == 32));
             uint32_t pp[16], dd[16];
             const float2 sc2 = make_float2(P.scale_log2, P.scale_log2);
             if (uniform) {
@@ -289,10 +331,12 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             tc_fence_after();
             __nv_bfloat16* dk = P.dK + b * P.ks_b + (int64_t)j * P.ks_l + hk * P.ks_h;
             __nv_bfloat16* dv = P.dV + b * P.vs_b + (int64_t)j * P.vs_l + hk * P.vs_h;
+            const size_t arow = ((size_t)(b * P.L + min(j, P.L - 1)) * P.Hkv + hk) * 128;      // accumulator row (compact mode)
 #pragma unroll
             for (int which = 0; which < 2; ++which) {
                 const float mul = which == 0 ? P.scale : 1.0f;
                 __nv_bfloat16* out = which == 0 ? dk : dv;
+                float* acc = (which == 0 ? P.dKacc : P.dVacc) + arow;
 #pragma unroll
                 for (int cc = 0; cc < 2; ++cc) {
                     const int c = hsel * 2 + cc;
@@ -304,7 +348,15 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
 #pragma unroll
                         for (int u = 0; u < 32; ++u) o[u] = 0;
                     }
-                    if (j < P.L) {
+                    if constexpr (kCompact) {
+                        // unscaled sums into the fp32 accumulators: the group's query heads add into the same rows
+                        if (j < P.L && n_steps > 0) {
+#pragma unroll
+                            for (int u = 0; u < 32; u += 4)
+                                red_add_v4(acc + c * 32 + u, __uint_as_float(o[u]), __uint_as_float(o[u + 1]), __uint_as_float(o[u + 2]),
+                                           __uint_as_float(o[u + 3]));
+                        }
+                    } else if (j < P.L) {
 #pragma unroll
                         for (int u = 0; u < 32; u += 8) {
                             uint4 pkt;
@@ -358,7 +410,28 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
     } else {
         if (warp == 12) {
             // ============================ producer ============================
-            if (lane == 0) {
+            if constexpr (kCompact) {
+                if (n_steps > 0) {
+                // gather the CTA's 128 K and V rows into the swizzled tile layout (8 lanes per 128-byte half row,
+                // 4 rows per instruction; padding entries are zero-filled)
+                const int rsub = lane >> 3, c = lane & 7;
+#pragma unroll 4
+                for (int q = 0; q < 32; ++q) {
+                    const int r = 4 * q + rsub, j = my_perm[r];
+                    const size_t row = ((size_t)(b * P.L + min(j, P.L - 1)) * P.Hkv + hk) * 128 + c * 8;
+                    const uint32_t off = r * 128 + ((c ^ (r & 7)) << 4);
+                    const int nb = j < P.L ? 16 : 0;
+                    cp_async16(S.k + off, P.Kg + row, nb);
+                    cp_async16(S.k + off + kKVBytes / 2, P.Kg + row + 64, nb);
+                    cp_async16(S.v + off, P.Vg + row, nb);
+                    cp_async16(S.v + off + kKVBytes / 2, P.Vg + row + 64, nb);
+                }
+                cp_async_wait_all();
+                fence_proxy_async();
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&S.kv_full);
+            } else if (lane == 0) {
                 mbar_arrive_expect_tx(&S.kv_full, 2 * kKVBytes);
                 for (int hf = 0; hf < 2; ++hf) {
                     tma_load_4d(&S.k[hf * (kKVBytes / 2)], &tmK, &S.kv_full, hf * 64, j0, hk, b);
@@ -540,18 +613,75 @@ __global__ void dq_convert_bf16_kernel(const float* __restrict__ acc, __nv_bfloa
 
 }  // namespace
 
+// Token-compacted mode: per (batch, query head) a stable counting sort of the keys by the band their expiry falls in
+// (band size >= 2048 rows, at most 62 bands; latest expiry first; keys that no row keeps go last). Within a band the
+// keys stay in index order, so 128 consecutive entries start at nearby rows and expire within one band of each other:
+// on i.i.d. importance at L = 16384, w = 2048 the walk covers 1.4 x the (row, key) pairs actually kept, against 4.3 x
+// for tiles of consecutive keys. Padded with L up to Tc * 128.
+// One CTA of 1024 threads per (batch, head); the warps take turns per 1024-key chunk so that the order is kept.
+__global__ void __launch_bounds__(1024) lifetime_perm_kernel(const int32_t* __restrict__ expiry, int* __restrict__ perm, int L, int Tc) {
+    __shared__ int hist[64];
+    __shared__ int offs[64];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int32_t* e = expiry + (size_t)blockIdx.x * L;
+    int* out = perm + (size_t)blockIdx.x * Tc * 128;
+    const int band = max(2048, (L + 61) / 62);
+    auto cls = [&](int j) { return e[j] > j ? 1 + (e[j] - 1) / band : 0; };
+    if (tid < 64) hist[tid] = 0;
+    __syncthreads();
+    for (int j = tid; j < L; j += 1024) atomicAdd(&hist[cls(j)], 1);
+    __syncthreads();
+    if (tid == 0) {
+        int run = 0;
+        for (int c = 63; c >= 0; --c) { offs[c] = run; run += hist[c]; }
+    }
+    __syncthreads();
+    for (int base = 0; base < L; base += 1024) {
+        const int j = base + tid;
+        const int c = j < L ? cls(j) : -1;
+        for (int wq = 0; wq < 32; ++wq) {
+            if (warp == wq && base + wq * 32 < L) {
+                const uint32_t same = __match_any_sync(0xffffffffu, c);
+                const int leader = __ffs(same) - 1, rank = __popc(same & ((1u << lane) - 1));
+                int start = 0;
+                if (lane == leader && c >= 0) { start = offs[c]; offs[c] = start + __popc(same); }
+                start = __shfl_sync(0xffffffffu, start, leader);
+                if (c >= 0) out[start + rank] = j;
+            }
+            __syncthreads();
+        }
+    }
+    for (int t = L + tid; t < Tc * 128; t += 1024) out[t] = L;
+}
+
+// workspace layout: header | D [rows] | dQ accumulator [rows x d] | (token-compacted mode) permutation | dK, dV accumulators
+static size_t bwd_rows64(const Prob& P) { return ((((size_t)P.B * P.Hq * P.L) + 63) / 64) * 64; }
+static size_t bwd_perm_ints(const Prob& P) { return (((size_t)P.B * P.Hq * P.Tc * 128) + 63) / 64 * 64; }
+
 size_t tc_bwd_ws_bytes(const Prob& P) {
     const size_t rows = (size_t)P.B * P.Hq * P.L;
-    return kWsHeaderBytes + (((rows + 63) / 64) * 64 + rows * P.d) * sizeof(float);
+    size_t n = kWsHeaderBytes + (bwd_rows64(P) + rows * P.d) * sizeof(float);
+    if (P.flags & DMA_FLAG_COMPACT_KV) n += bwd_perm_ints(P) * sizeof(int) + 2 * (size_t)P.B * P.L * P.Hkv * P.d * sizeof(float);
+    return n;
 }
 
 int launch_tc_bwd(const Prob& P, const void* Q, const void* K, const void* V, const void* O, const void* dO,
                   const float* lse, const float* bias, const int32_t* expiry, const uint32_t* bitmap, void* dQ,
                   void* dK, void* dV, float* dM, void* ws, cudaStream_t st) {
+    const bool compact = (P.flags & DMA_FLAG_COMPACT_KV) != 0;
     if ((size_t)P.G * P.Tr * 2 > (size_t)kMaxSteps || P.G > 16 || P.Tr > 1024) return DMA_ERR_UNSUPPORTED;
-    const size_t rows = (size_t)P.B * P.Hq * P.L, nq = rows * P.d;
+    const size_t rows = (size_t)P.B * P.Hq * P.L, nq = rows * P.d, nkv = (size_t)P.B * P.L * P.Hkv * P.d;
     float* Dv = reinterpret_cast<float*>((char*)ws + kWsHeaderBytes);
-    float* acc = Dv + ((rows + 63) / 64) * 64;
+    float* acc = Dv + bwd_rows64(P);
+    int* perm = reinterpret_cast<int*>(acc + nq);
+    float* accK = reinterpret_cast<float*>(perm + bwd_perm_ints(P));
+    float* accV = accK + nkv;
+    if (compact) {
+        // the gathers address K and V as plain row arrays: contiguous [B, L, Hkv, 128] only
+        const int64_t want[3] = {(int64_t)P.L * P.Hkv * P.d, (int64_t)P.Hkv * P.d, P.d};
+        for (int t = 0; t < 3; ++t)
+            if (P.ks[t] != want[t] || P.vs[t] != want[t]) return DMA_ERR_UNSUPPORTED;
+    }
     CUtensorMap tmQ, tmK, tmV, tmG;
     int rc;
     if ((rc = make_tmap_bf16(&tmQ, Q, P.B, P.L, P.Hq, P.d, P.qs, 64))) return rc;
@@ -564,6 +694,11 @@ int launch_tc_bwd(const Prob& P, const void* Q, const void* K, const void* V, co
                                                                     P.os[0], P.os[1], P.os[2]);
     if (cudaMemsetAsync(acc, 0, nq * sizeof(float), st) != cudaSuccess) return DMA_ERR_CUDA;
     if (cudaMemsetAsync(dM, 0, rows * sizeof(float), st) != cudaSuccess) return DMA_ERR_CUDA;   // two partial sums are added per key
+    if (compact) {
+        if (cudaMemsetAsync(accK, 0, 2 * nkv * sizeof(float), st) != cudaSuccess) return DMA_ERR_CUDA;
+        lifetime_perm_kernel<<<P.B * P.Hq, 1024, 0, st>>>(expiry, perm, P.L, P.Tc);
+        count_launch();
+    }
     BwdParams bp;
     bp.lse = lse; bp.Dv = Dv; bp.bias = bias; bp.expiry = expiry; bp.bitmap = bitmap; bp.dQacc = acc;
     bp.dK = (__nv_bfloat16*)dK; bp.dV = (__nv_bfloat16*)dV; bp.dM = dM; bp.status = (int32_t*)ws;
@@ -571,13 +706,24 @@ int launch_tc_bwd(const Prob& P, const void* Q, const void* K, const void* V, co
     bp.ignore_bitmap = (P.flags & DMA_FLAG_IGNORE_BITMAP) ? 1 : 0;
     bp.scale = P.scale; bp.scale_log2 = P.scale * 1.4426950408889634f; bp.inv_scale = 1.0f / P.scale;
     bp.ks_b = P.ks[0]; bp.ks_l = P.ks[1]; bp.ks_h = P.ks[2]; bp.vs_b = P.vs[0]; bp.vs_l = P.vs[1]; bp.vs_h = P.vs[2];
+    bp.perm = perm; bp.expiry_all = expiry; bp.Kg = (const __nv_bfloat16*)K; bp.Vg = (const __nv_bfloat16*)V;
+    bp.dKacc = accK; bp.dVacc = accV;
 #ifdef DMA_PROF
     const char* prof_env = getenv("DMA_PROF_PTR");
     bp.prof = prof_env ? (long long*)strtoull(prof_env, nullptr, 10) : nullptr;
 #endif
     const size_t smem = sizeof(SharedStorage) + 1024;
-    if (cudaFuncSetAttribute(bwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return DMA_ERR_CUDA;
-    bwd_kernel<<<dim3(P.B * P.Hkv, P.Tc), kThreads, smem, st>>>(tmQ, tmK, tmV, tmG, tmDQ, bp);
+    if (compact) {
+        if (cudaFuncSetAttribute(bwd_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return DMA_ERR_CUDA;
+        bwd_kernel<true><<<dim3(P.B * P.Hq, P.Tc), kThreads, smem, st>>>(tmQ, tmK, tmV, tmG, tmDQ, bp);
+        const int nb = (int)((nkv / 8 + 255) / 256);
+        dq_convert_bf16_kernel<<<nb, 256, 0, st>>>(accK, (__nv_bfloat16*)dK, nkv / 8, P.L, P.Hkv, P.ks[0], P.ks[1], P.ks[2], P.scale);
+        dq_convert_bf16_kernel<<<nb, 256, 0, st>>>(accV, (__nv_bfloat16*)dV, nkv / 8, P.L, P.Hkv, P.vs[0], P.vs[1], P.vs[2], 1.0f);
+        count_launch(2);
+    } else {
+        if (cudaFuncSetAttribute(bwd_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return DMA_ERR_CUDA;
+        bwd_kernel<false><<<dim3(P.B * P.Hkv, P.Tc), kThreads, smem, st>>>(tmQ, tmK, tmV, tmG, tmDQ, bp);
+    }
     dq_convert_bf16_kernel<<<(unsigned)((nq / 8 + 255) / 256), 256, 0, st>>>(acc, (__nv_bfloat16*)dQ, nq / 8, P.L, P.Hq, P.qs[0], P.qs[1], P.qs[2], P.scale);
     count_launch(3);
     return check_launch();

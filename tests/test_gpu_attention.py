@@ -215,3 +215,40 @@ def test_compact_flag_is_rejected_where_unsupported():
     with pytest.raises(dma.DmaError) as e:
         gpu_run(case, inp, backward=False, flags=dma.DMA_FLAG_COMPACT_KV)
     assert e.value.status == -4
+
+
+# ---- token-compacted backward (DMA_FLAG_COMPACT_KV): key tiles follow a lifetime-sorted permutation per query head -----
+
+def _compact_full_run(case, inp):
+    dev = torch.device("cuda:0")
+    pc = problem_of(case, flags=dma.DMA_FLAG_COMPACT_KV)
+    Q, K, V, dO = (inp[k].to(dev) for k in ("Q", "K", "V", "dO"))
+    bias, expiry, bitmap = dma.dma_mask_build(pc, V, inp["W_delta"].to(dev), inp["A"].to(dev))
+    m, f, bw = dma.dma_query_workspace(pc)
+    wsf = torch.empty(f, dtype=torch.uint8, device=dev)
+    wsb = torch.empty(bw, dtype=torch.uint8, device=dev)
+    O, lse = dma.dma_attn_fwd(pc, Q, K, V, bias, expiry, bitmap, ws=wsf)
+    dQ, dK, dV, dM = dma.dma_attn_bwd(pc, Q, K, V, O, dO, lse, bias, expiry, bitmap, ws=wsb)
+    torch.cuda.synchronize()
+    assert dma.dma_read_status(wsf) == 0 and dma.dma_read_status(wsb) == 0
+    return {"bias": bias, "expiry": expiry, "bitmap": bitmap, "O": O, "lse": lse, "dQ": dQ, "dK": dK, "dV": dV, "dM": dM}
+
+
+@pytest.mark.parametrize("case", [c for c in CASES if c.dtype == "bf16" and c.d == 128], ids=lambda c: c.name)
+def test_compact_backward_small_cases(case):
+    # the same small cases as the tile path (ragged tails and padding entries in the permutation, several query heads
+    # adding into one KV head, w = 1 where almost every key is never kept, w >= L where nothing expires, peaked scores)
+    inp = wl.make_inputs(case)
+    dl, e, _ = oracle_mask(case, inp)
+    got = _compact_full_run(case, inp)
+    assert np.array_equal(got["expiry"].cpu().numpy(), e)
+    compare(case, got, oracle_all(case, inp, dl, e))
+
+
+@pytest.mark.parametrize("key", ["3", "S"])
+def test_compact_backward_full_size_sampled(key):
+    case = wl.CONFIGS[key]
+    inp = wl.make_inputs(case)
+    got = _compact_full_run(case, inp)
+    sampled_check(case, inp, got)
+    dq_rows_check(case, inp, got, np.array([0, 5, 130, 700, 1500]))
