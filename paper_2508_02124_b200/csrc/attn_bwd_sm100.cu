@@ -126,6 +126,11 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
     const int j0 = kt * 128;
     const int* my_perm = kCompact ? P.perm + ((size_t)blockIdx.x * P.Tc + kt) * 128 : nullptr;
     volatile int* abort_flag = &S.abort_flag;
+    if constexpr (kCompact) {
+        // keys that no row keeps are sorted to the end of the permutation: a tile that starts with one holds nothing else
+        const int jf = my_perm[0];
+        if (jf >= P.L || P.expiry_all[(size_t)blockIdx.x * P.L + jf] <= jf) return;
+    }
 
     if (tid == 0) {
         mbar_init(&S.kv_full, 1);
@@ -575,16 +580,15 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
     if (tid == 0 && S.abort_flag) atomicExch(P.status, (int32_t)DMA_ERR_DEVICE_TIMEOUT);
 }
 
-// D_i = dO_i . O_i  (Alg. 2): one warp per (b, h, i), 16-byte loads
+// D_i = dO_i . O_i  (Alg. 2): 16 lanes per (b, h, i), 16-byte loads (a row of 128 bf16 is 16 x 16 bytes)
 __global__ void rowdot_bf16_kernel(const __nv_bfloat16* __restrict__ O, const __nv_bfloat16* __restrict__ dO,
                                    float* __restrict__ Dv, int B, int L, int Hq, int64_t os_b, int64_t os_l, int64_t os_h) {
-    const long row = (long)blockIdx.x * (blockDim.x / 32) + threadIdx.x / 32;
-    const int lane = threadIdx.x % 32;
-    if (row >= (long)B * Hq * L) return;
-    const int i = row % L, h = (row / L) % Hq, b = row / ((long)L * Hq);
-    const int64_t off = b * os_b + (int64_t)i * os_l + h * os_h + (lane & 15) * 8;
+    const long row = (long)blockIdx.x * (blockDim.x / 16) + threadIdx.x / 16;
+    const int sub = threadIdx.x % 16;
     float s = 0.0f;
-    if (lane < 16) {
+    if (row < (long)B * Hq * L) {
+        const int i = row % L, h = (row / L) % Hq, b = row / ((long)L * Hq);
+        const int64_t off = b * os_b + (int64_t)i * os_l + h * os_h + sub * 8;
         const uint4 a = *reinterpret_cast<const uint4*>(O + off), g = *reinterpret_cast<const uint4*>(dO + off);
         const uint32_t au[4] = {a.x, a.y, a.z, a.w}, gu[4] = {g.x, g.y, g.z, g.w};
 #pragma unroll
@@ -594,7 +598,7 @@ __global__ void rowdot_bf16_kernel(const __nv_bfloat16* __restrict__ O, const __
         }
     }
     for (int m = 8; m; m >>= 1) s += __shfl_xor_sync(0xffffffffu, s, m);
-    if (lane == 0) Dv[row] = s;
+    if (sub == 0 && row < (long)B * Hq * L) Dv[row] = s;
 }
 
 // fp32 accumulator [B, L, Hq, 128] (unscaled dS K sums) -> softmax scale applied -> bf16 dQ in the caller's layout; 8 elements per thread
@@ -690,7 +694,7 @@ int launch_tc_bwd(const Prob& P, const void* Q, const void* K, const void* V, co
     if ((rc = make_tmap_bf16(&tmV, V, P.B, P.L, P.Hkv, P.d, P.vs, 128))) return rc;
     CUtensorMap tmDQ;
     if ((rc = make_tmap_f32_rows(&tmDQ, acc, P.B, P.L, P.Hq, 16, 32))) return rc;
-    rowdot_bf16_kernel<<<(unsigned)((rows + 7) / 8), 256, 0, st>>>((const __nv_bfloat16*)O, (const __nv_bfloat16*)dO, Dv, P.B, P.L, P.Hq,
+    rowdot_bf16_kernel<<<(unsigned)((rows + 15) / 16), 256, 0, st>>>((const __nv_bfloat16*)O, (const __nv_bfloat16*)dO, Dv, P.B, P.L, P.Hq,
                                                                     P.os[0], P.os[1], P.os[2]);
     if (cudaMemsetAsync(acc, 0, nq * sizeof(float), st) != cudaSuccess) return DMA_ERR_CUDA;
     if (cudaMemsetAsync(dM, 0, rows * sizeof(float), st) != cudaSuccess) return DMA_ERR_CUDA;   // two partial sums are added per key

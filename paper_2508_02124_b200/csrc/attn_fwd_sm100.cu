@@ -857,28 +857,37 @@ int make_tmap_f32_rows(CUtensorMap* m, const void* base, int B, int L, int H, in
 
 // Token-compacted mode, per (batch, head, pair of query tiles): the ascending list of keys j that some row i of the
 // pair's 256 rows keeps, i.e. j <= i < expiry[j] for some i in [i0, i0 + 255]  <=>  j <= i0 + 255 and expiry[j] > max(i0, j).
-// At most w + 256 keys qualify. One warp per list: 32 keys per pass, ballot + popcount keep the order; the list is
-// padded with -1 to the next multiple of 128.
-__global__ void compact_lists_kernel(const int32_t* __restrict__ expiry, int* __restrict__ cidx, int* __restrict__ ccnt,
-                                     int L, int npairs, int cap, int nlists) {
-    const int list = blockIdx.x * (blockDim.x / 32) + threadIdx.x / 32, lane = threadIdx.x % 32;
-    if (list >= nlists) return;
+// At most w + 256 keys qualify. One CTA of 256 threads per list: 256 keys per pass, ballots and per-warp counts keep the
+// order; the list is padded with -1 to the next multiple of 128.
+__global__ void __launch_bounds__(256) compact_lists_kernel(const int32_t* __restrict__ expiry, int* __restrict__ cidx,
+                                                            int* __restrict__ ccnt, int L, int npairs, int cap) {
+    __shared__ int wsum[2][8];
+    const int list = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int bh = list / npairs, pair = list % npairs, i0 = pair * 256;
     const int32_t* e = expiry + (size_t)bh * L;
     int* out = cidx + (size_t)list * cap;
     const int jend = min(L, i0 + 256);
-    int n = 0;
-    for (int base = 0; base < jend; base += 32) {
-        const int j = base + lane;
+    int n = 0, buf = 0;
+    for (int base = 0; base < jend; base += 256, buf ^= 1) {
+        const int j = base + tid;
         const bool keep = j < jend && e[j] > max(i0, j);
         const uint32_t bal = __ballot_sync(0xffffffffu, keep);
-        const int pos = n + __popc(bal & ((1u << lane) - 1));
+        if (lane == 0) wsum[buf][warp] = __popc(bal);
+        __syncthreads();                                   // (the other buffer is free to be rewritten next pass)
+        int before = 0, total = 0;
+#pragma unroll
+        for (int wq = 0; wq < 8; ++wq) {
+            const int c = wsum[buf][wq];
+            before += wq < warp ? c : 0;
+            total += c;
+        }
+        const int pos = n + before + __popc(bal & ((1u << lane) - 1));
         if (keep && pos < cap) out[pos] = j;
-        n += __popc(bal);
+        n += total;
     }
     n = min(n, cap);
-    for (int t = n + lane; t < ((n + 127) / 128) * 128 && t < cap; t += 32) out[t] = -1;
-    if (lane == 0) ccnt[list] = n;
+    for (int t = n + tid; t < ((n + 127) / 128) * 128 && t < cap; t += 256) out[t] = -1;
+    if (tid == 0) ccnt[list] = n;
 }
 
 static int compact_cap(const Prob& P) { return ((P.w + 256 + 127) / 128) * 128; }
@@ -908,7 +917,7 @@ int launch_tc_fwd(const Prob& P, const void* Q, const void* K, const void* V, co
         const size_t nl = compact_lists(P);
         int* ccnt = reinterpret_cast<int*>((char*)ws + kWsHeaderBytes);
         int* cidx = reinterpret_cast<int*>((char*)ws + kWsHeaderBytes + ((nl * sizeof(int) + 255) / 256) * 256);
-        compact_lists_kernel<<<(unsigned)((nl + 3) / 4), 128, 0, st>>>(expiry, cidx, ccnt, P.L, (P.Tr + 1) / 2, compact_cap(P), (int)nl);
+        compact_lists_kernel<<<(unsigned)nl, 256, 0, st>>>(expiry, cidx, ccnt, P.L, (P.Tr + 1) / 2, compact_cap(P));
         count_launch();
         fp.cidx = cidx; fp.ccnt = ccnt; fp.ccap = compact_cap(P);
     }
