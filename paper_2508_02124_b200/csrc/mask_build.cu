@@ -177,13 +177,13 @@ __global__ void __launch_bounds__(kExpThreads) expiry_kernel(const float* __rest
         }
         __syncthreads();
         if (!done) {
-            int a = 0, z = kChunk;                // first position whose 64-bit key is greater than ours
-            while (a < z) {
-                const int mid = (a + z) >> 1;
-                const uint32_t h = hi[mid];
-                const bool greater = h > khi || (h == khi && lo[mid] > klo);
-                if (greater) z = mid; else a = mid + 1;
-            }
+            // a = first position whose 64-bit key is greater than ours: fixed-depth, branch-free lower bound on the
+            // high words (delta bits), then the (normally empty) run of equal high words is resolved by the low words
+            int a = 0;
+#pragma unroll
+            for (int s = kChunk / 2; s > 0; s >>= 1) a += hi[a + s - 1] < khi ? s : 0;
+            a += hi[a] < khi ? 1 : 0;                      // a = number of entries with hi < khi (0 .. kChunk)
+            while (a < kChunk && hi[a] == khi && lo[a] <= klo) ++a;
             const int n = kChunk - a;
             if (cnt + n >= w) { need = w - cnt; fin = c; done = true; }
             cnt += n;
