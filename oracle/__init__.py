@@ -187,3 +187,31 @@ def mask_backward(V, W, A, dM, Hq):
         dW[h] = np.einsum("bl,bld->d", dz, v)
         dV[:, :, hk, :] += dz[..., None] * W[h]
     return dV, dW, dA
+
+
+def decode(q, K, V, delta, w, scale=None):
+    """One decoding step (Sec. 3.2 with a single query at the end of the sequence; Alg. 1 with the per-key mask
+    M in R^N): the query of every (batch, head) sees all N cached keys, keeps the w with the largest dynamic weight
+    delta (ties to the lower index; all of them if N <= w) and attends to those with delta as the additive bias.
+    Plain numpy, fp64. q [B,Hq,d], K, V [B,N,Hkv,d], delta [B,Hq,N] (compared as given) ->
+    (o [B,Hq,d], lse [B,Hq], idx [B,Hq,min(w,N)] int32 ascending)."""
+    q = np.asarray(q, np.float64); K = np.asarray(K, np.float64); V = np.asarray(V, np.float64)
+    B, Hq, d = q.shape
+    N, Hkv = K.shape[1], K.shape[2]
+    G = Hq // Hkv
+    scale = d ** -0.5 if scale is None else scale
+    keep = min(w, N)
+    o = np.empty((B, Hq, d)); lse = np.empty((B, Hq)); idx = np.empty((B, Hq, keep), np.int32)
+    pos = np.arange(N)
+    for b in range(B):
+        for h in range(Hq):
+            dl = np.asarray(delta[b, h])
+            order = np.lexsort((pos, -dl.astype(np.float64)))[:keep]          # delta descending, then index ascending
+            sel = np.sort(order)
+            s = (K[b, sel, h // G, :] @ q[b, h]) * scale + dl[sel].astype(np.float64)
+            m = s.max()
+            p = np.exp(s - m)
+            o[b, h] = (p / p.sum()) @ V[b, sel, h // G, :]
+            lse[b, h] = m + np.log(p.sum())
+            idx[b, h] = sel
+    return o, lse, idx
