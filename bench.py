@@ -275,6 +275,31 @@ def main():
                             "step_ms": stage_ms["mask"] + c_ms + cb_ms, "tile_step_ms": sum(stage_ms.values()),
                             "dK_max_abs_diff_vs_tile_path": float((dKc.float() - dK.float()).abs().max())})
 
+    # ---- one decoding step over this workload's K / V as the cache (dma_delta_range + dma_decode), timed on its own
+    decode = None
+    if rank == 0:
+        pd = dma.problem(case.B, case.Hq, case.Hkv, case.L, case.d, case.w, dtype=case.torch_dtype)
+        dcache = torch.empty(case.B, case.Hq, case.L, dtype=torch.float32, device=dev)
+        dma.dma_delta_range(pd, V, W, A, dcache, 0, case.L)
+        qd = Q[:, -1].contiguous()
+        od, lsed = torch.empty_like(qd), torch.empty(case.B, case.Hq, dtype=torch.float32, device=dev)
+        ws_d = torch.empty(dma.dma_decode_workspace(pd), dtype=torch.uint8, device=dev)
+        for _ in range(3):
+            dma.dma_decode(pd, qd, K, V, dcache, od, lsed, None, False, ws_d)
+        d0, d1 = ev(), ev()
+        torch.cuda.synchronize()
+        d0.record()
+        for _ in range(20):
+            dma.dma_decode(pd, qd, K, V, dcache, od, lsed, None, False, ws_d)
+        d1.record()
+        torch.cuda.synchronize()
+        d_ms = d0.elapsed_time(d1) / 20
+        keep = min(case.w, case.L)
+        d_bytes = 2 * case.B * case.Hq * keep * case.d * K.element_size() + case.B * case.Hq * case.L * 4
+        decode = {"us_per_step": d_ms * 1e3, "cached_keys": case.L, "kept_keys": keep, "algorithmic_bytes": d_bytes,
+                  "gbs": d_bytes / (d_ms * 1e-3) / 1e9,
+                  "dense_kv_read_bytes": 2 * case.B * case.Hkv * case.L * case.d * K.element_size()}
+
     # ---- end to end through the host-buffer entry point: pinned host tensors in, results back on the host
     e2e = None
     if not args.no_e2e:
@@ -332,6 +357,9 @@ def main():
                      "traffic": NCU_TRAFFIC_BYTES.get(case.name, {}).get(dom) if tensor_path else None},
         "gpu_launches": launches, "clocks": clocks, "e2e": e2e,
     }
+    if decode is not None:
+        decode["frac_of_measured_hbm"] = decode["gbs"] / pk["hbm_gbs"]
+        out["decode"] = decode
     if compact is not None:
         out["compact"] = compact
     if mask_bwd is not None:

@@ -144,6 +144,24 @@ int dma_mask_bwd_workspace(const dma_problem_t* p, size_t* bytes);
 int dma_mask_bwd(const dma_problem_t* p, const void* V, const float* W_delta, const float* A, const float* bias,
                  const float* dM, void* dV, float* dW_delta, float* dA, void* ws, size_t ws_bytes, void* cuda_stream);
 
+/* Decoding (Sec. 3.2 for one query at the end of the sequence; Alg. 1 with the per-key mask M in R^N; the paper's
+ * decode benchmark): p->L is the number N of cached keys, k_stride / v_stride describe the K / V caches
+ * [B, >= N, Hkv, d] (a cache with spare capacity is a larger sequence stride), q and o are contiguous [B, Hq, d] in the
+ * problem's element type, delta is the cache of dynamic weights [B, Hq, delta_ld] fp32 (delta_ld >= N entries per row).
+ *
+ * dma_delta_range: delta[b,h,j] = exp(A[h] softplus(V[b,j,h/G,:] . W_delta[h,:])) for the keys j in [j_begin, j_end)
+ * only, with the same fixed fp32 arithmetic as dma_mask_build (bit-identical values): appends new keys to the cache.
+ *
+ * dma_decode: every (batch, query head) keeps the min(w, N) keys with the largest delta (ties to the lower index) and
+ * returns o = softmax(q . K_sel^T scale + delta_sel) V_sel and its log-sum-exp lse [B, Hq] (natural log). sel_idx, if
+ * not NULL, receives the kept key indices [B, Hq, min(w, N)] int32 in ascending order. Only the selected K and V rows
+ * are read. ws: dma_decode_workspace() bytes. All pointers device memory, 16-byte aligned. */
+int dma_delta_range(const dma_problem_t* p, const void* V, const float* W_delta, const float* A, float* delta, int64_t delta_ld,
+                    int32_t j_begin, int32_t j_end, void* cuda_stream);
+int dma_decode_workspace(const dma_problem_t* p, size_t* bytes);
+int dma_decode(const dma_problem_t* p, const void* q, const void* K, const void* V, const float* delta, int64_t delta_ld,
+               void* o, float* lse, int32_t* sel_idx, void* ws, size_t ws_bytes, void* cuda_stream);
+
 /* The whole hot path on HOST buffers (all contiguous, default strides only): copies Q,K,V,(dO),W_delta,A into the
  * caller's device arena, runs dma_mask_build, dma_attn_fwd and, if `backward` != 0, dma_attn_bwd on the stream,
  * copies O, lse (and dQ,dK,dV,dM) back and synchronises the stream before returning. h* pointers are HOST memory

@@ -18,7 +18,7 @@ DMA_FLAG_IGNORE_BITMAP, DMA_FLAG_SIMT, DMA_FLAG_COMPACT_KV = 1, 2, 4
 
 ENTRY_POINTS = ("dma_query_workspace", "dma_bitmap_words", "dma_mask_build", "dma_attn_fwd", "dma_attn_bwd",
                 "dma_read_status", "dma_launch_count", "dma_strerror", "dma_step_host_arena", "dma_step_host", "dma_mask_build_static", "dma_selftest_wait_timeout",
-                "dma_mask_bwd_workspace", "dma_mask_bwd")
+                "dma_mask_bwd_workspace", "dma_mask_bwd", "dma_delta_range", "dma_decode_workspace", "dma_decode")
 
 
 class DmaError(RuntimeError):
@@ -129,6 +129,35 @@ def dma_mask_bwd(p, V, W_delta, A, bias, dM, dV, dW_delta=None, dA=None, ws=None
     _check(lib().dma_mask_bwd(ctypes.byref(p), _ptr(V), _ptr(W_delta), _ptr(A), _ptr(bias), _ptr(dM), _ptr(dV), _ptr(dW_delta),
                               _ptr(dA), _ptr(ws), ctypes.c_size_t(ws.numel()), _stream()), "dma_mask_bwd")
     return dV, dW_delta, dA
+
+
+def dma_delta_range(p, V, W_delta, A, delta, j_begin, j_end):
+    """delta[b,h,j] for the keys j in [j_begin, j_end) of the cache V, written into the delta cache [B,Hq,ld]."""
+    _check(lib().dma_delta_range(ctypes.byref(p), _ptr(V), _ptr(W_delta), _ptr(A), _ptr(delta), ctypes.c_int64(delta.stride(1)),
+                                 ctypes.c_int32(j_begin), ctypes.c_int32(j_end), _stream()), "dma_delta_range")
+    return delta
+
+
+def dma_decode_workspace(p):
+    n = ctypes.c_size_t()
+    _check(lib().dma_decode_workspace(ctypes.byref(p), ctypes.byref(n)), "dma_decode_workspace")
+    return n.value
+
+
+def dma_decode(p, q, K, V, delta, o=None, lse=None, sel_idx=None, want_idx=False, ws=None):
+    """One decoding step over the cached keys; returns (o [B,Hq,d], lse [B,Hq], sel_idx or None)."""
+    dev = q.device
+    if o is None:
+        o = torch.empty_like(q)
+    if lse is None:
+        lse = torch.empty(p.B, p.Hq, dtype=torch.float32, device=dev)
+    if sel_idx is None and want_idx:
+        sel_idx = torch.empty(p.B, p.Hq, min(p.w, p.L), dtype=torch.int32, device=dev)
+    if ws is None:
+        ws = _ws(dma_decode_workspace(p), dev)
+    _check(lib().dma_decode(ctypes.byref(p), _ptr(q), _ptr(K), _ptr(V), _ptr(delta), ctypes.c_int64(delta.stride(1)), _ptr(o),
+                            _ptr(lse), _ptr(sel_idx), _ptr(ws), ctypes.c_size_t(ws.numel()), _stream()), "dma_decode")
+    return o, lse, sel_idx
 
 
 def dma_attn_fwd(p, Q, K, V, bias, expiry, bitmap, O=None, lse=None, ws=None):

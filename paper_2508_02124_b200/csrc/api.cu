@@ -135,6 +135,40 @@ int dma_mask_bwd(const dma_problem_t* p, const void* V, const float* W_delta, co
     return launch_mask_bwd(P, V, W_delta, A, bias, dM, dV, dW_delta, dA, ws, (cudaStream_t)cuda_stream);
 }
 
+int dma_delta_range(const dma_problem_t* p, const void* V, const float* W_delta, const float* A, float* delta, int64_t delta_ld,
+                    int32_t j_begin, int32_t j_end, void* cuda_stream) {
+    Prob P;
+    int rc = resolve(p, &P);
+    if (rc) return rc;
+    if (!V || !W_delta || !A || !delta) return DMA_ERR_NULL;
+    if (!aligned16(V) || !aligned16(W_delta) || !aligned16(delta)) return DMA_ERR_ALIGN;
+    if (j_begin < 0 || j_end > P.L || j_begin > j_end || delta_ld < P.L) return DMA_ERR_SHAPE;
+    if ((rc = device_ok())) return rc;
+    return launch_delta_range(P, V, W_delta, A, delta, delta_ld, j_begin, j_end, (cudaStream_t)cuda_stream);
+}
+
+int dma_decode_workspace(const dma_problem_t* p, size_t* bytes) {
+    Prob P;
+    int rc = resolve(p, &P);
+    if (rc) return rc;
+    if (!bytes) return DMA_ERR_NULL;
+    *bytes = decode_ws_bytes(P);
+    return DMA_OK;
+}
+
+int dma_decode(const dma_problem_t* p, const void* q, const void* K, const void* V, const float* delta, int64_t delta_ld,
+               void* o, float* lse, int32_t* sel_idx, void* ws, size_t ws_bytes, void* cuda_stream) {
+    Prob P;
+    int rc = resolve(p, &P);
+    if (rc) return rc;
+    if (!q || !K || !V || !delta || !o || !lse) return DMA_ERR_NULL;
+    if (!aligned16(q) || !aligned16(K) || !aligned16(V) || !aligned16(delta) || !aligned16(o)) return DMA_ERR_ALIGN;
+    if (delta_ld < P.L) return DMA_ERR_SHAPE;
+    if (!ws || ws_bytes < decode_ws_bytes(P) || !aligned16(ws)) return DMA_ERR_WORKSPACE;
+    if ((rc = device_ok())) return rc;
+    return launch_decode(P, q, K, V, delta, delta_ld, o, lse, sel_idx, ws, (cudaStream_t)cuda_stream);
+}
+
 int dma_attn_fwd(const dma_problem_t* p, const void* Q, const void* K, const void* V, const float* bias,
                  const int32_t* expiry, const uint32_t* bitmap, void* O, float* lse, void* ws, size_t ws_bytes,
                  void* cuda_stream) {

@@ -28,6 +28,11 @@ int check_launch();                                       // cudaGetLastError ->
 // stage launchers (each returns a dma_status); defined in the stage's .cu file
 size_t mask_ws_bytes(const Prob& P);
 size_t mask_bwd_ws_bytes(const Prob& P);
+int launch_delta_range(const Prob& P, const void* V, const float* W, const float* A, float* delta, int64_t ld, int j_begin,
+                       int j_end, cudaStream_t st);
+size_t decode_ws_bytes(const Prob& P);
+int launch_decode(const Prob& P, const void* q, const void* K, const void* V, const float* delta, int64_t ld, void* o, float* lse,
+                  int32_t* sel_idx, void* ws, cudaStream_t st);
 int launch_mask_bwd(const Prob& P, const void* V, const float* W, const float* A, const float* delta, const float* dM,
                     void* dV, float* dW, float* dA, void* ws, cudaStream_t st);
 int launch_mask_build(const Prob& P, const void* V, const float* W, const float* A, float* bias, int32_t* expiry,

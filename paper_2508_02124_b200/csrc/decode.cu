@@ -1,0 +1,335 @@
+// Decoding step (Sec. 3.2 for a single query at the end of the sequence; Alg. 1 with the per-key mask M in R^N, the
+// configuration of the paper's decode benchmark): every (batch, query head) keeps the w cached keys with the largest
+// dynamic weight delta (ties to the lower index; all N keys if N <= w) and attends to them with delta as the bias.
+// HBM / L2-bound: the delta row is scanned to select, then only the selected K and V rows are read.
+//
+// Kernels
+//   decode_select_kernel   per (batch, head): radix select over the 64-bit keys (delta bits << 32 | ~index) for the
+//                          threshold T with exactly min(w, N) keys >= T (three passes of 11 / 11 / 9 bits over the delta
+//                          bits, then the index cut among equal deltas)
+//   decode_index_kernel    optional: the selected indices in ascending order
+//   decode_attn_kernel     per (batch, head, split of <= 2048 keys): selected keys of the split are compacted into shared
+//                          memory; each warp then takes four of them per round (8 bytes of the K / V row per lane),
+//                          online softmax per warp, warps combined in shared memory -> partial (m, l, o)
+//   decode_combine_kernel  per (batch, head): the splits' partials -> o, log-sum-exp
+#include "common.cuh"
+
+namespace dma {
+namespace {
+
+constexpr int kSelThreads = 1024;
+constexpr int kSplitKeys = 2048;
+constexpr int kAttnThreads = 256;
+
+__device__ __forceinline__ unsigned long long key_of(float dl, int j) {
+    return ((unsigned long long)__float_as_uint(dl) << 32) | (unsigned long long)(0xFFFFFFFFu - (unsigned)j);
+}
+
+__global__ void __launch_bounds__(kSelThreads) decode_select_kernel(const float* __restrict__ delta, int64_t ld, int N, int w,
+                                                                    unsigned long long* __restrict__ thr) {
+    __shared__ int hist[2048];
+    __shared__ int s_scan[kSelThreads / 32];
+    __shared__ uint32_t s_prefix;
+    __shared__ int s_need, s_warp[kSelThreads / 32], s_found;
+    const int bh = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const float* dl = delta + (size_t)bh * ld;
+    if (N <= w) {
+        if (tid == 0) thr[bh] = 0ull;          // every key qualifies
+        return;
+    }
+    if (tid == 0) { s_prefix = 0u; s_need = w; }
+    __syncthreads();
+    // delta > 0 (sign bit clear): its bit pattern orders like the value. Three passes over bits [30:20], [19:9], [8:0]:
+    // keep the bin that holds the need-th largest among the keys matching the prefix so far. (Bits [30:20] = exponent
+    // and three mantissa bits spread a row over enough bins that the shared-memory adds rarely collide.)
+    const int shifts[3] = {20, 9, 0}, widths[3] = {11, 11, 9};
+    for (int pass = 0; pass < 3; ++pass) {
+        const int shift = shifts[pass], nb = 1 << widths[pass];
+        for (int t = tid; t < 2048; t += kSelThreads) hist[t] = 0;
+        __syncthreads();
+        const uint32_t prefix = s_prefix, himask = pass == 0 ? 0u : (0xFFFFFFFFu << (shift + widths[pass]));
+        for (int base = 0; base < N; base += 4 * kSelThreads) {
+            uint32_t u[4];
+#pragma unroll
+            for (int t = 0; t < 4; ++t) {
+                const int j = base + t * kSelThreads + tid;
+                u[t] = j < N ? __float_as_uint(dl[j]) : 0xFFFFFFFFu;          // never matches: deltas have the sign bit clear
+            }
+#pragma unroll
+            for (int t = 0; t < 4; ++t)
+                if (u[t] != 0xFFFFFFFFu && (u[t] & himask) == prefix) atomicAdd(&hist[(u[t] >> shift) & (nb - 1)], 1);
+        }
+        __syncthreads();
+        // suffix sums from the top bin: thread t owns bins [2t, 2t+1]; block-wide exclusive scan of the pair sums
+        const int b_hi = 2047 - 2 * tid, b_lo = b_hi - 1;            // descending bin order
+        const int c_hi = hist[b_hi], c_lo = hist[b_lo];
+        int incl = c_hi + c_lo;
+        for (int o = 1; o < 32; o <<= 1) {
+            const int v = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += v;
+        }
+        if (lane == 31) s_scan[warp] = incl;
+        __syncthreads();
+        int before = 0;
+        for (int wq = 0; wq < warp; ++wq) before += s_scan[wq];
+        const int excl = before + incl - (c_hi + c_lo);              // keys in bins above b_hi
+        const int need = s_need;
+        __syncthreads();
+        if (excl < need && need <= excl + c_hi) { s_need = need - excl; s_prefix = prefix | ((uint32_t)b_hi << shift); }
+        else if (excl + c_hi < need && need <= excl + c_hi + c_lo) { s_need = need - excl - c_hi; s_prefix = prefix | ((uint32_t)b_lo << shift); }
+        __syncthreads();
+    }
+    // s_prefix = delta bits of the threshold; s_need of the keys with exactly that delta are kept: those of lowest index
+    const uint32_t dstar = s_prefix;
+    const int need = s_need;
+    if (tid == 0) s_found = -1;
+    int seen = 0;
+    for (int base = 0; base < N; base += kSelThreads) {
+        const int j = base + tid;
+        const bool eq = j < N && __float_as_uint(dl[j]) == dstar;
+        const uint32_t bal = __ballot_sync(0xffffffffu, eq);
+        if (lane == 0) s_warp[warp] = __popc(bal);
+        __syncthreads();
+        int before = 0, total = 0;
+        for (int wq = 0; wq < kSelThreads / 32; ++wq) {
+            const int c = s_warp[wq];
+            before += wq < warp ? c : 0;
+            total += c;
+        }
+        const int rank = seen + before + __popc(bal & ((1u << lane) - 1));      // 0-based rank among the equal keys
+        if (eq && rank == need - 1) s_found = j;
+        seen += total;
+        __syncthreads();
+        if (seen >= need) break;
+    }
+    __syncthreads();
+    if (tid == 0) thr[bh] = key_of(__uint_as_float(dstar), s_found);
+}
+
+__global__ void __launch_bounds__(256) decode_index_kernel(const float* __restrict__ delta, int64_t ld, int N, int keep,
+                                                           const unsigned long long* __restrict__ thr, int32_t* __restrict__ idx) {
+    __shared__ int wsum[2][8];
+    const int bh = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const float* dl = delta + (size_t)bh * ld;
+    const unsigned long long T = thr[bh];
+    int n = 0, buf = 0;
+    for (int base = 0; base < N; base += 256, buf ^= 1) {
+        const int j = base + tid;
+        const bool sel = j < N && key_of(dl[j], j) >= T;
+        const uint32_t bal = __ballot_sync(0xffffffffu, sel);
+        if (lane == 0) wsum[buf][warp] = __popc(bal);
+        __syncthreads();
+        int before = 0, total = 0;
+#pragma unroll
+        for (int wq = 0; wq < 8; ++wq) {
+            const int c = wsum[buf][wq];
+            before += wq < warp ? c : 0;
+            total += c;
+        }
+        const int pos = n + before + __popc(bal & ((1u << lane) - 1));
+        if (sel && pos < keep) idx[(size_t)bh * keep + pos] = j;
+        n += total;
+    }
+}
+
+__device__ __forceinline__ void load4(const float* p, float (&v)[4]) {
+    const float4 a = *reinterpret_cast<const float4*>(p);
+    v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w;
+}
+__device__ __forceinline__ void load4(const __nv_bfloat16* p, float (&v)[4]) {
+    const uint2 a = *reinterpret_cast<const uint2*>(p);
+    v[0] = __uint_as_float(a.x << 16); v[1] = __uint_as_float(a.x & 0xffff0000u);
+    v[2] = __uint_as_float(a.y << 16); v[3] = __uint_as_float(a.y & 0xffff0000u);
+}
+
+// partial [bh][split][D + 2]: o (unnormalised, relative to m), m (log2 domain), l
+template <typename T, int D>
+__global__ void __launch_bounds__(kAttnThreads) decode_attn_kernel(const T* __restrict__ q, const T* __restrict__ K, const T* __restrict__ V,
+                                                                   const float* __restrict__ delta, int64_t ld,
+                                                                   const unsigned long long* __restrict__ thr, float* __restrict__ partial,
+                                                                   int N, int Hq, int G, float scale_log2, int nsplit,
+                                                                   int64_t ks_b, int64_t ks_l, int64_t ks_h, int64_t vs_b, int64_t vs_l,
+                                                                   int64_t vs_h) {
+    constexpr int LPK = D / 4;                 // lanes per key row (4 channels per lane)
+    constexpr int KPW = 32 / LPK;              // keys per warp instruction
+    __shared__ int list[kSplitKeys];
+    __shared__ int s_count, wsum[2][8];
+    __shared__ float s_part[8][D + 2];
+    const int split = blockIdx.x, bh = blockIdx.y, b = bh / Hq, h = bh % Hq, hk = h / G;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const float* dl = delta + (size_t)bh * ld;
+    const unsigned long long Tkey = thr[bh];
+    const int j_begin = split * kSplitKeys, j_end = min(N, j_begin + kSplitKeys);
+    // ordered compaction of the split's selected keys
+    int n = 0, buf = 0;
+    for (int base = j_begin; base < j_end; base += kAttnThreads, buf ^= 1) {
+        const int j = base + tid;
+        const bool sel = j < j_end && key_of(dl[j], j) >= Tkey;
+        const uint32_t bal = __ballot_sync(0xffffffffu, sel);
+        if (lane == 0) wsum[buf][warp] = __popc(bal);
+        __syncthreads();
+        int before = 0, total = 0;
+#pragma unroll
+        for (int wq = 0; wq < 8; ++wq) {
+            const int c = wsum[buf][wq];
+            before += wq < warp ? c : 0;
+            total += c;
+        }
+        if (sel) list[n + before + __popc(bal & ((1u << lane) - 1))] = j;
+        n += total;
+    }
+    if (tid == 0) s_count = n;
+    __syncthreads();
+    const int count = s_count;
+    // each warp: KPW keys per instruction (LPK lanes per key, 4 channels per lane), four such groups per round
+    const int sub = lane % LPK, grp = lane / LPK;
+    float qv[4];
+    load4(q + (size_t)bh * D + sub * 4, qv);
+    float m = -INFINITY, l = 0.0f, o[4] = {0.f, 0.f, 0.f, 0.f};
+    const T* Kb = K + b * ks_b + hk * ks_h + sub * 4;
+    const T* Vb = V + b * vs_b + hk * vs_h + sub * 4;
+    constexpr int kInFlight = 4;               // key rows whose K and V loads are in flight together, per lane group (8 was slower)
+    for (int base = warp * KPW * kInFlight; base < count; base += 8 * KPW * kInFlight) {
+        int jj[kInFlight];
+        float kv[kInFlight][4], vv[kInFlight][4], bias[kInFlight];
+#pragma unroll
+        for (int u = 0; u < kInFlight; ++u) {
+            const int e = base + u * KPW + grp;
+            jj[u] = e < count ? list[e] : -1;
+            if (jj[u] >= 0) {
+                load4(Kb + (int64_t)jj[u] * ks_l, kv[u]);
+                load4(Vb + (int64_t)jj[u] * vs_l, vv[u]);
+                bias[u] = dl[jj[u]];
+            } else {
+#pragma unroll
+                for (int c = 0; c < 4; ++c) { kv[u][c] = 0.0f; vv[u][c] = 0.0f; }
+                bias[u] = 0.0f;
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < kInFlight; ++u) {
+            float s = qv[0] * kv[u][0] + qv[1] * kv[u][1] + qv[2] * kv[u][2] + qv[3] * kv[u][3];
+#pragma unroll
+            for (int mm = 1; mm < LPK; mm <<= 1) s += __shfl_xor_sync(0xffffffffu, s, mm);
+            const float x = jj[u] >= 0 ? fmaf(s, scale_log2, bias[u] * 1.4426950408889634f) : -INFINITY;
+            const float m_new = fmaxf(m, x);
+            const float f = m_new == -INFINITY ? 1.0f : exp2f(m - m_new);
+            const float p = m_new == -INFINITY ? 0.0f : exp2f(x - m_new);
+            l = l * f + p;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) o[c] = o[c] * f + p * vv[u][c];
+            m = m_new;
+        }
+    }
+    // the KPW key groups of a warp hold different keys: merge them, then the warps, in shared memory
+#pragma unroll
+    for (int mm = LPK; mm < 32; mm <<= 1) {
+        const float m2 = __shfl_xor_sync(0xffffffffu, m, mm), l2 = __shfl_xor_sync(0xffffffffu, l, mm);
+        float o2[4];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) o2[c] = __shfl_xor_sync(0xffffffffu, o[c], mm);
+        const float mn = fmaxf(m, m2);
+        const float f1 = mn == -INFINITY ? 1.0f : exp2f(m - mn), f2 = mn == -INFINITY ? 1.0f : exp2f(m2 - mn);
+        l = l * f1 + l2 * f2;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) o[c] = o[c] * f1 + o2[c] * f2;
+        m = mn;
+    }
+    if (grp == 0) {
+#pragma unroll
+        for (int c = 0; c < 4; ++c) s_part[warp][sub * 4 + c] = o[c];
+        if (sub == 0) { s_part[warp][D] = m; s_part[warp][D + 1] = l; }
+    }
+    __syncthreads();
+    float* out = partial + ((size_t)bh * nsplit + split) * (D + 2);
+    float mx = -INFINITY;
+#pragma unroll
+    for (int wq = 0; wq < 8; ++wq) mx = fmaxf(mx, s_part[wq][D]);
+    for (int c = tid; c < D + 2; c += kAttnThreads) {
+        if (c == D) { out[c] = mx; continue; }
+        float acc = 0.0f;
+#pragma unroll
+        for (int wq = 0; wq < 8; ++wq) {
+            const float mw = s_part[wq][D];
+            const float f = (mw == -INFINITY || mx == -INFINITY) ? 0.0f : exp2f(mw - mx);
+            acc += s_part[wq][c] * f;                 // c == D + 1 is l
+        }
+        out[c] = acc;
+    }
+}
+
+template <typename T, int D>
+__global__ void __launch_bounds__(8 * D) decode_combine_kernel(const float* __restrict__ partial, T* __restrict__ o, float* __restrict__ lse,
+                                                               int nsplit) {
+    __shared__ float s_m[8], s_l[8], s_o[8][D];
+    const int bh = blockIdx.x, c = threadIdx.x % D, g = threadIdx.x / D;     // group g takes the splits s = g, g + 8, ...
+    const float* p = partial + (size_t)bh * nsplit * (D + 2);
+    float mx = -INFINITY;
+    for (int s = g; s < nsplit; s += 8) mx = fmaxf(mx, p[(size_t)s * (D + 2) + D]);
+    float l = 0.0f, acc = 0.0f;
+    for (int s = g; s < nsplit; s += 8) {
+        const float ms = p[(size_t)s * (D + 2) + D];
+        const float f = ms == -INFINITY ? 0.0f : exp2f(ms - mx);
+        l += p[(size_t)s * (D + 2) + D + 1] * f;
+        acc += p[(size_t)s * (D + 2) + c] * f;
+    }
+    s_o[g][c] = acc;
+    if (c == 0) { s_m[g] = mx; s_l[g] = l; }
+    __syncthreads();
+    if (g == 0) {
+        float m_all = -INFINITY;
+#pragma unroll
+        for (int q = 0; q < 8; ++q) m_all = fmaxf(m_all, s_m[q]);
+        float lt = 0.0f, at = 0.0f;
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            const float f = s_m[q] == -INFINITY ? 0.0f : exp2f(s_m[q] - m_all);
+            lt += s_l[q] * f;
+            at += s_o[q][c] * f;
+        }
+        const float v = lt > 0.0f ? at / lt : 0.0f;
+        if constexpr (sizeof(T) == 2) o[(size_t)bh * D + c] = __float2bfloat16_rn(v); else o[(size_t)bh * D + c] = v;
+        if (c == 0) lse[bh] = lt > 0.0f ? 0.6931471805599453f * (m_all + log2f(lt)) : -INFINITY;
+    }
+}
+
+template <typename T, int D>
+int launch_typed(const Prob& P, const void* q, const void* K, const void* V, const float* delta, int64_t ld, void* o, float* lse,
+                 const unsigned long long* thr, float* partial, int nsplit, cudaStream_t st) {
+    decode_attn_kernel<T, D><<<dim3(nsplit, P.B * P.Hq), kAttnThreads, 0, st>>>(
+        (const T*)q, (const T*)K, (const T*)V, delta, ld, thr, partial, P.L, P.Hq, P.G, P.scale * 1.4426950408889634f, nsplit, P.ks[0],
+        P.ks[1], P.ks[2], P.vs[0], P.vs[1], P.vs[2]);
+    decode_combine_kernel<T, D><<<P.B * P.Hq, 8 * D, 0, st>>>(partial, (T*)o, lse, nsplit);
+    count_launch(2);
+    return check_launch();
+}
+
+}  // namespace
+
+static int decode_splits(const Prob& P) { return (P.L + kSplitKeys - 1) / kSplitKeys; }
+
+size_t decode_ws_bytes(const Prob& P) {
+    const size_t bh = (size_t)P.B * P.Hq;
+    return kWsHeaderBytes + ((bh * sizeof(unsigned long long) + 255) / 256) * 256 + bh * decode_splits(P) * (P.d + 2) * sizeof(float);
+}
+
+int launch_decode(const Prob& P, const void* q, const void* K, const void* V, const float* delta, int64_t ld, void* o, float* lse,
+                  int32_t* sel_idx, void* ws, cudaStream_t st) {
+    const size_t bh = (size_t)P.B * P.Hq;
+    auto* thr = reinterpret_cast<unsigned long long*>((char*)ws + kWsHeaderBytes);
+    auto* partial = reinterpret_cast<float*>((char*)thr + ((bh * sizeof(unsigned long long) + 255) / 256) * 256);
+    decode_select_kernel<<<(unsigned)bh, kSelThreads, 0, st>>>(delta, ld, P.L, P.w, thr);
+    count_launch();
+    if (sel_idx) {
+        decode_index_kernel<<<(unsigned)bh, 256, 0, st>>>(delta, ld, P.L, P.w < P.L ? P.w : P.L, thr, sel_idx);
+        count_launch();
+    }
+    const int ns = decode_splits(P);
+    if (P.dtype == DMA_BF16)
+        return P.d == 128 ? launch_typed<__nv_bfloat16, 128>(P, q, K, V, delta, ld, o, lse, thr, partial, ns, st)
+                          : launch_typed<__nv_bfloat16, 64>(P, q, K, V, delta, ld, o, lse, thr, partial, ns, st);
+    return P.d == 128 ? launch_typed<float, 128>(P, q, K, V, delta, ld, o, lse, thr, partial, ns, st)
+                      : launch_typed<float, 64>(P, q, K, V, delta, ld, o, lse, thr, partial, ns, st);
+}
+
+}  // namespace dma

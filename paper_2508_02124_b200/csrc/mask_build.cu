@@ -78,14 +78,15 @@ __device__ __forceinline__ void load8(const __nv_bfloat16* p, float (&v)[8]) {
 template <typename T, int D>
 __global__ void __launch_bounds__(256) delta_kernel(const T* __restrict__ V, const float* __restrict__ W,
                                                     const float* __restrict__ A, float* __restrict__ delta,
-                                                    int L, int Hq, int G, int64_t vs_b, int64_t vs_l, int64_t vs_h) {
+                                                    int L, int Hq, int G, int64_t vs_b, int64_t vs_l, int64_t vs_h,
+                                                    int j_off, int64_t ld) {
     constexpr int LPR = D / 8;            // lanes per row
     constexpr int RPW = 32 / LPR;         // rows per warp and pass
     constexpr int kRows = 128;
     extern __shared__ float smem[];
     float* sW = smem;                     // [G][D]
     float* sOut = smem + G * D;           // [G][kRows]
-    const int hk = blockIdx.y, b = blockIdx.z, j0 = blockIdx.x * kRows;
+    const int hk = blockIdx.y, b = blockIdx.z, j0 = j_off + blockIdx.x * kRows;   // keys [j_off, L) of a row of ld entries
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int sub = lane % LPR, grp = lane / LPR;
     for (int i = tid; i < G * D; i += 256) sW[i] = W[(size_t)hk * G * D + i];
@@ -112,7 +113,7 @@ __global__ void __launch_bounds__(256) delta_kernel(const T* __restrict__ V, con
     __syncthreads();
     for (int i = tid; i < G * kRows; i += 256) {
         const int g = i / kRows, r = i % kRows;
-        if (j0 + r < L) delta[((size_t)b * Hq + hk * G + g) * L + j0 + r] = sOut[i];
+        if (j0 + r < L) delta[((size_t)b * Hq + hk * G + g) * ld + j0 + r] = sOut[i];
     }
 }
 
@@ -258,13 +259,27 @@ size_t mask_ws_bytes(const Prob& P) {
 }
 
 template <typename T, int D>
-static int launch_delta(const Prob& P, const void* V, const float* W, const float* A, float* bias, cudaStream_t st) {
-    dim3 grid((P.L + 127) / 128, P.Hkv, P.B);
+static int launch_delta(const Prob& P, const void* V, const float* W, const float* A, float* bias, cudaStream_t st,
+                        int j_begin = 0, int j_end = -1, int64_t ld = -1) {
+    if (j_end < 0) j_end = P.L;
+    if (ld < 0) ld = P.L;
+    if (j_end <= j_begin) return DMA_OK;
+    dim3 grid((j_end - j_begin + 127) / 128, P.Hkv, P.B);
     size_t smem = (size_t)P.G * (D + 128) * sizeof(float);
     if (smem > 48 * 1024) return DMA_ERR_UNSUPPORTED;
-    delta_kernel<T, D><<<grid, 256, smem, st>>>((const T*)V, W, A, bias, P.L, P.Hq, P.G, P.vs[0], P.vs[1], P.vs[2]);
+    delta_kernel<T, D><<<grid, 256, smem, st>>>((const T*)V, W, A, bias, j_end, P.Hq, P.G, P.vs[0], P.vs[1], P.vs[2], j_begin, ld);
     count_launch();
     return check_launch();
+}
+
+// delta for the keys [j_begin, j_end) only, into rows of ld entries (a decoding cache that grows)
+int launch_delta_range(const Prob& P, const void* V, const float* W, const float* A, float* delta, int64_t ld, int j_begin,
+                       int j_end, cudaStream_t st) {
+    if (P.dtype == DMA_BF16)
+        return P.d == 128 ? launch_delta<__nv_bfloat16, 128>(P, V, W, A, delta, st, j_begin, j_end, ld)
+                          : launch_delta<__nv_bfloat16, 64>(P, V, W, A, delta, st, j_begin, j_end, ld);
+    return P.d == 128 ? launch_delta<float, 128>(P, V, W, A, delta, st, j_begin, j_end, ld)
+                      : launch_delta<float, 64>(P, V, W, A, delta, st, j_begin, j_end, ld);
 }
 
 int launch_mask_build(const Prob& P, const void* V, const float* W, const float* A, float* bias, int32_t* expiry,
