@@ -57,7 +57,13 @@ __global__ void __launch_bounds__(kThreads) mask_bwd_kernel(const T* __restrict_
     const int hk = blockIdx.y, b = blockIdx.z, j0 = blockIdx.x * kRows;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int sub = lane % LPR, grp = lane / LPR;
+    float* sGD = sAcc + 8 * G * (D + 1);             // [G][kRows]: dM * delta of the CTA's keys, fetched in one batch
     for (int i = tid; i < G * D; i += kThreads) sW[i] = W[(size_t)hk * G * D + i];
+    for (int i = tid; i < G * kRows; i += kThreads) {
+        const int g = i / kRows, j = j0 + i % kRows;
+        const size_t at = ((size_t)b * Hq + hk * G + g) * L + j;
+        sGD[i] = j < L ? dM[at] * delta[at] : 0.0f;
+    }
     __syncthreads();
 
     float v[NR][8], upd[NR][8];
@@ -87,8 +93,7 @@ __global__ void __launch_bounds__(kThreads) mask_bwd_kernel(const T* __restrict_
             for (int c = 0; c < 8; ++c) z = fmaf(v[n][c], w[c], z);
 #pragma unroll
             for (int m = 1; m < LPR; m <<= 1) z += __shfl_xor_sync(0xffffffffu, z, m);
-            float gd = 0.0f;
-            if (j < L) gd = dM[((size_t)b * Hq + h) * L + j] * delta[((size_t)b * Hq + h) * L + j];
+            const float gd = sGD[g * kRows + (j - j0)];
             const float e = __expf(-fabsf(z));                       // in (0, 1]
             const float sp = fmaxf(z, 0.0f) + log1pf(e);
             const float sig = (z >= 0.0f ? 1.0f : e) / (1.0f + e);
@@ -161,7 +166,7 @@ template <typename T, int D>
 static int launch_typed(const Prob& P, const void* V, const float* W, const float* A, const float* delta, const float* dM,
                         void* dV, float* dW, float* dA, void* ws, cudaStream_t st) {
     const int nblk = (P.L + kRows - 1) / kRows;
-    const size_t smem = (size_t)P.G * (D + 8 * (D + 1)) * sizeof(float);
+    const size_t smem = (size_t)P.G * (D + 8 * (D + 1) + kRows) * sizeof(float);
     if (cudaFuncSetAttribute(mask_bwd_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return DMA_ERR_CUDA;
     mask_bwd_kernel<T, D><<<dim3(nblk, P.Hkv, P.B), kThreads, smem, st>>>((const T*)V, W, A, delta, dM, (T*)dV, (float*)ws, P.L, P.Hq,
                                                                             P.G, P.vs[0], P.vs[1], P.vs[2]);
