@@ -1,6 +1,7 @@
 // dma_step_host: the whole hot path (mask build, forward, optional backward) on HOST buffers, for callers that
 // keep their tensors in host memory and for end-to-end timing. Inputs are copied to a caller-provided device
-// arena, the three stages run on the caller's stream, results are copied back, and the stream is synchronised.
+// arena (on helper streams, overlapped with the kernels), the three stages run on the caller's stream, results are
+// copied back, and the stream is synchronised.
 #include "common.cuh"
 
 namespace dma {
@@ -75,29 +76,52 @@ int dma_step_host(const dma_problem_t* p, int backward, const void* hQ, const vo
     if (!dev_arena || arena_bytes < Lo.total || (reinterpret_cast<uintptr_t>(dev_arena) & 255)) return DMA_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)cuda_stream;
     char* a = (char*)dev_arena;
-    auto h2d = [&](size_t off, const void* src, size_t n) { return cudaMemcpyAsync(a + off, src, n, cudaMemcpyHostToDevice, st) == cudaSuccess; };
-    auto d2h = [&](void* dst, size_t off, size_t n) { return cudaMemcpyAsync(dst, a + off, n, cudaMemcpyDeviceToHost, st) == cudaSuccess; };
-    bool ok = h2d(Lo.Q, hQ, Lo.nq * Lo.esz) && h2d(Lo.K, hK, Lo.nk * Lo.esz) && h2d(Lo.V, hV, Lo.nk * Lo.esz) &&
-              h2d(Lo.W, hW_delta, (size_t)p->Hq * p->d * 4) && h2d(Lo.A, hA, (size_t)p->Hq * 4);
-    if (backward) ok = ok && h2d(Lo.dO, hdO, Lo.nq * Lo.esz);
-    if (!ok) return DMA_ERR_CUDA;
+    // Copies run on two helper streams of this call (created and destroyed here: no state is kept) so that they overlap
+    // the kernels on the caller's stream: V first (the mask build needs nothing else), then K and Q, then dO while the
+    // forward runs; O and lse go back while the backward runs. Events order the helpers after the work already on the
+    // caller's stream and the caller's stream after the last copy.
+    cudaStream_t s_in = nullptr, s_out = nullptr;
+    cudaEvent_t ev[7] = {};
+    auto cleanup = [&](int code) {
+        for (auto& e : ev) if (e) cudaEventDestroy(e);
+        if (s_in) cudaStreamDestroy(s_in);
+        if (s_out) cudaStreamDestroy(s_out);
+        return code;
+    };
+    if (cudaStreamCreateWithFlags(&s_in, cudaStreamNonBlocking) != cudaSuccess) return cleanup(DMA_ERR_CUDA);
+    if (cudaStreamCreateWithFlags(&s_out, cudaStreamNonBlocking) != cudaSuccess) return cleanup(DMA_ERR_CUDA);
+    for (auto& e : ev) if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) return cleanup(DMA_ERR_CUDA);
+    enum { kStart, kV, kKQ, kdO, kO, kG, kDone };
+    auto h2d = [&](size_t off, const void* src, size_t n) { return cudaMemcpyAsync(a + off, src, n, cudaMemcpyHostToDevice, s_in) == cudaSuccess; };
+    auto d2h = [&](void* dst, size_t off, size_t n) { return cudaMemcpyAsync(dst, a + off, n, cudaMemcpyDeviceToHost, s_out) == cudaSuccess; };
+    auto rec = [&](int e, cudaStream_t on) { return cudaEventRecord(ev[e], on) == cudaSuccess; };
+    auto wait = [&](cudaStream_t on, int e) { return cudaStreamWaitEvent(on, ev[e], 0) == cudaSuccess; };
+    bool ok = rec(kStart, st) && wait(s_in, kStart) && wait(s_out, kStart);
+    ok = ok && h2d(Lo.V, hV, Lo.nk * Lo.esz) && h2d(Lo.W, hW_delta, (size_t)p->Hq * p->d * 4) && h2d(Lo.A, hA, (size_t)p->Hq * 4) && rec(kV, s_in);
+    ok = ok && h2d(Lo.K, hK, Lo.nk * Lo.esz) && h2d(Lo.Q, hQ, Lo.nq * Lo.esz) && rec(kKQ, s_in);
+    if (backward) ok = ok && h2d(Lo.dO, hdO, Lo.nq * Lo.esz) && rec(kdO, s_in);
+    if (!ok) return cleanup(DMA_ERR_CUDA);
     float* bias = (float*)(a + Lo.bias);
     int32_t* expiry = (int32_t*)(a + Lo.expiry);
     uint32_t* bitmap = (uint32_t*)(a + Lo.bitmap);
-    if ((rc = dma_mask_build(p, a + Lo.V, (float*)(a + Lo.W), (float*)(a + Lo.A), bias, expiry, bitmap, a + Lo.ws_mask, Lo.m_ws, st))) return rc;
-    if ((rc = dma_attn_fwd(p, a + Lo.Q, a + Lo.K, a + Lo.V, bias, expiry, bitmap, a + Lo.O, (float*)(a + Lo.lse), a + Lo.ws_fwd, Lo.f_ws, st))) return rc;
-    ok = d2h(hO, Lo.O, Lo.nq * Lo.esz) && d2h(hlse, Lo.lse, Lo.nbh * 4);
+    if (!wait(st, kV)) return cleanup(DMA_ERR_CUDA);
+    if ((rc = dma_mask_build(p, a + Lo.V, (float*)(a + Lo.W), (float*)(a + Lo.A), bias, expiry, bitmap, a + Lo.ws_mask, Lo.m_ws, st))) return cleanup(rc);
+    if (!wait(st, kKQ)) return cleanup(DMA_ERR_CUDA);
+    if ((rc = dma_attn_fwd(p, a + Lo.Q, a + Lo.K, a + Lo.V, bias, expiry, bitmap, a + Lo.O, (float*)(a + Lo.lse), a + Lo.ws_fwd, Lo.f_ws, st))) return cleanup(rc);
+    ok = rec(kO, st) && wait(s_out, kO) && d2h(hO, Lo.O, Lo.nq * Lo.esz) && d2h(hlse, Lo.lse, Lo.nbh * 4);
     if (backward) {
+        if (!ok || !wait(st, kdO)) return cleanup(DMA_ERR_CUDA);
         if ((rc = dma_attn_bwd(p, a + Lo.Q, a + Lo.K, a + Lo.V, a + Lo.O, a + Lo.dO, (float*)(a + Lo.lse), bias, expiry, bitmap,
-                               a + Lo.dQ, a + Lo.dK, a + Lo.dV, (float*)(a + Lo.dM), a + Lo.ws_bwd, Lo.b_ws, st))) return rc;
-        ok = ok && d2h(hdQ, Lo.dQ, Lo.nq * Lo.esz) && d2h(hdK, Lo.dK, Lo.nk * Lo.esz) && d2h(hdV, Lo.dV, Lo.nk * Lo.esz) &&
-             d2h(hdM, Lo.dM, Lo.nbh * 4);
+                               a + Lo.dQ, a + Lo.dK, a + Lo.dV, (float*)(a + Lo.dM), a + Lo.ws_bwd, Lo.b_ws, st))) return cleanup(rc);
+        ok = rec(kG, st) && wait(s_out, kG) && d2h(hdQ, Lo.dQ, Lo.nq * Lo.esz) && d2h(hdK, Lo.dK, Lo.nk * Lo.esz) &&
+             d2h(hdV, Lo.dV, Lo.nk * Lo.esz) && d2h(hdM, Lo.dM, Lo.nbh * 4);
     }
-    if (!ok) return DMA_ERR_CUDA;
-    if (cudaStreamSynchronize(st) != cudaSuccess) return DMA_ERR_CUDA;
+    ok = ok && rec(kDone, s_out) && wait(st, kDone);
+    if (!ok) return cleanup(DMA_ERR_CUDA);
+    if (cudaStreamSynchronize(st) != cudaSuccess) return cleanup(DMA_ERR_CUDA);
     int s1 = dma_read_status(a + Lo.ws_fwd, st);
-    if (s1) return s1;
-    return backward ? dma_read_status(a + Lo.ws_bwd, st) : DMA_OK;
+    if (s1) return cleanup(s1);
+    return cleanup(backward ? dma_read_status(a + Lo.ws_bwd, st) : DMA_OK);
 }
 
 }  // extern "C"
