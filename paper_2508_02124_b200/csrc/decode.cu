@@ -4,9 +4,8 @@
 // HBM / L2-bound: the delta row is scanned to select, then only the selected K and V rows are read.
 //
 // Kernels
-//   decode_select_kernel   per (batch, head): radix select over the 64-bit keys (delta bits << 32 | ~index) for the
-//                          threshold T with exactly min(w, N) keys >= T (three passes of 11 / 11 / 9 bits over the delta
-//                          bits, then the index cut among equal deltas)
+//   decode_hist_kernel x3, decode_thr_kernel   radix select over the 64-bit keys (delta bits << 32 | ~index) for the
+//                          threshold T with exactly min(w, N) keys >= T, spread over CTAs of 8192 keys
 //   decode_index_kernel    optional: the selected indices in ascending order
 //   decode_attn_kernel     per (batch, head, split of <= 2048 keys): selected keys of the split are compacted into shared
 //                          memory; each warp then takes four of them per round (8 bytes of the K / V row per lane),
@@ -25,82 +24,125 @@ __device__ __forceinline__ unsigned long long key_of(float dl, int j) {
     return ((unsigned long long)__float_as_uint(dl) << 32) | (unsigned long long)(0xFFFFFFFFu - (unsigned)j);
 }
 
-__global__ void __launch_bounds__(kSelThreads) decode_select_kernel(const float* __restrict__ delta, int64_t ld, int N, int w,
-                                                                    unsigned long long* __restrict__ thr) {
+// Radix select of the min(w, N)-th largest key of every (batch, head) row, spread over many CTAs. Three histogram
+// passes over the delta bit patterns, bits [30:20], [19:9], [8:0] (delta > 0: the sign bit is clear and the pattern orders
+// like the value; exponent plus three mantissa bits spread a row over enough bins that shared-memory adds rarely
+// collide). Pass p: every CTA first re-derives the prefix chosen by the passes before it from their global histograms
+// (pick_bin: a 2048-bin suffix scan, identical in every CTA), then histograms the next bits of its 8192-key slice of the
+// row for the keys that match the prefix and adds the non-zero bins to the row's global histogram. A last kernel picks
+// the final bin and, only if several keys tie at the threshold delta and not all of them are wanted, walks the row in
+// index order for the cut. state[bh] = {prefix bits, keys still wanted inside the prefix}.
+struct SelState { uint32_t prefix; int need; };
+
+// hist: 2048 counters of one pass; returns through `st` the bin holding the need-th largest key (scanning from the top
+// bin) and the rank wanted inside it. Called by every thread of a CTA with kSelThreads / 4 = 256 threads.
+__device__ __forceinline__ void pick_bin(const int* __restrict__ hist, int shift, SelState& st, int* s_scan, SelState* s_out) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    int c[8], sum = 0;
+#pragma unroll
+    for (int t = 0; t < 8; ++t) { c[t] = hist[2047 - (8 * tid + t)]; sum += c[t]; }       // descending bin order
+    int incl = sum;
+    for (int o = 1; o < 32; o <<= 1) {
+        const int v = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += v;
+    }
+    if (lane == 31) s_scan[warp] = incl;
+    __syncthreads();
+    int before = 0;
+    for (int wq = 0; wq < warp; ++wq) before += s_scan[wq];
+    int excl = before + incl - sum;                       // keys in bins above this thread's first bin
+#pragma unroll
+    for (int t = 0; t < 8; ++t) {
+        if (excl < st.need && st.need <= excl + c[t]) {
+            s_out->prefix = st.prefix | ((uint32_t)(2047 - (8 * tid + t)) << shift);
+            s_out->need = st.need - excl;
+        }
+        excl += c[t];
+    }
+    __syncthreads();
+    st = *s_out;
+    __syncthreads();
+}
+
+constexpr int kSliceKeys = 8192;
+
+// pass = 0, 1, 2; ghist [3][BH][2048] zeroed before pass 0
+__global__ void __launch_bounds__(256) decode_hist_kernel(const float* __restrict__ delta, int64_t ld, int N, int w, int pass,
+                                                          int* __restrict__ ghist, int BH) {
     __shared__ int hist[2048];
-    __shared__ int s_scan[kSelThreads / 32];
-    __shared__ uint32_t s_prefix;
-    __shared__ int s_need, s_warp[kSelThreads / 32], s_found;
-    const int bh = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    __shared__ int s_scan[8];
+    __shared__ SelState s_out;
+    const int bh = blockIdx.y, tid = threadIdx.x;
+    if (N <= w) return;
     const float* dl = delta + (size_t)bh * ld;
+    const int shifts[3] = {20, 9, 0}, widths[3] = {11, 11, 9};
+    SelState st{0u, w};
+    for (int q = 0; q < pass; ++q) pick_bin(ghist + ((size_t)q * BH + bh) * 2048, shifts[q], st, s_scan, &s_out);
+    for (int t = tid; t < 2048; t += 256) hist[t] = 0;
+    __syncthreads();
+    const int shift = shifts[pass], nb = 1 << widths[pass];
+    const uint32_t himask = pass == 0 ? 0u : (0xFFFFFFFFu << (shift + widths[pass]));
+    const int j0 = blockIdx.x * kSliceKeys, j1 = min(N, j0 + kSliceKeys);
+    for (int base = j0; base < j1; base += 4 * 256) {
+        uint32_t u[4];
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+            const int j = base + t * 256 + tid;
+            u[t] = j < j1 ? __float_as_uint(dl[j]) : 0xFFFFFFFFu;              // never matches: deltas have the sign bit clear
+        }
+#pragma unroll
+        for (int t = 0; t < 4; ++t)
+            if (u[t] != 0xFFFFFFFFu && (u[t] & himask) == st.prefix) atomicAdd(&hist[(u[t] >> shift) & (nb - 1)], 1);
+    }
+    __syncthreads();
+    int* g = ghist + ((size_t)pass * BH + bh) * 2048;
+    for (int t = tid; t < 2048; t += 256)
+        if (hist[t]) atomicAdd(&g[t], hist[t]);
+}
+
+// one CTA per row: final pick; thr = (delta bits << 32) | ~index cut
+__global__ void __launch_bounds__(256) decode_thr_kernel(const float* __restrict__ delta, int64_t ld, int N, int w,
+                                                         const int* __restrict__ ghist, int BH, unsigned long long* __restrict__ thr) {
+    __shared__ int s_scan[8];
+    __shared__ SelState s_out;
+    __shared__ int s_warp[8], s_found;
+    const int bh = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     if (N <= w) {
         if (tid == 0) thr[bh] = 0ull;          // every key qualifies
         return;
     }
-    if (tid == 0) { s_prefix = 0u; s_need = w; }
-    __syncthreads();
-    // delta > 0 (sign bit clear): its bit pattern orders like the value. Three passes over bits [30:20], [19:9], [8:0]:
-    // keep the bin that holds the need-th largest among the keys matching the prefix so far. (Bits [30:20] = exponent
-    // and three mantissa bits spread a row over enough bins that the shared-memory adds rarely collide.)
-    const int shifts[3] = {20, 9, 0}, widths[3] = {11, 11, 9};
-    for (int pass = 0; pass < 3; ++pass) {
-        const int shift = shifts[pass], nb = 1 << widths[pass];
-        for (int t = tid; t < 2048; t += kSelThreads) hist[t] = 0;
-        __syncthreads();
-        const uint32_t prefix = s_prefix, himask = pass == 0 ? 0u : (0xFFFFFFFFu << (shift + widths[pass]));
-        for (int base = 0; base < N; base += 4 * kSelThreads) {
-            uint32_t u[4];
-#pragma unroll
-            for (int t = 0; t < 4; ++t) {
-                const int j = base + t * kSelThreads + tid;
-                u[t] = j < N ? __float_as_uint(dl[j]) : 0xFFFFFFFFu;          // never matches: deltas have the sign bit clear
-            }
-#pragma unroll
-            for (int t = 0; t < 4; ++t)
-                if (u[t] != 0xFFFFFFFFu && (u[t] & himask) == prefix) atomicAdd(&hist[(u[t] >> shift) & (nb - 1)], 1);
-        }
-        __syncthreads();
-        // suffix sums from the top bin: thread t owns bins [2t, 2t+1]; block-wide exclusive scan of the pair sums
-        const int b_hi = 2047 - 2 * tid, b_lo = b_hi - 1;            // descending bin order
-        const int c_hi = hist[b_hi], c_lo = hist[b_lo];
-        int incl = c_hi + c_lo;
-        for (int o = 1; o < 32; o <<= 1) {
-            const int v = __shfl_up_sync(0xffffffffu, incl, o);
-            if (lane >= o) incl += v;
-        }
-        if (lane == 31) s_scan[warp] = incl;
-        __syncthreads();
-        int before = 0;
-        for (int wq = 0; wq < warp; ++wq) before += s_scan[wq];
-        const int excl = before + incl - (c_hi + c_lo);              // keys in bins above b_hi
-        const int need = s_need;
-        __syncthreads();
-        if (excl < need && need <= excl + c_hi) { s_need = need - excl; s_prefix = prefix | ((uint32_t)b_hi << shift); }
-        else if (excl + c_hi < need && need <= excl + c_hi + c_lo) { s_need = need - excl - c_hi; s_prefix = prefix | ((uint32_t)b_lo << shift); }
-        __syncthreads();
+    const float* dl = delta + (size_t)bh * ld;
+    const int shifts[3] = {20, 9, 0};
+    SelState st{0u, w};
+    const int* g2 = ghist + ((size_t)2 * BH + bh) * 2048;
+    for (int q = 0; q < 3; ++q) pick_bin(ghist + ((size_t)q * BH + bh) * 2048, shifts[q], st, s_scan, &s_out);
+    // st.prefix = delta bits of the threshold; st.need of the keys with exactly that delta are kept, lowest index first
+    const uint32_t dstar = st.prefix;
+    const int equal = g2[dstar & 511];
+    if (st.need >= equal) {                    // every key with this delta is wanted: no cut inside the group
+        if (tid == 0) thr[bh] = (unsigned long long)dstar << 32;
+        return;
     }
-    // s_prefix = delta bits of the threshold; s_need of the keys with exactly that delta are kept: those of lowest index
-    const uint32_t dstar = s_prefix;
-    const int need = s_need;
     if (tid == 0) s_found = -1;
     int seen = 0;
-    for (int base = 0; base < N; base += kSelThreads) {
+    for (int base = 0; base < N; base += 256) {
         const int j = base + tid;
         const bool eq = j < N && __float_as_uint(dl[j]) == dstar;
         const uint32_t bal = __ballot_sync(0xffffffffu, eq);
         if (lane == 0) s_warp[warp] = __popc(bal);
         __syncthreads();
         int before = 0, total = 0;
-        for (int wq = 0; wq < kSelThreads / 32; ++wq) {
+#pragma unroll
+        for (int wq = 0; wq < 8; ++wq) {
             const int c = s_warp[wq];
             before += wq < warp ? c : 0;
             total += c;
         }
         const int rank = seen + before + __popc(bal & ((1u << lane) - 1));      // 0-based rank among the equal keys
-        if (eq && rank == need - 1) s_found = j;
+        if (eq && rank == st.need - 1) s_found = j;
         seen += total;
         __syncthreads();
-        if (seen >= need) break;
+        if (seen >= st.need) break;
     }
     __syncthreads();
     if (tid == 0) thr[bh] = key_of(__uint_as_float(dstar), s_found);
@@ -162,9 +204,18 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attn_kernel(const T* __re
     const int j_begin = split * kSplitKeys, j_end = min(N, j_begin + kSplitKeys);
     // ordered compaction of the split's selected keys
     int n = 0, buf = 0;
-    for (int base = j_begin; base < j_end; base += kAttnThreads, buf ^= 1) {
+    float dpre[kSplitKeys / kAttnThreads];          // the split's deltas of this thread, all loads in flight together
+#pragma unroll
+    for (int t = 0; t < kSplitKeys / kAttnThreads; ++t) {
+        const int j = j_begin + t * kAttnThreads + tid;
+        dpre[t] = j < j_end ? dl[j] : 0.0f;
+    }
+#pragma unroll
+    for (int t = 0; t < kSplitKeys / kAttnThreads; ++t, buf ^= 1) {
+        const int base = j_begin + t * kAttnThreads;
+        if (base >= j_end) break;
         const int j = base + tid;
-        const bool sel = j < j_end && key_of(dl[j], j) >= Tkey;
+        const bool sel = j < j_end && key_of(dpre[t], j) >= Tkey;
         const uint32_t bal = __ballot_sync(0xffffffffu, sel);
         if (lane == 0) wsum[buf][warp] = __popc(bal);
         __syncthreads();
@@ -308,17 +359,28 @@ int launch_typed(const Prob& P, const void* q, const void* K, const void* V, con
 
 static int decode_splits(const Prob& P) { return (P.L + kSplitKeys - 1) / kSplitKeys; }
 
+static size_t decode_hist_bytes(const Prob& P) { return (size_t)3 * P.B * P.Hq * 2048 * sizeof(int); }
+
 size_t decode_ws_bytes(const Prob& P) {
     const size_t bh = (size_t)P.B * P.Hq;
-    return kWsHeaderBytes + ((bh * sizeof(unsigned long long) + 255) / 256) * 256 + bh * decode_splits(P) * (P.d + 2) * sizeof(float);
+    return kWsHeaderBytes + ((bh * sizeof(unsigned long long) + 255) / 256) * 256 + decode_hist_bytes(P) +
+           bh * decode_splits(P) * (P.d + 2) * sizeof(float);
 }
 
 int launch_decode(const Prob& P, const void* q, const void* K, const void* V, const float* delta, int64_t ld, void* o, float* lse,
                   int32_t* sel_idx, void* ws, cudaStream_t st) {
     const size_t bh = (size_t)P.B * P.Hq;
     auto* thr = reinterpret_cast<unsigned long long*>((char*)ws + kWsHeaderBytes);
-    auto* partial = reinterpret_cast<float*>((char*)thr + ((bh * sizeof(unsigned long long) + 255) / 256) * 256);
-    decode_select_kernel<<<(unsigned)bh, kSelThreads, 0, st>>>(delta, ld, P.L, P.w, thr);
+    int* ghist = reinterpret_cast<int*>((char*)thr + ((bh * sizeof(unsigned long long) + 255) / 256) * 256);
+    auto* partial = reinterpret_cast<float*>((char*)ghist + decode_hist_bytes(P));
+    if (P.w < P.L) {
+        if (cudaMemsetAsync(ghist, 0, decode_hist_bytes(P), st) != cudaSuccess) return DMA_ERR_CUDA;
+        const dim3 grid((P.L + kSliceKeys - 1) / kSliceKeys, (unsigned)bh);
+        for (int pass = 0; pass < 3; ++pass)
+            decode_hist_kernel<<<grid, 256, 0, st>>>(delta, ld, P.L, P.w, pass, ghist, (int)bh);
+        count_launch(3);
+    }
+    decode_thr_kernel<<<(unsigned)bh, 256, 0, st>>>(delta, ld, P.L, P.w, ghist, (int)bh, thr);
     count_launch();
     if (sel_idx) {
         decode_index_kernel<<<(unsigned)bh, 256, 0, st>>>(delta, ld, P.L, P.w < P.L ? P.w : P.L, thr, sel_idx);
