@@ -142,16 +142,28 @@ __global__ void __launch_bounds__(kThreads) mask_bwd_kernel(const T* __restrict_
     }
 }
 
-// dW[h][c] and dA[h]: sum of the per-CTA partials over batches and key blocks, in index order
-__global__ void mask_bwd_reduce_kernel(const float* __restrict__ partial, float* __restrict__ dW, float* __restrict__ dA,
-                                       int B, int Hkv, int G, int D, int nblk) {
+// dW[h][c] and dA[h]: sum of the per-CTA partials over batches and key blocks. kGroups groups of threads each add every
+// kGroups-th partial in index order, then the group sums are added in group order: a fixed order, whatever the schedule.
+template <int D>
+__global__ void __launch_bounds__((D == 128 ? 4 : 8) * (D + 1)) mask_bwd_reduce_kernel(const float* __restrict__ partial, float* __restrict__ dW,
+                                                                     float* __restrict__ dA, int B, int Hkv, int G, int nblk) {
+    constexpr int kGroups = D == 128 ? 4 : 8;      // kGroups * (D + 1) threads <= 1024
+    __shared__ float part[kGroups][D + 1];
     const int h = blockIdx.x, hk = h / G, g = h % G;
-    for (int c = threadIdx.x; c <= D; c += blockDim.x) {
-        float s = 0.0f;
-        for (int b = 0; b < B; ++b)
-            for (int k = 0; k < nblk; ++k)
-                s += partial[((((size_t)b * Hkv + hk) * nblk + k) * G + g) * (D + 1) + c];
-        if (c < D) dW[(size_t)h * D + c] = s; else dA[h] = s;
+    const int c = threadIdx.x % (D + 1), grp = threadIdx.x / (D + 1);
+    float s = 0.0f;
+    const int total = B * nblk;
+    for (int t = grp; t < total; t += kGroups) {
+        const int b = t / nblk, k = t % nblk;
+        s += partial[((((size_t)b * Hkv + hk) * nblk + k) * G + g) * (D + 1) + c];
+    }
+    part[grp][c] = s;
+    __syncthreads();
+    if (grp == 0) {
+        float tot = 0.0f;
+#pragma unroll
+        for (int q = 0; q < kGroups; ++q) tot += part[q][c];
+        if (c < D) dW[(size_t)h * D + c] = tot; else dA[h] = tot;
     }
 }
 
@@ -170,7 +182,7 @@ static int launch_typed(const Prob& P, const void* V, const float* W, const floa
     if (cudaFuncSetAttribute(mask_bwd_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return DMA_ERR_CUDA;
     mask_bwd_kernel<T, D><<<dim3(nblk, P.Hkv, P.B), kThreads, smem, st>>>((const T*)V, W, A, delta, dM, (T*)dV, (float*)ws, P.L, P.Hq,
                                                                             P.G, P.vs[0], P.vs[1], P.vs[2]);
-    mask_bwd_reduce_kernel<<<P.Hq, 160, 0, st>>>((const float*)ws, dW, dA, P.B, P.Hkv, P.G, D, nblk);
+    mask_bwd_reduce_kernel<D><<<P.Hq, (D == 128 ? 4 : 8) * (D + 1), 0, st>>>((const float*)ws, dW, dA, P.B, P.Hkv, P.G, nblk);
     count_launch(2);
     return check_launch();
 }
