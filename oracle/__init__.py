@@ -74,6 +74,20 @@ def delta(V, W, A, Hq):
     return z, dl
 
 
+def delta_full(V, W, A):
+    """Eq. (delta_calc) with the full sampling weights: V [B,L,Hkv,d], W [Hq, Hkv*d] (one row per query head over the
+    flattened value row), A [Hq] -> (z, delta) [B,Hq,L] fp32 in the fixed operation order of the C source."""
+    V = _c(V, np.float32); W = _c(W, np.float32); A = _c(A, np.float32)
+    B, L, Hkv, d = V.shape
+    Hq = W.shape[0]
+    assert W.shape == (Hq, Hkv * d) and A.shape == (Hq,)
+    z = np.empty((B, Hq, L), np.float32)
+    dl = np.empty((B, Hq, L), np.float32)
+    rc = lib().dmao_delta_full(_p(V), _p(W), _p(A), B, L, Hq, Hkv, d, _p(z), _p(dl))
+    assert rc == 0, rc
+    return z, dl
+
+
 def select_definition(dl, w):
     """delta [..., L] -> keep [..., L, L] uint8 by the per-row sort definition."""
     dl = _c(dl, np.float32)
@@ -187,6 +201,30 @@ def mask_backward(V, W, A, dM, Hq):
         dW[h] = np.einsum("bl,bld->d", dz, v)
         dV[:, :, hk, :] += dz[..., None] * W[h]
     return dV, dW, dA
+
+
+def mask_backward_full(V, W, A, dM):
+    """mask_backward for the full sampling weights W [Hq, Hkv*d] (every query head reads the whole value row):
+
+        z = vrow . W_h  (vrow = the Hkv*d channels of key j),  g = dM delta,  dA_h = sum g softplus(z),
+        dz = g A_h sigmoid(z),  dW_h = sum dz vrow,  dVrow[j] = sum_h dz W_h
+
+    Plain numpy, fp64. V [B,L,Hkv,d], A [Hq], dM [B,Hq,L] -> (dV like V, dW like W, dA [Hq])."""
+    V = np.asarray(V, np.float64); W = np.asarray(W, np.float64); A = np.asarray(A, np.float64)
+    dM = np.asarray(dM, np.float64)
+    B, L, Hkv, d = V.shape
+    rows = V.reshape(B, L, Hkv * d)
+    dRows = np.zeros_like(rows); dW = np.zeros_like(W); dA = np.zeros_like(A)
+    for h in range(W.shape[0]):
+        z = rows @ W[h]                                      # [B, L]
+        e = np.exp(-np.abs(z))
+        sp = np.maximum(z, 0.0) + np.log1p(e)
+        g = dM[:, h, :] * np.exp(A[h] * sp)
+        dA[h] = (g * sp).sum()
+        dz = g * A[h] * np.where(z >= 0, 1.0, e) / (1.0 + e)
+        dW[h] = np.einsum("bl,blc->c", dz, rows)
+        dRows += dz[..., None] * W[h]
+    return dRows.reshape(V.shape), dW, dA
 
 
 def decode(q, K, V, delta, w, scale=None):

@@ -6,7 +6,8 @@
 // kernels. Every routine follows the definition (or the algorithm's steps) in the paper's order:
 // no tiling, no fusion, no SIMD intrinsics; OpenMP only spreads independent rows / keys over cores.
 //
-//   delta            Eq. (delta_calc) of Sec. 4.1 and the listing of App. A: dt = exp(A * softplus(v . W))
+//   delta            Eq. (delta_calc) of Sec. 4.1 and the listing of App. A: dt = exp(A * softplus(v . W)), with
+//                    W per head over the head's own d channels, or (delta_full) over all Hkv*d channels of the row
 //   selection        Eq. (mask_combine) of Sec. 4.1 read per query row as the App. A listing does
 //                    (top-w over the causally visible keys), ties broken toward the lower index
 //   block bitmap     the Judge(M_j) block test of Alg. 1 / Alg. 2, per (query tile, key tile)
@@ -311,6 +312,30 @@ int dmao_delta(const float* V, const float* W, const float* A, int B, int L, int
             for (int j = 0; j < L; ++j) {
                 const float* v = V + (((size_t)b * L + j) * Hkv + h / G) * d;
                 float z = dot_spec(v, W + (size_t)h * d, d);
+                float sp = softplus_spec(z);
+                size_t o = ((size_t)b * Hq + h) * L + j;
+                if (z_out) z_out[o] = z;
+                delta[o] = exp_spec(A[h] * sp);
+            }
+    return 0;
+}
+
+// Eq. (delta_calc) with the sampling weights as the paper states them, a map from all heads' value channels to
+// one score per head (App. A listing: a linear layer over the value row flattened to Hkv*d channels):
+//   z[b,h,j] = sum_{h'} V[b,j,h',:] . W[h, h'*d : (h'+1)*d]
+// delta-v1 order: the per-head dot products as above, added over h' = 0, 1, ... from left to right (one rounded
+// addition each, starting from the h' = 0 term).
+int dmao_delta_full(const float* V, const float* W, const float* A, int B, int L, int Hq, int Hkv, int d,
+                    float* z_out, float* delta) {
+    if (d % 8 || (d / 8) & (d / 8 - 1) || d > 512) return -1;
+#pragma omp parallel for collapse(2)
+    for (int b = 0; b < B; ++b)
+        for (int h = 0; h < Hq; ++h)
+            for (int j = 0; j < L; ++j) {
+                const float* v = V + ((size_t)b * L + j) * Hkv * d;
+                const float* w = W + (size_t)h * Hkv * d;
+                float z = dot_spec(v, w, d);
+                for (int hk = 1; hk < Hkv; ++hk) z = z + dot_spec(v + (size_t)hk * d, w + (size_t)hk * d, d);
                 float sp = softplus_spec(z);
                 size_t o = ((size_t)b * Hq + h) * L + j;
                 if (z_out) z_out[o] = z;
