@@ -238,6 +238,37 @@ def main():
         g_bytes = 3 * V.numel() * V.element_size() + 2 * bias.numel() * 4
         mask_bwd = {"ms": g_ms, "algorithmic_bytes": g_bytes, "gbs": g_bytes / (g_ms * 1e-3) / 1e9}
 
+    # ---- full sampling weights (DMA_FLAG_FULL_DELTA: W over all Hkv*d channels of the value row), timed on their own:
+    # the mask build and its backward with a [Hq, Hkv*d] weight; 2 Hq Hkv d flop per key for z, three times that in the backward
+    full_delta = None
+    try:
+        pf = dma.problem(case.B, case.Hq, case.Hkv, case.L, case.d, case.w, dtype=case.torch_dtype,
+                         flags=args.flags | dma.DMA_FLAG_FULL_DELTA)
+        Wf = wl.full_delta_weights(case).to(dev)
+        bias_f, exp_f, bmp_f = torch.empty_like(bias), torch.empty_like(expiry), torch.empty_like(bitmap)
+        ws_fm = torch.empty(dma.dma_query_workspace(pf)[0], dtype=torch.uint8, device=dev)
+        run_f = [lambda: dma.dma_mask_build(pf, V, Wf, A, bias_f, exp_f, bmp_f, ws_fm)]
+        if case.backward:
+            ws_fg = torch.empty(dma.dma_mask_bwd_workspace(pf), dtype=torch.uint8, device=dev)
+            dWf, dAf = torch.empty_like(Wf), torch.empty_like(A)
+            run_f.append(lambda: dma.dma_mask_bwd(pf, V, Wf, A, bias_f, dM, dV, dWf, dAf, ws_fg))
+        times = []
+        for f in run_f:
+            for _ in range(3):
+                f()
+            g0, g1 = ev(), ev()
+            barrier()
+            g0.record()
+            for _ in range(10):
+                f()
+            g1.record()
+            barrier()
+            times.append(g0.elapsed_time(g1) / 10)
+        zflop = 2.0 * case.B * case.L * case.Hq * case.Hkv * case.d
+        full_delta = {"mask_build_ms": times[0], "mask_bwd_ms": times[1] if len(times) > 1 else None, "z_gflop": zflop / 1e9}
+    except dma.DmaError as e:
+        full_delta = {"unsupported": str(e)}
+
     # ---- token-compacted forward (DMA_FLAG_COMPACT_KV), timed on its own: same outputs, O(L w d) work
     compact = None
     if case.dtype == "bf16" and case.d == 128 and not (args.flags & dma.DMA_FLAG_SIMT):
@@ -362,6 +393,8 @@ def main():
         out["decode"] = decode
     if compact is not None:
         out["compact"] = compact
+    if full_delta is not None:
+        out["full_delta"] = full_delta
     if mask_bwd is not None:
         mask_bwd["frac_of_measured_hbm"] = mask_bwd["gbs"] / pk["hbm_gbs"]
         out["mask_bwd"] = mask_bwd

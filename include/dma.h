@@ -47,7 +47,7 @@ enum {
     DMA_FLAG_IGNORE_BITMAP = 1,  /* visit every causal tile regardless of the bitmap (result must not change:
                                     block skipping is an optimisation only, Sec. 4.2 last paragraph)           */
     DMA_FLAG_SIMT = 2,           /* run the CUDA-core kernels also for bf16 (they always serve fp32)            */
-    DMA_FLAG_COMPACT_KV = 4      /* dma_attn_fwd and dma_attn_bwd, bf16, d = 128, contiguous K and V: token-compacted
+    DMA_FLAG_COMPACT_KV = 4,     /* dma_attn_fwd and dma_attn_bwd, bf16, d = 128, contiguous K and V: token-compacted
                                     execution (Sec. 3.3, computational sparsity: O(L w d) instead of O(L^2 d) work).
                                     Forward: each pair of query tiles gathers only the keys that one of its 256 rows
                                     keeps (at most w + 256) instead of walking every active 128-key tile. Backward: a CTA
@@ -56,6 +56,13 @@ enum {
                                     the first key and the last expiry; dK, dV are summed over the group in fp32. Same
                                     results up to rounding; needs the larger workspaces dma_query_workspace reports for
                                     it; ignores the bitmap */
+    DMA_FLAG_FULL_DELTA = 8      /* the sampling weights as Eq. (delta_calc) states them: W_delta (and dW_delta) is
+                                    [Hq, Hkv*d], one row per query head over ALL channels of the value row (the linear
+                                    layer of the App. A listing), z[b,h,j] = sum_{h'} V[b,j,h',:] . W_delta[h, h'*d:(h'+1)*d].
+                                    Without the flag W_delta is [Hq, d] and head h reads only its own KV head (the
+                                    block-diagonal special case). Read by dma_mask_build, dma_mask_build_static,
+                                    dma_delta_range, dma_mask_bwd, dma_mask_bwd_workspace and dma_step_host; needs
+                                    roundup(Hq, d/8) * (Hkv*d + 64) * 4 <= 200 KiB */
 };
 
 typedef struct {

@@ -14,7 +14,7 @@ LIB_PATH = os.path.join(_PKG, "libdma_b200.so")
 _lib = None
 
 DMA_BF16, DMA_FP32 = 0, 1
-DMA_FLAG_IGNORE_BITMAP, DMA_FLAG_SIMT, DMA_FLAG_COMPACT_KV = 1, 2, 4
+DMA_FLAG_IGNORE_BITMAP, DMA_FLAG_SIMT, DMA_FLAG_COMPACT_KV, DMA_FLAG_FULL_DELTA = 1, 2, 4, 8
 
 ENTRY_POINTS = ("dma_query_workspace", "dma_bitmap_words", "dma_mask_build", "dma_attn_fwd", "dma_attn_bwd",
                 "dma_read_status", "dma_launch_count", "dma_strerror", "dma_step_host_arena", "dma_step_host", "dma_mask_build_static", "dma_selftest_wait_timeout",
@@ -118,10 +118,10 @@ def dma_mask_bwd_workspace(p):
 
 
 def dma_mask_bwd(p, V, W_delta, A, bias, dM, dV, dW_delta=None, dA=None, ws=None):
-    """Adds the mask path's contribution to dV in place; returns (dV, dW_delta [Hq,d] fp32, dA [Hq] fp32)."""
+    """Adds the mask path's contribution to dV in place; returns (dV, dW_delta fp32 shaped like W_delta, dA [Hq] fp32)."""
     dev = V.device
     if dW_delta is None:
-        dW_delta = torch.empty(p.Hq, p.d, dtype=torch.float32, device=dev)
+        dW_delta = torch.empty(p.Hq, p.Hkv * p.d if p.flags & DMA_FLAG_FULL_DELTA else p.d, dtype=torch.float32, device=dev)
     if dA is None:
         dA = torch.empty(p.Hq, dtype=torch.float32, device=dev)
     if ws is None:

@@ -117,6 +117,93 @@ __global__ void __launch_bounds__(256) delta_kernel(const T* __restrict__ V, con
     }
 }
 
+// Full sampling weights (Eq. delta_calc as stated: all Hkv*D channels of the value row feed every head's score, the
+// linear layer of the App. A listing): z[h] = sum over KV heads hk of (v_hk . W[h, hk*D : (hk+1)*D]), the per-head dot
+// products formed as in delta_kernel (8-channel fma chains, pairwise tree over adjacent chunks) and added over hk
+// from left to right. One CTA owns 64 keys of one batch and all heads. A group of D/8 lanes owns two rows; it forms the
+// chains of D/8 heads at a time and adds them with a transposing butterfly (at each step a lane keeps half of its
+// values and hands the other half to its partner: the same additions as the plain butterfly, a quarter of the
+// shuffles), after which lane `sub` holds the dot product of head bitrev(sub) and carries that head's running sum.
+constexpr int kFullRows = 64;
+
+template <typename T, int D>
+__global__ void __launch_bounds__(256) delta_full_kernel(const T* __restrict__ V, const float* __restrict__ W,
+                                                         const float* __restrict__ A, float* __restrict__ delta,
+                                                         int L, int Hq, int Hkv, int64_t vs_b, int64_t vs_l,
+                                                         int64_t vs_h, int j_off, int64_t ld) {
+    constexpr int LPR = D / 8;            // lanes per row = heads per batch
+    constexpr int RPW = 32 / LPR;         // row groups per warp
+    constexpr int kPass = 16 * RPW;       // rows per pass of the CTA (two per lane group)
+    extern __shared__ float smem[];
+    const int C = Hkv * D, HqP = (Hq + LPR - 1) / LPR * LPR;
+    float* sW = smem;                     // [HqP][C], rows beyond Hq zero
+    float* sZ = smem + (size_t)HqP * C;   // [HqP][kFullRows]
+    const int b = blockIdx.y, j0 = j_off + blockIdx.x * kFullRows;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int sub = lane % LPR, grp = lane / LPR;
+    int mine = 0;                         // the head (within a batch) this lane ends up with: sub, bit-reversed
+#pragma unroll
+    for (int m = 1, t = LPR >> 1; m < LPR; m <<= 1, t >>= 1) mine |= (sub & m) ? t : 0;
+    for (int i = tid; i < HqP * C; i += 256) sW[i] = i < Hq * C ? W[i] : 0.0f;
+    __syncthreads();
+    for (int r0 = 0; r0 < kFullRows; r0 += kPass) {
+        int r[2];
+        r[0] = r0 + warp * 2 * RPW + grp;
+        r[1] = r[0] + RPW;
+        for (int hk = 0; hk < Hkv; ++hk) {
+            float v[2][8];
+#pragma unroll
+            for (int n = 0; n < 2; ++n) {
+                if (j0 + r[n] < L) {
+                    load8(V + b * vs_b + (int64_t)(j0 + r[n]) * vs_l + hk * vs_h + sub * 8, v[n]);
+                } else {
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) v[n][c] = 0.0f;
+                }
+            }
+            for (int hb = 0; hb < HqP; hb += LPR) {
+                float p[2][LPR];
+#pragma unroll
+                for (int q = 0; q < LPR; ++q) {
+                    const float* wp = sW + (size_t)(hb + q) * C + hk * D + sub * 8;
+                    const float4 wa = *reinterpret_cast<const float4*>(wp), wb = *reinterpret_cast<const float4*>(wp + 4);
+                    const float w[8] = {wa.x, wa.y, wa.z, wa.w, wb.x, wb.y, wb.z, wb.w};
+#pragma unroll
+                    for (int n = 0; n < 2; ++n) {
+                        float a = 0.0f;
+#pragma unroll
+                        for (int c = 0; c < 8; ++c) a = __fmaf_rn(v[n][c], w[c], a);
+                        p[n][q] = a;
+                    }
+                }
+#pragma unroll
+                for (int m = 1, keep = LPR >> 1; m < LPR; m <<= 1, keep >>= 1) {
+                    const bool up = (sub & m) != 0;
+#pragma unroll
+                    for (int n = 0; n < 2; ++n)
+#pragma unroll
+                        for (int q = 0; q < keep; ++q) {
+                            const float stay = up ? p[n][q + keep] : p[n][q];
+                            const float give = up ? p[n][q] : p[n][q + keep];
+                            p[n][q] = __fadd_rn(stay, __shfl_xor_sync(0xffffffffu, give, m));
+                        }
+                }
+                const int h = hb + mine;
+#pragma unroll
+                for (int n = 0; n < 2; ++n) {
+                    float* z = sZ + h * kFullRows + r[n];
+                    *z = hk == 0 ? p[n][0] : __fadd_rn(*z, p[n][0]);
+                }
+            }
+        }
+    }
+    __syncthreads();
+    for (int i = tid; i < Hq * kFullRows; i += 256) {
+        const int h = i / kFullRows, r = i % kFullRows;
+        if (j0 + r < L) delta[((size_t)b * Hq + h) * ld + j0 + r] = delta_fixed(sZ[i], A[h]);
+    }
+}
+
 // ---- selection --------------------------------------------------------------------------------------------
 // Order: key a beats key b iff (delta_a, -a) > (delta_b, -b). delta > 0, so its bit pattern orders like the
 // value and one unsigned 64-bit compare decides.
@@ -264,6 +351,17 @@ static int launch_delta(const Prob& P, const void* V, const float* W, const floa
     if (j_end < 0) j_end = P.L;
     if (ld < 0) ld = P.L;
     if (j_end <= j_begin) return DMA_OK;
+    if (P.flags & DMA_FLAG_FULL_DELTA) {
+        const size_t HqP = (size_t)(P.Hq + D / 8 - 1) / (D / 8) * (D / 8);
+        const size_t bytes = (HqP * P.Hkv * D + HqP * kFullRows) * sizeof(float);
+        if (bytes > 200 * 1024) return DMA_ERR_UNSUPPORTED;
+        if (cudaFuncSetAttribute(delta_full_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess)
+            return DMA_ERR_CUDA;
+        delta_full_kernel<T, D><<<dim3((j_end - j_begin + kFullRows - 1) / kFullRows, P.B), 256, bytes, st>>>(
+            (const T*)V, W, A, bias, j_end, P.Hq, P.Hkv, P.vs[0], P.vs[1], P.vs[2], j_begin, ld);
+        count_launch();
+        return check_launch();
+    }
     dim3 grid((j_end - j_begin + 127) / 128, P.Hkv, P.B);
     size_t smem = (size_t)P.G * (D + 128) * sizeof(float);
     if (smem > 48 * 1024) return DMA_ERR_UNSUPPORTED;

@@ -167,9 +167,192 @@ __global__ void __launch_bounds__((D == 128 ? 4 : 8) * (D + 1)) mask_bwd_reduce_
     }
 }
 
+// ---- full sampling weights: W [Hq, C], C = Hkv * D channels of the value row feed every head ----------------
+// One CTA owns R consecutive keys of one batch with their whole value rows in shared memory (fp32):
+//   1  z[h][row]: warp per RW rows, lanes stride the channels, W read once per warp from L2
+//   2  dz[row][h] = dM delta A sigmoid(z), gs[h][row] = dM delta softplus(z)
+//   3  dW partial [h][col] = sum_rows dz v: a thread owns a column and walks the rows (no cross-thread sums)
+//   4  the value tile is overwritten by sum_h dz W[h][col], then added to dV
+// partial [B * blocks][Hq][C + 1]; mask_bwd_full_reduce_kernel adds them in a fixed order.
+template <typename T, int RW>
+__global__ void __launch_bounds__(kThreads) mask_bwd_full_kernel(const T* __restrict__ V, const float* __restrict__ W,
+                                                                 const float* __restrict__ A, const float* __restrict__ delta,
+                                                                 const float* __restrict__ dM, T* __restrict__ dV,
+                                                                 float* __restrict__ partial, int L, int Hq, int Hkv, int D,
+                                                                 int64_t vs_b, int64_t vs_l, int64_t vs_h) {
+    constexpr int R = RW * 8;
+    extern __shared__ float smem[];
+    const int C = Hkv * D, HqP = (Hq + 7) & ~7;
+    float* sV = smem;                              // [R][C]
+    float* sDz = sV + (size_t)R * C;               // [R][HqP], heads beyond Hq hold 0
+    float* sZ = sDz + (size_t)R * HqP;             // [Hq][R]: z, then dM delta softplus(z)
+    const int b = blockIdx.y, j0 = blockIdx.x * R;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int C8 = C / 8, D8 = D / 8;
+
+    for (int i = tid; i < R * C8; i += kThreads) {
+        const int row = i / C8, ch = i % C8, j = j0 + row;
+        float v[8];
+        if (j < L) {
+            load8f(V + b * vs_b + (int64_t)j * vs_l + (ch / D8) * vs_h + (ch % D8) * 8, v);
+        } else {
+#pragma unroll
+            for (int c = 0; c < 8; ++c) v[c] = 0.0f;
+        }
+        store8f(sV + (size_t)row * C + ch * 8, v);
+    }
+    for (int i = tid; i < R * HqP; i += kThreads) sDz[i] = 0.0f;
+    __syncthreads();
+
+    // z: a warp owns HB heads at a time and all R rows; lanes stride the channels, so W is read once per CTA and each
+    // value feeds HB fmas. The per-lane sums are added across lanes by a transposing butterfly (a lane keeps half of
+    // its rows at each step), which leaves row (lane mod RL) of every head in the lane.
+    constexpr int HB = 128 / R < 16 ? 128 / R : 16;
+    constexpr int RL = R < 32 ? R : 32;            // rows reduced together
+    for (int h0 = warp * HB; h0 < Hq; h0 += 8 * HB) {
+        float acc[HB][R];
+#pragma unroll
+        for (int q = 0; q < HB; ++q)
+#pragma unroll
+            for (int r = 0; r < R; ++r) acc[q][r] = 0.0f;
+        for (int col = lane; col < C; col += 32) {
+            float w[HB];
+#pragma unroll
+            for (int q = 0; q < HB; ++q) w[q] = h0 + q < Hq ? __ldg(W + (size_t)(h0 + q) * C + col) : 0.0f;
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                const float v = sV[(size_t)r * C + col];
+#pragma unroll
+                for (int q = 0; q < HB; ++q) acc[q][r] = fmaf(v, w[q], acc[q][r]);
+            }
+        }
+#pragma unroll
+        for (int q = 0; q < HB; ++q) {
+#pragma unroll
+            for (int base = 0; base < R; base += RL) {
+#pragma unroll
+                for (int keep = RL >> 1; keep >= 1; keep >>= 1) {
+                    const bool up = (lane & keep) != 0;
+#pragma unroll
+                    for (int r = 0; r < keep; ++r) {
+                        const float stay = up ? acc[q][base + r + keep] : acc[q][base + r];
+                        const float give = up ? acc[q][base + r] : acc[q][base + r + keep];
+                        acc[q][base + r] = stay + __shfl_xor_sync(0xffffffffu, give, keep);
+                    }
+                }
+#pragma unroll
+                for (int m = RL; m < 32; m <<= 1) acc[q][base] += __shfl_xor_sync(0xffffffffu, acc[q][base], m);
+                if (lane < RL && h0 + q < Hq) sZ[(h0 + q) * R + base + lane] = acc[q][base];
+            }
+        }
+    }
+    __syncthreads();
+
+    for (int i = tid; i < Hq * R; i += kThreads) {
+        const int h = i / R, row = i % R, j = j0 + row;
+        float dz = 0.0f, gs = 0.0f;
+        if (j < L) {
+            const size_t at = ((size_t)b * Hq + h) * L + j;
+            const float gd = dM[at] * delta[at];
+            const float z = sZ[i];
+            const float e = __expf(-fabsf(z));
+            gs = gd * (fmaxf(z, 0.0f) + log1pf(e));
+            dz = gd * A[h] * ((z >= 0.0f ? 1.0f : e) / (1.0f + e));
+        }
+        sDz[row * HqP + h] = dz;
+        sZ[i] = gs;
+    }
+    __syncthreads();
+
+    float* out = partial + ((size_t)b * gridDim.x + blockIdx.x) * Hq * (C + 1);
+    for (int col = tid; col < C; col += kThreads) {
+        for (int hc = 0; hc < HqP; hc += 8) {
+            float acc[8];
+#pragma unroll
+            for (int q = 0; q < 8; ++q) acc[q] = 0.0f;
+            for (int row = 0; row < R; ++row) {
+                const float v = sV[(size_t)row * C + col];
+                const float4 a = *reinterpret_cast<const float4*>(sDz + row * HqP + hc);
+                const float4 c = *reinterpret_cast<const float4*>(sDz + row * HqP + hc + 4);
+                acc[0] = fmaf(a.x, v, acc[0]); acc[1] = fmaf(a.y, v, acc[1]); acc[2] = fmaf(a.z, v, acc[2]); acc[3] = fmaf(a.w, v, acc[3]);
+                acc[4] = fmaf(c.x, v, acc[4]); acc[5] = fmaf(c.y, v, acc[5]); acc[6] = fmaf(c.z, v, acc[6]); acc[7] = fmaf(c.w, v, acc[7]);
+            }
+#pragma unroll
+            for (int q = 0; q < 8; ++q)
+                if (hc + q < Hq) out[(size_t)(hc + q) * (C + 1) + col] = acc[q];
+        }
+    }
+    if (tid < Hq) {
+        float t = 0.0f;
+        for (int row = 0; row < R; ++row) t += sZ[tid * R + row];
+        out[(size_t)tid * (C + 1) + C] = t;
+    }
+    __syncthreads();   // every thread is done with the values of its columns' neighbours: the tile may be overwritten
+
+    for (int col = tid; col < C; col += kThreads) {
+        for (int hc = 0; hc < HqP; hc += 8) {
+            float w[8];
+#pragma unroll
+            for (int q = 0; q < 8; ++q) w[q] = hc + q < Hq ? __ldg(W + (size_t)(hc + q) * C + col) : 0.0f;
+            for (int row = 0; row < R; ++row) {
+                const float4 a = *reinterpret_cast<const float4*>(sDz + row * HqP + hc);
+                const float4 c = *reinterpret_cast<const float4*>(sDz + row * HqP + hc + 4);
+                float u = a.x * w[0];
+                u = fmaf(a.y, w[1], u); u = fmaf(a.z, w[2], u); u = fmaf(a.w, w[3], u);
+                u = fmaf(c.x, w[4], u); u = fmaf(c.y, w[5], u); u = fmaf(c.z, w[6], u); u = fmaf(c.w, w[7], u);
+                float* dst = sV + (size_t)row * C + col;
+                *dst = hc == 0 ? u : *dst + u;
+            }
+        }
+    }
+    __syncthreads();
+
+    for (int i = tid; i < R * C8; i += kThreads) {
+        const int row = i / C8, ch = i % C8, j = j0 + row;
+        if (j < L) {
+            T* p = dV + b * vs_b + (int64_t)j * vs_l + (ch / D8) * vs_h + (ch % D8) * 8;
+            float cur[8];
+            load8f(p, cur);
+#pragma unroll
+            for (int c = 0; c < 8; ++c) cur[c] += sV[(size_t)row * C + ch * 8 + c];
+            store8f(p, cur);
+        }
+    }
+}
+
+// dW [Hq][C] and dA [Hq] from partial [n][Hq][C + 1]: four groups of threads each add every fourth partial in index order,
+// then the group sums are added in group order.
+__global__ void __launch_bounds__(512) mask_bwd_full_reduce_kernel(const float* __restrict__ partial, float* __restrict__ dW,
+                                                                   float* __restrict__ dA, int n, int Hq, int C) {
+    __shared__ float part[4][128];
+    const int h = blockIdx.y, c = blockIdx.x * 128 + (threadIdx.x & 127), grp = threadIdx.x >> 7;
+    float s = 0.0f;
+    if (c <= C)
+        for (int t = grp; t < n; t += 4) s += partial[((size_t)t * Hq + h) * (C + 1) + c];
+    part[grp][threadIdx.x & 127] = s;
+    __syncthreads();
+    if (grp == 0 && c <= C) {
+        const float tot = ((part[0][threadIdx.x] + part[1][threadIdx.x]) + part[2][threadIdx.x]) + part[3][threadIdx.x];
+        if (c < C) dW[(size_t)h * C + c] = tot; else dA[h] = tot;
+    }
+}
+
+// rows per CTA: the largest of 64, 32, 16, 8 whose tile fits 200 KiB of shared memory (0: none does)
+static int full_rows(const Prob& P) {
+    const size_t C = (size_t)P.Hkv * P.d, HqP = (P.Hq + 7) & ~7;
+    for (int R = 64; R >= 8; R >>= 1)
+        if ((R * C + R * HqP + (size_t)P.Hq * R) * sizeof(float) <= 200 * 1024) return R;
+    return 0;
+}
+
 }  // namespace
 
 size_t mask_bwd_ws_bytes(const Prob& P) {
+    if (P.flags & DMA_FLAG_FULL_DELTA) {
+        const int R = full_rows(P);
+        if (R == 0) return 0;
+        return (size_t)P.B * ((P.L + R - 1) / R) * P.Hq * ((size_t)P.Hkv * P.d + 1) * sizeof(float);
+    }
     const size_t nblk = (size_t)(P.L + kRows - 1) / kRows;
     return (size_t)P.B * P.Hkv * nblk * P.G * (P.d + 1) * sizeof(float);
 }
@@ -187,8 +370,38 @@ static int launch_typed(const Prob& P, const void* V, const float* W, const floa
     return check_launch();
 }
 
+template <typename T, int RW>
+static int launch_full(const Prob& P, const void* V, const float* W, const float* A, const float* delta, const float* dM,
+                       void* dV, float* dW, float* dA, void* ws, cudaStream_t st) {
+    constexpr int R = RW * 8;
+    const int nblk = (P.L + R - 1) / R, C = P.Hkv * P.d, HqP = (P.Hq + 7) & ~7;
+    const size_t smem = ((size_t)R * C + (size_t)R * HqP + (size_t)P.Hq * R) * sizeof(float);
+    if (cudaFuncSetAttribute(mask_bwd_full_kernel<T, RW>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+        return DMA_ERR_CUDA;
+    mask_bwd_full_kernel<T, RW><<<dim3(nblk, P.B), kThreads, smem, st>>>((const T*)V, W, A, delta, dM, (T*)dV, (float*)ws, P.L, P.Hq,
+                                                                          P.Hkv, P.d, P.vs[0], P.vs[1], P.vs[2]);
+    mask_bwd_full_reduce_kernel<<<dim3((C + 1 + 127) / 128, P.Hq), 512, 0, st>>>((const float*)ws, dW, dA, P.B * nblk, P.Hq, C);
+    count_launch(2);
+    return check_launch();
+}
+
+template <typename T>
+static int launch_full_rows(const Prob& P, const void* V, const float* W, const float* A, const float* delta, const float* dM,
+                            void* dV, float* dW, float* dA, void* ws, cudaStream_t st) {
+    switch (full_rows(P)) {
+        case 64: return launch_full<T, 8>(P, V, W, A, delta, dM, dV, dW, dA, ws, st);
+        case 32: return launch_full<T, 4>(P, V, W, A, delta, dM, dV, dW, dA, ws, st);
+        case 16: return launch_full<T, 2>(P, V, W, A, delta, dM, dV, dW, dA, ws, st);
+        case 8: return launch_full<T, 1>(P, V, W, A, delta, dM, dV, dW, dA, ws, st);
+    }
+    return DMA_ERR_UNSUPPORTED;
+}
+
 int launch_mask_bwd(const Prob& P, const void* V, const float* W, const float* A, const float* delta, const float* dM,
                     void* dV, float* dW, float* dA, void* ws, cudaStream_t st) {
+    if (P.flags & DMA_FLAG_FULL_DELTA)
+        return P.dtype == DMA_BF16 ? launch_full_rows<__nv_bfloat16>(P, V, W, A, delta, dM, dV, dW, dA, ws, st)
+                                   : launch_full_rows<float>(P, V, W, A, delta, dM, dV, dW, dA, ws, st);
     if (P.G > 16) return DMA_ERR_UNSUPPORTED;
     if (P.dtype == DMA_BF16) {
         return P.d == 128 ? launch_typed<__nv_bfloat16, 128>(P, V, W, A, delta, dM, dV, dW, dA, ws, st)

@@ -18,7 +18,7 @@ struct Arena {
 
 struct Layout {
     size_t Q, K, V, dO, O, dQ, dK, dV, W, A, bias, expiry, bitmap, lse, dM, ws_mask, ws_fwd, ws_bwd, total;
-    size_t nq, nk, nbh, nbmp, m_ws, f_ws, b_ws, esz;
+    size_t nq, nk, nbh, nbmp, m_ws, f_ws, b_ws, esz, wbytes;
 };
 
 int make_layout(const dma_problem_t* p, int backward, Layout* Lo) {
@@ -36,7 +36,8 @@ int make_layout(const dma_problem_t* p, int backward, Layout* Lo) {
     Arena a;
     Lo->Q = a.take(Lo->nq * Lo->esz); Lo->K = a.take(Lo->nk * Lo->esz); Lo->V = a.take(Lo->nk * Lo->esz);
     Lo->O = a.take(Lo->nq * Lo->esz);
-    Lo->W = a.take((size_t)P.Hq * P.d * 4); Lo->A = a.take((size_t)P.Hq * 4);
+    Lo->wbytes = (size_t)P.Hq * ((P.flags & DMA_FLAG_FULL_DELTA) ? P.Hkv * P.d : P.d) * 4;
+    Lo->W = a.take(Lo->wbytes); Lo->A = a.take((size_t)P.Hq * 4);
     Lo->bias = a.take(Lo->nbh * 4); Lo->expiry = a.take(Lo->nbh * 4); Lo->bitmap = a.take(Lo->nbmp * 4);
     Lo->lse = a.take(Lo->nbh * 4);
     Lo->ws_mask = a.take(Lo->m_ws); Lo->ws_fwd = a.take(Lo->f_ws);
@@ -97,7 +98,7 @@ int dma_step_host(const dma_problem_t* p, int backward, const void* hQ, const vo
     auto rec = [&](int e, cudaStream_t on) { return cudaEventRecord(ev[e], on) == cudaSuccess; };
     auto wait = [&](cudaStream_t on, int e) { return cudaStreamWaitEvent(on, ev[e], 0) == cudaSuccess; };
     bool ok = rec(kStart, st) && wait(s_in, kStart) && wait(s_out, kStart);
-    ok = ok && h2d(Lo.V, hV, Lo.nk * Lo.esz) && h2d(Lo.W, hW_delta, (size_t)p->Hq * p->d * 4) && h2d(Lo.A, hA, (size_t)p->Hq * 4) && rec(kV, s_in);
+    ok = ok && h2d(Lo.V, hV, Lo.nk * Lo.esz) && h2d(Lo.W, hW_delta, Lo.wbytes) && h2d(Lo.A, hA, (size_t)p->Hq * 4) && rec(kV, s_in);
     ok = ok && h2d(Lo.K, hK, Lo.nk * Lo.esz) && h2d(Lo.Q, hQ, Lo.nq * Lo.esz) && rec(kKQ, s_in);
     if (backward) ok = ok && h2d(Lo.dO, hdO, Lo.nq * Lo.esz) && rec(kdO, s_in);
     if (!ok) return cleanup(DMA_ERR_CUDA);

@@ -74,6 +74,14 @@ def _structured_z(case: Case, g: torch.Generator) -> torch.Tensor:
     return z
 
 
+def full_delta_weights(case: Case) -> torch.Tensor:
+    """Sampling weights over the whole value row, [Hq, Hkv*d] fp32 ~ N(0, 1/(Hkv*d)) (the z scale of the per-head
+    recipe), from the case's seed."""
+    g = torch.Generator().manual_seed(case.seed + 77)
+    c = case.Hkv * case.d
+    return (torch.randn(case.Hq, c, generator=g) / math.sqrt(c)).contiguous()
+
+
 def make_inputs(case: Case) -> dict:
     """CPU tensors: Q,dO [B,L,Hq,d]; K,V [B,L,Hkv,d] in the case's dtype; W_delta [Hq,d], A [Hq] fp32."""
     g = torch.Generator().manual_seed(case.seed)
