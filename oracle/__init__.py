@@ -107,6 +107,20 @@ def select_expiry(dl, w):
     return e
 
 
+def select_expiry_varlen(dl, w, cu_seqlens):
+    """Selection for a batch of sequences packed along the key axis (sequence s owns the keys cu[s] <= j < cu[s+1]):
+    every sequence is selected on its own (Sec. 4.1 applied per sequence: a row sees only the keys of its own
+    sequence up to itself), so the result is select_expiry of each slice, shifted to packed indices. Key j is then
+    kept by the rows j <= i < expiry[j] of the packed axis, and expiry[j] never passes the end of j's sequence."""
+    dl = _c(dl, np.float32)
+    cu = [int(c) for c in cu_seqlens]
+    assert cu[0] == 0 and cu[-1] == dl.shape[-1] and all(a < b for a, b in zip(cu, cu[1:]))
+    e = np.empty(dl.shape, np.int32)
+    for s0, s1 in zip(cu, cu[1:]):
+        e[..., s0:s1] = select_expiry(dl[..., s0:s1], w) + s0
+    return e
+
+
 def keep_from_expiry(e):
     e = _c(e, np.int32)
     L = e.shape[-1]
