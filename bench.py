@@ -306,6 +306,36 @@ def main():
                             "step_ms": stage_ms["mask"] + c_ms + cb_ms, "tile_step_ms": sum(stage_ms.values()),
                             "dK_max_abs_diff_vs_tile_path": float((dKc.float() - dK.float()).abs().max())})
 
+    # ---- the same tensors read as 12 documents packed along the sequence axis (dma_mask_build_varlen; the attention
+    # kernels are unchanged): the bitmap becomes block-diagonal and tile skipping removes the other documents' tiles
+    varlen = None
+    if case.L >= 4096:
+        cu = wl.packed_cu_seqlens(case.L, 12, seed=31)
+        cu_t = torch.tensor(cu, dtype=torch.int32, device=dev)
+        bias_v, exp_v, bmp_v = torch.empty_like(bias), torch.empty_like(expiry), torch.empty_like(bitmap)
+        Ov, lsev = torch.empty_like(O), torch.empty_like(lse)
+        stages = [lambda: dma.dma_mask_build_varlen(p, V, W, A, cu_t, bias_v, exp_v, bmp_v, ws_m),
+                  lambda: dma.dma_attn_fwd(p, Q, K, V, bias_v, exp_v, bmp_v, Ov, lsev, ws_f)]
+        if case.backward:
+            stages.append(lambda: dma.dma_attn_bwd(p, Q, K, V, Ov, dO, lsev, bias_v, exp_v, bmp_v, dQ, dK, dV, dM, ws_b))
+        v_ms = []
+        for f in stages:
+            for _ in range(3):
+                f()
+            g0, g1 = ev(), ev()
+            barrier()
+            g0.record()
+            for _ in range(10):
+                f()
+            g1.record()
+            barrier()
+            v_ms.append(g0.elapsed_time(g1) / 10)
+        act_v = int(sum(bin(int(x) & 0xFFFFFFFF).count("1") for x in bmp_v.cpu().numpy().ravel()))
+        v_step = sum(v_ms)
+        varlen = {"documents": 12, "lengths": [b - a for a, b in zip(cu, cu[1:])], "mask_ms": v_ms[0], "fwd_ms": v_ms[1],
+                  "bwd_ms": v_ms[2] if case.backward else None, "step_ms": v_step, "active_tiles": act_v,
+                  "tflops_executed_tiles": tile_flops(act_v, case.d, case.backward) / (v_step * 1e-3) / 1e12}
+
     # ---- one decoding step over this workload's K / V as the cache (dma_delta_range + dma_decode), timed on its own
     decode = None
     if rank == 0:
@@ -395,6 +425,8 @@ def main():
         out["compact"] = compact
     if full_delta is not None:
         out["full_delta"] = full_delta
+    if varlen is not None:
+        out["varlen"] = varlen
     if mask_bwd is not None:
         mask_bwd["frac_of_measured_hbm"] = mask_bwd["gbs"] / pk["hbm_gbs"]
         out["mask_bwd"] = mask_bwd

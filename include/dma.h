@@ -118,6 +118,18 @@ int dma_mask_build(const dma_problem_t* p, const void* V, const float* W_delta, 
 int dma_mask_build_static(const dma_problem_t* p, const void* V, const float* W_delta, const float* A,
                           float* bias, int32_t* expiry, uint32_t* bitmap, void* cuda_stream);
 
+/* Mask generation for sequences packed along the sequence axis (variable-length batches; the method applied to each
+ * sequence on its own). cu_seqlens: DEVICE memory, nseq + 1 int32, cu[0] = 0 < cu[1] < ... < cu[nseq] = L: sequence s
+ * owns positions cu[s] <= j < cu[s+1] of every batch entry. Row i sees the keys of its own sequence up to itself and
+ * keeps the min(w, visible) best of them. Same outputs as dma_mask_build in packed coordinates: key j is kept by the
+ * rows j <= i < expiry[j], and expiry[j] never passes the end of j's sequence, so no row reaches into another
+ * sequence. dma_attn_fwd, dma_attn_bwd and dma_mask_bwd take the triple as it is: nothing else changes for packed
+ * batches (the bitmap becomes block-diagonal, so whole key tiles of other sequences are skipped). The contents of
+ * cu_seqlens are not checked (reading them would synchronise); offsets outside [0, L] are clamped. */
+int dma_mask_build_varlen(const dma_problem_t* p, const void* V, const float* W_delta, const float* A,
+                          const int32_t* cu_seqlens, int32_t nseq, float* bias, int32_t* expiry, uint32_t* bitmap,
+                          void* ws, size_t ws_bytes, void* cuda_stream);
+
 /* Forward (Sec. 4.2, Eq. (attention_output), Alg. 1): for each row i of head h
  *   s_j = q_i . k_j * scale + bias[j]   over keys with j <= i < expiry[j];   p = softmax(s);   O_i = sum p_j v_j
  *   lse_i = log sum_j exp(s_j)   (natural log; replaces Alg. 1's (l, m) pair)

@@ -18,7 +18,8 @@ DMA_FLAG_IGNORE_BITMAP, DMA_FLAG_SIMT, DMA_FLAG_COMPACT_KV, DMA_FLAG_FULL_DELTA 
 
 ENTRY_POINTS = ("dma_query_workspace", "dma_bitmap_words", "dma_mask_build", "dma_attn_fwd", "dma_attn_bwd",
                 "dma_read_status", "dma_launch_count", "dma_strerror", "dma_step_host_arena", "dma_step_host", "dma_mask_build_static", "dma_selftest_wait_timeout",
-                "dma_mask_bwd_workspace", "dma_mask_bwd", "dma_delta_range", "dma_decode_workspace", "dma_decode")
+                "dma_mask_bwd_workspace", "dma_mask_bwd", "dma_delta_range", "dma_decode_workspace", "dma_decode",
+                "dma_mask_build_varlen")
 
 
 class DmaError(RuntimeError):
@@ -108,6 +109,26 @@ def dma_mask_build(p, V, W_delta, A, bias=None, expiry=None, bitmap=None, ws=Non
         ws = _ws(dma_query_workspace(p)[0], dev)
     _check(lib().dma_mask_build(ctypes.byref(p), _ptr(V), _ptr(W_delta), _ptr(A), _ptr(bias), _ptr(expiry), _ptr(bitmap),
                                 _ptr(ws), ctypes.c_size_t(ws.numel()), _stream()), "dma_mask_build")
+    return bias, expiry, bitmap
+
+
+def dma_mask_build_varlen(p, V, W_delta, A, cu_seqlens, bias=None, expiry=None, bitmap=None, ws=None):
+    """dma_mask_build for sequences packed along the sequence axis; cu_seqlens: int32 device tensor [nseq + 1]."""
+    dev = V.device
+    assert cu_seqlens.dtype == torch.int32 and cu_seqlens.is_cuda and cu_seqlens.is_contiguous()
+    if bias is None:
+        bias = torch.empty(p.B, p.Hq, p.L, dtype=torch.float32, device=dev)
+    if expiry is None:
+        expiry = torch.empty(p.B, p.Hq, p.L, dtype=torch.int32, device=dev)
+    if bitmap is None:
+        tm, tn = (p.tile_m or 128), (p.tile_n or 128)
+        Tr, Tc = -(-p.L // tm), -(-p.L // tn)
+        bitmap = torch.empty(p.B, p.Hq, Tr, (Tc + 31) // 32, dtype=torch.int32, device=dev)
+    if ws is None:
+        ws = _ws(dma_query_workspace(p)[0], dev)
+    _check(lib().dma_mask_build_varlen(ctypes.byref(p), _ptr(V), _ptr(W_delta), _ptr(A), _ptr(cu_seqlens),
+                                       ctypes.c_int32(cu_seqlens.numel() - 1), _ptr(bias), _ptr(expiry), _ptr(bitmap),
+                                       _ptr(ws), ctypes.c_size_t(ws.numel()), _stream()), "dma_mask_build_varlen")
     return bias, expiry, bitmap
 
 

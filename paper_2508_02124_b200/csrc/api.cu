@@ -113,6 +113,21 @@ int dma_mask_build(const dma_problem_t* p, const void* V, const float* W_delta, 
     return launch_mask_build(P, V, W_delta, A, bias, expiry, bitmap, ws, (cudaStream_t)cuda_stream);
 }
 
+int dma_mask_build_varlen(const dma_problem_t* p, const void* V, const float* W_delta, const float* A,
+                          const int32_t* cu_seqlens, int32_t nseq, float* bias, int32_t* expiry, uint32_t* bitmap,
+                          void* ws, size_t ws_bytes, void* cuda_stream) {
+    Prob P;
+    int rc = resolve(p, &P);
+    if (rc) return rc;
+    if (!V || !W_delta || !A || !cu_seqlens || !bias || !expiry || !bitmap) return DMA_ERR_NULL;
+    if (nseq < 1 || nseq > P.L) return DMA_ERR_SHAPE;
+    if (!aligned16(V) || !aligned16(W_delta) || !aligned16(bias) || !aligned16(expiry) || !aligned16(bitmap))
+        return DMA_ERR_ALIGN;
+    if (!ws || ws_bytes < mask_ws_bytes(P) || !aligned16(ws)) return DMA_ERR_WORKSPACE;
+    if ((rc = device_ok())) return rc;
+    return launch_mask_build(P, V, W_delta, A, bias, expiry, bitmap, ws, (cudaStream_t)cuda_stream, cu_seqlens, nseq);
+}
+
 int dma_mask_bwd_workspace(const dma_problem_t* p, size_t* bytes) {
     Prob P;
     int rc = resolve(p, &P);

@@ -235,23 +235,44 @@ __global__ void __launch_bounds__(kChunk) chunk_sort_kernel(const float* __restr
 // words, the next one already in flight) and every thread counts its beaters chunk by chunk with a binary search
 // until the count reaches w. Phase 2: the warp locates, lane by lane, the remaining need-th beater inside that
 // lane's final chunk with coalesced 32-key loads and a ballot.
+// kVarlen: sequences packed along the key axis (sequence s owns the keys cu[s] <= j < cu[s+1]). A key competes only
+// with the keys of its own sequence [s0, s1): chunks before s0 count nothing, a chunk that straddles s0 or s1 is
+// counted entry by entry with the index test, the walk ends at s1, and L is replaced by s1.
+template <bool kVarlen>
 __global__ void __launch_bounds__(kExpThreads) expiry_kernel(const float* __restrict__ delta,
                                                              const unsigned long long* __restrict__ sorted,
-                                                             int32_t* __restrict__ expiry, int L, int w, int nchunk) {
+                                                             int32_t* __restrict__ expiry, int L, int w, int nchunk,
+                                                             const int32_t* __restrict__ cu, int nseq) {
     constexpr int kPer = kChunk / kExpThreads;
     __shared__ uint32_t shi[2][kChunk], slo[2][kChunk];
+    __shared__ int c_first;
     const int bh = blockIdx.y, t = threadIdx.x, lane = t & 31, j = blockIdx.x * kExpThreads + t;
     const float* dl = delta + (size_t)bh * L;
     const unsigned long long* srt = sorted + (size_t)bh * nchunk * kChunk;
     const bool valid = j < L;
     const unsigned long long key = valid ? sort_key(dl[j], j) : ~0ull;
     const uint32_t khi = (uint32_t)(key >> 32), klo = (uint32_t)key;
+    int s0 = 0, s1 = L;
+    if (kVarlen) {
+        if (valid) {
+            int lo = 0, hi = nseq;                         // largest s with cu[s] <= j
+            while (hi - lo > 1) {
+                const int mid = (lo + hi) >> 1;
+                if (cu[mid] <= j) lo = mid; else hi = mid;
+            }
+            s0 = max(cu[lo], 0);
+            s1 = min(cu[lo + 1], L);
+        }
+        if (t == 0) c_first = s0 / kChunk;                 // the CTA's first key has the smallest sequence start
+        __syncthreads();
+    }
+    const int c_begin = kVarlen ? c_first : 0;
     int cnt = 0, fin = -1, need = 0;
     bool done = !valid;
     unsigned long long nxt[kPer];
 #pragma unroll
-    for (int u = 0; u < kPer; ++u) nxt[u] = srt[u * kExpThreads + t];
-    for (int c = 0; c < nchunk; ++c) {
+    for (int u = 0; u < kPer; ++u) nxt[u] = srt[(size_t)c_begin * kChunk + u * kExpThreads + t];
+    for (int c = c_begin; c < nchunk; ++c) {
         uint32_t* hi = shi[c & 1];
         uint32_t* lo = slo[c & 1];
 #pragma unroll
@@ -264,33 +285,48 @@ __global__ void __launch_bounds__(kExpThreads) expiry_kernel(const float* __rest
             for (int u = 0; u < kPer; ++u) nxt[u] = srt[(size_t)(c + 1) * kChunk + u * kExpThreads + t];
         }
         __syncthreads();
+        if (kVarlen && !done && c * kChunk >= s1) done = true;          // past the end of the sequence: expiry = s1
         if (!done) {
-            // a = first position whose 64-bit key is greater than ours: fixed-depth, branch-free lower bound on the
-            // high words (delta bits), then the (normally empty) run of equal high words is resolved by the low words
-            int a = 0;
+            int n;
+            if (!kVarlen || (c * kChunk >= s0 && (c + 1) * kChunk <= s1)) {
+                // a = first position whose 64-bit key is greater than ours: fixed-depth, branch-free lower bound on
+                // the high words (delta bits), then the (normally empty) run of equal high words is resolved by the
+                // low words
+                int a = 0;
 #pragma unroll
-            for (int s = kChunk / 2; s > 0; s >>= 1) a += hi[a + s - 1] < khi ? s : 0;
-            a += hi[a] < khi ? 1 : 0;                      // a = number of entries with hi < khi (0 .. kChunk)
-            while (a < kChunk && hi[a] == khi && lo[a] <= klo) ++a;
-            const int n = kChunk - a;
+                for (int s = kChunk / 2; s > 0; s >>= 1) a += hi[a + s - 1] < khi ? s : 0;
+                a += hi[a] < khi ? 1 : 0;                      // a = number of entries with hi < khi (0 .. kChunk)
+                while (a < kChunk && hi[a] == khi && lo[a] <= klo) ++a;
+                n = kChunk - a;
+            } else if ((c + 1) * kChunk <= s0) {
+                n = 0;
+            } else {
+                n = 0;
+                for (int a = 0; a < kChunk; ++a) {
+                    const int idx = (int)(0xFFFFFFFFu - lo[a]);
+                    const bool beats = hi[a] > khi || (hi[a] == khi && lo[a] > klo);
+                    n += (beats && idx >= s0 && idx < s1) ? 1 : 0;
+                }
+            }
             if (cnt + n >= w) { need = w - cnt; fin = c; done = true; }
             cnt += n;
         }
         if (__syncthreads_and(done)) break;
     }
     // phase 2, warp-cooperative: lane `src` broadcasts (chunk, key, need); the warp scans that chunk 32 keys at a time
-    int e = L;
+    int e = s1;
     const uint32_t pending = __ballot_sync(0xffffffffu, fin >= 0);
     for (uint32_t rest = pending; rest; rest &= rest - 1) {
         const int src = __ffs(rest) - 1;
         const int base = __shfl_sync(0xffffffffu, fin, src) * kChunk;
         const uint32_t bhi = __shfl_sync(0xffffffffu, khi, src), blo = __shfl_sync(0xffffffffu, klo, src);
+        const int b0 = __shfl_sync(0xffffffffu, s0, src), b1 = __shfl_sync(0xffffffffu, s1, src);
         int nd = __shfl_sync(0xffffffffu, need, src);
         const unsigned long long bkey = ((unsigned long long)bhi << 32) | blo;
-        int found = L;
+        int found = b1;
         for (int g = 0; g < kChunk; g += 32) {
             const int k = base + g + lane;
-            const bool beat = k < L && sort_key(dl[k], k) > bkey;
+            const bool beat = k >= b0 && k < b1 && sort_key(dl[k], k) > bkey;
             uint32_t m = __ballot_sync(0xffffffffu, beat);
             const int pc = __popc(m);
             if (nd <= pc) {
@@ -381,7 +417,7 @@ int launch_delta_range(const Prob& P, const void* V, const float* W, const float
 }
 
 int launch_mask_build(const Prob& P, const void* V, const float* W, const float* A, float* bias, int32_t* expiry,
-                      uint32_t* bitmap, void* ws, cudaStream_t st) {
+                      uint32_t* bitmap, void* ws, cudaStream_t st, const int32_t* cu, int nseq) {
     int rc;
     if (P.dtype == DMA_BF16)
         rc = P.d == 128 ? launch_delta<__nv_bfloat16, 128>(P, V, W, A, bias, st)
@@ -392,14 +428,16 @@ int launch_mask_build(const Prob& P, const void* V, const float* W, const float*
 
     const int BH = P.B * P.Hq;
     const int nchunk = (P.L + kChunk - 1) / kChunk;
-    if (P.w >= P.L) {   // every visible key is kept
+    if (P.w >= P.L && !cu) {   // every visible key is kept
         size_t n = (size_t)BH * P.L;
         fill_i32_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(expiry, n, P.L);
         count_launch();
     } else {
         auto* sorted = reinterpret_cast<unsigned long long*>((char*)ws + kWsHeaderBytes);
         chunk_sort_kernel<<<dim3(nchunk, BH), kChunk, 0, st>>>(bias, sorted, P.L, nchunk);
-        expiry_kernel<<<dim3((P.L + kExpThreads - 1) / kExpThreads, BH), kExpThreads, 0, st>>>(bias, sorted, expiry, P.L, P.w, nchunk);
+        const dim3 grid((P.L + kExpThreads - 1) / kExpThreads, BH);
+        if (cu) expiry_kernel<true><<<grid, kExpThreads, 0, st>>>(bias, sorted, expiry, P.L, P.w, nchunk, cu, nseq);
+        else expiry_kernel<false><<<grid, kExpThreads, 0, st>>>(bias, sorted, expiry, P.L, P.w, nchunk, nullptr, 0);
         count_launch(2);
     }
     if ((rc = check_launch())) return rc;

@@ -82,6 +82,20 @@ def full_delta_weights(case: Case) -> torch.Tensor:
     return (torch.randn(case.Hq, c, generator=g) / math.sqrt(c)).contiguous()
 
 
+def packed_cu_seqlens(L: int, nseq: int, seed: int) -> list:
+    """Sequence offsets [0, ..., L] of nseq documents packed into L positions: log-normal lengths (a few long
+    documents, many short ones, as in packed pre-training batches), every length >= 1, nothing aligned to a tile."""
+    g = torch.Generator().manual_seed(seed)
+    wts = torch.exp(torch.randn(nseq, generator=g))
+    lens = torch.clamp((wts / wts.sum() * (L - nseq)).floor().long() + 1, min=1)
+    lens[-1] += L - int(lens.sum())
+    assert int(lens.min()) >= 1
+    cu = [0]
+    for n in lens.tolist():
+        cu.append(cu[-1] + n)
+    return cu
+
+
 def make_inputs(case: Case) -> dict:
     """CPU tensors: Q,dO [B,L,Hq,d]; K,V [B,L,Hkv,d] in the case's dtype; W_delta [Hq,d], A [Hq] fp32."""
     g = torch.Generator().manual_seed(case.seed)

@@ -1,0 +1,122 @@
+"""GPU parity for sequences packed along the sequence axis (dma_mask_build_varlen): the mask bit for bit against the
+oracle's per-sequence selection, and the unchanged attention kernels on the resulting block-diagonal masks."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2508_02124_b200 import binding as dma
+from paper_2508_02124_b200 import workloads as wl
+from helpers import assert_close, f64, problem_of, round_to
+from test_gpu_attention import compare, oracle_all
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+C1, C2 = wl.CONFIGS["1"], wl.CONFIGS["2"]
+
+SMALL = [
+    (wl.small(C1, L=37, w=4, name="varlen fp32 tiny"), [0, 5, 6, 20, 37]),
+    (wl.small(C1, B=2, L=600, w=64, name="varlen fp32 boundaries inside a chunk"), [0, 100, 255, 256, 257, 511, 600]),
+    (wl.small(C1, L=300, w=500, name="varlen fp32 w above every length"), [0, 140, 300]),
+    (wl.small(C2, B=1, Hq=4, Hkv=2, L=1000, w=129, backward=True, name="varlen bf16 ragged gqa"), [0, 1, 333, 334, 900, 1000]),
+    (wl.small(C2, B=2, Hq=4, Hkv=1, L=1536, w=200, backward=True, name="varlen bf16 three documents"), [0, 700, 829, 1536]),
+    (wl.small(C2, B=1, Hq=2, Hkv=2, L=1024, w=64, backward=True, name="varlen bf16 tile-aligned"), [0, 256, 512, 1024]),
+    (wl.small(C2, B=1, Hq=4, Hkv=4, L=512, w=64, d=64, backward=True, name="varlen bf16 d64"), [0, 77, 300, 512]),
+]
+
+
+def run(case, cu, flags=0, backward=True):
+    inp = wl.make_inputs(case)
+    p = problem_of(case, flags=flags)
+    Q, K, V, dO = (inp[k].to(DEV) for k in ("Q", "K", "V", "dO"))
+    cu_t = torch.tensor(cu, dtype=torch.int32, device=DEV)
+    bias, expiry, bitmap = dma.dma_mask_build_varlen(p, V, inp["W_delta"].to(DEV), inp["A"].to(DEV), cu_t)
+    O, lse = dma.dma_attn_fwd(p, Q, K, V, bias, expiry, bitmap)
+    got = {"bias": bias, "expiry": expiry, "bitmap": bitmap, "O": O, "lse": lse}
+    if backward:
+        dQ, dK, dV, dM = dma.dma_attn_bwd(p, Q, K, V, O, dO, lse, bias, expiry, bitmap)
+        got.update(dQ=dQ, dK=dK, dV=dV, dM=dM)
+    torch.cuda.synchronize()
+    return inp, got
+
+
+def oracle_varlen_mask(case, inp, cu):
+    _, dl = oracle.delta(inp["V"].float().numpy(), inp["W_delta"].numpy(), inp["A"].numpy(), case.Hq)
+    e = oracle.select_expiry_varlen(dl, min(case.w, case.L), cu)
+    return dl, e, oracle.bitmap_from_expiry(e)
+
+
+@pytest.mark.parametrize("case,cu", SMALL, ids=lambda v: v.name if hasattr(v, "name") else "")
+def test_mask_and_attention_small(case, cu):
+    inp, got = run(case, cu)
+    dl, e, bmp = oracle_varlen_mask(case, inp, cu)
+    assert np.array_equal(got["bias"].cpu().numpy().view(np.uint32), dl.view(np.uint32))
+    assert np.array_equal(got["expiry"].cpu().numpy(), e)
+    assert np.array_equal(got["bitmap"].cpu().numpy().view(np.uint32), bmp)
+    compare(case, got, oracle_all(case, inp, dl, e))
+
+
+@pytest.mark.parametrize("case,cu", [c for c in SMALL if c[0].dtype == "bf16" and c[0].d == 128],
+                         ids=lambda v: v.name if hasattr(v, "name") else "")
+def test_token_compacted_kernels_on_packed_sequences(case, cu):
+    inp, got = run(case, cu, flags=dma.DMA_FLAG_COMPACT_KV)
+    dl, e, _ = oracle_varlen_mask(case, inp, cu)
+    compare(case, got, oracle_all(case, inp, dl, e))
+
+
+def test_one_sequence_equals_the_plain_mask_build():
+    case = wl.small(C2, B=1, Hq=4, Hkv=2, L=2000, w=300, name="varlen one sequence")
+    inp = wl.make_inputs(case)
+    p = problem_of(case)
+    V, W, A = inp["V"].to(DEV), inp["W_delta"].to(DEV), inp["A"].to(DEV)
+    a = dma.dma_mask_build(p, V, W, A)
+    b = dma.dma_mask_build_varlen(p, V, W, A, torch.tensor([0, case.L], dtype=torch.int32, device=DEV))
+    torch.cuda.synchronize()
+    for x, y in zip(a, b):
+        assert torch.equal(x, y)
+
+
+def test_config3_packed_documents():
+    """Config 3's shapes with 12 packed documents: expiry and bitmap bit-exact at full size; O, lse, dK, dV, dM on sampled
+    rows and keys; no key tile of another document is ever active."""
+    case = wl.CONFIGS["3"]
+    cu = wl.packed_cu_seqlens(case.L, 12, seed=31)
+    inp, got = run(case, cu)
+    dl, e, bmp = oracle_varlen_mask(case, inp, cu)
+    assert np.array_equal(got["expiry"].cpu().numpy(), e)
+    assert np.array_equal(got["bitmap"].cpu().numpy().view(np.uint32), bmp)
+    seq_of = np.searchsorted(np.asarray(cu), np.arange(case.L), side="right") - 1
+    words = got["bitmap"].cpu().numpy().view(np.uint32)
+    Tr = words.shape[2]
+    for qt in range(Tr):
+        first_seq_start = cu[seq_of[qt * 128]]
+        for kt in range(first_seq_start // 128):                 # tiles wholly before the first document of the query tile
+            assert not (words[:, :, qt, kt // 32] >> np.uint32(kt % 32) & np.uint32(1)).any()
+    Q, K, V, dO = (f64(inp[k]) for k in ("Q", "K", "V", "dO"))
+    rng = np.random.default_rng(5)
+    L = case.L
+    rows = np.unique(np.concatenate([[0, L - 1], np.asarray(cu[1:-1]) - 1, np.asarray(cu[1:-1]), rng.integers(0, L, 12)])).astype(np.int32)
+    O, lse = oracle.forward(Q, K, V, dl.astype(np.float64), expiry=e, rows=rows)
+    assert_close(got["O"][:, rows], O, case.dtype, "O rows")
+    assert_close(got["lse"][:, :, rows], lse, case.dtype, "lse rows", lse=True)
+    # keys of the last document: only its rows can keep them
+    s0 = cu[-2]
+    keys = np.unique(np.concatenate([[s0, L - 1], rng.integers(s0, L, 5)])).astype(np.int32)
+    tail = np.arange(s0, L, dtype=np.int32)
+    Ot, _ = oracle.forward(Q, K, V, dl.astype(np.float64), expiry=e, rows=tail)
+    Ostored = np.zeros_like(Q)
+    Ostored[:, tail] = round_to(case, Ot)
+    _, dK, dV, dM = oracle.backward(Q, K, V, dO, dl.astype(np.float64), expiry=e, keys=keys, want_dq=False, O=Ostored)
+    assert_close(got["dK"][:, keys], dK, case.dtype, "dK keys")
+    assert_close(got["dV"][:, keys], dV, case.dtype, "dV keys")
+    assert_close(got["dM"][:, :, keys], dM, case.dtype, "dM keys")
+
+
+def test_argument_checks():
+    case = wl.small(C2, B=1, Hq=2, Hkv=1, L=128, d=128, w=32, name="varlen args")
+    p = problem_of(case)
+    inp = wl.make_inputs(case)
+    V, W, A = inp["V"].to(DEV), inp["W_delta"].to(DEV), inp["A"].to(DEV)
+    with pytest.raises(dma.DmaError) as err:
+        dma.dma_mask_build_varlen(p, V, W, A, torch.zeros(1, dtype=torch.int32, device=DEV))     # nseq = 0
+    assert err.value.status == -2
