@@ -121,6 +121,29 @@ def select_expiry_varlen(dl, w, cu_seqlens):
     return e
 
 
+def select_noncausal(dl, w):
+    """Selection without the causal fill (the App. A listing with an all-zero causal_m): every row sees every key, so
+    all rows of a head keep the same min(w, L) keys, the best under (delta descending, index ascending). Returned in the
+    interval form of the non-causal mode: expiry[j] = L for a kept key, 0 otherwise (key j is kept by rows i < expiry[j])."""
+    dl = _c(dl, np.float32)
+    L = dl.shape[-1]
+    flat = dl.reshape(-1, L)
+    e = np.zeros(flat.shape, np.int32)
+    pos = np.arange(L)
+    for r in range(flat.shape[0]):
+        order = np.lexsort((pos, -flat[r].astype(np.float64)))
+        e[r, order[:min(int(w), L)]] = L
+    return e.reshape(dl.shape)
+
+
+def keep_from_expiry_noncausal(e):
+    e = _c(e, np.int32)
+    L = e.shape[-1]
+    keep = np.empty(e.shape + (L,), np.uint8)
+    assert lib().dmao_keep_from_expiry_noncausal(_p(e), e.size // L, L, _p(keep)) == 0
+    return keep
+
+
 def keep_from_expiry(e):
     e = _c(e, np.int32)
     L = e.shape[-1]
@@ -149,7 +172,7 @@ def bitmap_from_expiry(e, bm=128, bn=128):
     return bmp
 
 
-def forward(Q, K, V, bias, expiry=None, keep=None, scale=None, rows=None, dtype=np.float64):
+def forward(Q, K, V, bias, expiry=None, keep=None, scale=None, rows=None, dtype=np.float64, causal=True):
     """Eq. (attention_output). Returns (O, LSE). With ``rows`` only those query rows are evaluated and the
     outputs are compact: O [B,len(rows),Hq,d], LSE [B,Hq,len(rows)]."""
     Q = _c(Q, dtype); K = _c(K, dtype); V = _c(V, dtype); bias = _c(bias, dtype)
@@ -162,12 +185,13 @@ def forward(Q, K, V, bias, expiry=None, keep=None, scale=None, rows=None, dtype=
     LSE = np.empty((B, Hq, R), dtype)
     f = lib().dmao_fwd_f64 if dtype == np.float64 else lib().dmao_fwd_f32
     rc = f(_p(Q), _p(K), _p(V), _p(bias), _p(expiry), _p(keep), B, L, Hq, Hkv, d, ctypes.c_double(scale),
-           _p(rows), 0 if rows is None else len(rows), _p(O), _p(LSE))
+           _p(rows), 0 if rows is None else len(rows), _p(O), _p(LSE), int(bool(causal)))
     assert rc == 0, rc
     return O, LSE
 
 
-def backward(Q, K, V, dO, bias, expiry=None, keep=None, scale=None, keys=None, want_dq=True, dtype=np.float64, O=None):
+def backward(Q, K, V, dO, bias, expiry=None, keep=None, scale=None, keys=None, want_dq=True, dtype=np.float64, O=None,
+             causal=True):
     """Sec. 4.3 gradients with the mask and bias values held fixed. Returns (dQ, dK, dV, dM). With ``keys`` only
     those keys are evaluated: dK,dV [B,len(keys),Hkv,d], dM [B,Hq,len(keys)] (dQ stays full, or None).
     ``O`` is the stored forward output that Alg. 2 reads for D = rowsum(dO o O); None = the exact output."""
@@ -183,7 +207,8 @@ def backward(Q, K, V, dO, bias, expiry=None, keep=None, scale=None, keys=None, w
     dM = np.empty((B, Hq, NK), dtype)
     f = lib().dmao_bwd_f64 if dtype == np.float64 else lib().dmao_bwd_f32
     rc = f(_p(Q), _p(K), _p(V), _p(O), _p(dO), _p(bias), _p(expiry), _p(keep), B, L, Hq, Hkv, d,
-           ctypes.c_double(scale), _p(keys), 0 if keys is None else len(keys), _p(dQ), _p(dK), _p(dV), _p(dM))
+           ctypes.c_double(scale), _p(keys), 0 if keys is None else len(keys), _p(dQ), _p(dK), _p(dV), _p(dM),
+           int(bool(causal)))
     assert rc == 0, rc
     return dQ, dK, dV, dM
 

@@ -115,12 +115,16 @@ struct Problem {
     const T *Q, *K, *V, *bias;
     const int32_t* expiry;   // [B,Hq,L] or null
     const uint8_t* keep;     // [B,Hq,L,L] or null (definition form; tiny cases)
+    int causal;              // 1: row i sees keys j <= i (the listing's causal fill); 0: every row sees every key
+                             // (the listing with an all-zero causal_m), key j kept by the rows i < expiry[j]
+    int jlast(int i) const { return causal ? i : L - 1; }    // last key row i can see
+    int ifirst(int j) const { return causal ? j : 0; }       // first row that can see key j
     int G() const { return Hq / Hkv; }
     const T* q(int b, int i, int h) const { return Q + (((size_t)b * L + i) * Hq + h) * d; }
     const T* k(int b, int j, int hk) const { return K + (((size_t)b * L + j) * Hkv + hk) * d; }
     const T* v(int b, int j, int hk) const { return V + (((size_t)b * L + j) * Hkv + hk) * d; }
     bool kept(int b, int h, int i, int j) const {
-        if (j > i) return false;
+        if (causal && j > i) return false;
         size_t bh = (size_t)b * Hq + h;
         if (keep) return keep[(bh * L + i) * L + j] != 0;
         return expiry[bh * L + j] > i;
@@ -137,7 +141,7 @@ void row_forward(const Problem<T>& P, int b, int h, int i, std::vector<int>& idx
     const T* bias = P.bias + ((size_t)b * P.Hq + h) * P.L;
     idx.clear();
     p.clear();
-    for (int j = 0; j <= i; ++j)
+    for (int j = 0; j <= P.jlast(i); ++j)
         if (P.kept(b, h, i, j)) idx.push_back(j);
     T m = -INFINITY;
     for (int j : idx) {
@@ -205,7 +209,7 @@ int backward(const Problem<T>& P, const T* Ostored, const T* dO, const int32_t* 
         for (int b = 0; b < P.B; ++b)
             for (int h = 0; h < Hq; ++h)
                 for (int t = 0; t < nkeys; ++t)
-                    for (int i = keys[t]; i < L; ++i)
+                    for (int i = P.ifirst(keys[t]); i < L; ++i)
                         if (P.kept(b, h, i, keys[t])) need[((size_t)b * Hq + h) * L + i] = 1;
         if (dQ) std::fill(need.begin(), need.end(), 1);
     }
@@ -260,7 +264,7 @@ int backward(const Problem<T>& P, const T* Ostored, const T* dO, const int32_t* 
         for (int h = hk * G; h < (hk + 1) * G; ++h) {
             size_t bh = (size_t)b * Hq + h;
             T dm = 0;
-            for (int i = j; i < L; ++i) {
+            for (int i = P.ifirst(j); i < L; ++i) {
                 if (!P.kept(b, h, i, j)) continue;
                 const T* qi = P.q(b, i, h);
                 const T* doi = dO + (((size_t)b * L + i) * Hq + h) * d;
@@ -284,8 +288,9 @@ int backward(const Problem<T>& P, const T* Ostored, const T* dO, const int32_t* 
 
 template <class T>
 Problem<T> make_problem(int B, int L, int Hq, int Hkv, int d, double scale, const T* Q, const T* K,
-                        const T* V, const T* bias, const int32_t* expiry, const uint8_t* keep) {
+                        const T* V, const T* bias, const int32_t* expiry, const uint8_t* keep, int causal) {
     Problem<T> P;
+    P.causal = causal;
     P.B = B; P.L = L; P.Hq = Hq; P.Hkv = Hkv; P.d = d;
     P.scale = (T)scale;
     P.Q = Q; P.K = K; P.V = V; P.bias = bias; P.expiry = expiry; P.keep = keep;
@@ -410,6 +415,14 @@ int dmao_bitmap_definition(const uint8_t* keep, int BH, int L, int bm, int bn, u
     return 0;
 }
 
+// Non-causal mode: key j is kept by the rows 0 <= i < expiry[j] (expiry is L for the w selected keys, 0 otherwise).
+int dmao_keep_from_expiry_noncausal(const int32_t* expiry, int BH, int L, uint8_t* keep) {
+    for (int bh = 0; bh < BH; ++bh)
+        for (int i = 0; i < L; ++i)
+            for (int j = 0; j < L; ++j) keep[((size_t)bh * L + i) * L + j] = expiry[(size_t)bh * L + j] > i ? 1 : 0;
+    return 0;
+}
+
 int dmao_bitmap_from_expiry(const int32_t* expiry, int BH, int L, int bm, int bn, uint32_t* bitmap) {
     const int Tr = (L + bm - 1) / bm, Tc = (L + bn - 1) / bn, Wd = (Tc + 31) / 32;
     std::memset(bitmap, 0, (size_t)BH * Tr * Wd * 4);
@@ -429,9 +442,9 @@ int dmao_bitmap_from_expiry(const int32_t* expiry, int BH, int L, int bm, int bn
 #define DMAO_FWD(NAME, T)                                                                            \
     int NAME(const T* Q, const T* K, const T* V, const T* bias, const int32_t* expiry,               \
              const uint8_t* keep, int B, int L, int Hq, int Hkv, int d, double scale,                \
-             const int32_t* rows, int nrows, T* O, T* LSE) {                                         \
+             const int32_t* rows, int nrows, T* O, T* LSE, int causal) {                             \
         if (Hq % Hkv || (!expiry && !keep)) return -1;                                               \
-        return forward<T>(make_problem<T>(B, L, Hq, Hkv, d, scale, Q, K, V, bias, expiry, keep),    \
+        return forward<T>(make_problem<T>(B, L, Hq, Hkv, d, scale, Q, K, V, bias, expiry, keep, causal), \
                           rows, nrows, O, LSE);                                                      \
     }
 DMAO_FWD(dmao_fwd_f32, float)
@@ -440,9 +453,9 @@ DMAO_FWD(dmao_fwd_f64, double)
 #define DMAO_BWD(NAME, T)                                                                            \
     int NAME(const T* Q, const T* K, const T* V, const T* Ostored, const T* dO, const T* bias,       \
              const int32_t* expiry, const uint8_t* keep, int B, int L, int Hq, int Hkv, int d, double scale, \
-             const int32_t* keys, int nkeys, T* dQ, T* dK, T* dV, T* dM) {                           \
+             const int32_t* keys, int nkeys, T* dQ, T* dK, T* dV, T* dM, int causal) {               \
         if (Hq % Hkv || (!expiry && !keep)) return -1;                                               \
-        return backward<T>(make_problem<T>(B, L, Hq, Hkv, d, scale, Q, K, V, bias, expiry, keep),   \
+        return backward<T>(make_problem<T>(B, L, Hq, Hkv, d, scale, Q, K, V, bias, expiry, keep, causal), \
                            Ostored, dO, keys, nkeys, dQ, dK, dV, dM);                                         \
     }
 DMAO_BWD(dmao_bwd_f32, float)
