@@ -336,6 +336,37 @@ def main():
                   "bwd_ms": v_ms[2] if case.backward else None, "step_ms": v_step, "active_tiles": act_v,
                   "tflops_executed_tiles": tile_flops(act_v, case.d, case.backward) / (v_step * 1e-3) / 1e12}
 
+    # ---- non-causal mode (causal = 0: every row of a head keeps the same min(w, L) keys; bf16 d = 128 runs token-compacted):
+    # dense attention of L rows over w gathered keys per head
+    noncausal = None
+    if case.dtype == "bf16" and case.d == 128 and not (args.flags & dma.DMA_FLAG_SIMT):
+        pn = dma.problem(case.B, case.Hq, case.Hkv, case.L, case.d, case.w, dtype=case.torch_dtype, causal=0, flags=args.flags)
+        mn, fn_, bn_ = dma.dma_query_workspace(pn)
+        ws_nm, ws_nf, ws_nb = (torch.empty(n, dtype=torch.uint8, device=dev) for n in (mn, fn_, bn_))
+        bias_n, exp_n, bmp_n = torch.empty_like(bias), torch.empty_like(expiry), torch.empty_like(bitmap)
+        On, lsen = torch.empty_like(O), torch.empty_like(lse)
+        stages = [lambda: dma.dma_mask_build(pn, V, W, A, bias_n, exp_n, bmp_n, ws_nm),
+                  lambda: dma.dma_attn_fwd(pn, Q, K, V, bias_n, exp_n, bmp_n, On, lsen, ws_nf)]
+        if case.backward:
+            stages.append(lambda: dma.dma_attn_bwd(pn, Q, K, V, On, dO, lsen, bias_n, exp_n, bmp_n, dQ, dK, dV, dM, ws_nb))
+        n_ms = []
+        for f in stages:
+            for _ in range(3):
+                f()
+            g0, g1 = ev(), ev()
+            barrier()
+            g0.record()
+            for _ in range(10):
+                f()
+            g1.record()
+            barrier()
+            n_ms.append(g0.elapsed_time(g1) / 10)
+        assert dma.dma_read_status(ws_nf) == 0 and (not case.backward or dma.dma_read_status(ws_nb) == 0), "device status (non-causal)"
+        keep = min(case.w, case.L)
+        pair_flops = (4 + (10 if case.backward else 0)) * case.B * case.Hq * case.L * keep * case.d   # per kept (row, key) pair
+        noncausal = {"mask_ms": n_ms[0], "fwd_ms": n_ms[1], "bwd_ms": n_ms[2] if case.backward else None, "step_ms": sum(n_ms),
+                     "kept_keys_per_head": keep, "tflops_kept_pairs": pair_flops / (sum(n_ms) * 1e-3) / 1e12}
+
     # ---- one decoding step over this workload's K / V as the cache (dma_delta_range + dma_decode), timed on its own
     decode = None
     if rank == 0:
@@ -427,6 +458,8 @@ def main():
         out["full_delta"] = full_delta
     if varlen is not None:
         out["varlen"] = varlen
+    if noncausal is not None:
+        out["noncausal"] = noncausal
     if mask_bwd is not None:
         mask_bwd["frac_of_measured_hbm"] = mask_bwd["gbs"] / pk["hbm_gbs"]
         out["mask_bwd"] = mask_bwd

@@ -68,7 +68,12 @@ enum {
 typedef struct {
     int32_t B, Hq, Hkv, L, d;    /* d in {64, 128}; Hq % Hkv == 0; L >= 1 (query and key length are equal)      */
     int32_t w;                   /* keep window of Eq. (mask_combine), >= 1; values above L act as L            */
-    int32_t causal;              /* must be 1: key j is visible to row i iff j <= i                             */
+    int32_t causal;              /* 1: key j is visible to row i iff j <= i. 0 (non-causal, the App. A listing with an
+                                    all-zero causal mask): every row sees every key, so all rows of a head keep the same
+                                    min(w, L) keys; expiry[j] is then L for a kept key and 0 otherwise, key j is kept by the
+                                    rows 0 <= i < expiry[j], and every bitmap row of a head is the same. bf16 with d = 128
+                                    always runs token-compacted in this mode (DMA_FLAG_COMPACT_KV is implied: contiguous K
+                                    and V, the larger workspaces); dma_mask_build_varlen needs causal = 1              */
     int32_t dtype;               /* DMA_BF16 | DMA_FP32                                                         */
     int32_t tile_m, tile_n;      /* bitmap granularity (query rows x keys per bit); 0,0 = 128,128               */
     int32_t flags;               /* DMA_FLAG_*                                                                  */

@@ -27,13 +27,13 @@ int resolve(const dma_problem_t* p, Prob* o) {
     if (!p) return DMA_ERR_NULL;
     if (p->B < 1 || p->Hq < 1 || p->Hkv < 1 || p->L < 1 || p->w < 1 || p->Hq % p->Hkv) return DMA_ERR_SHAPE;
     if (p->d != 64 && p->d != 128) return DMA_ERR_UNSUPPORTED;
-    if (p->causal != 1) return DMA_ERR_UNSUPPORTED;
+    if (p->causal != 0 && p->causal != 1) return DMA_ERR_UNSUPPORTED;
     if (p->dtype != DMA_BF16 && p->dtype != DMA_FP32) return DMA_ERR_UNSUPPORTED;
     if ((p->tile_m == 0) != (p->tile_n == 0) || p->tile_m < 0 || p->tile_n < 0) return DMA_ERR_SHAPE;
     if (!(p->softmax_scale >= 0.0f) || std::isinf(p->softmax_scale)) return DMA_ERR_SHAPE;
     o->B = p->B; o->Hq = p->Hq; o->Hkv = p->Hkv; o->L = p->L; o->d = p->d; o->G = p->Hq / p->Hkv;
     o->w = p->w < p->L ? p->w : p->L;
-    o->dtype = p->dtype; o->flags = p->flags;
+    o->dtype = p->dtype; o->flags = p->flags; o->causal = p->causal;
     o->bm = p->tile_m ? p->tile_m : 128;
     o->bn = p->tile_n ? p->tile_n : 128;
     o->Tr = (p->L + o->bm - 1) / o->bm;
@@ -43,6 +43,9 @@ int resolve(const dma_problem_t* p, Prob* o) {
     if (!fill_strides(p->q_stride, o->qs, p->L, p->Hq, p->d) || !fill_strides(p->k_stride, o->ks, p->L, p->Hkv, p->d) ||
         !fill_strides(p->v_stride, o->vs, p->L, p->Hkv, p->d) || !fill_strides(p->o_stride, o->os, p->L, p->Hq, p->d))
         return DMA_ERR_ALIGN;
+    // non-causal: all rows of a head keep the same keys, so the tensor-core path always runs token-compacted
+    if (!o->causal && o->dtype == DMA_BF16 && o->d == 128 && o->bm == 128 && o->bn == 128 && !(o->flags & DMA_FLAG_SIMT))
+        o->flags |= DMA_FLAG_COMPACT_KV;
     return DMA_OK;
 }
 
@@ -121,6 +124,7 @@ int dma_mask_build_varlen(const dma_problem_t* p, const void* V, const float* W_
     if (rc) return rc;
     if (!V || !W_delta || !A || !cu_seqlens || !bias || !expiry || !bitmap) return DMA_ERR_NULL;
     if (nseq < 1 || nseq > P.L) return DMA_ERR_SHAPE;
+    if (!P.causal) return DMA_ERR_UNSUPPORTED;
     if (!aligned16(V) || !aligned16(W_delta) || !aligned16(bias) || !aligned16(expiry) || !aligned16(bitmap))
         return DMA_ERR_ALIGN;
     if (!ws || ws_bytes < mask_ws_bytes(P) || !aligned16(ws)) return DMA_ERR_WORKSPACE;

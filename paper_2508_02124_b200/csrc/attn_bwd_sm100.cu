@@ -73,6 +73,7 @@ struct BwdParams {
     // groups keys of similar lifetime; a CTA owns 128 consecutive entries of one query head's permutation
     const int* perm;
     const int32_t* expiry_all;
+    int causal;                // 0: key j is visible to every row (token-compacted mode only): its first row is 0 instead of j
     const __nv_bfloat16* Kg;    // K, V as contiguous [B, L, Hkv, 128] row arrays
     const __nv_bfloat16* Vg;
     float* dKacc;               // fp32 [B, L, Hkv, 128] accumulators (several query heads add into one KV head's rows)
@@ -129,7 +130,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
     if constexpr (kCompact) {
         // keys that no row keeps are sorted to the end of the permutation: a tile that starts with one holds nothing else
         const int jf = my_perm[0];
-        if (jf >= P.L || P.expiry_all[(size_t)blockIdx.x * P.L + jf] <= jf) return;
+        if (jf >= P.L || P.expiry_all[(size_t)blockIdx.x * P.L + jf] <= (P.causal ? jf : 0)) return;
     }
 
     if (tid == 0) {
@@ -162,7 +163,8 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             for (int t = 0; t < 4; ++t) {
                 const int j = my_perm[lane + 32 * t];
                 const int e = j < P.L ? P.expiry_all[(size_t)blockIdx.x * P.L + j] : 0;
-                if (e > j) { jmin = min(jmin, j); emax = max(emax, e); }
+                const int first = P.causal ? j : 0;
+                if (e > first) { jmin = min(jmin, first); emax = max(emax, e); }
             }
             for (int o = 16; o; o >>= 1) {
                 jmin = min(jmin, __shfl_xor_sync(0xffffffffu, jmin, o));
@@ -220,6 +222,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
         const int quad = warp & 3, hsel = warp >> 2;
         const int r = quad * 32 + lane;                     // key within the tile = TMEM lane
         const int j = kCompact ? my_perm[r] : j0 + r;           // token-compacted mode: padding entries hold L
+        const int jf = (kCompact && !P.causal) ? 0 : j;         // first row that can see the key
         const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
         float bj = 0.0f;
         float2 dm2 = make_float2(0.0f, 0.0f);
@@ -235,7 +238,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                 if (cur_g >= 0 && j < P.L) atomicAdd(&P.dM[(size_t)(bh - (g - cur_g)) * P.L + j], dm2.x + dm2.y);
                 dm2 = make_float2(0.0f, 0.0f);
                 bj = j < P.L ? P.bias[(size_t)bh * P.L + j] * 1.4426950408889634f : 0.0f;
-                len = j < P.L ? P.expiry[(size_t)bh * P.L + j] - j : 0;
+                len = j < P.L ? max(0, P.expiry[(size_t)bh * P.L + j] - jf) : 0;
                 cur_g = g;
             }
             PROF_WAIT(0, ok = mbar_wait_warp(&S.sdp_full, n & 1, abort_flag) && mbar_wait_warp(&S.qd_full[st], (n / kStages) & 1, abort_flag));
@@ -257,8 +260,8 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
 #endif
             // valid columns of this thread within its 32: col in [lo, lo + width)
             const int c0 = hsel * 32;
-            const int lo = max(0, j - i0 - c0);
-            const int width = max(0, min(32, j - i0 - c0 + len) - lo);
+            const int lo = max(0, jf - i0 - c0);
+            const int width = max(0, min(32, jf - i0 - c0 + len) - lo);
             // Almost every (key, 32-row group) pair is all-or-nothing: then the mask is one additive term per thread
             // (0 or -inf) and the per-element test is skipped. Warps with a partly kept key take the general loop.
             const bool uniform = __all_sync(0xffffffffu, width == 0 || (lo == 0 && width == 32));
@@ -623,14 +626,14 @@ __global__ void dq_convert_bf16_kernel(const float* __restrict__ acc, __nv_bfloa
 // on i.i.d. importance at L = 16384, w = 2048 the walk covers 1.4 x the (row, key) pairs actually kept, against 4.3 x
 // for tiles of consecutive keys. Padded with L up to Tc * 128.
 // One CTA of 1024 threads per (batch, head); the warps take turns per 1024-key chunk so that the order is kept.
-__global__ void __launch_bounds__(1024) lifetime_perm_kernel(const int32_t* __restrict__ expiry, int* __restrict__ perm, int L, int Tc) {
+__global__ void __launch_bounds__(1024) lifetime_perm_kernel(const int32_t* __restrict__ expiry, int* __restrict__ perm, int L, int Tc, int causal) {
     __shared__ int hist[64];
     __shared__ int offs[64];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int32_t* e = expiry + (size_t)blockIdx.x * L;
     int* out = perm + (size_t)blockIdx.x * Tc * 128;
     const int band = max(2048, (L + 61) / 62);
-    auto cls = [&](int j) { return e[j] > j ? 1 + (e[j] - 1) / band : 0; };
+    auto cls = [&](int j) { return e[j] > (causal ? j : 0) ? 1 + (e[j] - 1) / band : 0; };
     if (tid < 64) hist[tid] = 0;
     __syncthreads();
     for (int j = tid; j < L; j += 1024) atomicAdd(&hist[cls(j)], 1);
@@ -673,6 +676,7 @@ int launch_tc_bwd(const Prob& P, const void* Q, const void* K, const void* V, co
                   const float* lse, const float* bias, const int32_t* expiry, const uint32_t* bitmap, void* dQ,
                   void* dK, void* dV, float* dM, void* ws, cudaStream_t st) {
     const bool compact = (P.flags & DMA_FLAG_COMPACT_KV) != 0;
+    if (!P.causal && !compact) return DMA_ERR_UNSUPPORTED;
     if ((size_t)P.G * P.Tr * 2 > (size_t)kMaxSteps || P.G > 16 || P.Tr > 1024) return DMA_ERR_UNSUPPORTED;
     const size_t rows = (size_t)P.B * P.Hq * P.L, nq = rows * P.d, nkv = (size_t)P.B * P.L * P.Hkv * P.d;
     float* Dv = reinterpret_cast<float*>((char*)ws + kWsHeaderBytes);
@@ -700,7 +704,7 @@ int launch_tc_bwd(const Prob& P, const void* Q, const void* K, const void* V, co
     if (cudaMemsetAsync(dM, 0, rows * sizeof(float), st) != cudaSuccess) return DMA_ERR_CUDA;   // two partial sums are added per key
     if (compact) {
         if (cudaMemsetAsync(accK, 0, 2 * nkv * sizeof(float), st) != cudaSuccess) return DMA_ERR_CUDA;
-        lifetime_perm_kernel<<<P.B * P.Hq, 1024, 0, st>>>(expiry, perm, P.L, P.Tc);
+        lifetime_perm_kernel<<<P.B * P.Hq, 1024, 0, st>>>(expiry, perm, P.L, P.Tc, P.causal);
         count_launch();
     }
     BwdParams bp;
@@ -710,7 +714,7 @@ int launch_tc_bwd(const Prob& P, const void* Q, const void* K, const void* V, co
     bp.ignore_bitmap = (P.flags & DMA_FLAG_IGNORE_BITMAP) ? 1 : 0;
     bp.scale = P.scale; bp.scale_log2 = P.scale * 1.4426950408889634f; bp.inv_scale = 1.0f / P.scale;
     bp.ks_b = P.ks[0]; bp.ks_l = P.ks[1]; bp.ks_h = P.ks[2]; bp.vs_b = P.vs[0]; bp.vs_l = P.vs[1]; bp.vs_h = P.vs[2];
-    bp.perm = perm; bp.expiry_all = expiry; bp.Kg = (const __nv_bfloat16*)K; bp.Vg = (const __nv_bfloat16*)V;
+    bp.perm = perm; bp.expiry_all = expiry; bp.causal = P.causal; bp.Kg = (const __nv_bfloat16*)K; bp.Vg = (const __nv_bfloat16*)V;
     bp.dKacc = accK; bp.dVacc = accV;
 #ifdef DMA_PROF
     const char* prof_env = getenv("DMA_PROF_PTR");

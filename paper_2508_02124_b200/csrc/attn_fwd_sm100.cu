@@ -76,6 +76,7 @@ struct FwdParams {
     const __nv_bfloat16* Kg;                   // K and V as contiguous [B, L, Hkv, 128] row arrays
     const __nv_bfloat16* Vg;
     int ccap, Hkv;
+    int causal;                                // 0: key j is visible to every row (token-compacted mode only)
     int64_t os_b, os_l, os_h;
 #ifdef DMA_PROF
     long long* prof;                           // role timing (development builds only): cycles per phase of CTA (0, 0)
@@ -495,8 +496,9 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
 #pragma unroll
                     for (int w = 0; w < 2; ++w) {
                         const int i0 = (w ? qt1 : qt0) * 128;
-                        const bool dead = jv[t] < 0 || ev[t] <= i0 || jv[t] > i0 + 127;
-                        const bool mixed = !dead && (ev[t] < i0 + 128 || jv[t] > i0);
+                        const int first = P.causal ? jv[t] : 0;             // first row that can see the key
+                        const bool dead = jv[t] < 0 || ev[t] <= i0 || first > i0 + 127;
+                        const bool mixed = !dead && (ev[t] < i0 + 128 || first > i0);
                         b0[w][t] = dead ? kNegBig : w0;
                         flags[w] |= __ballot_sync(0xffffffffu, mixed) ? (1u << t) : 0u;
                     }
@@ -509,7 +511,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
 #pragma unroll
                 for (int t = 0; t < 4; ++t) {
                     const int c = lane + 32 * t;
-                    S.jidx[st][c] = jv[t] >= 0 ? jv[t] : 0x7fffffff;                   // padding: never <= a row index
+                    S.jidx[st][c] = jv[t] >= 0 ? (P.causal ? jv[t] : 0) : 0x7fffffff;  // first row of the key; padding: never <= a row index
                     S.len[st][c] = ev[t];
 #pragma unroll
                     for (int w = 0; w < 2; ++w)
@@ -860,17 +862,17 @@ int make_tmap_f32_rows(CUtensorMap* m, const void* base, int B, int L, int H, in
 // At most w + 256 keys qualify. One CTA of 256 threads per list: 256 keys per pass, ballots and per-warp counts keep the
 // order; the list is padded with -1 to the next multiple of 128.
 __global__ void __launch_bounds__(256) compact_lists_kernel(const int32_t* __restrict__ expiry, int* __restrict__ cidx,
-                                                            int* __restrict__ ccnt, int L, int npairs, int cap) {
+                                                            int* __restrict__ ccnt, int L, int npairs, int cap, int causal) {
     __shared__ int wsum[2][8];
     const int list = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int bh = list / npairs, pair = list % npairs, i0 = pair * 256;
     const int32_t* e = expiry + (size_t)bh * L;
     int* out = cidx + (size_t)list * cap;
-    const int jend = min(L, i0 + 256);
+    const int jend = causal ? min(L, i0 + 256) : L;     // non-causal: key j is kept by the rows i < expiry[j], whatever j
     int n = 0, buf = 0;
     for (int base = 0; base < jend; base += 256, buf ^= 1) {
         const int j = base + tid;
-        const bool keep = j < jend && e[j] > max(i0, j);
+        const bool keep = j < jend && e[j] > (causal ? max(i0, j) : i0);
         const uint32_t bal = __ballot_sync(0xffffffffu, keep);
         if (lane == 0) wsum[buf][warp] = __popc(bal);
         __syncthreads();                                   // (the other buffer is free to be rewritten next pass)
@@ -907,7 +909,8 @@ int launch_tc_fwd(const Prob& P, const void* Q, const void* K, const void* V, co
     int rc;
     if ((rc = make_tmap_bf16(&tmQ, Q, P.B, P.L, P.Hq, P.d, P.qs, 128))) return rc;
     FwdParams fp;
-    fp.cidx = nullptr; fp.ccnt = nullptr; fp.ccap = 0; fp.Hkv = P.Hkv;
+    fp.cidx = nullptr; fp.ccnt = nullptr; fp.ccap = 0; fp.Hkv = P.Hkv; fp.causal = P.causal;
+    if (!P.causal && !compact) return DMA_ERR_UNSUPPORTED;
     if (compact) {
         // the gathers address K and V as plain row arrays: contiguous [B, L, Hkv, 128] only
         const int64_t want[3] = {(int64_t)P.L * P.Hkv * P.d, (int64_t)P.Hkv * P.d, P.d};
@@ -917,7 +920,7 @@ int launch_tc_fwd(const Prob& P, const void* Q, const void* K, const void* V, co
         const size_t nl = compact_lists(P);
         int* ccnt = reinterpret_cast<int*>((char*)ws + kWsHeaderBytes);
         int* cidx = reinterpret_cast<int*>((char*)ws + kWsHeaderBytes + ((nl * sizeof(int) + 255) / 256) * 256);
-        compact_lists_kernel<<<(unsigned)nl, 256, 0, st>>>(expiry, cidx, ccnt, P.L, (P.Tr + 1) / 2, compact_cap(P));
+        compact_lists_kernel<<<(unsigned)nl, 256, 0, st>>>(expiry, cidx, ccnt, P.L, (P.Tr + 1) / 2, compact_cap(P), P.causal);
         count_launch();
         fp.cidx = cidx; fp.ccnt = ccnt; fp.ccap = compact_cap(P);
     }

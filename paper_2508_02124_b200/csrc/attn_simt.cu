@@ -53,7 +53,7 @@ __global__ void __launch_bounds__(NT) simt_fwd_kernel(const T* __restrict__ Q, c
 #pragma unroll
         for (int c = 0; c < D / 16; ++c) acc[a][c] = 0.0f;
 
-    const int last = min(i0 + BM, L) - 1;            // last query row of the tile
+    const int last = P.causal ? min(i0 + BM, L) - 1 : L - 1;   // last key any row of the tile can see
     for (int j0 = 0; j0 <= last; j0 += BN) {
         if (use_bitmap && !bitmap_test(bitmap, P.Tr, P.Wd, bh, i0 / P.bm, j0 / P.bn)) continue;
         __syncthreads();
@@ -86,7 +86,7 @@ __global__ void __launch_bounds__(NT) simt_fwd_kernel(const T* __restrict__ Q, c
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
                 int r = ty + 16 * a, cc = tx + 16 * c, i = i0 + r, j = j0 + cc;
-                bool ok = j <= i && i < sE[cc];
+                bool ok = (j <= i || !P.causal) && i < sE[cc];
                 sS[r * LDS + cc] = ok ? s[a][c] * P.scale + sB[cc] : -INFINITY;
             }
         __syncthreads();
@@ -204,7 +204,7 @@ __global__ void __launch_bounds__(NT) simt_bwd_kernel(const T* __restrict__ Q, c
             sE[tid] = j < L ? expiry[(size_t)bh * L + j] : 0;
             sdM[tid] = 0.0f;
         }
-        for (int i0 = (j0 / BM) * BM; i0 < L; i0 += BM) {
+        for (int i0 = P.causal ? (j0 / BM) * BM : 0; i0 < L; i0 += BM) {
             if (use_bitmap && !bitmap_test(bitmap, P.Tr, P.Wd, bh, i0 / P.bm, j0 / P.bn)) continue;
             __syncthreads();
             load_tile(sQ, LDQ, Q + b * P.qs[0] + h * P.qs[2], P.qs[1], i0, L, D);
@@ -240,7 +240,7 @@ __global__ void __launch_bounds__(NT) simt_bwd_kernel(const T* __restrict__ Q, c
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
                     int r = ty + 16 * a, cc = tx + 16 * c, i = i0 + r, j = j0 + cc;
-                    bool ok = j <= i && i < sE[cc] && i < L;
+                    bool ok = (j <= i || !P.causal) && i < sE[cc] && i < L;
                     float p = ok ? __expf(s[a][c] * P.scale + sB[cc] - sLse[r]) : 0.0f;
                     float ds = p * (dp[a][c] - sDv[r]);
                     sP[r * LDS + cc] = p;

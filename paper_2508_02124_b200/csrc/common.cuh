@@ -16,6 +16,7 @@ struct Prob {
     int B, Hq, Hkv, L, d, G;
     int w;                 // min(w, L)
     int dtype, flags;
+    int causal;            // 1: key j visible to rows i >= j; 0: to every row (the key's first row is 0 instead of j)
     int bm, bn, Tr, Tc, Wd;   // bitmap tile sizes, tile counts, uint32 words per bitmap row
     float scale;
     int64_t qs[3], ks[3], vs[3], os[3];   // batch, seq, head strides in elements

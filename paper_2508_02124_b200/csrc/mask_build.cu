@@ -238,12 +238,15 @@ __global__ void __launch_bounds__(kChunk) chunk_sort_kernel(const float* __restr
 // kVarlen: sequences packed along the key axis (sequence s owns the keys cu[s] <= j < cu[s+1]). A key competes only
 // with the keys of its own sequence [s0, s1): chunks before s0 count nothing, a chunk that straddles s0 or s1 is
 // counted entry by entry with the index test, the walk ends at s1, and L is replaced by s1.
-template <bool kVarlen>
+// kMode 2 (non-causal): every row sees every key, so a key is kept by all rows (expiry L) iff fewer than w keys of the
+// whole head beat it, and by none (expiry 0) otherwise: phase 1 alone, over all chunks.
+template <int kMode>
 __global__ void __launch_bounds__(kExpThreads) expiry_kernel(const float* __restrict__ delta,
                                                              const unsigned long long* __restrict__ sorted,
                                                              int32_t* __restrict__ expiry, int L, int w, int nchunk,
                                                              const int32_t* __restrict__ cu, int nseq) {
     constexpr int kPer = kChunk / kExpThreads;
+    constexpr bool kVarlen = kMode == 1, kAllRows = kMode == 2;
     __shared__ uint32_t shi[2][kChunk], slo[2][kChunk];
     __shared__ int c_first;
     const int bh = blockIdx.y, t = threadIdx.x, lane = t & 31, j = blockIdx.x * kExpThreads + t;
@@ -315,7 +318,7 @@ __global__ void __launch_bounds__(kExpThreads) expiry_kernel(const float* __rest
     }
     // phase 2, warp-cooperative: lane `src` broadcasts (chunk, key, need); the warp scans that chunk 32 keys at a time
     int e = s1;
-    const uint32_t pending = __ballot_sync(0xffffffffu, fin >= 0);
+    const uint32_t pending = kAllRows ? 0u : __ballot_sync(0xffffffffu, fin >= 0);
     for (uint32_t rest = pending; rest; rest &= rest - 1) {
         const int src = __ffs(rest) - 1;
         const int base = __shfl_sync(0xffffffffu, fin, src) * kChunk;
@@ -338,6 +341,7 @@ __global__ void __launch_bounds__(kExpThreads) expiry_kernel(const float* __rest
         }
         if (lane == src) e = max(j, found);
     }
+    if (kAllRows) e = fin >= 0 ? 0 : L;
     if (valid) expiry[(size_t)bh * L + j] = e;
 }
 
@@ -348,8 +352,9 @@ __global__ void fill_i32_kernel(int32_t* p, size_t n, int32_t v) {
 
 // One CTA per (key tile, head): key j is kept by rows [j, expiry[j]), i.e. by query tiles j/bm .. (expiry[j]-1)/bm.
 // A difference array over query tiles forms the union; bits are OR-ed into the (pre-zeroed) bitmap.
+// (non-causal mode: key j is kept by rows [0, expiry[j]), so its interval of query tiles starts at tile 0)
 __global__ void __launch_bounds__(128) bitmap_kernel(const int32_t* __restrict__ expiry, uint32_t* __restrict__ bitmap,
-                                                     int L, int bm, int bn, int Tr, int Wd) {
+                                                     int L, int bm, int bn, int Tr, int Wd, int causal) {
     extern __shared__ int diff[];                 // [Tr + 1]
     const int kt = blockIdx.x, bh = blockIdx.y, t = threadIdx.x;
     for (int i = t; i <= Tr; i += blockDim.x) diff[i] = 0;
@@ -357,8 +362,8 @@ __global__ void __launch_bounds__(128) bitmap_kernel(const int32_t* __restrict__
     const int jend = min(L, (kt + 1) * bn);
     for (int j = kt * bn + t; j < jend; j += blockDim.x) {
         const int e = expiry[(size_t)bh * L + j];
-        if (e > j) {
-            atomicAdd(&diff[j / bm], 1);
+        if (e > (causal ? j : 0)) {
+            atomicAdd(&diff[causal ? j / bm : 0], 1);
             atomicAdd(&diff[(e - 1) / bm + 1], -1);
         }
     }
@@ -436,8 +441,9 @@ int launch_mask_build(const Prob& P, const void* V, const float* W, const float*
         auto* sorted = reinterpret_cast<unsigned long long*>((char*)ws + kWsHeaderBytes);
         chunk_sort_kernel<<<dim3(nchunk, BH), kChunk, 0, st>>>(bias, sorted, P.L, nchunk);
         const dim3 grid((P.L + kExpThreads - 1) / kExpThreads, BH);
-        if (cu) expiry_kernel<true><<<grid, kExpThreads, 0, st>>>(bias, sorted, expiry, P.L, P.w, nchunk, cu, nseq);
-        else expiry_kernel<false><<<grid, kExpThreads, 0, st>>>(bias, sorted, expiry, P.L, P.w, nchunk, nullptr, 0);
+        if (cu) expiry_kernel<1><<<grid, kExpThreads, 0, st>>>(bias, sorted, expiry, P.L, P.w, nchunk, cu, nseq);
+        else if (!P.causal) expiry_kernel<2><<<grid, kExpThreads, 0, st>>>(bias, sorted, expiry, P.L, P.w, nchunk, nullptr, 0);
+        else expiry_kernel<0><<<grid, kExpThreads, 0, st>>>(bias, sorted, expiry, P.L, P.w, nchunk, nullptr, 0);
         count_launch(2);
     }
     if ((rc = check_launch())) return rc;
@@ -445,7 +451,7 @@ int launch_mask_build(const Prob& P, const void* V, const float* W, const float*
     if (cudaMemsetAsync(bitmap, 0, (size_t)BH * P.Tr * P.Wd * sizeof(uint32_t), st) != cudaSuccess) return DMA_ERR_CUDA;
     size_t smem = (size_t)(P.Tr + 1) * sizeof(int);
     if (smem > 48 * 1024) return DMA_ERR_UNSUPPORTED;
-    bitmap_kernel<<<dim3(P.Tc, BH), 128, smem, st>>>(expiry, bitmap, P.L, P.bm, P.bn, P.Tr, P.Wd);
+    bitmap_kernel<<<dim3(P.Tc, BH), 128, smem, st>>>(expiry, bitmap, P.L, P.bm, P.bn, P.Tr, P.Wd, P.causal);
     count_launch();
     return check_launch();
 }
