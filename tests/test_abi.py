@@ -41,7 +41,7 @@ def test_argument_validation(lib):
     assert dma.dma_bitmap_words(ok) == 4 * 2 * 1
     for bad, code in ((dma.problem(1, 3, 2, 256, 64, 32), -2), (dma.problem(1, 4, 2, 0, 64, 32), -2),
                       (dma.problem(1, 4, 2, 256, 64, 0), -2), (dma.problem(1, 4, 2, 256, 96, 32), -4),
-                      (dma.problem(1, 4, 2, 256, 64, 32, causal=0), -4), (dma.problem(1, 4, 2, 256, 64, 32, tile_m=64), -2)):
+                      (dma.problem(1, 4, 2, 256, 64, 32, causal=2), -4), (dma.problem(1, 4, 2, 256, 64, 32, tile_m=64), -2)):
         with pytest.raises(dma.DmaError) as e:
             dma.dma_query_workspace(bad)
         assert e.value.status == code
