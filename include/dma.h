@@ -189,8 +189,10 @@ int dma_decode(const dma_problem_t* p, const void* q, const void* K, const void*
 /* The whole hot path on HOST buffers (all contiguous, default strides only): copies Q,K,V,(dO),W_delta,A into the
  * caller's device arena, runs dma_mask_build, dma_attn_fwd and, if `backward` != 0, dma_attn_bwd on the stream,
  * copies O, lse (and dQ,dK,dV,dM) back and synchronises the stream before returning. The copies run on two helper
- * streams that exist only for the duration of the call, so that they overlap the kernels (V first, then K and Q, dO during
- * the forward, O and lse during the backward). h* pointers are HOST memory
+ * streams that exist only for the duration of the call, so that they overlap the kernels; the step is cut into
+ * independent (batch entry, group of KV heads) problems (up to four head groups, addressed inside the full tensors by
+ * strides) so that the next group's inputs arrive and the previous group's results leave while a group computes; the
+ * results are those of the device entry points on the same inputs. h* pointers are HOST memory
  * (pinned memory makes the copies asynchronous and faster); dev_arena is DEVICE memory, 256-byte aligned, of at
  * least dma_step_host_arena() bytes; hdO, hdQ, hdK, hdV, hdM may be NULL when `backward` is 0. */
 int dma_step_host_arena(const dma_problem_t* p, int backward, size_t* bytes);

@@ -2,10 +2,17 @@
 // keep their tensors in host memory and for end-to-end timing. Inputs are copied to a caller-provided device
 // arena (on helper streams, overlapped with the kernels), the three stages run on the caller's stream, results are
 // copied back, and the stream is synchronised.
+//
+// Every (batch entry, group of KV heads) is an independent problem (the mask is per head, dK and dV are summed only
+// inside a KV head's group of query heads), so the step is cut into such groups and pipelined: while group g runs its
+// kernels, group g + 1's inputs arrive and group g - 1's results leave. A group is addressed inside the full tensors
+// by pointer offsets and the full tensors' strides (the kernels take strides), its copies are strided 2-D copies.
 #include "common.cuh"
 
 namespace dma {
 namespace {
+
+constexpr int kMaxGroups = 64;
 
 struct Arena {
     size_t off = 0;
@@ -19,7 +26,25 @@ struct Arena {
 struct Layout {
     size_t Q, K, V, dO, O, dQ, dK, dV, W, A, bias, expiry, bitmap, lse, dM, ws_mask, ws_fwd, ws_bwd, total;
     size_t nq, nk, nbh, nbmp, m_ws, f_ws, b_ws, esz, wbytes;
+    int head_groups;       // groups of KV heads per batch entry (1 = whole batch entries)
+    int groups;            // B * head_groups
 };
+
+// Head groups per batch entry: up to 4, a divisor of Hkv, and only where every per-group pointer stays 16-byte aligned,
+// the group is independent (the full sampling weights read all KV heads; the token-compacted kernels want contiguous
+// K and V) and a group's K / V rows are at least 512 bytes wide (measured at L = 16384, 32 / 8 heads: 4 groups of
+// 512-byte rows 10.2 ms per step, 8 groups of 256-byte rows 14.6 ms, one group 14.8 ms: short rows slow the copies down).
+int pick_head_groups(const Prob& P) {
+    if (P.flags & (DMA_FLAG_FULL_DELTA | DMA_FLAG_COMPACT_KV)) return 1;
+    const size_t esz = P.dtype == DMA_BF16 ? 2 : 4;
+    for (int g = 4; g > 1; --g) {
+        if (P.Hkv % g || (size_t)(P.Hkv / g) * P.d * esz < 512) continue;
+        const size_t hq = (size_t)P.Hq / g;
+        if ((hq * P.L) % 4 || (hq * P.Tr * P.Wd) % 4 || hq % 4) continue;
+        return g;
+    }
+    return 1;
+}
 
 int make_layout(const dma_problem_t* p, int backward, Layout* Lo) {
     Prob P;
@@ -28,6 +53,13 @@ int make_layout(const dma_problem_t* p, int backward, Layout* Lo) {
     for (int i = 0; i < 3; ++i)
         if (p->q_stride[i] || p->k_stride[i] || p->v_stride[i] || p->o_stride[i]) return DMA_ERR_UNSUPPORTED;
     if ((rc = dma_query_workspace(p, &Lo->m_ws, &Lo->f_ws, &Lo->b_ws))) return rc;
+    Lo->head_groups = pick_head_groups(P);
+    if ((size_t)P.B * Lo->head_groups > (size_t)kMaxGroups) Lo->head_groups = 1;
+    Lo->groups = P.B <= kMaxGroups ? P.B * Lo->head_groups : 1;
+    if (Lo->groups == 1) Lo->head_groups = 1;
+    // one status header per group in front of each workspace (a group's header is never inside a later group's data)
+    Lo->f_ws += (size_t)Lo->groups * kWsHeaderBytes;
+    Lo->b_ws += (size_t)Lo->groups * kWsHeaderBytes;
     Lo->esz = P.dtype == DMA_BF16 ? 2 : 4;
     Lo->nq = (size_t)P.B * P.L * P.Hq * P.d;
     Lo->nk = (size_t)P.B * P.L * P.Hkv * P.d;
@@ -77,52 +109,122 @@ int dma_step_host(const dma_problem_t* p, int backward, const void* hQ, const vo
     if (!dev_arena || arena_bytes < Lo.total || (reinterpret_cast<uintptr_t>(dev_arena) & 255)) return DMA_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)cuda_stream;
     char* a = (char*)dev_arena;
+    const int NG = Lo.groups, HG = Lo.head_groups;
+    const int L = p->L, d = p->d, nqh = p->Hq / HG, nkh = p->Hkv / HG;
+    const size_t esz = Lo.esz;
+
     // Copies run on two helper streams of this call (created and destroyed here: no state is kept) so that they overlap
-    // the kernels on the caller's stream: V first (the mask build needs nothing else), then K and Q, then dO while the
-    // forward runs; O and lse go back while the backward runs. Events order the helpers after the work already on the
-    // caller's stream and the caller's stream after the last copy.
+    // the kernels on the caller's stream. Per group: V first (the mask build needs nothing else), then K and Q, then dO;
+    // O and lse go back while the group's backward runs, the gradients while the next group computes. Events order the
+    // helpers after the work already on the caller's stream and the caller's stream after the last copy.
+    enum { kV, kKQ, kdO, kO, kG, kPerGroup };
     cudaStream_t s_in = nullptr, s_out = nullptr;
-    cudaEvent_t ev[7] = {};
+    cudaEvent_t ev_start = nullptr, ev_done = nullptr;
+    cudaEvent_t ev[kMaxGroups * kPerGroup] = {};
     auto cleanup = [&](int code) {
-        for (auto& e : ev) if (e) cudaEventDestroy(e);
+        for (int i = 0; i < NG * kPerGroup; ++i) if (ev[i]) cudaEventDestroy(ev[i]);
+        if (ev_start) cudaEventDestroy(ev_start);
+        if (ev_done) cudaEventDestroy(ev_done);
         if (s_in) cudaStreamDestroy(s_in);
         if (s_out) cudaStreamDestroy(s_out);
         return code;
     };
     if (cudaStreamCreateWithFlags(&s_in, cudaStreamNonBlocking) != cudaSuccess) return cleanup(DMA_ERR_CUDA);
     if (cudaStreamCreateWithFlags(&s_out, cudaStreamNonBlocking) != cudaSuccess) return cleanup(DMA_ERR_CUDA);
-    for (auto& e : ev) if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) return cleanup(DMA_ERR_CUDA);
-    enum { kStart, kV, kKQ, kdO, kO, kG, kDone };
-    auto h2d = [&](size_t off, const void* src, size_t n) { return cudaMemcpyAsync(a + off, src, n, cudaMemcpyHostToDevice, s_in) == cudaSuccess; };
-    auto d2h = [&](void* dst, size_t off, size_t n) { return cudaMemcpyAsync(dst, a + off, n, cudaMemcpyDeviceToHost, s_out) == cudaSuccess; };
-    auto rec = [&](int e, cudaStream_t on) { return cudaEventRecord(ev[e], on) == cudaSuccess; };
-    auto wait = [&](cudaStream_t on, int e) { return cudaStreamWaitEvent(on, ev[e], 0) == cudaSuccess; };
-    bool ok = rec(kStart, st) && wait(s_in, kStart) && wait(s_out, kStart);
-    ok = ok && h2d(Lo.V, hV, Lo.nk * Lo.esz) && h2d(Lo.W, hW_delta, Lo.wbytes) && h2d(Lo.A, hA, (size_t)p->Hq * 4) && rec(kV, s_in);
-    ok = ok && h2d(Lo.K, hK, Lo.nk * Lo.esz) && h2d(Lo.Q, hQ, Lo.nq * Lo.esz) && rec(kKQ, s_in);
-    if (backward) ok = ok && h2d(Lo.dO, hdO, Lo.nq * Lo.esz) && rec(kdO, s_in);
-    if (!ok) return cleanup(DMA_ERR_CUDA);
-    float* bias = (float*)(a + Lo.bias);
-    int32_t* expiry = (int32_t*)(a + Lo.expiry);
-    uint32_t* bitmap = (uint32_t*)(a + Lo.bitmap);
-    if (!wait(st, kV)) return cleanup(DMA_ERR_CUDA);
-    if ((rc = dma_mask_build(p, a + Lo.V, (float*)(a + Lo.W), (float*)(a + Lo.A), bias, expiry, bitmap, a + Lo.ws_mask, Lo.m_ws, st))) return cleanup(rc);
-    if (!wait(st, kKQ)) return cleanup(DMA_ERR_CUDA);
-    if ((rc = dma_attn_fwd(p, a + Lo.Q, a + Lo.K, a + Lo.V, bias, expiry, bitmap, a + Lo.O, (float*)(a + Lo.lse), a + Lo.ws_fwd, Lo.f_ws, st))) return cleanup(rc);
-    ok = rec(kO, st) && wait(s_out, kO) && d2h(hO, Lo.O, Lo.nq * Lo.esz) && d2h(hlse, Lo.lse, Lo.nbh * 4);
-    if (backward) {
-        if (!ok || !wait(st, kdO)) return cleanup(DMA_ERR_CUDA);
-        if ((rc = dma_attn_bwd(p, a + Lo.Q, a + Lo.K, a + Lo.V, a + Lo.O, a + Lo.dO, (float*)(a + Lo.lse), bias, expiry, bitmap,
-                               a + Lo.dQ, a + Lo.dK, a + Lo.dV, (float*)(a + Lo.dM), a + Lo.ws_bwd, Lo.b_ws, st))) return cleanup(rc);
-        ok = rec(kG, st) && wait(s_out, kG) && d2h(hdQ, Lo.dQ, Lo.nq * Lo.esz) && d2h(hdK, Lo.dK, Lo.nk * Lo.esz) &&
-             d2h(hdV, Lo.dV, Lo.nk * Lo.esz) && d2h(hdM, Lo.dM, Lo.nbh * 4);
+    if (cudaEventCreateWithFlags(&ev_start, cudaEventDisableTiming) != cudaSuccess) return cleanup(DMA_ERR_CUDA);
+    if (cudaEventCreateWithFlags(&ev_done, cudaEventDisableTiming) != cudaSuccess) return cleanup(DMA_ERR_CUDA);
+    for (int i = 0; i < NG * kPerGroup; ++i)
+        if (cudaEventCreateWithFlags(&ev[i], cudaEventDisableTiming) != cudaSuccess) return cleanup(DMA_ERR_CUDA);
+
+    // a [rows x width] block of a [rows x pitch] tensor; width == pitch is one plain copy
+    auto copy2d = [&](void* dst, const void* src, size_t pitch, size_t width, size_t rows, cudaMemcpyKind kind, cudaStream_t on) {
+        if (width == pitch) return cudaMemcpyAsync(dst, src, width * rows, kind, on) == cudaSuccess;
+        return cudaMemcpy2DAsync(dst, pitch, src, pitch, width, rows, kind, on) == cudaSuccess;
+    };
+    auto rec = [&](cudaEvent_t e, cudaStream_t on) { return cudaEventRecord(e, on) == cudaSuccess; };
+    auto wait = [&](cudaStream_t on, cudaEvent_t e) { return cudaStreamWaitEvent(on, e, 0) == cudaSuccess; };
+
+    struct Group { size_t q, k, h, bmp; int hq0; };
+    auto group_of = [&](int g) {
+        const int b = g / HG, hg = g % HG;
+        Group G;
+        G.hq0 = hg * nqh;
+        G.q = ((size_t)b * L * p->Hq + (size_t)hg * nqh) * d;          // elements into Q, O, dO, dQ
+        G.k = ((size_t)b * L * p->Hkv + (size_t)hg * nkh) * d;         // elements into K, V, dK, dV
+        G.h = ((size_t)b * p->Hq + (size_t)hg * nqh) * L;              // entries into bias, expiry, lse, dM
+        G.bmp = ((size_t)b * p->Hq + (size_t)hg * nqh) * ((Lo.nbmp / p->B) / p->Hq);
+        return G;
+    };
+    const size_t q_pitch = (size_t)p->Hq * d * esz, q_width = (size_t)nqh * d * esz;
+    const size_t k_pitch = (size_t)p->Hkv * d * esz, k_width = (size_t)nkh * d * esz;
+
+    bool ok = rec(ev_start, st) && wait(s_in, ev_start) && wait(s_out, ev_start);
+    ok = ok && cudaMemcpyAsync(a + Lo.W, hW_delta, Lo.wbytes, cudaMemcpyHostToDevice, s_in) == cudaSuccess &&
+         cudaMemcpyAsync(a + Lo.A, hA, (size_t)p->Hq * 4, cudaMemcpyHostToDevice, s_in) == cudaSuccess;
+    for (int g = 0; g < NG && ok; ++g) {
+        const Group G = group_of(g);
+        cudaEvent_t* e = ev + g * kPerGroup;
+        const cudaMemcpyKind in = cudaMemcpyHostToDevice;
+        ok = copy2d(a + Lo.V + G.k * esz, (const char*)hV + G.k * esz, k_pitch, k_width, L, in, s_in) && rec(e[kV], s_in) &&
+             copy2d(a + Lo.K + G.k * esz, (const char*)hK + G.k * esz, k_pitch, k_width, L, in, s_in) &&
+             copy2d(a + Lo.Q + G.q * esz, (const char*)hQ + G.q * esz, q_pitch, q_width, L, in, s_in) && rec(e[kKQ], s_in);
+        if (backward) ok = ok && copy2d(a + Lo.dO + G.q * esz, (const char*)hdO + G.q * esz, q_pitch, q_width, L, in, s_in) && rec(e[kdO], s_in);
     }
-    ok = ok && rec(kDone, s_out) && wait(st, kDone);
+    if (!ok) return cleanup(DMA_ERR_CUDA);
+
+    dma_problem_t sub = *p;
+    sub.B = 1; sub.Hq = nqh; sub.Hkv = nkh;
+    const int64_t qs[3] = {(int64_t)L * p->Hq * d, (int64_t)p->Hq * d, d}, ks[3] = {(int64_t)L * p->Hkv * d, (int64_t)p->Hkv * d, d};
+    for (int i = 0; i < 3; ++i) { sub.q_stride[i] = sub.o_stride[i] = qs[i]; sub.k_stride[i] = sub.v_stride[i] = ks[i]; }
+    const size_t f_ws = Lo.f_ws - (size_t)NG * kWsHeaderBytes, b_ws = Lo.b_ws - (size_t)NG * kWsHeaderBytes;
+    const size_t w_per_head = Lo.wbytes / 4 / p->Hq;
+    for (int g = 0; g < NG; ++g) {
+        const Group G = group_of(g);
+        cudaEvent_t* e = ev + g * kPerGroup;
+        float* bias = (float*)(a + Lo.bias) + G.h;
+        int32_t* expiry = (int32_t*)(a + Lo.expiry) + G.h;
+        uint32_t* bitmap = (uint32_t*)(a + Lo.bitmap) + G.bmp;
+        float* lse = (float*)(a + Lo.lse) + G.h;
+        char* wsf = a + Lo.ws_fwd + (size_t)g * kWsHeaderBytes;
+        if (!wait(st, e[kV])) return cleanup(DMA_ERR_CUDA);
+        if ((rc = dma_mask_build(&sub, a + Lo.V + G.k * esz, (float*)(a + Lo.W) + G.hq0 * w_per_head, (float*)(a + Lo.A) + G.hq0, bias,
+                                 expiry, bitmap, a + Lo.ws_mask, Lo.m_ws, st))) return cleanup(rc);
+        if (!wait(st, e[kKQ])) return cleanup(DMA_ERR_CUDA);
+        if ((rc = dma_attn_fwd(&sub, a + Lo.Q + G.q * esz, a + Lo.K + G.k * esz, a + Lo.V + G.k * esz, bias, expiry, bitmap,
+                               a + Lo.O + G.q * esz, lse, wsf, f_ws, st))) return cleanup(rc);
+        const cudaMemcpyKind out = cudaMemcpyDeviceToHost;
+        ok = rec(e[kO], st) && wait(s_out, e[kO]) &&
+             copy2d((char*)hO + G.q * esz, a + Lo.O + G.q * esz, q_pitch, q_width, L, out, s_out) &&
+             cudaMemcpyAsync(hlse + G.h, lse, (size_t)nqh * L * 4, out, s_out) == cudaSuccess;
+        if (backward) {
+            char* wsb = a + Lo.ws_bwd + (size_t)g * kWsHeaderBytes;
+            float* dM = (float*)(a + Lo.dM) + G.h;
+            if (!ok || !wait(st, e[kdO])) return cleanup(DMA_ERR_CUDA);
+            if ((rc = dma_attn_bwd(&sub, a + Lo.Q + G.q * esz, a + Lo.K + G.k * esz, a + Lo.V + G.k * esz, a + Lo.O + G.q * esz,
+                                   a + Lo.dO + G.q * esz, lse, bias, expiry, bitmap, a + Lo.dQ + G.q * esz, a + Lo.dK + G.k * esz,
+                                   a + Lo.dV + G.k * esz, dM, wsb, b_ws, st))) return cleanup(rc);
+            ok = rec(e[kG], st) && wait(s_out, e[kG]) &&
+                 copy2d((char*)hdQ + G.q * esz, a + Lo.dQ + G.q * esz, q_pitch, q_width, L, out, s_out) &&
+                 copy2d((char*)hdK + G.k * esz, a + Lo.dK + G.k * esz, k_pitch, k_width, L, out, s_out) &&
+                 copy2d((char*)hdV + G.k * esz, a + Lo.dV + G.k * esz, k_pitch, k_width, L, out, s_out) &&
+                 cudaMemcpyAsync(hdM + G.h, dM, (size_t)nqh * L * 4, out, s_out) == cudaSuccess;
+        }
+        if (!ok) return cleanup(DMA_ERR_CUDA);
+    }
+    ok = rec(ev_done, s_out) && wait(st, ev_done);
     if (!ok) return cleanup(DMA_ERR_CUDA);
     if (cudaStreamSynchronize(st) != cudaSuccess) return cleanup(DMA_ERR_CUDA);
-    int s1 = dma_read_status(a + Lo.ws_fwd, st);
-    if (s1) return cleanup(s1);
-    return cleanup(backward ? dma_read_status(a + Lo.ws_bwd, st) : DMA_OK);
+    // the groups' status words (one header each in front of the forward and of the backward workspace)
+    static_assert(kWsHeaderBytes % 4 == 0, "header");
+    int32_t heads[kMaxGroups * (kWsHeaderBytes / 4)];
+    for (int pass = 0; pass < (backward ? 2 : 1); ++pass) {
+        const char* src = a + (pass ? Lo.ws_bwd : Lo.ws_fwd);
+        if (cudaMemcpyAsync(heads, src, (size_t)NG * kWsHeaderBytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return cleanup(DMA_ERR_CUDA);
+        if (cudaStreamSynchronize(st) != cudaSuccess) return cleanup(DMA_ERR_CUDA);
+        for (int g = 0; g < NG; ++g)
+            if (heads[g * (kWsHeaderBytes / 4)] != 0) return cleanup(DMA_ERR_DEVICE_TIMEOUT);
+    }
+    return cleanup(DMA_OK);
 }
 
 }  // extern "C"
