@@ -230,11 +230,69 @@ __global__ void __launch_bounds__(kChunk) chunk_sort_kernel(const float* __restr
     sorted[((size_t)bh * nchunk + c) * kChunk + t] = s[t];   // ascending
 }
 
+// Work assignment of the expiry kernel. A key's walk over the sorted chunks ends once w keys have beaten it, after
+// about w / q keys if a fraction q of the head beats it: weak keys stop early, and the keys that fewer than w keys
+// beat at all walk the whole row to learn that their expiry is L. Threads of a CTA walk together, so the keys are
+// handed out in the order of a coarse rank (a counting sort on 12 bits of delta: exponent and top four mantissa bits),
+// which gives the keys of a CTA walks of similar length, and a key whose whole class ranks below w (or, in the
+// non-causal mode, at or above w) is tagged so that it does not walk at all.
+// perm[bh][pos] = key index | (tag << 30); tag 1: fewer than w keys beat it; tag 2: at least w keys beat it.
+constexpr int kRankBins = 4096;
+
+__global__ void __launch_bounds__(1024) rank_perm_kernel(const float* __restrict__ delta, uint32_t* __restrict__ perm, int L, int w) {
+    __shared__ int hist[kRankBins];      // counts, then the next free position of each class
+    __shared__ int wsum[32];
+    __shared__ uint8_t tag[kRankBins];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const float* dl = delta + (size_t)blockIdx.x * L;
+    uint32_t* out = perm + (size_t)blockIdx.x * L;
+    auto bin = [](float v) { return (int)((__float_as_uint(v) >> 19) & (kRankBins - 1)); };   // delta > 0: bit 31 is clear
+    for (int i = tid; i < kRankBins; i += 1024) hist[i] = 0;
+    __syncthreads();
+    for (int j = tid; j < L; j += 1024) atomicAdd(&hist[bin(dl[j])], 1);
+    __syncthreads();
+    // classes in descending order of delta: thread t owns the four classes kRankBins - 1 - 4t - {0, 1, 2, 3}
+    int c[4], run = 0;
+#pragma unroll
+    for (int u = 0; u < 4; ++u) { c[u] = hist[kRankBins - 1 - 4 * tid - u]; run += c[u]; }
+    int incl = run;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int t = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += t;
+    }
+    if (lane == 31) wsum[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+        int v = wsum[lane];
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int t = __shfl_up_sync(0xffffffffu, v, o);
+            if (lane >= o) v += t;
+        }
+        wsum[lane] = v;
+    }
+    __syncthreads();
+    int start = incl - run + (warp ? wsum[warp - 1] : 0);      // keys in classes above this thread's
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+        const int b = kRankBins - 1 - 4 * tid - u;
+        hist[b] = start;
+        tag[b] = start + c[u] <= w ? 1 : (start >= w ? 2 : 0);   // ranks of the class: [start, start + count)
+        start += c[u];
+    }
+    __syncthreads();
+    for (int j = tid; j < L; j += 1024) {
+        const int b = bin(dl[j]);
+        out[atomicAdd(&hist[b], 1)] = (uint32_t)j | ((uint32_t)tag[b] << 30);
+    }
+}
+
 // expiry[j] = max(j, index of the w-th key in index order that beats j), or L if fewer than w keys beat it.
 // Phase 1: the CTA walks the sorted chunks together (each staged once in shared memory as separate high / low
 // words, the next one already in flight) and every thread counts its beaters chunk by chunk with a binary search
-// until the count reaches w. Phase 2: the warp locates, lane by lane, the remaining need-th beater inside that
-// lane's final chunk with coalesced 32-key loads and a ballot.
+// until the count reaches w. Phase 2: each thread locates the remaining need-th beater inside its final chunk, in index
+// order, 32 keys at a time.
 // kVarlen: sequences packed along the key axis (sequence s owns the keys cu[s] <= j < cu[s+1]). A key competes only
 // with the keys of its own sequence [s0, s1): chunks before s0 count nothing, a chunk that straddles s0 or s1 is
 // counted entry by entry with the index test, the walk ends at s1, and L is replaced by s1.
@@ -244,15 +302,24 @@ template <int kMode>
 __global__ void __launch_bounds__(kExpThreads) expiry_kernel(const float* __restrict__ delta,
                                                              const unsigned long long* __restrict__ sorted,
                                                              int32_t* __restrict__ expiry, int L, int w, int nchunk,
-                                                             const int32_t* __restrict__ cu, int nseq) {
+                                                             const int32_t* __restrict__ cu, int nseq,
+                                                             const uint32_t* __restrict__ perm) {
     constexpr int kPer = kChunk / kExpThreads;
     constexpr bool kVarlen = kMode == 1, kAllRows = kMode == 2;
-    __shared__ uint32_t shi[2][kChunk], slo[2][kChunk];
+    static_assert(kChunk == 256 && kPer == 1, "the level-order layout below is written for 256-key chunks");
+    // sbf: the high words once more, in level order of the implicit search tree over the first 255 sorted entries (root at
+    // index 1, children of k at 2k and 2k + 1; the largest entry sits in slot 0). The probes of one search level are
+    // then neighbours in memory, so the first five levels of a warp's 32 searches cost one shared-memory access each;
+    // probing the sorted array itself puts every early level into a single bank (addresses 128 apart, 64 apart, ...).
+    __shared__ uint32_t shi[2][kChunk], slo[2][kChunk], sbf[2][kChunk];
     __shared__ int c_first;
-    const int bh = blockIdx.y, t = threadIdx.x, lane = t & 31, j = blockIdx.x * kExpThreads + t;
+    const int bh = blockIdx.y, t = threadIdx.x, lane = t & 31, slot = blockIdx.x * kExpThreads + t;
     const float* dl = delta + (size_t)bh * L;
     const unsigned long long* srt = sorted + (size_t)bh * nchunk * kChunk;
-    const bool valid = j < L;
+    const bool valid = slot < L;
+    // packed sequences keep the index order (perm == nullptr): a CTA's keys then share their documents' boundary chunks
+    const uint32_t entry = valid ? (perm ? perm[(size_t)bh * L + slot] : (uint32_t)slot) : 0u;
+    const int j = (int)(entry & 0x3FFFFFFFu), tag = (int)(entry >> 30);     // rank order: see rank_perm_kernel
     const unsigned long long key = valid ? sort_key(dl[j], j) : ~0ull;
     const uint32_t khi = (uint32_t)(key >> 32), klo = (uint32_t)key;
     int s0 = 0, s1 = L;
@@ -266,22 +333,30 @@ __global__ void __launch_bounds__(kExpThreads) expiry_kernel(const float* __rest
             s0 = max(cu[lo], 0);
             s1 = min(cu[lo + 1], L);
         }
-        if (t == 0) c_first = s0 / kChunk;                 // the CTA's first key has the smallest sequence start
+        if (t == 0) c_first = nchunk;
+        __syncthreads();
+        if (valid && tag != 1) atomicMin(&c_first, s0 / kChunk);   // the walk starts at the earliest sequence of the CTA's keys
         __syncthreads();
     }
     const int c_begin = kVarlen ? c_first : 0;
     int cnt = 0, fin = -1, need = 0;
-    bool done = !valid;
+    // tag 1: fewer than w keys of the whole head beat the key, so it is never dropped; tag 2 (used in the non-causal
+    // mode only): at least w beat it
+    const bool dropped = kAllRows && tag == 2;
+    bool done = !valid || tag == 1 || dropped;
     unsigned long long nxt[kPer];
 #pragma unroll
-    for (int u = 0; u < kPer; ++u) nxt[u] = srt[(size_t)c_begin * kChunk + u * kExpThreads + t];
-    for (int c = c_begin; c < nchunk; ++c) {
+    for (int u = 0; u < kPer; ++u) nxt[u] = c_begin < nchunk ? srt[(size_t)c_begin * kChunk + u * kExpThreads + t] : 0ull;
+    bool all_done = __syncthreads_and(done);               // a CTA of keys that need no walk (see rank_perm_kernel)
+    for (int c = c_begin; c < nchunk && !all_done; ++c) {
         uint32_t* hi = shi[c & 1];
         uint32_t* lo = slo[c & 1];
-#pragma unroll
-        for (int u = 0; u < kPer; ++u) {
-            hi[u * kExpThreads + t] = (uint32_t)(nxt[u] >> 32);
-            lo[u * kExpThreads + t] = (uint32_t)nxt[u];
+        uint32_t* bf = sbf[c & 1];
+        {
+            hi[t] = (uint32_t)(nxt[0] >> 32);
+            lo[t] = (uint32_t)nxt[0];
+            const int p1 = t + 1, z = __ffs(p1) - 1;                       // in-order position (1-based) and its level from the leaves
+            bf[t == kChunk - 1 ? 0 : (1 << (7 - z)) + (p1 >> (z + 1))] = (uint32_t)(nxt[0] >> 32);
         }
         if (c + 1 < nchunk) {
 #pragma unroll
@@ -295,10 +370,14 @@ __global__ void __launch_bounds__(kExpThreads) expiry_kernel(const float* __rest
                 // a = first position whose 64-bit key is greater than ours: fixed-depth, branch-free lower bound on
                 // the high words (delta bits), then the (normally empty) run of equal high words is resolved by the
                 // low words
-                int a = 0;
+                int a = 0, k = 1;
 #pragma unroll
-                for (int s = kChunk / 2; s > 0; s >>= 1) a += hi[a + s - 1] < khi ? s : 0;
-                a += hi[a] < khi ? 1 : 0;                      // a = number of entries with hi < khi (0 .. kChunk)
+                for (int s = kChunk / 2; s > 0; s >>= 1) {     // node k is the sorted entry a + s - 1
+                    const int right = bf[k] < khi ? 1 : 0;
+                    a += right ? s : 0;
+                    k = 2 * k + right;
+                }
+                a += (a == kChunk - 1 && bf[0] < khi) ? 1 : 0;   // a = number of entries with hi < khi (0 .. kChunk)
                 while (a < kChunk && hi[a] == khi && lo[a] <= klo) ++a;
                 n = kChunk - a;
             } else if ((c + 1) * kChunk <= s0) {
@@ -314,23 +393,23 @@ __global__ void __launch_bounds__(kExpThreads) expiry_kernel(const float* __rest
             if (cnt + n >= w) { need = w - cnt; fin = c; done = true; }
             cnt += n;
         }
-        if (__syncthreads_and(done)) break;
+        all_done = __syncthreads_and(done);
     }
-    // phase 2, warp-cooperative: lane `src` broadcasts (chunk, key, need); the warp scans that chunk 32 keys at a time
+    // phase 2: each thread scans its final chunk in index order, 32 keys at a time (32 independent loads), until the
+    // remaining need-th beater is found
     int e = s1;
-    const uint32_t pending = kAllRows ? 0u : __ballot_sync(0xffffffffu, fin >= 0);
-    for (uint32_t rest = pending; rest; rest &= rest - 1) {
-        const int src = __ffs(rest) - 1;
-        const int base = __shfl_sync(0xffffffffu, fin, src) * kChunk;
-        const uint32_t bhi = __shfl_sync(0xffffffffu, khi, src), blo = __shfl_sync(0xffffffffu, klo, src);
-        const int b0 = __shfl_sync(0xffffffffu, s0, src), b1 = __shfl_sync(0xffffffffu, s1, src);
-        int nd = __shfl_sync(0xffffffffu, need, src);
-        const unsigned long long bkey = ((unsigned long long)bhi << 32) | blo;
-        int found = b1;
+    if (!kAllRows && fin >= 0) {
+        const int base = fin * kChunk;
+        int nd = need, found = s1;
         for (int g = 0; g < kChunk; g += 32) {
-            const int k = base + g + lane;
-            const bool beat = k >= b0 && k < b1 && sort_key(dl[k], k) > bkey;
-            uint32_t m = __ballot_sync(0xffffffffu, beat);
+            uint32_t m = 0u;
+#pragma unroll
+            for (int u = 0; u < 32; ++u) {
+                const int k = base + g + u;
+                const bool in = k >= s0 && k < s1;
+                const float v = in ? __ldg(dl + k) : 0.0f;
+                m |= (in && sort_key(v, k) > key) ? 1u << u : 0u;
+            }
             const int pc = __popc(m);
             if (nd <= pc) {
                 for (int r = 1; r < nd; ++r) m &= m - 1;          // drop the nd-1 lowest beaters
@@ -339,9 +418,9 @@ __global__ void __launch_bounds__(kExpThreads) expiry_kernel(const float* __rest
             }
             nd -= pc;
         }
-        if (lane == src) e = max(j, found);
+        e = max(j, found);
     }
-    if (kAllRows) e = fin >= 0 ? 0 : L;
+    if (kAllRows) e = (fin >= 0 || dropped) ? 0 : L;
     if (valid) expiry[(size_t)bh * L + j] = e;
 }
 
@@ -381,9 +460,10 @@ __global__ void __launch_bounds__(128) bitmap_kernel(const int32_t* __restrict__
 
 constexpr int kStaticChunk = kChunk;
 
+// workspace: header | sorted chunks (8 bytes per padded key) | rank permutation (4 bytes per padded key)
 size_t mask_ws_bytes(const Prob& P) {
     const size_t nchunk = (P.L + kChunk - 1) / kChunk;
-    return kWsHeaderBytes + (size_t)P.B * P.Hq * nchunk * kChunk * sizeof(unsigned long long);
+    return kWsHeaderBytes + (size_t)P.B * P.Hq * nchunk * kChunk * (sizeof(unsigned long long) + sizeof(uint32_t));
 }
 
 template <typename T, int D>
@@ -439,12 +519,14 @@ int launch_mask_build(const Prob& P, const void* V, const float* W, const float*
         count_launch();
     } else {
         auto* sorted = reinterpret_cast<unsigned long long*>((char*)ws + kWsHeaderBytes);
+        uint32_t* perm = reinterpret_cast<uint32_t*>(sorted + (size_t)BH * nchunk * kChunk);
         chunk_sort_kernel<<<dim3(nchunk, BH), kChunk, 0, st>>>(bias, sorted, P.L, nchunk);
+        if (!cu) rank_perm_kernel<<<BH, 1024, 0, st>>>(bias, perm, P.L, P.w);
         const dim3 grid((P.L + kExpThreads - 1) / kExpThreads, BH);
-        if (cu) expiry_kernel<1><<<grid, kExpThreads, 0, st>>>(bias, sorted, expiry, P.L, P.w, nchunk, cu, nseq);
-        else if (!P.causal) expiry_kernel<2><<<grid, kExpThreads, 0, st>>>(bias, sorted, expiry, P.L, P.w, nchunk, nullptr, 0);
-        else expiry_kernel<0><<<grid, kExpThreads, 0, st>>>(bias, sorted, expiry, P.L, P.w, nchunk, nullptr, 0);
-        count_launch(2);
+        if (cu) expiry_kernel<1><<<grid, kExpThreads, 0, st>>>(bias, sorted, expiry, P.L, P.w, nchunk, cu, nseq, nullptr);
+        else if (!P.causal) expiry_kernel<2><<<grid, kExpThreads, 0, st>>>(bias, sorted, expiry, P.L, P.w, nchunk, nullptr, 0, perm);
+        else expiry_kernel<0><<<grid, kExpThreads, 0, st>>>(bias, sorted, expiry, P.L, P.w, nchunk, nullptr, 0, perm);
+        count_launch(cu ? 2 : 3);
     }
     if ((rc = check_launch())) return rc;
 
@@ -465,8 +547,8 @@ int launch_mask_build(const Prob& P, const void* V, const float* W, const float*
 // once per device with cudaGetSymbolAddress and that pointer is what the kernels receive.
 // ---------------------------------------------------------------------------------------------------------------
 namespace {
-constexpr size_t kStaticKeys = 1u << 20;   // 1 Mi sort keys = 8 MiB: B * Hq * roundup(L, 256) must not exceed this
-static __device__ __align__(256) unsigned long long g_static_scratch[dma::kWsHeaderBytes / 8 + kStaticKeys];
+constexpr size_t kStaticKeys = 1u << 20;   // 1 Mi sort keys (8 MiB) and their rank permutation (4 MiB): B * Hq * roundup(L, 256) must not exceed this
+static __device__ __align__(256) unsigned long long g_static_scratch[dma::kWsHeaderBytes / 8 + kStaticKeys + kStaticKeys / 2];
 constexpr int kMaxDevices = 64;
 void* g_static_ptr[kMaxDevices];            // per-device address of g_static_scratch (0 = not looked up yet)
 std::mutex g_static_mutex;
