@@ -391,6 +391,56 @@ def main():
         decode = {"us_per_step": d_ms * 1e3, "cached_keys": case.L, "kept_keys": keep, "algorithmic_bytes": d_bytes,
                   "gbs": d_bytes / (d_ms * 1e-3) / 1e9,
                   "dense_kv_read_bytes": 2 * case.B * case.Hkv * case.L * case.d * K.element_size()}
+        # the same with the kept set carried from step to step (dma_decode_step): 24 consecutive steps that append the
+        # workload's last 24 keys one at a time (delta of the new key + the step), the first 4 untimed
+        n_inc = 24
+        if case.L > n_inc + 1:
+            probs = [dma.problem(case.B, case.Hq, case.Hkv, n, case.d, case.w, dtype=case.torch_dtype) for n in range(case.L - n_inc, case.L + 1)]
+            for pp in probs:
+                for sdst, ssrc in ((pp.k_stride, K.stride()), (pp.v_stride, V.stride())):
+                    sdst[0], sdst[1], sdst[2] = ssrc[0], ssrc[1], ssrc[2]
+            state = dma.dma_decode_state(probs[0], dev)
+            dma.dma_decode_state_init(probs[0], dcache, state, ws_d)
+            i0, i1 = ev(), ev()
+            for t, pp in enumerate(probs[1:]):
+                if t == 4:
+                    torch.cuda.synchronize()
+                    i0.record()
+                dma.dma_delta_range(pp, V, W, A, dcache, pp.L - 1, pp.L)
+                dma.dma_decode_step(pp, qd, K, V, dcache, state, od, lsed, ws_d)
+            i1.record()
+            torch.cuda.synchronize()
+            inc_ms = i0.elapsed_time(i1) / (n_inc - 4)
+            inc_bytes = 2 * case.B * case.Hq * keep * (case.d * K.element_size() + 4 + 4)      # K, V rows, delta and index of the kept keys
+            decode.update({"incremental_us_per_step": inc_ms * 1e3, "incremental_algorithmic_bytes": inc_bytes,
+                           "incremental_gbs": inc_bytes / (inc_ms * 1e-3) / 1e9})
+            # the same two loops captured once in CUDA graphs and replayed: the device time without the host's launch cost
+            # (seven and four small kernels per step: the eager numbers above are bound by the submission rate)
+            try:
+                g_full = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g_full):
+                    for _ in range(20):
+                        dma.dma_decode(pd, qd, K, V, dcache, od, lsed, None, False, ws_d)
+                dma.dma_decode_state_init(probs[0], dcache, state, ws_d)
+                g_inc = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g_inc):
+                    for pp in probs[1:21]:
+                        dma.dma_delta_range(pp, V, W, A, dcache, pp.L - 1, pp.L)
+                        dma.dma_decode_step(pp, qd, K, V, dcache, state, od, lsed, ws_d)
+                for name, gr, reinit in (("graph_us_per_step", g_full, False), ("incremental_graph_us_per_step", g_inc, True)):
+                    ts = []
+                    for _ in range(4):
+                        if reinit:
+                            dma.dma_decode_state_init(probs[0], dcache, state, ws_d)
+                        torch.cuda.synchronize()
+                        d0.record()
+                        gr.replay()
+                        d1.record()
+                        torch.cuda.synchronize()
+                        ts.append(d0.elapsed_time(d1) / 20)
+                    decode[name] = min(ts[1:]) * 1e3
+            except RuntimeError as e:          # capture refused: keep the eager numbers
+                decode["graph_error"] = str(e)[:200]
 
     # ---- end to end through the host-buffer entry point: pinned host tensors in, results back on the host
     e2e = None

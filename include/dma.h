@@ -186,6 +186,24 @@ int dma_decode_workspace(const dma_problem_t* p, size_t* bytes);
 int dma_decode(const dma_problem_t* p, const void* q, const void* K, const void* V, const float* delta, int64_t delta_ld,
                void* o, float* lse, int32_t* sel_idx, void* ws, size_t ws_bytes, void* cuda_stream);
 
+/* Decoding with a carried state: one key is appended per step, so the set of the w best keys changes by at most one
+ * member (the new key enters iff it beats the weakest kept key or the set is not full, and that weakest key leaves).
+ * A step then costs O(w) whatever the number of cached keys: no scan of the delta row.
+ *   state: device memory, dma_decode_state_bytes() bytes ([B, Hq] rows of 8 int32 of header (count, position and 64-bit
+ *          order key of the weakest kept key) and p->w int32 kept key indices in no particular order), 16-byte aligned,
+ *          owned by the caller; it depends on B, Hq and w only.
+ *   dma_decode_state_init: the state for the first N = p->L cached keys (the selection of dma_decode).
+ *   dma_decode_step: p->L = N counts the cached keys INCLUDING the key appended for this step (index N - 1), whose
+ *          K, V and delta entries are already in the caches; `state` describes the first N - 1 keys on entry and all N
+ *          on return. o, lse as dma_decode: the same keys are selected, so the results agree up to summation order.
+ *          (N = 1 with a state whose count is 0, e.g. zero-filled memory, starts a sequence.)
+ *   ws: dma_decode_workspace() bytes of the same problem. */
+int dma_decode_state_bytes(const dma_problem_t* p, size_t* bytes);
+int dma_decode_state_init(const dma_problem_t* p, const float* delta, int64_t delta_ld, void* state, void* ws, size_t ws_bytes,
+                          void* cuda_stream);
+int dma_decode_step(const dma_problem_t* p, const void* q, const void* K, const void* V, const float* delta, int64_t delta_ld,
+                    void* state, void* o, float* lse, void* ws, size_t ws_bytes, void* cuda_stream);
+
 /* The whole hot path on HOST buffers (all contiguous, default strides only): copies Q,K,V,(dO),W_delta,A into the
  * caller's device arena, runs dma_mask_build, dma_attn_fwd and, if `backward` != 0, dma_attn_bwd on the stream,
  * copies O, lse (and dQ,dK,dV,dM) back and synchronises the stream before returning. The copies run on two helper

@@ -19,7 +19,7 @@ DMA_FLAG_IGNORE_BITMAP, DMA_FLAG_SIMT, DMA_FLAG_COMPACT_KV, DMA_FLAG_FULL_DELTA 
 ENTRY_POINTS = ("dma_query_workspace", "dma_bitmap_words", "dma_mask_build", "dma_attn_fwd", "dma_attn_bwd",
                 "dma_read_status", "dma_launch_count", "dma_strerror", "dma_step_host_arena", "dma_step_host", "dma_mask_build_static", "dma_selftest_wait_timeout",
                 "dma_mask_bwd_workspace", "dma_mask_bwd", "dma_delta_range", "dma_decode_workspace", "dma_decode",
-                "dma_mask_build_varlen")
+                "dma_mask_build_varlen", "dma_decode_state_bytes", "dma_decode_state_init", "dma_decode_step")
 
 
 class DmaError(RuntimeError):
@@ -179,6 +179,41 @@ def dma_decode(p, q, K, V, delta, o=None, lse=None, sel_idx=None, want_idx=False
     _check(lib().dma_decode(ctypes.byref(p), _ptr(q), _ptr(K), _ptr(V), _ptr(delta), ctypes.c_int64(delta.stride(1)), _ptr(o),
                             _ptr(lse), _ptr(sel_idx), _ptr(ws), ctypes.c_size_t(ws.numel()), _stream()), "dma_decode")
     return o, lse, sel_idx
+
+
+def dma_decode_state(p, device):
+    """Zero-filled incremental decoding state for (B, Hq, w): int32 [B*Hq, 8 + roundup(w, 4)] (count 0 everywhere)."""
+    n = ctypes.c_size_t()
+    _check(lib().dma_decode_state_bytes(ctypes.byref(p), ctypes.byref(n)), "dma_decode_state_bytes")
+    return torch.zeros(p.B * p.Hq, n.value // 4 // (p.B * p.Hq), dtype=torch.int32, device=device)
+
+
+def dma_decode_state_init(p, delta, state, ws=None):
+    if ws is None:
+        ws = _ws(dma_decode_workspace(p), delta.device)
+    _check(lib().dma_decode_state_init(ctypes.byref(p), _ptr(delta), ctypes.c_int64(delta.stride(1)), _ptr(state), _ptr(ws),
+                                       ctypes.c_size_t(ws.numel()), _stream()), "dma_decode_state_init")
+    return state
+
+
+def dma_decode_step(p, q, K, V, delta, state, o=None, lse=None, ws=None):
+    """One decoding step with the carried state (p.L counts the cached keys including the one just appended)."""
+    dev = q.device
+    if o is None:
+        o = torch.empty_like(q)
+    if lse is None:
+        lse = torch.empty(p.B, p.Hq, dtype=torch.float32, device=dev)
+    if ws is None:
+        ws = _ws(dma_decode_workspace(p), dev)
+    _check(lib().dma_decode_step(ctypes.byref(p), _ptr(q), _ptr(K), _ptr(V), _ptr(delta), ctypes.c_int64(delta.stride(1)),
+                                 _ptr(state), _ptr(o), _ptr(lse), _ptr(ws), ctypes.c_size_t(ws.numel()), _stream()), "dma_decode_step")
+    return o, lse
+
+
+def decode_state_sets(state, w):
+    """The kept index sets of a state tensor: list over rows of sorted Python lists."""
+    st = state.cpu()
+    return [sorted(st[r, 8:8 + int(st[r, 0])].tolist()) for r in range(st.shape[0])]
 
 
 def dma_attn_fwd(p, Q, K, V, bias, expiry, bitmap, O=None, lse=None, ws=None):

@@ -33,6 +33,7 @@ int resolve(const dma_problem_t* p, Prob* o) {
     if (!(p->softmax_scale >= 0.0f) || std::isinf(p->softmax_scale)) return DMA_ERR_SHAPE;
     o->B = p->B; o->Hq = p->Hq; o->Hkv = p->Hkv; o->L = p->L; o->d = p->d; o->G = p->Hq / p->Hkv;
     o->w = p->w < p->L ? p->w : p->L;
+    o->w_cap = p->w;
     o->dtype = p->dtype; o->flags = p->flags; o->causal = p->causal;
     o->bm = p->tile_m ? p->tile_m : 128;
     o->bn = p->tile_n ? p->tile_n : 128;
@@ -186,6 +187,41 @@ int dma_decode(const dma_problem_t* p, const void* q, const void* K, const void*
     if (!ws || ws_bytes < decode_ws_bytes(P) || !aligned16(ws)) return DMA_ERR_WORKSPACE;
     if ((rc = device_ok())) return rc;
     return launch_decode(P, q, K, V, delta, delta_ld, o, lse, sel_idx, ws, (cudaStream_t)cuda_stream);
+}
+
+int dma_decode_state_bytes(const dma_problem_t* p, size_t* bytes) {
+    Prob P;
+    int rc = resolve(p, &P);
+    if (rc) return rc;
+    if (!bytes) return DMA_ERR_NULL;
+    *bytes = decode_state_bytes(P);
+    return DMA_OK;
+}
+
+int dma_decode_state_init(const dma_problem_t* p, const float* delta, int64_t delta_ld, void* state, void* ws, size_t ws_bytes,
+                          void* cuda_stream) {
+    Prob P;
+    int rc = resolve(p, &P);
+    if (rc) return rc;
+    if (!delta || !state) return DMA_ERR_NULL;
+    if (!aligned16(delta) || !aligned16(state)) return DMA_ERR_ALIGN;
+    if (delta_ld < P.L) return DMA_ERR_SHAPE;
+    if (!ws || ws_bytes < decode_ws_bytes(P) || !aligned16(ws)) return DMA_ERR_WORKSPACE;
+    if ((rc = device_ok())) return rc;
+    return launch_decode_state_init(P, delta, delta_ld, (int*)state, ws, (cudaStream_t)cuda_stream);
+}
+
+int dma_decode_step(const dma_problem_t* p, const void* q, const void* K, const void* V, const float* delta, int64_t delta_ld,
+                    void* state, void* o, float* lse, void* ws, size_t ws_bytes, void* cuda_stream) {
+    Prob P;
+    int rc = resolve(p, &P);
+    if (rc) return rc;
+    if (!q || !K || !V || !delta || !state || !o || !lse) return DMA_ERR_NULL;
+    if (!aligned16(q) || !aligned16(K) || !aligned16(V) || !aligned16(delta) || !aligned16(state) || !aligned16(o)) return DMA_ERR_ALIGN;
+    if (delta_ld < P.L) return DMA_ERR_SHAPE;
+    if (!ws || ws_bytes < decode_ws_bytes(P) || !aligned16(ws)) return DMA_ERR_WORKSPACE;
+    if ((rc = device_ok())) return rc;
+    return launch_decode_step(P, q, K, V, delta, delta_ld, (int*)state, o, lse, ws, (cudaStream_t)cuda_stream);
 }
 
 int dma_attn_fwd(const dma_problem_t* p, const void* Q, const void* K, const void* V, const float* bias,

@@ -15,6 +15,7 @@ constexpr int kWsHeaderBytes = 256;   // every workspace starts with this header
 struct Prob {
     int B, Hq, Hkv, L, d, G;
     int w;                 // min(w, L)
+    int w_cap;             // w as given (the capacity of an incremental decoding state)
     int dtype, flags;
     int causal;            // 1: key j visible to rows i >= j; 0: to every row (the key's first row is 0 instead of j)
     int bm, bn, Tr, Tc, Wd;   // bitmap tile sizes, tile counts, uint32 words per bitmap row
@@ -32,6 +33,10 @@ size_t mask_bwd_ws_bytes(const Prob& P);
 int launch_delta_range(const Prob& P, const void* V, const float* W, const float* A, float* delta, int64_t ld, int j_begin,
                        int j_end, cudaStream_t st);
 size_t decode_ws_bytes(const Prob& P);
+size_t decode_state_bytes(const Prob& P);
+int launch_decode_state_init(const Prob& P, const float* delta, int64_t ld, int* state, void* ws, cudaStream_t st);
+int launch_decode_step(const Prob& P, const void* q, const void* K, const void* V, const float* delta, int64_t ld, int* state,
+                       void* o, float* lse, void* ws, cudaStream_t st);
 int launch_decode(const Prob& P, const void* q, const void* K, const void* V, const float* delta, int64_t ld, void* o, float* lse,
                   int32_t* sel_idx, void* ws, cudaStream_t st);
 int launch_mask_bwd(const Prob& P, const void* V, const float* W, const float* A, const float* delta, const float* dM,

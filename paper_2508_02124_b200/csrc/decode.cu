@@ -149,7 +149,8 @@ __global__ void __launch_bounds__(256) decode_thr_kernel(const float* __restrict
 }
 
 __global__ void __launch_bounds__(256) decode_index_kernel(const float* __restrict__ delta, int64_t ld, int N, int keep,
-                                                           const unsigned long long* __restrict__ thr, int32_t* __restrict__ idx) {
+                                                           const unsigned long long* __restrict__ thr, int32_t* __restrict__ idx,
+                                                           int64_t idx_stride) {
     __shared__ int wsum[2][8];
     const int bh = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const float* dl = delta + (size_t)bh * ld;
@@ -169,7 +170,7 @@ __global__ void __launch_bounds__(256) decode_index_kernel(const float* __restri
             total += c;
         }
         const int pos = n + before + __popc(bal & ((1u << lane) - 1));
-        if (sel && pos < keep) idx[(size_t)bh * keep + pos] = j;
+        if (sel && pos < keep) idx[(size_t)bh * idx_stride + pos] = j;
         n += total;
     }
 }
@@ -185,53 +186,18 @@ __device__ __forceinline__ void load4(const __nv_bfloat16* p, float (&v)[4]) {
 }
 
 // partial [bh][split][D + 2]: o (unnormalised, relative to m), m (log2 domain), l
+// The attention part shared by the two decoding kernels: `list` (shared memory) holds `count` key indices of this CTA.
+// Each warp takes four of them per round (8 bytes of the K / V row per lane), online softmax per warp, then the warps are
+// combined in shared memory and the CTA's partial (o relative to m, m in the log2 domain, l) is written.
 template <typename T, int D>
-__global__ void __launch_bounds__(kAttnThreads) decode_attn_kernel(const T* __restrict__ q, const T* __restrict__ K, const T* __restrict__ V,
-                                                                   const float* __restrict__ delta, int64_t ld,
-                                                                   const unsigned long long* __restrict__ thr, float* __restrict__ partial,
-                                                                   int N, int Hq, int G, float scale_log2, int nsplit,
-                                                                   int64_t ks_b, int64_t ks_l, int64_t ks_h, int64_t vs_b, int64_t vs_l,
-                                                                   int64_t vs_h) {
+__device__ __forceinline__ void decode_attend(const int* list, int count, const T* __restrict__ q, const T* __restrict__ K,
+                                              const T* __restrict__ V, const float* __restrict__ dl, float* __restrict__ out,
+                                              int bh, int b, int hk, float scale_log2, int64_t ks_b, int64_t ks_l, int64_t ks_h,
+                                              int64_t vs_b, int64_t vs_l, int64_t vs_h) {
     constexpr int LPK = D / 4;                 // lanes per key row (4 channels per lane)
     constexpr int KPW = 32 / LPK;              // keys per warp instruction
-    __shared__ int list[kSplitKeys];
-    __shared__ int s_count, wsum[2][8];
     __shared__ float s_part[8][D + 2];
-    const int split = blockIdx.x, bh = blockIdx.y, b = bh / Hq, h = bh % Hq, hk = h / G;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const float* dl = delta + (size_t)bh * ld;
-    const unsigned long long Tkey = thr[bh];
-    const int j_begin = split * kSplitKeys, j_end = min(N, j_begin + kSplitKeys);
-    // ordered compaction of the split's selected keys
-    int n = 0, buf = 0;
-    float dpre[kSplitKeys / kAttnThreads];          // the split's deltas of this thread, all loads in flight together
-#pragma unroll
-    for (int t = 0; t < kSplitKeys / kAttnThreads; ++t) {
-        const int j = j_begin + t * kAttnThreads + tid;
-        dpre[t] = j < j_end ? dl[j] : 0.0f;
-    }
-#pragma unroll
-    for (int t = 0; t < kSplitKeys / kAttnThreads; ++t, buf ^= 1) {
-        const int base = j_begin + t * kAttnThreads;
-        if (base >= j_end) break;
-        const int j = base + tid;
-        const bool sel = j < j_end && key_of(dpre[t], j) >= Tkey;
-        const uint32_t bal = __ballot_sync(0xffffffffu, sel);
-        if (lane == 0) wsum[buf][warp] = __popc(bal);
-        __syncthreads();
-        int before = 0, total = 0;
-#pragma unroll
-        for (int wq = 0; wq < 8; ++wq) {
-            const int c = wsum[buf][wq];
-            before += wq < warp ? c : 0;
-            total += c;
-        }
-        if (sel) list[n + before + __popc(bal & ((1u << lane) - 1))] = j;
-        n += total;
-    }
-    if (tid == 0) s_count = n;
-    __syncthreads();
-    const int count = s_count;
     // each warp: KPW keys per instruction (LPK lanes per key, 4 channels per lane), four such groups per round
     const int sub = lane % LPK, grp = lane / LPK;
     float qv[4];
@@ -292,7 +258,6 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attn_kernel(const T* __re
         if (sub == 0) { s_part[warp][D] = m; s_part[warp][D + 1] = l; }
     }
     __syncthreads();
-    float* out = partial + ((size_t)bh * nsplit + split) * (D + 2);
     float mx = -INFINITY;
 #pragma unroll
     for (int wq = 0; wq < 8; ++wq) mx = fmaxf(mx, s_part[wq][D]);
@@ -310,8 +275,163 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attn_kernel(const T* __re
 }
 
 template <typename T, int D>
+__global__ void __launch_bounds__(kAttnThreads) decode_attn_kernel(const T* __restrict__ q, const T* __restrict__ K, const T* __restrict__ V,
+                                                                   const float* __restrict__ delta, int64_t ld,
+                                                                   const unsigned long long* __restrict__ thr, float* __restrict__ partial,
+                                                                   int N, int Hq, int G, float scale_log2, int nsplit,
+                                                                   int64_t ks_b, int64_t ks_l, int64_t ks_h, int64_t vs_b, int64_t vs_l,
+                                                                   int64_t vs_h) {
+    constexpr int LPK = D / 4;                 // lanes per key row (4 channels per lane)
+    constexpr int KPW = 32 / LPK;              // keys per warp instruction
+    __shared__ int list[kSplitKeys];
+    __shared__ int s_count, wsum[2][8];
+    const int split = blockIdx.x, bh = blockIdx.y, b = bh / Hq, h = bh % Hq, hk = h / G;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const float* dl = delta + (size_t)bh * ld;
+    const unsigned long long Tkey = thr[bh];
+    const int j_begin = split * kSplitKeys, j_end = min(N, j_begin + kSplitKeys);
+    // ordered compaction of the split's selected keys
+    int n = 0, buf = 0;
+    float dpre[kSplitKeys / kAttnThreads];          // the split's deltas of this thread, all loads in flight together
+#pragma unroll
+    for (int t = 0; t < kSplitKeys / kAttnThreads; ++t) {
+        const int j = j_begin + t * kAttnThreads + tid;
+        dpre[t] = j < j_end ? dl[j] : 0.0f;
+    }
+#pragma unroll
+    for (int t = 0; t < kSplitKeys / kAttnThreads; ++t, buf ^= 1) {
+        const int base = j_begin + t * kAttnThreads;
+        if (base >= j_end) break;
+        const int j = base + tid;
+        const bool sel = j < j_end && key_of(dpre[t], j) >= Tkey;
+        const uint32_t bal = __ballot_sync(0xffffffffu, sel);
+        if (lane == 0) wsum[buf][warp] = __popc(bal);
+        __syncthreads();
+        int before = 0, total = 0;
+#pragma unroll
+        for (int wq = 0; wq < 8; ++wq) {
+            const int c = wsum[buf][wq];
+            before += wq < warp ? c : 0;
+            total += c;
+        }
+        if (sel) list[n + before + __popc(bal & ((1u << lane) - 1))] = j;
+        n += total;
+    }
+    if (tid == 0) s_count = n;
+    __syncthreads();
+    decode_attend<T, D>(list, s_count, q, K, V, dl, partial + ((size_t)bh * nsplit + split) * (D + 2), bh, b, hk, scale_log2, ks_b, ks_l,
+                        ks_h, vs_b, vs_l, vs_h);
+}
+
+// ---- incremental decoding: the kept set is carried from step to step --------------------------------------------------
+// One key is appended per step, so the set of the w best keys changes by at most one member: the new key enters iff it
+// beats the weakest kept key (or the set is not full yet), and that weakest key leaves. The state of a (batch, head) row:
+//   int32 [0] count (<= w)   [1] position of the weakest kept key in the list   [2..3] its 64-bit sort key   [4..7] unused
+//   int32 [8 .. 8 + w)       the kept key indices, in no particular order
+// A step costs O(w), whatever the number of cached keys: no scan of the delta row.
+constexpr int kStateHeader = 8;
+constexpr int kListSplit = 128;            // kept keys per CTA of the list attention kernel (256: 4 us slower per step at w = 2048)
+
+__device__ __forceinline__ int state_stride(int w_cap) { return kStateHeader + ((w_cap + 3) & ~3); }
+
+// what the appended key N - 1 does to a row's set: 0 nothing, 1 appended (set not full), 2 replaces the weakest
+__device__ __forceinline__ int step_mode(const int* hdr, int w_cap, unsigned long long kn) {
+    const int count = hdr[0];
+    if (count < w_cap) return 1;
+    const unsigned long long kmin = ((unsigned long long)(unsigned)hdr[3] << 32) | (unsigned)hdr[2];
+    return kn > kmin ? 2 : 0;
+}
+
+// weakest key of the row's list (entry `skip_pos`, if >= 0, reads as key `skip_j`): written to the header by thread 0
+__device__ __forceinline__ void store_weakest(int* hdr, const int* kept, int count, const float* dl, int skip_pos, int skip_j) {
+    __shared__ unsigned long long s_key[32];
+    __shared__ int s_pos[32];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarp = blockDim.x >> 5;
+    unsigned long long best = ~0ull;
+    int pos = -1;
+    for (int i = tid; i < count; i += blockDim.x) {
+        const int j = i == skip_pos ? skip_j : kept[i];
+        const unsigned long long k = key_of(dl[j], j);
+        if (k < best) { best = k; pos = i; }
+    }
+    for (int o = 16; o; o >>= 1) {
+        const unsigned long long k2 = __shfl_xor_sync(0xffffffffu, best, o);
+        const int p2 = __shfl_xor_sync(0xffffffffu, pos, o);
+        if (k2 < best) { best = k2; pos = p2; }
+    }
+    if (lane == 0) { s_key[warp] = best; s_pos[warp] = pos; }
+    __syncthreads();
+    if (tid == 0) {
+        for (int wq = 1; wq < nwarp; ++wq)
+            if (s_key[wq] < best) { best = s_key[wq]; pos = s_pos[wq]; }
+        hdr[1] = pos;
+        hdr[2] = (int)(uint32_t)best;
+        hdr[3] = (int)(uint32_t)(best >> 32);
+    }
+}
+
+// after decode_index_kernel has written the kept indices of the first N keys: count and weakest key
+__global__ void __launch_bounds__(256) decode_state_init_kernel(const float* __restrict__ delta, int64_t ld, int keep, int w_cap,
+                                                                int* __restrict__ state) {
+    const int bh = blockIdx.x;
+    int* hdr = state + (size_t)bh * state_stride(w_cap);
+    if (threadIdx.x == 0) hdr[0] = keep;
+    store_weakest(hdr, hdr + kStateHeader, keep, delta + (size_t)bh * ld, -1, 0);
+}
+
+// attention over the row's kept list as it is AFTER the appended key N - 1 is taken into account (the stored state still
+// describes the first N - 1 keys; decode_state_update_kernel brings it up to date afterwards)
+template <typename T, int D>
+__global__ void __launch_bounds__(kAttnThreads) decode_list_attn_kernel(const T* __restrict__ q, const T* __restrict__ K,
+                                                                        const T* __restrict__ V, const float* __restrict__ delta,
+                                                                        int64_t ld, const int* __restrict__ state, int w_cap,
+                                                                        float* __restrict__ partial, int N, int Hq, int G,
+                                                                        float scale_log2, int nsplit, int64_t ks_b, int64_t ks_l,
+                                                                        int64_t ks_h, int64_t vs_b, int64_t vs_l, int64_t vs_h) {
+    __shared__ int list[kListSplit];
+    const int split = blockIdx.x, bh = blockIdx.y, b = bh / Hq, h = bh % Hq, hk = h / G;
+    const int tid = threadIdx.x;
+    const float* dl = delta + (size_t)bh * ld;
+    const int* hdr = state + (size_t)bh * state_stride(w_cap);
+    const int* kept = hdr + kStateHeader;
+    const int newj = N - 1, count = hdr[0];
+    const int mode = step_mode(hdr, w_cap, key_of(dl[newj], newj));
+    const int eff = count + (mode == 1 ? 1 : 0), weakest = hdr[1];
+    const int e = split * kListSplit + tid;
+    if (tid < kListSplit && e < eff) list[tid] = (e >= count || (mode == 2 && e == weakest)) ? newj : kept[e];
+    __syncthreads();
+    decode_attend<T, D>(list, max(0, min(kListSplit, eff - split * kListSplit)), q, K, V, dl,
+                        partial + ((size_t)bh * nsplit + split) * (D + 2), bh, b, hk, scale_log2, ks_b, ks_l, ks_h, vs_b, vs_l, vs_h);
+}
+
+// brings a row's state up to date with the appended key N - 1 (every thread of the CTA takes part)
+__device__ __forceinline__ void decode_state_update(const float* __restrict__ delta, int64_t ld, int N, int w_cap,
+                                                    int* __restrict__ state, int bh) {
+    const float* dl = delta + (size_t)bh * ld;
+    int* hdr = state + (size_t)bh * state_stride(w_cap);
+    int* kept = hdr + kStateHeader;
+    const int newj = N - 1, count = hdr[0], weakest = hdr[1];
+    const unsigned long long kn = key_of(dl[newj], newj);
+    const int mode = step_mode(hdr, w_cap, kn);
+    __syncthreads();                                   // every thread has read the header before anyone rewrites it
+    if (mode == 0) return;
+    if (mode == 1) {                                   // the appended key has the largest index: on equal delta it is the weakest
+        if (threadIdx.x == 0) {
+            const unsigned long long kmin = ((unsigned long long)(unsigned)hdr[3] << 32) | (unsigned)hdr[2];
+            kept[count] = newj;
+            hdr[0] = count + 1;
+            if (count == 0 || kn < kmin) { hdr[1] = count; hdr[2] = (int)(uint32_t)kn; hdr[3] = (int)(uint32_t)(kn >> 32); }
+        }
+        return;
+    }
+    store_weakest(hdr, kept, count, dl, weakest, newj);
+    if (threadIdx.x == 0) kept[weakest] = newj;
+}
+
+template <typename T, int D>
 __global__ void __launch_bounds__(8 * D) decode_combine_kernel(const float* __restrict__ partial, T* __restrict__ o, float* __restrict__ lse,
-                                                               int nsplit) {
+                                                               int nsplit, const float* __restrict__ delta = nullptr, int64_t ld = 0,
+                                                               int N = 0, int w_cap = 0, int* __restrict__ state = nullptr) {
     __shared__ float s_m[8], s_l[8], s_o[8][D];
     const int bh = blockIdx.x, c = threadIdx.x % D, g = threadIdx.x / D;     // group g takes the splits s = g, g + 8, ...
     const float* p = partial + (size_t)bh * nsplit * (D + 2);
@@ -342,6 +462,8 @@ __global__ void __launch_bounds__(8 * D) decode_combine_kernel(const float* __re
         if constexpr (sizeof(T) == 2) o[(size_t)bh * D + c] = __float2bfloat16_rn(v); else o[(size_t)bh * D + c] = v;
         if (c == 0) lse[bh] = lt > 0.0f ? 0.6931471805599453f * (m_all + log2f(lt)) : -INFINITY;
     }
+    // incremental decoding: the attention kernel has read the row's state, which can now take in the appended key
+    if (state) decode_state_update(delta, ld, N, w_cap, state, bh);
 }
 
 template <typename T, int D>
@@ -361,10 +483,18 @@ static int decode_splits(const Prob& P) { return (P.L + kSplitKeys - 1) / kSplit
 
 static size_t decode_hist_bytes(const Prob& P) { return (size_t)3 * P.B * P.Hq * 2048 * sizeof(int); }
 
+static int list_splits(const Prob& P) { return (P.w_cap + kListSplit - 1) / kListSplit; }
+
+// header | thresholds | histograms | partials of the larger of the two attention kernels' split counts
 size_t decode_ws_bytes(const Prob& P) {
     const size_t bh = (size_t)P.B * P.Hq;
+    const size_t splits = (size_t)(decode_splits(P) > list_splits(P) ? decode_splits(P) : list_splits(P));
     return kWsHeaderBytes + ((bh * sizeof(unsigned long long) + 255) / 256) * 256 + decode_hist_bytes(P) +
-           bh * decode_splits(P) * (P.d + 2) * sizeof(float);
+           bh * splits * (P.d + 2) * sizeof(float);
+}
+
+size_t decode_state_bytes(const Prob& P) {
+    return (size_t)P.B * P.Hq * (kStateHeader + ((P.w_cap + 3) & ~3)) * sizeof(int);
 }
 
 int launch_decode(const Prob& P, const void* q, const void* K, const void* V, const float* delta, int64_t ld, void* o, float* lse,
@@ -383,7 +513,7 @@ int launch_decode(const Prob& P, const void* q, const void* K, const void* V, co
     decode_thr_kernel<<<(unsigned)bh, 256, 0, st>>>(delta, ld, P.L, P.w, ghist, (int)bh, thr);
     count_launch();
     if (sel_idx) {
-        decode_index_kernel<<<(unsigned)bh, 256, 0, st>>>(delta, ld, P.L, P.w < P.L ? P.w : P.L, thr, sel_idx);
+        decode_index_kernel<<<(unsigned)bh, 256, 0, st>>>(delta, ld, P.L, P.w, thr, sel_idx, P.w);
         count_launch();
     }
     const int ns = decode_splits(P);
@@ -392,6 +522,52 @@ int launch_decode(const Prob& P, const void* q, const void* K, const void* V, co
                           : launch_typed<__nv_bfloat16, 64>(P, q, K, V, delta, ld, o, lse, thr, partial, ns, st);
     return P.d == 128 ? launch_typed<float, 128>(P, q, K, V, delta, ld, o, lse, thr, partial, ns, st)
                       : launch_typed<float, 64>(P, q, K, V, delta, ld, o, lse, thr, partial, ns, st);
+}
+
+// Builds the incremental state from the first N = P.L cached keys: the select kernels, the kept indices into the state's
+// lists, then count and weakest key.
+int launch_decode_state_init(const Prob& P, const float* delta, int64_t ld, int* state, void* ws, cudaStream_t st) {
+    const size_t bh = (size_t)P.B * P.Hq;
+    auto* thr = reinterpret_cast<unsigned long long*>((char*)ws + kWsHeaderBytes);
+    int* ghist = reinterpret_cast<int*>((char*)thr + ((bh * sizeof(unsigned long long) + 255) / 256) * 256);
+    if (P.w < P.L) {
+        if (cudaMemsetAsync(ghist, 0, decode_hist_bytes(P), st) != cudaSuccess) return DMA_ERR_CUDA;
+        const dim3 grid((P.L + kSliceKeys - 1) / kSliceKeys, (unsigned)bh);
+        for (int pass = 0; pass < 3; ++pass)
+            decode_hist_kernel<<<grid, 256, 0, st>>>(delta, ld, P.L, P.w, pass, ghist, (int)bh);
+        count_launch(3);
+    }
+    decode_thr_kernel<<<(unsigned)bh, 256, 0, st>>>(delta, ld, P.L, P.w, ghist, (int)bh, thr);
+    const int stride = kStateHeader + ((P.w_cap + 3) & ~3);
+    decode_index_kernel<<<(unsigned)bh, 256, 0, st>>>(delta, ld, P.L, P.w, thr, state + kStateHeader, stride);
+    decode_state_init_kernel<<<(unsigned)bh, 256, 0, st>>>(delta, ld, P.w, P.w_cap, state);
+    count_launch(3);
+    return check_launch();
+}
+
+template <typename T, int D>
+static int launch_step_typed(const Prob& P, const void* q, const void* K, const void* V, const float* delta, int64_t ld, int* state,
+                             void* o, float* lse, float* partial, cudaStream_t st) {
+    const int ns = list_splits(P);
+    decode_list_attn_kernel<T, D><<<dim3(ns, P.B * P.Hq), kAttnThreads, 0, st>>>(
+        (const T*)q, (const T*)K, (const T*)V, delta, ld, state, P.w_cap, partial, P.L, P.Hq, P.G, P.scale * 1.4426950408889634f, ns,
+        P.ks[0], P.ks[1], P.ks[2], P.vs[0], P.vs[1], P.vs[2]);
+    decode_combine_kernel<T, D><<<P.B * P.Hq, 8 * D, 0, st>>>(partial, (T*)o, lse, ns, delta, ld, P.L, P.w_cap, state);
+    count_launch(2);
+    return check_launch();
+}
+
+// One decoding step with the carried state: P.L counts the cached keys INCLUDING the one appended for this step.
+int launch_decode_step(const Prob& P, const void* q, const void* K, const void* V, const float* delta, int64_t ld, int* state,
+                       void* o, float* lse, void* ws, cudaStream_t st) {
+    const size_t bh = (size_t)P.B * P.Hq;
+    auto* partial = reinterpret_cast<float*>((char*)ws + kWsHeaderBytes + ((bh * sizeof(unsigned long long) + 255) / 256) * 256 +
+                                             decode_hist_bytes(P));
+    if (P.dtype == DMA_BF16)
+        return P.d == 128 ? launch_step_typed<__nv_bfloat16, 128>(P, q, K, V, delta, ld, state, o, lse, partial, st)
+                          : launch_step_typed<__nv_bfloat16, 64>(P, q, K, V, delta, ld, state, o, lse, partial, st);
+    return P.d == 128 ? launch_step_typed<float, 128>(P, q, K, V, delta, ld, state, o, lse, partial, st)
+                      : launch_step_typed<float, 64>(P, q, K, V, delta, ld, state, o, lse, partial, st);
 }
 
 }  // namespace dma

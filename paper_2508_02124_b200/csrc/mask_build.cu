@@ -91,7 +91,8 @@ __global__ void __launch_bounds__(256) delta_kernel(const T* __restrict__ V, con
     const int sub = lane % LPR, grp = lane / LPR;
     for (int i = tid; i < G * D; i += 256) sW[i] = W[(size_t)hk * G * D + i];
     __syncthreads();
-    for (int r0 = warp * RPW; r0 < kRows; r0 += 8 * RPW) {
+    const int rows = min(kRows, L - j0);                   // a short range (one appended key) does not walk 128 row slots
+    for (int r0 = warp * RPW; r0 < rows; r0 += 8 * RPW) {
         const int r = r0 + grp, j = j0 + r;
         float v[8];
         if (j < L) {
