@@ -110,6 +110,13 @@ def test_config3_packed_documents():
     assert_close(got["dK"][:, keys], dK, case.dtype, "dK keys")
     assert_close(got["dV"][:, keys], dV, case.dtype, "dV keys")
     assert_close(got["dM"][:, :, keys], dM, case.dtype, "dM keys")
+    # the token-compacted kernels on the same packed batch, against the same oracle samples
+    _, gc = run(case, cu, flags=dma.DMA_FLAG_COMPACT_KV)
+    assert_close(gc["O"][:, rows], O, case.dtype, "compact O rows")
+    assert_close(gc["lse"][:, :, rows], lse, case.dtype, "compact lse rows", lse=True)
+    assert_close(gc["dK"][:, keys], dK, case.dtype, "compact dK keys")
+    assert_close(gc["dV"][:, keys], dV, case.dtype, "compact dV keys")
+    assert_close(gc["dM"][:, :, keys], dM, case.dtype, "compact dM keys")
 
 
 def test_argument_checks():
