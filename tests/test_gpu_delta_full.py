@@ -112,3 +112,25 @@ def test_too_many_weights_for_shared_memory_is_refused():
     with pytest.raises(dma.DmaError) as e:
         dma.dma_mask_build(p, V, W, A)
     assert e.value.status == -4
+
+
+def test_with_packed_documents_and_without_the_causal_mask():
+    """The full projection only changes delta: the packed-document and the non-causal selections on top of it stay exact."""
+    case = wl.small(wl.CONFIGS["2"], B=1, Hq=4, Hkv=2, L=900, d=128, w=100, name="full-delta modes")
+    inp = wl.make_inputs(case)
+    W = wl.full_delta_weights(case)
+    _, dl = oracle.delta_full(inp["V"].float().numpy(), W.numpy(), inp["A"].numpy())
+    V, A = inp["V"].to(DEV), inp["A"].to(DEV)
+    cu = [0, 17, 300, 301, 900]
+    p = problem_of(case, flags=FULL)
+    bias, expiry, bitmap = dma.dma_mask_build_varlen(p, V, W.to(DEV), A, torch.tensor(cu, dtype=torch.int32, device=DEV))
+    torch.cuda.synchronize()
+    e = oracle.select_expiry_varlen(dl, case.w, cu)
+    assert np.array_equal(bias.cpu().numpy().view(np.uint32), dl.view(np.uint32))
+    assert np.array_equal(expiry.cpu().numpy(), e)
+    assert np.array_equal(bitmap.cpu().numpy().view(np.uint32), oracle.bitmap_from_expiry(e))
+    pn = dma.problem(case.B, case.Hq, case.Hkv, case.L, case.d, case.w, dtype=case.torch_dtype, causal=0, flags=FULL)
+    bias, expiry, _ = dma.dma_mask_build(pn, V, W.to(DEV), A)
+    torch.cuda.synchronize()
+    assert np.array_equal(bias.cpu().numpy().view(np.uint32), dl.view(np.uint32))
+    assert np.array_equal(expiry.cpu().numpy(), oracle.select_noncausal(dl, case.w))

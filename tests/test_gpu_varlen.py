@@ -22,6 +22,8 @@ SMALL = [
     (wl.small(C2, B=2, Hq=4, Hkv=1, L=1536, w=200, backward=True, name="varlen bf16 three documents"), [0, 700, 829, 1536]),
     (wl.small(C2, B=1, Hq=2, Hkv=2, L=1024, w=64, backward=True, name="varlen bf16 tile-aligned"), [0, 256, 512, 1024]),
     (wl.small(C2, B=1, Hq=4, Hkv=4, L=512, w=64, d=64, backward=True, name="varlen bf16 d64"), [0, 77, 300, 512]),
+    (wl.small(C2, B=1, Hq=2, Hkv=1, L=700, w=1, backward=True, name="varlen bf16 w=1"), [0, 130, 131, 400, 700]),
+    (wl.small(C1, B=1, L=40, w=3, name="varlen fp32 every document one token"), list(range(41))),
 ]
 
 
