@@ -154,6 +154,26 @@ def test_full_size_configs_sampled(key):
         dq_rows_check(case, inp, got, np.array([0, 5, 130, 700, 1500]))
 
 
+def test_largest_supported_lengths():
+    """The longest sequences the tensor-core kernels take: forward at L = 131072 (1024 key tiles, the schedule's capacity),
+    tile path and token-compacted; forward + backward at L = 65536 with a group of 4 query heads per KV head (the backward's
+    step-list capacity). Sampled rows and keys against the oracle."""
+    fwd = wl.small(wl.CONFIGS["5"], B=1, Hq=4, Hkv=2, L=131072, w=4096, backward=False, name="max L forward")
+    inp = wl.make_inputs(fwd)
+    got = gpu_run(fwd, inp, backward=False)
+    sampled_check(fwd, inp, got, nrows=10, forward_only=True)
+    gc = gpu_run(fwd, inp, backward=False, flags=dma.DMA_FLAG_COMPACT_KV)
+    sampled_check(fwd, inp, gc, nrows=10, forward_only=True)
+    with pytest.raises(dma.DmaError) as e:                        # one tile more is refused, not mis-executed
+        too_long = wl.small(fwd, L=131072 + 128)
+        dma.dma_attn_fwd(problem_of(too_long), got["O"], got["O"], got["O"], got["bias"], got["expiry"], got["bitmap"])
+    assert e.value.status == -4
+    both = wl.small(wl.CONFIGS["3"], B=1, Hq=4, Hkv=1, L=65536, w=2048, backward=True, name="max L backward")
+    inp = wl.make_inputs(both)
+    got = gpu_run(both, inp)
+    sampled_check(both, inp, got, nrows=8, nkeys=4)
+
+
 def test_bounded_wait_reports_timeout_and_context_survives():
     # a wait that nothing satisfies gives up after its limit and leaves a status, instead of hanging the GPU
     dev = torch.device("cuda:0")
