@@ -47,7 +47,7 @@ enum {
     DMA_FLAG_IGNORE_BITMAP = 1,  /* visit every causal tile regardless of the bitmap (result must not change:
                                     block skipping is an optimisation only, Sec. 4.2 last paragraph)           */
     DMA_FLAG_SIMT = 2,           /* run the CUDA-core kernels also for bf16 (they always serve fp32)            */
-    DMA_FLAG_COMPACT_KV = 4,     /* dma_attn_fwd and dma_attn_bwd, bf16, d = 128, contiguous K and V: token-compacted
+    DMA_FLAG_COMPACT_KV = 4,     /* dma_attn_fwd and dma_attn_bwd, bf16, d = 128: token-compacted
                                     execution (Sec. 3.3, computational sparsity: O(L w d) instead of O(L^2 d) work).
                                     Forward: each pair of query tiles gathers only the keys that one of its 256 rows
                                     keeps (at most w + 256) instead of walking every active 128-key tile. Backward: a CTA
@@ -72,8 +72,8 @@ typedef struct {
                                     all-zero causal mask): every row sees every key, so all rows of a head keep the same
                                     min(w, L) keys; expiry[j] is then L for a kept key and 0 otherwise, key j is kept by the
                                     rows 0 <= i < expiry[j], and every bitmap row of a head is the same. bf16 with d = 128
-                                    always runs token-compacted in this mode (DMA_FLAG_COMPACT_KV is implied: contiguous K
-                                    and V, the larger workspaces); dma_mask_build_varlen needs causal = 1              */
+                                    always runs token-compacted in this mode (DMA_FLAG_COMPACT_KV is implied: the larger
+                                    workspaces); dma_mask_build_varlen needs causal = 1              */
     int32_t dtype;               /* DMA_BF16 | DMA_FP32                                                         */
     int32_t tile_m, tile_n;      /* bitmap granularity (query rows x keys per bit); 0,0 = 128,128               */
     int32_t flags;               /* DMA_FLAG_*                                                                  */

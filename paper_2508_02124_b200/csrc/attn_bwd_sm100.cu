@@ -74,7 +74,7 @@ struct BwdParams {
     const int* perm;
     const int32_t* expiry_all;
     int causal;                // 0: key j is visible to every row (token-compacted mode only): its first row is 0 instead of j
-    const __nv_bfloat16* Kg;    // K, V as contiguous [B, L, Hkv, 128] row arrays
+    const __nv_bfloat16* Kg;    // K, V base pointers for the row gathers (ks_*, vs_* strides)
     const __nv_bfloat16* Vg;
     float* dKacc;               // fp32 [B, L, Hkv, 128] accumulators (several query heads add into one KV head's rows)
     float* dVacc;
@@ -426,13 +426,14 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
 #pragma unroll 4
                 for (int q = 0; q < 32; ++q) {
                     const int r = 4 * q + rsub, j = my_perm[r];
-                    const size_t row = ((size_t)(b * P.L + min(j, P.L - 1)) * P.Hkv + hk) * 128 + c * 8;
+                    const int64_t jr = min(j, P.L - 1);
+                    const int64_t krow = b * P.ks_b + jr * P.ks_l + hk * P.ks_h + c * 8, vrow = b * P.vs_b + jr * P.vs_l + hk * P.vs_h + c * 8;
                     const uint32_t off = r * 128 + ((c ^ (r & 7)) << 4);
                     const int nb = j < P.L ? 16 : 0;
-                    cp_async16(S.k + off, P.Kg + row, nb);
-                    cp_async16(S.k + off + kKVBytes / 2, P.Kg + row + 64, nb);
-                    cp_async16(S.v + off, P.Vg + row, nb);
-                    cp_async16(S.v + off + kKVBytes / 2, P.Vg + row + 64, nb);
+                    cp_async16(S.k + off, P.Kg + krow, nb);
+                    cp_async16(S.k + off + kKVBytes / 2, P.Kg + krow + 64, nb);
+                    cp_async16(S.v + off, P.Vg + vrow, nb);
+                    cp_async16(S.v + off + kKVBytes / 2, P.Vg + vrow + 64, nb);
                 }
                 cp_async_wait_all();
                 fence_proxy_async();
@@ -684,12 +685,6 @@ int launch_tc_bwd(const Prob& P, const void* Q, const void* K, const void* V, co
     int* perm = reinterpret_cast<int*>(acc + nq);
     float* accK = reinterpret_cast<float*>(perm + bwd_perm_ints(P));
     float* accV = accK + nkv;
-    if (compact) {
-        // the gathers address K and V as plain row arrays: contiguous [B, L, Hkv, 128] only
-        const int64_t want[3] = {(int64_t)P.L * P.Hkv * P.d, (int64_t)P.Hkv * P.d, P.d};
-        for (int t = 0; t < 3; ++t)
-            if (P.ks[t] != want[t] || P.vs[t] != want[t]) return DMA_ERR_UNSUPPORTED;
-    }
     CUtensorMap tmQ, tmK, tmV, tmG;
     int rc;
     if ((rc = make_tmap_bf16(&tmQ, Q, P.B, P.L, P.Hq, P.d, P.qs, 64))) return rc;

@@ -73,11 +73,12 @@ struct FwdParams {
     // pair keeps, padded with -1 to a multiple of 128 (ccap entries per list), and its length
     const int* cidx;
     const int* ccnt;
-    const __nv_bfloat16* Kg;                   // K and V as contiguous [B, L, Hkv, 128] row arrays
+    const __nv_bfloat16* Kg;                   // K and V base pointers for the row gathers (strides below)
     const __nv_bfloat16* Vg;
     int ccap, Hkv;
     int causal;                                // 0: key j is visible to every row (token-compacted mode only)
     int64_t os_b, os_l, os_h;
+    int64_t ks_b, ks_l, ks_h, vs_b, vs_l, vs_h;
 #ifdef DMA_PROF
     long long* prof;                           // role timing (development builds only): cycles per phase of CTA (0, 0)
 #endif
@@ -405,7 +406,8 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                         tma_load_4d(&S.q[w][hf * (kTileBytes / 2)], &tmQ, &S.q_full, hf * 64, (qt0 + w) * 128, h, b);
             }
             const int* list = P.cidx + ((size_t)bh * npairs + pair) * P.ccap;
-            const __nv_bfloat16* src = (isK ? P.Kg : P.Vg) + (size_t)hk * 128 + (lane & 7) * 8;
+            const int64_t row_stride = isK ? P.ks_l : P.vs_l;
+            const __nv_bfloat16* src = (isK ? P.Kg + b * P.ks_b + hk * P.ks_h : P.Vg + b * P.vs_b + hk * P.vs_h) + (lane & 7) * 8;
             const int rsub = lane >> 3;
             const uint32_t sw0 = (uint32_t)(((lane & 7) ^ rsub) << 4), sw1 = (uint32_t)(((lane & 7) ^ (rsub + 4)) << 4);
             int jrow[32];
@@ -424,7 +426,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
 #pragma unroll
                 for (int q = 0; q < 32; ++q) {
                     const int j = jrow[q];
-                    const __nv_bfloat16* row = src + (size_t)(b * P.L + max(j, 0)) * P.Hkv * 128;
+                    const __nv_bfloat16* row = src + (int64_t)max(j, 0) * row_stride;
                     uint8_t* d = dst + q * 512 + ((q & 1) ? sw1 : sw0);          // row r = 4q + rsub, chunk c ^ (r & 7)
                     cp_async16(d, row, j >= 0 ? 16 : 0);
                     cp_async16(d + kTileBytes / 2, row + 64, j >= 0 ? 16 : 0);
@@ -912,10 +914,6 @@ int launch_tc_fwd(const Prob& P, const void* Q, const void* K, const void* V, co
     fp.cidx = nullptr; fp.ccnt = nullptr; fp.ccap = 0; fp.Hkv = P.Hkv; fp.causal = P.causal;
     if (!P.causal && !compact) return DMA_ERR_UNSUPPORTED;
     if (compact) {
-        // the gathers address K and V as plain row arrays: contiguous [B, L, Hkv, 128] only
-        const int64_t want[3] = {(int64_t)P.L * P.Hkv * P.d, (int64_t)P.Hkv * P.d, P.d};
-        for (int t = 0; t < 3; ++t)
-            if (P.ks[t] != want[t] || P.vs[t] != want[t]) return DMA_ERR_UNSUPPORTED;
         if (compact_cap(P) / 128 > kMaxSched) return DMA_ERR_UNSUPPORTED;
         const size_t nl = compact_lists(P);
         int* ccnt = reinterpret_cast<int*>((char*)ws + kWsHeaderBytes);
@@ -935,6 +933,7 @@ int launch_tc_fwd(const Prob& P, const void* Q, const void* K, const void* V, co
     fp.inv_scale = 1.0f / P.scale;
     fp.rescale_gap = kRescaleThreshold / fp.scale_log2;
     fp.os_b = P.os[0]; fp.os_l = P.os[1]; fp.os_h = P.os[2];
+    fp.ks_b = P.ks[0]; fp.ks_l = P.ks[1]; fp.ks_h = P.ks[2]; fp.vs_b = P.vs[0]; fp.vs_l = P.vs[1]; fp.vs_h = P.vs[2];
 #ifdef DMA_PROF
     const char* prof_env = getenv("DMA_PROF_PTR");
     fp.prof = prof_env ? (long long*)strtoull(prof_env, nullptr, 10) : nullptr;

@@ -31,11 +31,10 @@ struct Layout {
 };
 
 // Head groups per batch entry: up to 4, a divisor of Hkv, and only where every per-group pointer stays 16-byte aligned,
-// the group is independent (the full sampling weights read all KV heads; the token-compacted kernels want contiguous
-// K and V) and a group's K / V rows are at least 512 bytes wide (measured at L = 16384, 32 / 8 heads: 4 groups of
+// the group is independent (the full sampling weights read all KV heads) and a group's K / V rows are at least 512 bytes wide (measured at L = 16384, 32 / 8 heads: 4 groups of
 // 512-byte rows 10.2 ms per step, 8 groups of 256-byte rows 14.6 ms, one group 14.8 ms: short rows slow the copies down).
 int pick_head_groups(const Prob& P) {
-    if (P.flags & (DMA_FLAG_FULL_DELTA | DMA_FLAG_COMPACT_KV)) return 1;
+    if (P.flags & DMA_FLAG_FULL_DELTA) return 1;
     const size_t esz = P.dtype == DMA_BF16 ? 2 : 4;
     for (int g = 4; g > 1; --g) {
         if (P.Hkv % g || (size_t)(P.Hkv / g) * P.d * esz < 512) continue;

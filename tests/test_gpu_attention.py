@@ -237,6 +237,37 @@ def test_compact_flag_is_rejected_where_unsupported():
     assert e.value.status == -4
 
 
+def test_compact_kernels_on_strided_k_and_v():
+    """K and V living inside larger buffers (spare sequence capacity, extra heads between the used ones): the gathers follow
+    the descriptor's strides; results equal those on packed copies of the same data."""
+    dev = torch.device("cuda:0")
+    case = wl.small(C2, B=2, Hq=4, Hkv=2, L=700, w=96, backward=True, name="compact-strided")
+    inp = wl.make_inputs(case)
+    ref = gpu_run(case, inp, flags=dma.DMA_FLAG_COMPACT_KV)
+    B, L, Hkv, d = case.B, case.L, case.Hkv, case.d
+    cap, Hbig = L + 52, 2 * Hkv + 1
+    bigK = torch.randn(B, cap, Hbig, d).to(case.torch_dtype).to(dev)
+    bigV = torch.randn(B, cap, Hbig, d).to(case.torch_dtype).to(dev)
+    Kv, Vv = bigK[:, :L, 1:1 + 2 * Hkv:2], bigV[:, :L, 1:1 + 2 * Hkv:2]          # every other head, starting at head 1
+    Kv.copy_(inp["K"].to(dev)); Vv.copy_(inp["V"].to(dev))
+    p = problem_of(case, flags=dma.DMA_FLAG_COMPACT_KV)
+    for sdst, t in ((p.k_stride, Kv), (p.v_stride, Vv)):
+        sdst[0], sdst[1], sdst[2] = t.stride(0), t.stride(1), t.stride(2)
+    Q, dO = inp["Q"].to(dev), inp["dO"].to(dev)
+    O, lse = dma.dma_attn_fwd(p, Q, Kv, Vv, ref["bias"], ref["expiry"], ref["bitmap"])
+    dK, dV = torch.zeros_like(bigK), torch.zeros_like(bigV)
+    dKv, dVv = dK[:, :L, 1:1 + 2 * Hkv:2], dV[:, :L, 1:1 + 2 * Hkv:2]
+    dQ, _, _, dM = dma.dma_attn_bwd(p, Q, Kv, Vv, O, dO, lse, ref["bias"], ref["expiry"], ref["bitmap"], dK=dKv, dV=dVv)
+    torch.cuda.synchronize()
+    assert torch.equal(O, ref["O"]) and torch.equal(lse, ref["lse"])
+    assert_close(dKv, f64(ref["dK"]), case.dtype, "dK (strided)")
+    assert_close(dVv, f64(ref["dV"]), case.dtype, "dV (strided)")
+    assert_close(dQ, f64(ref["dQ"]), case.dtype, "dQ (strided)")
+    assert_close(dM, f64(ref["dM"]), case.dtype, "dM (strided)")
+    untouched = torch.ones(Hbig, dtype=torch.bool); untouched[1:1 + 2 * Hkv:2] = False
+    assert float(dK[:, :, untouched].abs().max()) == 0.0 and float(dK[:, L:].abs().max()) == 0.0
+
+
 # ---- token-compacted backward (DMA_FLAG_COMPACT_KV): key tiles follow a lifetime-sorted permutation per query head -----
 
 def _compact_full_run(case, inp):
