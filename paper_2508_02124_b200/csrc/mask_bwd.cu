@@ -174,8 +174,10 @@ __global__ void __launch_bounds__((D == 128 ? 4 : 8) * (D + 1)) mask_bwd_reduce_
 //   3  dW partial [h][col] = sum_rows dz v: a thread owns a column and walks the rows (no cross-thread sums)
 //   4  the value tile is overwritten by sum_h dz W[h][col], then added to dV
 // partial [B * blocks][Hq][C + 1]; mask_bwd_full_reduce_kernel adds them in a fixed order.
+constexpr int kFullThreads = 512;     // 16 warps: the kernel is bound by instruction issue and latency, not by registers
+
 template <typename T, int RW>
-__global__ void __launch_bounds__(kThreads) mask_bwd_full_kernel(const T* __restrict__ V, const float* __restrict__ W,
+__global__ void __launch_bounds__(kFullThreads) mask_bwd_full_kernel(const T* __restrict__ V, const float* __restrict__ W,
                                                                  const float* __restrict__ A, const float* __restrict__ delta,
                                                                  const float* __restrict__ dM, T* __restrict__ dV,
                                                                  float* __restrict__ partial, int L, int Hq, int Hkv, int D,
@@ -190,7 +192,7 @@ __global__ void __launch_bounds__(kThreads) mask_bwd_full_kernel(const T* __rest
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int C8 = C / 8, D8 = D / 8;
 
-    for (int i = tid; i < R * C8; i += kThreads) {
+    for (int i = tid; i < R * C8; i += kFullThreads) {
         const int row = i / C8, ch = i % C8, j = j0 + row;
         float v[8];
         if (j < L) {
@@ -201,15 +203,15 @@ __global__ void __launch_bounds__(kThreads) mask_bwd_full_kernel(const T* __rest
         }
         store8f(sV + (size_t)row * C + ch * 8, v);
     }
-    for (int i = tid; i < R * HqP; i += kThreads) sDz[i] = 0.0f;
+    for (int i = tid; i < R * HqP; i += kFullThreads) sDz[i] = 0.0f;
     __syncthreads();
 
     // z: a warp owns HB heads at a time and all R rows; lanes stride the channels, so W is read once per CTA and each
     // value feeds HB fmas. The per-lane sums are added across lanes by a transposing butterfly (a lane keeps half of
     // its rows at each step), which leaves row (lane mod RL) of every head in the lane.
-    constexpr int HB = 128 / R < 16 ? 128 / R : 16;
+    constexpr int HB = 64 / R > 1 ? 64 / R : 1;     // 64 accumulators per thread
     constexpr int RL = R < 32 ? R : 32;            // rows reduced together
-    for (int h0 = warp * HB; h0 < Hq; h0 += 8 * HB) {
+    for (int h0 = warp * HB; h0 < Hq; h0 += (kFullThreads / 32) * HB) {
         float acc[HB][R];
 #pragma unroll
         for (int q = 0; q < HB; ++q)
@@ -248,7 +250,7 @@ __global__ void __launch_bounds__(kThreads) mask_bwd_full_kernel(const T* __rest
     }
     __syncthreads();
 
-    for (int i = tid; i < Hq * R; i += kThreads) {
+    for (int i = tid; i < Hq * R; i += kFullThreads) {
         const int h = i / R, row = i % R, j = j0 + row;
         float dz = 0.0f, gs = 0.0f;
         if (j < L) {
@@ -265,7 +267,7 @@ __global__ void __launch_bounds__(kThreads) mask_bwd_full_kernel(const T* __rest
     __syncthreads();
 
     float* out = partial + ((size_t)b * gridDim.x + blockIdx.x) * Hq * (C + 1);
-    for (int col = tid; col < C; col += kThreads) {
+    for (int col = tid; col < C; col += kFullThreads) {
         for (int hc = 0; hc < HqP; hc += 8) {
             float acc[8];
 #pragma unroll
@@ -289,7 +291,7 @@ __global__ void __launch_bounds__(kThreads) mask_bwd_full_kernel(const T* __rest
     }
     __syncthreads();   // every thread is done with the values of its columns' neighbours: the tile may be overwritten
 
-    for (int col = tid; col < C; col += kThreads) {
+    for (int col = tid; col < C; col += kFullThreads) {
         for (int hc = 0; hc < HqP; hc += 8) {
             float w[8];
 #pragma unroll
@@ -307,7 +309,7 @@ __global__ void __launch_bounds__(kThreads) mask_bwd_full_kernel(const T* __rest
     }
     __syncthreads();
 
-    for (int i = tid; i < R * C8; i += kThreads) {
+    for (int i = tid; i < R * C8; i += kFullThreads) {
         const int row = i / C8, ch = i % C8, j = j0 + row;
         if (j < L) {
             T* p = dV + b * vs_b + (int64_t)j * vs_l + (ch / D8) * vs_h + (ch % D8) * 8;
@@ -378,7 +380,7 @@ static int launch_full(const Prob& P, const void* V, const float* W, const float
     const size_t smem = ((size_t)R * C + (size_t)R * HqP + (size_t)P.Hq * R) * sizeof(float);
     if (cudaFuncSetAttribute(mask_bwd_full_kernel<T, RW>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return DMA_ERR_CUDA;
-    mask_bwd_full_kernel<T, RW><<<dim3(nblk, P.B), kThreads, smem, st>>>((const T*)V, W, A, delta, dM, (T*)dV, (float*)ws, P.L, P.Hq,
+    mask_bwd_full_kernel<T, RW><<<dim3(nblk, P.B), kFullThreads, smem, st>>>((const T*)V, W, A, delta, dM, (T*)dV, (float*)ws, P.L, P.Hq,
                                                                           P.Hkv, P.d, P.vs[0], P.vs[1], P.vs[2]);
     mask_bwd_full_reduce_kernel<<<dim3((C + 1 + 127) / 128, P.Hq), 512, 0, st>>>((const float*)ws, dW, dA, P.B * nblk, P.Hq, C);
     count_launch(2);
