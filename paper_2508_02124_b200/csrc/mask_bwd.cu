@@ -79,26 +79,48 @@ __global__ void __launch_bounds__(kThreads) mask_bwd_kernel(const T* __restrict_
 #pragma unroll
         for (int c = 0; c < 8; ++c) upd[n][c] = 0.0f;
     }
+    // z of every (row, head) pair of the lane group, then softplus / sigmoid ONCE per pair (the LPR lanes of a group would
+    // all repeat the same forty instructions): lane `sub` takes the pairs sub, sub + LPR, ... and leaves dz and
+    // dM delta softplus(z) in shared memory for the whole group
+    float* sDz = sGD + G * kRows;                     // [8 warps][RPW][NR * G]
+    float* sGs = sDz + 8 * RPW * NR * G;              // same shape
+    float* myDz = sDz + (warp * RPW + grp) * NR * G;
+    float* myGs = sGs + (warp * RPW + grp) * NR * G;
     for (int g = 0; g < G; ++g) {
-        const int h = hk * G + g;
-        const float a = A[h];
-        float w[8], pw[8], pa = 0.0f;
+        float w[8];
 #pragma unroll
-        for (int c = 0; c < 8; ++c) { w[c] = sW[g * D + sub * 8 + c]; pw[c] = 0.0f; }
+        for (int c = 0; c < 8; ++c) w[c] = sW[g * D + sub * 8 + c];
 #pragma unroll
         for (int n = 0; n < NR; ++n) {
-            const int j = j0 + warp * RPW + n * 8 * RPW + grp;
             float z = 0.0f;
 #pragma unroll
             for (int c = 0; c < 8; ++c) z = fmaf(v[n][c], w[c], z);
 #pragma unroll
             for (int m = 1; m < LPR; m <<= 1) z += __shfl_xor_sync(0xffffffffu, z, m);
-            const float gd = sGD[g * kRows + (j - j0)];
-            const float e = __expf(-fabsf(z));                       // in (0, 1]
-            const float sp = fmaxf(z, 0.0f) + log1pf(e);
-            const float sig = (z >= 0.0f ? 1.0f : e) / (1.0f + e);
-            const float dz = gd * a * sig;
-            if (sub == 0) pa += gd * sp;
+            if (sub == 0) myDz[n * G + g] = z;
+        }
+    }
+    __syncwarp();
+    for (int pr = sub; pr < NR * G; pr += LPR) {
+        const int n = pr / G, g = pr % G;
+        const int j = j0 + warp * RPW + n * 8 * RPW + grp;
+        const float z = myDz[pr];
+        const float gd = sGD[g * kRows + (j - j0)];
+        const float e = __expf(-fabsf(z));                       // in (0, 1]
+        const float sp = fmaxf(z, 0.0f) + log1pf(e);
+        const float sig = (z >= 0.0f ? 1.0f : e) / (1.0f + e);
+        myDz[pr] = gd * A[hk * G + g] * sig;
+        myGs[pr] = gd * sp;
+    }
+    __syncwarp();
+    for (int g = 0; g < G; ++g) {
+        float w[8], pw[8], pa = 0.0f;
+#pragma unroll
+        for (int c = 0; c < 8; ++c) { w[c] = sW[g * D + sub * 8 + c]; pw[c] = 0.0f; }
+#pragma unroll
+        for (int n = 0; n < NR; ++n) {
+            const float dz = myDz[n * G + g];
+            if (sub == 0) pa += myGs[n * G + g];
 #pragma unroll
             for (int c = 0; c < 8; ++c) {
                 pw[c] = fmaf(dz, v[n][c], pw[c]);
@@ -363,7 +385,7 @@ template <typename T, int D>
 static int launch_typed(const Prob& P, const void* V, const float* W, const float* A, const float* delta, const float* dM,
                         void* dV, float* dW, float* dA, void* ws, cudaStream_t st) {
     const int nblk = (P.L + kRows - 1) / kRows;
-    const size_t smem = (size_t)P.G * (D + 8 * (D + 1) + kRows) * sizeof(float);
+    const size_t smem = (size_t)P.G * (D + 8 * (D + 1) + 3 * kRows) * sizeof(float);
     if (cudaFuncSetAttribute(mask_bwd_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return DMA_ERR_CUDA;
     mask_bwd_kernel<T, D><<<dim3(nblk, P.Hkv, P.B), kThreads, smem, st>>>((const T*)V, W, A, delta, dM, (T*)dV, (float*)ws, P.L, P.Hq,
                                                                             P.G, P.vs[0], P.vs[1], P.vs[2]);
