@@ -108,13 +108,13 @@ __global__ void __launch_bounds__(256) delta_kernel(const T* __restrict__ V, con
             for (int c = 0; c < 8; ++c) p = __fmaf_rn(v[c], w[c], p);
 #pragma unroll
             for (int m = 1; m < LPR; m <<= 1) p = __fadd_rn(p, __shfl_xor_sync(0xffffffffu, p, m));
-            if (sub == g % LPR) sOut[g * kRows + r] = delta_fixed(p, A[hk * G + g]);
+            if (sub == g % LPR) sOut[g * kRows + r] = p;      // z; softplus and exp follow, one (row, head) pair per thread
         }
     }
     __syncthreads();
     for (int i = tid; i < G * kRows; i += 256) {
         const int g = i / kRows, r = i % kRows;
-        if (j0 + r < L) delta[((size_t)b * Hq + hk * G + g) * ld + j0 + r] = sOut[i];
+        if (j0 + r < L) delta[((size_t)b * Hq + hk * G + g) * ld + j0 + r] = delta_fixed(sOut[i], A[hk * G + g]);
     }
 }
 
