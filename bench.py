@@ -367,6 +367,28 @@ def main():
         noncausal = {"mask_ms": n_ms[0], "fwd_ms": n_ms[1], "bwd_ms": n_ms[2] if case.backward else None, "step_ms": sum(n_ms),
                      "kept_keys_per_head": keep, "tflops_kept_pairs": pair_flops / (sum(n_ms) * 1e-3) / 1e12}
 
+    # ---- prefill in pieces: the last 2048 rows of the sequence against all its keys (dma_attn_fwd_chunk), timed on its own
+    chunk = None
+    if case.dtype == "bf16" and case.d == 128 and case.L >= 4096 and not (args.flags & dma.DMA_FLAG_SIMT):
+        q_len = 2048
+        q_begin = case.L - q_len
+        Qc = Q[:, q_begin:].contiguous()
+        Oc2, lsec2 = torch.empty_like(Qc), torch.empty(case.B, case.Hq, q_len, dtype=torch.float32, device=dev)
+        pcc = dma.problem(case.B, case.Hq, case.Hkv, case.L, case.d, case.w, dtype=case.torch_dtype, flags=args.flags | dma.DMA_FLAG_COMPACT_KV)
+        ws_ch = torch.empty(dma.dma_query_workspace(pcc)[1], dtype=torch.uint8, device=dev)
+        for _ in range(3):
+            dma.dma_attn_fwd_chunk(p, q_begin, Qc, K, V, bias, expiry, Oc2, lsec2, ws_ch)
+        g0, g1 = ev(), ev()
+        barrier()
+        g0.record()
+        for _ in range(10):
+            dma.dma_attn_fwd_chunk(p, q_begin, Qc, K, V, bias, expiry, Oc2, lsec2, ws_ch)
+        g1.record()
+        barrier()
+        ch_ms = g0.elapsed_time(g1) / 10
+        chunk = {"q_begin": q_begin, "q_len": q_len, "ms": ch_ms,
+                 "max_abs_diff_vs_full_forward": float((Oc2.float() - O[:, q_begin:].float()).abs().max())}
+
     # ---- one decoding step over this workload's K / V as the cache (dma_delta_range + dma_decode), timed on its own
     decode = None
     if rank == 0:
@@ -510,6 +532,8 @@ def main():
         out["varlen"] = varlen
     if noncausal is not None:
         out["noncausal"] = noncausal
+    if chunk is not None:
+        out["fwd_chunk"] = chunk
     if mask_bwd is not None:
         mask_bwd["frac_of_measured_hbm"] = mask_bwd["gbs"] / pk["hbm_gbs"]
         out["mask_bwd"] = mask_bwd

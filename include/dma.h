@@ -144,6 +144,16 @@ int dma_attn_fwd(const dma_problem_t* p, const void* Q, const void* K, const voi
                  const float* bias, const int32_t* expiry, const uint32_t* bitmap,
                  void* O, float* lse, void* ws, size_t ws_bytes, void* cuda_stream);
 
+/* Forward for a chunk of query rows (prefill in pieces over a KV cache; the same computation as dma_attn_fwd restricted
+ * to the rows q_begin <= i < q_begin + q_len of the sequence of p->L keys, bottom-right aligned when q_begin + q_len = L):
+ * Q and O are [B, q_len, Hq, d] (q_stride / o_stride, all 0 = packed with q_len rows), lse is [B, Hq, q_len]; K, V, bias
+ * and expiry are those of the whole sequence (the mask built over all p->L keys). q_begin and q_len need no alignment.
+ * bf16 with d = 128 runs the token-compacted kernel (its workspace size: dma_query_workspace with DMA_FLAG_COMPACT_KV set);
+ * the other cases run the CUDA-core kernel. No bitmap is needed. */
+int dma_attn_fwd_chunk(const dma_problem_t* p, int32_t q_begin, int32_t q_len, const void* Q, const void* K, const void* V,
+                       const float* bias, const int32_t* expiry, void* O, float* lse, void* ws, size_t ws_bytes,
+                       void* cuda_stream);
+
 /* Backward (Sec. 4.3, Alg. 2, Eqs. (grad_v), (grad_s), (grad_m), (grad_qk)), mask and bias values held fixed:
  *   D_i = dO_i . O_i;  p_ij = exp(s_ij - lse_i);  dP_ij = dO_i . v_j;  dS_ij = p_ij (dP_ij - D_i)
  *   dV_j = sum_i p_ij dO_i;  dK_j = scale sum_i dS_ij q_i;  dQ_i = scale sum_j dS_ij k_j;  dM[b,h,j] = sum_i dS_ij

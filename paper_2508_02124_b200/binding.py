@@ -19,7 +19,8 @@ DMA_FLAG_IGNORE_BITMAP, DMA_FLAG_SIMT, DMA_FLAG_COMPACT_KV, DMA_FLAG_FULL_DELTA 
 ENTRY_POINTS = ("dma_query_workspace", "dma_bitmap_words", "dma_mask_build", "dma_attn_fwd", "dma_attn_bwd",
                 "dma_read_status", "dma_launch_count", "dma_strerror", "dma_step_host_arena", "dma_step_host", "dma_mask_build_static", "dma_selftest_wait_timeout",
                 "dma_mask_bwd_workspace", "dma_mask_bwd", "dma_delta_range", "dma_decode_workspace", "dma_decode",
-                "dma_mask_build_varlen", "dma_decode_state_bytes", "dma_decode_state_init", "dma_decode_step")
+                "dma_mask_build_varlen", "dma_decode_state_bytes", "dma_decode_state_init", "dma_decode_step",
+                "dma_attn_fwd_chunk")
 
 
 class DmaError(RuntimeError):
@@ -226,6 +227,23 @@ def dma_attn_fwd(p, Q, K, V, bias, expiry, bitmap, O=None, lse=None, ws=None):
         ws = _ws(dma_query_workspace(p)[1], Q.device)
     _check(lib().dma_attn_fwd(ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(bias), _ptr(expiry), _ptr(bitmap), _ptr(O),
                               _ptr(lse), _ptr(ws), ctypes.c_size_t(ws.numel()), _stream()), "dma_attn_fwd")
+    return O, lse
+
+
+def dma_attn_fwd_chunk(p, q_begin, Q, K, V, bias, expiry, O=None, lse=None, ws=None):
+    """Forward for the query rows q_begin .. q_begin + Q.shape[1] - 1 of a sequence of p.L keys; returns (O like Q, lse [B,Hq,q_len])."""
+    q_len = Q.shape[1]
+    if O is None:
+        O = torch.empty_like(Q)
+    if lse is None:
+        lse = torch.empty(p.B, p.Hq, q_len, dtype=torch.float32, device=Q.device)
+    if ws is None:
+        pc = dma_problem_t.from_buffer_copy(bytes(p))
+        pc.flags |= DMA_FLAG_COMPACT_KV
+        ws = _ws(dma_query_workspace(pc)[1], Q.device)
+    _check(lib().dma_attn_fwd_chunk(ctypes.byref(p), ctypes.c_int32(q_begin), ctypes.c_int32(q_len), _ptr(Q), _ptr(K), _ptr(V),
+                                    _ptr(bias), _ptr(expiry), _ptr(O), _ptr(lse), _ptr(ws), ctypes.c_size_t(ws.numel()), _stream()),
+           "dma_attn_fwd_chunk")
     return O, lse
 
 

@@ -34,6 +34,7 @@ int resolve(const dma_problem_t* p, Prob* o) {
     o->B = p->B; o->Hq = p->Hq; o->Hkv = p->Hkv; o->L = p->L; o->d = p->d; o->G = p->Hq / p->Hkv;
     o->w = p->w < p->L ? p->w : p->L;
     o->w_cap = p->w;
+    o->Lq = p->L; o->q_off = 0;
     o->dtype = p->dtype; o->flags = p->flags; o->causal = p->causal;
     o->bm = p->tile_m ? p->tile_m : 128;
     o->bn = p->tile_n ? p->tile_n : 128;
@@ -243,6 +244,36 @@ int dma_attn_fwd(const dma_problem_t* p, const void* Q, const void* K, const voi
     if (cudaMemsetAsync(ws, 0, kWsHeaderBytes, st) != cudaSuccess) return DMA_ERR_CUDA;
     if (tc) return launch_tc_fwd(P, Q, K, V, bias, expiry, bitmap, O, lse, ws, st);
     return launch_simt_fwd(P, Q, K, V, bias, expiry, bitmap, O, lse, st);
+}
+
+int dma_attn_fwd_chunk(const dma_problem_t* p, int32_t q_begin, int32_t q_len, const void* Q, const void* K, const void* V,
+                       const float* bias, const int32_t* expiry, void* O, float* lse, void* ws, size_t ws_bytes,
+                       void* cuda_stream) {
+    Prob P;
+    int rc = resolve(p, &P);
+    if (rc) return rc;
+    if (!Q || !K || !V || !bias || !expiry || !O || !lse) return DMA_ERR_NULL;
+    if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || !aligned16(bias) || !aligned16(expiry) ||
+        !aligned16(lse))
+        return DMA_ERR_ALIGN;
+    if (q_begin < 0 || q_len < 1 || (int64_t)q_begin + q_len > P.L) return DMA_ERR_SHAPE;
+    P.Lq = q_len; P.q_off = q_begin;
+    bool q_default = true, o_default = true;
+    for (int t = 0; t < 3; ++t) { q_default = q_default && p->q_stride[t] == 0; o_default = o_default && p->o_stride[t] == 0; }
+    const int64_t packed[3] = {(int64_t)q_len * P.Hq * P.d, (int64_t)P.Hq * P.d, P.d};     // [B, q_len, Hq, d]
+    for (int t = 0; t < 3; ++t) {
+        if (q_default) P.qs[t] = packed[t];
+        if (o_default) P.os[t] = packed[t];
+    }
+    const bool tc = use_tensor_cores(P);
+    if (tc) P.flags |= DMA_FLAG_COMPACT_KV;            // the gathered-key kernel has no tile alignment between rows and keys
+    const size_t need = tc ? tc_fwd_ws_bytes(P) : (size_t)kWsHeaderBytes;
+    if (!ws || ws_bytes < need || !aligned16(ws)) return DMA_ERR_WORKSPACE;
+    if ((rc = device_ok())) return rc;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    if (cudaMemsetAsync(ws, 0, kWsHeaderBytes, st) != cudaSuccess) return DMA_ERR_CUDA;
+    if (tc) return launch_tc_fwd(P, Q, K, V, bias, expiry, nullptr, O, lse, ws, st);
+    return launch_simt_fwd(P, Q, K, V, bias, expiry, nullptr, O, lse, st);
 }
 
 int dma_attn_bwd(const dma_problem_t* p, const void* Q, const void* K, const void* V, const void* O, const void* dO,

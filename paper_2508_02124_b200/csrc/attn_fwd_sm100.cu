@@ -77,6 +77,7 @@ struct FwdParams {
     const __nv_bfloat16* Vg;
     int ccap, Hkv;
     int causal;                                // 0: key j is visible to every row (token-compacted mode only)
+    int Lq, q_off, Trq;                        // chunk of query rows (token-compacted mode only): Q, O, lse hold rows q_off .. q_off + Lq - 1; Trq = its 128-row tiles
     int64_t os_b, os_l, os_h;
     int64_t ks_b, ks_l, ks_h, vs_b, vs_l, vs_h;
 #ifdef DMA_PROF
@@ -110,10 +111,10 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
     const int tid = threadIdx.x, lane = tid & 31;
     const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);      // warp-uniform to the compiler: role branches stay uniform
     const int bh = blockIdx.x, b = bh / P.Hq, h = bh % P.Hq, hk = h / P.G;
-    const int npairs = (P.Tr + 1) / 2;
+    const int npairs = (P.Trq + 1) / 2;
     const int pair = npairs - 1 - (int)blockIdx.y;          // heaviest query tiles first
-    const int qt0 = 2 * pair, qt1 = 2 * pair + 1;
-    const bool has1 = qt1 < P.Tr;
+    const int qt0 = 2 * pair, qt1 = 2 * pair + 1;           // query tiles inside the chunk (the whole sequence unless P.q_off / P.Lq say otherwise)
+    const bool has1 = qt1 < P.Trq;
     volatile int* abort_flag = &S.abort_flag;
 
     if (tid == 0) {
@@ -174,7 +175,8 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
         const int w = warp >> 2;
         const int r = tid & 127;
         const int qt = w ? qt1 : qt0;
-        const int i = qt * 128 + r;
+        const int il = qt * 128 + r;                        // row inside Q, O, lse
+        const int i = P.q_off + il;                         // its position in the sequence
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
         const uint32_t tS = tmem + lane_base + w * 128;
         const uint32_t tO = tmem + lane_base + 256 + w * 128;
@@ -366,7 +368,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
         if (ok && exists) {
             tc_fence_after();
             const float inv = l > 0.0f ? 1.0f / l : 0.0f;
-            __nv_bfloat16* orow = P.O + b * P.os_b + (int64_t)i * P.os_l + h * P.os_h;
+            __nv_bfloat16* orow = P.O + b * P.os_b + (int64_t)il * P.os_l + h * P.os_h;
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
                 uint32_t o[32];
@@ -377,7 +379,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
 #pragma unroll
                     for (int u = 0; u < 32; ++u) o[u] = 0;
                 }
-                if (i < P.L) {
+                if (il < P.Lq) {
 #pragma unroll
                     for (int u = 0; u < 32; u += 8) {
                         uint4 pkt;
@@ -389,7 +391,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                     }
                 }
             }
-            if (i < P.L) P.lse[(size_t)bh * P.L + i] = l > 0.0f ? 0.6931471805599453f * ((m_ref * P.scale_log2 - r_ref) + log2f(l)) : -INFINITY;
+            if (il < P.Lq) P.lse[(size_t)bh * P.Lq + il] = l > 0.0f ? 0.6931471805599453f * ((m_ref * P.scale_log2 - r_ref) + log2f(l)) : -INFINITY;
         }
     } else {
         setmaxnreg_dec<88>();   // 4 warps x 80 registers released = 8 warps x 40 acquired above
@@ -497,7 +499,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                     b1[t] = (uint32_t)__bfloat16_as_ushort(lo);
 #pragma unroll
                     for (int w = 0; w < 2; ++w) {
-                        const int i0 = (w ? qt1 : qt0) * 128;
+                        const int i0 = P.q_off + (w ? qt1 : qt0) * 128;
                         const int first = P.causal ? jv[t] : 0;             // first row that can see the key
                         const bool dead = jv[t] < 0 || ev[t] <= i0 || first > i0 + 127;
                         const bool mixed = !dead && (ev[t] < i0 + 128 || first > i0);
@@ -864,10 +866,11 @@ int make_tmap_f32_rows(CUtensorMap* m, const void* base, int B, int L, int H, in
 // At most w + 256 keys qualify. One CTA of 256 threads per list: 256 keys per pass, ballots and per-warp counts keep the
 // order; the list is padded with -1 to the next multiple of 128.
 __global__ void __launch_bounds__(256) compact_lists_kernel(const int32_t* __restrict__ expiry, int* __restrict__ cidx,
-                                                            int* __restrict__ ccnt, int L, int npairs, int cap, int causal) {
+                                                            int* __restrict__ ccnt, int L, int npairs, int cap, int causal,
+                                                            int q_off) {
     __shared__ int wsum[2][8];
     const int list = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int bh = list / npairs, pair = list % npairs, i0 = pair * 256;
+    const int bh = list / npairs, pair = list % npairs, i0 = q_off + pair * 256;
     const int32_t* e = expiry + (size_t)bh * L;
     int* out = cidx + (size_t)list * cap;
     const int jend = causal ? min(L, i0 + 256) : L;     // non-causal: key j is kept by the rows i < expiry[j], whatever j
@@ -909,16 +912,19 @@ int launch_tc_fwd(const Prob& P, const void* Q, const void* K, const void* V, co
     if (P.Tc > kMaxSched) return DMA_ERR_UNSUPPORTED;
     CUtensorMap tmQ, tmK, tmV;
     int rc;
-    if ((rc = make_tmap_bf16(&tmQ, Q, P.B, P.L, P.Hq, P.d, P.qs, 128))) return rc;
+    const int Trq = (P.Lq + 127) / 128, npairs = (Trq + 1) / 2;
+    if ((P.Lq != P.L || P.q_off != 0) && !compact) return DMA_ERR_UNSUPPORTED;
+    if ((rc = make_tmap_bf16(&tmQ, Q, P.B, P.Lq, P.Hq, P.d, P.qs, 128))) return rc;
     FwdParams fp;
     fp.cidx = nullptr; fp.ccnt = nullptr; fp.ccap = 0; fp.Hkv = P.Hkv; fp.causal = P.causal;
+    fp.Lq = P.Lq; fp.q_off = P.q_off; fp.Trq = Trq;
     if (!P.causal && !compact) return DMA_ERR_UNSUPPORTED;
     if (compact) {
         if (compact_cap(P) / 128 > kMaxSched) return DMA_ERR_UNSUPPORTED;
-        const size_t nl = compact_lists(P);
+        const size_t nl = (size_t)P.B * P.Hq * npairs;
         int* ccnt = reinterpret_cast<int*>((char*)ws + kWsHeaderBytes);
         int* cidx = reinterpret_cast<int*>((char*)ws + kWsHeaderBytes + ((nl * sizeof(int) + 255) / 256) * 256);
-        compact_lists_kernel<<<(unsigned)nl, 256, 0, st>>>(expiry, cidx, ccnt, P.L, (P.Tr + 1) / 2, compact_cap(P), P.causal);
+        compact_lists_kernel<<<(unsigned)nl, 256, 0, st>>>(expiry, cidx, ccnt, P.L, npairs, compact_cap(P), P.causal, P.q_off);
         count_launch();
         fp.cidx = cidx; fp.ccnt = ccnt; fp.ccap = compact_cap(P);
     }
@@ -939,7 +945,7 @@ int launch_tc_fwd(const Prob& P, const void* Q, const void* K, const void* V, co
     fp.prof = prof_env ? (long long*)strtoull(prof_env, nullptr, 10) : nullptr;
 #endif
     const size_t smem = sizeof(SharedStorage) + 1024;
-    dim3 grid(P.B * P.Hq, (P.Tr + 1) / 2);
+    dim3 grid(P.B * P.Hq, npairs);
     if (compact) {
         if (cudaFuncSetAttribute(fwd_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return DMA_ERR_CUDA;
         fwd_kernel<true><<<grid, kThreads, smem, st>>>(tmQ, tmK, tmV, fp);

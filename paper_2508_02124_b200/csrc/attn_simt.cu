@@ -39,13 +39,14 @@ __global__ void __launch_bounds__(NT) simt_fwd_kernel(const T* __restrict__ Q, c
     int* sE = reinterpret_cast<int*>(sB + BN);   // expiry of the tile [BN]
 
     const int qt = blockIdx.x, h = blockIdx.y, b = blockIdx.z, hk = h / P.G, bh = b * P.Hq + h;
-    const int i0 = qt * BM, L = P.L;
+    const int i0 = qt * BM, L = P.L;                 // i0: first row of the tile inside the chunk; row i0 + r is position ia0 + r
+    const int ia0 = P.q_off + i0;
     const int tid = threadIdx.x, ty = tid / 16, tx = tid % 16;
     const T* q = Q + b * P.qs[0] + h * P.qs[2];
     const T* k = K + b * P.ks[0] + hk * P.ks[2];
     const T* v = V + b * P.vs[0] + hk * P.vs[2];
 
-    load_tile(sQ, LDQ, q, P.qs[1], i0, L, D);
+    load_tile(sQ, LDQ, q, P.qs[1], i0, P.Lq, D);
     if (tid < BM) { sM[tid] = -INFINITY; sL[tid] = 0.0f; }
     float acc[4][D / 16];
 #pragma unroll
@@ -53,9 +54,9 @@ __global__ void __launch_bounds__(NT) simt_fwd_kernel(const T* __restrict__ Q, c
 #pragma unroll
         for (int c = 0; c < D / 16; ++c) acc[a][c] = 0.0f;
 
-    const int last = P.causal ? min(i0 + BM, L) - 1 : L - 1;   // last key any row of the tile can see
+    const int last = P.causal ? min(ia0 + BM, L) - 1 : L - 1;  // last key any row of the tile can see
     for (int j0 = 0; j0 <= last; j0 += BN) {
-        if (use_bitmap && !bitmap_test(bitmap, P.Tr, P.Wd, bh, i0 / P.bm, j0 / P.bn)) continue;
+        if (use_bitmap && !bitmap_test(bitmap, P.Tr, P.Wd, bh, ia0 / P.bm, j0 / P.bn)) continue;
         __syncthreads();
         load_tile(sK, LDQ, k, P.ks[1], j0, L, D);
         load_tile(sV, D, v, P.vs[1], j0, L, D);
@@ -85,7 +86,7 @@ __global__ void __launch_bounds__(NT) simt_fwd_kernel(const T* __restrict__ Q, c
         for (int a = 0; a < 4; ++a)
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
-                int r = ty + 16 * a, cc = tx + 16 * c, i = i0 + r, j = j0 + cc;
+                int r = ty + 16 * a, cc = tx + 16 * c, i = ia0 + r, j = j0 + cc;
                 bool ok = (j <= i || !P.causal) && i < sE[cc];
                 sS[r * LDS + cc] = ok ? s[a][c] * P.scale + sB[cc] : -INFINITY;
             }
@@ -136,12 +137,12 @@ __global__ void __launch_bounds__(NT) simt_fwd_kernel(const T* __restrict__ Q, c
 #pragma unroll
     for (int a = 0; a < 4; ++a) {
         int r = ty + 16 * a, i = i0 + r;
-        if (i >= L) continue;
+        if (i >= P.Lq) continue;
         float l = sL[r], inv = l > 0.0f ? 1.0f / l : 0.0f;
         T* o = O + b * P.os[0] + (int64_t)i * P.os[1] + h * P.os[2];
 #pragma unroll
         for (int c = 0; c < D / 16; ++c) store_as(o + tx + 16 * c, acc[a][c] * inv);
-        if (tx == 0) lse[(size_t)bh * L + i] = l > 0.0f ? sM[r] + logf(l) : -INFINITY;
+        if (tx == 0) lse[(size_t)bh * P.Lq + i] = l > 0.0f ? sM[r] + logf(l) : -INFINITY;
     }
 }
 
@@ -324,9 +325,10 @@ int fwd_t(const Prob& P, const void* Q, const void* K, const void* V, const floa
     size_t smem = (size_t)(2 * BM * (D + 1) + BN * D + BM * (BN + 1) + 3 * BM + 2 * BN) * sizeof(float);
     auto kern = simt_fwd_kernel<T, D>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return DMA_ERR_CUDA;
-    int use_bitmap = !(P.flags & DMA_FLAG_IGNORE_BITMAP) && P.bm % BM == 0 && P.bn % BN == 0;
-    kern<<<dim3((P.L + BM - 1) / BM, P.Hq, P.B), NT, smem, st>>>((const T*)Q, (const T*)K, (const T*)V, bias, expiry,
-                                                                 bitmap, (T*)O, lse, P, use_bitmap);
+    // a chunk of query rows that does not start on a bitmap row boundary (or comes without a bitmap) visits every key tile
+    int use_bitmap = bitmap && !(P.flags & DMA_FLAG_IGNORE_BITMAP) && P.bm % BM == 0 && P.bn % BN == 0 && P.q_off % BM == 0;
+    kern<<<dim3((P.Lq + BM - 1) / BM, P.Hq, P.B), NT, smem, st>>>((const T*)Q, (const T*)K, (const T*)V, bias, expiry,
+                                                                  bitmap, (T*)O, lse, P, use_bitmap);
     count_launch();
     return check_launch();
 }

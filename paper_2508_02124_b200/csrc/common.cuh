@@ -19,6 +19,7 @@ struct Prob {
     int dtype, flags;
     int causal;            // 1: key j visible to rows i >= j; 0: to every row (the key's first row is 0 instead of j)
     int bm, bn, Tr, Tc, Wd;   // bitmap tile sizes, tile counts, uint32 words per bitmap row
+    int Lq, q_off;            // forward over a chunk of query rows: Q, O, lse hold the rows q_off .. q_off + Lq - 1 (Lq = L, q_off = 0: all)
     float scale;
     int64_t qs[3], ks[3], vs[3], os[3];   // batch, seq, head strides in elements
 };
