@@ -18,6 +18,9 @@
  *   - Every entry point returns 0 (DMA_OK) or a negative dma_status code; nothing is thrown across the ABI.
  *     On an error return no kernel has been launched. Outputs are fully overwritten (no pre-zeroing needed).
  *   - There is no CPU path: without a CUDA device of compute capability 10.x the calls return DMA_ERR_CUDA.
+ *   - The calls that take a stream only enqueue work on it: they allocate nothing and do not synchronise, so they can be
+ *     captured into a CUDA graph. Exceptions: dma_step_host, dma_read_status and dma_selftest_wait_timeout synchronise
+ *     the stream, and the first dma_mask_build_static call on a device looks up a symbol address.
  */
 #ifndef DMA_B200_H
 #define DMA_B200_H

@@ -174,6 +174,37 @@ def test_largest_supported_lengths():
     sampled_check(both, inp, got, nrows=8, nkeys=4)
 
 
+def test_whole_step_can_be_captured_in_a_cuda_graph():
+    """The stream entry points only enqueue work (no allocation, no synchronisation): mask build, forward and backward are
+    captured once and replayed; the replay reproduces the eager results."""
+    dev = torch.device("cuda:0")
+    case = wl.small(C2, B=1, Hq=8, Hkv=2, L=1024, w=256, backward=True, name="graph")
+    inp = wl.make_inputs(case)
+    eager = gpu_run(case, inp)
+    p = problem_of(case)
+    Q, K, V, dO = (inp[k].to(dev) for k in ("Q", "K", "V", "dO"))
+    W, A = inp["W_delta"].to(dev), inp["A"].to(dev)
+    m_ws, f_ws, b_ws = (torch.empty(n, dtype=torch.uint8, device=dev) for n in dma.dma_query_workspace(p))
+    bias, expiry, bitmap = (torch.empty_like(eager[k]) for k in ("bias", "expiry", "bitmap"))
+    O, lse = torch.empty_like(eager["O"]), torch.empty_like(eager["lse"])
+    dQ, dK, dV, dM = (torch.empty_like(eager[k]) for k in ("dQ", "dK", "dV", "dM"))
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        dma.dma_mask_build(p, V, W, A, bias, expiry, bitmap, m_ws)
+        dma.dma_attn_fwd(p, Q, K, V, bias, expiry, bitmap, O, lse, f_ws)
+        dma.dma_attn_bwd(p, Q, K, V, O, dO, lse, bias, expiry, bitmap, dQ, dK, dV, dM, b_ws)
+    for _ in range(2):
+        for t in (bias, expiry, bitmap, O, lse, dQ, dK, dV, dM):
+            t.zero_()
+        g.replay()
+        torch.cuda.synchronize()
+        assert dma.dma_read_status(f_ws) == 0 and dma.dma_read_status(b_ws) == 0
+        for k, t in (("bias", bias), ("expiry", expiry), ("bitmap", bitmap), ("O", O), ("lse", lse), ("dK", dK), ("dV", dV)):
+            assert torch.equal(t, eager[k]), k
+        assert_close(dQ, f64(eager["dQ"]), case.dtype, "dQ (replayed)")        # atomics: order-dependent rounding
+        assert_close(dM, f64(eager["dM"]), case.dtype, "dM (replayed)")
+
+
 def test_bounded_wait_reports_timeout_and_context_survives():
     # a wait that nothing satisfies gives up after its limit and leaves a status, instead of hanging the GPU
     dev = torch.device("cuda:0")
