@@ -489,6 +489,20 @@ def main():
         assert torch.equal(hO, O.cpu()), "host-buffer path disagrees with the device path"
         e2e = {"value": world * tile_flops(active, case.d, case.backward) / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s",
                "ms_per_step": e2e_ms, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+        # the same call with DMA_FLAG_COMPACT_KV (same outputs up to rounding, O(L w d) work): reported beside the headline
+        if case.dtype == "bf16" and case.d == 128 and not (args.flags & dma.DMA_FLAG_SIMT):
+            pce = dma.problem(case.B, case.Hq, case.Hkv, case.L, case.d, case.w, dtype=case.torch_dtype,
+                              flags=args.flags | dma.DMA_FLAG_COMPACT_KV)
+            arena_c = torch.empty(dma.dma_step_host_arena(pce, case.backward), dtype=torch.uint8, device=dev)
+            call_c = lambda: dma.dma_step_host(pce, case.backward, hin[0], hin[1], hin[2], hin[3], hin[4], hin[5], hO, hlse, hdQ, hdK, hdV, hdM, arena_c)
+            call_c(); call_c()
+            barrier()
+            t2.record()
+            for _ in range(n_e2e):
+                call_c()
+            t3.record()
+            barrier()
+            e2e["compact_ms_per_step"] = replicas.max_over_ranks(t2.elapsed_time(t3) / n_e2e, dev)
 
     if rank != 0:
         if dist is not None:
