@@ -16,7 +16,6 @@
 namespace dma {
 namespace {
 
-constexpr int kSelThreads = 1024;
 constexpr int kSplitKeys = 2048;
 constexpr int kAttnThreads = 256;
 
@@ -35,7 +34,7 @@ __device__ __forceinline__ unsigned long long key_of(float dl, int j) {
 struct SelState { uint32_t prefix; int need; };
 
 // hist: 2048 counters of one pass; returns through `st` the bin holding the need-th largest key (scanning from the top
-// bin) and the rank wanted inside it. Called by every thread of a CTA with kSelThreads / 4 = 256 threads.
+// bin) and the rank wanted inside it. Called by every thread of a CTA of 256 threads.
 __device__ __forceinline__ void pick_bin(const int* __restrict__ hist, int shift, SelState& st, int* s_scan, SelState* s_out) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     int c[8], sum = 0;
@@ -281,8 +280,6 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attn_kernel(const T* __re
                                                                    int N, int Hq, int G, float scale_log2, int nsplit,
                                                                    int64_t ks_b, int64_t ks_l, int64_t ks_h, int64_t vs_b, int64_t vs_l,
                                                                    int64_t vs_h) {
-    constexpr int LPK = D / 4;                 // lanes per key row (4 channels per lane)
-    constexpr int KPW = 32 / LPK;              // keys per warp instruction
     __shared__ int list[kSplitKeys];
     __shared__ int s_count, wsum[2][8];
     const int split = blockIdx.x, bh = blockIdx.y, b = bh / Hq, h = bh % Hq, hk = h / G;

@@ -314,7 +314,7 @@ __global__ void __launch_bounds__(kExpThreads) expiry_kernel(const float* __rest
     // probing the sorted array itself puts every early level into a single bank (addresses 128 apart, 64 apart, ...).
     __shared__ uint32_t shi[2][kChunk], slo[2][kChunk], sbf[2][kChunk];
     __shared__ int c_first;
-    const int bh = blockIdx.y, t = threadIdx.x, lane = t & 31, slot = blockIdx.x * kExpThreads + t;
+    const int bh = blockIdx.y, t = threadIdx.x, slot = blockIdx.x * kExpThreads + t;
     const float* dl = delta + (size_t)bh * L;
     const unsigned long long* srt = sorted + (size_t)bh * nchunk * kChunk;
     const bool valid = slot < L;
