@@ -193,14 +193,15 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             if (!use_bit(entry, w)) continue;
             PROF_T(t_a);
             const int st = it % kStages, j0 = (int)(entry & 0xFFFFF) * 128;
-            // the stagers' flag is there long before the S product: read it while waiting for S
-            ok = mbar_wait_warp(&S.k_full[st], (it / kStages) & 1, abort_flag);
-            if (!ok) break;
-            const uint32_t tile_flags = S.fast[st][w];
-            const bool fast_tile = kCompact || tile_flags != 0;      // token-compacted mode: the flags are a chunk mask instead
             ok = mbar_wait_warp(&S.s_full[w], n_used & 1, abort_flag);
             if (!ok) break;
             tc_fence_after();
+            // The stagers' flag is read only now. The S product was issued after k_full[st] completed, so the flag of THIS
+            // iteration is in place. (Waiting on k_full[st] here instead is wrong: a tile that skipped earlier key tiles
+            // has not followed that barrier's phases, and a parity wait on a barrier it is a whole phase ahead of returns
+            // at once, before the stager has written the flag.)
+            const uint32_t tile_flags = S.fast[st][w];
+            const bool fast_tile = kCompact || tile_flags != 0;      // token-compacted mode: the flags are a chunk mask instead
             PROF_T(t_b);
             PROF_ADD(0, t_b - t_a);
             if ((warp & 3) == 0 && lane == 0) TRACE(it, w * 4 + 0);

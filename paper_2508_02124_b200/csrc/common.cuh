@@ -52,6 +52,8 @@ int launch_simt_bwd(const Prob& P, const void* Q, const void* K, const void* V, 
                     const float* lse, const float* bias, const int32_t* expiry, const uint32_t* bitmap, void* dQ,
                     void* dK, void* dV, float* dM, void* ws, cudaStream_t st);
 
+int launch_pad64(const void* src, void* dst, int B, int L, int H, const int64_t (&s)[3], cudaStream_t st);
+int launch_unpad64(const void* src, void* dst, int B, int L, int H, const int64_t (&s)[3], cudaStream_t st);
 size_t tc_fwd_ws_bytes(const Prob& P);
 int launch_tc_fwd(const Prob& P, const void* Q, const void* K, const void* V, const float* bias,
                   const int32_t* expiry, const uint32_t* bitmap, void* O, float* lse, void* ws, cudaStream_t st);

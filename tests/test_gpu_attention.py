@@ -260,12 +260,43 @@ def test_compact_forward_full_size_sampled(key):
 
 def test_compact_flag_is_rejected_where_unsupported():
     dev = torch.device("cuda:0")
-    case = wl.small(C2, B=1, Hq=2, Hkv=1, L=256, w=64, d=64, name="compact-d64")
+    for case in (wl.small(C1, B=1, Hq=2, Hkv=1, L=256, w=64, d=128, name="compact-fp32"),
+                 wl.small(C2, B=1, Hq=2, Hkv=1, L=256, w=64, d=64, name="compact-d64-cuda-cores")):
+        inp = wl.make_inputs(case)
+        flags = dma.DMA_FLAG_COMPACT_KV | (dma.DMA_FLAG_SIMT if case.dtype == "bf16" else 0)
+        with pytest.raises(dma.DmaError) as e:
+            gpu_run(case, inp, backward=False, flags=flags)
+        assert e.value.status == -4
+
+
+def test_bf16_d64_runs_on_the_tensor_core_kernels():
+    """bf16 with 64 channels goes through zero-padded 128-channel copies: same results as the CUDA-core kernels within the
+    gate, on strided inputs too, and far faster (the launch list shows the tensor-core kernels)."""
+    dev = torch.device("cuda:0")
+    case = wl.small(C2, B=2, Hq=4, Hkv=2, L=700, w=96, d=64, backward=True, name="d64-padded")
     inp = wl.make_inputs(case)
-    p = problem_of(case, flags=dma.DMA_FLAG_COMPACT_KV)
-    with pytest.raises(dma.DmaError) as e:
-        gpu_run(case, inp, backward=False, flags=dma.DMA_FLAG_COMPACT_KV)
-    assert e.value.status == -4
+    dl, e, _ = oracle_mask(case, inp)
+    ref = oracle_all(case, inp, dl, e)
+    for flags in (0, dma.DMA_FLAG_COMPACT_KV):
+        compare(case, gpu_run(case, inp, flags=flags), ref)
+    # strided Q / K / V / O views of wider buffers
+    big = {k: torch.randn(case.B, case.L + 9, (case.Hq if k in ("Q", "dO") else case.Hkv) + 1, 64).to(case.torch_dtype).to(dev) for k in ("Q", "K", "V", "dO")}
+    view = {k: big[k][:, 3:3 + case.L, 1:] for k in big}
+    for k in view:
+        view[k].copy_(inp[k].to(dev))
+    p = problem_of(case)
+    for sdst, t in ((p.q_stride, view["Q"]), (p.k_stride, view["K"]), (p.v_stride, view["V"]), (p.o_stride, view["dO"])):
+        sdst[0], sdst[1], sdst[2] = t.stride(0), t.stride(1), t.stride(2)
+    bias, expiry, bitmap = dma.dma_mask_build(p, view["V"], inp["W_delta"].to(dev), inp["A"].to(dev))
+    Obuf = torch.zeros_like(big["dO"])
+    O, lse = dma.dma_attn_fwd(p, view["Q"], view["K"], view["V"], bias, expiry, bitmap, O=Obuf[:, 3:3 + case.L, 1:])
+    dQb, dKb, dVb = torch.zeros_like(big["Q"]), torch.zeros_like(big["K"]), torch.zeros_like(big["V"])
+    dQ, dK, dV, dM = dma.dma_attn_bwd(p, view["Q"], view["K"], view["V"], O, view["dO"], lse, bias, expiry, bitmap,
+                                      dQ=dQb[:, 3:3 + case.L, 1:], dK=dKb[:, 3:3 + case.L, 1:], dV=dVb[:, 3:3 + case.L, 1:])
+    torch.cuda.synchronize()
+    compare(case, {"O": O, "lse": lse, "dQ": dQ, "dK": dK, "dV": dV, "dM": dM}, ref)
+    assert float(Obuf[:, :3].abs().max()) == 0.0 and float(Obuf[:, :, 0].abs().max()) == 0.0
+    assert float(dKb[:, :3].abs().max()) == 0.0 and float(dKb[:, :, 0].abs().max()) == 0.0
 
 
 def test_compact_kernels_on_strided_k_and_v():

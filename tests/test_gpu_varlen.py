@@ -22,6 +22,7 @@ SMALL = [
     (wl.small(C2, B=2, Hq=4, Hkv=1, L=1536, w=200, backward=True, name="varlen bf16 three documents"), [0, 700, 829, 1536]),
     (wl.small(C2, B=1, Hq=2, Hkv=2, L=1024, w=64, backward=True, name="varlen bf16 tile-aligned"), [0, 256, 512, 1024]),
     (wl.small(C2, B=1, Hq=4, Hkv=4, L=512, w=64, d=64, backward=True, name="varlen bf16 d64"), [0, 77, 300, 512]),
+    (wl.small(C2, B=1, Hq=4, Hkv=4, L=512, w=64, d=128, backward=True, name="varlen bf16 late entry"), [0, 77, 300, 512]),
     (wl.small(C2, B=1, Hq=2, Hkv=1, L=700, w=1, backward=True, name="varlen bf16 w=1"), [0, 130, 131, 400, 700]),
     (wl.small(C1, B=1, L=40, w=3, name="varlen fp32 every document one token"), list(range(41))),
 ]
@@ -64,6 +65,30 @@ def test_token_compacted_kernels_on_packed_sequences(case, cu):
     inp, got = run(case, cu, flags=dma.DMA_FLAG_COMPACT_KV)
     dl, e, _ = oracle_varlen_mask(case, inp, cu)
     compare(case, got, oracle_all(case, inp, dl, e))
+
+
+def test_query_tile_whose_first_key_tiles_belong_to_another_document():
+    """Regression: the second query tile of a CTA's pair starts a new document, so it skips the key tiles its partner
+    still needs and enters the walk late, at a tile that takes the per-element path. It once read that tile's fast-path
+    flag before the stager had written it (the outcome depended on where the tensors lay in memory). Several placements
+    of Q, K, V, tensor-core kernel against the CUDA-core kernel."""
+    case = wl.small(C2, B=1, Hq=4, Hkv=4, L=512, w=64, d=128, backward=False, name="varlen late entry")
+    cu = torch.tensor([0, 77, 300, 512], dtype=torch.int32, device=DEV)
+    inp = wl.make_inputs(case)
+    p, ps = problem_of(case), problem_of(case, flags=dma.DMA_FLAG_SIMT)
+    n = case.L * case.Hq * case.d
+    big = torch.empty(3 * n + (4 << 20), dtype=torch.bfloat16, device=DEV)
+    W, A = inp["W_delta"].to(DEV), inp["A"].to(DEV)
+    for trial in range(12):
+        off = trial * 0x12340 * 4
+        Q, K, V = (big[off + t * n:off + (t + 1) * n].view(1, case.L, case.Hq, case.d) for t in range(3))
+        Q.copy_(inp["Q"]); K.copy_(inp["K"]); V.copy_(inp["V"])
+        bias, expiry, bitmap = dma.dma_mask_build_varlen(p, V, W, A, cu)
+        ref, lref = dma.dma_attn_fwd(ps, Q, K, V, bias, expiry, bitmap)
+        O, lse = dma.dma_attn_fwd(p, Q, K, V, bias, expiry, bitmap)
+        torch.cuda.synchronize()
+        assert float((O.float() - ref.float()).abs().max()) <= 3e-2, trial
+        assert float((lse - lref).abs().max()) <= 1e-3 * max(1.0, float(lref.abs().max())), trial
 
 
 def test_one_sequence_equals_the_plain_mask_build():
