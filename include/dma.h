@@ -142,7 +142,8 @@ int dma_mask_build_varlen(const dma_problem_t* p, const void* V, const float* W_
  *   s_j = q_i . k_j * scale + bias[j]   over keys with j <= i < expiry[j];   p = softmax(s);   O_i = sum p_j v_j
  *   lse_i = log sum_j exp(s_j)   (natural log; replaces Alg. 1's (l, m) pair)
  * Key tiles whose bitmap bit is 0 are neither loaded nor computed. Any self-consistent (bias, expiry, bitmap)
- * triple is accepted. bf16: tcgen05/TMA kernel, d = 128 (d = 64 runs the CUDA-core kernel); fp32: CUDA-core kernel. */
+ * triple is accepted. bf16: tcgen05/TMA kernel for d = 128; d = 64 runs the same kernel on zero-padded 128-channel copies
+ * held in the workspace (forward and backward; dma_query_workspace reports the larger sizes); fp32: CUDA-core kernel. */
 int dma_attn_fwd(const dma_problem_t* p, const void* Q, const void* K, const void* V,
                  const float* bias, const int32_t* expiry, const uint32_t* bitmap,
                  void* O, float* lse, void* ws, size_t ws_bytes, void* cuda_stream);
