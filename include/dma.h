@@ -58,7 +58,9 @@ enum {
                                     lifetime-sorted permutation built per call) and walks only the query tiles between
                                     the first key and the last expiry; dK, dV are summed over the group in fp32. Same
                                     results up to rounding; needs the larger workspaces dma_query_workspace reports for
-                                    it; ignores the bitmap */
+                                    it; ignores the bitmap. The mask must keep at most w keys per row, as every mask
+                                    of dma_mask_build does (an injected mask that keeps more needs p->w raised to its
+                                    largest per-row count: the gathered lists are sized w + 256) */
     DMA_FLAG_FULL_DELTA = 8      /* the sampling weights as Eq. (delta_calc) states them: W_delta (and dW_delta) is
                                     [Hq, Hkv*d], one row per query head over ALL channels of the value row (the linear
                                     layer of the App. A listing), z[b,h,j] = sum_{h'} V[b,j,h',:] . W_delta[h, h'*d:(h'+1)*d].

@@ -63,3 +63,41 @@ def test_tensor_core_kernels_equal_the_cuda_core_kernels(seed):
             scale = max(1.0, float(b.abs().max()))
             tol = (1e-3 if k == "lse" else 4e-2) * scale
             assert float((a - b).abs().max()) <= tol, (seed, flags, k, float((a - b).abs().max()), scale, cu, case)
+
+
+@pytest.mark.parametrize("seed", range(8))
+def test_arbitrary_interval_masks(seed):
+    """Any self-consistent (bias, expiry, bitmap) triple is accepted: lifetimes drawn at random (one row, tens of rows,
+    hundreds, the whole rest of the sequence) instead of a top-w selection, the bitmap from the oracle's interval rule.
+    Every key is kept at least by its own row, so no row is empty."""
+    import oracle
+    r = np.random.default_rng(100 + seed)
+    Hkv, G = int(r.choice([1, 2])), int(r.choice([1, 2, 4]))
+    L = int(r.choice([256, 640, 1100]))
+    case = wl.small(wl.CONFIGS["2"], B=1, Hq=Hkv * G, Hkv=Hkv, L=L, w=L, d=128, backward=True, seed=2000 + seed, name=f"interval-{seed}")
+    inp = wl.make_inputs(case)
+    Hq = case.Hq
+    kind = r.integers(0, 10, (1, Hq, L))
+    life = np.where(kind < 3, 1, np.where(kind < 6, r.integers(1, 64, (1, Hq, L)), np.where(kind < 9, r.integers(64, L + 1, (1, Hq, L)), L)))
+    if seed % 2:
+        life[:, :, 128:256] = 1                                   # a whole key tile that only its own rows keep
+    e = np.minimum(np.arange(L)[None, None, :] + life, L).astype(np.int32)
+    bias = r.uniform(0.5, 6.0, (1, Hq, L)).astype(np.float32)
+    bitmap = oracle.bitmap_from_expiry(e)
+    Q, K, V, dO = (inp[k].to(DEV) for k in ("Q", "K", "V", "dO"))
+    bias_t, e_t, bmp_t = torch.from_numpy(bias).to(DEV), torch.from_numpy(e).to(DEV), torch.from_numpy(bitmap.view(np.int32)).to(DEV)
+    ref = None
+    for flags in (dma.DMA_FLAG_SIMT, 0, dma.DMA_FLAG_COMPACT_KV):
+        p = dma.problem(1, Hq, Hkv, L, 128, L, flags=flags)
+        O, lse = dma.dma_attn_fwd(p, Q, K, V, bias_t, e_t, bmp_t)
+        dQ, dK, dV, dM = dma.dma_attn_bwd(p, Q, K, V, O, dO, lse, bias_t, e_t, bmp_t)
+        torch.cuda.synchronize()
+        out = {"O": O, "lse": lse, "dQ": dQ, "dK": dK, "dV": dV, "dM": dM}
+        assert all(bool(torch.isfinite(t.float()).all()) for t in out.values()), (seed, flags)
+        if ref is None:
+            ref = out
+            continue
+        for k, t in out.items():
+            a, b = t.float(), ref[k].float()
+            scale = max(1.0, float(b.abs().max()))
+            assert float((a - b).abs().max()) <= (1e-3 if k == "lse" else 4e-2) * scale, (seed, flags, k, float((a - b).abs().max()), scale)
