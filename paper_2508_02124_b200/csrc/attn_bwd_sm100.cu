@@ -241,7 +241,8 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                 len = j < P.L ? max(0, P.expiry[(size_t)bh * P.L + j] - jf) : 0;
                 cur_g = g;
             }
-            PROF_WAIT(0, ok = mbar_wait_warp(&S.sdp_full, n & 1, abort_flag) && mbar_wait_warp(&S.qd_full[st], (n / kStages) & 1, abort_flag));
+            // (S^T and dP^T were issued after the step's Q / dO stage was full: nothing else of that stage is read here)
+            PROF_WAIT(0, ok = mbar_wait_warp(&S.sdp_full, n & 1, abort_flag));
             if (!ok) break;
             tc_fence_after();
             uint32_t sr[32], pr[32];
