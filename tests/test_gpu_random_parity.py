@@ -1,6 +1,7 @@
-"""Randomised parity of the mask build against the oracle, bit for bit: random sizes (including L below one chunk and
+"""Randomised parity. The mask build against the oracle, bit for bit: random sizes (including L below one chunk and
 ragged tails), window sizes around and above L, element types, head groupings, the three selection modes (causal, packed
-documents, non-causal) and both sampling-weight shapes."""
+documents, non-causal) and both sampling-weight shapes. The mask backward against the oracle, and forward chunks at random
+positions against the whole forward."""
 import numpy as np
 import pytest
 import torch
