@@ -83,3 +83,15 @@ def test_state_after_steps_equals_a_fresh_init():
     # the recorded weakest key is the same key in both (its position in the list may differ)
     a, b = state.cpu(), fresh.cpu()
     assert torch.equal(a[:, 2:4], b[:, 2:4])
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_random_sequences(seed):
+    r = np.random.default_rng(40 + seed)
+    Hkv, G = int(r.choice([1, 2, 3])), int(r.choice([1, 2, 4]))
+    w = int(r.choice([1, 5, 64, 130, 257]))
+    n0 = int(r.choice([0, 1, w // 2, w, w + 17, 3 * w]))
+    steps = int(r.integers(10, 40))
+    case = wl.small(wl.CONFIGS["2"], B=int(r.choice([1, 2])), Hq=Hkv * G, Hkv=Hkv, L=n0 + steps + int(r.integers(0, 9)), d=int(r.choice([64, 128])),
+                    w=w, dtype=str(r.choice(["bf16", "fp32"])), backward=False, seed=6000 + seed, name=f"decode-step-random-{seed}")
+    run(case, n0, steps, seed=seed, tie_head=bool(seed % 3 == 0))
