@@ -12,10 +12,12 @@ from paper_2508_02124_b200 import workloads as wl
 pytestmark = pytest.mark.gpu
 
 
-def build_both(case, inp, out):
+def build_both(case, inp, out, causal=1, full=False):
     dev = torch.device("cuda:0")
-    p = dma.problem(case.B, case.Hq, case.Hkv, case.L, case.d, case.w, dtype=case.torch_dtype)
-    V, W, A = inp["V"].to(dev), inp["W_delta"].to(dev), inp["A"].to(dev)
+    p = dma.problem(case.B, case.Hq, case.Hkv, case.L, case.d, case.w, dtype=case.torch_dtype, causal=causal,
+                    flags=dma.DMA_FLAG_FULL_DELTA if full else 0)
+    V, A = inp["V"].to(dev), inp["A"].to(dev)
+    W = (wl.full_delta_weights(case) if full else inp["W_delta"]).to(dev)
     ref = dma.dma_mask_build(p, V, W, A)
     for t in out:
         t.fill_(-1)                                   # outputs are preallocated by the caller and fully overwritten
@@ -37,6 +39,8 @@ def test_static_scratch_matches_workspace_version_on_consecutive_calls():
         inp = wl.make_inputs(case)
         build_both(case, inp, out)
         build_both(case, inp, out)
+        build_both(case, inp, out, causal=0)                      # the non-causal selection and the full sampling weights
+        build_both(case, inp, out, full=True)                     # go through the same scratch
 
 
 def test_static_scratch_rejects_oversized_problems():
