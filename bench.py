@@ -218,6 +218,11 @@ def main():
         stage_ms["mask"] += e[0].elapsed_time(e[1]); stage_ms["fwd"] += e[1].elapsed_time(e[2]); stage_ms["bwd"] += e[2].elapsed_time(e[3])
     stage_ms = {k: v / args.steps for k, v in stage_ms.items()}
     ms = replicas.max_over_ranks(total_ms / args.steps, dev)
+    per_step = sorted(e[0].elapsed_time(e[3]) for e in evs)                 # each step's own span (events around its stages)
+    step_stats = {"median_ms": per_step[len(per_step) // 2], "min_ms": per_step[0], "max_ms": per_step[-1]}
+    # useful work: 4 d (forward) resp. 10 d (backward) flop per kept (row, key) pair, whatever the tile granularity
+    kept_pairs = int((expiry.long() - torch.arange(case.L, device=dev)).clamp_(min=0).sum().item())
+    useful_flops = kept_pairs * (4 + (10 if case.backward else 0)) * case.d
 
     # ---- mask-generation backward (bias gradient on to W_delta, A and V), timed on its own after the step: it is
     # not part of the headline metric. HBM-bound: V read once, dV read and written once, bias and dM read once.
@@ -534,6 +539,8 @@ def main():
                      "unit": "TFLOP/s", "frac": achieved / pk["bf16_sustained"],
                      "traffic": NCU_TRAFFIC_BYTES.get(case.name, {}).get(dom) if tensor_path else None},
         "gpu_launches": launches, "clocks": clocks, "e2e": e2e,
+        "step_ms": step_stats, "kept_pairs": kept_pairs, "useful_tflop_per_step": useful_flops / 1e12,
+        "useful_tflops": world * useful_flops / (ms * 1e-3) / 1e12,
     }
     if decode is not None:
         decode["frac_of_measured_hbm"] = decode["gbs"] / pk["hbm_gbs"]
