@@ -1,4 +1,6 @@
-"""CPU oracle for Dynamic Mask Attention: thin ctypes access to ``dma_oracle.cpp``.
+"""CPU oracle for Dynamic Mask Attention: ctypes access to ``dma_oracle.cpp`` (delta in the pinned fp32 arithmetic, the
+selection in definition and interval form, bitmaps, forward, backward) plus the parts that are plain numpy in fp64
+(mask-generation backward, decoding step, non-causal and packed-sequence selection).
 
 TEST INFRASTRUCTURE ONLY: imported by the tests, by the smoke check and by the benchmark's
 CPU-baseline leg. The product package never imports it and it never imports the product package.
