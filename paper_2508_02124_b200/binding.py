@@ -61,13 +61,26 @@ def dma_strerror(status):
 def problem(B, Hq, Hkv, L, d, w, dtype=torch.bfloat16, causal=1, tile_m=0, tile_n=0, flags=0, softmax_scale=0.0):
     p = dma_problem_t()
     p.B, p.Hq, p.Hkv, p.L, p.d, p.w, p.causal = B, Hq, Hkv, L, d, w, causal
-    p.dtype = DMA_BF16 if dtype == torch.bfloat16 else DMA_FP32
+    if dtype in (torch.bfloat16, torch.float32):
+        p.dtype = DMA_BF16 if dtype == torch.bfloat16 else DMA_FP32
+    elif type(dtype) is int and dtype in (DMA_BF16, DMA_FP32):
+        p.dtype = dtype
+    else:
+        raise TypeError(f"element type {dtype!r}: torch.bfloat16, torch.float32, DMA_BF16 or DMA_FP32")
     p.tile_m, p.tile_n, p.flags, p.softmax_scale = tile_m, tile_n, flags, softmax_scale
     return p
 
 
 def _ptr(t):
     return ctypes.c_void_p(0 if t is None else t.data_ptr())
+
+
+def _elem(p, *tensors):
+    """The library reads Q, K, V, ... as the problem's element type; a tensor of another type would be read out of bounds."""
+    want = torch.bfloat16 if p.dtype == DMA_BF16 else torch.float32
+    for t in tensors:
+        if t is not None and t.dtype != want:
+            raise TypeError(f"tensor of {t.dtype} passed for a problem whose element type is {want}")
 
 
 def _stream():
@@ -97,6 +110,7 @@ def _ws(nbytes, device):
 
 def dma_mask_build(p, V, W_delta, A, bias=None, expiry=None, bitmap=None, ws=None):
     """Returns (bias [B,Hq,L] fp32, expiry [B,Hq,L] int32, bitmap [B,Hq,Tr,ceil(Tc/32)] int32-typed uint32 words)."""
+    _elem(p, V)
     dev = V.device
     if bias is None:
         bias = torch.empty(p.B, p.Hq, p.L, dtype=torch.float32, device=dev)
@@ -115,6 +129,7 @@ def dma_mask_build(p, V, W_delta, A, bias=None, expiry=None, bitmap=None, ws=Non
 
 def dma_mask_build_varlen(p, V, W_delta, A, cu_seqlens, bias=None, expiry=None, bitmap=None, ws=None):
     """dma_mask_build for sequences packed along the sequence axis; cu_seqlens: int32 device tensor [nseq + 1]."""
+    _elem(p, V)
     dev = V.device
     assert cu_seqlens.dtype == torch.int32 and cu_seqlens.is_cuda and cu_seqlens.is_contiguous()
     if bias is None:
@@ -141,6 +156,7 @@ def dma_mask_bwd_workspace(p):
 
 def dma_mask_bwd(p, V, W_delta, A, bias, dM, dV, dW_delta=None, dA=None, ws=None):
     """Adds the mask path's contribution to dV in place; returns (dV, dW_delta fp32 shaped like W_delta, dA [Hq] fp32)."""
+    _elem(p, V, dV)
     dev = V.device
     if dW_delta is None:
         dW_delta = torch.empty(p.Hq, p.Hkv * p.d if p.flags & DMA_FLAG_FULL_DELTA else p.d, dtype=torch.float32, device=dev)
@@ -155,6 +171,7 @@ def dma_mask_bwd(p, V, W_delta, A, bias, dM, dV, dW_delta=None, dA=None, ws=None
 
 def dma_delta_range(p, V, W_delta, A, delta, j_begin, j_end):
     """delta[b,h,j] for the keys j in [j_begin, j_end) of the cache V, written into the delta cache [B,Hq,ld]."""
+    _elem(p, V)
     _check(lib().dma_delta_range(ctypes.byref(p), _ptr(V), _ptr(W_delta), _ptr(A), _ptr(delta), ctypes.c_int64(delta.stride(1)),
                                  ctypes.c_int32(j_begin), ctypes.c_int32(j_end), _stream()), "dma_delta_range")
     return delta
@@ -168,6 +185,7 @@ def dma_decode_workspace(p):
 
 def dma_decode(p, q, K, V, delta, o=None, lse=None, sel_idx=None, want_idx=False, ws=None):
     """One decoding step over the cached keys; returns (o [B,Hq,d], lse [B,Hq], sel_idx or None)."""
+    _elem(p, q, K, V, o)
     dev = q.device
     if o is None:
         o = torch.empty_like(q)
@@ -199,6 +217,7 @@ def dma_decode_state_init(p, delta, state, ws=None):
 
 def dma_decode_step(p, q, K, V, delta, state, o=None, lse=None, ws=None):
     """One decoding step with the carried state (p.L counts the cached keys including the one just appended)."""
+    _elem(p, q, K, V, o)
     dev = q.device
     if o is None:
         o = torch.empty_like(q)
@@ -219,6 +238,7 @@ def decode_state_sets(state, w):
 
 def dma_attn_fwd(p, Q, K, V, bias, expiry, bitmap, O=None, lse=None, ws=None):
     """Returns (O like Q, lse [B,Hq,L] fp32)."""
+    _elem(p, Q, K, V, O)
     if O is None:
         O = torch.empty_like(Q)
     if lse is None:
@@ -232,6 +252,7 @@ def dma_attn_fwd(p, Q, K, V, bias, expiry, bitmap, O=None, lse=None, ws=None):
 
 def dma_attn_fwd_chunk(p, q_begin, Q, K, V, bias, expiry, O=None, lse=None, ws=None):
     """Forward for the query rows q_begin .. q_begin + Q.shape[1] - 1 of a sequence of p.L keys; returns (O like Q, lse [B,Hq,q_len])."""
+    _elem(p, Q, K, V, O)
     q_len = Q.shape[1]
     if O is None:
         O = torch.empty_like(Q)
@@ -249,6 +270,7 @@ def dma_attn_fwd_chunk(p, q_begin, Q, K, V, bias, expiry, O=None, lse=None, ws=N
 
 def dma_attn_bwd(p, Q, K, V, O, dO, lse, bias, expiry, bitmap, dQ=None, dK=None, dV=None, dM=None, ws=None):
     """Returns (dQ like Q, dK like K, dV like V, dM [B,Hq,L] fp32)."""
+    _elem(p, Q, K, V, O, dO, dQ, dK, dV)
     dQ = torch.empty_like(Q) if dQ is None else dQ
     dK = torch.empty_like(K) if dK is None else dK
     dV = torch.empty_like(V) if dV is None else dV
@@ -286,6 +308,7 @@ def dma_step_host(p, backward, hQ, hK, hV, hdO, hW, hA, hO, hlse, hdQ, hdK, hdV,
 def dma_mask_build_static(p, V, W_delta, A, bias, expiry, bitmap):
     """dma_mask_build without a workspace: the scratch is a fixed array inside the library (see include/dma.h for
     the size limit and the sharing rules). Outputs must be preallocated by the caller; nothing is allocated here."""
+    _elem(p, V)
     _check(lib().dma_mask_build_static(ctypes.byref(p), _ptr(V), _ptr(W_delta), _ptr(A), _ptr(bias), _ptr(expiry),
                                        _ptr(bitmap), _stream()), "dma_mask_build_static")
     return bias, expiry, bitmap

@@ -67,3 +67,16 @@ def test_no_cpu_fallback(lib):
     a = ctypes.c_void_p(4096)
     assert lib.dma_mask_build(ctypes.byref(ok), a, a, a, a, a, a, a, ctypes.c_size_t(1 << 30), ctypes.c_void_p(0)) == -6
     assert lib.dma_attn_fwd(ctypes.byref(ok), *([a] * 9), ctypes.c_size_t(1 << 30), ctypes.c_void_p(0)) == -6
+
+
+def test_binding_refuses_tensors_of_another_element_type():
+    # the library would read them with the problem's element size; the binding stops that before any call
+    p = dma.problem(1, 2, 2, 8, 64, 4, dtype=dma.DMA_FP32)
+    assert p.dtype == dma.DMA_FP32 and dma.problem(1, 2, 2, 8, 64, 4).dtype == dma.DMA_BF16
+    V = torch.zeros(1, 8, 2, 64, dtype=torch.bfloat16)
+    with pytest.raises(TypeError):
+        dma.dma_mask_build(p, V, None, None)
+    with pytest.raises(TypeError):
+        dma.dma_attn_fwd(p, V, V, V, None, None, None)
+    with pytest.raises(TypeError):
+        dma.problem(1, 2, 2, 8, 64, 4, dtype=torch.float16)
