@@ -27,7 +27,9 @@ struct Layout {
     size_t Q, K, V, dO, O, dQ, dK, dV, W, A, bias, expiry, bitmap, lse, dM, ws_mask, ws_fwd, ws_bwd, total;
     size_t nq, nk, nbh, nbmp, m_ws, f_ws, b_ws, esz, wbytes;
     int head_groups;       // groups of KV heads per batch entry (1 = whole batch entries)
-    int groups;            // B * head_groups
+    int groups;            // B * head_groups (1: the whole problem at once)
+    int group_batch;       // batch entries per group: 1, or B when there is a single group
+    size_t gh, gbmp;       // entries of a group's block of bias / expiry / lse / dM and of its bitmap, padded to 256 bytes
 };
 
 // Head groups per batch entry: up to 4, a divisor of Hkv, and only where every per-group pointer stays 16-byte aligned,
@@ -39,7 +41,7 @@ int pick_head_groups(const Prob& P) {
     for (int g = 4; g > 1; --g) {
         if (P.Hkv % g || (size_t)(P.Hkv / g) * P.d * esz < 512) continue;
         const size_t hq = (size_t)P.Hq / g;
-        if ((hq * P.L) % 4 || (hq * P.Tr * P.Wd) % 4 || hq % 4) continue;
+        if (hq % 4) continue;                       // W_delta and A of a group start at its first query head
         return g;
     }
     return 1;
@@ -69,13 +71,20 @@ int make_layout(const dma_problem_t* p, int backward, Layout* Lo) {
     Lo->O = a.take(Lo->nq * Lo->esz);
     Lo->wbytes = (size_t)P.Hq * ((P.flags & DMA_FLAG_FULL_DELTA) ? P.Hkv * P.d : P.d) * 4;
     Lo->W = a.take(Lo->wbytes); Lo->A = a.take((size_t)P.Hq * 4);
-    Lo->bias = a.take(Lo->nbh * 4); Lo->expiry = a.take(Lo->nbh * 4); Lo->bitmap = a.take(Lo->nbmp * 4);
-    Lo->lse = a.take(Lo->nbh * 4);
+    // per-head vectors and the bitmap live in one padded block per group, so that every group's pointers are aligned
+    // whatever Hq * L is
+    Lo->group_batch = Lo->groups == 1 ? P.B : 1;
+    const size_t hq_g = (size_t)Lo->group_batch * (P.Hq / Lo->head_groups);
+    Lo->gh = (hq_g * P.L + 63) / 64 * 64;
+    Lo->gbmp = (hq_g * P.Tr * P.Wd + 63) / 64 * 64;
+    const size_t vec = (size_t)Lo->groups * Lo->gh * 4;
+    Lo->bias = a.take(vec); Lo->expiry = a.take(vec); Lo->bitmap = a.take((size_t)Lo->groups * Lo->gbmp * 4);
+    Lo->lse = a.take(vec);
     Lo->ws_mask = a.take(Lo->m_ws); Lo->ws_fwd = a.take(Lo->f_ws);
     if (backward) {
         Lo->dO = a.take(Lo->nq * Lo->esz); Lo->dQ = a.take(Lo->nq * Lo->esz);
         Lo->dK = a.take(Lo->nk * Lo->esz); Lo->dV = a.take(Lo->nk * Lo->esz);
-        Lo->dM = a.take(Lo->nbh * 4); Lo->ws_bwd = a.take(Lo->b_ws);
+        Lo->dM = a.take(vec); Lo->ws_bwd = a.take(Lo->b_ws);
     }
     Lo->total = a.off;
     return DMA_OK;
@@ -110,6 +119,9 @@ int dma_step_host(const dma_problem_t* p, int backward, const void* hQ, const vo
     char* a = (char*)dev_arena;
     const int NG = Lo.groups, HG = Lo.head_groups;
     const int L = p->L, d = p->d, nqh = p->Hq / HG, nkh = p->Hkv / HG;
+    const int GB = Lo.group_batch;                 // batch entries per group
+    const size_t rows = (size_t)GB * L;            // sequence rows per group (batch entries are contiguous)
+    const size_t hl = (size_t)GB * nqh * L;        // entries of a group's per-head vectors
     const size_t esz = Lo.esz;
 
     // Copies run on two helper streams of this call (created and destroyed here: no state is kept) so that they overlap
@@ -143,15 +155,14 @@ int dma_step_host(const dma_problem_t* p, int backward, const void* hQ, const vo
     auto rec = [&](cudaEvent_t e, cudaStream_t on) { return cudaEventRecord(e, on) == cudaSuccess; };
     auto wait = [&](cudaStream_t on, cudaEvent_t e) { return cudaStreamWaitEvent(on, e, 0) == cudaSuccess; };
 
-    struct Group { size_t q, k, h, bmp; int hq0; };
+    struct Group { size_t q, k, h; int hq0; };
     auto group_of = [&](int g) {
         const int b = g / HG, hg = g % HG;
         Group G;
         G.hq0 = hg * nqh;
         G.q = ((size_t)b * L * p->Hq + (size_t)hg * nqh) * d;          // elements into Q, O, dO, dQ
         G.k = ((size_t)b * L * p->Hkv + (size_t)hg * nkh) * d;         // elements into K, V, dK, dV
-        G.h = ((size_t)b * p->Hq + (size_t)hg * nqh) * L;              // entries into bias, expiry, lse, dM
-        G.bmp = ((size_t)b * p->Hq + (size_t)hg * nqh) * ((Lo.nbmp / p->B) / p->Hq);
+        G.h = ((size_t)b * p->Hq + (size_t)hg * nqh) * L;              // entries into the host's lse and dM
         return G;
     };
     const size_t q_pitch = (size_t)p->Hq * d * esz, q_width = (size_t)nqh * d * esz;
@@ -164,15 +175,15 @@ int dma_step_host(const dma_problem_t* p, int backward, const void* hQ, const vo
         const Group G = group_of(g);
         cudaEvent_t* e = ev + g * kPerGroup;
         const cudaMemcpyKind in = cudaMemcpyHostToDevice;
-        ok = copy2d(a + Lo.V + G.k * esz, (const char*)hV + G.k * esz, k_pitch, k_width, L, in, s_in) && rec(e[kV], s_in) &&
-             copy2d(a + Lo.K + G.k * esz, (const char*)hK + G.k * esz, k_pitch, k_width, L, in, s_in) &&
-             copy2d(a + Lo.Q + G.q * esz, (const char*)hQ + G.q * esz, q_pitch, q_width, L, in, s_in) && rec(e[kKQ], s_in);
-        if (backward) ok = ok && copy2d(a + Lo.dO + G.q * esz, (const char*)hdO + G.q * esz, q_pitch, q_width, L, in, s_in) && rec(e[kdO], s_in);
+        ok = copy2d(a + Lo.V + G.k * esz, (const char*)hV + G.k * esz, k_pitch, k_width, rows, in, s_in) && rec(e[kV], s_in) &&
+             copy2d(a + Lo.K + G.k * esz, (const char*)hK + G.k * esz, k_pitch, k_width, rows, in, s_in) &&
+             copy2d(a + Lo.Q + G.q * esz, (const char*)hQ + G.q * esz, q_pitch, q_width, rows, in, s_in) && rec(e[kKQ], s_in);
+        if (backward) ok = ok && copy2d(a + Lo.dO + G.q * esz, (const char*)hdO + G.q * esz, q_pitch, q_width, rows, in, s_in) && rec(e[kdO], s_in);
     }
     if (!ok) return cleanup(DMA_ERR_CUDA);
 
     dma_problem_t sub = *p;
-    sub.B = 1; sub.Hq = nqh; sub.Hkv = nkh;
+    sub.B = GB; sub.Hq = nqh; sub.Hkv = nkh;
     const int64_t qs[3] = {(int64_t)L * p->Hq * d, (int64_t)p->Hq * d, d}, ks[3] = {(int64_t)L * p->Hkv * d, (int64_t)p->Hkv * d, d};
     for (int i = 0; i < 3; ++i) { sub.q_stride[i] = sub.o_stride[i] = qs[i]; sub.k_stride[i] = sub.v_stride[i] = ks[i]; }
     const size_t f_ws = Lo.f_ws - (size_t)NG * kWsHeaderBytes, b_ws = Lo.b_ws - (size_t)NG * kWsHeaderBytes;
@@ -180,10 +191,10 @@ int dma_step_host(const dma_problem_t* p, int backward, const void* hQ, const vo
     for (int g = 0; g < NG; ++g) {
         const Group G = group_of(g);
         cudaEvent_t* e = ev + g * kPerGroup;
-        float* bias = (float*)(a + Lo.bias) + G.h;
-        int32_t* expiry = (int32_t*)(a + Lo.expiry) + G.h;
-        uint32_t* bitmap = (uint32_t*)(a + Lo.bitmap) + G.bmp;
-        float* lse = (float*)(a + Lo.lse) + G.h;
+        float* bias = (float*)(a + Lo.bias) + (size_t)g * Lo.gh;
+        int32_t* expiry = (int32_t*)(a + Lo.expiry) + (size_t)g * Lo.gh;
+        uint32_t* bitmap = (uint32_t*)(a + Lo.bitmap) + (size_t)g * Lo.gbmp;
+        float* lse = (float*)(a + Lo.lse) + (size_t)g * Lo.gh;
         char* wsf = a + Lo.ws_fwd + (size_t)g * kWsHeaderBytes;
         if (!wait(st, e[kV])) return cleanup(DMA_ERR_CUDA);
         if ((rc = dma_mask_build(&sub, a + Lo.V + G.k * esz, (float*)(a + Lo.W) + G.hq0 * w_per_head, (float*)(a + Lo.A) + G.hq0, bias,
@@ -193,20 +204,20 @@ int dma_step_host(const dma_problem_t* p, int backward, const void* hQ, const vo
                                a + Lo.O + G.q * esz, lse, wsf, f_ws, st))) return cleanup(rc);
         const cudaMemcpyKind out = cudaMemcpyDeviceToHost;
         ok = rec(e[kO], st) && wait(s_out, e[kO]) &&
-             copy2d((char*)hO + G.q * esz, a + Lo.O + G.q * esz, q_pitch, q_width, L, out, s_out) &&
-             cudaMemcpyAsync(hlse + G.h, lse, (size_t)nqh * L * 4, out, s_out) == cudaSuccess;
+             copy2d((char*)hO + G.q * esz, a + Lo.O + G.q * esz, q_pitch, q_width, rows, out, s_out) &&
+             cudaMemcpyAsync(hlse + G.h, lse, hl * 4, out, s_out) == cudaSuccess;
         if (backward) {
             char* wsb = a + Lo.ws_bwd + (size_t)g * kWsHeaderBytes;
-            float* dM = (float*)(a + Lo.dM) + G.h;
+            float* dM = (float*)(a + Lo.dM) + (size_t)g * Lo.gh;
             if (!ok || !wait(st, e[kdO])) return cleanup(DMA_ERR_CUDA);
             if ((rc = dma_attn_bwd(&sub, a + Lo.Q + G.q * esz, a + Lo.K + G.k * esz, a + Lo.V + G.k * esz, a + Lo.O + G.q * esz,
                                    a + Lo.dO + G.q * esz, lse, bias, expiry, bitmap, a + Lo.dQ + G.q * esz, a + Lo.dK + G.k * esz,
                                    a + Lo.dV + G.k * esz, dM, wsb, b_ws, st))) return cleanup(rc);
             ok = rec(e[kG], st) && wait(s_out, e[kG]) &&
-                 copy2d((char*)hdQ + G.q * esz, a + Lo.dQ + G.q * esz, q_pitch, q_width, L, out, s_out) &&
-                 copy2d((char*)hdK + G.k * esz, a + Lo.dK + G.k * esz, k_pitch, k_width, L, out, s_out) &&
-                 copy2d((char*)hdV + G.k * esz, a + Lo.dV + G.k * esz, k_pitch, k_width, L, out, s_out) &&
-                 cudaMemcpyAsync(hdM + G.h, dM, (size_t)nqh * L * 4, out, s_out) == cudaSuccess;
+                 copy2d((char*)hdQ + G.q * esz, a + Lo.dQ + G.q * esz, q_pitch, q_width, rows, out, s_out) &&
+                 copy2d((char*)hdK + G.k * esz, a + Lo.dK + G.k * esz, k_pitch, k_width, rows, out, s_out) &&
+                 copy2d((char*)hdV + G.k * esz, a + Lo.dV + G.k * esz, k_pitch, k_width, rows, out, s_out) &&
+                 cudaMemcpyAsync(hdM + G.h, dM, hl * 4, out, s_out) == cudaSuccess;
         }
         if (!ok) return cleanup(DMA_ERR_CUDA);
     }

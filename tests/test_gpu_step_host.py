@@ -35,6 +35,10 @@ def host_step(case, inp, flags=0, W=None):
     wl.small(C2, B=3, Hq=4, Hkv=2, L=333, w=50, backward=True, name="host bf16 ragged: batch groups only"),
     wl.small(C2, B=2, Hq=8, Hkv=4, L=512, w=64, backward=False, name="host bf16 forward only"),
     wl.small(C1, B=2, Hq=8, Hkv=2, L=256, w=64, name="host fp32"),
+    # Hq * L not a multiple of four: a batch entry's vectors would start off a 16-byte boundary inside [B, Hq, L] arrays
+    wl.small(C2, B=3, Hq=1, Hkv=1, L=333, w=64, backward=True, name="host bf16 one head, odd length"),
+    wl.small(C2, B=2, Hq=2, Hkv=2, L=1, w=64, d=64, backward=True, name="host bf16 single key"),
+    wl.small(C2, B=70, Hq=2, Hkv=1, L=130, w=20, backward=True, name="host bf16 more batch entries than groups"),
 ], ids=lambda c: c.name)
 def test_equals_the_device_entry_points(case):
     inp = wl.make_inputs(case)
