@@ -47,6 +47,7 @@ def test_static_scratch_rejects_oversized_problems():
     dev = torch.device("cuda:0")
     p = dma.problem(1, 32, 8, 65536, 128, 4096)      # 2 Mi sort keys: over the 1 Mi limit
     a = torch.empty(64, dtype=torch.float32, device=dev)
+    v = torch.empty(64, dtype=torch.bfloat16, device=dev)     # refused before anything is read
     with pytest.raises(dma.DmaError) as e:
-        dma.dma_mask_build_static(p, a, a, a, a, a.view(torch.int32), a.view(torch.int32))
+        dma.dma_mask_build_static(p, v, a, a, a, a.view(torch.int32), a.view(torch.int32))
     assert e.value.status == -5
