@@ -102,3 +102,47 @@ def test_arbitrary_interval_masks(seed):
             a, b = t.float(), ref[k].float()
             scale = max(1.0, float(b.abs().max()))
             assert float((a - b).abs().max()) <= (1e-3 if k == "lse" else 4e-2) * scale, (seed, flags, k, float((a - b).abs().max()), scale)
+
+
+def test_two_host_threads_on_two_streams():
+    """The library keeps no state between calls (workspaces are the caller's): two host threads, each on its own stream with
+    its own problem and workspaces, get the results of a serial run (O, lse, dK, dV bit for bit; dQ, dM within tolerance)."""
+    import threading
+    cases = [wl.small(wl.CONFIGS["2"], B=1, Hq=4, Hkv=2, L=1536, w=200, backward=True, seed=71, name="thread-a"),
+             wl.small(wl.CONFIGS["2"], B=2, Hq=2, Hkv=1, L=900, w=64, d=64, backward=True, seed=72, name="thread-b")]
+
+    def step(case, inp, flags):
+        p = dma.problem(case.B, case.Hq, case.Hkv, case.L, case.d, case.w, flags=flags)
+        mask = dma.dma_mask_build(p, inp["V"], inp["W_delta"], inp["A"])
+        O, lse = dma.dma_attn_fwd(p, inp["Q"], inp["K"], inp["V"], *mask)
+        g = dma.dma_attn_bwd(p, inp["Q"], inp["K"], inp["V"], O, inp["dO"], lse, *mask)
+        return dict(zip(("O", "lse", "dQ", "dK", "dV", "dM"), (O, lse) + tuple(g)))
+
+    inps = [{k: v.to(DEV) for k, v in wl.make_inputs(c).items() if isinstance(v, torch.Tensor)} for c in cases]
+    serial = [[step(c, i, f) for f in (0, dma.DMA_FLAG_COMPACT_KV)] for c, i in zip(cases, inps)]
+    torch.cuda.synchronize()
+    errors = []
+
+    def worker(idx):
+        try:
+            with torch.cuda.stream(torch.cuda.Stream()):
+                for rep in range(12):
+                    for f, ref in zip((0, dma.DMA_FLAG_COMPACT_KV), serial[idx]):
+                        out = step(cases[idx], inps[idx], f)
+                        torch.cuda.current_stream().synchronize()
+                        for k in ("O", "lse", "dK", "dV"):
+                            if not torch.equal(out[k], ref[k]):
+                                errors.append((idx, rep, f, k))
+                        for k in ("dQ", "dM"):
+                            a, b = out[k].float(), ref[k].float()
+                            if float((a - b).abs().max()) > 2e-2 * max(1.0, float(b.abs().max())):
+                                errors.append((idx, rep, f, k))
+        except Exception as ex:                                   # surfaced in the main thread below
+            errors.append((idx, repr(ex)))
+
+    threads = [threading.Thread(target=worker, args=(i,)) for i in range(2)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    assert not errors, errors[:5]
