@@ -138,7 +138,7 @@ def main():
     ap.add_argument("--workload", default="3", help="key of workloads.CONFIGS (3 = 16K training step, the headline)")
     ap.add_argument("--impl", default="dma", choices=["dma", "reference"])
     ap.add_argument("--ref-rows", type=int, default=4096, help="rows of the oracle sample per step (--impl reference)")
-    ap.add_argument("--cpu-rows", type=int, default=8192, help="rows of the oracle sample for cpu_baseline (0 = skip)")
+    ap.add_argument("--cpu-rows", type=int, default=16384, help="rows of the oracle sample for cpu_baseline (0 = skip)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--flags", type=int, default=0, help="dma_problem_t.flags (1 = ignore the bitmap, 2 = CUDA-core kernels)")
     ap.add_argument("--seq-len", type=int, default=0, help="override the workload's sequence length (profiling of a smaller case)")
