@@ -164,7 +164,9 @@ int dma_attn_fwd_chunk(const dma_problem_t* p, int32_t q_begin, int32_t q_len, c
  *   D_i = dO_i . O_i;  p_ij = exp(s_ij - lse_i);  dP_ij = dO_i . v_j;  dS_ij = p_ij (dP_ij - D_i)
  *   dV_j = sum_i p_ij dO_i;  dK_j = scale sum_i dS_ij q_i;  dQ_i = scale sum_j dS_ij k_j;  dM[b,h,j] = sum_i dS_ij
  * dK and dV are summed over the Hq/Hkv query heads that share a KV head; dM is per query head.
- * dQ is accumulated with floating-point atomics: its rounding depends on execution order. */
+ * dQ is accumulated with floating-point atomics: its rounding depends on execution order. dK, dV (and O, lse of the
+ * forward) are reproducible bit for bit from run to run on the tile path and the CUDA-core path; with
+ * DMA_FLAG_COMPACT_KV dK and dV are accumulated with atomics too (one CTA per query head) and vary in the last bits. */
 int dma_attn_bwd(const dma_problem_t* p, const void* Q, const void* K, const void* V,
                  const void* O, const void* dO, const float* lse,
                  const float* bias, const int32_t* expiry, const uint32_t* bitmap,
