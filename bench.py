@@ -28,7 +28,7 @@ METRIC = "dma_fwd_bwd_executed_tile_tflops"
 NOMINAL_BF16_TFLOPS = 2250.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from one ncu capture of this
 # command at full size (profiles/dram_traffic_cfg3_train16k.md); other workloads: not captured.
-NCU_TRAFFIC_BYTES = {"cfg3-train-16k": {"bwd": 3.62e9, "fwd": 0.513e9}}
+NCU_TRAFFIC_BYTES = {"cfg3-train-16k": {"bwd": 1.12e9, "fwd": 0.511e9}}
 
 
 def tile_flops(active_tiles, d, backward, bm=128, bn=128):
