@@ -714,15 +714,15 @@ int launch_tc_bwd(const Prob& P, const void* Q, const void* K, const void* V, co
     bp.B = P.B; bp.Hq = P.Hq; bp.Hkv = P.Hkv; bp.G = P.G; bp.L = P.L; bp.Tr = P.Tr; bp.Tc = P.Tc; bp.Wd = P.Wd;
     bp.ignore_bitmap = (P.flags & DMA_FLAG_IGNORE_BITMAP) ? 1 : 0;
     {
-        // CTA start order (tile path): all key tiles of a few (batch, KV head) entries before the next few, so that the
+        // CTA start order: all key tiles of a few (batch, KV head) entries before the next few, so that the
         // rows those CTAs stream (Q, dO) and add to (the fp32 dQ accumulator: 8 bytes per element and query head in all)
         // stay in L2 while they are in use. About 160 MB of such rows per group was the best of the orders measured at
         // L = 16384 with 32 / 8 heads (two KV heads per group: 1.3 % faster in a long run than all eight at once; one
         // KV head per group starts the heaviest CTAs of the last group too late).
         const int gx = compact ? P.B * P.Hq : P.B * P.Hkv;
         int sg = gx;
-        if (!compact) {
-            const double per_entry = (double)P.G * P.L * 128 * 8;
+        {
+            const double per_entry = (double)(compact ? 1 : P.G) * P.L * 128 * 8;     // token-compacted mode: an entry is one query head
             int want = (int)(160.0 * 1024 * 1024 / per_entry);
             want = want < 1 ? 1 : want;
             for (sg = want < gx ? want : gx; gx % sg; --sg) {}
