@@ -215,6 +215,24 @@ def backward(Q, K, V, dO, bias, expiry=None, keep=None, scale=None, keys=None, w
     return dQ, dK, dV, dM
 
 
+def backward_dq_rows(Q, K, V, dO, bias, rows, expiry=None, keep=None, scale=None, dtype=np.float64, O=None, causal=True):
+    """dQ of Sec. 4.3 (Eq. grad_qk) on the listed query rows only (dQ_i depends on row i alone): [B,len(rows),Hq,d].
+    ``O`` is the stored forward output of those rows, compact [B,len(rows),Hq,d], that Alg. 2 reads for D; None = the
+    exact output."""
+    Q = _c(Q, dtype); K = _c(K, dtype); V = _c(V, dtype); dO = _c(dO, dtype); bias = _c(bias, dtype); O = _c(O, dtype)
+    expiry = _c(expiry, np.int32); keep = _c(keep, np.uint8); rows = _c(rows, np.int32)
+    B, L, Hq, d = Q.shape
+    Hkv = K.shape[2]
+    scale = d ** -0.5 if scale is None else scale
+    assert O is None or O.shape == (B, len(rows), Hq, d)
+    dQ = np.empty((B, len(rows), Hq, d), dtype)
+    f = lib().dmao_dq_rows_f64 if dtype == np.float64 else lib().dmao_dq_rows_f32
+    rc = f(_p(Q), _p(K), _p(V), _p(O), _p(dO), _p(bias), _p(expiry), _p(keep), B, L, Hq, Hkv, d,
+           ctypes.c_double(scale), _p(rows), len(rows), _p(dQ), int(bool(causal)))
+    assert rc == 0, rc
+    return dQ
+
+
 def mask_backward(V, W, A, dM, Hq):
     """Gradient of the mask-generation bias path (Sec. 4.3: the bias gradient dM reaches the sampling weights and
     the gate; Eq. delta_calc differentiated with the top-w selection held fixed). Plain numpy, fp64:

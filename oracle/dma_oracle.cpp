@@ -286,6 +286,44 @@ int backward(const Problem<T>& P, const T* Ostored, const T* dO, const int32_t* 
     return 0;
 }
 
+// dQ of Sec. 4.3 (Eq. grad_qk, first line) on a subset of query rows. dQ_i depends on row i alone:
+// dQ_i = scale * sum_{j in I_i} dS_ij k_j with dS_ij = p_ij (dO_i . v_j - D_i), D_i = dO_i . O_i (Alg. 2 reads
+// the stored O: Ostored holds it for the listed rows, compact [B,nrows,Hq,d]; null = the exact o of this row).
+// The same statements as pass 1 of `backward`, restricted to the listed rows; output compact [B,nrows,Hq,d].
+template <class T>
+int backward_dq_rows(const Problem<T>& P, const T* Ostored, const T* dO, const int32_t* rows, int nrows, T* dQ) {
+    const int L = P.L, d = P.d, Hq = P.Hq, G = P.G();
+    const long total = (long)P.B * Hq * nrows;
+#pragma omp parallel
+    {
+        std::vector<int> idx;
+        std::vector<T> p, o(d);
+#pragma omp for schedule(dynamic, 1)
+        for (long t = 0; t < total; ++t) {
+            int r = (int)(t % nrows);
+            int h = (int)((t / nrows) % Hq);
+            int b = (int)(t / ((long)nrows * Hq));
+            const int i = rows[r], hk = h / G;
+            row_forward(P, b, h, i, idx, p, o.data(), (T*)nullptr);
+            const T* doi = dO + (((size_t)b * L + i) * Hq + h) * d;
+            const T* oi = Ostored ? Ostored + (((size_t)b * nrows + r) * Hq + h) * d : o.data();
+            T Di = 0;
+            for (int c = 0; c < d; ++c) Di += doi[c] * oi[c];
+            T* dqi = dQ + (((size_t)b * nrows + r) * Hq + h) * d;
+            for (int c = 0; c < d; ++c) dqi[c] = 0;
+            for (size_t u = 0; u < idx.size(); ++u) {
+                const T* vj = P.v(b, idx[u], hk);
+                const T* kj = P.k(b, idx[u], hk);
+                T dp = 0;
+                for (int c = 0; c < d; ++c) dp += doi[c] * vj[c];
+                T ds = p[u] * (dp - Di);
+                for (int c = 0; c < d; ++c) dqi[c] += ds * kj[c] * P.scale;
+            }
+        }
+    }
+    return 0;
+}
+
 template <class T>
 Problem<T> make_problem(int B, int L, int Hq, int Hkv, int d, double scale, const T* Q, const T* K,
                         const T* V, const T* bias, const int32_t* expiry, const uint8_t* keep, int causal) {
@@ -460,5 +498,16 @@ DMAO_FWD(dmao_fwd_f64, double)
     }
 DMAO_BWD(dmao_bwd_f32, float)
 DMAO_BWD(dmao_bwd_f64, double)
+
+#define DMAO_DQ_ROWS(NAME, T)                                                                        \
+    int NAME(const T* Q, const T* K, const T* V, const T* Ostored, const T* dO, const T* bias,       \
+             const int32_t* expiry, const uint8_t* keep, int B, int L, int Hq, int Hkv, int d, double scale, \
+             const int32_t* rows, int nrows, T* dQ, int causal) {                                    \
+        if (Hq % Hkv || (!expiry && !keep) || !rows) return -1;                                      \
+        return backward_dq_rows<T>(make_problem<T>(B, L, Hq, Hkv, d, scale, Q, K, V, bias, expiry, keep, causal), \
+                                   Ostored, dO, rows, nrows, dQ);                                    \
+    }
+DMAO_DQ_ROWS(dmao_dq_rows_f32, float)
+DMAO_DQ_ROWS(dmao_dq_rows_f64, double)
 
 }  // extern "C"

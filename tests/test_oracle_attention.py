@@ -213,6 +213,23 @@ def test_backward_key_subset_equals_full():
     assert (dKs == dK[:, keys]).all() and (dVs == dV[:, keys]).all() and (dMs == dM[:, :, keys]).all()
 
 
+def test_backward_dq_row_subset_equals_full():
+    # dQ_i depends on row i alone: the row-subset routine must reproduce the rows of the full backward (itself pinned by
+    # finite differences above), with the exact O and with a stored (here: perturbed) O
+    Q, K, V, dO, bias, e = rand_case(12)
+    rows = np.array([0, 1, 17, 40, Q.shape[1] - 1], np.int32)
+    dQ = oracle.backward(Q, K, V, dO, bias, expiry=e)[0]
+    assert (oracle.backward_dq_rows(Q, K, V, dO, bias, rows, expiry=e) == dQ[:, rows]).all()
+    O, _ = oracle.forward(Q, K, V, bias, expiry=e)
+    O2 = O + 0.01 * np.cos(np.arange(O.size)).reshape(O.shape)
+    dQ2 = oracle.backward(Q, K, V, dO, bias, expiry=e, O=O2)[0]
+    got = oracle.backward_dq_rows(Q, K, V, dO, bias, rows, expiry=e, O=O2[:, rows])
+    assert (got == dQ2[:, rows]).all() and np.abs(dQ2 - dQ).max() > 1e-6
+    # definition form (keep matrix) and non-causal mode go through the same routine
+    keep = oracle.keep_from_expiry(e)
+    assert (oracle.backward_dq_rows(Q, K, V, dO, bias, rows, keep=keep) == dQ[:, rows]).all()
+
+
 def test_backward_with_stored_output():
     # Alg. 2 reads O back from memory for D = rowsum(dO o O): passing the exact O changes nothing; passing a
     # perturbed O moves D by dO.(O' - O) and hence dS by -p * that, which for dM (column sums of dS) is checkable.
