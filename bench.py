@@ -26,9 +26,27 @@ from paper_2508_02124_b200 import workloads as wl  # noqa: E402
 
 METRIC = "dma_fwd_bwd_executed_tile_tflops"
 NOMINAL_BF16_TFLOPS = 2250.0
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from one ncu capture of this
-# command at full size (profiles/dram_traffic_cfg3_train16k.md); other workloads: not captured.
-NCU_TRAFFIC_BYTES = {"cfg3-train-16k": {"bwd": 1.12e9, "fwd": 0.511e9}}
+
+
+def ncu_traffic(workload, kernel):
+    """dram__bytes_read.sum + dram__bytes_write.sum per launch of a kernel on a workload, from the ncu captures
+    summarised in profiles/dram_traffic.json; None where nothing was captured."""
+    try:
+        with open(os.path.join(ROOT, "profiles", "dram_traffic.json")) as f:
+            return json.load(f).get(workload, {}).get(kernel)
+    except (OSError, ValueError):
+        return None
+
+
+def algorithmic_bytes(case, kernel):
+    """Lower bound of the HBM traffic of one launch: every input read once, every output written once."""
+    e = 2 if case.dtype == "bf16" else 4
+    q = case.B * case.L * case.Hq * case.d * e
+    kv = case.B * case.L * case.Hkv * case.d * e
+    rows = case.B * case.Hq * case.L * 4
+    if kernel == "fwd":
+        return 2 * q + 2 * kv + 3 * rows                      # Q, O; K, V; bias, expiry, lse
+    return 2 * q + 2 * kv + 2 * kv + 4 * rows + 2 * case.B * case.L * case.Hq * case.d * 4   # Q, dO; K, V; dK, dV; bias, expiry, lse, D, dM; fp32 dQ accumulator read + written
 
 
 def tile_flops(active_tiles, d, backward, bm=128, bn=128):
@@ -80,9 +98,10 @@ class ClockSampler:
             return out
         sm = sorted(float(r[0]) for r in rows)
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        reasons = [n for k, n in enumerate(names) if any("Active" in r[3 + k] and "Not" not in r[3 + k] for r in rows)]
+        on = lambda r, k: "Active" in r[3 + k] and "Not" not in r[3 + k]
+        reasons = [n for k, n in enumerate(names) if any(on(r, k) for r in rows)]
         out.update(sm_mhz=sm[len(sm) // 2], sm_max_mhz=float(rows[0][1]), reasons=reasons, samples=len(rows),
-                   power_w_max=max(float(r[2]) for r in rows))
+                   power_w_max=max(float(r[2]) for r in rows), power_cap_frac=sum(on(r, 3) for r in rows) / len(rows))
         return out
 
 
@@ -165,7 +184,10 @@ def main():
         dist.init_process_group("nccl", device_id=dev)
 
     inp = wl.make_inputs(case)
-    p = dma.problem(case.B, case.Hq, case.Hkv, case.L, case.d, case.w, dtype=case.torch_dtype, flags=args.flags)
+    # the headline metric (TFLOP/s on executed tiles) is defined on the tile-walking kernels: DMA_FLAG_TILE_PATH; what the
+    # library runs when left to choose is timed below as `best_path`
+    tile_flag = dma.DMA_FLAG_TILE_PATH if not (args.flags & (dma.DMA_FLAG_COMPACT_KV | dma.DMA_FLAG_SIMT)) and case.causal else 0
+    p = dma.problem(case.B, case.Hq, case.Hkv, case.L, case.d, case.w, dtype=case.torch_dtype, flags=args.flags | tile_flag)
     Q, K, V, dO, W, A = (inp[k].to(dev) for k in ("Q", "K", "V", "dO", "W_delta", "A"))
     m_ws, f_ws, b_ws = dma.dma_query_workspace(p)
     ws_m, ws_f, ws_b = (torch.empty(n, dtype=torch.uint8, device=dev) for n in (m_ws, f_ws, b_ws))
@@ -207,10 +229,16 @@ def main():
     launches0 = dma.dma_launch_count()
     t0, t1 = ev(), ev()
     barrier()
+    dma.dma_kernel_timing(True)            # event pairs around fwd_kernel / bwd_kernel alone (the library's measurement hook)
     t0.record()
     evs = [step(timed=True) for _ in range(args.steps)]
     t1.record()
     barrier()
+    dma.dma_kernel_timing(False)
+    kernel_ms = {"fwd": [], "bwd": []}
+    for stage, t_ms in dma.dma_kernel_timing_read():
+        kernel_ms[stage].append(t_ms)
+    kernel_ms = {k: (sum(v) / len(v) if v else None) for k, v in kernel_ms.items()}
     launches = dma.dma_launch_count() - launches0
     clocks = sampler.stop() if sampler else None
     total_ms = t0.elapsed_time(t1)
@@ -310,6 +338,38 @@ def main():
             compact.update({"bwd_ms": cb_ms, "tile_bwd_ms": stage_ms["bwd"], "bwd_speedup_over_tile_skipping": stage_ms["bwd"] / cb_ms,
                             "step_ms": stage_ms["mask"] + c_ms + cb_ms, "tile_step_ms": sum(stage_ms.values()),
                             "dK_max_abs_diff_vs_tile_path": float((dKc.float() - dK.float()).abs().max())})
+
+    # ---- the step as a caller gets it with default flags: the library picks tile-walking or token-compacted kernels from the
+    # descriptor (w against L); timed like the headline step, reported as wall time and as TFLOP/s on kept (row, key) pairs
+    best_path = None
+    if not (args.flags & (dma.DMA_FLAG_COMPACT_KV | dma.DMA_FLAG_TILE_PATH)):
+        pa = dma.problem(case.B, case.Hq, case.Hkv, case.L, case.d, case.w, dtype=case.torch_dtype, flags=args.flags)
+        sizes_a = dma.dma_query_workspace(pa)
+        ws_am, ws_af, ws_ab = (torch.empty(n, dtype=torch.uint8, device=dev) for n in sizes_a)
+        Oa, lsea = torch.empty_like(O), torch.empty_like(lse)
+        dQa, dKa, dVa, dMa = torch.empty_like(dQ), torch.empty_like(dK), torch.empty_like(dV), torch.empty_like(dM)
+
+        def step_a():
+            dma.dma_mask_build(pa, V, W, A, bias, expiry, bitmap, ws_am)
+            dma.dma_attn_fwd(pa, Q, K, V, bias, expiry, bitmap, Oa, lsea, ws_af)
+            if case.backward:
+                dma.dma_attn_bwd(pa, Q, K, V, Oa, dO, lsea, bias, expiry, bitmap, dQa, dKa, dVa, dMa, ws_ab)
+
+        for _ in range(3):
+            step_a()
+        n_a = max(3, min(args.steps, 20))
+        a0, a1 = ev(), ev()
+        barrier()
+        a0.record()
+        for _ in range(n_a):
+            step_a()
+        a1.record()
+        barrier()
+        assert dma.dma_read_status(ws_af) == 0 and (not case.backward or dma.dma_read_status(ws_ab) == 0), "device status (default flags)"
+        a_ms = replicas.max_over_ranks(a0.elapsed_time(a1) / n_a, dev)
+        best_path = {"ms_per_step": a_ms, "path": "tile" if sizes_a[1] == dma.dma_query_workspace(p)[1] else "token-compacted",
+                     "useful_tflops": world * useful_flops / (a_ms * 1e-3) / 1e12,
+                     "speedup_over_tile_path": ms / a_ms, "max_abs_diff_O_vs_tile_path": float((Oa.float() - O.float()).abs().max())}
 
     # ---- the same tensors read as 12 documents packed along the sequence axis (dma_mask_build_varlen; the attention
     # kernels are unchanged): the bitmap becomes block-diagonal and tile skipping removes the other documents' tiles
@@ -517,9 +577,30 @@ def main():
     flops = tile_flops(active, case.d, case.backward)
     value = world * flops / (ms * 1e-3) / 1e12
     dom = "bwd" if case.backward else "fwd"
-    dom_flops = tile_flops(active, case.d, False) * (2.5 if case.backward else 1.0)
-    achieved = dom_flops / (stage_ms[dom] * 1e-3) / 1e12
     tensor_path = case.dtype == "bf16" and case.d == 128 and not (args.flags & dma.DMA_FLAG_SIMT)
+    # Roofline of the dominant KERNEL (its own event pair, not the stage with its small pre / post kernels). The denominator
+    # follows the clocks sampled during the timed region: the burst cuBLAS peak when the run was not power-capped (median SM
+    # clock near the maximum, sw_power_cap active in a minority of samples), the sustained one otherwise; both fractions are printed.
+    kflops = {"fwd": tile_flops(active, case.d, False), "bwd": tile_flops(active, case.d, False) * 2.5}
+    capped = bool(clocks and clocks.get("sm_mhz") and (clocks["sm_mhz"] < 0.95 * clocks["sm_max_mhz"] or clocks.get("power_cap_frac", 0.0) > 0.5))
+    peak_kind = "sustained" if capped else "burst"
+    peak = pk["bf16_sustained"] if capped else pk["bf16_burst"]
+
+    def kernel_roofline(kind):
+        t_ms = kernel_ms.get(kind) or stage_ms[kind]
+        ach = kflops[kind] / (t_ms * 1e-3) / 1e12
+        return {"bound": "tensor" if tensor_path else "alu", "kernel": f"{kind}_kernel", "ms": t_ms,
+                "timed": "event pair around the kernel alone" if kernel_ms.get(kind) else "stage time",
+                "achieved": ach, "peak": peak, "peak_source": f"{pk['source']} {peak_kind} cuBLAS bf16 (chosen from the sampled clocks)",
+                "unit": "TFLOP/s", "frac": ach / peak, "frac_burst": ach / pk["bf16_burst"], "frac_sustained": ach / pk["bf16_sustained"],
+                "frac_nominal": ach / NOMINAL_BF16_TFLOPS,
+                "traffic": ncu_traffic(case.name, kind + "_kernel") if tensor_path else None,
+                "algorithmic_bytes": algorithmic_bytes(case, kind)}
+
+    roofline = kernel_roofline(dom)
+    if case.backward:
+        roofline["forward"] = kernel_roofline("fwd")
+    dom_flops = kflops[dom]
     out = {
         "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -530,14 +611,13 @@ def main():
         "stage_ms": stage_ms, "active_tiles": active, "causal_tiles": causal_tiles(case),
         "executed_tile_tflop_per_step": flops / 1e12,
         "frac_of_nominal_bf16_peak": value / world / NOMINAL_BF16_TFLOPS,
-        "frac_of_measured_bf16_peak": value / world / pk["bf16_sustained"],
+        "frac_of_measured_bf16_peak": value / world / peak, "measured_peak_used": peak_kind,
+        "frac_of_measured_bf16_burst_peak": value / world / pk["bf16_burst"],
+        "frac_of_measured_bf16_sustained_peak": value / world / pk["bf16_sustained"],
         "fwd_tflops": tile_flops(active, case.d, False) / (stage_ms["fwd"] * 1e-3) / 1e12,
         "bwd_tflops": (dom_flops / (stage_ms["bwd"] * 1e-3) / 1e12) if case.backward else None,
         "dense_causal_equivalent_speedup": causal_tiles(case) / max(active, 1),
-        "roofline": {"bound": "tensor" if tensor_path else "alu", "kernel": f"dma_attn_{dom} (stage time, includes its pre/post kernels)",
-                     "achieved": achieved, "peak": pk["bf16_sustained"], "peak_source": pk["source"] + " sustained cuBLAS bf16",
-                     "unit": "TFLOP/s", "frac": achieved / pk["bf16_sustained"],
-                     "traffic": NCU_TRAFFIC_BYTES.get(case.name, {}).get(dom) if tensor_path else None},
+        "roofline": roofline, "kernel_ms": kernel_ms,
         "gpu_launches": launches, "clocks": clocks, "e2e": e2e,
         "step_ms": step_stats, "kept_pairs": kept_pairs, "useful_tflop_per_step": useful_flops / 1e12,
         "useful_tflops": world * useful_flops / (ms * 1e-3) / 1e12,
@@ -545,6 +625,8 @@ def main():
     if decode is not None:
         decode["frac_of_measured_hbm"] = decode["gbs"] / pk["hbm_gbs"]
         out["decode"] = decode
+    if best_path is not None:
+        out["best_path"] = best_path
     if compact is not None:
         out["compact"] = compact
     if full_delta is not None:

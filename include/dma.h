@@ -8,9 +8,11 @@
  *
  * Conventions
  *   - Unless a parameter is marked HOST, every pointer is a DEVICE pointer owned by the caller, 16-byte
- *     aligned. The library allocates no device memory, keeps no state between calls, enqueues work only
- *     on the caller's stream (a cudaStream_t passed as void*; NULL = default stream) and does not
- *     synchronise, except in dma_read_status and dma_step_host.
+ *     aligned. The library allocates no device memory, enqueues work only on the caller's stream (a
+ *     cudaStream_t passed as void*; NULL = default stream) and does not synchronise, except in
+ *     dma_read_status and dma_step_host. What it keeps between calls is bookkeeping only: the process-wide
+ *     launch counter behind dma_launch_count, and for dma_mask_build_static the fixed scratch array in the
+ *     device image with its per-device address; no result depends on an earlier call.
  *   - Element type of Q,K,V,O,dO,dQ,dK,dV is `dtype` (bf16 or fp32). bias, lse, dM, W_delta, A are fp32.
  *   - Q,O,dO,dQ are [B, L, Hq, d]; K,V,dK,dV are [B, L, Hkv, d]; d is contiguous; the batch, sequence and
  *     head strides are given in elements in the problem descriptor (0 = contiguous default). bias, expiry,
@@ -40,7 +42,10 @@ typedef enum {
     DMA_ERR_UNSUPPORTED = -4,    /* valid request outside what is implemented (see each call)       */
     DMA_ERR_WORKSPACE = -5,      /* workspace NULL or smaller than dma_query_workspace reports      */
     DMA_ERR_CUDA = -6,           /* a CUDA runtime / driver call failed (launch, descriptor, device)*/
-    DMA_ERR_DEVICE_TIMEOUT = -7  /* a bounded device-side wait gave up (read via dma_read_status)    */
+    DMA_ERR_DEVICE_TIMEOUT = -7, /* a bounded device-side wait gave up (read via dma_read_status)    */
+    DMA_ERR_MASK_OVERFLOW = -8   /* token-compacted execution met a mask that keeps more than w keys in a row: the
+                                    gathered key lists are sized for w (read via dma_read_status; the outputs of
+                                    that call are not valid)                                          */
 } dma_status;
 
 enum { DMA_BF16 = 0, DMA_FP32 = 1 };
@@ -50,7 +55,7 @@ enum {
     DMA_FLAG_IGNORE_BITMAP = 1,  /* visit every causal tile regardless of the bitmap (result must not change:
                                     block skipping is an optimisation only, Sec. 4.2 last paragraph)           */
     DMA_FLAG_SIMT = 2,           /* run the CUDA-core kernels also for bf16 (they always serve fp32)            */
-    DMA_FLAG_COMPACT_KV = 4,     /* dma_attn_fwd and dma_attn_bwd, bf16, d = 128: token-compacted
+    DMA_FLAG_COMPACT_KV = 4,     /* dma_attn_fwd and dma_attn_bwd, bf16: token-compacted
                                     execution (Sec. 3.3, computational sparsity: O(L w d) instead of O(L^2 d) work).
                                     Forward: each pair of query tiles gathers only the keys that one of its 256 rows
                                     keeps (at most w + 256) instead of walking every active 128-key tile. Backward: a CTA
@@ -60,7 +65,18 @@ enum {
                                     results up to rounding; needs the larger workspaces dma_query_workspace reports for
                                     it; ignores the bitmap. The mask must keep at most w keys per row, as every mask
                                     of dma_mask_build does (an injected mask that keeps more needs p->w raised to its
-                                    largest per-row count: the gathered lists are sized w + 256) */
+                                    largest per-row count: the gathered lists are sized w + 256; a list that overflows
+                                    leaves DMA_ERR_MASK_OVERFLOW in the workspace status word).
+                                    WITHOUT this flag and without DMA_FLAG_TILE_PATH the library chooses: causal bf16
+                                    problems on the tensor-core kernels with L >= 2048 and 4 w <= L run token-compacted
+                                    (there the tile-walking kernels spend most of their work on (row, key) pairs the mask
+                                    drops; from w = L/2 on the tile-walking kernels are the faster ones), everything else
+                                    walks tiles. The choice depends on the descriptor alone, so dma_query_workspace,
+                                    dma_attn_fwd and dma_attn_bwd agree on it */
+    DMA_FLAG_TILE_PATH = 16,     /* dma_attn_fwd and dma_attn_bwd: always walk the bitmap's active 128 x 128 tiles (Alg. 1 /
+                                    Alg. 2 with block skipping), never the token-compacted kernels. For masks whose kept
+                                    keys cluster (packed documents, banded importance) tile skipping alone can be the
+                                    faster choice; DMA_FLAG_IGNORE_BITMAP and DMA_FLAG_SIMT imply it */
     DMA_FLAG_FULL_DELTA = 8      /* the sampling weights as Eq. (delta_calc) states them: W_delta (and dW_delta) is
                                     [Hq, Hkv*d], one row per query head over ALL channels of the value row (the linear
                                     layer of the App. A listing), z[b,h,j] = sum_{h'} V[b,j,h',:] . W_delta[h, h'*d:(h'+1)*d].
@@ -121,7 +137,10 @@ int dma_mask_build(const dma_problem_t* p, const void* V, const float* W_delta, 
  *   Limit: B * Hq * roundup(L, 256) <= 1,048,576 sort keys; beyond that it returns DMA_ERR_WORKSPACE and launches
  *   nothing (use dma_mask_build with a caller-provided workspace instead).
  *   The first call on each device looks up the array's device address (that device must be current, as for
- *   every call); make that first call before starting any stream capture.
+ *   every call); make that first call before starting any stream capture. The address is remembered per device
+ *   ordinal for the life of the process: it belongs to the device's primary context, so a process that calls
+ *   cudaDeviceReset, or that runs this entry point under a context of its own (driver API) instead of the primary
+ *   one, must not use it afterwards (use dma_mask_build there).
  *   All calls on a device share the one array. Nothing in it has to start at zero (each call rewrites what it
  *   reads), but two calls whose kernels overlap on the GPU, from different streams or threads, race on it:
  *   serialise them. */
@@ -236,7 +255,8 @@ int dma_step_host(const dma_problem_t* p, int backward, const void* hQ, const vo
                   const float* hW_delta, const float* hA, void* hO, float* hlse, void* hdQ, void* hdK, void* hdV,
                   float* hdM, void* dev_arena, size_t arena_bytes, void* cuda_stream);
 
-/* Synchronises the stream and returns the device status word of a workspace (0 or DMA_ERR_DEVICE_TIMEOUT). */
+/* Synchronises the stream and returns the device status word of a workspace: 0, DMA_ERR_DEVICE_TIMEOUT or
+ * DMA_ERR_MASK_OVERFLOW. */
 int dma_read_status(const void* ws, void* cuda_stream);
 
 /* Self-test of the bounded device-side waits (every mbarrier wait in the kernels gives up after a cycle limit, raises
@@ -247,6 +267,16 @@ int dma_selftest_wait_timeout(void* ws, size_t ws_bytes, void* cuda_stream);
 
 /* Number of kernels the library has launched in this process (all entry points), for accounting. */
 long long dma_launch_count(void);
+
+/* Measurement hook (a property of the library; the paper has no counterpart). While recording is on, every dma_attn_fwd
+ * and dma_attn_bwd call brackets its MAIN kernel (the attention kernel itself, not the small kernels before and after it:
+ * key lists, D = rowsum(dO o O), accumulator conversion) with a pair of CUDA events on the caller's stream; up to 4096
+ * pairs are kept, in call order. dma_kernel_timing(1) discards earlier records and starts recording, dma_kernel_timing(0)
+ * stops. dma_kernel_timing_read waits for the recorded events and writes the elapsed milliseconds of each recorded
+ * launch to ms[] and its stage to which[] (0 = forward, 1 = backward), at most `capacity` of them; *count receives the
+ * number recorded. HOST pointers. Do not record while capturing a CUDA graph. */
+int dma_kernel_timing(int enable);
+int dma_kernel_timing_read(float* ms, int32_t* which, int32_t capacity, int32_t* count);
 
 const char* dma_strerror(int status);
 

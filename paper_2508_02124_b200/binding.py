@@ -14,13 +14,13 @@ LIB_PATH = os.path.join(_PKG, "libdma_b200.so")
 _lib = None
 
 DMA_BF16, DMA_FP32 = 0, 1
-DMA_FLAG_IGNORE_BITMAP, DMA_FLAG_SIMT, DMA_FLAG_COMPACT_KV, DMA_FLAG_FULL_DELTA = 1, 2, 4, 8
+DMA_FLAG_IGNORE_BITMAP, DMA_FLAG_SIMT, DMA_FLAG_COMPACT_KV, DMA_FLAG_FULL_DELTA, DMA_FLAG_TILE_PATH = 1, 2, 4, 8, 16
 
 ENTRY_POINTS = ("dma_query_workspace", "dma_bitmap_words", "dma_mask_build", "dma_attn_fwd", "dma_attn_bwd",
                 "dma_read_status", "dma_launch_count", "dma_strerror", "dma_step_host_arena", "dma_step_host", "dma_mask_build_static", "dma_selftest_wait_timeout",
                 "dma_mask_bwd_workspace", "dma_mask_bwd", "dma_delta_range", "dma_decode_workspace", "dma_decode",
                 "dma_mask_build_varlen", "dma_decode_state_bytes", "dma_decode_state_init", "dma_decode_step",
-                "dma_attn_fwd_chunk")
+                "dma_attn_fwd_chunk", "dma_kernel_timing", "dma_kernel_timing_read")
 
 
 class DmaError(RuntimeError):
@@ -290,6 +290,20 @@ def dma_read_status(ws):
 
 def dma_launch_count():
     return lib().dma_launch_count()
+
+
+def dma_kernel_timing(enable):
+    """Starts (discarding earlier records) or stops the recording of event pairs around each attention call's main kernel."""
+    _check(lib().dma_kernel_timing(int(bool(enable))), "dma_kernel_timing")
+
+
+def dma_kernel_timing_read(capacity=4096):
+    """[(stage, ms), ...] of the launches recorded so far, in call order; stage is "fwd" or "bwd"."""
+    ms = (ctypes.c_float * capacity)()
+    which = (ctypes.c_int32 * capacity)()
+    n = ctypes.c_int32()
+    _check(lib().dma_kernel_timing_read(ms, which, capacity, ctypes.byref(n)), "dma_kernel_timing_read")
+    return [("bwd" if which[i] else "fwd", float(ms[i])) for i in range(min(n.value, capacity))]
 
 
 def dma_step_host_arena(p, backward):

@@ -1,6 +1,8 @@
 // C-ABI entry points (include/dma.h): argument validation, defaults, dispatch to the stage launchers.
 #include <atomic>
 #include <cmath>
+#include <mutex>
+#include <vector>
 
 #include "common.cuh"
 #include "sm100_ptx.cuh"
@@ -10,6 +12,35 @@ namespace dma {
 static std::atomic<long long> g_launches{0};
 void count_launch(int n) { g_launches += n; }
 int check_launch() { return cudaGetLastError() == cudaSuccess ? DMA_OK : DMA_ERR_CUDA; }
+
+// ---- dma_kernel_timing: event pairs around the main kernel of each attention call while recording is on ----------
+namespace {
+struct TimedLaunch { cudaEvent_t before, after; int which; bool closed; };
+constexpr size_t kMaxTimed = 4096;
+std::mutex g_timing_mutex;
+std::vector<TimedLaunch> g_timed;
+std::atomic<bool> g_timing_on{false};
+void timing_clear() {
+    for (TimedLaunch& t : g_timed) { cudaEventDestroy(t.before); cudaEventDestroy(t.after); }
+    g_timed.clear();
+}
+}  // namespace
+
+void timing_mark(int which, bool after, cudaStream_t st) {
+    if (!g_timing_on.load(std::memory_order_relaxed)) return;
+    std::lock_guard<std::mutex> lock(g_timing_mutex);
+    if (!after) {
+        if (g_timed.size() >= kMaxTimed) return;
+        TimedLaunch t{nullptr, nullptr, which, false};
+        if (cudaEventCreate(&t.before) != cudaSuccess) return;
+        if (cudaEventCreate(&t.after) != cudaSuccess) { cudaEventDestroy(t.before); return; }
+        cudaEventRecord(t.before, st);
+        g_timed.push_back(t);
+    } else if (!g_timed.empty() && !g_timed.back().closed && g_timed.back().which == which) {
+        cudaEventRecord(g_timed.back().after, st);
+        g_timed.back().closed = true;
+    }
+}
 
 static bool fill_strides(const int64_t in[3], int64_t out[3], int L, int H, int d) {
     if (in[0] == 0 && in[1] == 0 && in[2] == 0) {
@@ -45,9 +76,18 @@ int resolve(const dma_problem_t* p, Prob* o) {
     if (!fill_strides(p->q_stride, o->qs, p->L, p->Hq, p->d) || !fill_strides(p->k_stride, o->ks, p->L, p->Hkv, p->d) ||
         !fill_strides(p->v_stride, o->vs, p->L, p->Hkv, p->d) || !fill_strides(p->o_stride, o->os, p->L, p->Hq, p->d))
         return DMA_ERR_ALIGN;
-    // non-causal: all rows of a head keep the same keys, so the tensor-core path always runs token-compacted
-    if (!o->causal && o->dtype == DMA_BF16 && o->bm == 128 && o->bn == 128 && !(o->flags & DMA_FLAG_SIMT))
+    const bool tc_shape = o->dtype == DMA_BF16 && o->bm == 128 && o->bn == 128 && !(o->flags & DMA_FLAG_SIMT);
+    if (o->flags & DMA_FLAG_IGNORE_BITMAP) o->flags |= DMA_FLAG_TILE_PATH;
+    if ((o->flags & DMA_FLAG_TILE_PATH) && (o->flags & DMA_FLAG_COMPACT_KV)) return DMA_ERR_UNSUPPORTED;
+    if (!o->causal && tc_shape) {
+        // non-causal: all rows of a head keep the same keys, so the tensor-core path always runs token-compacted
+        if (o->flags & DMA_FLAG_TILE_PATH) return DMA_ERR_UNSUPPORTED;
         o->flags |= DMA_FLAG_COMPACT_KV;
+    } else if (tc_shape && !(o->flags & (DMA_FLAG_COMPACT_KV | DMA_FLAG_TILE_PATH)) && o->L >= 2048 && 4ll * o->w <= o->L) {
+        // the library's choice (a function of the descriptor alone): with a window of at most a quarter of the
+        // sequence the token-compacted kernels do O(L w d) work where walking tiles does O(L^2 d) on scattered masks
+        o->flags |= DMA_FLAG_COMPACT_KV;
+    }
     return DMA_OK;
 }
 
@@ -363,7 +403,7 @@ int dma_read_status(const void* ws, void* cuda_stream) {
     cudaStream_t st = (cudaStream_t)cuda_stream;
     if (cudaMemcpyAsync(&word, ws, sizeof(word), cudaMemcpyDeviceToHost, st) != cudaSuccess) return DMA_ERR_CUDA;
     if (cudaStreamSynchronize(st) != cudaSuccess) return DMA_ERR_CUDA;
-    return word == 0 ? DMA_OK : DMA_ERR_DEVICE_TIMEOUT;
+    return word == 0 ? DMA_OK : word == DMA_ERR_MASK_OVERFLOW ? DMA_ERR_MASK_OVERFLOW : DMA_ERR_DEVICE_TIMEOUT;
 }
 
 int dma_selftest_wait_timeout(void* ws, size_t ws_bytes, void* cuda_stream) {
@@ -379,6 +419,30 @@ int dma_selftest_wait_timeout(void* ws, size_t ws_bytes, void* cuda_stream) {
 
 long long dma_launch_count(void) { return g_launches.load(); }
 
+int dma_kernel_timing(int enable) {
+    std::lock_guard<std::mutex> lock(g_timing_mutex);
+    if (enable) timing_clear();
+    g_timing_on.store(enable != 0);
+    return DMA_OK;
+}
+
+int dma_kernel_timing_read(float* ms, int32_t* which, int32_t capacity, int32_t* count) {
+    if (!count || (capacity > 0 && (!ms || !which))) return DMA_ERR_NULL;
+    std::lock_guard<std::mutex> lock(g_timing_mutex);
+    int n = 0;
+    for (const TimedLaunch& t : g_timed) {
+        if (!t.closed) continue;
+        if (n < capacity) {
+            if (cudaEventSynchronize(t.after) != cudaSuccess || cudaEventElapsedTime(&ms[n], t.before, t.after) != cudaSuccess)
+                return DMA_ERR_CUDA;
+            which[n] = t.which;
+        }
+        ++n;
+    }
+    *count = n;
+    return DMA_OK;
+}
+
 const char* dma_strerror(int status) {
     switch (status) {
         case DMA_OK: return "ok";
@@ -389,6 +453,7 @@ const char* dma_strerror(int status) {
         case DMA_ERR_WORKSPACE: return "workspace missing, misaligned or smaller than dma_query_workspace reports";
         case DMA_ERR_CUDA: return "CUDA call failed or no sm_100 device";
         case DMA_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait expired";
+        case DMA_ERR_MASK_OVERFLOW: return "token-compacted execution: the mask keeps more than w keys in a row";
         default: return "unknown status";
     }
 }

@@ -738,9 +738,11 @@ int launch_tc_bwd(const Prob& P, const void* Q, const void* K, const void* V, co
     bp.prof = prof_env ? (long long*)strtoull(prof_env, nullptr, 10) : nullptr;
 #endif
     const size_t smem = sizeof(SharedStorage) + 1024;
+    timing_mark(1, false, st);
     if (compact) {
         if (cudaFuncSetAttribute(bwd_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return DMA_ERR_CUDA;
         bwd_kernel<true><<<dim3(P.B * P.Hq, P.Tc), kThreads, smem, st>>>(tmQ, tmK, tmV, tmG, tmDQ, bp);
+        timing_mark(1, true, st);
         const int nb = (int)((nkv / 8 + 255) / 256);
         dq_convert_bf16_kernel<<<nb, 256, 0, st>>>(accK, (__nv_bfloat16*)dK, nkv / 8, P.L, P.Hkv, P.ks[0], P.ks[1], P.ks[2], P.scale);
         dq_convert_bf16_kernel<<<nb, 256, 0, st>>>(accV, (__nv_bfloat16*)dV, nkv / 8, P.L, P.Hkv, P.vs[0], P.vs[1], P.vs[2], 1.0f);
@@ -748,6 +750,7 @@ int launch_tc_bwd(const Prob& P, const void* Q, const void* K, const void* V, co
     } else {
         if (cudaFuncSetAttribute(bwd_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return DMA_ERR_CUDA;
         bwd_kernel<false><<<dim3(P.B * P.Hkv, P.Tc), kThreads, smem, st>>>(tmQ, tmK, tmV, tmG, tmDQ, bp);
+        timing_mark(1, true, st);
     }
     dq_convert_bf16_kernel<<<(unsigned)((nq / 8 + 255) / 256), 256, 0, st>>>(acc, (__nv_bfloat16*)dQ, nq / 8, P.L, P.Hq, P.qs[0], P.qs[1], P.qs[2], P.scale);
     count_launch(3);

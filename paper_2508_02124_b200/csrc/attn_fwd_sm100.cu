@@ -868,7 +868,7 @@ int make_tmap_f32_rows(CUtensorMap* m, const void* base, int B, int L, int H, in
 // order; the list is padded with -1 to the next multiple of 128.
 __global__ void __launch_bounds__(256) compact_lists_kernel(const int32_t* __restrict__ expiry, int* __restrict__ cidx,
                                                             int* __restrict__ ccnt, int L, int npairs, int cap, int causal,
-                                                            int q_off) {
+                                                            int q_off, int32_t* __restrict__ status) {
     __shared__ int wsum[2][8];
     const int list = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int bh = list / npairs, pair = list % npairs, i0 = q_off + pair * 256;
@@ -893,6 +893,8 @@ __global__ void __launch_bounds__(256) compact_lists_kernel(const int32_t* __res
         if (keep && pos < cap) out[pos] = j;
         n += total;
     }
+    // more kept keys than the list holds (a mask that keeps more than w keys in some row): reported, not truncated silently
+    if (n > cap && tid == 0) atomicExch(status, (int32_t)DMA_ERR_MASK_OVERFLOW);
     n = min(n, cap);
     for (int t = n + tid; t < ((n + 127) / 128) * 128 && t < cap; t += 256) out[t] = -1;
     if (tid == 0) ccnt[list] = n;
@@ -925,7 +927,7 @@ int launch_tc_fwd(const Prob& P, const void* Q, const void* K, const void* V, co
         const size_t nl = (size_t)P.B * P.Hq * npairs;
         int* ccnt = reinterpret_cast<int*>((char*)ws + kWsHeaderBytes);
         int* cidx = reinterpret_cast<int*>((char*)ws + kWsHeaderBytes + ((nl * sizeof(int) + 255) / 256) * 256);
-        compact_lists_kernel<<<(unsigned)nl, 256, 0, st>>>(expiry, cidx, ccnt, P.L, npairs, compact_cap(P), P.causal, P.q_off);
+        compact_lists_kernel<<<(unsigned)nl, 256, 0, st>>>(expiry, cidx, ccnt, P.L, npairs, compact_cap(P), P.causal, P.q_off, (int32_t*)ws);
         count_launch();
         fp.cidx = cidx; fp.ccnt = ccnt; fp.ccap = compact_cap(P);
     }
@@ -947,6 +949,7 @@ int launch_tc_fwd(const Prob& P, const void* Q, const void* K, const void* V, co
 #endif
     const size_t smem = sizeof(SharedStorage) + 1024;
     dim3 grid(P.B * P.Hq, npairs);
+    timing_mark(0, false, st);
     if (compact) {
         if (cudaFuncSetAttribute(fwd_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return DMA_ERR_CUDA;
         fwd_kernel<true><<<grid, kThreads, smem, st>>>(tmQ, tmK, tmV, fp);
@@ -954,6 +957,7 @@ int launch_tc_fwd(const Prob& P, const void* Q, const void* K, const void* V, co
         if (cudaFuncSetAttribute(fwd_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return DMA_ERR_CUDA;
         fwd_kernel<false><<<grid, kThreads, smem, st>>>(tmQ, tmK, tmV, fp);
     }
+    timing_mark(0, true, st);
     count_launch();
     return check_launch();
 }

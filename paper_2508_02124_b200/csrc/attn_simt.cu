@@ -327,8 +327,10 @@ int fwd_t(const Prob& P, const void* Q, const void* K, const void* V, const floa
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return DMA_ERR_CUDA;
     // a chunk of query rows that does not start on a bitmap row boundary (or comes without a bitmap) visits every key tile
     int use_bitmap = bitmap && !(P.flags & DMA_FLAG_IGNORE_BITMAP) && P.bm % BM == 0 && P.bn % BN == 0 && P.q_off % BM == 0;
+    timing_mark(0, false, st);
     kern<<<dim3((P.Lq + BM - 1) / BM, P.Hq, P.B), NT, smem, st>>>((const T*)Q, (const T*)K, (const T*)V, bias, expiry,
                                                                   bitmap, (T*)O, lse, P, use_bitmap);
+    timing_mark(0, true, st);
     count_launch();
     return check_launch();
 }
@@ -346,9 +348,11 @@ int bwd_t(const Prob& P, const void* Q, const void* K, const void* V, const void
     auto kern = simt_bwd_kernel<T, D>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return DMA_ERR_CUDA;
     int use_bitmap = !(P.flags & DMA_FLAG_IGNORE_BITMAP) && P.bm % BM == 0 && P.bn % BN == 0;
+    timing_mark(1, false, st);
     kern<<<dim3((P.L + BN - 1) / BN, P.Hkv, P.B), NT, smem, st>>>((const T*)Q, (const T*)K, (const T*)V, (const T*)dO,
                                                                   lse, Dv, bias, expiry, bitmap, acc, (T*)dK, (T*)dV,
                                                                   dM, P, use_bitmap);
+    timing_mark(1, true, st);
     dq_convert_kernel<T><<<(unsigned)((nq + 255) / 256), 256, 0, st>>>(acc, (T*)dQ, P);
     count_launch(3);
     return check_launch();

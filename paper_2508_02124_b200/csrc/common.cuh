@@ -26,6 +26,8 @@ struct Prob {
 
 int resolve(const dma_problem_t* p, Prob* out);          // validation + defaults; returns dma_status
 void count_launch(int n = 1);
+// measurement hook (dma_kernel_timing): brackets a stage's main kernel with a pair of CUDA events while recording is on
+void timing_mark(int which, bool after, cudaStream_t st);
 int check_launch();                                       // cudaGetLastError -> dma_status
 
 // stage launchers (each returns a dma_status); defined in the stage's .cu file

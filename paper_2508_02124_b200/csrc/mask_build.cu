@@ -502,9 +502,22 @@ int launch_delta_range(const Prob& P, const void* V, const float* W, const float
                       : launch_delta<float, 64>(P, V, W, A, delta, st, j_begin, j_end, ld);
 }
 
+// size limits of the stage's kernels (shared-memory footprints), checked before anything is enqueued
+static int mask_build_limits(const Prob& P) {
+    if (P.flags & DMA_FLAG_FULL_DELTA) {
+        const size_t lanes = (size_t)P.d / 8, HqP = (P.Hq + lanes - 1) / lanes * lanes;
+        if ((HqP * P.Hkv * P.d + HqP * kFullRows) * sizeof(float) > 200 * 1024) return DMA_ERR_UNSUPPORTED;
+    } else if ((size_t)P.G * (P.d + 128) * sizeof(float) > 48 * 1024) {
+        return DMA_ERR_UNSUPPORTED;
+    }
+    if ((size_t)(P.Tr + 1) * sizeof(int) > 48 * 1024) return DMA_ERR_UNSUPPORTED;
+    return DMA_OK;
+}
+
 int launch_mask_build(const Prob& P, const void* V, const float* W, const float* A, float* bias, int32_t* expiry,
                       uint32_t* bitmap, void* ws, cudaStream_t st, const int32_t* cu, int nseq) {
     int rc;
+    if ((rc = mask_build_limits(P))) return rc;          // an error return means that no kernel has been launched
     if (P.dtype == DMA_BF16)
         rc = P.d == 128 ? launch_delta<__nv_bfloat16, 128>(P, V, W, A, bias, st)
                         : launch_delta<__nv_bfloat16, 64>(P, V, W, A, bias, st);
@@ -565,8 +578,9 @@ extern "C" int dma_mask_build_static(const dma_problem_t* p, const void* V, cons
     if (bits & 15) return DMA_ERR_ALIGN;
     const size_t keys = (size_t)P.B * P.Hq * ((P.L + dma::kStaticChunk - 1) / dma::kStaticChunk) * dma::kStaticChunk;
     if (keys > kStaticKeys) return DMA_ERR_WORKSPACE;          // larger problems must use dma_mask_build
-    int dev = -1;
+    int dev = -1, major = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return DMA_ERR_CUDA;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess || major != 10) return DMA_ERR_CUDA;
     void* scratch;
     {
         std::lock_guard<std::mutex> lock(g_static_mutex);

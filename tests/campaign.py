@@ -29,6 +29,7 @@ from paper_2508_02124_b200 import binding as dma  # noqa: E402
 from paper_2508_02124_b200 import workloads as wl  # noqa: E402
 
 DEV = "cuda:0"
+TILE = dma.DMA_FLAG_TILE_PATH          # the tile-walking kernels; 0 leaves the choice to the library
 C2 = wl.CONFIGS["2"]
 
 
@@ -101,13 +102,13 @@ def attention(T):
         W, A = inp["W_delta"].to(DEV), inp["A"].to(DEV)
         if not causal:
             A = A * 0.25              # one key set per head: with the causal recipe's gates every row would be one-hot
-        p_of = lambda flags: dma.problem(B, case.Hq, Hkv, L, d, w, flags=flags, causal=causal)
+        p_of = lambda flags: dma.problem(B, case.Hq, Hkv, L, d, w, flags=flags if causal else flags & ~TILE, causal=causal)
         if varlen:
             mask = dma.dma_mask_build_varlen(p_of(0), v["V"], W, A, torch.tensor(cu, dtype=torch.int32, device=DEV))
         else:
             mask = dma.dma_mask_build(p_of(0), v["V"], W, A)
         ref = None
-        for flags in (dma.DMA_FLAG_SIMT, 0, dma.DMA_FLAG_COMPACT_KV, 0, dma.DMA_FLAG_COMPACT_KV):
+        for flags in (dma.DMA_FLAG_SIMT, TILE, dma.DMA_FLAG_COMPACT_KV, TILE, dma.DMA_FLAG_COMPACT_KV, 0):
             p = p_of(flags)
             O, lse = dma.dma_attn_fwd(p, v["Q"], v["K"], v["V"], *mask)
             g = dma.dma_attn_bwd(p, v["Q"], v["K"], v["V"], ref["O"] if ref else O, v["dO"], ref["lse"] if ref else lse, *mask)
@@ -262,13 +263,13 @@ def strided(T):
         L, w = int(r.choice([1, 130, 257, 512, 777, 1024, 2048])), int(r.choice([1, 31, 64, 129, 500, 3000]))
         d, B = int(r.choice([64, 128])), int(r.choice([1, 2]))
         dtn = str(r.choice(["bf16", "bf16", "bf16", "fp32"]))
-        flags = int(r.choice([0, dma.DMA_FLAG_COMPACT_KV, dma.DMA_FLAG_SIMT])) if dtn == "bf16" else 0
+        flags = int(r.choice([0, TILE, dma.DMA_FLAG_COMPACT_KV, dma.DMA_FLAG_SIMT])) if dtn == "bf16" else 0
         causal = int(r.random() < 0.8)
         case = wl.small(C2, B=B, Hq=Hkv * G, Hkv=Hkv, L=L, w=w, d=d, dtype=dtn, backward=True, seed=T.seed, name="campaign strided")
         inp = wl.make_inputs(case)
         Q, K, V, dO = (inp[k].to(DEV) for k in ("Q", "K", "V", "dO"))
         W, A = inp["W_delta"].to(DEV), inp["A"].to(DEV) * (1.0 if causal else 0.25)
-        mk = lambda: dma.problem(B, case.Hq, Hkv, L, d, w, dtype=case.torch_dtype, flags=flags, causal=causal)
+        mk = lambda: dma.problem(B, case.Hq, Hkv, L, d, w, dtype=case.torch_dtype, flags=flags if causal else flags & ~TILE, causal=causal)
         p0 = mk()
         m0 = dma.dma_mask_build(p0, V, W, A)
         O0, lse0 = dma.dma_attn_fwd(p0, Q, K, V, *m0)
@@ -347,7 +348,7 @@ def large(T):
             bad.append("expiry")
         if not np.array_equal(mask[2].cpu().numpy().view(np.uint32), oracle.bitmap_from_expiry(e).view(np.uint32)):
             bad.append("bitmap")
-        outs = run_all_paths(p_of, Q, K, V, dO, mask, (0, dma.DMA_FLAG_COMPACT_KV))
+        outs = run_all_paths(p_of, Q, K, V, dO, mask, (TILE, dma.DMA_FLAG_COMPACT_KV))
         bad += ["tile against compacted: " + k for k in outs[0] if not close(outs[1][k], outs[0][k], 1e-3 if k == "lse" else 8e-2)]
         edge = (L // 128) * 128
         rows = np.unique(np.concatenate([r.integers(0, L, 6), [0, L - 1, edge - 1, min(L - 1, edge)]])).astype(np.int32)

@@ -92,7 +92,7 @@ def test_skipped_tiles_do_not_change_the_result_on_a_banded_mask():
     active = ((bmp[..., t // 32] >> (t % 32)) & 1).sum()
     assert active < 0.8 * case.B * case.Hq * T * (T + 1) / 2           # the mask really has holes
     ref = oracle_all(case, inp, dl, e)
-    compare(case, gpu_run(case, inp), ref)
+    compare(case, gpu_run(case, inp, flags=dma.DMA_FLAG_TILE_PATH), ref)
     compare(case, gpu_run(case, inp, flags=dma.DMA_FLAG_IGNORE_BITMAP), ref)
 
 
@@ -131,27 +131,59 @@ def sampled_check(case, inp, got, nrows=24, nkeys=6, seed=0, forward_only=False)
     assert np.abs(lhs - rhs).max() <= 2e-2 * max(1.0, np.abs(rhs).max())
 
 
-def dq_rows_check(case, inp, got, rows):
-    """dQ on sampled rows: a one-head-group slice of the problem keeps the oracle's cost bounded."""
+def dq_rows(case):
+    """Sampled query rows for dQ: the dense-causal region (rows below w keep every visible key) AND the region where
+    the mask drops keys (rows at and beyond w), including both sides of a tile boundary and the last row."""
+    L, w = case.L, min(case.w, case.L)
+    rows = [0, 5, 130, min(700, L - 1), w - 1, min(w, L - 1), min(w + 1, L - 1), L // 2, (L // 2) | 1, 3 * L // 4 + 77,
+            L - 129, L - 128, L - 1]
+    return np.unique(np.clip(np.array(rows, np.int64), 0, L - 1)).astype(np.int32)
+
+
+def dq_rows_check(case, inp, got, rows=None):
+    """dQ on sampled rows, every head, against the oracle's row-subset routine (dQ_i depends on row i alone); Alg. 2's D
+    uses the oracle's own forward output of those rows rounded to the element type."""
+    rows = dq_rows(case) if rows is None else rows
     dl, e, _ = oracle_mask(case, inp)
-    G = case.Hq // case.Hkv
-    Q, K, V, dO = (f64(inp[k][:, :, :n]) for k, n in (("Q", G), ("K", 1), ("V", 1), ("dO", G)))
-    Lr = int(rows.max()) + 1                       # causal: rows < Lr only see keys < Lr
-    et = np.minimum(e[:, :G, :Lr], Lr)
-    Ot, _ = oracle.forward(Q[:, :Lr], K[:, :Lr], V[:, :Lr], dl[:, :G, :Lr].astype(np.float64), expiry=et)
-    dQ, _, _, _ = oracle.backward(Q[:, :Lr], K[:, :Lr], V[:, :Lr], dO[:, :Lr], dl[:, :G, :Lr].astype(np.float64),
-                                  expiry=et, keys=np.array([0], np.int32), O=round_to(case, Ot))
-    assert_close(got["dQ"][:, rows, :G], dQ[:, rows], case.dtype, "dQ rows")
+    Q, K, V, dO = (f64(inp[k]) for k in ("Q", "K", "V", "dO"))
+    bias = dl.astype(np.float64)
+    Or, _ = oracle.forward(Q, K, V, bias, expiry=e, rows=rows)
+    dQ = oracle.backward_dq_rows(Q, K, V, dO, bias, rows, expiry=e, O=round_to(case, Or))
+    assert_close(got["dQ"][:, rows], dQ, case.dtype, "dQ rows")
 
 
-@pytest.mark.parametrize("key", ["2", "3", "3x3", "4w256", "4w8192", "5", "S"])
+@pytest.mark.parametrize("key", ["2", "3", "3x3", "4w256", "4w2048", "4w8192", "5", "S"])
 def test_full_size_configs_sampled(key):
     case = wl.CONFIGS[key]
     inp = wl.make_inputs(case)
-    got = gpu_run(case, inp, backward=case.backward)
+    got = gpu_run(case, inp, backward=case.backward, flags=dma.DMA_FLAG_TILE_PATH)       # the tile-walking kernels (Alg. 1 / Alg. 2)
     sampled_check(case, inp, got)
     if case.backward:
-        dq_rows_check(case, inp, got, np.array([0, 5, 130, 700, 1500]))
+        dq_rows_check(case, inp, got)
+
+
+def test_default_flags_choose_the_path_from_the_descriptor():
+    """Without DMA_FLAG_COMPACT_KV / DMA_FLAG_TILE_PATH the library picks token-compacted execution for causal bf16 problems
+    with L >= 2048 and 4 w <= L and the tile-walking kernels otherwise: O and lse are the bits of the explicitly chosen path,
+    the injected over-full mask is reported (DMA_ERR_MASK_OVERFLOW) instead of being truncated silently."""
+    dev = torch.device("cuda:0")
+    for key, chosen in (("4w2048", dma.DMA_FLAG_COMPACT_KV), ("4w4096", dma.DMA_FLAG_TILE_PATH)):
+        case = wl.small(wl.CONFIGS[key], Hq=4, Hkv=4, name="auto " + key)
+        inp = wl.make_inputs(case)
+        a, b = gpu_run(case, inp, backward=False), gpu_run(case, inp, backward=False, flags=chosen)
+        assert torch.equal(a["O"], b["O"]) and torch.equal(a["lse"], b["lse"]), key
+        sizes = [dma.dma_query_workspace(problem_of(case, flags=f)) for f in (0, chosen)]
+        assert sizes[0] == sizes[1], key
+    # a mask that keeps every visible key, declared with w = 64: the gathered lists (w + 256 entries) overflow
+    case = wl.small(C2, B=1, Hq=2, Hkv=1, L=2048, w=64, name="overfull")
+    inp = wl.make_inputs(case)
+    p = problem_of(case, flags=dma.DMA_FLAG_COMPACT_KV)
+    e = torch.full((1, 2, case.L), case.L, dtype=torch.int32, device=dev)
+    bias = torch.zeros(1, 2, case.L, dtype=torch.float32, device=dev)
+    bmp = torch.from_numpy(oracle.bitmap_from_expiry(e.cpu().numpy()).view(np.int32)).to(dev)
+    ws = torch.empty(dma.dma_query_workspace(p)[1], dtype=torch.uint8, device=dev)
+    dma.dma_attn_fwd(p, inp["Q"].to(dev), inp["K"].to(dev), inp["V"].to(dev), bias, e, bmp, ws=ws)
+    assert dma.dma_read_status(ws) == -8
 
 
 def test_largest_supported_lengths():
@@ -160,18 +192,19 @@ def test_largest_supported_lengths():
     step-list capacity). Sampled rows and keys against the oracle."""
     fwd = wl.small(wl.CONFIGS["5"], B=1, Hq=4, Hkv=2, L=131072, w=4096, backward=False, name="max L forward")
     inp = wl.make_inputs(fwd)
-    got = gpu_run(fwd, inp, backward=False)
+    got = gpu_run(fwd, inp, backward=False, flags=dma.DMA_FLAG_TILE_PATH)
     sampled_check(fwd, inp, got, nrows=10, forward_only=True)
     gc = gpu_run(fwd, inp, backward=False, flags=dma.DMA_FLAG_COMPACT_KV)
     sampled_check(fwd, inp, gc, nrows=10, forward_only=True)
     with pytest.raises(dma.DmaError) as e:                        # one tile more is refused, not mis-executed
         too_long = wl.small(fwd, L=131072 + 128)
-        dma.dma_attn_fwd(problem_of(too_long), got["O"], got["O"], got["O"], got["bias"], got["expiry"], got["bitmap"])
+        dma.dma_attn_fwd(problem_of(too_long, flags=dma.DMA_FLAG_TILE_PATH), got["O"], got["O"], got["O"], got["bias"], got["expiry"], got["bitmap"])
     assert e.value.status == -4
     both = wl.small(wl.CONFIGS["3"], B=1, Hq=4, Hkv=1, L=65536, w=2048, backward=True, name="max L backward")
     inp = wl.make_inputs(both)
-    got = gpu_run(both, inp)
+    got = gpu_run(both, inp, flags=dma.DMA_FLAG_TILE_PATH)
     sampled_check(both, inp, got, nrows=8, nkeys=4)
+    dq_rows_check(both, inp, got)
 
 
 def test_whole_step_can_be_captured_in_a_cuda_graph():
@@ -243,10 +276,11 @@ def test_compact_forward_small_cases(kw):
     case = wl.small(C2, name="compact-small", backward=False, **kw)
     inp = wl.make_inputs(case)
     got = _compact_run(case, inp)
-    e = got["expiry"].cpu().numpy()
+    dl, e, _ = oracle_mask(case, inp)                     # the oracle's own mask, not the GPU's
+    assert np.array_equal(got["expiry"].cpu().numpy(), e)
     ref = oracle.forward(inp["Q"].double().numpy(), inp["K"].double().numpy(), inp["V"].double().numpy(),
-                         got["bias"].double().cpu().numpy(), expiry=e, scale=case.d ** -0.5)
-    assert_close(got["O"], round_to(case, ref[0]), case.dtype, "compact O")
+                         dl.astype(np.float64), expiry=e, scale=case.d ** -0.5)
+    assert_close(got["O"], ref[0], case.dtype, "compact O")
     assert_close(got["lse"], ref[1], case.dtype, "compact lse", lse=True)
 
 
@@ -358,10 +392,10 @@ def test_compact_backward_small_cases(case):
     compare(case, got, oracle_all(case, inp, dl, e))
 
 
-@pytest.mark.parametrize("key", ["3", "S"])
+@pytest.mark.parametrize("key", ["3", "4w256", "4w2048", "S"])
 def test_compact_backward_full_size_sampled(key):
     case = wl.CONFIGS[key]
     inp = wl.make_inputs(case)
     got = _compact_full_run(case, inp)
     sampled_check(case, inp, got)
-    dq_rows_check(case, inp, got, np.array([0, 5, 130, 700, 1500]))
+    dq_rows_check(case, inp, got)

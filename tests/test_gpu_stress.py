@@ -49,7 +49,7 @@ def test_tensor_core_kernels_equal_the_cuda_core_kernels(seed):
     p0 = mk(0)
     bias, expiry, bitmap = dma.dma_mask_build_varlen(p0, V, W, A, cu_t)
     ref = None
-    for flags in (dma.DMA_FLAG_SIMT, 0, dma.DMA_FLAG_COMPACT_KV, 0):
+    for flags in (dma.DMA_FLAG_SIMT, dma.DMA_FLAG_TILE_PATH, dma.DMA_FLAG_COMPACT_KV, 0):
         p = mk(flags)
         O, lse = dma.dma_attn_fwd(p, Q, K, V, bias, expiry, bitmap)
         dQ, dK, dV, dM = dma.dma_attn_bwd(p, Q, K, V, O, dO, lse, bias, expiry, bitmap)
@@ -88,7 +88,7 @@ def test_arbitrary_interval_masks(seed):
     Q, K, V, dO = (inp[k].to(DEV) for k in ("Q", "K", "V", "dO"))
     bias_t, e_t, bmp_t = torch.from_numpy(bias).to(DEV), torch.from_numpy(e).to(DEV), torch.from_numpy(bitmap.view(np.int32)).to(DEV)
     ref = None
-    for flags in (dma.DMA_FLAG_SIMT, 0, dma.DMA_FLAG_COMPACT_KV):
+    for flags in (dma.DMA_FLAG_SIMT, dma.DMA_FLAG_TILE_PATH, dma.DMA_FLAG_COMPACT_KV, 0):
         p = dma.problem(1, Hq, Hkv, L, 128, L, flags=flags)
         O, lse = dma.dma_attn_fwd(p, Q, K, V, bias_t, e_t, bmp_t)
         dQ, dK, dV, dM = dma.dma_attn_bwd(p, Q, K, V, O, dO, lse, bias_t, e_t, bmp_t)

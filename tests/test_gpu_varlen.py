@@ -108,7 +108,7 @@ def test_config3_packed_documents():
     rows and keys; no key tile of another document is ever active."""
     case = wl.CONFIGS["3"]
     cu = wl.packed_cu_seqlens(case.L, 12, seed=31)
-    inp, got = run(case, cu)
+    inp, got = run(case, cu, flags=dma.DMA_FLAG_TILE_PATH)
     dl, e, bmp = oracle_varlen_mask(case, inp, cu)
     assert np.array_equal(got["expiry"].cpu().numpy(), e)
     assert np.array_equal(got["bitmap"].cpu().numpy().view(np.uint32), bmp)

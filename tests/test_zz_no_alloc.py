@@ -43,6 +43,26 @@ def test_static_scratch_matches_workspace_version_on_consecutive_calls():
         build_both(case, inp, out, full=True)                     # go through the same scratch
 
 
+def test_static_scratch_at_exactly_its_limit():
+    # 32 heads x 32768 keys = 1,048,576 sort keys: the rank permutation ends on the array's last byte. V is the
+    # recipe's noise; the check is bit-equality with the workspace version, twice in a row.
+    dev = torch.device("cuda:0")
+    case = wl.small(wl.CONFIGS["3"], B=1, Hq=32, Hkv=8, L=32768, d=64, w=1000, name="static-limit")
+    g = torch.Generator().manual_seed(77)
+    inp = {"V": torch.randn(case.B, case.L, case.Hkv, case.d, generator=g).to(case.torch_dtype),
+           "W_delta": torch.randn(case.Hq, case.d, generator=g) / 8.0, "A": torch.rand(case.Hq, generator=g) * 1.5 + 0.5}
+    T = case.L // 128
+    out = (torch.empty(case.B, case.Hq, case.L, dtype=torch.float32, device=dev),
+           torch.empty(case.B, case.Hq, case.L, dtype=torch.int32, device=dev),
+           torch.empty(case.B, case.Hq, T, (T + 31) // 32, dtype=torch.int32, device=dev))
+    build_both(case, inp, out)
+    build_both(case, inp, out)
+    one_more = dma.problem(case.B, case.Hq, case.Hkv, case.L + 1, case.d, case.w)      # one key over: a whole new chunk per head
+    with pytest.raises(dma.DmaError) as e:
+        dma.dma_mask_build_static(one_more, inp["V"].to(dev), inp["W_delta"].to(dev), inp["A"].to(dev), *out)
+    assert e.value.status == -5
+
+
 def test_static_scratch_rejects_oversized_problems():
     dev = torch.device("cuda:0")
     p = dma.problem(1, 32, 8, 65536, 128, 4096)      # 2 Mi sort keys: over the 1 Mi limit
