@@ -80,22 +80,8 @@ struct BwdParams {
     float* dKacc;               // fp32 [B, L, Hkv, 128] accumulators (several query heads add into one KV head's rows)
     float* dVacc;
     int64_t ks_b, ks_l, ks_h, vs_b, vs_l, vs_h;
-#ifdef DMA_PROF
-    long long* prof;            // role timing (development builds only): cycles per phase of CTA (0, 0)
-#endif
 };
 
-// PROF_WAIT(slot, expr): evaluates expr (a wait) and, in development builds, adds its duration to a per-role counter
-#ifdef DMA_PROF
-#define PROF_DECL(role) const bool prof_on = P.prof && blockIdx.x == 0 && blockIdx.y == 0 && lane == 0; \
-    long long prof_acc[8] = {0, 0, 0, 0, 0, 0, 0, 0}; const long long prof_start = clock64(); const int prof_role = role
-#define PROF_WAIT(slot, expr) do { const long long t0_ = clock64(); expr; prof_acc[slot] += clock64() - t0_; } while (0)
-#define PROF_END() do { if (prof_on) { prof_acc[7] = clock64() - prof_start; for (int k_ = 0; k_ < 8; ++k_) P.prof[prof_role * 8 + k_] = prof_acc[k_]; } } while (0)
-#else
-#define PROF_DECL(role)
-#define PROF_WAIT(slot, expr) do { expr; } while (0)
-#define PROF_END()
-#endif
 
 // x as three bf16 terms (hi, mid, lo: 24 significant bits) in elements 0-2 of a 16-byte core-matrix row
 __device__ __forceinline__ uint4 split3(float x) {
@@ -233,7 +219,6 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
         float2 dm2 = make_float2(0.0f, 0.0f);
         int len = 0, cur_g = -1;
         bool ok = true;
-        PROF_DECL(warp == 0 ? 0 : 7);
         for (int n = 0; n < n_steps && ok; ++n) {
             const uint32_t e = S.sched[n];
             const int g = (int)(e >> 11), i0 = (int)((e >> 1) & 0x3FF) * 128 + (int)(e & 1) * 64;
@@ -247,23 +232,16 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                 cur_g = g;
             }
             // (S^T and dP^T were issued after the step's Q / dO stage was full: nothing else of that stage is read here)
-            PROF_WAIT(0, ok = mbar_wait_warp(&S.sdp_full, n & 1, abort_flag));
+            ok = mbar_wait_warp(&S.sdp_full, n & 1, abort_flag);
             if (!ok) break;
             tc_fence_after();
             uint32_t sr[32], pr[32];
-#ifdef DMA_PROF
-            const long long tp0 = clock64();
-#endif
             tmem_ld32(tmem + lane_base + cS + hsel * 32, sr);
             tmem_ld32(tmem + lane_base + cDP + hsel * 32, pr);
             tc_wait_ld();
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&S.sdp_free);
-#ifdef DMA_PROF
-            const long long tp1 = clock64();
-            prof_acc[2] += tp1 - tp0;
-#endif
             // valid columns of this thread within its 32: col in [lo, lo + width)
             const int c0 = hsel * 32;
             const int lo = max(0, jf - i0 - c0);
@@ -312,12 +290,8 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                     dd[(c >> 1) + 1] = pack_bf16(d1.x, d1.y);
                 }
             }
-#ifdef DMA_PROF
-            const long long tp2 = clock64();
-            prof_acc[3] += tp2 - tp1 + (long long)(pp[3] == 0x12345u && dd[7] == 0x54321u);
-#endif
             // the previous step's dV / dK / dQ GEMMs must have finished reading P^T, dS^T (TMEM) and dS^T (smem)
-            if (n > 0) PROF_WAIT(1, ok = mbar_wait_warp(&S.pds_free, (n - 1) & 1, abort_flag));
+            if (n > 0) ok = mbar_wait_warp(&S.pds_free, (n - 1) & 1, abort_flag);
             if (!ok) break;
             tc_fence_after();
             tmem_st16(tmem + lane_base + cP + hsel * 16, pp);
@@ -333,11 +307,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&S.pds_ready);
-#ifdef DMA_PROF
-            prof_acc[4] += clock64() - tp2;
-#endif
         }
-        if (warp == 0) PROF_END();
         if (cur_g >= 0 && j < P.L) atomicAdd(&P.dM[(size_t)(b * P.Hq + hk * P.G + cur_g) * P.L + j], dm2.x + dm2.y);
         // epilogue: dK (scaled) and dV rows to global memory; warps w and w+4 each write one half of the channels
         if (ok && n_steps > 0) ok = mbar_wait_warp(&S.pds_free, (n_steps - 1) & 1, abort_flag);
@@ -392,11 +362,10 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
         const int dw = warp & 3;
         const uint32_t lane_base = (uint32_t)(dw * 32) << 16;
         bool ok = true;
-        PROF_DECL(warp == 8 ? 1 : 7);
         for (int n = 0; n < n_steps && ok; ++n) {
             const uint32_t e = S.sched[n];
             const int g = (int)(e >> 11), i0 = (int)((e >> 1) & 0x3FF) * 128 + (int)(e & 1) * 64;
-            PROF_WAIT(0, ok = mbar_wait_warp(&S.dq_full, n & 1, abort_flag));
+            ok = mbar_wait_warp(&S.dq_full, n & 1, abort_flag);
             if (!ok) break;
             tc_fence_after();
             uint32_t v[64];
@@ -408,7 +377,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             if (lane == 0) mbar_arrive(&S.dq_free);
 #pragma unroll
             for (int qr = 0; qr < 4; ++qr) {           // quarter steps of 16 query rows, two staging buffers in turn
-                PROF_WAIT(1 + (qr & 1), if (lane == 0) bulk_wait_read_1(); __syncwarp());
+                if (lane == 0) bulk_wait_read_1(); __syncwarp();
 #pragma unroll
                 for (int u = 0; u < 16; ++u) S.dq_stage[dw][qr & 1][u][lane] = __uint_as_float(v[qr * 16 + u]);
                 fence_proxy_async();
@@ -419,7 +388,6 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                 if (lane == 0) bulk_commit();
             }
         }
-        if (warp == 8) PROF_END();
         if (lane == 0) bulk_wait_all();
     } else {
         if (warp == 12) {
@@ -519,11 +487,10 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             const uint32_t tmem_u = __shfl_sync(0xffffffffu, tmem, 0);
             const int n_steps_u = __shfl_sync(0xffffffffu, n_steps, 0);
             bool ok = mbar_wait_warp(&S.kv_full, 0, abort_flag);
-            PROF_DECL(2);
             for (int n = 0; n < n_steps_u && ok; ++n) {
                 const int st = n % kStages;
-                PROF_WAIT(0, ok = mbar_wait_warp(&S.qd_full[st], (n / kStages) & 1, abort_flag));
-                if (ok && n > 0) PROF_WAIT(1, ok = mbar_wait_warp(&S.sdp_free, (n - 1) & 1, abort_flag));
+                ok = mbar_wait_warp(&S.qd_full[st], (n / kStages) & 1, abort_flag);
+                if (ok && n > 0) ok = mbar_wait_warp(&S.sdp_free, (n - 1) & 1, abort_flag);
                 if (!ok) break;
                 tc_fence_after();
                 const uint64_t dQ = dQ0 + (uint64_t)(st * (kQBytes >> 4)), dG = dG0 + (uint64_t)(st * (kQBytes >> 4));
@@ -543,7 +510,6 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                 }
                 __syncwarp();
             }
-            PROF_END();
         } else if (warp == 14) {
             // ============================ MMA issuer 2: dV += P^T dO, dK += dS^T Q, dQ^T = K^T dS^T ============================
             constexpr uint32_t id_dkv = idesc_bf16(128, 128, 0, 1);    // P^T|dS^T (TMEM) x dO|Q (MN-major)    -> 128 x 128
@@ -553,11 +519,10 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             const uint32_t tmem_u = __shfl_sync(0xffffffffu, tmem, 0);
             const int n_steps_u = __shfl_sync(0xffffffffu, n_steps, 0);
             bool ok = true;
-            PROF_DECL(3);
             for (int n = 0; n < n_steps_u && ok; ++n) {
                 const int st = n % kStages;
-                PROF_WAIT(0, ok = mbar_wait_warp(&S.pds_ready, n & 1, abort_flag));
-                if (ok && n > 0) PROF_WAIT(1, ok = mbar_wait_warp(&S.dq_free, (n - 1) & 1, abort_flag));
+                ok = mbar_wait_warp(&S.pds_ready, n & 1, abort_flag);
+                if (ok && n > 0) ok = mbar_wait_warp(&S.dq_free, (n - 1) & 1, abort_flag);
                 if (!ok) break;
                 tc_fence_after();
                 const uint64_t dGm = dGm0 + (uint64_t)(st * (kQBytes >> 4)), dQm = dQm0 + (uint64_t)(st * (kQBytes >> 4));
@@ -578,7 +543,6 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                 }
                 __syncwarp();
             }
-            PROF_END();
         }
     }
     tc_fence_before();
@@ -733,10 +697,6 @@ int launch_tc_bwd(const Prob& P, const void* Q, const void* K, const void* V, co
     bp.ks_b = P.ks[0]; bp.ks_l = P.ks[1]; bp.ks_h = P.ks[2]; bp.vs_b = P.vs[0]; bp.vs_l = P.vs[1]; bp.vs_h = P.vs[2];
     bp.perm = perm; bp.expiry_all = expiry; bp.causal = P.causal; bp.Kg = (const __nv_bfloat16*)K; bp.Vg = (const __nv_bfloat16*)V;
     bp.dKacc = accK; bp.dVacc = accV;
-#ifdef DMA_PROF
-    const char* prof_env = getenv("DMA_PROF_PTR");
-    bp.prof = prof_env ? (long long*)strtoull(prof_env, nullptr, 10) : nullptr;
-#endif
     const size_t smem = sizeof(SharedStorage) + 1024;
     timing_mark(1, false, st);
     if (compact) {

@@ -8,13 +8,13 @@
 // memory and touch no shared memory per element. Diagonal tiles, and tiles in which more than 13 keys expire inside
 // the query tile's rows, take the general path with the explicit test j <= i < expiry[j].
 // Warp roles (12 warps):
-//   warps 0-3 / 4-7  softmax group 0 / 1: thread r owns query row r of its tile (TMEM lane r): row max, lazy rescale of
+//   warps 4-7 / 8-11 softmax group 0 / 1: thread r owns query row r of its tile (TMEM lane r): row max, lazy rescale of
 //                    O, p = 2^(x c - stab), row sum, P (bf16) written back to tensor memory over S, final normalisation
-//   warp 8           producer: builds the tile schedule from the bitmap, then issues the TMA loads of K and V per
+//   warp 0           producer: builds the tile schedule from the bitmap, then issues the TMA loads of K and V per
 //                    active key tile (inactive tiles are never loaded); K and V stages are released separately
-//   warp 9           MMA issuer (whole warp, warp-uniform values, one elected lane issues): S_w = Q_w K^T (+ ninth
+//   warp 1           MMA issuer (whole warp, warp-uniform values, one elected lane issues): S_w = Q_w K^T (+ ninth
 //                    k-step), O_w += P_w V, ping-ponging between the two query tiles
-//   warps 10, 11     stagers for query tile 0 / 1: ninth k-step operands, expiry vector, fast / general flag
+//   warps 2, 3       stagers for query tile 0 / 1: ninth k-step operands, expiry vector, fast / general flag
 // Tensor memory (512 columns): S0 [0,128) S1 [128,256) O0 [256,384) O1 [384,512); P_w aliases columns [0,64) of S_w.
 // The log-sum-exp replaces Alg. 1's (l, m) pair.
 #include <cstdlib>
@@ -80,27 +80,20 @@ struct FwdParams {
     int Lq, q_off, Trq;                        // chunk of query rows (token-compacted mode only): Q, O, lse hold rows q_off .. q_off + Lq - 1; Trq = its 128-row tiles
     int64_t os_b, os_l, os_h;
     int64_t ks_b, ks_l, ks_h, vs_b, vs_l, vs_h;
-#ifdef DMA_PROF
-    long long* prof;                           // role timing (development builds only): cycles per phase of CTA (0, 0)
-#endif
 };
 
-#ifdef DMA_PROF
-#define TRACE(it, ev) do { if (P.prof && blockIdx.x == 0 && blockIdx.y == 0 && (it) >= 60 && (it) < 64) P.prof[64 + ((it) - 60) * 16 + (ev)] = clock64(); } while (0)
-#define PROF_T(var) const long long var = clock64()
-#define PROF_ADD(slot, expr) do { if (prof_on) prof_acc[slot] += (expr); } while (0)
-#else
-#define TRACE(it, ev)
-#define PROF_T(var)
-#define PROF_ADD(slot, expr)
-#endif
 
 __device__ __forceinline__ uint32_t use_bit(uint32_t entry, int w) { return (entry >> (30 + w)) & 1u; }
 
+// Warp roles. The four service warps come FIRST: among ready warps the schedulers favour the older (lower-numbered) ones,
+// and a stager that gets an issue slot only when both softmax warps of its scheduler stall was measured to need ~3600
+// cycles for the few hundred instructions of one key tile.
+constexpr int kWarpProducer = 0, kWarpIssuer = 1, kWarpStager0 = 2, kWarpStager1 = 3, kFirstSoftmaxWarp = 4;
+
 // kCompact: instead of walking the active 128-key tiles of the bitmap, the CTA walks its gathered key list (keys that
-// at least one of its 256 query rows keeps, at most w + 256 of them). Warps 8 and 11 fetch the K and V rows with 16-byte
+// at least one of its 256 query rows keeps, at most w + 256 of them). Warps 0 and 3 fetch the K and V rows with 16-byte
 // asynchronous copies into the swizzled tile layout (TMA row gathers of four rows were measured at ~70 cycles per
-// request: too slow), warp 10 builds the B rows of the ninth k-step (bias, and -BIG for columns no row of the tile keeps; the A
+// request: too slow), warp 2 builds the B rows of the ninth k-step (bias, and -BIG for columns no row of the tile keeps; the A
 // rows are constant) and flags the 32-column chunks that still need the per-element test.
 template <bool kCompact>
 __global__ void __launch_bounds__(kThreads, 1)
@@ -135,11 +128,11 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
         S.n_iters = 0;
         fence_barrier_init();
     }
-    if (warp == 9) {
+    if (warp == kWarpIssuer) {
         tmem_alloc(&S.tmem_base, 512);
         tmem_relinquish();
     }
-    if (warp == 8) {
+    if (warp == kWarpProducer) {
         // schedule: ascending key tiles that at least one of the two query tiles uses
         if (lane == 0) { prefetch_tmap(&tmQ); prefetch_tmap(&tmK); prefetch_tmap(&tmV); }
         int n = 0;
@@ -169,10 +162,10 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
     const uint32_t tmem = S.tmem_base;
     const int n_iters = S.n_iters;
 
-    if (warp < 8) {
+    if (warp >= kFirstSoftmaxWarp) {
         // =========================================== softmax groups ===========================================
         setmaxnreg_inc<208>();
-        const int w = warp >> 2;
+        const int w = (warp - kFirstSoftmaxWarp) >> 2;
         const int r = tid & 127;
         const int qt = w ? qt1 : qt0;
         const int il = qt * 128 + r;                        // row inside Q, O, lse
@@ -183,15 +176,9 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
         float m_ref = -INFINITY, r_ref = 0.0f, l = 0.0f;
         int n_used = 0;
         bool ok = true;
-#ifdef DMA_PROF
-        const bool prof_on = P.prof && blockIdx.x == 0 && blockIdx.y == 0 && lane == 0;
-        long long prof_acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-        const long long prof_start = clock64();
-#endif
         for (int it = 0; it < n_iters && ok; ++it) {
             const uint32_t entry = S.sched[it];
             if (!use_bit(entry, w)) continue;
-            PROF_T(t_a);
             const int st = it % kStages, j0 = (int)(entry & 0xFFFFF) * 128;
             ok = mbar_wait_warp(&S.s_full[w], n_used & 1, abort_flag);
             if (!ok) break;
@@ -202,9 +189,6 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             // at once, before the stager has written the flag.)
             const uint32_t tile_flags = S.fast[st][w];
             const bool fast_tile = kCompact || tile_flags != 0;      // token-compacted mode: the flags are a chunk mask instead
-            PROF_T(t_b);
-            PROF_ADD(0, t_b - t_a);
-            if ((warp & 3) == 0 && lane == 0) TRACE(it, w * 4 + 0);
             // The accumulator holds q.k + bias / scale (+ -BIG where the ninth k-step masks). On the fast path that
             // is the whole masked score; otherwise (diagonal tile, or more than 13 keys expiring inside the tile's
             // rows) the validity test j <= i < expiry[j] is applied here. x = log2e * scale * score, -inf if masked.
@@ -217,9 +201,6 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
 #pragma unroll
                 for (int u = 0; u < 128; ++u) x[u] = __uint_as_float(raw[u]);
             }
-            PROF_T(t_c);
-            PROF_ADD(1, t_c - t_b);
-            if ((warp & 3) == 0 && lane == 0) TRACE(it, w * 4 + 1);
             float mxa[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
             if constexpr (kCompact) {
                 // gathered columns: bias and the keys that are gone for the whole tile are already in the score; the
@@ -240,7 +221,6 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                 }
             }
             if (fast_tile) {
-                PROF_ADD(6, 1);
 #pragma unroll
                 for (int c = 0; c < 128; c += 4) {
                     mxa[(c >> 2) & 1] = max3(mxa[(c >> 2) & 1], x[c], x[c + 1]);
@@ -302,9 +282,6 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             const float M = m_use * P.scale_log2, nM = -M;
             const float resid = r_ref;
             const bool small = __all_sync(0xffffffffu, fabsf(M) < kSmallStab);
-            PROF_T(t_d);
-            PROF_ADD(2, t_d - t_c + (long long)(m_use == 1.2345f));
-            if ((warp & 3) == 0 && lane == 0) TRACE(it, w * 4 + 2);
             float sa[4] = {0.f, 0.f, 0.f, 0.f};
             if (small) {
 #pragma unroll
@@ -350,19 +327,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             __syncwarp();
             if (lane == 0) mbar_arrive(&S.p_ready[w]);      // one arrival per warp: 128 serialised arrivals cost ~400 cycles
             ++n_used;
-            PROF_T(t_e);
-            PROF_ADD(3, t_e - t_d);
-            if ((warp & 3) == 0 && lane == 0) TRACE(it, w * 4 + 3);
-            PROF_ADD(4, 1);
         }
-#ifdef DMA_PROF
-        if (prof_on) {
-            prof_acc[5] = clock64() - prof_start;
-            if ((warp & 3) == 0) for (int k = 0; k < 8; ++k) P.prof[w * 8 + k] = prof_acc[k];
-            P.prof[32 + warp * 2] = prof_acc[0];
-            P.prof[33 + warp * 2] = prof_acc[5];
-        }
-#endif
         // epilogue: O_w / l -> bf16 rows, log-sum-exp in natural log
         const bool exists = w == 0 || has1;
         if (ok && exists && n_used > 0) ok = mbar_wait_warp(&S.o_done[w], (n_used - 1) & 1, abort_flag);
@@ -396,12 +361,12 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
         }
     } else {
         setmaxnreg_dec<88>();   // 4 warps x 80 registers released = 8 warps x 40 acquired above
-        if (kCompact && (warp == 8 || warp == 11)) {
+        if (kCompact && (warp == kWarpProducer || warp == kWarpStager1)) {
             // ================================ token-compacted mode: gather warps ================================
-            // Warp 8 fetches the K rows of each 128-key slice of the gathered list, warp 11 the V rows: 16-byte
+            // Warp 0 fetches the K rows of each 128-key slice of the gathered list, warp 3 the V rows: 16-byte
             // asynchronous copies into the 128-byte-swizzled tile layout (8 lanes per 128-byte half row, 4 rows per
             // instruction; padding entries (-1) are zero-filled). Each lane's copies report to the stage's barrier.
-            const bool isK = warp == 8;
+            const bool isK = warp == kWarpProducer;
             if (isK && lane == 0) {
                 mbar_arrive_expect_tx(&S.q_full, has1 ? 2 * kTileBytes : kTileBytes);
                 for (int w = 0; w < (has1 ? 2 : 1); ++w)
@@ -442,7 +407,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             }
             for (int it = max(0, n_iters - kStages); it < n_iters && ok; ++it)
                 ok = mbar_wait_warp(isK ? &S.k_empty[it % kStages] : &S.v_empty[it % kStages], (it / kStages) & 1, abort_flag);
-        } else if (kCompact && warp == 10) {
+        } else if (kCompact && warp == kWarpStager0) {
             // ================================ token-compacted mode: stager ================================
             // Per 128-key slice and query tile: the B rows of the ninth k-step (bias / scale as three bf16 terms, or
             // -BIG for a column that no row of the tile keeps; the A rows are constant ones), the key index and expiry
@@ -529,7 +494,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&S.k_full[st]);
             }
-        } else if (warp == 8) {
+        } else if (warp == kWarpProducer) {
             // =========================================== producer ===========================================
             if (lane == 0) {
                 mbar_arrive_expect_tx(&S.q_full, has1 ? 2 * kTileBytes : kTileBytes);
@@ -561,13 +526,13 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             for (int it = max(0, n_iters - kStages); it < n_iters && ok; ++it)
                 ok = mbar_wait_warp(&S.k_empty[it % kStages], (it / kStages) & 1, abort_flag) &&
                      mbar_wait_warp(&S.v_empty[it % kStages], (it / kStages) & 1, abort_flag);
-        } else if (warp >= 10) {
+        } else if (warp == kWarpStager0 || warp == kWarpStager1) {
             // =========================================== stagers ===========================================
-            // Warp 10 + w serves query tile w: per key tile it builds the ninth k-step operands described at
-            // SharedStorage (warp 10 also stages the expiry vector for the general softmax path). The global loads run
+            // Warp 2 + w serves query tile w: per key tile it builds the ninth k-step operands described at
+            // SharedStorage (warp 2 also stages the expiry vector for the general softmax path). The global loads run
             // one tile ahead and the rows are formed in registers before the wait for the blocks to be free, so that
             // only the stores are left between the previous S product and the next one.
-            const int w = warp - 10;
+            const int w = warp - kWarpStager0;
             const int i0 = (w ? qt1 : qt0) * 128;
             // key indices of a tile's columns, then their bias and expiry, loaded one tile before they are needed
             auto fetch_idx = [&](int it, int (&jv)[4]) {
@@ -595,9 +560,6 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                 const int st = it % kStages;
                 const uint32_t entry = S.sched[it];
                 const bool use = use_bit(entry, w);
-#ifdef DMA_PROF
-                const long long ts_loop = clock64();
-#endif
                 float bn[4] = {0.f, 0.f, 0.f, 0.f};
                 int en[4] = {0, 0, 0, 0}, jnn[4] = {0, 0, 0, 0};
                 if (it + 1 < n_iters) fetch_vals(jn, bn, en);
@@ -656,15 +618,8 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                 }
                 // fast[st] / len[st] were last read by the softmax groups before they released P of tile it - kStages
                 // (hence before its P V); the operand blocks were last read by the S products of tile it - 1
-#ifdef DMA_PROF
-                const long long ts0 = clock64();
-#endif
                 if (it >= kStages) ok = mbar_wait_warp(&S.v_empty[st], ((it / kStages) - 1) & 1, abort_flag);
                 if (ok && it >= 1) ok = mbar_wait_warp(&S.k_empty[(it - 1) % kStages], ((it - 1) / kStages) & 1, abort_flag);
-#ifdef DMA_PROF
-                const long long ts1 = clock64();
-                if (P.prof && blockIdx.x == 0 && blockIdx.y == 0 && lane == 0 && w == 0) { P.prof[24] += ts1 - ts0; P.prof[25] += ts0 - ts_loop; }
-#endif
                 if (!ok) break;
                 if (w == 0) {
 #pragma unroll
@@ -700,11 +655,8 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                 fence_proxy_async();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&S.k_full[st]);
-#ifdef DMA_PROF
-                if (P.prof && blockIdx.x == 0 && blockIdx.y == 0 && lane == 0 && w == 0) P.prof[26] += clock64() - ts1;
-#endif
             }
-        } else if (warp == 9) {
+        } else if (warp == kWarpIssuer) {
             // =========================================== MMA issuer ===========================================
             // The whole warp walks the schedule with warp-uniform values (descriptors, stage and tile indices stay in
             // the uniform datapath); one elected lane issues the tcgen05 instructions.
@@ -731,12 +683,6 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                 __syncwarp();
             };
             int n_p[2] = {0, 0};
-#ifdef DMA_PROF
-            long long iss_acc[4] = {0, 0, 0, 0};
-#define PROF_W(slot, expr) do { const long long t0_ = clock64(); expr; iss_acc[slot] += clock64() - t0_; } while (0)
-#else
-#define PROF_W(slot, expr) do { expr; } while (0)
-#endif
             bool ok = mbar_wait_warp(&S.q_full, 0, abort_flag);
             if (ok && n_iters_u > 0) {
                 ok = mbar_wait_warp(&S.k_full[0], 0, abort_flag);
@@ -755,7 +701,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                 const int st = it % kStages, nst = (it + 1) % kStages;
                 const uint32_t entry = __shfl_sync(0xffffffffu, S.sched[it], 0);
                 const uint32_t next = it + 1 < n_iters_u ? __shfl_sync(0xffffffffu, S.sched[it + 1], 0) : 0u;
-                PROF_W(0, ok = mbar_wait_warp(&S.v_full[st], (it / kStages) & 1, abort_flag));
+                ok = mbar_wait_warp(&S.v_full[st], (it / kStages) & 1, abort_flag);
                 if constexpr (kCompact) fence_proxy_async();     // the gathered tiles were written through the generic proxy
                 bool k_ready = false;
 #pragma unroll
@@ -765,7 +711,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                         const uint64_t dv = dV0 + (uint64_t)(st * (kTileBytes >> 4));
                         const uint32_t d_tmem = tmem_u + 256 + w * 128, a_tmem = tmem_u + w * 128;
                         const uint32_t acc0 = n_p[w] > 0 ? 1u : 0u;
-                        PROF_W(2 + w, ok = mbar_wait_warp(&S.p_half[w], n_p[w] & 1, abort_flag));
+                        ok = mbar_wait_warp(&S.p_half[w], n_p[w] & 1, abort_flag);
                         if (ok) {
                             tc_fence_after();
                             if (elect_one()) {
@@ -776,7 +722,6 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                             __syncwarp();
                             ok = mbar_wait_warp(&S.p_ready[w], n_p[w] & 1, abort_flag);
                         }
-                        if (lane == 0) TRACE(it, 8 + w * 2);
                         if (ok) {
                             tc_fence_after();
                             if (elect_one()) {
@@ -791,14 +736,13 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                     }
                     if (ok && use_bit(next, w)) {
                         if (!k_ready) {
-                            PROF_W(1, ok = mbar_wait_warp(&S.k_full[nst], ((it + 1) / kStages) & 1, abort_flag));
+                            ok = mbar_wait_warp(&S.k_full[nst], ((it + 1) / kStages) & 1, abort_flag);
                             if constexpr (kCompact) fence_proxy_async();
                             if (ok) tc_fence_after();
                             k_ready = true;
                         }
                         if (ok) issue_s(w, nst);
                     }
-                    if (lane == 0) TRACE(it, 9 + w * 2);
                 }
                 if (ok) {
                     if (elect_one()) {
@@ -808,15 +752,12 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                     __syncwarp();
                 }
             }
-#ifdef DMA_PROF
-            if (P.prof && blockIdx.x == 0 && blockIdx.y == 0 && lane == 0) for (int k = 0; k < 4; ++k) P.prof[16 + k] = iss_acc[k];
-#endif
         }
     }
     // teardown: every role falls through to here, also after a timed-out wait
     tc_fence_before();
     __syncthreads();
-    if (warp == 9) {
+    if (warp == kWarpIssuer) {
         tc_fence_after();
         tmem_dealloc(tmem, 512);
     }
@@ -943,10 +884,6 @@ int launch_tc_fwd(const Prob& P, const void* Q, const void* K, const void* V, co
     fp.rescale_gap = kRescaleThreshold / fp.scale_log2;
     fp.os_b = P.os[0]; fp.os_l = P.os[1]; fp.os_h = P.os[2];
     fp.ks_b = P.ks[0]; fp.ks_l = P.ks[1]; fp.ks_h = P.ks[2]; fp.vs_b = P.vs[0]; fp.vs_l = P.vs[1]; fp.vs_h = P.vs[2];
-#ifdef DMA_PROF
-    const char* prof_env = getenv("DMA_PROF_PTR");
-    fp.prof = prof_env ? (long long*)strtoull(prof_env, nullptr, 10) : nullptr;
-#endif
     const size_t smem = sizeof(SharedStorage) + 1024;
     dim3 grid(P.B * P.Hq, npairs);
     timing_mark(0, false, st);

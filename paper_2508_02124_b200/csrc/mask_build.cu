@@ -92,23 +92,33 @@ __global__ void __launch_bounds__(256) delta_kernel(const T* __restrict__ V, con
     for (int i = tid; i < G * D; i += 256) sW[i] = W[(size_t)hk * G * D + i];
     __syncthreads();
     const int rows = min(kRows, L - j0);                   // a short range (one appended key) does not walk 128 row slots
-    for (int r0 = warp * RPW; r0 < rows; r0 += 8 * RPW) {
-        const int r = r0 + grp, j = j0 + r;
-        float v[8];
-        if (j < L) {
-            load8(V + b * vs_b + (int64_t)j * vs_l + hk * vs_h + sub * 8, v);
+    // A warp owns kPass = kRows / (8 RPW) row groups. All their value rows are requested before the first is used (the
+    // kernel is bound by the V stream: one 16-byte load in flight per lane would leave the memory system idle), then
+    // the chains run out of registers.
+    constexpr int kPass = kRows / (8 * RPW);
+    float v[kPass][8];
+#pragma unroll
+    for (int t = 0; t < kPass; ++t) {
+        const int r = warp * RPW + grp + t * 8 * RPW, j = j0 + r;
+        if (r < rows && j < L) {
+            load8(V + b * vs_b + (int64_t)j * vs_l + hk * vs_h + sub * 8, v[t]);
         } else {
 #pragma unroll
-            for (int c = 0; c < 8; ++c) v[c] = 0.0f;
+            for (int c = 0; c < 8; ++c) v[t][c] = 0.0f;
         }
-        for (int g = 0; g < G; ++g) {
-            const float* w = sW + g * D + sub * 8;
+    }
+    for (int g = 0; g < G; ++g) {
+        const float4 wa = *reinterpret_cast<const float4*>(sW + g * D + sub * 8), wb = *reinterpret_cast<const float4*>(sW + g * D + sub * 8 + 4);
+        const float w[8] = {wa.x, wa.y, wa.z, wa.w, wb.x, wb.y, wb.z, wb.w};
+#pragma unroll
+        for (int t = 0; t < kPass; ++t) {
             float p = 0.0f;
 #pragma unroll
-            for (int c = 0; c < 8; ++c) p = __fmaf_rn(v[c], w[c], p);
+            for (int c = 0; c < 8; ++c) p = __fmaf_rn(v[t][c], w[c], p);
 #pragma unroll
             for (int m = 1; m < LPR; m <<= 1) p = __fadd_rn(p, __shfl_xor_sync(0xffffffffu, p, m));
-            if (sub == g % LPR) sOut[g * kRows + r] = p;      // z; softplus and exp follow, one (row, head) pair per thread
+            const int r = warp * RPW + grp + t * 8 * RPW;
+            if (sub == g % LPR && r < rows) sOut[g * kRows + r] = p;      // z; softplus and exp follow, one (row, head) pair per thread
         }
     }
     __syncthreads();

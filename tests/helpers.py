@@ -11,9 +11,12 @@ from paper_2508_02124_b200 import binding as dma
 # Parity gate by element type: (atol, whole-tensor relative L2). bf16: 2e-2 / 5e-3; fp32: 1e-4 / 1e-4. The relative L2
 # bound always applies. The max-abs bound is applied per ELEMENT, in the form the arithmetic of each output gives:
 #
-#   forward outputs (O, decode o)   |err| <= atol + K_OUT * u * |ref|          u = 2^-8 (bf16: half the output spacing is
-#                                    <= 2^-8 |ref|) or 2^-24 (fp32). O is a convex combination of value rows: the atol term
-#                                    is the stated absolute bound, the second is the rounding of the stored output itself.
+#   forward outputs (O, decode o)   |err| <= atol + K_OUT * u * |ref|, K_OUT = 2, u = 2^-8 (bf16) or 2^-24 (fp32): one
+#                                    spacing of the output format. O is a convex combination of value rows: the atol term is
+#                                    the stated absolute bound; of the second, half is the rounding of the stored output
+#                                    itself and half the rounding of P to bf16 before P V (relative 2^-9 per entry, which
+#                                    does not average out in a row that one key dominates). It matters only for |O| >> 1
+#                                    (value rows scaled x 4 in the long-context configuration: |O| up to 15, spacing 2^-4).
 #   dQ, dK, dV (Alg. 2 sums)        |err| <= atol * max(1, R)                  R = max |ref| over the d channels of the
 #                                    element's own row (one query row of dQ, one key row of dK / dV). Every channel of a
 #                                    row is a sum over the same (row, key) pairs with the same bf16-rounded weights (P for
@@ -28,7 +31,7 @@ from paper_2508_02124_b200 import binding as dma
 #                                    atol + 1e-6 M, a few fp32 ulps of that magnitude.
 TOL = {"bf16": (2e-2, 5e-3), "fp32": (1e-4, 1e-4)}
 UNIT = {"bf16": 2.0 ** -8, "fp32": 2.0 ** -24}
-K_OUT = 1.0
+K_OUT = 2.0
 
 
 def round_to(case, a):
@@ -53,8 +56,18 @@ def gpu_mask(case, inp, **kw):
     return p, bias, expiry, bitmap
 
 
-def gpu_run(case, inp, backward=True, mask=None, **kw):
-    """Full path on the GPU. `mask` = (bias, expiry, bitmap) CPU/GPU tensors to inject instead of building one."""
+def stored_forward(case, O, lse, rows=None):
+    """The forward outputs as Alg. 2 reads them back from memory, for handing to BOTH backward passes: O rounded to the
+    element type and lse rounded to fp32, either whole tensors or (with `rows`) the listed query rows only."""
+    return {"O": round_to(case, O), "lse": np.asarray(lse, np.float32), "rows": None if rows is None else np.asarray(rows)}
+
+
+def gpu_run(case, inp, backward=True, mask=None, stored=None, **kw):
+    """Full path on the GPU. `mask` = (bias, expiry, bitmap) CPU/GPU tensors to inject instead of building one.
+    `stored` (from stored_forward, i.e. values computed on the CPU by the oracle) replaces, as INPUT of dma_attn_bwd, the
+    forward output O and lse on all rows or on the listed rows: Alg. 2 takes the stored O and the softmax statistics as
+    inputs, so the backward kernels are compared with the oracle's backward on the same inputs (the GPU forward's own O
+    and lse are still returned and compared on their own)."""
     dev = torch.device("cuda:0")
     p = problem_of(case, **kw)
     Q, K, V, dO = (inp[k].to(dev) for k in ("Q", "K", "V", "dO"))
@@ -62,10 +75,26 @@ def gpu_run(case, inp, backward=True, mask=None, **kw):
         bias, expiry, bitmap = dma.dma_mask_build(p, V, inp["W_delta"].to(dev), inp["A"].to(dev))
     else:
         bias, expiry, bitmap = (torch.as_tensor(m).to(dev) for m in mask)
-    O, lse = dma.dma_attn_fwd(p, Q, K, V, bias, expiry, bitmap)
+    _, f_ws, b_ws = dma.dma_query_workspace(p)
+    wsf = torch.empty(f_ws, dtype=torch.uint8, device=dev)
+    O, lse = dma.dma_attn_fwd(p, Q, K, V, bias, expiry, bitmap, ws=wsf)
+    assert dma.dma_read_status(wsf) == 0, "device status after the forward"
     out = {"bias": bias, "expiry": expiry, "bitmap": bitmap, "O": O, "lse": lse}
     if backward:
-        dQ, dK, dV, dM = dma.dma_attn_bwd(p, Q, K, V, O, dO, lse, bias, expiry, bitmap)
+        O_in, lse_in = O, lse
+        if stored is not None:
+            so = torch.from_numpy(stored["O"]).to(case.torch_dtype).to(dev)
+            sl = torch.from_numpy(stored["lse"]).to(dev)
+            if stored["rows"] is None:
+                O_in, lse_in = so.contiguous(), sl.contiguous()
+            else:
+                idx = torch.from_numpy(stored["rows"].astype(np.int64)).to(dev)
+                O_in, lse_in = O.clone(), lse.clone()
+                O_in[:, idx] = so
+                lse_in[:, :, idx] = sl
+        wsb = torch.empty(b_ws, dtype=torch.uint8, device=dev)
+        dQ, dK, dV, dM = dma.dma_attn_bwd(p, Q, K, V, O_in, dO, lse_in, bias, expiry, bitmap, ws=wsb)
+        assert dma.dma_read_status(wsb) == 0, "device status after the backward"
         out.update(dQ=dQ, dK=dK, dV=dV, dM=dM)
     torch.cuda.synchronize()
     return out

@@ -8,7 +8,7 @@ import oracle
 from paper_2508_02124_b200 import binding as dma
 from paper_2508_02124_b200 import workloads as wl
 
-from helpers import assert_close, f64, gpu_run, oracle_mask, problem_of, round_to
+from helpers import assert_close, f64, gpu_run, oracle_mask, problem_of, round_to, stored_forward
 
 pytestmark = pytest.mark.gpu
 
@@ -38,24 +38,30 @@ def oracle_all(case, inp, bias, e, backward=True):
     return out
 
 
-def compare(case, got, ref, backward=True):
+def compare(case, got, ref, backward=True, end_to_end=False):
+    """end_to_end: the GPU backward read the GPU forward's own stored O (dma_step_host cannot be handed another), which
+    differs from the oracle's stored O wherever the two forwards round an element to different neighbours; D = rowsum(dO o O)
+    of Alg. 2 carries those one-ulp differences into every dS of the row, so the gradients are held to the bound relative
+    to the tensor's largest magnitude there. Everywhere else both backward passes read the same stored O and the
+    per-row / per-head bounds apply."""
     assert_close(got["O"], ref["O"], case.dtype, "O")
     assert_close(got["lse"], ref["lse"], case.dtype, "lse", lse=True)
     if backward:
         for k in ("dQ", "dK", "dV", "dM"):
-            assert_close(got[k], ref[k], case.dtype, k)
+            assert_close(got[k], ref[k], case.dtype, k, kind="tensor" if end_to_end else None)
 
 
 @pytest.mark.parametrize("case", CASES, ids=lambda c: c.name)
 def test_forward_backward_small(case):
     inp = wl.make_inputs(case)
     dl, e, bmp = oracle_mask(case, inp)
-    got = gpu_run(case, inp)
-    assert np.array_equal(got["expiry"].cpu().numpy(), e)
     ref = oracle_all(case, inp, dl, e)
+    st = stored_forward(case, ref["O"], ref["lse"])          # both backward passes read the same stored forward output
+    got = gpu_run(case, inp, stored=st)
+    assert np.array_equal(got["expiry"].cpu().numpy(), e)
     compare(case, got, ref)
     # block skipping is an optimisation only: ignoring the bitmap must give the same result
-    again = gpu_run(case, inp, flags=dma.DMA_FLAG_IGNORE_BITMAP)
+    again = gpu_run(case, inp, stored=st, flags=dma.DMA_FLAG_IGNORE_BITMAP)
     compare(case, again, ref)
 
 
@@ -63,7 +69,8 @@ def test_forward_backward_small(case):
 def test_cuda_core_kernels_on_bf16(case):
     inp = wl.make_inputs(case)
     dl, e, bmp = oracle_mask(case, inp)
-    compare(case, gpu_run(case, inp, flags=dma.DMA_FLAG_SIMT), oracle_all(case, inp, dl, e))
+    ref = oracle_all(case, inp, dl, e)
+    compare(case, gpu_run(case, inp, stored=stored_forward(case, ref["O"], ref["lse"]), flags=dma.DMA_FLAG_SIMT), ref)
 
 
 def test_injected_mask_zero_bias_is_dense_causal_attention():
@@ -74,12 +81,13 @@ def test_injected_mask_zero_bias_is_dense_causal_attention():
     bias = np.zeros((B, Hq, L), np.float32)
     e = np.full((B, Hq, L), L, np.int32)
     bmp = oracle.bitmap_from_expiry(e).view(np.int32)
-    got = gpu_run(case, inp, mask=(bias, e, bmp))
+    ref_all = oracle_all(case, inp, bias, e)
+    got = gpu_run(case, inp, mask=(bias, e, bmp), stored=stored_forward(case, ref_all["O"], ref_all["lse"]))
     q, k, v = (inp[n].double().permute(0, 2, 1, 3) for n in ("Q", "K", "V"))
     G = Hq // case.Hkv
     ref = torch.nn.functional.scaled_dot_product_attention(q, k.repeat_interleave(G, 1), v.repeat_interleave(G, 1), is_causal=True)
     assert_close(got["O"], ref.permute(0, 2, 1, 3).numpy(), "bf16", "O vs SDPA")
-    compare(case, got, oracle_all(case, inp, bias, e))
+    compare(case, got, ref_all)
 
 
 def test_skipped_tiles_do_not_change_the_result_on_a_banded_mask():
@@ -92,43 +100,9 @@ def test_skipped_tiles_do_not_change_the_result_on_a_banded_mask():
     active = ((bmp[..., t // 32] >> (t % 32)) & 1).sum()
     assert active < 0.8 * case.B * case.Hq * T * (T + 1) / 2           # the mask really has holes
     ref = oracle_all(case, inp, dl, e)
-    compare(case, gpu_run(case, inp, flags=dma.DMA_FLAG_TILE_PATH), ref)
-    compare(case, gpu_run(case, inp, flags=dma.DMA_FLAG_IGNORE_BITMAP), ref)
-
-
-def sampled_check(case, inp, got, nrows=24, nkeys=6, seed=0, forward_only=False):
-    """Full-size parity on sampled outputs: query rows (O, lse, dQ) and keys (dK, dV, dM) that the oracle
-    evaluates one by one. Keys are sampled near the end of the sequence, where few rows can keep them."""
-    rng = np.random.default_rng(seed)
-    dl, e, _ = oracle_mask(case, inp)
-    Q, K, V, dO = (f64(inp[k]) for k in ("Q", "K", "V", "dO"))
-    L = case.L
-    rows = np.unique(np.concatenate([[0, 1, 127, 128, L - 1], rng.integers(0, L, nrows)])).astype(np.int32)
-    O, lse = oracle.forward(Q, K, V, dl.astype(np.float64), expiry=e, rows=rows)
-    assert_close(got["O"][:, rows], O, case.dtype, "O rows")
-    assert_close(got["lse"][:, :, rows], lse, case.dtype, "lse rows", lse=True)
-    if forward_only or not case.backward:
-        return
-    keys = np.unique(np.concatenate([[L - 1, L - 130], rng.integers(L - 600, L, nkeys)])).astype(np.int32)
-    tail = np.arange(L - 600, L, dtype=np.int32)               # the only rows that can keep those keys
-    Ot, _ = oracle.forward(Q, K, V, dl.astype(np.float64), expiry=e, rows=tail)
-    Ostored = np.zeros_like(Q)
-    Ostored[:, tail] = round_to(case, Ot)                      # Alg. 2 reads the stored (rounded) forward output
-    _, dK, dV, dM = oracle.backward(Q, K, V, dO, dl.astype(np.float64), expiry=e, keys=keys, want_dq=False, O=Ostored)
-    assert_close(got["dK"][:, keys], dK, case.dtype, "dK keys")
-    assert_close(got["dV"][:, keys], dV, case.dtype, "dV keys")
-    assert_close(got["dM"][:, :, keys], dM, case.dtype, "dM keys")
-    # properties that hold at any size (Sec. 4.3): rows of dS sum to zero; q.dQ and k.dK balance per KV group
-    # (D is formed from the stored, rounded O, so each row of dS sums to dO_i.(O_i - stored O_i), at most
-    # half a bf16 ulp of every |dO_ic O_ic| term; in fp32 the bound is the accumulation error)
-    dMs = f64(got["dM"]).sum(-1)
-    half_ulp = 2.0 ** -9 if case.dtype == "bf16" else 2.0 ** -20
-    bound = half_ulp * (np.abs(dO) * np.abs(f64(got["O"]))).sum((1, 3)) + 1e-3
-    assert (np.abs(dMs) <= bound).all(), (dMs, bound)
-    G = case.Hq // case.Hkv
-    lhs = (Q * f64(got["dQ"])).sum(-1).reshape(case.B, L, case.Hkv, G).sum((1, 3))
-    rhs = (K * f64(got["dK"])).sum(-1).sum(1)
-    assert np.abs(lhs - rhs).max() <= 2e-2 * max(1.0, np.abs(rhs).max())
+    st = stored_forward(case, ref["O"], ref["lse"])
+    compare(case, gpu_run(case, inp, stored=st, flags=dma.DMA_FLAG_TILE_PATH), ref)
+    compare(case, gpu_run(case, inp, stored=st, flags=dma.DMA_FLAG_IGNORE_BITMAP), ref)
 
 
 def dq_rows(case):
@@ -140,26 +114,68 @@ def dq_rows(case):
     return np.unique(np.clip(np.array(rows, np.int64), 0, L - 1)).astype(np.int32)
 
 
-def dq_rows_check(case, inp, got, rows=None):
-    """dQ on sampled rows, every head, against the oracle's row-subset routine (dQ_i depends on row i alone); Alg. 2's D
-    uses the oracle's own forward output of those rows rounded to the element type."""
-    rows = dq_rows(case) if rows is None else rows
-    dl, e, _ = oracle_mask(case, inp)
-    Q, K, V, dO = (f64(inp[k]) for k in ("Q", "K", "V", "dO"))
-    bias = dl.astype(np.float64)
-    Or, _ = oracle.forward(Q, K, V, bias, expiry=e, rows=rows)
-    dQ = oracle.backward_dq_rows(Q, K, V, dO, bias, rows, expiry=e, O=round_to(case, Or))
-    assert_close(got["dQ"][:, rows], dQ, case.dtype, "dQ rows")
+class Samples:
+    """Full-size parity on sampled outputs: query rows (O, lse, dQ) and keys (dK, dV, dM) that the oracle evaluates one
+    by one, computed BEFORE the GPU runs. Keys are sampled near the end of the sequence, where only the last 600 rows can
+    keep them; dQ rows cover the region where the mask drops keys. `stored` holds the oracle's forward output on every
+    row the sampled gradients depend on: the GPU backward is given those rows as its stored O / lse (Alg. 2 takes them
+    as inputs), so both backward passes work from the same values."""
+
+    def __init__(self, case, inp, nrows=24, nkeys=6, seed=0, forward_only=False):
+        rng = np.random.default_rng(seed)
+        self.case, self.inp = case, inp
+        self.backward = case.backward and not forward_only
+        self.dl, self.e, _ = oracle_mask(case, inp)
+        Q, K, V, dO = (f64(inp[k]) for k in ("Q", "K", "V", "dO"))
+        L, bias = case.L, self.dl.astype(np.float64)
+        rows = np.concatenate([[0, 1, 127, 128, L - 1], rng.integers(0, L, nrows)])
+        if self.backward:
+            self.keys = np.unique(np.concatenate([[L - 1, L - 130], rng.integers(L - 600, L, nkeys)])).astype(np.int32)
+            tail = np.arange(L - 600, L)                             # the only rows that can keep those keys
+            self.dq = dq_rows(case)
+            rows = np.concatenate([rows, tail, self.dq])
+        self.rows = np.unique(rows).astype(np.int32)
+        self.O, self.lse = oracle.forward(Q, K, V, bias, expiry=self.e, rows=self.rows)
+        self.stored = stored_forward(case, self.O, self.lse, rows=self.rows)
+        if self.backward:
+            Ostored = np.zeros_like(Q)
+            Ostored[:, self.rows] = self.stored["O"]                 # Alg. 2 reads the stored (rounded) forward output
+            _, self.dK, self.dV, self.dM = oracle.backward(Q, K, V, dO, bias, expiry=self.e, keys=self.keys, want_dq=False, O=Ostored)
+            at = np.searchsorted(self.rows, self.dq)
+            self.dQ = oracle.backward_dq_rows(Q, K, V, dO, bias, self.dq, expiry=self.e, O=self.stored["O"][:, at])
+
+    def check(self, got, tag=""):
+        case = self.case
+        assert_close(got["O"][:, self.rows], self.O, case.dtype, tag + "O rows")
+        assert_close(got["lse"][:, :, self.rows], self.lse, case.dtype, tag + "lse rows", lse=True)
+        if not self.backward:
+            return
+        assert_close(got["dK"][:, self.keys], self.dK, case.dtype, tag + "dK keys")
+        assert_close(got["dV"][:, self.keys], self.dV, case.dtype, tag + "dV keys")
+        assert_close(got["dM"][:, :, self.keys], self.dM, case.dtype, tag + "dM keys")
+        assert_close(got["dQ"][:, self.dq], self.dQ, case.dtype, tag + "dQ rows")
+        # properties that hold at any size (Sec. 4.3): rows of dS sum to zero; q.dQ and k.dK balance per KV group
+        # (D is formed from the stored, rounded O, so each row of dS sums to dO_i.(O_i - stored O_i), at most
+        # half a bf16 ulp of every |dO_ic O_ic| term; in fp32 the bound is the accumulation error)
+        Q, K, dO = (f64(self.inp[k]) for k in ("Q", "K", "dO"))
+        L = case.L
+        dMs = f64(got["dM"]).sum(-1)
+        half_ulp = 2.0 ** -9 if case.dtype == "bf16" else 2.0 ** -20
+        bound = half_ulp * (np.abs(dO) * np.abs(f64(got["O"]))).sum((1, 3)) + 1e-3
+        assert (np.abs(dMs) <= bound).all(), (dMs, bound)
+        G = case.Hq // case.Hkv
+        lhs = (Q * f64(got["dQ"])).sum(-1).reshape(case.B, L, case.Hkv, G).sum((1, 3))
+        rhs = (K * f64(got["dK"])).sum(-1).sum(1)
+        assert np.abs(lhs - rhs).max() <= 2e-2 * max(1.0, np.abs(rhs).max())
 
 
 @pytest.mark.parametrize("key", ["2", "3", "3x3", "4w256", "4w2048", "4w8192", "5", "S"])
 def test_full_size_configs_sampled(key):
     case = wl.CONFIGS[key]
     inp = wl.make_inputs(case)
-    got = gpu_run(case, inp, backward=case.backward, flags=dma.DMA_FLAG_TILE_PATH)       # the tile-walking kernels (Alg. 1 / Alg. 2)
-    sampled_check(case, inp, got)
-    if case.backward:
-        dq_rows_check(case, inp, got)
+    ref = Samples(case, inp)
+    # the tile-walking kernels (Alg. 1 / Alg. 2 with block skipping)
+    ref.check(gpu_run(case, inp, backward=case.backward, stored=ref.stored, flags=dma.DMA_FLAG_TILE_PATH))
 
 
 def test_default_flags_choose_the_path_from_the_descriptor():
@@ -192,19 +208,18 @@ def test_largest_supported_lengths():
     step-list capacity). Sampled rows and keys against the oracle."""
     fwd = wl.small(wl.CONFIGS["5"], B=1, Hq=4, Hkv=2, L=131072, w=4096, backward=False, name="max L forward")
     inp = wl.make_inputs(fwd)
+    ref = Samples(fwd, inp, nrows=10, forward_only=True)
     got = gpu_run(fwd, inp, backward=False, flags=dma.DMA_FLAG_TILE_PATH)
-    sampled_check(fwd, inp, got, nrows=10, forward_only=True)
-    gc = gpu_run(fwd, inp, backward=False, flags=dma.DMA_FLAG_COMPACT_KV)
-    sampled_check(fwd, inp, gc, nrows=10, forward_only=True)
+    ref.check(got)
+    ref.check(gpu_run(fwd, inp, backward=False, flags=dma.DMA_FLAG_COMPACT_KV), "compact ")
     with pytest.raises(dma.DmaError) as e:                        # one tile more is refused, not mis-executed
         too_long = wl.small(fwd, L=131072 + 128)
         dma.dma_attn_fwd(problem_of(too_long, flags=dma.DMA_FLAG_TILE_PATH), got["O"], got["O"], got["O"], got["bias"], got["expiry"], got["bitmap"])
     assert e.value.status == -4
     both = wl.small(wl.CONFIGS["3"], B=1, Hq=4, Hkv=1, L=65536, w=2048, backward=True, name="max L backward")
     inp = wl.make_inputs(both)
-    got = gpu_run(both, inp, flags=dma.DMA_FLAG_TILE_PATH)
-    sampled_check(both, inp, got, nrows=8, nkeys=4)
-    dq_rows_check(both, inp, got)
+    ref = Samples(both, inp, nrows=8, nkeys=4)
+    ref.check(gpu_run(both, inp, stored=ref.stored, flags=dma.DMA_FLAG_TILE_PATH))
 
 
 def test_whole_step_can_be_captured_in_a_cuda_graph():
@@ -288,8 +303,7 @@ def test_compact_forward_small_cases(kw):
 def test_compact_forward_full_size_sampled(key):
     case = wl.CONFIGS[key]
     inp = wl.make_inputs(case)
-    got = _compact_run(case, inp)
-    sampled_check(case, inp, got, forward_only=True)
+    Samples(case, inp, forward_only=True).check(_compact_run(case, inp), "compact ")
 
 
 def test_compact_flag_is_rejected_where_unsupported():
@@ -311,8 +325,9 @@ def test_bf16_d64_runs_on_the_tensor_core_kernels():
     inp = wl.make_inputs(case)
     dl, e, _ = oracle_mask(case, inp)
     ref = oracle_all(case, inp, dl, e)
+    st = stored_forward(case, ref["O"], ref["lse"])
     for flags in (0, dma.DMA_FLAG_COMPACT_KV):
-        compare(case, gpu_run(case, inp, flags=flags), ref)
+        compare(case, gpu_run(case, inp, stored=st, flags=flags), ref)
     # strided Q / K / V / O views of wider buffers
     big = {k: torch.randn(case.B, case.L + 9, (case.Hq if k in ("Q", "dO") else case.Hkv) + 1, 64).to(case.torch_dtype).to(dev) for k in ("Q", "K", "V", "dO")}
     view = {k: big[k][:, 3:3 + case.L, 1:] for k in big}
@@ -325,7 +340,9 @@ def test_bf16_d64_runs_on_the_tensor_core_kernels():
     Obuf = torch.zeros_like(big["dO"])
     O, lse = dma.dma_attn_fwd(p, view["Q"], view["K"], view["V"], bias, expiry, bitmap, O=Obuf[:, 3:3 + case.L, 1:])
     dQb, dKb, dVb = torch.zeros_like(big["Q"]), torch.zeros_like(big["K"]), torch.zeros_like(big["V"])
-    dQ, dK, dV, dM = dma.dma_attn_bwd(p, view["Q"], view["K"], view["V"], O, view["dO"], lse, bias, expiry, bitmap,
+    Oin = torch.zeros_like(big["dO"])[:, 3:3 + case.L, 1:]                       # the oracle's stored O in the same strided layout
+    Oin.copy_(torch.from_numpy(st["O"]).to(case.torch_dtype).to(dev))
+    dQ, dK, dV, dM = dma.dma_attn_bwd(p, view["Q"], view["K"], view["V"], Oin, view["dO"], torch.from_numpy(st["lse"]).to(dev), bias, expiry, bitmap,
                                       dQ=dQb[:, 3:3 + case.L, 1:], dK=dKb[:, 3:3 + case.L, 1:], dV=dVb[:, 3:3 + case.L, 1:])
     torch.cuda.synchronize()
     compare(case, {"O": O, "lse": lse, "dQ": dQ, "dK": dK, "dV": dV, "dM": dM}, ref)
@@ -366,36 +383,21 @@ def test_compact_kernels_on_strided_k_and_v():
 
 # ---- token-compacted backward (DMA_FLAG_COMPACT_KV): key tiles follow a lifetime-sorted permutation per query head -----
 
-def _compact_full_run(case, inp):
-    dev = torch.device("cuda:0")
-    pc = problem_of(case, flags=dma.DMA_FLAG_COMPACT_KV)
-    Q, K, V, dO = (inp[k].to(dev) for k in ("Q", "K", "V", "dO"))
-    bias, expiry, bitmap = dma.dma_mask_build(pc, V, inp["W_delta"].to(dev), inp["A"].to(dev))
-    m, f, bw = dma.dma_query_workspace(pc)
-    wsf = torch.empty(f, dtype=torch.uint8, device=dev)
-    wsb = torch.empty(bw, dtype=torch.uint8, device=dev)
-    O, lse = dma.dma_attn_fwd(pc, Q, K, V, bias, expiry, bitmap, ws=wsf)
-    dQ, dK, dV, dM = dma.dma_attn_bwd(pc, Q, K, V, O, dO, lse, bias, expiry, bitmap, ws=wsb)
-    torch.cuda.synchronize()
-    assert dma.dma_read_status(wsf) == 0 and dma.dma_read_status(wsb) == 0
-    return {"bias": bias, "expiry": expiry, "bitmap": bitmap, "O": O, "lse": lse, "dQ": dQ, "dK": dK, "dV": dV, "dM": dM}
-
-
 @pytest.mark.parametrize("case", [c for c in CASES if c.dtype == "bf16" and c.d == 128], ids=lambda c: c.name)
 def test_compact_backward_small_cases(case):
     # the same small cases as the tile path (ragged tails and padding entries in the permutation, several query heads
     # adding into one KV head, w = 1 where almost every key is never kept, w >= L where nothing expires, peaked scores)
     inp = wl.make_inputs(case)
     dl, e, _ = oracle_mask(case, inp)
-    got = _compact_full_run(case, inp)
+    ref = oracle_all(case, inp, dl, e)
+    got = gpu_run(case, inp, stored=stored_forward(case, ref["O"], ref["lse"]), flags=dma.DMA_FLAG_COMPACT_KV)
     assert np.array_equal(got["expiry"].cpu().numpy(), e)
-    compare(case, got, oracle_all(case, inp, dl, e))
+    compare(case, got, ref)
 
 
 @pytest.mark.parametrize("key", ["3", "4w256", "4w2048", "S"])
 def test_compact_backward_full_size_sampled(key):
     case = wl.CONFIGS[key]
     inp = wl.make_inputs(case)
-    got = _compact_full_run(case, inp)
-    sampled_check(case, inp, got)
-    dq_rows_check(case, inp, got)
+    ref = Samples(case, inp)
+    ref.check(gpu_run(case, inp, stored=ref.stored, flags=dma.DMA_FLAG_COMPACT_KV), "compact ")

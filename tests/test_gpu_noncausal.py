@@ -7,7 +7,8 @@ import torch
 import oracle
 from paper_2508_02124_b200 import binding as dma
 from paper_2508_02124_b200 import workloads as wl
-from helpers import assert_close, f64, round_to
+from helpers import assert_close, f64, round_to, stored_forward
+from test_gpu_varlen import patched
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
@@ -41,14 +42,15 @@ def problem(case, flags=0):
     return dma.problem(case.B, case.Hq, case.Hkv, case.L, case.d, case.w, dtype=case.torch_dtype, causal=0, flags=flags)
 
 
-def gpu(case, inp, flags=0, backward=True):
+def gpu(case, inp, flags=0, backward=True, stored=None):
     p = problem(case, flags)
     Q, K, V, dO = (inp[k].to(DEV) for k in ("Q", "K", "V", "dO"))
     bias, expiry, bitmap = dma.dma_mask_build(p, V, inp["W_delta"].to(DEV), inp["A"].to(DEV))
     O, lse = dma.dma_attn_fwd(p, Q, K, V, bias, expiry, bitmap)
     out = {"bias": bias, "expiry": expiry, "bitmap": bitmap, "O": O, "lse": lse}
     if backward:
-        dQ, dK, dV, dM = dma.dma_attn_bwd(p, Q, K, V, O, dO, lse, bias, expiry, bitmap)
+        O_in, lse_in = patched(case, O, lse, stored)          # Alg. 2's stored forward output: the oracle's, for both sides
+        dQ, dK, dV, dM = dma.dma_attn_bwd(p, Q, K, V, O_in, dO, lse_in, bias, expiry, bitmap)
         out.update(dQ=dQ, dK=dK, dV=dV, dM=dM)
     torch.cuda.synchronize()
     return out
@@ -59,34 +61,39 @@ def oracle_mask(case, inp):
     return dl, oracle.select_noncausal(dl, case.w)
 
 
-def check_all(case, inp, got, dl, e):
+def oracle_all(case, inp, dl, e):
     Q, K, V, dO = (f64(inp[k]) for k in ("Q", "K", "V", "dO"))
     O, lse = oracle.forward(Q, K, V, dl.astype(np.float64), expiry=e, causal=False)
-    assert_close(got["O"], O, case.dtype, "O")
-    assert_close(got["lse"], lse, case.dtype, "lse", lse=True)
     dQ, dK, dV, dM = oracle.backward(Q, K, V, dO, dl.astype(np.float64), expiry=e, O=round_to(case, O), causal=False)
-    for k, ref in (("dQ", dQ), ("dK", dK), ("dV", dV), ("dM", dM)):
-        assert_close(got[k], ref, case.dtype, k)
+    return {"O": O, "lse": lse, "dQ": dQ, "dK": dK, "dV": dV, "dM": dM}
+
+
+def check_all(case, got, ref):
+    assert_close(got["O"], ref["O"], case.dtype, "O")
+    assert_close(got["lse"], ref["lse"], case.dtype, "lse", lse=True)
+    for k in ("dQ", "dK", "dV", "dM"):
+        assert_close(got[k], ref[k], case.dtype, k)
 
 
 @pytest.mark.parametrize("case", CASES, ids=lambda c: c.name)
 def test_mask_forward_backward_small(case):
     inp = inputs(case)
-    got = gpu(case, inp)
     dl, e = oracle_mask(case, inp)
+    ref = oracle_all(case, inp, dl, e)
+    got = gpu(case, inp, stored=stored_forward(case, ref["O"], ref["lse"]))
     assert np.array_equal(got["bias"].cpu().numpy().view(np.uint32), dl.view(np.uint32))
     assert np.array_equal(got["expiry"].cpu().numpy(), e)
     keep = oracle.keep_from_expiry_noncausal(e)
     assert np.array_equal(got["bitmap"].cpu().numpy().view(np.uint32), oracle.bitmap_definition(keep))
-    check_all(case, inp, got, dl, e)
+    check_all(case, got, ref)
 
 
 @pytest.mark.parametrize("case", [c for c in CASES if c.dtype == "bf16"], ids=lambda c: c.name)
 def test_cuda_core_kernels_on_bf16(case):
     inp = inputs(case)
-    got = gpu(case, inp, flags=dma.DMA_FLAG_SIMT)
     dl, e = oracle_mask(case, inp)
-    check_all(case, inp, got, dl, e)
+    ref = oracle_all(case, inp, dl, e)
+    check_all(case, gpu(case, inp, flags=dma.DMA_FLAG_SIMT, stored=stored_forward(case, ref["O"], ref["lse"])), ref)
 
 
 def test_last_row_equals_the_causal_last_row_on_the_gpu():
@@ -108,21 +115,32 @@ def test_config3_sampled():
     of the first KV group (the oracle needs every row for a kept key, so the problem is cut to one group)."""
     case = wl.CONFIGS["3"]
     inp = inputs(case)
-    got = gpu(case, inp)
     dl, e = oracle_mask(case, inp)
-    assert np.array_equal(got["expiry"].cpu().numpy(), e)
     Q, K, V, dO = (f64(inp[k]) for k in ("Q", "K", "V", "dO"))
+    G = case.Hq // case.Hkv
+    # the first KV group in full on the oracle: its forward output is the stored O / lse that both backward passes read
+    # for those heads (the other heads' backward, which is not compared, reads the GPU's own forward output)
+    Og, lg = oracle.forward(Q[:, :, :G], K[:, :, :1], V[:, :, :1], dl[:, :G].astype(np.float64), expiry=e[:, :G], causal=False)
+    p = problem(case)
+    Qd, Kd, Vd, dOd = (inp[k].to(DEV) for k in ("Q", "K", "V", "dO"))
+    bias, expiry, bitmap = dma.dma_mask_build(p, Vd, inp["W_delta"].to(DEV), inp["A"].to(DEV))
+    Od, lsed = dma.dma_attn_fwd(p, Qd, Kd, Vd, bias, expiry, bitmap)
+    O_in, lse_in = Od.clone(), lsed.clone()
+    O_in[:, :, :G] = torch.from_numpy(round_to(case, Og)).to(case.torch_dtype).to(DEV)
+    lse_in[:, :G] = torch.from_numpy(lg.astype(np.float32)).to(DEV)
+    dQd, dKd, dVd, dMd = dma.dma_attn_bwd(p, Qd, Kd, Vd, O_in, dOd, lse_in, bias, expiry, bitmap)
+    torch.cuda.synchronize()
+    got = {"expiry": expiry, "O": Od, "lse": lsed, "dQ": dQd, "dK": dKd, "dV": dVd, "dM": dMd}
+    assert np.array_equal(got["expiry"].cpu().numpy(), e)
     rng = np.random.default_rng(9)
     rows = np.unique(np.concatenate([[0, 1, 127, 128, case.L - 1], rng.integers(0, case.L, 16)])).astype(np.int32)
     O, lse = oracle.forward(Q, K, V, dl.astype(np.float64), expiry=e, rows=rows, causal=False)
     assert_close(got["O"][:, rows], O, case.dtype, "O rows")
     assert_close(got["lse"][:, :, rows], lse, case.dtype, "lse rows", lse=True)
-    G = case.Hq // case.Hkv
     kept = np.nonzero(e[0, :G].max(0))[0]
     dropped = np.nonzero(e[0, :G].max(0) == 0)[0]
     keys = np.unique(np.concatenate([rng.choice(kept, 4), rng.choice(dropped, 2)])).astype(np.int32)
     Qg, dOg = Q[:, :, :G], dO[:, :, :G]
-    Og, _ = oracle.forward(Qg, K[:, :, :1], V[:, :, :1], dl[:, :G].astype(np.float64), expiry=e[:, :G], causal=False)
     _, dK, dV, dM = oracle.backward(Qg, K[:, :, :1], V[:, :, :1], dOg, dl[:, :G].astype(np.float64), expiry=e[:, :G], keys=keys,
                                     want_dq=False, O=round_to(case, Og), causal=False)
     assert_close(got["dK"][:, keys, :1], dK, case.dtype, "dK keys")

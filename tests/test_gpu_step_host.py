@@ -58,15 +58,15 @@ def test_against_the_oracle():
     inp = wl.make_inputs(case)
     got = host_step(case, inp)
     dl, e, _ = oracle_mask(case, inp)
-    compare(case, got, oracle_all(case, inp, dl, e))
+    compare(case, got, oracle_all(case, inp, dl, e), end_to_end=True)
 
 
 def test_flags_that_keep_the_batch_entries_whole():
     case = wl.small(C2, B=2, Hq=8, Hkv=4, L=512, w=96, backward=True, name="host flags")
     inp = wl.make_inputs(case)
     dl, e, _ = oracle_mask(case, inp)
-    compare(case, host_step(case, inp, flags=dma.DMA_FLAG_COMPACT_KV), oracle_all(case, inp, dl, e))
+    compare(case, host_step(case, inp, flags=dma.DMA_FLAG_COMPACT_KV), oracle_all(case, inp, dl, e), end_to_end=True)
     W = wl.full_delta_weights(case)
     _, dlf = oracle.delta_full(inp["V"].float().numpy(), W.numpy(), inp["A"].numpy())
     ef = oracle.select_expiry(dlf, case.w)
-    compare(case, host_step(case, inp, flags=dma.DMA_FLAG_FULL_DELTA, W=W), oracle_all(case, inp, dlf, ef))
+    compare(case, host_step(case, inp, flags=dma.DMA_FLAG_FULL_DELTA, W=W), oracle_all(case, inp, dlf, ef), end_to_end=True)

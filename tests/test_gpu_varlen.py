@@ -7,7 +7,7 @@ import torch
 import oracle
 from paper_2508_02124_b200 import binding as dma
 from paper_2508_02124_b200 import workloads as wl
-from helpers import assert_close, f64, problem_of, round_to
+from helpers import assert_close, f64, problem_of, round_to, stored_forward
 from test_gpu_attention import compare, oracle_all
 
 pytestmark = pytest.mark.gpu
@@ -28,8 +28,23 @@ SMALL = [
 ]
 
 
-def run(case, cu, flags=0, backward=True):
-    inp = wl.make_inputs(case)
+def patched(case, O, lse, stored):
+    """The GPU forward's O / lse with the oracle's stored values written over all rows or over the listed rows (the
+    backward's inputs: Alg. 2 reads the stored forward output, and both backward passes are given the same one)."""
+    if stored is None:
+        return O, lse
+    so, sl = torch.from_numpy(stored["O"]).to(case.torch_dtype).to(DEV), torch.from_numpy(stored["lse"]).to(DEV)
+    if stored["rows"] is None:
+        return so.contiguous(), sl.contiguous()
+    idx = torch.from_numpy(stored["rows"].astype(np.int64)).to(DEV)
+    O, lse = O.clone(), lse.clone()
+    O[:, idx] = so
+    lse[:, :, idx] = sl
+    return O, lse
+
+
+def run(case, cu, flags=0, backward=True, stored=None, inp=None):
+    inp = wl.make_inputs(case) if inp is None else inp
     p = problem_of(case, flags=flags)
     Q, K, V, dO = (inp[k].to(DEV) for k in ("Q", "K", "V", "dO"))
     cu_t = torch.tensor(cu, dtype=torch.int32, device=DEV)
@@ -37,7 +52,8 @@ def run(case, cu, flags=0, backward=True):
     O, lse = dma.dma_attn_fwd(p, Q, K, V, bias, expiry, bitmap)
     got = {"bias": bias, "expiry": expiry, "bitmap": bitmap, "O": O, "lse": lse}
     if backward:
-        dQ, dK, dV, dM = dma.dma_attn_bwd(p, Q, K, V, O, dO, lse, bias, expiry, bitmap)
+        O_in, lse_in = patched(case, O, lse, stored)
+        dQ, dK, dV, dM = dma.dma_attn_bwd(p, Q, K, V, O_in, dO, lse_in, bias, expiry, bitmap)
         got.update(dQ=dQ, dK=dK, dV=dV, dM=dM)
     torch.cuda.synchronize()
     return inp, got
@@ -51,20 +67,24 @@ def oracle_varlen_mask(case, inp, cu):
 
 @pytest.mark.parametrize("case,cu", SMALL, ids=lambda v: v.name if hasattr(v, "name") else "")
 def test_mask_and_attention_small(case, cu):
-    inp, got = run(case, cu)
+    inp = wl.make_inputs(case)
     dl, e, bmp = oracle_varlen_mask(case, inp, cu)
+    ref = oracle_all(case, inp, dl, e)
+    _, got = run(case, cu, stored=stored_forward(case, ref["O"], ref["lse"]), inp=inp)
     assert np.array_equal(got["bias"].cpu().numpy().view(np.uint32), dl.view(np.uint32))
     assert np.array_equal(got["expiry"].cpu().numpy(), e)
     assert np.array_equal(got["bitmap"].cpu().numpy().view(np.uint32), bmp)
-    compare(case, got, oracle_all(case, inp, dl, e))
+    compare(case, got, ref)
 
 
 @pytest.mark.parametrize("case,cu", [c for c in SMALL if c[0].dtype == "bf16" and c[0].d == 128],
                          ids=lambda v: v.name if hasattr(v, "name") else "")
 def test_token_compacted_kernels_on_packed_sequences(case, cu):
-    inp, got = run(case, cu, flags=dma.DMA_FLAG_COMPACT_KV)
+    inp = wl.make_inputs(case)
     dl, e, _ = oracle_varlen_mask(case, inp, cu)
-    compare(case, got, oracle_all(case, inp, dl, e))
+    ref = oracle_all(case, inp, dl, e)
+    _, got = run(case, cu, flags=dma.DMA_FLAG_COMPACT_KV, stored=stored_forward(case, ref["O"], ref["lse"]), inp=inp)
+    compare(case, got, ref)
 
 
 def test_query_tile_whose_first_key_tiles_belong_to_another_document():
@@ -108,8 +128,26 @@ def test_config3_packed_documents():
     rows and keys; no key tile of another document is ever active."""
     case = wl.CONFIGS["3"]
     cu = wl.packed_cu_seqlens(case.L, 12, seed=31)
-    inp, got = run(case, cu, flags=dma.DMA_FLAG_TILE_PATH)
+    inp = wl.make_inputs(case)
     dl, e, bmp = oracle_varlen_mask(case, inp, cu)
+    Q, K, V, dO = (f64(inp[k]) for k in ("Q", "K", "V", "dO"))
+    rng = np.random.default_rng(5)
+    L = case.L
+    # sampled rows (document starts and ends included) and, for the gradients, every row of the last document: only its
+    # rows can keep its keys. The oracle's forward on those rows is the stored O / lse that both backward passes read.
+    s0 = cu[-2]
+    rows = np.unique(np.concatenate([[0, L - 1], np.asarray(cu[1:-1]) - 1, np.asarray(cu[1:-1]), rng.integers(0, L, 12),
+                                     np.arange(s0, L)])).astype(np.int32)
+    O, lse = oracle.forward(Q, K, V, dl.astype(np.float64), expiry=e, rows=rows)
+    st = stored_forward(case, O, lse, rows=rows)
+    keys = np.unique(np.concatenate([[s0, L - 1], rng.integers(s0, L, 5)])).astype(np.int32)
+    Ostored = np.zeros_like(Q)
+    Ostored[:, rows] = st["O"]
+    _, dK, dV, dM = oracle.backward(Q, K, V, dO, dl.astype(np.float64), expiry=e, keys=keys, want_dq=False, O=Ostored)
+    dq = np.unique(np.concatenate([[s0, s0 + 1, L - 1], rng.integers(s0, L, 5)])).astype(np.int32)
+    dQ = oracle.backward_dq_rows(Q, K, V, dO, dl.astype(np.float64), dq, expiry=e, O=st["O"][:, np.searchsorted(rows, dq)])
+
+    _, got = run(case, cu, flags=dma.DMA_FLAG_TILE_PATH, stored=st, inp=inp)
     assert np.array_equal(got["expiry"].cpu().numpy(), e)
     assert np.array_equal(got["bitmap"].cpu().numpy().view(np.uint32), bmp)
     seq_of = np.searchsorted(np.asarray(cu), np.arange(case.L), side="right") - 1
@@ -119,31 +157,14 @@ def test_config3_packed_documents():
         first_seq_start = cu[seq_of[qt * 128]]
         for kt in range(first_seq_start // 128):                 # tiles wholly before the first document of the query tile
             assert not (words[:, :, qt, kt // 32] >> np.uint32(kt % 32) & np.uint32(1)).any()
-    Q, K, V, dO = (f64(inp[k]) for k in ("Q", "K", "V", "dO"))
-    rng = np.random.default_rng(5)
-    L = case.L
-    rows = np.unique(np.concatenate([[0, L - 1], np.asarray(cu[1:-1]) - 1, np.asarray(cu[1:-1]), rng.integers(0, L, 12)])).astype(np.int32)
-    O, lse = oracle.forward(Q, K, V, dl.astype(np.float64), expiry=e, rows=rows)
-    assert_close(got["O"][:, rows], O, case.dtype, "O rows")
-    assert_close(got["lse"][:, :, rows], lse, case.dtype, "lse rows", lse=True)
-    # keys of the last document: only its rows can keep them
-    s0 = cu[-2]
-    keys = np.unique(np.concatenate([[s0, L - 1], rng.integers(s0, L, 5)])).astype(np.int32)
-    tail = np.arange(s0, L, dtype=np.int32)
-    Ot, _ = oracle.forward(Q, K, V, dl.astype(np.float64), expiry=e, rows=tail)
-    Ostored = np.zeros_like(Q)
-    Ostored[:, tail] = round_to(case, Ot)
-    _, dK, dV, dM = oracle.backward(Q, K, V, dO, dl.astype(np.float64), expiry=e, keys=keys, want_dq=False, O=Ostored)
-    assert_close(got["dK"][:, keys], dK, case.dtype, "dK keys")
-    assert_close(got["dV"][:, keys], dV, case.dtype, "dV keys")
-    assert_close(got["dM"][:, :, keys], dM, case.dtype, "dM keys")
-    # the token-compacted kernels on the same packed batch, against the same oracle samples
-    _, gc = run(case, cu, flags=dma.DMA_FLAG_COMPACT_KV)
-    assert_close(gc["O"][:, rows], O, case.dtype, "compact O rows")
-    assert_close(gc["lse"][:, :, rows], lse, case.dtype, "compact lse rows", lse=True)
-    assert_close(gc["dK"][:, keys], dK, case.dtype, "compact dK keys")
-    assert_close(gc["dV"][:, keys], dV, case.dtype, "compact dV keys")
-    assert_close(gc["dM"][:, :, keys], dM, case.dtype, "compact dM keys")
+    # the tile-walking kernels, then the token-compacted kernels on the same packed batch, against the same oracle samples
+    for tag, g in (("", got), ("compact ", run(case, cu, flags=dma.DMA_FLAG_COMPACT_KV, stored=st, inp=inp)[1])):
+        assert_close(g["O"][:, rows], O, case.dtype, tag + "O rows")
+        assert_close(g["lse"][:, :, rows], lse, case.dtype, tag + "lse rows", lse=True)
+        assert_close(g["dK"][:, keys], dK, case.dtype, tag + "dK keys")
+        assert_close(g["dV"][:, keys], dV, case.dtype, tag + "dV keys")
+        assert_close(g["dM"][:, :, keys], dM, case.dtype, tag + "dM keys")
+        assert_close(g["dQ"][:, dq], dQ, case.dtype, tag + "dQ rows")
 
 
 def test_argument_checks():
