@@ -77,6 +77,12 @@ enum {
                                     Alg. 2 with block skipping), never the token-compacted kernels. For masks whose kept
                                     keys cluster (packed documents, banded importance) tile skipping alone can be the
                                     faster choice; DMA_FLAG_IGNORE_BITMAP and DMA_FLAG_SIMT imply it */
+    DMA_FLAG_BLOCK_SKIP = 32,    /* dma_attn_fwd, tensor-core kernels: MMA-block skipping inside executed tiles (the finer
+                                    granularity below the 128 x 128 tile: "if there are no active tokens in the MMA block,
+                                    skip"). The P V product leaves out the 16-key blocks in which no key can be kept by the
+                                    query tile's rows; P is exactly zero there, so O and lse are the same bits. Off by
+                                    default: on the benchmark masks well under 5 % of the blocks of executed tiles are dead,
+                                    and the bookkeeping costs the kernel more than the multiplications it saves */
     DMA_FLAG_FULL_DELTA = 8      /* the sampling weights as Eq. (delta_calc) states them: W_delta (and dW_delta) is
                                     [Hq, Hkv*d], one row per query head over ALL channels of the value row (the linear
                                     layer of the App. A listing), z[b,h,j] = sum_{h'} V[b,j,h',:] . W_delta[h, h'*d:(h'+1)*d].

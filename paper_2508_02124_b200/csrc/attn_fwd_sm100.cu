@@ -48,8 +48,9 @@ struct SharedStorage {
     alignas(16) int len[kStages][128];        // expiry[j] (0 beyond L): row i keeps key j iff j <= i < expiry[j]
     alignas(16) int jidx[kStages][128];       // token-compacted mode: the key index of each gathered column
     int thr[2][16];                           // stager scratch: row thresholds of the keys that expire inside the tile
-    uint32_t fast[kStages][2];                // 1: the extra k-step carries the whole mask of this (key tile, query tile);
-                                              // token-compacted mode: bit q = 32-column chunk q needs the per-element test
+    uint32_t fast[kStages][2];                // bit 0: the extra k-step carries the whole mask of this (key tile, query tile);
+                                              // token-compacted mode: bit q (0-3) = 32-column chunk q needs the per-element test;
+                                              // bits 8-15: 16-key blocks that hold a key some row of the query tile may keep
     uint32_t sched[kMaxSched];                // key tile | use by tile 0 << 30 | use by tile 1 << 31
     uint64_t q_full, k_full[kStages], v_full[kStages], k_empty[kStages], v_empty[kStages];
     uint64_t s_full[2], p_half[2], p_ready[2], o_done[2];
@@ -95,7 +96,9 @@ constexpr int kWarpProducer = 0, kWarpIssuer = 1, kWarpStager0 = 2, kWarpStager1
 // asynchronous copies into the swizzled tile layout (TMA row gathers of four rows were measured at ~70 cycles per
 // request: too slow), warp 2 builds the B rows of the ninth k-step (bias, and -BIG for columns no row of the tile keeps; the A
 // rows are constant) and flags the 32-column chunks that still need the per-element test.
-template <bool kCompact>
+// kBlockSkip: MMA-block skipping inside executed tiles (DMA_FLAG_BLOCK_SKIP), a separate instantiation so that the
+// default kernel carries none of its code (the kernel is sensitive to the size of its service warps' loops).
+template <bool kCompact, bool kBlockSkip>
 __global__ void __launch_bounds__(kThreads, 1)
 fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
            const __grid_constant__ CUtensorMap tmV, const FwdParams P) {
@@ -188,7 +191,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             // has not followed that barrier's phases, and a parity wait on a barrier it is a whole phase ahead of returns
             // at once, before the stager has written the flag.)
             const uint32_t tile_flags = S.fast[st][w];
-            const bool fast_tile = kCompact || tile_flags != 0;      // token-compacted mode: the flags are a chunk mask instead
+            const bool fast_tile = kCompact || (tile_flags & 1u) != 0;      // token-compacted mode: the low bits are a chunk mask instead
             // The accumulator holds q.k + bias / scale (+ -BIG where the ninth k-step masks). On the fast path that
             // is the whole masked score; otherwise (diagonal tile, or more than 13 keys expiring inside the tile's
             // rows) the validity test j <= i < expiry[j] is applied here. x = log2e * scale * score, -inf if masked.
@@ -453,7 +456,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                     for (int t = 0; t < 4; ++t) jnn[t] = list[(it + 2) * 128 + lane + 32 * t];
                 }
                 // rows and flags are formed in registers before the waits
-                uint32_t b0[2][4], b1[4], flags[2] = {0u, 0u};
+                uint32_t b0[2][4], b1[4], flags[2] = {0u, 0u}, live[2] = {0u, 0u};
 #pragma unroll
                 for (int t = 0; t < 4; ++t) {
                     const float bsc = bv[t] * P.inv_scale;
@@ -471,6 +474,10 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                         const bool mixed = !dead && (ev[t] < i0 + 128 || first > i0);
                         b0[w][t] = dead ? kNegBig : w0;
                         flags[w] |= __ballot_sync(0xffffffffu, mixed) ? (1u << t) : 0u;
+                        if constexpr (kBlockSkip) {
+                            const uint32_t alive = __ballot_sync(0xffffffffu, !dead);
+                            live[w] |= ((alive & 0xFFFFu) ? 1u : 0u) << (2 * t) | ((alive >> 16) ? 1u : 0u) << (2 * t + 1);
+                        }
                     }
                 }
                 // the vectors of this stage were last read by the softmax groups before they released P of tile
@@ -489,7 +496,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                             make_uint4(b0[w][t], b0[w][t] == kNegBig ? 0u : b1[t], 0u, 0u);
                     jv[t] = jn[t]; bv[t] = bn[t]; ev[t] = en[t]; jn[t] = jnn[t];
                 }
-                if (lane < 2) S.fast[st][lane] = lane ? flags[1] : flags[0];
+                if (lane < 2) S.fast[st][lane] = (lane ? flags[1] : flags[0]) | ((kBlockSkip ? (lane ? live[1] : live[0]) : 0xFFu) << 8);
                 fence_proxy_async();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&S.k_full[st]);
@@ -567,6 +574,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                 uint32_t b0[4], b1[4], aw[4][7];
                 int hot[4];
                 bool fast = false;
+                uint32_t live8 = 0xFFu;
                 if (use) {
                     // general path needed: the tile holds keys that enter inside the query tile's rows (the diagonal tile)
                     const bool diag = (int)(entry & 0xFFFFF) == (w ? qt1 : qt0);
@@ -577,6 +585,14 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                         dead[t] = ev[t] <= i0;
                         mixed[t] = !dead[t] && ev[t] < i0 + 128;
                         bal[t] = __ballot_sync(0xffffffffu, mixed[t]);
+                    }
+                    if constexpr (kBlockSkip) {
+                        live8 = 0u;
+#pragma unroll
+                        for (int t = 0; t < 4; ++t) {
+                            const uint32_t alive = __ballot_sync(0xffffffffu, !dead[t]);     // keys 32 t .. 32 t + 31
+                            live8 |= ((alive & 0xFFFFu) ? 1u : 0u) << (2 * t) | ((alive >> 16) ? 1u : 0u) << (2 * t + 1);
+                        }
                     }
                     const int cnt = __popc(bal[0]) + __popc(bal[1]) + __popc(bal[2]) + __popc(bal[3]);
                     fast = !diag && cnt <= kMaskSlots;
@@ -643,7 +659,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                         *reinterpret_cast<uint4*>(arow) = make_uint4(kOne | (kOne << 16), aw[t][0], aw[t][1], aw[t][2]);
                         *reinterpret_cast<uint4*>(arow + 128) = make_uint4(aw[t][3], aw[t][4], aw[t][5], aw[t][6]);
                     }
-                    if (lane == 0) S.fast[st][w] = fast ? 1u : 0u;
+                    if (lane == 0) S.fast[st][w] = (fast ? 1u : 0u) | (live8 << 8);
                 }
 #pragma unroll
                 for (int t = 0; t < 4; ++t) {
@@ -668,6 +684,13 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             const uint64_t dA0 = smem_desc_plain(smem_u32(S.aext[0]), 128, 256), dB0 = smem_desc_plain(smem_u32(S.bext[0]), 128, 256);
             const uint32_t tmem_u = __shfl_sync(0xffffffffu, tmem, 0);
             const int n_iters_u = __shfl_sync(0xffffffffu, n_iters, 0);
+            // MMA-block skipping (the finer granularity inside an active tile): the stager marks the 16-key blocks of the key
+            // tile in which some key may be kept by the query tile's rows, and P V multiplies the marked blocks only (P is
+            // exactly zero in the others, so the result does not change). The S product is always multiplied in full: leaving
+            // out a dead 64-key half was built and measured (the issuer then needs the marks BEFORE the issue, a shared-memory
+            // load on the critical path: 1.98 -> 2.55 ms at L = 16384), so it stayed out.
+            uint32_t live[2] = {0xFFu, 0xFFu};          // marks of the key tile whose S product was issued last, per query tile
+            bool o_started[2] = {false, false};         // the O accumulator has been written (first product: no accumulate)
             auto issue_s = [&](int w, int st) {
                 const uint64_t dq = dQ0 + (uint64_t)(w * (kTileBytes >> 4)), dk = dK0 + (uint64_t)(st * (kTileBytes >> 4));
                 const uint32_t d_tmem = tmem_u + w * 128;
@@ -681,6 +704,9 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                     tc_commit(&S.s_full[w]);
                 }
                 __syncwarp();
+                // the block marks of this key tile, for its P V product later on: read AFTER the issue (a shared-memory load
+                // costs hundreds of cycles while the MMAs stream their operands, and the S products are on the critical path)
+                if constexpr (kBlockSkip) live[w] = *reinterpret_cast<volatile uint32_t*>(&S.fast[st][w]) >> 8;     // (every lane reads the same word; first used at the P V issue)
             };
             int n_p[2] = {0, 0};
             bool ok = mbar_wait_warp(&S.q_full, 0, abort_flag);
@@ -710,14 +736,27 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                         // P V in two halves of 64 keys: the first runs while the softmax group still forms the second
                         const uint64_t dv = dV0 + (uint64_t)(st * (kTileBytes >> 4));
                         const uint32_t d_tmem = tmem_u + 256 + w * 128, a_tmem = tmem_u + w * 128;
-                        const uint32_t acc0 = n_p[w] > 0 ? 1u : 0u;
+                        // blocks to multiply; an accumulator that has never been written takes block 0 in any case (P is zero there)
+                        const uint32_t l8 = !kBlockSkip ? 0xFFu : (!o_started[w] && live[w] == 0u) ? 1u : live[w];
+                        const uint32_t acc0 = o_started[w] ? 1u : 0u;
                         ok = mbar_wait_warp(&S.p_half[w], n_p[w] & 1, abort_flag);
                         if (ok) {
                             tc_fence_after();
                             if (elect_one()) {
+                                if (l8 == 0xFFu) {                                   // the common case: every block
 #pragma unroll
-                                for (int kk = 0; kk < 4; ++kk)
-                                    mma_ts(d_tmem, a_tmem + kk * 8, dv + (uint64_t)((kk * 2048) >> 4), idesc_pv, kk > 0 ? 1u : acc0);
+                                    for (int kk = 0; kk < 4; ++kk)
+                                        mma_ts(d_tmem, a_tmem + kk * 8, dv + (uint64_t)((kk * 2048) >> 4), idesc_pv, kk > 0 ? 1u : acc0);
+                                } else {
+                                    uint32_t acc = acc0;
+#pragma unroll
+                                    for (int kk = 0; kk < 4; ++kk) {
+                                        if ((l8 >> kk) & 1u) {
+                                            mma_ts(d_tmem, a_tmem + kk * 8, dv + (uint64_t)((kk * 2048) >> 4), idesc_pv, acc);
+                                            acc = 1u;
+                                        }
+                                    }
+                                }
                             }
                             __syncwarp();
                             ok = mbar_wait_warp(&S.p_ready[w], n_p[w] & 1, abort_flag);
@@ -725,12 +764,24 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                         if (ok) {
                             tc_fence_after();
                             if (elect_one()) {
+                                if (l8 == 0xFFu) {
 #pragma unroll
-                                for (int kk = 4; kk < 8; ++kk)
-                                    mma_ts(d_tmem, a_tmem + kk * 8, dv + (uint64_t)((kk * 2048) >> 4), idesc_pv, 1u);
+                                    for (int kk = 4; kk < 8; ++kk)
+                                        mma_ts(d_tmem, a_tmem + kk * 8, dv + (uint64_t)((kk * 2048) >> 4), idesc_pv, 1u);
+                                } else {
+                                    uint32_t acc = (acc0 || (l8 & 0x0Fu)) ? 1u : 0u;
+#pragma unroll
+                                    for (int kk = 4; kk < 8; ++kk) {
+                                        if ((l8 >> kk) & 1u) {
+                                            mma_ts(d_tmem, a_tmem + kk * 8, dv + (uint64_t)((kk * 2048) >> 4), idesc_pv, acc);
+                                            acc = 1u;
+                                        }
+                                    }
+                                }
                                 tc_commit(&S.o_done[w]);
                             }
                             __syncwarp();
+                            o_started[w] = o_started[w] || l8 != 0u;
                             ++n_p[w];
                         }
                     }
@@ -887,13 +938,11 @@ int launch_tc_fwd(const Prob& P, const void* Q, const void* K, const void* V, co
     const size_t smem = sizeof(SharedStorage) + 1024;
     dim3 grid(P.B * P.Hq, npairs);
     timing_mark(0, false, st);
-    if (compact) {
-        if (cudaFuncSetAttribute(fwd_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return DMA_ERR_CUDA;
-        fwd_kernel<true><<<grid, kThreads, smem, st>>>(tmQ, tmK, tmV, fp);
-    } else {
-        if (cudaFuncSetAttribute(fwd_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return DMA_ERR_CUDA;
-        fwd_kernel<false><<<grid, kThreads, smem, st>>>(tmQ, tmK, tmV, fp);
-    }
+    const bool block_skip = (P.flags & DMA_FLAG_BLOCK_SKIP) != 0;
+    auto kern = compact ? (block_skip ? fwd_kernel<true, true> : fwd_kernel<true, false>)
+                        : (block_skip ? fwd_kernel<false, true> : fwd_kernel<false, false>);
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return DMA_ERR_CUDA;
+    kern<<<grid, kThreads, smem, st>>>(tmQ, tmK, tmV, fp);
     timing_mark(0, true, st);
     count_launch();
     return check_launch();

@@ -202,6 +202,43 @@ def test_default_flags_choose_the_path_from_the_descriptor():
     assert dma.dma_read_status(ws) == -8
 
 
+def test_mma_block_skipping_does_not_change_the_result():
+    """With DMA_FLAG_BLOCK_SKIP the P V product of an executed tile leaves out the 16-key MMA blocks in which no key can be
+    kept by the query tile's rows. P is exactly zero there, so O and lse must be the bits of the run with every block
+    multiplied, on masks that really have such blocks: a banded importance
+    pattern, packed documents whose boundaries fall inside key tiles, and the gathered lists of the token-compacted kernels.
+    The same outputs are held to the oracle in the tests above."""
+    dev = torch.device("cuda:0")
+    banded = wl.small(wl.CONFIGS["S"], L=4096, w=200, Hq=6, Hkv=2, backward=False, name="block-skip banded")
+    packed = wl.small(C2, B=1, Hq=4, Hkv=2, L=3000, w=300, backward=False, name="block-skip packed")
+    for case, cu in ((banded, None), (packed, [0, 70, 1000, 1111, 1900, 2500, 3000])):
+        inp = wl.make_inputs(case)
+        Q, K, V = (inp[k].to(dev) for k in ("Q", "K", "V"))
+        p0 = problem_of(case, flags=dma.DMA_FLAG_TILE_PATH)
+        if cu is None:
+            mask = dma.dma_mask_build(p0, V, inp["W_delta"].to(dev), inp["A"].to(dev))
+        else:
+            mask = dma.dma_mask_build_varlen(p0, V, inp["W_delta"].to(dev), inp["A"].to(dev), torch.tensor(cu, dtype=torch.int32, device=dev))
+        # the mask must contain dead 16-key blocks inside active tiles, or the test checks nothing
+        e = mask[1].cpu().numpy()
+        bmp = mask[2].cpu().numpy().view(np.uint32)
+        dead_blocks = 0
+        for qt in range(case.L // 128):
+            for kt in range(qt):                                                   # off-diagonal tiles: a key is dead iff it expired before the tile's rows
+                if (bmp[0, 0, qt, kt // 32] >> np.uint32(kt % 32)) & np.uint32(1):
+                    blk = (e[0, 0, kt * 128:(kt + 1) * 128].reshape(8, 16) <= qt * 128).all(1)
+                    dead_blocks += int(blk.sum())
+        assert dead_blocks > 0, case.name
+        for path in (dma.DMA_FLAG_TILE_PATH, dma.DMA_FLAG_COMPACT_KV):
+            outs = []
+            for extra in (dma.DMA_FLAG_BLOCK_SKIP, 0):
+                p = problem_of(case, flags=path | extra)
+                ws = torch.empty(dma.dma_query_workspace(p)[1], dtype=torch.uint8, device=dev)
+                outs.append(dma.dma_attn_fwd(p, Q, K, V, *mask, ws=ws))
+                assert dma.dma_read_status(ws) == 0
+            assert torch.equal(outs[0][0], outs[1][0]) and torch.equal(outs[0][1], outs[1][1]), (case.name, path)
+
+
 def test_largest_supported_lengths():
     """The longest sequences the tensor-core kernels take: forward at L = 131072 (1024 key tiles, the schedule's capacity),
     tile path and token-compacted; forward + backward at L = 65536 with a group of 4 query heads per KV head (the backward's
