@@ -83,6 +83,11 @@ enum {
                                     query tile's rows; P is exactly zero there, so O and lse are the same bits. Off by
                                     default: on the benchmark masks well under 5 % of the blocks of executed tiles are dead,
                                     and the bookkeeping costs the kernel more than the multiplications it saves */
+    DMA_FLAG_DETERMINISTIC = 64, /* dma_attn_bwd with token-compacted execution: the query heads of a group write their dK / dV
+                                    contributions to accumulators of their own (Hq/Hkv times the accumulator space: the
+                                    larger workspace dma_query_workspace reports) and a last pass adds them in head order,
+                                    so dK and dV are the same bits from run to run, as on the tile path. dQ stays a sum of
+                                    floating-point atomics on every path */
     DMA_FLAG_FULL_DELTA = 8      /* the sampling weights as Eq. (delta_calc) states them: W_delta (and dW_delta) is
                                     [Hq, Hkv*d], one row per query head over ALL channels of the value row (the linear
                                     layer of the App. A listing), z[b,h,j] = sum_{h'} V[b,j,h',:] . W_delta[h, h'*d:(h'+1)*d].
@@ -191,7 +196,8 @@ int dma_attn_fwd_chunk(const dma_problem_t* p, int32_t q_begin, int32_t q_len, c
  * dK and dV are summed over the Hq/Hkv query heads that share a KV head; dM is per query head.
  * dQ is accumulated with floating-point atomics: its rounding depends on execution order. dK, dV (and O, lse of the
  * forward) are reproducible bit for bit from run to run on the tile path and the CUDA-core path; with
- * DMA_FLAG_COMPACT_KV dK and dV are accumulated with atomics too (one CTA per query head) and vary in the last bits. */
+ * token-compacted execution dK and dV are accumulated with atomics too (one CTA per query head) and vary in the last
+ * bits unless DMA_FLAG_DETERMINISTIC is set. */
 int dma_attn_bwd(const dma_problem_t* p, const void* Q, const void* K, const void* V,
                  const void* O, const void* dO, const float* lse,
                  const float* bias, const int32_t* expiry, const uint32_t* bitmap,

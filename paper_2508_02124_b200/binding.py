@@ -15,7 +15,7 @@ _lib = None
 
 DMA_BF16, DMA_FP32 = 0, 1
 DMA_FLAG_IGNORE_BITMAP, DMA_FLAG_SIMT, DMA_FLAG_COMPACT_KV, DMA_FLAG_FULL_DELTA, DMA_FLAG_TILE_PATH = 1, 2, 4, 8, 16
-DMA_FLAG_BLOCK_SKIP = 32
+DMA_FLAG_BLOCK_SKIP, DMA_FLAG_DETERMINISTIC = 32, 64
 
 ENTRY_POINTS = ("dma_query_workspace", "dma_bitmap_words", "dma_mask_build", "dma_attn_fwd", "dma_attn_bwd",
                 "dma_read_status", "dma_launch_count", "dma_strerror", "dma_step_host_arena", "dma_step_host", "dma_mask_build_static", "dma_selftest_wait_timeout",

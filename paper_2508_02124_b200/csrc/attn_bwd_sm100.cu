@@ -79,6 +79,8 @@ struct BwdParams {
     const __nv_bfloat16* Vg;
     float* dKacc;               // fp32 [B, L, Hkv, 128] accumulators (several query heads add into one KV head's rows)
     float* dVacc;
+    int64_t acc_slot;           // 0: the group's heads add into one accumulator with atomics; else: elements between the
+                                // per-head slots [G][B, L, Hkv, 128], written with plain stores and summed in head order afterwards
     int64_t ks_b, ks_l, ks_h, vs_b, vs_l, vs_h;
 };
 
@@ -315,7 +317,8 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             tc_fence_after();
             __nv_bfloat16* dk = P.dK + b * P.ks_b + (int64_t)j * P.ks_l + hk * P.ks_h;
             __nv_bfloat16* dv = P.dV + b * P.vs_b + (int64_t)j * P.vs_l + hk * P.vs_h;
-            const size_t arow = ((size_t)(b * P.L + min(j, P.L - 1)) * P.Hkv + hk) * 128;      // accumulator row (compact mode)
+            const size_t arow = ((size_t)(b * P.L + min(j, P.L - 1)) * P.Hkv + hk) * 128 +      // accumulator row (compact mode)
+                                (kCompact ? (size_t)(hq_c % P.G) * (size_t)P.acc_slot : 0);
 #pragma unroll
             for (int which = 0; which < 2; ++which) {
                 const float mul = which == 0 ? P.scale : 1.0f;
@@ -335,10 +338,17 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                     if constexpr (kCompact) {
                         // unscaled sums into the fp32 accumulators: the group's query heads add into the same rows
                         if (j < P.L && n_steps > 0) {
+                            if (P.acc_slot) {          // this (key, query head) pair is written by this thread alone
 #pragma unroll
-                            for (int u = 0; u < 32; u += 4)
-                                red_add_v4(acc + c * 32 + u, __uint_as_float(o[u]), __uint_as_float(o[u + 1]), __uint_as_float(o[u + 2]),
-                                           __uint_as_float(o[u + 3]));
+                                for (int u = 0; u < 32; u += 4)
+                                    *reinterpret_cast<float4*>(acc + c * 32 + u) = make_float4(__uint_as_float(o[u]), __uint_as_float(o[u + 1]),
+                                                                                              __uint_as_float(o[u + 2]), __uint_as_float(o[u + 3]));
+                            } else {
+#pragma unroll
+                                for (int u = 0; u < 32; u += 4)
+                                    red_add_v4(acc + c * 32 + u, __uint_as_float(o[u]), __uint_as_float(o[u + 1]), __uint_as_float(o[u + 2]),
+                                               __uint_as_float(o[u + 3]));
+                            }
                         }
                     } else if (j < P.L) {
 #pragma unroll
@@ -575,14 +585,20 @@ __global__ void rowdot_bf16_kernel(const __nv_bfloat16* __restrict__ O, const __
     if (sub == 0 && row < (long)B * Hq * L) Dv[row] = s;
 }
 
-// fp32 accumulator [B, L, Hq, 128] (unscaled dS K sums) -> softmax scale applied -> bf16 dQ in the caller's layout; 8 elements per thread
+// fp32 accumulator [B, L, Hq, 128] (unscaled dS K sums) -> softmax scale applied -> bf16 dQ in the caller's layout; 8 elements per thread.
+// nslots > 1: the accumulator is nslots copies, slot_stride elements apart, added here in slot order (a fixed order: the
+// result is then the same bits from run to run).
 __global__ void dq_convert_bf16_kernel(const float* __restrict__ acc, __nv_bfloat16* __restrict__ dQ, size_t n8, int L, int Hq,
-                                       int64_t qs_b, int64_t qs_l, int64_t qs_h, float scale) {
+                                       int64_t qs_b, int64_t qs_l, int64_t qs_h, float scale, int nslots = 1, int64_t slot_stride = 0) {
     const size_t t = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (t >= n8) return;
     const size_t e = t * 8;
     const int c = e % 128, h = (e / 128) % Hq, i = (e / ((size_t)128 * Hq)) % L, b = e / ((size_t)128 * Hq * L);
-    const float4 a = *reinterpret_cast<const float4*>(acc + e), bb = *reinterpret_cast<const float4*>(acc + e + 4);
+    float4 a = *reinterpret_cast<const float4*>(acc + e), bb = *reinterpret_cast<const float4*>(acc + e + 4);
+    for (int sl = 1; sl < nslots; ++sl) {
+        const float4 a2 = *reinterpret_cast<const float4*>(acc + (size_t)sl * slot_stride + e), b2 = *reinterpret_cast<const float4*>(acc + (size_t)sl * slot_stride + e + 4);
+        a.x += a2.x; a.y += a2.y; a.z += a2.z; a.w += a2.w; bb.x += b2.x; bb.y += b2.y; bb.z += b2.z; bb.w += b2.w;
+    }
     uint4 o;
     o.x = ptx::pack_bf16(a.x * scale, a.y * scale); o.y = ptx::pack_bf16(a.z * scale, a.w * scale);
     o.z = ptx::pack_bf16(bb.x * scale, bb.y * scale); o.w = ptx::pack_bf16(bb.z * scale, bb.w * scale);
@@ -639,7 +655,8 @@ static size_t bwd_perm_ints(const Prob& P) { return (((size_t)P.B * P.Hq * P.Tc 
 size_t tc_bwd_ws_bytes(const Prob& P) {
     const size_t rows = (size_t)P.B * P.Hq * P.L;
     size_t n = kWsHeaderBytes + (bwd_rows64(P) + rows * P.d) * sizeof(float);
-    if (P.flags & DMA_FLAG_COMPACT_KV) n += bwd_perm_ints(P) * sizeof(int) + 2 * (size_t)P.B * P.L * P.Hkv * P.d * sizeof(float);
+    const size_t slots = (P.flags & DMA_FLAG_DETERMINISTIC) ? (size_t)P.G : 1;      // per-head dK / dV accumulators
+    if (P.flags & DMA_FLAG_COMPACT_KV) n += bwd_perm_ints(P) * sizeof(int) + 2 * slots * (size_t)P.B * P.L * P.Hkv * P.d * sizeof(float);
     return n;
 }
 
@@ -653,8 +670,9 @@ int launch_tc_bwd(const Prob& P, const void* Q, const void* K, const void* V, co
     float* Dv = reinterpret_cast<float*>((char*)ws + kWsHeaderBytes);
     float* acc = Dv + bwd_rows64(P);
     int* perm = reinterpret_cast<int*>(acc + nq);
+    const size_t slots = (compact && (P.flags & DMA_FLAG_DETERMINISTIC)) ? (size_t)P.G : 1;
     float* accK = reinterpret_cast<float*>(perm + bwd_perm_ints(P));
-    float* accV = accK + nkv;
+    float* accV = accK + slots * nkv;
     CUtensorMap tmQ, tmK, tmV, tmG;
     int rc;
     if ((rc = make_tmap_bf16(&tmQ, Q, P.B, P.L, P.Hq, P.d, P.qs, 64))) return rc;
@@ -668,7 +686,7 @@ int launch_tc_bwd(const Prob& P, const void* Q, const void* K, const void* V, co
     if (cudaMemsetAsync(acc, 0, nq * sizeof(float), st) != cudaSuccess) return DMA_ERR_CUDA;
     if (cudaMemsetAsync(dM, 0, rows * sizeof(float), st) != cudaSuccess) return DMA_ERR_CUDA;   // two partial sums are added per key
     if (compact) {
-        if (cudaMemsetAsync(accK, 0, 2 * nkv * sizeof(float), st) != cudaSuccess) return DMA_ERR_CUDA;
+        if (cudaMemsetAsync(accK, 0, 2 * slots * nkv * sizeof(float), st) != cudaSuccess) return DMA_ERR_CUDA;
         lifetime_perm_kernel<<<P.B * P.Hq, 1024, 0, st>>>(expiry, perm, P.L, P.Tc, P.causal);
         count_launch();
     }
@@ -696,7 +714,7 @@ int launch_tc_bwd(const Prob& P, const void* Q, const void* K, const void* V, co
     bp.scale = P.scale; bp.scale_log2 = P.scale * 1.4426950408889634f; bp.inv_scale = 1.0f / P.scale;
     bp.ks_b = P.ks[0]; bp.ks_l = P.ks[1]; bp.ks_h = P.ks[2]; bp.vs_b = P.vs[0]; bp.vs_l = P.vs[1]; bp.vs_h = P.vs[2];
     bp.perm = perm; bp.expiry_all = expiry; bp.causal = P.causal; bp.Kg = (const __nv_bfloat16*)K; bp.Vg = (const __nv_bfloat16*)V;
-    bp.dKacc = accK; bp.dVacc = accV;
+    bp.dKacc = accK; bp.dVacc = accV; bp.acc_slot = slots > 1 ? (int64_t)nkv : 0;
     const size_t smem = sizeof(SharedStorage) + 1024;
     timing_mark(1, false, st);
     if (compact) {
@@ -704,8 +722,8 @@ int launch_tc_bwd(const Prob& P, const void* Q, const void* K, const void* V, co
         bwd_kernel<true><<<dim3(P.B * P.Hq, P.Tc), kThreads, smem, st>>>(tmQ, tmK, tmV, tmG, tmDQ, bp);
         timing_mark(1, true, st);
         const int nb = (int)((nkv / 8 + 255) / 256);
-        dq_convert_bf16_kernel<<<nb, 256, 0, st>>>(accK, (__nv_bfloat16*)dK, nkv / 8, P.L, P.Hkv, P.ks[0], P.ks[1], P.ks[2], P.scale);
-        dq_convert_bf16_kernel<<<nb, 256, 0, st>>>(accV, (__nv_bfloat16*)dV, nkv / 8, P.L, P.Hkv, P.vs[0], P.vs[1], P.vs[2], 1.0f);
+        dq_convert_bf16_kernel<<<nb, 256, 0, st>>>(accK, (__nv_bfloat16*)dK, nkv / 8, P.L, P.Hkv, P.ks[0], P.ks[1], P.ks[2], P.scale, (int)slots, (int64_t)nkv);
+        dq_convert_bf16_kernel<<<nb, 256, 0, st>>>(accV, (__nv_bfloat16*)dV, nkv / 8, P.L, P.Hkv, P.vs[0], P.vs[1], P.vs[2], 1.0f, (int)slots, (int64_t)nkv);
         count_launch(2);
     } else {
         if (cudaFuncSetAttribute(bwd_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return DMA_ERR_CUDA;

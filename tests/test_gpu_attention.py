@@ -432,6 +432,24 @@ def test_compact_backward_small_cases(case):
     compare(case, got, ref)
 
 
+def test_compact_backward_deterministic_option():
+    """DMA_FLAG_DETERMINISTIC: the query heads of a group write dK / dV contributions to accumulators of their own, added in
+    head order: the same bits from run to run (four heads per KV head here), and the same parity with the oracle."""
+    case = wl.small(C2, B=2, Hq=8, Hkv=2, L=1100, w=150, backward=True, name="compact deterministic")
+    inp = wl.make_inputs(case)
+    dl, e, _ = oracle_mask(case, inp)
+    ref = oracle_all(case, inp, dl, e)
+    st = stored_forward(case, ref["O"], ref["lse"])
+    flags = dma.DMA_FLAG_COMPACT_KV | dma.DMA_FLAG_DETERMINISTIC
+    runs = [gpu_run(case, inp, stored=st, flags=flags) for _ in range(3)]
+    compare(case, runs[0], ref)
+    for r in runs[1:]:
+        assert torch.equal(r["dK"], runs[0]["dK"]) and torch.equal(r["dV"], runs[0]["dV"])
+    plain = gpu_run(case, inp, stored=st, flags=dma.DMA_FLAG_COMPACT_KV)
+    assert_close(plain["dK"], f64(runs[0]["dK"]), case.dtype, "dK (atomic against ordered sums)")
+    assert dma.dma_query_workspace(problem_of(case, flags=flags))[2] > dma.dma_query_workspace(problem_of(case, flags=dma.DMA_FLAG_COMPACT_KV))[2]
+
+
 @pytest.mark.parametrize("key", ["3", "4w256", "4w2048", "S"])
 def test_compact_backward_full_size_sampled(key):
     case = wl.CONFIGS[key]
