@@ -28,7 +28,7 @@ namespace {
 using namespace ptx;
 
 constexpr int kStages = 3;
-constexpr int kMaxSteps = 4096;
+constexpr int kMaxSteps = 8192;              // 64-row steps of one CTA: G * ceil(L / 128) * 2 (L = 131072 with four query heads per KV head)
 constexpr int kThreads = 512;
 constexpr uint32_t kKVBytes = 128 * 128 * 2;   // K or V tile: two 16 KB halves (channels 0-63 | 64-127)
 constexpr uint32_t kQBytes = 64 * 128 * 2;     // Q or dO step tile (64 rows): two 8 KB halves

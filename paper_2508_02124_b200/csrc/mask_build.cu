@@ -9,6 +9,7 @@
 //                       chunk by chunk with a binary search in each sorted chunk
 //   bitmap_kernel       per key tile: union of the query-tile intervals its keys are kept in
 #include <mutex>
+#include <type_traits>
 
 #include "common.cuh"
 
@@ -72,59 +73,135 @@ __device__ __forceinline__ void load8(const __nv_bfloat16* p, float (&v)[8]) {
     }
 }
 
-// One CTA: kRows consecutive keys of one (batch, KV head); writes delta for the G query heads of the group.
-// A group of D/8 lanes owns a row: each lane forms the fma chain over its 8 channels, an xor butterfly adds
-// adjacent partials pairwise (IEEE addition commutes, so every lane of the group holds the same sum).
+// eight consecutive channels of one value row, as loaded (converted to fp32 only when the chain runs)
+struct Raw8f { float4 a, b; };
+__device__ __forceinline__ Raw8f load_raw8(const float* p) { return {*reinterpret_cast<const float4*>(p), *reinterpret_cast<const float4*>(p + 4)}; }
+__device__ __forceinline__ uint4 load_raw8(const __nv_bfloat16* p) { return *reinterpret_cast<const uint4*>(p); }
+__device__ __forceinline__ void widen8(const Raw8f& r, float (&v)[8]) {
+    v[0] = r.a.x; v[1] = r.a.y; v[2] = r.a.z; v[3] = r.a.w; v[4] = r.b.x; v[5] = r.b.y; v[6] = r.b.z; v[7] = r.b.w;
+}
+__device__ __forceinline__ void widen8(const uint4& a, float (&v)[8]) {
+    const uint32_t u[4] = {a.x, a.y, a.z, a.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        v[2 * i] = __uint_as_float(u[i] << 16);
+        v[2 * i + 1] = __uint_as_float(u[i] & 0xffff0000u);
+    }
+}
+template <typename T> struct RawOf { using type = uint4; };
+template <> struct RawOf<float> { using type = Raw8f; };
+
+// Sum over the LPR lanes of a row group of NB per-lane partials (one per head of a block of NB heads), in the order of the
+// xor butterfly (adjacent lanes first: a balanced pairwise tree over the row's 8-channel chunks). The first log2(NB) levels
+// are "transposing": a lane keeps half of its values and hands the other half to its partner, so the block costs
+// log2(NB) + ... shuffles in all instead of NB log2(LPR) (the additions are the same, and IEEE addition commutes, so the
+// bits are those of the plain butterfly). On return p[0] of lane `sub` is the complete sum of head bitrev(sub mod NB) of
+// the block (the same value in every lane of the group with those low bits).
+template <int NB, int LPR>
+__device__ __forceinline__ void block_reduce(float (&p)[NB], int sub) {
+    int keep = NB >> 1;
+#pragma unroll
+    for (int m = 1; m < LPR; m <<= 1) {
+        if (keep >= 1) {
+            const bool up = (sub & m) != 0;
+#pragma unroll
+            for (int q = 0; q < NB / 2; ++q) {
+                if (q < keep) {
+                    const float stay = up ? p[q + keep] : p[q];
+                    const float give = up ? p[q] : p[q + keep];
+                    p[q] = __fadd_rn(stay, __shfl_xor_sync(0xffffffffu, give, m));
+                }
+            }
+            keep >>= 1;
+        } else {
+            p[0] = __fadd_rn(p[0], __shfl_xor_sync(0xffffffffu, p[0], m));
+        }
+    }
+}
+
+// One CTA: tiles of kRows consecutive keys of one (batch, KV head), taken in turn with the other CTAs of that pair (grid-
+// stride); writes delta for the G query heads of the group. A group of D/8 lanes owns a row: each lane forms the fma chain
+// over its 8 channels, an xor butterfly adds adjacent partials pairwise (IEEE addition commutes, so every lane of the group
+// holds the same sum). The kernel streams V once and is bound by that stream, so it is built around memory-level
+// parallelism: a warp requests ALL value rows of its NEXT tile (kPass 16-byte loads per lane) before it runs the chains of
+// the current one, W is staged once per CTA, and softplus / exp of tile t (one (row, head) pair per thread, from the z
+// values in shared memory) overlap the chains of tile t + 1 (two z buffers, one barrier per tile).
 template <typename T, int D>
-__global__ void __launch_bounds__(256) delta_kernel(const T* __restrict__ V, const float* __restrict__ W,
+__global__ void __launch_bounds__(256, sizeof(T) == 2 ? 2 : 1) delta_kernel(const T* __restrict__ V, const float* __restrict__ W,
                                                     const float* __restrict__ A, float* __restrict__ delta,
                                                     int L, int Hq, int G, int64_t vs_b, int64_t vs_l, int64_t vs_h,
                                                     int j_off, int64_t ld) {
     constexpr int LPR = D / 8;            // lanes per row
     constexpr int RPW = 32 / LPR;         // rows per warp and pass
     constexpr int kRows = 128;
+    constexpr int kPass = kRows / (8 * RPW);
+    using Raw = typename RawOf<T>::type;
     extern __shared__ float smem[];
     float* sW = smem;                     // [G][D]
-    float* sOut = smem + G * D;           // [G][kRows]
-    const int hk = blockIdx.y, b = blockIdx.z, j0 = j_off + blockIdx.x * kRows;   // keys [j_off, L) of a row of ld entries
+    float* sOut = smem + G * D;           // [2][G][kRows]
+    const int hk = blockIdx.y, b = blockIdx.z;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int sub = lane % LPR, grp = lane / LPR;
-    for (int i = tid; i < G * D; i += 256) sW[i] = W[(size_t)hk * G * D + i];
-    __syncthreads();
-    const int rows = min(kRows, L - j0);                   // a short range (one appended key) does not walk 128 row slots
-    // A warp owns kPass = kRows / (8 RPW) row groups. All their value rows are requested before the first is used (the
-    // kernel is bound by the V stream: one 16-byte load in flight per lane would leave the memory system idle), then
-    // the chains run out of registers.
-    constexpr int kPass = kRows / (8 * RPW);
-    float v[kPass][8];
-#pragma unroll
-    for (int t = 0; t < kPass; ++t) {
-        const int r = warp * RPW + grp + t * 8 * RPW, j = j0 + r;
-        if (r < rows && j < L) {
-            load8(V + b * vs_b + (int64_t)j * vs_l + hk * vs_h + sub * 8, v[t]);
-        } else {
-#pragma unroll
-            for (int c = 0; c < 8; ++c) v[t][c] = 0.0f;
-        }
-    }
-    for (int g = 0; g < G; ++g) {
-        const float4 wa = *reinterpret_cast<const float4*>(sW + g * D + sub * 8), wb = *reinterpret_cast<const float4*>(sW + g * D + sub * 8 + 4);
-        const float w[8] = {wa.x, wa.y, wa.z, wa.w, wb.x, wb.y, wb.z, wb.w};
+    const int ntiles = (L - j_off + kRows - 1) / kRows;        // keys [j_off, L) of a row of ld entries
+    const T* Vb = V + b * vs_b + hk * vs_h + sub * 8;
+    auto request = [&](int tile, Raw (&raw)[kPass]) {
+        const int j0 = j_off + tile * kRows;
 #pragma unroll
         for (int t = 0; t < kPass; ++t) {
-            float p = 0.0f;
-#pragma unroll
-            for (int c = 0; c < 8; ++c) p = __fmaf_rn(v[t][c], w[c], p);
-#pragma unroll
-            for (int m = 1; m < LPR; m <<= 1) p = __fadd_rn(p, __shfl_xor_sync(0xffffffffu, p, m));
-            const int r = warp * RPW + grp + t * 8 * RPW;
-            if (sub == g % LPR && r < rows) sOut[g * kRows + r] = p;      // z; softplus and exp follow, one (row, head) pair per thread
+            const int j = j0 + warp * RPW + grp + t * 8 * RPW;
+            if (tile < ntiles && j < L) raw[t] = load_raw8(Vb + (int64_t)j * vs_l);
+            else raw[t] = Raw{};
         }
-    }
+    };
+    Raw cur[kPass], nxt[kPass];
+    request(blockIdx.x, cur);
+    for (int i = tid; i < G * D; i += 256) sW[i] = W[(size_t)hk * G * D + i];
     __syncthreads();
-    for (int i = tid; i < G * kRows; i += 256) {
-        const int g = i / kRows, r = i % kRows;
-        if (j0 + r < L) delta[((size_t)b * Hq + hk * G + g) * ld + j0 + r] = delta_fixed(sOut[i], A[hk * G + g]);
+    int buf = 0;
+    for (int tile = blockIdx.x; tile < ntiles; tile += gridDim.x, buf ^= 1) {
+        request(tile + gridDim.x, nxt);
+        const int j0 = j_off + tile * kRows, rows = min(kRows, L - j0);
+        float* z = sOut + buf * G * kRows;
+        // heads in blocks of 4 (then 2, then 1): the chains of a block, then one transposing reduction per pass
+        auto block = [&](int g0, auto nb_tag) {
+            constexpr int NB = decltype(nb_tag)::value;
+            float w[NB][8];
+#pragma unroll
+            for (int q = 0; q < NB; ++q) {
+                const float4 wa = *reinterpret_cast<const float4*>(sW + (g0 + q) * D + sub * 8), wb = *reinterpret_cast<const float4*>(sW + (g0 + q) * D + sub * 8 + 4);
+                w[q][0] = wa.x; w[q][1] = wa.y; w[q][2] = wa.z; w[q][3] = wa.w; w[q][4] = wb.x; w[q][5] = wb.y; w[q][6] = wb.z; w[q][7] = wb.w;
+            }
+            int mine = 0;                 // head of the block this lane ends up with: the low bits of sub, reversed
+#pragma unroll
+            for (int m = 1, t = NB >> 1; m < NB; m <<= 1, t >>= 1) mine |= (sub & m) ? t : 0;
+#pragma unroll
+            for (int t = 0; t < kPass; ++t) {
+                if (warp * RPW + t * 8 * RPW >= rows) continue;      // (warp-uniform) a short range, e.g. the one appended key of a decoding step
+                float v[8], p[NB];
+                widen8(cur[t], v);
+#pragma unroll
+                for (int q = 0; q < NB; ++q) {
+                    float a = 0.0f;
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) a = __fmaf_rn(v[c], w[q][c], a);
+                    p[q] = a;
+                }
+                block_reduce<NB, LPR>(p, sub);
+                const int r = warp * RPW + grp + t * 8 * RPW;
+                if (sub < NB && r < rows) z[(g0 + mine) * kRows + r] = p[0];
+            }
+        };
+        int g0 = 0;
+        for (; g0 + 4 <= G; g0 += 4) block(g0, std::integral_constant<int, 4>{});
+        if (g0 + 2 <= G) { block(g0, std::integral_constant<int, 2>{}); g0 += 2; }
+        if (g0 < G) block(g0, std::integral_constant<int, 1>{});
+        __syncthreads();                  // z of this tile is complete (and the other buffer's readers of two tiles ago are long done)
+        for (int i = tid; i < G * kRows; i += 256) {
+            const int g = i / kRows, r = i % kRows;
+            if (r < rows) delta[((size_t)b * Hq + hk * G + g) * ld + j0 + r] = delta_fixed(z[i], A[hk * G + g]);
+        }
+#pragma unroll
+        for (int t = 0; t < kPass; ++t) cur[t] = nxt[t];
     }
 }
 
@@ -494,8 +571,13 @@ static int launch_delta(const Prob& P, const void* V, const float* W, const floa
         count_launch();
         return check_launch();
     }
-    dim3 grid((j_end - j_begin + 127) / 128, P.Hkv, P.B);
-    size_t smem = (size_t)P.G * (D + 128) * sizeof(float);
+    // two CTAs per SM in all (what the register file holds at once), each walking its (batch, KV head) pair's tiles grid-stride; short ranges (one appended key
+    // of a decoding step) get one CTA per tile
+    const int ntiles = (j_end - j_begin + 127) / 128;
+    int per_pair = (2 * 148 + P.Hkv * P.B - 1) / (P.Hkv * P.B);
+    per_pair = per_pair < 1 ? 1 : per_pair > ntiles ? ntiles : per_pair;
+    dim3 grid(per_pair, P.Hkv, P.B);
+    size_t smem = (size_t)P.G * (D + 2 * 128) * sizeof(float);
     if (smem > 48 * 1024) return DMA_ERR_UNSUPPORTED;
     delta_kernel<T, D><<<grid, 256, smem, st>>>((const T*)V, W, A, bias, j_end, P.Hq, P.G, P.vs[0], P.vs[1], P.vs[2], j_begin, ld);
     count_launch();
@@ -517,7 +599,7 @@ static int mask_build_limits(const Prob& P) {
     if (P.flags & DMA_FLAG_FULL_DELTA) {
         const size_t lanes = (size_t)P.d / 8, HqP = (P.Hq + lanes - 1) / lanes * lanes;
         if ((HqP * P.Hkv * P.d + HqP * kFullRows) * sizeof(float) > 200 * 1024) return DMA_ERR_UNSUPPORTED;
-    } else if ((size_t)P.G * (P.d + 128) * sizeof(float) > 48 * 1024) {
+    } else if ((size_t)P.G * (P.d + 2 * 128) * sizeof(float) > 48 * 1024) {
         return DMA_ERR_UNSUPPORTED;
     }
     if ((size_t)(P.Tr + 1) * sizeof(int) > 48 * 1024) return DMA_ERR_UNSUPPORTED;

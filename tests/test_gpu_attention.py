@@ -240,23 +240,24 @@ def test_mma_block_skipping_does_not_change_the_result():
 
 
 def test_largest_supported_lengths():
-    """The longest sequences the tensor-core kernels take: forward at L = 131072 (1024 key tiles, the schedule's capacity),
-    tile path and token-compacted; forward + backward at L = 65536 with a group of 4 query heads per KV head (the backward's
-    step-list capacity). Sampled rows and keys against the oracle."""
-    fwd = wl.small(wl.CONFIGS["5"], B=1, Hq=4, Hkv=2, L=131072, w=4096, backward=False, name="max L forward")
-    inp = wl.make_inputs(fwd)
-    ref = Samples(fwd, inp, nrows=10, forward_only=True)
-    got = gpu_run(fwd, inp, backward=False, flags=dma.DMA_FLAG_TILE_PATH)
+    """The longest sequences the tensor-core kernels take: L = 131072 (1024 key tiles, the forward schedule's capacity; with
+    a group of 4 query heads per KV head also the capacity of the backward's step list), forward and backward, tile path and
+    token-compacted. Sampled rows and keys against the oracle, dQ on rows where the mask drops keys."""
+    case = wl.small(wl.CONFIGS["3"], B=1, Hq=4, Hkv=1, L=131072, w=2048, backward=True, name="max L")
+    inp = wl.make_inputs(case)
+    ref = Samples(case, inp, nrows=8, nkeys=4)
+    got = gpu_run(case, inp, stored=ref.stored, flags=dma.DMA_FLAG_TILE_PATH)
     ref.check(got)
-    ref.check(gpu_run(fwd, inp, backward=False, flags=dma.DMA_FLAG_COMPACT_KV), "compact ")
+    ref.check(gpu_run(case, inp, stored=ref.stored, flags=dma.DMA_FLAG_COMPACT_KV), "compact ")
     with pytest.raises(dma.DmaError) as e:                        # one tile more is refused, not mis-executed
-        too_long = wl.small(fwd, L=131072 + 128)
+        too_long = wl.small(case, L=131072 + 128)
         dma.dma_attn_fwd(problem_of(too_long, flags=dma.DMA_FLAG_TILE_PATH), got["O"], got["O"], got["O"], got["bias"], got["expiry"], got["bitmap"])
     assert e.value.status == -4
-    both = wl.small(wl.CONFIGS["3"], B=1, Hq=4, Hkv=1, L=65536, w=2048, backward=True, name="max L backward")
-    inp = wl.make_inputs(both)
-    ref = Samples(both, inp, nrows=8, nkeys=4)
-    ref.check(gpu_run(both, inp, stored=ref.stored, flags=dma.DMA_FLAG_TILE_PATH))
+    with pytest.raises(dma.DmaError) as e:                        # eight heads per KV head at this length: the tile path's step list is too short
+        wide = problem_of(wl.small(case, Hq=8), flags=dma.DMA_FLAG_TILE_PATH)
+        ws = torch.empty(dma.dma_query_workspace(wide)[2], dtype=torch.uint8, device="cuda:0")
+        dma.dma_attn_bwd(wide, got["O"], got["O"], got["O"], got["O"], got["O"], got["lse"], got["bias"], got["expiry"], got["bitmap"], ws=ws)
+    assert e.value.status == -4
 
 
 def test_whole_step_can_be_captured_in_a_cuda_graph():
