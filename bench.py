@@ -395,10 +395,24 @@ def main():
             g1.record()
             barrier()
             v_ms.append(g0.elapsed_time(g1) / 10)
+        # MMA-block skipping inside executed tiles (DMA_FLAG_BLOCK_SKIP): the same forward with the dead 16-key blocks of P V left out
+        pbs = dma.problem(case.B, case.Hq, case.Hkv, case.L, case.d, case.w, dtype=case.torch_dtype, flags=p.flags | dma.DMA_FLAG_BLOCK_SKIP)
+        bs_ms = None
+        if case.dtype == "bf16" and case.d == 128 and not (args.flags & dma.DMA_FLAG_SIMT):
+            for _ in range(3):
+                dma.dma_attn_fwd(pbs, Q, K, V, bias_v, exp_v, bmp_v, Ov, lsev, ws_f)
+            g0, g1 = ev(), ev()
+            barrier()
+            g0.record()
+            for _ in range(10):
+                dma.dma_attn_fwd(pbs, Q, K, V, bias_v, exp_v, bmp_v, Ov, lsev, ws_f)
+            g1.record()
+            barrier()
+            bs_ms = g0.elapsed_time(g1) / 10
         act_v = int(sum(bin(int(x) & 0xFFFFFFFF).count("1") for x in bmp_v.cpu().numpy().ravel()))
         v_step = sum(v_ms)
         varlen = {"documents": 12, "lengths": [b - a for a, b in zip(cu, cu[1:])], "mask_ms": v_ms[0], "fwd_ms": v_ms[1],
-                  "bwd_ms": v_ms[2] if case.backward else None, "step_ms": v_step, "active_tiles": act_v,
+                  "bwd_ms": v_ms[2] if case.backward else None, "step_ms": v_step, "active_tiles": act_v, "fwd_ms_block_skip": bs_ms,
                   "tflops_executed_tiles": tile_flops(act_v, case.d, case.backward) / (v_step * 1e-3) / 1e12}
 
     # ---- non-causal mode (causal = 0: every row of a head keeps the same min(w, L) keys; bf16 d = 128 runs token-compacted):

@@ -490,7 +490,7 @@ __global__ void __launch_bounds__(kAttnThreads) decode_attn_kernel(const T* __re
 // One key is appended per step, so the set of the w best keys changes by at most one member: the new key enters iff it
 // beats the weakest kept key (or the set is not full yet), and that weakest key leaves. The state of a (batch, head) row:
 //   int32 [0] count (<= w)   [1] position of the weakest kept key in the list   [2..3] its 64-bit sort key
-//         [4] ticket counter of the step kernel's CTAs (zero between calls)   [5..7] unused
+//         [4..7] unused
 //   int32 [8 .. 8 + w)       the kept key indices, in no particular order
 // A step costs O(w), whatever the number of cached keys: no scan of the delta row.
 constexpr int kStateHeader = 8;
@@ -539,7 +539,7 @@ __global__ void __launch_bounds__(256) decode_state_init_kernel(const float* __r
                                                                 int* __restrict__ state) {
     const int bh = blockIdx.x;
     int* hdr = state + (size_t)bh * state_stride(w_cap);
-    if (threadIdx.x == 0) { hdr[0] = keep; hdr[4] = 0; }      // count; the step kernels' ticket
+    if (threadIdx.x == 0) hdr[0] = keep;
     store_weakest(hdr, hdr + kStateHeader, keep, delta + (size_t)bh * ld, -1, 0);
 }
 
@@ -572,11 +572,10 @@ __device__ __forceinline__ void decode_state_update(const float* __restrict__ de
 template <typename T, int D>
 __global__ void __launch_bounds__(kAttnThreads) decode_list_attn_kernel(const T* __restrict__ q, const T* __restrict__ K,
                                                                         const T* __restrict__ V, const float* __restrict__ delta,
-                                                                        int64_t ld, int* state, int w_cap,
+                                                                        int64_t ld, const int* __restrict__ state, int w_cap,
                                                                         float* __restrict__ partial, int N, int Hq, int G,
                                                                         float scale_log2, int nsplit, int64_t ks_b, int64_t ks_l,
-                                                                        int64_t ks_h, int64_t vs_b, int64_t vs_l, int64_t vs_h,
-                                                                        T* __restrict__ o, float* __restrict__ lse) {
+                                                                        int64_t ks_h, int64_t vs_b, int64_t vs_l, int64_t vs_h) {
     __shared__ int list[kListSplit];
     const int split = blockIdx.x, bh = blockIdx.y, b = bh / Hq, h = bh % Hq, hk = h / G;
     const int tid = threadIdx.x;
@@ -591,14 +590,52 @@ __global__ void __launch_bounds__(kAttnThreads) decode_list_attn_kernel(const T*
     __syncthreads();
     decode_attend<T, D>(list, max(0, min(kListSplit, eff - split * kListSplit)), q, K, V, dl,
                         partial + ((size_t)bh * nsplit + split) * (D + 2), bh, b, hk, scale_log2, ks_b, ks_l, ks_h, vs_b, vs_l, vs_h);
-    // the row's last CTA (ticket: word 4 of the state header, zero between calls) combines the partials and then, every
-    // CTA of the row having read the state, lets the state take in the appended key
-    if (last_of_row(state + (size_t)bh * state_stride(w_cap) + 4, nsplit)) {
-        combine_row<T, D>(partial, o, lse, nsplit, bh);
-        __syncthreads();
-        decode_state_update(delta, ld, N, w_cap, state, bh);
-    }
 }
+
+// The step's second kernel, one CTA of 8 D threads per row: the splits' partials -> o, log-sum-exp, and then, every CTA of
+// the attention kernel having read the row's state, the state takes in the appended key. (Doing this in the attention
+// kernel's last CTA per row, as dma_decode does, was measured slower here, 16.5 -> 20.7 us per step: the state must then be
+// writable in the attention kernel, whose loads of the kept list no longer take the read-only path, and the update, which
+// scans the w kept keys, runs on 256 threads at the end of the row's critical path instead of 8 D.)
+template <typename T, int D>
+__global__ void __launch_bounds__(8 * D) decode_step_combine_kernel(const float* __restrict__ partial, T* __restrict__ o, float* __restrict__ lse,
+                                                                    int nsplit, const float* __restrict__ delta, int64_t ld,
+                                                                    int N, int w_cap, int* __restrict__ state) {
+    __shared__ float s_m[8], s_l[8], s_o[8][D];
+    const int bh = blockIdx.x, c = threadIdx.x % D, g = threadIdx.x / D;     // group g takes the splits s = g, g + 8, ...
+    const float* p = partial + (size_t)bh * nsplit * (D + 2);
+    float mx = -INFINITY;
+    for (int s = g; s < nsplit; s += 8) mx = fmaxf(mx, p[(size_t)s * (D + 2) + D]);
+    float l = 0.0f, acc = 0.0f;
+    for (int s = g; s < nsplit; s += 8) {
+        const float ms = p[(size_t)s * (D + 2) + D];
+        const float f = ms == -INFINITY ? 0.0f : exp2f(ms - mx);
+        l += p[(size_t)s * (D + 2) + D + 1] * f;
+        acc += p[(size_t)s * (D + 2) + c] * f;
+    }
+    s_o[g][c] = acc;
+    if (c == 0) { s_m[g] = mx; s_l[g] = l; }
+    __syncthreads();
+    if (g == 0) {
+        float m_all = -INFINITY;
+#pragma unroll
+        for (int q = 0; q < 8; ++q) m_all = fmaxf(m_all, s_m[q]);
+        float lt = 0.0f, at = 0.0f;
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            const float f = s_m[q] == -INFINITY ? 0.0f : exp2f(s_m[q] - m_all);
+            lt += s_l[q] * f;
+            at += s_o[q][c] * f;
+        }
+        const float v = lt > 0.0f ? at / lt : 0.0f;
+        if constexpr (sizeof(T) == 2) o[(size_t)bh * D + c] = __float2bfloat16_rn(v); else o[(size_t)bh * D + c] = v;
+        if (c == 0) lse[bh] = lt > 0.0f ? 0.6931471805599453f * (m_all + log2f(lt)) : -INFINITY;
+    }
+    // incremental decoding: the attention kernel has read the row's state, which can now take in the appended key
+    if (state) decode_state_update(delta, ld, N, w_cap, state, bh);
+}
+
+
 
 template <typename T, int D>
 int launch_typed(const Prob& P, const void* q, const void* K, const void* V, const float* delta, int64_t ld, void* o, float* lse,
@@ -714,8 +751,9 @@ static int launch_step_typed(const Prob& P, const void* q, const void* K, const 
     const int ns = list_splits(P);
     decode_list_attn_kernel<T, D><<<dim3(ns, P.B * P.Hq), kAttnThreads, 0, st>>>(
         (const T*)q, (const T*)K, (const T*)V, delta, ld, state, P.w_cap, partial, P.L, P.Hq, P.G, P.scale * 1.4426950408889634f, ns,
-        P.ks[0], P.ks[1], P.ks[2], P.vs[0], P.vs[1], P.vs[2], (T*)o, lse);
-    count_launch();
+        P.ks[0], P.ks[1], P.ks[2], P.vs[0], P.vs[1], P.vs[2]);
+    decode_step_combine_kernel<T, D><<<P.B * P.Hq, 8 * D, 0, st>>>(partial, (T*)o, lse, ns, delta, ld, P.L, P.w_cap, state);
+    count_launch(2);
     return check_launch();
 }
 

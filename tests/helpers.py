@@ -22,10 +22,13 @@ from paper_2508_02124_b200 import binding as dma
 #                                    row is a sum over the same (row, key) pairs with the same bf16-rounded weights (P for
 #                                    dV, dS for dQ / dK; Eqs. grad_v, grad_qk), so the rounding error of a row scales with
 #                                    that row's magnitude, not with the element's own value (channels cancel differently).
-#   dM (Eq. grad_m, column sums)    |err| <= atol * max(1, H)                  H = max |ref| over the keys of the element's
-#                                    (batch, head). dM_j = sum_i P_ij (dP_ij - D_i) cancels almost completely for a key
-#                                    that many rows attend to alone, and D is formed from the STORED bf16 O (Alg. 2), so
-#                                    its error follows the head's gradient scale, not |dM_j|.
+#   dM (Eq. grad_m, column sums)    |err| <= atol + u * |ref| per element. dM_j = sum_i dS_ij is a per-thread fp32 sum of fp32
+#                                    dS values in the kernels (nothing is rounded to bf16 on the way), so once both backward
+#                                    passes read the same stored O it agrees with the oracle to ~1e-5 relative (measured worst
+#                                    ratio against this bound: 0.02). Where the GPU backward must read the GPU forward's own O
+#                                    (dma_step_host) the bound relative to the tensor's largest magnitude applies instead: D is
+#                                    formed from the stored bf16 O (Alg. 2) and dM_j = sum_i P_ij (dP_ij - D_i) cancels almost
+#                                    completely for a key that many rows attend to alone.
 #   other sums (dW, dA of the mask backward, ...)  |err| <= atol * max(1, M), M = max |ref| of the tensor.
 #   log-sum-exp                      fp32 whatever the element type, carries the bias magnitude (1e2..1e4):
 #                                    atol + 1e-6 M, a few fp32 ulps of that magnitude.
@@ -124,7 +127,7 @@ def _kind_of(what):
     if any(t in ("dQ", "dK", "dV") for t in w):
         return "row"
     if "dM" in w:
-        return "head"
+        return "elem"
     if any(t in ("O", "o") for t in w):
         return "out"
     return "tensor"
@@ -138,8 +141,8 @@ def element_tolerance(ref, dtype, kind):
         return atol + K_OUT * UNIT[dtype] * a
     if kind == "row":                              # [..., d]: the element's own channel row
         return atol * np.maximum(1.0, a.max(-1, keepdims=True)) + 0.0 * a
-    if kind == "head":                             # [B, Hq, keys]: the element's own (batch, head)
-        return atol * np.maximum(1.0, a.max(-1, keepdims=True)) + 0.0 * a
+    if kind == "elem":                             # fp32 sums of fp32 terms: the stated bound plus one unit of the element type
+        return atol + UNIT[dtype] * a
     if kind == "lse":
         return atol + 1e-6 * (a.max() if a.size else 0.0) + 0.0 * a
     assert kind == "tensor", kind
@@ -148,7 +151,7 @@ def element_tolerance(ref, dtype, kind):
 
 def assert_close(got, ref, dtype, what, lse=False, kind=None):
     """Gate of the header: relative L2 over the whole tensor and the per-element max-abs bound of the tensor's kind
-    ("out", "row", "head", "tensor", "lse"; inferred from the tensor's name in `what` when not given)."""
+    ("out", "row", "elem", "tensor", "lse"; inferred from the tensor's name in `what` when not given)."""
     g = f64(got) if isinstance(got, torch.Tensor) else np.asarray(got, np.float64)
     ref = np.asarray(ref, np.float64)
     kind = "lse" if lse else (kind or _kind_of(what))
