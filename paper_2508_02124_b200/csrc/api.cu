@@ -94,74 +94,24 @@ int resolve(const dma_problem_t* p, Prob* o) {
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 
 static bool use_tensor_cores(const Prob& P) {
-    return P.dtype == DMA_BF16 && P.d == 128 && P.bm == 128 && P.bn == 128 && !(P.flags & DMA_FLAG_SIMT);
+    return P.dtype == DMA_BF16 && (P.d == 128 || P.d == 64) && P.bm == 128 && P.bn == 128 && !(P.flags & DMA_FLAG_SIMT);
 }
 
-// bf16 with 64 channels: the same kernels on zero-padded 128-channel copies held in the workspace (see pad64.cu)
-static bool use_padded(const Prob& P) {
-    return P.dtype == DMA_BF16 && P.d == 64 && P.bm == 128 && P.bn == 128 && !(P.flags & DMA_FLAG_SIMT);
-}
+static size_t fwd_ws_any(const Prob& P) { return use_tensor_cores(P) ? tc_fwd_ws_bytes(P) : (size_t)kWsHeaderBytes; }
 
-static size_t align256(size_t n) { return (n + 255) / 256 * 256; }
-
-// the 128-channel problem the padded copies form: packed [B, rows, H, 128] tensors, the caller's softmax scale
-static Prob padded_problem(const Prob& P) {
-    Prob R = P;
-    R.d = 128;
-    const int64_t q[3] = {(int64_t)P.Lq * P.Hq * 128, (int64_t)P.Hq * 128, 128}, k[3] = {(int64_t)P.L * P.Hkv * 128, (int64_t)P.Hkv * 128, 128};
-    for (int t = 0; t < 3; ++t) { R.qs[t] = R.os[t] = q[t]; R.ks[t] = R.vs[t] = k[t]; }
-    return R;
-}
-
-static size_t fwd_ws_any(const Prob& P) {
-    if (use_tensor_cores(P)) return tc_fwd_ws_bytes(P);
-    if (!use_padded(P)) return (size_t)kWsHeaderBytes;
-    const size_t nq = (size_t)P.B * P.Lq * P.Hq * 128 * 2, nk = (size_t)P.B * P.L * P.Hkv * 128 * 2;
-    return align256(tc_fwd_ws_bytes(padded_problem(P))) + 2 * align256(nq) + 2 * align256(nk);        // Q, O, K, V
-}
-
-static size_t bwd_ws_any(const Prob& P) {
-    if (use_tensor_cores(P)) return tc_bwd_ws_bytes(P);
-    if (!use_padded(P)) return simt_bwd_ws_bytes(P);
-    const size_t nq = (size_t)P.B * P.L * P.Hq * 128 * 2, nk = (size_t)P.B * P.L * P.Hkv * 128 * 2;
-    return align256(tc_bwd_ws_bytes(padded_problem(P))) + 4 * align256(nq) + 4 * align256(nk);        // Q, O, dO, dQ, K, V, dK, dV
-}
+static size_t bwd_ws_any(const Prob& P) { return use_tensor_cores(P) ? tc_bwd_ws_bytes(P) : simt_bwd_ws_bytes(P); }
 
 static int fwd_any(const Prob& P, const void* Q, const void* K, const void* V, const float* bias, const int32_t* expiry,
                    const uint32_t* bitmap, void* O, float* lse, void* ws, cudaStream_t st) {
     if (use_tensor_cores(P)) return launch_tc_fwd(P, Q, K, V, bias, expiry, bitmap, O, lse, ws, st);
-    if (!use_padded(P)) return launch_simt_fwd(P, Q, K, V, bias, expiry, bitmap, O, lse, st);
-    const Prob R = padded_problem(P);
-    const size_t nq = align256((size_t)P.B * P.Lq * P.Hq * 128 * 2), nk = align256((size_t)P.B * P.L * P.Hkv * 128 * 2);
-    char* base = (char*)ws + align256(tc_fwd_ws_bytes(R));
-    char *Qp = base, *Op = Qp + nq, *Kp = Op + nq, *Vp = Kp + nk;
-    int rc;
-    if ((rc = launch_pad64(Q, Qp, P.B, P.Lq, P.Hq, P.qs, st))) return rc;
-    if ((rc = launch_pad64(K, Kp, P.B, P.L, P.Hkv, P.ks, st))) return rc;
-    if ((rc = launch_pad64(V, Vp, P.B, P.L, P.Hkv, P.vs, st))) return rc;
-    if ((rc = launch_tc_fwd(R, Qp, Kp, Vp, bias, expiry, bitmap, Op, lse, ws, st))) return rc;
-    return launch_unpad64(Op, O, P.B, P.Lq, P.Hq, P.os, st);
+    return launch_simt_fwd(P, Q, K, V, bias, expiry, bitmap, O, lse, st);
 }
 
 static int bwd_any(const Prob& P, const void* Q, const void* K, const void* V, const void* O, const void* dO, const float* lse,
                    const float* bias, const int32_t* expiry, const uint32_t* bitmap, void* dQ, void* dK, void* dV, float* dM,
                    void* ws, cudaStream_t st) {
     if (use_tensor_cores(P)) return launch_tc_bwd(P, Q, K, V, O, dO, lse, bias, expiry, bitmap, dQ, dK, dV, dM, ws, st);
-    if (!use_padded(P)) return launch_simt_bwd(P, Q, K, V, O, dO, lse, bias, expiry, bitmap, dQ, dK, dV, dM, ws, st);
-    const Prob R = padded_problem(P);
-    const size_t nq = align256((size_t)P.B * P.L * P.Hq * 128 * 2), nk = align256((size_t)P.B * P.L * P.Hkv * 128 * 2);
-    char* base = (char*)ws + align256(tc_bwd_ws_bytes(R));
-    char *Qp = base, *Op = Qp + nq, *dOp = Op + nq, *dQp = dOp + nq, *Kp = dQp + nq, *Vp = Kp + nk, *dKp = Vp + nk, *dVp = dKp + nk;
-    int rc;
-    if ((rc = launch_pad64(Q, Qp, P.B, P.L, P.Hq, P.qs, st))) return rc;
-    if ((rc = launch_pad64(O, Op, P.B, P.L, P.Hq, P.os, st))) return rc;
-    if ((rc = launch_pad64(dO, dOp, P.B, P.L, P.Hq, P.os, st))) return rc;
-    if ((rc = launch_pad64(K, Kp, P.B, P.L, P.Hkv, P.ks, st))) return rc;
-    if ((rc = launch_pad64(V, Vp, P.B, P.L, P.Hkv, P.vs, st))) return rc;
-    if ((rc = launch_tc_bwd(R, Qp, Kp, Vp, Op, dOp, lse, bias, expiry, bitmap, dQp, dKp, dVp, dM, ws, st))) return rc;
-    if ((rc = launch_unpad64(dQp, dQ, P.B, P.L, P.Hq, P.qs, st))) return rc;
-    if ((rc = launch_unpad64(dKp, dK, P.B, P.L, P.Hkv, P.ks, st))) return rc;
-    return launch_unpad64(dVp, dV, P.B, P.L, P.Hkv, P.vs, st);
+    return launch_simt_bwd(P, Q, K, V, O, dO, lse, bias, expiry, bitmap, dQ, dK, dV, dM, ws, st);
 }
 
 static int device_ok() {
@@ -342,7 +292,7 @@ int dma_attn_fwd(const dma_problem_t* p, const void* Q, const void* K, const voi
     if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || !aligned16(bias) || !aligned16(expiry) ||
         !aligned16(lse))
         return DMA_ERR_ALIGN;
-    const bool tc = use_tensor_cores(P) || use_padded(P);
+    const bool tc = use_tensor_cores(P);
     if ((P.flags & DMA_FLAG_COMPACT_KV) && !tc) return DMA_ERR_UNSUPPORTED;
     if (!ws || ws_bytes < fwd_ws_any(P) || !aligned16(ws)) return DMA_ERR_WORKSPACE;
     if ((rc = device_ok())) return rc;
@@ -370,7 +320,7 @@ int dma_attn_fwd_chunk(const dma_problem_t* p, int32_t q_begin, int32_t q_len, c
         if (q_default) P.qs[t] = packed[t];
         if (o_default) P.os[t] = packed[t];
     }
-    if (use_tensor_cores(P) || use_padded(P)) P.flags |= DMA_FLAG_COMPACT_KV;   // the gathered-key kernel has no tile alignment between rows and keys
+    if (use_tensor_cores(P)) P.flags |= DMA_FLAG_COMPACT_KV;   // the gathered-key kernel has no tile alignment between rows and keys
     if (!ws || ws_bytes < fwd_ws_any(P) || !aligned16(ws)) return DMA_ERR_WORKSPACE;
     if ((rc = device_ok())) return rc;
     cudaStream_t st = (cudaStream_t)cuda_stream;
@@ -388,7 +338,7 @@ int dma_attn_bwd(const dma_problem_t* p, const void* Q, const void* K, const voi
     if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || !aligned16(dO) || !aligned16(dQ) ||
         !aligned16(dK) || !aligned16(dV) || !aligned16(dM) || !aligned16(lse))
         return DMA_ERR_ALIGN;
-    const bool tc = use_tensor_cores(P) || use_padded(P);
+    const bool tc = use_tensor_cores(P);
     if ((P.flags & DMA_FLAG_COMPACT_KV) && !tc) return DMA_ERR_UNSUPPORTED;
     if (!ws || ws_bytes < bwd_ws_any(P) || !aligned16(ws)) return DMA_ERR_WORKSPACE;
     if ((rc = device_ok())) return rc;

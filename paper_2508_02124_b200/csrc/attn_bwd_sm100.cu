@@ -1,4 +1,4 @@
-// Tensor-core backward (Sec. 4.3, Alg. 2) for bf16, d = 128, on sm_100a.
+// Tensor-core backward (Sec. 4.3, Alg. 2) for bf16, d = 128 or 64, on sm_100a.
 //
 // One CTA owns one 128-key tile of one KV head and, as in Alg. 2's outer loop, keeps dK, dV (fp32, tensor memory)
 // and dM (registers) for it while walking the query heads of the group and their active query tiles in steps of
@@ -9,7 +9,10 @@
 //   P^T  = exp2(c S^T + log2e bias_j) where j <= i < expiry[j], else 0;   dS^T = P^T o dP^T
 //   dV  += P^T dO           dK  += dS^T Q                      (TMEM x smem  -> TMEM, 128 columns each)
 //   dQ^T = K^T dS^T                                            (smem x smem  -> TMEM, 64 columns), staged in shared memory
-//                                                              and added to the fp32 dQ accumulator by TMA reduce-adds
+//                                                              and added to the fp32 dQ accumulator by bulk reduce-adds
+// The dQ accumulator is blocked: 16 rows x 32 channels of one head are 2 KB of consecutive floats, so that a staged
+// quarter step leaves as ONE contiguous bulk reduce-add (as a tile of a [B, L, Hq, d] tensor map the same 2 KB were 16
+// strided 128-byte rows, and issuing that request took the drain warp ~350 cycles: the drain was as long as the step).
 // Shared-memory bandwidth is the scarce resource (operand reads of the smem x smem MMAs alone take ~1400 of a step's
 // ~2250 cycles), so the compute warps read nothing from shared memory per element.
 // Warp roles (16 warps): warps 0-7 compute (thread = key; warps w and w+4 share the 32 TMEM lanes of quadrant w%4 and
@@ -17,6 +20,10 @@
 // warps 13 and 14 MMA issuers (S^T, dP^T | dV, dK, dQ^T; whole warps with warp-uniform values, one elected lane
 // issues), warp 15 stages the ninth k-step operand of each step's query rows.
 // TMEM columns: dK [0,128) dV [128,256) S^T [256,320) dP^T [320,384) P^T [384,416) dS^T [416,448) dQ^T [448,512).
+// kD = 64 (its own instantiations): K, V, Q and dO tiles are one swizzled half tile each (the second half of every buffer
+// stays unused), S^T and dP^T have four k-steps and the ninth, dK and dV take 64 columns. dQ^T = K^T dS^T keeps M = 128:
+// its upper 64 lanes multiply whatever the unused half of the K buffer holds and are never read (rows of an MMA do not
+// mix), so drain warps 2 and 3 only follow the barriers.
 #include <cstdlib>
 
 #include "common.cuh"
@@ -63,7 +70,8 @@ struct BwdParams {
     const int32_t* expiry;
     const uint32_t* bitmap;
     int sched_group;            // (batch, head) entries per scheduling group, a divisor of gridDim.x
-    float* dQacc;               // [B, L, Hq, 128] fp32, zeroed
+    float* dQacc;               // fp32, zeroed, blocked: [B, Hq, Lblk, d / 32][16 rows][32 channels]
+    int Lblk;                   // 16-row blocks per head: 8 * Tr (rows padded to whole 128-row tiles)
     __nv_bfloat16* dK;
     __nv_bfloat16* dV;
     float* dM;
@@ -99,11 +107,12 @@ __device__ __forceinline__ uint4 split3(float x) {
 // same query rows, so the walk over query tiles [first key's tile, last expiry's tile] wastes little. K and V rows
 // are gathered once with 16-byte asynchronous copies; dK and dV are added to fp32 accumulators (the query heads of a
 // group meet there), dM is written directly.
-template <bool kCompact>
+template <bool kCompact, int kD>
 __global__ void __launch_bounds__(kThreads, 1)
 bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
-           const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmG,
-           const __grid_constant__ CUtensorMap tmDQ, const BwdParams P) {
+           const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmG, const BwdParams P) {
+    static_assert(kD == 128 || kD == 64, "head dimensions of the tensor-core kernels");
+    constexpr int kHalves = kD / 64;                 // 64-channel (128-byte) swizzled half tiles per operand tile
     extern __shared__ uint8_t smem_raw[];
     SharedStorage& S = *reinterpret_cast<SharedStorage*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const int tid = threadIdx.x, lane = tid & 31;
@@ -317,7 +326,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             tc_fence_after();
             __nv_bfloat16* dk = P.dK + b * P.ks_b + (int64_t)j * P.ks_l + hk * P.ks_h;
             __nv_bfloat16* dv = P.dV + b * P.vs_b + (int64_t)j * P.vs_l + hk * P.vs_h;
-            const size_t arow = ((size_t)(b * P.L + min(j, P.L - 1)) * P.Hkv + hk) * 128 +      // accumulator row (compact mode)
+            const size_t arow = ((size_t)(b * P.L + min(j, P.L - 1)) * P.Hkv + hk) * kD +      // accumulator row (compact mode)
                                 (kCompact ? (size_t)(hq_c % P.G) * (size_t)P.acc_slot : 0);
 #pragma unroll
             for (int which = 0; which < 2; ++which) {
@@ -325,8 +334,8 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                 __nv_bfloat16* out = which == 0 ? dk : dv;
                 float* acc = (which == 0 ? P.dKacc : P.dVacc) + arow;
 #pragma unroll
-                for (int cc = 0; cc < 2; ++cc) {
-                    const int c = hsel * 2 + cc;
+                for (int cc = 0; cc < kHalves; ++cc) {
+                    const int c = hsel * kHalves + cc;
                     uint32_t o[32];
                     if (n_steps > 0) {
                         tmem_ld32(tmem + lane_base + (which == 0 ? cDK : cDV) + c * 32, o);
@@ -379,12 +388,15 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             if (!ok) break;
             tc_fence_after();
             uint32_t v[64];
-            tmem_ld32(tmem + lane_base + cDQ, *reinterpret_cast<uint32_t(*)[32]>(&v[0]));
-            tmem_ld32(tmem + lane_base + cDQ + 32, *reinterpret_cast<uint32_t(*)[32]>(&v[32]));
-            tc_wait_ld();
+            if (dw * 32 < kD) {
+                tmem_ld32(tmem + lane_base + cDQ, *reinterpret_cast<uint32_t(*)[32]>(&v[0]));
+                tmem_ld32(tmem + lane_base + cDQ + 32, *reinterpret_cast<uint32_t(*)[32]>(&v[32]));
+                tc_wait_ld();
+            }
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&S.dq_free);
+            if (dw * 32 >= kD) continue;               // (no channels of this warp)
 #pragma unroll
             for (int qr = 0; qr < 4; ++qr) {           // quarter steps of 16 query rows, two staging buffers in turn
                 if (lane == 0) bulk_wait_read_1(); __syncwarp();
@@ -392,8 +404,9 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                 for (int u = 0; u < 16; ++u) S.dq_stage[dw][qr & 1][u][lane] = __uint_as_float(v[qr * 16 + u]);
                 fence_proxy_async();
                 __syncwarp();
-                if (lane == 0 && i0 + qr * 16 < P.L) {
-                    tma_reduce_add_4d(&tmDQ, &S.dq_stage[dw][qr & 1][0][0], dw * 32, hk * P.G + g, i0 + qr * 16, b);   // rows beyond L are clipped
+                if (lane == 0 && i0 + qr * 16 < P.L) {       // (rows beyond L inside the block land in the accumulator's padding)
+                    float* blk = P.dQacc + ((((size_t)(b * P.Hq + hk * P.G + g) * P.Lblk + (i0 >> 4) + qr) * (kD / 32) + dw) << 9);
+                    bulk_reduce_add_f32(blk, &S.dq_stage[dw][qr & 1][0][0], 2048);
                 }
                 if (lane == 0) bulk_commit();
             }
@@ -415,9 +428,9 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                     const uint32_t off = r * 128 + ((c ^ (r & 7)) << 4);
                     const int nb = j < P.L ? 16 : 0;
                     cp_async16(S.k + off, P.Kg + krow, nb);
-                    cp_async16(S.k + off + kKVBytes / 2, P.Kg + krow + 64, nb);
+                    if constexpr (kD == 128) cp_async16(S.k + off + kKVBytes / 2, P.Kg + krow + 64, nb);
                     cp_async16(S.v + off, P.Vg + vrow, nb);
-                    cp_async16(S.v + off + kKVBytes / 2, P.Vg + vrow + 64, nb);
+                    if constexpr (kD == 128) cp_async16(S.v + off + kKVBytes / 2, P.Vg + vrow + 64, nb);
                 }
                 cp_async_wait_all();
                 fence_proxy_async();
@@ -425,8 +438,8 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&S.kv_full);
             } else if (lane == 0) {
-                mbar_arrive_expect_tx(&S.kv_full, 2 * kKVBytes);
-                for (int hf = 0; hf < 2; ++hf) {
+                mbar_arrive_expect_tx(&S.kv_full, kHalves * kKVBytes);
+                for (int hf = 0; hf < kHalves; ++hf) {
                     tma_load_4d(&S.k[hf * (kKVBytes / 2)], &tmK, &S.kv_full, hf * 64, j0, hk, b);
                     tma_load_4d(&S.v[hf * (kKVBytes / 2)], &tmV, &S.kv_full, hf * 64, j0, hk, b);
                 }
@@ -439,8 +452,8 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                 if (n >= kStages) ok = mbar_wait_warp(&S.qd_empty[st], ((n / kStages) - 1) & 1, abort_flag);
                 if (!ok) break;
                 if (lane == 0) {
-                    mbar_arrive_expect_tx(&S.qd_full[st], 2 * kQBytes);
-                    for (int hf = 0; hf < 2; ++hf) {
+                    mbar_arrive_expect_tx(&S.qd_full[st], kHalves * kQBytes);
+                    for (int hf = 0; hf < kHalves; ++hf) {
                         tma_load_4d(&S.q[st][hf * (kQBytes / 2)], &tmQ, &S.qd_full[st], hf * 64, i0, h, b);
                         tma_load_4d(&S.g[st][hf * (kQBytes / 2)], &tmG, &S.qd_full[st], hf * 64, i0, h, b);
                     }
@@ -507,12 +520,12 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                 const uint64_t dX = dX0 + (uint64_t)(st * (2048 >> 4));
                 if (elect_one()) {
 #pragma unroll
-                    for (int kk = 0; kk < 8; ++kk)
+                    for (int kk = 0; kk < kD / 16; ++kk)
                         mma_ss(tmem_u + cS, dK + (uint64_t)(((kk >> 2) * (kKVBytes / 2) + (kk & 3) * 32) >> 4),
                                dQ + (uint64_t)(((kk >> 2) * (kQBytes / 2) + (kk & 3) * 32) >> 4), id_sdp, kk > 0);
                     mma_ss(tmem_u + cS, dOnesLo, dX, id_sdp, 1u);          // S^T  += 1 (x) (-lse / scale)
 #pragma unroll
-                    for (int kk = 0; kk < 8; ++kk)
+                    for (int kk = 0; kk < kD / 16; ++kk)
                         mma_ss(tmem_u + cDP, dV + (uint64_t)(((kk >> 2) * (kKVBytes / 2) + (kk & 3) * 32) >> 4),
                                dG + (uint64_t)(((kk >> 2) * (kQBytes / 2) + (kk & 3) * 32) >> 4), id_sdp, kk > 0);
                     mma_ss(tmem_u + cDP, dOnesHi, dX, id_sdp, 1u);         // dP^T += 1 (x) (-D)
@@ -522,7 +535,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             }
         } else if (warp == 14) {
             // ============================ MMA issuer 2: dV += P^T dO, dK += dS^T Q, dQ^T = K^T dS^T ============================
-            constexpr uint32_t id_dkv = idesc_bf16(128, 128, 0, 1);    // P^T|dS^T (TMEM) x dO|Q (MN-major)    -> 128 x 128
+            constexpr uint32_t id_dkv = idesc_bf16(128, kD, 0, 1);     // P^T|dS^T (TMEM) x dO|Q (MN-major)    -> 128 x d
             constexpr uint32_t id_dq = idesc_bf16(128, 64, 1, 1);      // K^T (MN-major) x dS^T (MN-major)     -> 128 x 64
             const uint64_t dKt = smem_desc_sw128(smem_u32(S.k), kKVBytes / 2, 1024), dDs = smem_desc_sw128(smem_u32(S.ds), 16, 1024);
             const uint64_t dGm0 = smem_desc_sw128(smem_u32(S.g[0]), kQBytes / 2, 1024), dQm0 = smem_desc_sw128(smem_u32(S.q[0]), kQBytes / 2, 1024);
@@ -564,11 +577,12 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
     if (tid == 0 && S.abort_flag) atomicExch(P.status, (int32_t)DMA_ERR_DEVICE_TIMEOUT);
 }
 
-// D_i = dO_i . O_i  (Alg. 2): 16 lanes per (b, h, i), 16-byte loads (a row of 128 bf16 is 16 x 16 bytes)
+// D_i = dO_i . O_i  (Alg. 2): kLanes = d / 8 lanes per (b, h, i), 16-byte loads (a row of 128 bf16 is 16 x 16 bytes)
+template <int kLanes>
 __global__ void rowdot_bf16_kernel(const __nv_bfloat16* __restrict__ O, const __nv_bfloat16* __restrict__ dO,
                                    float* __restrict__ Dv, int B, int L, int Hq, int64_t os_b, int64_t os_l, int64_t os_h) {
-    const long row = (long)blockIdx.x * (blockDim.x / 16) + threadIdx.x / 16;
-    const int sub = threadIdx.x % 16;
+    const long row = (long)blockIdx.x * (blockDim.x / kLanes) + threadIdx.x / kLanes;
+    const int sub = threadIdx.x % kLanes;
     float s = 0.0f;
     if (row < (long)B * Hq * L) {
         const int i = row % L, h = (row / L) % Hq, b = row / ((long)L * Hq);
@@ -581,24 +595,39 @@ __global__ void rowdot_bf16_kernel(const __nv_bfloat16* __restrict__ O, const __
             s = fmaf(__uint_as_float(au[t] & 0xffff0000u), __uint_as_float(gu[t] & 0xffff0000u), s);
         }
     }
-    for (int m = 8; m; m >>= 1) s += __shfl_xor_sync(0xffffffffu, s, m);
+    for (int m = kLanes / 2; m; m >>= 1) s += __shfl_xor_sync(0xffffffffu, s, m);
     if (sub == 0 && row < (long)B * Hq * L) Dv[row] = s;
 }
 
-// fp32 accumulator [B, L, Hq, 128] (unscaled dS K sums) -> softmax scale applied -> bf16 dQ in the caller's layout; 8 elements per thread.
+// fp32 accumulator [B, L, Hq, d] (unscaled dS K sums) -> softmax scale applied -> bf16 dQ in the caller's layout; 8 elements per thread.
 // nslots > 1: the accumulator is nslots copies, slot_stride elements apart, added here in slot order (a fixed order: the
 // result is then the same bits from run to run).
 __global__ void dq_convert_bf16_kernel(const float* __restrict__ acc, __nv_bfloat16* __restrict__ dQ, size_t n8, int L, int Hq,
-                                       int64_t qs_b, int64_t qs_l, int64_t qs_h, float scale, int nslots = 1, int64_t slot_stride = 0) {
+                                       int64_t qs_b, int64_t qs_l, int64_t qs_h, float scale, int d, int nslots = 1, int64_t slot_stride = 0) {
     const size_t t = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (t >= n8) return;
     const size_t e = t * 8;
-    const int c = e % 128, h = (e / 128) % Hq, i = (e / ((size_t)128 * Hq)) % L, b = e / ((size_t)128 * Hq * L);
+    const int c = e % d, h = (e / d) % Hq, i = (e / ((size_t)d * Hq)) % L, b = e / ((size_t)d * Hq * L);
     float4 a = *reinterpret_cast<const float4*>(acc + e), bb = *reinterpret_cast<const float4*>(acc + e + 4);
     for (int sl = 1; sl < nslots; ++sl) {
         const float4 a2 = *reinterpret_cast<const float4*>(acc + (size_t)sl * slot_stride + e), b2 = *reinterpret_cast<const float4*>(acc + (size_t)sl * slot_stride + e + 4);
         a.x += a2.x; a.y += a2.y; a.z += a2.z; a.w += a2.w; bb.x += b2.x; bb.y += b2.y; bb.z += b2.z; bb.w += b2.w;
     }
+    uint4 o;
+    o.x = ptx::pack_bf16(a.x * scale, a.y * scale); o.y = ptx::pack_bf16(a.z * scale, a.w * scale);
+    o.z = ptx::pack_bf16(bb.x * scale, bb.y * scale); o.w = ptx::pack_bf16(bb.z * scale, bb.w * scale);
+    *reinterpret_cast<uint4*>(dQ + b * qs_b + (int64_t)i * qs_l + h * qs_h + c) = o;
+}
+
+// blocked fp32 dQ accumulator (see BwdParams::dQacc) -> softmax scale applied -> bf16 dQ in the caller's layout; 8 elements per thread
+__global__ void dq_unblock_bf16_kernel(const float* __restrict__ acc, __nv_bfloat16* __restrict__ dQ, size_t n8, int L, int Hq, int Lblk,
+                                       int64_t qs_b, int64_t qs_l, int64_t qs_h, float scale, int d) {
+    const size_t t = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= n8) return;
+    const size_t e = t * 8;                       // element of the packed [B, L, Hq, d] order
+    const int c = e % d, h = (e / d) % Hq, i = (e / ((size_t)d * Hq)) % L, b = e / ((size_t)d * Hq * L);
+    const float* src = acc + (((((size_t)(b * Hq + h) * Lblk + (i >> 4)) * (d >> 5) + (c >> 5)) * 16 + (i & 15)) << 5) + (c & 31);
+    const float4 a = *reinterpret_cast<const float4*>(src), bb = *reinterpret_cast<const float4*>(src + 4);
     uint4 o;
     o.x = ptx::pack_bf16(a.x * scale, a.y * scale); o.y = ptx::pack_bf16(a.z * scale, a.w * scale);
     o.z = ptx::pack_bf16(bb.x * scale, bb.y * scale); o.w = ptx::pack_bf16(bb.z * scale, bb.w * scale);
@@ -648,13 +677,13 @@ __global__ void __launch_bounds__(1024) lifetime_perm_kernel(const int32_t* __re
     for (int t = L + tid; t < Tc * 128; t += 1024) out[t] = L;
 }
 
-// workspace layout: header | D [rows] | dQ accumulator [rows x d] | (token-compacted mode) permutation | dK, dV accumulators
+// workspace layout: header | D [rows] | dQ accumulator [B x Hq x (Tr x 128) x d] | (token-compacted mode) permutation | dK, dV accumulators
 static size_t bwd_rows64(const Prob& P) { return ((((size_t)P.B * P.Hq * P.L) + 63) / 64) * 64; }
+static size_t bwd_acc_floats(const Prob& P) { return (size_t)P.B * P.Hq * P.Tr * 128 * P.d; }     // rows padded to whole query tiles
 static size_t bwd_perm_ints(const Prob& P) { return (((size_t)P.B * P.Hq * P.Tc * 128) + 63) / 64 * 64; }
 
 size_t tc_bwd_ws_bytes(const Prob& P) {
-    const size_t rows = (size_t)P.B * P.Hq * P.L;
-    size_t n = kWsHeaderBytes + (bwd_rows64(P) + rows * P.d) * sizeof(float);
+    size_t n = kWsHeaderBytes + (bwd_rows64(P) + bwd_acc_floats(P)) * sizeof(float);
     const size_t slots = (P.flags & DMA_FLAG_DETERMINISTIC) ? (size_t)P.G : 1;      // per-head dK / dV accumulators
     if (P.flags & DMA_FLAG_COMPACT_KV) n += bwd_perm_ints(P) * sizeof(int) + 2 * slots * (size_t)P.B * P.L * P.Hkv * P.d * sizeof(float);
     return n;
@@ -669,7 +698,7 @@ int launch_tc_bwd(const Prob& P, const void* Q, const void* K, const void* V, co
     const size_t rows = (size_t)P.B * P.Hq * P.L, nq = rows * P.d, nkv = (size_t)P.B * P.L * P.Hkv * P.d;
     float* Dv = reinterpret_cast<float*>((char*)ws + kWsHeaderBytes);
     float* acc = Dv + bwd_rows64(P);
-    int* perm = reinterpret_cast<int*>(acc + nq);
+    int* perm = reinterpret_cast<int*>(acc + bwd_acc_floats(P));
     const size_t slots = (compact && (P.flags & DMA_FLAG_DETERMINISTIC)) ? (size_t)P.G : 1;
     float* accK = reinterpret_cast<float*>(perm + bwd_perm_ints(P));
     float* accV = accK + slots * nkv;
@@ -679,11 +708,13 @@ int launch_tc_bwd(const Prob& P, const void* Q, const void* K, const void* V, co
     if ((rc = make_tmap_bf16(&tmG, dO, P.B, P.L, P.Hq, P.d, P.os, 64))) return rc;
     if ((rc = make_tmap_bf16(&tmK, K, P.B, P.L, P.Hkv, P.d, P.ks, 128))) return rc;
     if ((rc = make_tmap_bf16(&tmV, V, P.B, P.L, P.Hkv, P.d, P.vs, 128))) return rc;
-    CUtensorMap tmDQ;
-    if ((rc = make_tmap_f32_rows(&tmDQ, acc, P.B, P.L, P.Hq, 16, 32))) return rc;
-    rowdot_bf16_kernel<<<(unsigned)((rows + 15) / 16), 256, 0, st>>>((const __nv_bfloat16*)O, (const __nv_bfloat16*)dO, Dv, P.B, P.L, P.Hq,
-                                                                    P.os[0], P.os[1], P.os[2]);
-    if (cudaMemsetAsync(acc, 0, nq * sizeof(float), st) != cudaSuccess) return DMA_ERR_CUDA;
+    if (P.d == 128)
+        rowdot_bf16_kernel<16><<<(unsigned)((rows + 15) / 16), 256, 0, st>>>((const __nv_bfloat16*)O, (const __nv_bfloat16*)dO, Dv, P.B, P.L, P.Hq,
+                                                                            P.os[0], P.os[1], P.os[2]);
+    else
+        rowdot_bf16_kernel<8><<<(unsigned)((rows + 31) / 32), 256, 0, st>>>((const __nv_bfloat16*)O, (const __nv_bfloat16*)dO, Dv, P.B, P.L, P.Hq,
+                                                                           P.os[0], P.os[1], P.os[2]);
+    if (cudaMemsetAsync(acc, 0, bwd_acc_floats(P) * sizeof(float), st) != cudaSuccess) return DMA_ERR_CUDA;
     if (cudaMemsetAsync(dM, 0, rows * sizeof(float), st) != cudaSuccess) return DMA_ERR_CUDA;   // two partial sums are added per key
     if (compact) {
         if (cudaMemsetAsync(accK, 0, 2 * slots * nkv * sizeof(float), st) != cudaSuccess) return DMA_ERR_CUDA;
@@ -691,7 +722,7 @@ int launch_tc_bwd(const Prob& P, const void* Q, const void* K, const void* V, co
         count_launch();
     }
     BwdParams bp;
-    bp.lse = lse; bp.Dv = Dv; bp.bias = bias; bp.expiry = expiry; bp.bitmap = bitmap; bp.dQacc = acc;
+    bp.lse = lse; bp.Dv = Dv; bp.bias = bias; bp.expiry = expiry; bp.bitmap = bitmap; bp.dQacc = acc; bp.Lblk = P.Tr * 8;
     bp.dK = (__nv_bfloat16*)dK; bp.dV = (__nv_bfloat16*)dV; bp.dM = dM; bp.status = (int32_t*)ws;
     bp.B = P.B; bp.Hq = P.Hq; bp.Hkv = P.Hkv; bp.G = P.G; bp.L = P.L; bp.Tr = P.Tr; bp.Tc = P.Tc; bp.Wd = P.Wd;
     bp.ignore_bitmap = (P.flags & DMA_FLAG_IGNORE_BITMAP) ? 1 : 0;
@@ -704,7 +735,7 @@ int launch_tc_bwd(const Prob& P, const void* Q, const void* K, const void* V, co
         const int gx = compact ? P.B * P.Hq : P.B * P.Hkv;
         int sg = gx;
         {
-            const double per_entry = (double)(compact ? 1 : P.G) * P.L * 128 * 8;     // token-compacted mode: an entry is one query head
+            const double per_entry = (double)(compact ? 1 : P.G) * P.L * P.d * 8;     // token-compacted mode: an entry is one query head
             int want = (int)(160.0 * 1024 * 1024 / per_entry);
             want = want < 1 ? 1 : want;
             for (sg = want < gx ? want : gx; gx % sg; --sg) {}
@@ -718,19 +749,21 @@ int launch_tc_bwd(const Prob& P, const void* Q, const void* K, const void* V, co
     const size_t smem = sizeof(SharedStorage) + 1024;
     timing_mark(1, false, st);
     if (compact) {
-        if (cudaFuncSetAttribute(bwd_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return DMA_ERR_CUDA;
-        bwd_kernel<true><<<dim3(P.B * P.Hq, P.Tc), kThreads, smem, st>>>(tmQ, tmK, tmV, tmG, tmDQ, bp);
+        auto kern = P.d == 128 ? bwd_kernel<true, 128> : bwd_kernel<true, 64>;
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return DMA_ERR_CUDA;
+        kern<<<dim3(P.B * P.Hq, P.Tc), kThreads, smem, st>>>(tmQ, tmK, tmV, tmG, bp);
         timing_mark(1, true, st);
         const int nb = (int)((nkv / 8 + 255) / 256);
-        dq_convert_bf16_kernel<<<nb, 256, 0, st>>>(accK, (__nv_bfloat16*)dK, nkv / 8, P.L, P.Hkv, P.ks[0], P.ks[1], P.ks[2], P.scale, (int)slots, (int64_t)nkv);
-        dq_convert_bf16_kernel<<<nb, 256, 0, st>>>(accV, (__nv_bfloat16*)dV, nkv / 8, P.L, P.Hkv, P.vs[0], P.vs[1], P.vs[2], 1.0f, (int)slots, (int64_t)nkv);
+        dq_convert_bf16_kernel<<<nb, 256, 0, st>>>(accK, (__nv_bfloat16*)dK, nkv / 8, P.L, P.Hkv, P.ks[0], P.ks[1], P.ks[2], P.scale, P.d, (int)slots, (int64_t)nkv);
+        dq_convert_bf16_kernel<<<nb, 256, 0, st>>>(accV, (__nv_bfloat16*)dV, nkv / 8, P.L, P.Hkv, P.vs[0], P.vs[1], P.vs[2], 1.0f, P.d, (int)slots, (int64_t)nkv);
         count_launch(2);
     } else {
-        if (cudaFuncSetAttribute(bwd_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return DMA_ERR_CUDA;
-        bwd_kernel<false><<<dim3(P.B * P.Hkv, P.Tc), kThreads, smem, st>>>(tmQ, tmK, tmV, tmG, tmDQ, bp);
+        auto kern = P.d == 128 ? bwd_kernel<false, 128> : bwd_kernel<false, 64>;
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return DMA_ERR_CUDA;
+        kern<<<dim3(P.B * P.Hkv, P.Tc), kThreads, smem, st>>>(tmQ, tmK, tmV, tmG, bp);
         timing_mark(1, true, st);
     }
-    dq_convert_bf16_kernel<<<(unsigned)((nq / 8 + 255) / 256), 256, 0, st>>>(acc, (__nv_bfloat16*)dQ, nq / 8, P.L, P.Hq, P.qs[0], P.qs[1], P.qs[2], P.scale);
+    dq_unblock_bf16_kernel<<<(unsigned)((nq / 8 + 255) / 256), 256, 0, st>>>(acc, (__nv_bfloat16*)dQ, nq / 8, P.L, P.Hq, P.Tr * 8, P.qs[0], P.qs[1], P.qs[2], P.scale, P.d);
     count_launch(3);
     return check_launch();
 }

@@ -1,4 +1,4 @@
-// Tensor-core forward (Sec. 4.2, Alg. 1) for bf16, d = 128, on sm_100a: TMA-staged Q/K/V tiles, tcgen05 MMAs with
+// Tensor-core forward (Sec. 4.2, Alg. 1) for bf16, d = 128 or 64, on sm_100a: TMA-staged Q/K/V tiles, tcgen05 MMAs with
 // accumulators in tensor memory, online softmax in registers, bitmap-driven tile skipping.
 //
 // One CTA owns two consecutive 128-row query tiles of one (batch, head) and walks the union of their active key
@@ -16,6 +16,8 @@
 //                    k-step), O_w += P_w V, ping-ponging between the two query tiles
 //   warps 2, 3       stagers for query tile 0 / 1: ninth k-step operands, expiry vector, fast / general flag
 // Tensor memory (512 columns): S0 [0,128) S1 [128,256) O0 [256,384) O1 [384,512); P_w aliases columns [0,64) of S_w.
+// kD = 64 (its own instantiations): Q, K and V tiles are one 16 KB half tile each (the second half of every buffer stays
+// unused), S = Q K^T has four k-steps and the ninth, O_w takes 64 columns.
 // The log-sum-exp replaces Alg. 1's (l, m) pair.
 #include <cstdlib>
 
@@ -98,10 +100,13 @@ constexpr int kWarpProducer = 0, kWarpIssuer = 1, kWarpStager0 = 2, kWarpStager1
 // rows are constant) and flags the 32-column chunks that still need the per-element test.
 // kBlockSkip: MMA-block skipping inside executed tiles (DMA_FLAG_BLOCK_SKIP), a separate instantiation so that the
 // default kernel carries none of its code (the kernel is sensitive to the size of its service warps' loops).
-template <bool kCompact, bool kBlockSkip>
+template <bool kCompact, bool kBlockSkip, int kD>
 __global__ void __launch_bounds__(kThreads, 1)
 fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
            const __grid_constant__ CUtensorMap tmV, const FwdParams P) {
+    static_assert(kD == 128 || kD == 64, "head dimensions of the tensor-core kernels");
+    constexpr int kHalves = kD / 64;                         // 64-channel (128-byte) swizzled half tiles per operand tile
+    constexpr uint32_t kLoadBytes = kHalves * (kTileBytes / 2);
     extern __shared__ uint8_t smem_raw[];
     SharedStorage& S = *reinterpret_cast<SharedStorage*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const int tid = threadIdx.x, lane = tid & 31;
@@ -264,7 +269,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                 const float r_new = stab_resid(m_new);
                 const float f = (m_new == -INFINITY) ? 1.0f : (m_ref == -INFINITY) ? 0.0f : ex2(fmaf(m_ref - m_new, P.scale_log2, r_new - r_ref));
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
+                for (int c = 0; c < kD / 32; ++c) {
                     uint32_t o[32];
                     tmem_ld32(tO + c * 32, o);
                     tc_wait_ld();
@@ -339,7 +344,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             const float inv = l > 0.0f ? 1.0f / l : 0.0f;
             __nv_bfloat16* orow = P.O + b * P.os_b + (int64_t)il * P.os_l + h * P.os_h;
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
+            for (int c = 0; c < kD / 32; ++c) {
                 uint32_t o[32];
                 if (n_used > 0) {
                     tmem_ld32(tO + c * 32, o);
@@ -371,9 +376,9 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             // instruction; padding entries (-1) are zero-filled). Each lane's copies report to the stage's barrier.
             const bool isK = warp == kWarpProducer;
             if (isK && lane == 0) {
-                mbar_arrive_expect_tx(&S.q_full, has1 ? 2 * kTileBytes : kTileBytes);
+                mbar_arrive_expect_tx(&S.q_full, has1 ? 2 * kLoadBytes : kLoadBytes);
                 for (int w = 0; w < (has1 ? 2 : 1); ++w)
-                    for (int hf = 0; hf < 2; ++hf)
+                    for (int hf = 0; hf < kHalves; ++hf)
                         tma_load_4d(&S.q[w][hf * (kTileBytes / 2)], &tmQ, &S.q_full, hf * 64, (qt0 + w) * 128, h, b);
             }
             const int* list = P.cidx + ((size_t)bh * npairs + pair) * P.ccap;
@@ -400,7 +405,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                     const __nv_bfloat16* row = src + (int64_t)max(j, 0) * row_stride;
                     uint8_t* d = dst + q * 512 + ((q & 1) ? sw1 : sw0);          // row r = 4q + rsub, chunk c ^ (r & 7)
                     cp_async16(d, row, j >= 0 ? 16 : 0);
-                    cp_async16(d + kTileBytes / 2, row + 64, j >= 0 ? 16 : 0);
+                    if constexpr (kD == 128) cp_async16(d + kTileBytes / 2, row + 64, j >= 0 ? 16 : 0);
                 }
                 cp_async_arrive(full);
                 if (it + 1 < n_iters) {
@@ -504,9 +509,9 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
         } else if (warp == kWarpProducer) {
             // =========================================== producer ===========================================
             if (lane == 0) {
-                mbar_arrive_expect_tx(&S.q_full, has1 ? 2 * kTileBytes : kTileBytes);
+                mbar_arrive_expect_tx(&S.q_full, has1 ? 2 * kLoadBytes : kLoadBytes);
                 for (int w = 0; w < (has1 ? 2 : 1); ++w)
-                    for (int hf = 0; hf < 2; ++hf)
+                    for (int hf = 0; hf < kHalves; ++hf)
                         tma_load_4d(&S.q[w][hf * (kTileBytes / 2)], &tmQ, &S.q_full, hf * 64, (qt0 + w) * 128, h, b);
             }
             // K and V of a stage are released separately (K once its S = Q K^T products are done, V after P V), so
@@ -517,16 +522,16 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                 if (it >= kStages) ok = mbar_wait_warp(&S.k_empty[st], ((it / kStages) - 1) & 1, abort_flag);
                 if (!ok) break;
                 if (lane == 0) {
-                    mbar_arrive_expect_tx(&S.k_full[st], kTileBytes);
+                    mbar_arrive_expect_tx(&S.k_full[st], kLoadBytes);
                     tma_load_4d(&S.k[st][0], &tmK, &S.k_full[st], 0, j0, hk, b);
-                    tma_load_4d(&S.k[st][kTileBytes / 2], &tmK, &S.k_full[st], 64, j0, hk, b);
+                    if constexpr (kD == 128) tma_load_4d(&S.k[st][kTileBytes / 2], &tmK, &S.k_full[st], 64, j0, hk, b);
                 }
                 if (it >= kStages) ok = mbar_wait_warp(&S.v_empty[st], ((it / kStages) - 1) & 1, abort_flag);
                 if (!ok) break;
                 if (lane == 0) {
-                    mbar_arrive_expect_tx(&S.v_full[st], kTileBytes);
+                    mbar_arrive_expect_tx(&S.v_full[st], kLoadBytes);
                     tma_load_4d(&S.v[st][0], &tmV, &S.v_full[st], 0, j0, hk, b);
-                    tma_load_4d(&S.v[st][kTileBytes / 2], &tmV, &S.v_full[st], 64, j0, hk, b);
+                    if constexpr (kD == 128) tma_load_4d(&S.v[st][kTileBytes / 2], &tmV, &S.v_full[st], 64, j0, hk, b);
                 }
             }
             // tail: the last stages' release arrivals must land before the CTA's shared memory is given up
@@ -677,7 +682,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             // The whole warp walks the schedule with warp-uniform values (descriptors, stage and tile indices stay in
             // the uniform datapath); one elected lane issues the tcgen05 instructions.
             constexpr uint32_t idesc_s = idesc_bf16(128, 128, 0, 0);     // Q (K-major) x K (K-major)
-            constexpr uint32_t idesc_pv = idesc_bf16(128, 128, 0, 1);    // P (TMEM)    x V (MN-major)
+            constexpr uint32_t idesc_pv = idesc_bf16(128, kD, 0, 1);     // P (TMEM)    x V (MN-major)
             // operand descriptors are formed once; a stage, query tile or k-step only moves the 16-byte address field
             const uint64_t dQ0 = smem_desc_sw128(smem_u32(S.q[0]), 16, 1024), dK0 = smem_desc_sw128(smem_u32(S.k[0]), 16, 1024);
             const uint64_t dV0 = smem_desc_sw128(smem_u32(S.v[0]), kTileBytes / 2, 1024);
@@ -696,7 +701,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                 const uint32_t d_tmem = tmem_u + w * 128;
                 if (elect_one()) {
 #pragma unroll
-                    for (int kk = 0; kk < 8; ++kk) {
+                    for (int kk = 0; kk < kD / 16; ++kk) {
                         const uint32_t off = ((kk >> 2) * (kTileBytes / 2) + (kk & 3) * 32) >> 4;
                         mma_ss(d_tmem, dq + off, dk + off, idesc_s, kk > 0);
                     }
@@ -841,19 +846,6 @@ int make_tmap_bf16(CUtensorMap* m, const void* base, int B, int L, int H, int d,
     return r == CUDA_SUCCESS ? DMA_OK : DMA_ERR_CUDA;
 }
 
-int make_tmap_f32_rows(CUtensorMap* m, const void* base, int B, int L, int H, int rows, int channels) {
-    EncodeTiledFn enc = get_encode_tiled();
-    if (!enc) return DMA_ERR_CUDA;
-    cuuint64_t dims[4] = {128, (cuuint64_t)H, (cuuint64_t)L, (cuuint64_t)B};
-    cuuint64_t str[3] = {128 * 4, (cuuint64_t)H * 128 * 4, (cuuint64_t)L * H * 128 * 4};
-    cuuint32_t box[4] = {(cuuint32_t)channels, 1, (cuuint32_t)rows, 1};
-    cuuint32_t estr[4] = {1, 1, 1, 1};
-    CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, const_cast<void*>(base), dims, str, box, estr,
-                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
-                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    return r == CUDA_SUCCESS ? DMA_OK : DMA_ERR_CUDA;
-}
-
 // Token-compacted mode, per (batch, head, pair of query tiles): the ascending list of keys j that some row i of the
 // pair's 256 rows keeps, i.e. j <= i < expiry[j] for some i in [i0, i0 + 255]  <=>  j <= i0 + 255 and expiry[j] > max(i0, j).
 // At most w + 256 keys qualify. One CTA of 256 threads per list: 256 keys per pass, ballots and per-warp counts keep the
@@ -939,8 +931,10 @@ int launch_tc_fwd(const Prob& P, const void* Q, const void* K, const void* V, co
     dim3 grid(P.B * P.Hq, npairs);
     timing_mark(0, false, st);
     const bool block_skip = (P.flags & DMA_FLAG_BLOCK_SKIP) != 0;
-    auto kern = compact ? (block_skip ? fwd_kernel<true, true> : fwd_kernel<true, false>)
-                        : (block_skip ? fwd_kernel<false, true> : fwd_kernel<false, false>);
+    auto kern = P.d == 128 ? (compact ? (block_skip ? fwd_kernel<true, true, 128> : fwd_kernel<true, false, 128>)
+                                      : (block_skip ? fwd_kernel<false, true, 128> : fwd_kernel<false, false, 128>))
+                           : (compact ? (block_skip ? fwd_kernel<true, true, 64> : fwd_kernel<true, false, 64>)
+                                      : (block_skip ? fwd_kernel<false, true, 64> : fwd_kernel<false, false, 64>));
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return DMA_ERR_CUDA;
     kern<<<grid, kThreads, smem, st>>>(tmQ, tmK, tmV, fp);
     timing_mark(0, true, st);

@@ -5,10 +5,15 @@
 // Kernels
 //   delta_kernel        V read once (HBM-bound); z, softplus, exp in a fixed fp32 operation order
 //   chunk_sort_kernel   256-key chunks of (delta bits, ~index) keys sorted in shared memory
-//   expiry_kernel       per key: the index of the w-th key (in index order) that beats it, by counting beaters
-//                       chunk by chunk with a binary search in each sorted chunk
+//   tree_merge_kernel, expiry_tree_kernel
+//                       selection as a rank tree: the merge passes that finish the sort leave one bit per key and level,
+//                       and a key's expiry (the w-th smallest index among the keys that beat it) is a walk of log2(L) steps
+//   rank_perm_kernel, expiry_kernel
+//                       the chunk-walking selection (packed sequences; the entry point with static scratch): per key, beaters
+//                       are counted chunk by chunk with a binary search in each sorted chunk
 //   bitmap_kernel       per key tile: union of the query-tile intervals its keys are kept in
 #include <mutex>
+#include <utility>
 #include <type_traits>
 
 #include "common.cuh"
@@ -299,23 +304,249 @@ __device__ __forceinline__ unsigned long long sort_key(float dl, int j) {
     return ((unsigned long long)__float_as_uint(dl) << 32) | (unsigned long long)(0xFFFFFFFFu - (unsigned)j);
 }
 
+// lev == nullptr: chunks written in ascending order (the chunk-walking expiry kernel). Otherwise (rank-tree selection,
+// see tree_merge_kernel): chunks written in DESCENDING order, padding keys carry their index, and the kernel also emits
+// the eight lowest levels of the tree (node sizes 256 ... 2) by splitting the sorted chunk on one index bit per level.
 __global__ void __launch_bounds__(kChunk) chunk_sort_kernel(const float* __restrict__ delta,
-                                                            unsigned long long* __restrict__ sorted, int L, int nchunk) {
-    __shared__ unsigned long long s[kChunk];
+                                                            unsigned long long* __restrict__ sorted, int L, int nchunk,
+                                                            uint2* __restrict__ lev, int m) {
+    __shared__ unsigned long long s[2][kChunk];
     const int bh = blockIdx.y, c = blockIdx.x, t = threadIdx.x, j = c * kChunk + t;
-    s[t] = j < L ? sort_key(delta[(size_t)bh * L + j], j) : 0ull;   // padding sorts below every real key
-    __syncthreads();
-    for (int k = 2; k <= kChunk; k <<= 1)
-        for (int m = k >> 1; m > 0; m >>= 1) {
-            int o = t ^ m;
-            if (o > t) {
-                unsigned long long a = s[t], b = s[o];
-                bool up = (t & k) == 0;
-                if ((a > b) == up) { s[t] = b; s[o] = a; }
+    // padding sorts below every real key (delta > 0); in the rank-tree form it keeps its index in the low word
+    unsigned long long v = j < L ? sort_key(delta[(size_t)bh * L + j], j) : (lev ? (unsigned long long)(0xFFFFFFFFu - (unsigned)j) : 0ull);
+    // bitonic network, ascending; thread t holds position t. Partners less than 32 apart exchange by shuffle, the six
+    // wider exchanges go through shared memory (two buffers in turn: one barrier each).
+    int nb = 0;
+#pragma unroll
+    for (int k = 2; k <= kChunk; k <<= 1) {
+        const bool up = (t & k) == 0;
+#pragma unroll
+        for (int mm = k >> 1; mm > 0; mm >>= 1) {
+            unsigned long long o;
+            if (mm >= 32) {
+                s[nb][t] = v;
+                __syncthreads();
+                o = s[nb][t ^ mm];
+                nb ^= 1;
+            } else {
+                o = __shfl_xor_sync(0xffffffffu, v, mm);
             }
-            __syncthreads();
+            const bool want_min = ((t & mm) == 0) == up;
+            v = want_min ? (v < o ? v : o) : (v > o ? v : o);
         }
-    sorted[((size_t)bh * nchunk + c) * kChunk + t] = s[t];   // ascending
+    }
+    if (!lev) {
+        sorted[((size_t)bh * nchunk + c) * kChunk + t] = v;      // ascending
+        return;
+    }
+    s[0][t] = v;
+    __syncthreads();
+    const unsigned long long mine = s[0][kChunk - 1 - t];        // position t of the descending order
+    sorted[((size_t)bh * nchunk + c) * kChunk + t] = mine;
+    // Levels with node size Bs = 256, 128, ..., 2: a node is an aligned block of Bs key indices, its sequence the block's
+    // keys in descending order, its bit the half of the block a key lies in. Splitting a node's sequence stably on that
+    // bit gives the sequences of its two children.
+    __shared__ uint8_t cur[2][kChunk];
+    __shared__ uint32_t wbits[kChunk / 32];
+    const int lane = t & 31, warp = t >> 5;
+    const size_t W = (size_t)nchunk * (kChunk / 32);
+    cur[0][t] = (uint8_t)((0xFFFFFFFFu - (uint32_t)mine) & (kChunk - 1));
+    __syncthreads();
+#pragma unroll
+    for (int lv = 0; lv < 8; ++lv) {
+        const int Bs = kChunk >> lv, v = cur[lv & 1][t], bit = (v >> (7 - lv)) & 1;
+        const uint32_t bal = __ballot_sync(0xffffffffu, bit);
+        if (lane == 0) wbits[warp] = bal;
+        __syncthreads();
+        const int node_start = t & ~(Bs - 1);
+        uint32_t cumw = 0;                                      // ones of the node before this word
+        for (int k = node_start >> 5; k < warp; ++k) cumw += __popc(wbits[k]);
+        const uint32_t below = (1u << lane) - 1u, in_node = Bs >= 32 ? 0xffffffffu : (((1u << Bs) - 1u) << (node_start & 31));
+        const int ones_before = (int)cumw + __popc(bal & below & in_node);
+        if (lane == 0) lev[((size_t)bh * m + (m - 8 + lv)) * W + (size_t)c * (kChunk / 32) + warp] = make_uint2(cumw, bal);
+        const int npos = node_start + (bit ? Bs / 2 + ones_before : (t - node_start) - ones_before);
+        cur[(lv + 1) & 1][npos] = (uint8_t)v;
+        __syncthreads();
+    }
+}
+
+// ---- selection as a rank tree -------------------------------------------------------------------------------
+// expiry[j] is the w-th smallest INDEX among the keys that beat j, i.e. among the first r entries of the head's keys in
+// descending order, r = rank of j. That is a quantile query on a prefix, answered by a tree over key indices: the node of an
+// aligned block of 2^k indices stores, for the block's keys in descending order, one bit per key (lower / upper half of
+// the block) with running counts. A query walks from the root to a leaf: with c = how many of the first r keys lie in the
+// node and z of them in its lower half, the k-th smallest index is in the lower half iff k <= z. log2(L) steps of one
+// 8-byte load each, for every key in parallel, whatever w.
+// The tree is what a bottom-up merge sort leaves behind: merging the sorted lower and upper half of a block yields the
+// block's sorted sequence, and "this output came from the upper half" is the node's bit. chunk_sort_kernel builds the
+// levels up to 256 keys; one tree_merge_kernel launch per level does the rest (runs of R keys -> runs of 2R).
+// Level l (0 = root) of head bh lives at lev[(bh * m + l) * W + position / 32]: x = ones of the node before this word,
+// y = the bits. A trailing run shorter than R (L is not a power of two) merges with what exists; the nodes stay
+// left-aligned, which is all a query needs (it never looks past the real keys).
+constexpr int kMergeThreads = 256;
+constexpr int kBlockKeys = 4096;      // keys one CTA of tree_block_kernel merges in shared memory
+constexpr int kBlockThreads = 1024;
+
+// Levels with nodes of 512 ... 4096 keys in one launch: a CTA holds 4096 keys (16 sorted chunks) in shared memory and
+// merges runs of R = 256, 512, 1024, 2048. Every key finds its place by rank: its position in its own run plus the
+// number of keys of the sibling run that go before it (a binary search in the sibling run). A node's bit is the bit
+// log2(R) of the key's index (upper or lower half of the block of 2R indices), read off the merged sequence.
+__global__ void __launch_bounds__(kBlockThreads) tree_block_kernel(const unsigned long long* __restrict__ src,
+                                                                   unsigned long long* __restrict__ dst,
+                                                                   uint2* __restrict__ lev, int Lc, int m) {
+    extern __shared__ __align__(16) unsigned long long sk[];         // two buffers of kBlockKeys keys
+    __shared__ uint32_t wpop[kBlockKeys / 32], wexcl[kBlockKeys / 32];
+    const int bh = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int base = blockIdx.x * kBlockKeys, nreal = min(kBlockKeys, Lc - base);
+    const size_t Wl = (size_t)Lc / 32;
+    unsigned long long* cur = sk;
+    unsigned long long* nxt = sk + kBlockKeys;
+#pragma unroll
+    for (int k = 0; k < kBlockKeys / kBlockThreads; ++k) {
+        const int i = tid + k * kBlockThreads;
+        cur[i] = i < nreal ? src[(size_t)bh * Lc + base + i] : 0ull;
+    }
+    __syncthreads();
+    int l = m - 9;
+    for (int R = kChunk, sh = 8; R < kBlockKeys && R < Lc; R *= 2, ++sh, --l) {
+#pragma unroll
+        for (int k = 0; k < kBlockKeys / kBlockThreads; ++k) {
+            const int i = tid + k * kBlockThreads;
+            if (i < nreal) {
+                const unsigned long long key = cur[i];
+                const int pair = i & ~(2 * R - 1), own = i & (R - 1);
+                const int sib = pair + ((i & R) ? 0 : R);
+                const unsigned long long* sv = cur + sib;
+                int lo = 0, hi = max(0, min(R, nreal - sib));    // keys of the sibling run that go before this one
+                while (lo < hi) {
+                    const int mid = (lo + hi) >> 1;
+                    if (sv[mid] > key) lo = mid + 1; else hi = mid;
+                }
+                nxt[pair + own + lo] = key;
+            }
+        }
+        __syncthreads();
+        // bits and running counts of the merged nodes
+        uint32_t bal[kBlockKeys / kBlockThreads];
+#pragma unroll
+        for (int k = 0; k < kBlockKeys / kBlockThreads; ++k) {
+            const int i = tid + k * kBlockThreads;
+            const bool bit = i < nreal && (((0xFFFFFFFFu - (uint32_t)nxt[i]) >> sh) & 1u);
+            bal[k] = __ballot_sync(0xffffffffu, bit);
+            if (lane == 0) wpop[k * 32 + warp] = __popc(bal[k]);
+        }
+        __syncthreads();
+        if (warp == 0) {                                         // exclusive scan over the 128 words
+            uint32_t a[4], run = 0;
+#pragma unroll
+            for (int u = 0; u < 4; ++u) { a[u] = wpop[lane * 4 + u]; run += a[u]; }
+            uint32_t incl = run;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const uint32_t y = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += y;
+            }
+            uint32_t ex = incl - run;
+#pragma unroll
+            for (int u = 0; u < 4; ++u) { wexcl[lane * 4 + u] = ex; ex += a[u]; }
+        }
+        __syncthreads();
+        if (lane == 0) {
+#pragma unroll
+            for (int k = 0; k < kBlockKeys / kBlockThreads; ++k) {
+                const int wi = k * 32 + warp;                    // word of this block
+                if (wi * 32 < nreal) {
+                    const int node_first = (wi * 32 & ~(2 * R - 1)) >> 5;
+                    lev[((size_t)bh * m + l) * Wl + (size_t)(base >> 5) + wi] = make_uint2(wexcl[wi] - wexcl[node_first], bal[k]);
+                }
+            }
+        }
+        unsigned long long* tmp = cur; cur = nxt; nxt = tmp;
+        __syncthreads();
+    }
+#pragma unroll
+    for (int k = 0; k < kBlockKeys / kBlockThreads; ++k) {
+        const int i = tid + k * kBlockThreads;
+        if (i < nreal) dst[(size_t)bh * Lc + base + i] = cur[i];
+    }
+}
+
+__global__ void __launch_bounds__(kMergeThreads) tree_merge_kernel(const unsigned long long* __restrict__ src,
+                                                                   unsigned long long* __restrict__ dst,
+                                                                   uint2* __restrict__ lev_l, int Lc, int R, int m) {
+    __shared__ unsigned long long sA[kMergeThreads], sB[kMergeThreads];
+    __shared__ int s_a0;
+    const int bh = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int o0 = blockIdx.x * kMergeThreads;                   // first output position of this CTA within the head
+    const int base = o0 & ~(2 * R - 1), t0 = o0 - base;
+    const int na = min(R, Lc - base), nb = max(0, min(R, Lc - base - R));
+    const unsigned long long* A = src + (size_t)bh * Lc + base;
+    const unsigned long long* Bv = A + R;
+    // a0 = how many of the first t0 outputs of the pair come from A: the first i for which "A[i] goes before the last B
+    // taken" fails. 32 probes per round, each round cuts the interval 32-fold.
+    if (warp == 0) {
+        int lo = max(0, t0 - nb), hi = min(t0, na);
+        while (lo < hi) {
+            const int len = hi - lo, stride = (len + 31) / 32;
+            const int i = lo + lane * stride;
+            const bool pr = i < hi && A[i] > Bv[t0 - i - 1];      // (i < hi implies i < na and t0 - i > 0)
+            const int cnt = __popc(__ballot_sync(0xffffffffu, pr));
+            if (cnt == 0) { hi = lo; break; }
+            const int last_true = lo + (cnt - 1) * stride;
+            lo = last_true + 1;
+            hi = min(hi, last_true + stride);
+        }
+        if (lane == 0) s_a0 = lo;
+    }
+    __syncthreads();
+    const int a0 = s_a0, b0 = t0 - a0;
+    const int la = min(kMergeThreads, na - a0), lb = min(kMergeThreads, nb - b0);
+    sA[tid] = tid < la ? A[a0 + tid] : 0ull;
+    sB[tid] = tid < lb ? Bv[b0 + tid] : 0ull;
+    __syncthreads();
+    const int x = tid;
+    const bool exists = t0 + x < na + nb;
+    int lo = max(0, x - lb), hi = min(x, la);
+    while (lo < hi) {
+        const int mid = (lo + hi) >> 1;
+        if (sA[mid] > sB[x - mid - 1]) lo = mid + 1; else hi = mid;
+    }
+    const int i = lo;                                            // outputs before x that come from A
+    const bool takeA = i < la && (x - i >= lb || sA[i] > sB[x - i]);
+    if (exists) dst[(size_t)bh * Lc + o0 + x] = takeA ? sA[i] : sB[x - i];
+    const uint32_t bal = __ballot_sync(0xffffffffu, exists && !takeA);
+    if (lane == 0 && exists) lev_l[(size_t)bh * m * (Lc / 32) + (o0 + x) / 32] = make_uint2((uint32_t)(b0 + x - i), bal);
+}
+
+// One thread per rank r of a head: the key at rank r, the walk down the tree, expiry[j] = max(j, index found).
+// kAllRows (non-causal): every row sees every key, so the key is kept by all rows iff fewer than w keys beat it.
+template <bool kAllRows>
+__global__ void __launch_bounds__(256) expiry_tree_kernel(const unsigned long long* __restrict__ sorted, const uint2* __restrict__ lev,
+                                                          int32_t* __restrict__ expiry, int L, int Lc, int w, int m) {
+    const int r = blockIdx.x * 256 + threadIdx.x, bh = blockIdx.y;
+    if (r >= L) return;                                          // ranks from L on are padding
+    const int j = (int)(0xFFFFFFFFu - (uint32_t)sorted[(size_t)bh * Lc + r]);
+    int e;
+    if (r < w) {
+        e = L;                                                   // fewer than w keys beat it: never dropped
+    } else if (kAllRows) {
+        e = 0;
+    } else {
+        const size_t W = (size_t)Lc / 32;
+        const uint2* lv = lev + (size_t)bh * m * W;
+        int k = w, c = r, s = 0;                                 // k-th smallest among the first c entries of the node starting at s
+        for (int l = 0; l < m; ++l, lv += W) {
+            const int half = 1 << (m - 1 - l);
+            const int q = s + c - 1;                             // last entry of the prefix (c >= k >= 1)
+            const uint2 wd = lv[q >> 5];
+            const uint32_t upto = (2u << (q & 31)) - 1u, from = ~((1u << (s & 31)) - 1u);     // a node smaller than a word starts inside it
+            const int ones = (int)wd.x + __popc(wd.y & upto & from);
+            const int zeros = c - ones;
+            if (k <= zeros) c = zeros; else { k -= zeros; c = ones; s += half; }
+        }
+        e = max(j, s);
+    }
+    expiry[(size_t)bh * L + j] = e;
 }
 
 // Work assignment of the expiry kernel. A key's walk over the sorted chunks ends once w keys have beaten it, after
@@ -548,10 +779,19 @@ __global__ void __launch_bounds__(128) bitmap_kernel(const int32_t* __restrict__
 
 constexpr int kStaticChunk = kChunk;
 
-// workspace: header | sorted chunks (8 bytes per padded key) | rank permutation (4 bytes per padded key)
+// levels of the rank tree over a head of Lc (a multiple of 256) keys: the smallest m with 2^m >= Lc
+static int tree_levels(int Lc) {
+    int m = 8;
+    while ((1ll << m) < Lc) ++m;
+    return m;
+}
+
+// workspace: header | two buffers of sort keys (8 bytes per padded key each: the merge passes alternate between them) |
+// the rank tree (m levels of 8 bytes per 32 padded keys). The chunk-walking selection (packed sequences, and the
+// entry point with static scratch) uses the first 12 bytes per padded key of the same region: sorted chunks | rank permutation.
 size_t mask_ws_bytes(const Prob& P) {
-    const size_t nchunk = (P.L + kChunk - 1) / kChunk;
-    return kWsHeaderBytes + (size_t)P.B * P.Hq * nchunk * kChunk * (sizeof(unsigned long long) + sizeof(uint32_t));
+    const size_t nchunk = (P.L + kChunk - 1) / kChunk, keys = (size_t)P.B * P.Hq * nchunk * kChunk;
+    return kWsHeaderBytes + keys * 2 * sizeof(unsigned long long) + keys / 32 * tree_levels((int)(nchunk * kChunk)) * sizeof(uint2);
 }
 
 template <typename T, int D>
@@ -607,7 +847,7 @@ static int mask_build_limits(const Prob& P) {
 }
 
 int launch_mask_build(const Prob& P, const void* V, const float* W, const float* A, float* bias, int32_t* expiry,
-                      uint32_t* bitmap, void* ws, cudaStream_t st, const int32_t* cu, int nseq) {
+                      uint32_t* bitmap, void* ws, cudaStream_t st, const int32_t* cu, int nseq, bool small_scratch) {
     int rc;
     if ((rc = mask_build_limits(P))) return rc;          // an error return means that no kernel has been launched
     if (P.dtype == DMA_BF16)
@@ -623,10 +863,35 @@ int launch_mask_build(const Prob& P, const void* V, const float* W, const float*
         size_t n = (size_t)BH * P.L;
         fill_i32_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(expiry, n, P.L);
         count_launch();
+    } else if (!cu && !small_scratch) {
+        // rank tree: sorted chunks and the low levels, one merge pass per further level, then one walk per key
+        const int Lc = nchunk * kChunk, m = tree_levels(Lc);
+        const size_t keys = (size_t)BH * Lc, Wl = (size_t)Lc / 32;
+        auto* buf0 = reinterpret_cast<unsigned long long*>((char*)ws + kWsHeaderBytes);
+        auto* buf1 = buf0 + keys;
+        uint2* lev = reinterpret_cast<uint2*>(buf1 + keys);
+        chunk_sort_kernel<<<dim3(nchunk, BH), kChunk, 0, st>>>(bias, buf0, P.L, nchunk, lev, m);
+        int launches = 2;
+        if (Lc > kChunk) {
+            const size_t smem = 2 * (size_t)kBlockKeys * sizeof(unsigned long long);
+            if (cudaFuncSetAttribute(tree_block_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return DMA_ERR_CUDA;
+            tree_block_kernel<<<dim3((Lc + kBlockKeys - 1) / kBlockKeys, BH), kBlockThreads, smem, st>>>(buf0, buf1, lev, Lc, m);
+            std::swap(buf0, buf1);
+            ++launches;
+        }
+        int l = m - 13;                                          // level of the nodes of 2 * kBlockKeys keys
+        for (int R = kBlockKeys; R < Lc; R *= 2, --l, ++launches) {
+            tree_merge_kernel<<<dim3(Lc / kMergeThreads, BH), kMergeThreads, 0, st>>>(buf0, buf1, lev + (size_t)l * Wl, Lc, R, m);
+            std::swap(buf0, buf1);
+        }
+        const dim3 grid((P.L + 255) / 256, BH);
+        if (P.causal) expiry_tree_kernel<false><<<grid, 256, 0, st>>>(buf0, lev, expiry, P.L, Lc, P.w, m);
+        else expiry_tree_kernel<true><<<grid, 256, 0, st>>>(buf0, lev, expiry, P.L, Lc, P.w, m);
+        count_launch(launches);
     } else {
         auto* sorted = reinterpret_cast<unsigned long long*>((char*)ws + kWsHeaderBytes);
         uint32_t* perm = reinterpret_cast<uint32_t*>(sorted + (size_t)BH * nchunk * kChunk);
-        chunk_sort_kernel<<<dim3(nchunk, BH), kChunk, 0, st>>>(bias, sorted, P.L, nchunk);
+        chunk_sort_kernel<<<dim3(nchunk, BH), kChunk, 0, st>>>(bias, sorted, P.L, nchunk, nullptr, 0);
         if (!cu) rank_perm_kernel<<<BH, 1024, 0, st>>>(bias, perm, P.L, P.w);
         const dim3 grid((P.L + kExpThreads - 1) / kExpThreads, BH);
         if (cu) expiry_kernel<1><<<grid, kExpThreads, 0, st>>>(bias, sorted, expiry, P.L, P.w, nchunk, cu, nseq, nullptr);
@@ -683,5 +948,5 @@ extern "C" int dma_mask_build_static(const dma_problem_t* p, const void* V, cons
         }
         scratch = g_static_ptr[dev];
     }
-    return dma::launch_mask_build(P, V, W_delta, A, bias, expiry, bitmap, scratch, (cudaStream_t)cuda_stream);
+    return dma::launch_mask_build(P, V, W_delta, A, bias, expiry, bitmap, scratch, (cudaStream_t)cuda_stream, nullptr, 0, true);
 }

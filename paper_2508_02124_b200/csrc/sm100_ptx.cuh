@@ -93,6 +93,13 @@ __device__ __forceinline__ void tma_reduce_add_4d(const CUtensorMap* m, const vo
         ::"l"(reinterpret_cast<uint64_t>(m)), "r"(smem_u32(src)), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
         : "memory");
 }
+// reduce-add of one contiguous block (bytes: a multiple of 16, both addresses 16-byte aligned) from shared memory into
+// global memory; bulk-group tracked
+__device__ __forceinline__ void bulk_reduce_add_f32(float* dst, const void* src, uint32_t bytes) {
+    asm volatile("cp.reduce.async.bulk.global.shared::cta.bulk_group.add.f32 [%0], [%1], %2;"
+                 ::"l"(dst), "r"(smem_u32(src)), "r"(bytes)
+                 : "memory");
+}
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_read_all() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 // at most one bulk group of this thread may still be reading its shared-memory source
@@ -309,8 +316,5 @@ EncodeTiledFn get_encode_tiled();
 // 128-byte swizzle, out-of-range rows read as zero. Coordinates: (channel, seq, head, batch).
 int make_tmap_bf16(CUtensorMap* m, const void* base, int B, int L, int H, int d, const int64_t strides[3], int rows);
 
-// fp32 tensor [B, L, H, 128] contiguous: box = 128 channels x `rows` sequence positions of one head, no swizzle.
-// Coordinates: (channel, head, seq, batch). Used as the destination of the dQ reduce-add.
-int make_tmap_f32_rows(CUtensorMap* m, const void* base, int B, int L, int H, int rows, int channels = 128);
 
 }  // namespace dma
