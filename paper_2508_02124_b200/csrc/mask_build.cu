@@ -384,19 +384,50 @@ __global__ void __launch_bounds__(kChunk) chunk_sort_kernel(const float* __restr
 // y = the bits. A trailing run shorter than R (L is not a power of two) merges with what exists; the nodes stay
 // left-aligned, which is all a query needs (it never looks past the real keys).
 constexpr int kMergeThreads = 256;
+constexpr int kMergeOut = 1024;       // outputs per CTA of tree_merge_kernel (four per thread)
 constexpr int kBlockKeys = 4096;      // keys one CTA of tree_block_kernel merges in shared memory
 constexpr int kBlockThreads = 1024;
 
+// Four consecutive outputs of the merge of two descending runs A (na keys) and B (nb keys), starting at output x:
+// i = how many of the first x outputs come from A (the first i for which "A[i] goes before the last B taken" fails), then
+// four merge steps. Keys are distinct and non-zero; 0 stands for "run exhausted". Returns i; prov bit u = output u came from B.
+__device__ __forceinline__ int merge4(const unsigned long long* A, int na, const unsigned long long* B, int nb, int x,
+                                      unsigned long long (&out)[4], uint32_t& prov) {
+    int lo = max(0, x - nb), hi = min(x, na);
+    while (lo < hi) {
+        const int mid = (lo + hi) >> 1;
+        if (A[mid] > B[x - mid - 1]) lo = mid + 1; else hi = mid;
+    }
+    int i = lo, k = x - lo;
+    unsigned long long a = i < na ? A[i] : 0ull, b = k < nb ? B[k] : 0ull;
+    prov = 0u;
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+        const bool takeA = a > b;
+        out[u] = takeA ? a : b;
+        prov |= takeA ? 0u : 1u << u;
+        if (takeA) { ++i; a = i < na ? A[i] : 0ull; } else { ++k; b = k < nb ? B[k] : 0ull; }
+    }
+    return lo;
+}
+
+// the 32-bit word of eight neighbouring threads' four provenance bits each (valid in the lanes with lane % 8 == 0)
+__device__ __forceinline__ uint32_t gather_nibbles(uint32_t prov, int lane) {
+    uint32_t wv = prov << (4 * (lane & 7));
+    wv |= __shfl_xor_sync(0xffffffffu, wv, 1);
+    wv |= __shfl_xor_sync(0xffffffffu, wv, 2);
+    wv |= __shfl_xor_sync(0xffffffffu, wv, 4);
+    return wv;
+}
+
 // Levels with nodes of 512 ... 4096 keys in one launch: a CTA holds 4096 keys (16 sorted chunks) in shared memory and
-// merges runs of R = 256, 512, 1024, 2048. Every key finds its place by rank: its position in its own run plus the
-// number of keys of the sibling run that go before it (a binary search in the sibling run). A node's bit is the bit
-// log2(R) of the key's index (upper or lower half of the block of 2R indices), read off the merged sequence.
+// merges runs of R = 256, 512, 1024, 2048, four consecutive outputs per thread. A node's bit says whether the output came
+// from the upper run, and the count of such outputs before a word is the word's position minus the A keys taken so far.
 __global__ void __launch_bounds__(kBlockThreads) tree_block_kernel(const unsigned long long* __restrict__ src,
                                                                    unsigned long long* __restrict__ dst,
                                                                    uint2* __restrict__ lev, int Lc, int m) {
     extern __shared__ __align__(16) unsigned long long sk[];         // two buffers of kBlockKeys keys
-    __shared__ uint32_t wpop[kBlockKeys / 32], wexcl[kBlockKeys / 32];
-    const int bh = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int bh = blockIdx.y, tid = threadIdx.x, lane = tid & 31;
     const int base = blockIdx.x * kBlockKeys, nreal = min(kBlockKeys, Lc - base);
     const size_t Wl = (size_t)Lc / 32;
     unsigned long long* cur = sk;
@@ -407,60 +438,21 @@ __global__ void __launch_bounds__(kBlockThreads) tree_block_kernel(const unsigne
         cur[i] = i < nreal ? src[(size_t)bh * Lc + base + i] : 0ull;
     }
     __syncthreads();
+    const int o = 4 * tid;                                       // this thread's outputs: o .. o + 3 of the block
     int l = m - 9;
-    for (int R = kChunk, sh = 8; R < kBlockKeys && R < Lc; R *= 2, ++sh, --l) {
-#pragma unroll
-        for (int k = 0; k < kBlockKeys / kBlockThreads; ++k) {
-            const int i = tid + k * kBlockThreads;
-            if (i < nreal) {
-                const unsigned long long key = cur[i];
-                const int pair = i & ~(2 * R - 1), own = i & (R - 1);
-                const int sib = pair + ((i & R) ? 0 : R);
-                const unsigned long long* sv = cur + sib;
-                int lo = 0, hi = max(0, min(R, nreal - sib));    // keys of the sibling run that go before this one
-                while (lo < hi) {
-                    const int mid = (lo + hi) >> 1;
-                    if (sv[mid] > key) lo = mid + 1; else hi = mid;
-                }
-                nxt[pair + own + lo] = key;
-            }
+    for (int R = kChunk; R < kBlockKeys && R < Lc; R *= 2, --l) {
+        const int pair = o & ~(2 * R - 1), x = o - pair;
+        const int na = max(0, min(R, nreal - pair)), nb = max(0, min(R, nreal - pair - R));
+        unsigned long long out[4];
+        uint32_t prov;
+        const int i0 = merge4(cur + pair, na, cur + pair + R, nb, x, out, prov);
+        const bool exists = o < nreal;                           // (runs are whole chunks: all four outputs exist or none)
+        if (exists) {
+            *reinterpret_cast<ulonglong2*>(nxt + o) = make_ulonglong2(out[0], out[1]);
+            *reinterpret_cast<ulonglong2*>(nxt + o + 2) = make_ulonglong2(out[2], out[3]);
         }
-        __syncthreads();
-        // bits and running counts of the merged nodes
-        uint32_t bal[kBlockKeys / kBlockThreads];
-#pragma unroll
-        for (int k = 0; k < kBlockKeys / kBlockThreads; ++k) {
-            const int i = tid + k * kBlockThreads;
-            const bool bit = i < nreal && (((0xFFFFFFFFu - (uint32_t)nxt[i]) >> sh) & 1u);
-            bal[k] = __ballot_sync(0xffffffffu, bit);
-            if (lane == 0) wpop[k * 32 + warp] = __popc(bal[k]);
-        }
-        __syncthreads();
-        if (warp == 0) {                                         // exclusive scan over the 128 words
-            uint32_t a[4], run = 0;
-#pragma unroll
-            for (int u = 0; u < 4; ++u) { a[u] = wpop[lane * 4 + u]; run += a[u]; }
-            uint32_t incl = run;
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const uint32_t y = __shfl_up_sync(0xffffffffu, incl, o);
-                if (lane >= o) incl += y;
-            }
-            uint32_t ex = incl - run;
-#pragma unroll
-            for (int u = 0; u < 4; ++u) { wexcl[lane * 4 + u] = ex; ex += a[u]; }
-        }
-        __syncthreads();
-        if (lane == 0) {
-#pragma unroll
-            for (int k = 0; k < kBlockKeys / kBlockThreads; ++k) {
-                const int wi = k * 32 + warp;                    // word of this block
-                if (wi * 32 < nreal) {
-                    const int node_first = (wi * 32 & ~(2 * R - 1)) >> 5;
-                    lev[((size_t)bh * m + l) * Wl + (size_t)(base >> 5) + wi] = make_uint2(wexcl[wi] - wexcl[node_first], bal[k]);
-                }
-            }
-        }
+        const uint32_t wv = gather_nibbles(exists ? prov : 0u, lane);
+        if ((lane & 7) == 0 && exists) lev[((size_t)bh * m + l) * Wl + (size_t)((base + o) >> 5)] = make_uint2((uint32_t)(x - i0), wv);
         unsigned long long* tmp = cur; cur = nxt; nxt = tmp;
         __syncthreads();
     }
@@ -471,19 +463,20 @@ __global__ void __launch_bounds__(kBlockThreads) tree_block_kernel(const unsigne
     }
 }
 
+// One level per launch for runs of R >= 4096 keys: a CTA produces 1024 consecutive outputs of one pair of runs. Warp 0
+// finds where they start in the two runs (32 probes per round), the CTA stages up to 1024 keys of each run in shared
+// memory, and every thread merges four outputs from there.
 __global__ void __launch_bounds__(kMergeThreads) tree_merge_kernel(const unsigned long long* __restrict__ src,
                                                                    unsigned long long* __restrict__ dst,
                                                                    uint2* __restrict__ lev_l, int Lc, int R, int m) {
-    __shared__ unsigned long long sA[kMergeThreads], sB[kMergeThreads];
+    __shared__ __align__(16) unsigned long long sA[kMergeOut], sB[kMergeOut];
     __shared__ int s_a0;
     const int bh = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int o0 = blockIdx.x * kMergeThreads;                   // first output position of this CTA within the head
+    const int o0 = blockIdx.x * kMergeOut;                       // first output position of this CTA within the head
     const int base = o0 & ~(2 * R - 1), t0 = o0 - base;
     const int na = min(R, Lc - base), nb = max(0, min(R, Lc - base - R));
     const unsigned long long* A = src + (size_t)bh * Lc + base;
     const unsigned long long* Bv = A + R;
-    // a0 = how many of the first t0 outputs of the pair come from A: the first i for which "A[i] goes before the last B
-    // taken" fails. 32 probes per round, each round cuts the interval 32-fold.
     if (warp == 0) {
         int lo = max(0, t0 - nb), hi = min(t0, na);
         while (lo < hi) {
@@ -500,22 +493,26 @@ __global__ void __launch_bounds__(kMergeThreads) tree_merge_kernel(const unsigne
     }
     __syncthreads();
     const int a0 = s_a0, b0 = t0 - a0;
-    const int la = min(kMergeThreads, na - a0), lb = min(kMergeThreads, nb - b0);
-    sA[tid] = tid < la ? A[a0 + tid] : 0ull;
-    sB[tid] = tid < lb ? Bv[b0 + tid] : 0ull;
-    __syncthreads();
-    const int x = tid;
-    const bool exists = t0 + x < na + nb;
-    int lo = max(0, x - lb), hi = min(x, la);
-    while (lo < hi) {
-        const int mid = (lo + hi) >> 1;
-        if (sA[mid] > sB[x - mid - 1]) lo = mid + 1; else hi = mid;
+    const int la = min(kMergeOut, na - a0), lb = min(kMergeOut, nb - b0);
+#pragma unroll
+    for (int k = 0; k < kMergeOut / kMergeThreads; ++k) {
+        const int i = tid + k * kMergeThreads;
+        sA[i] = i < la ? A[a0 + i] : 0ull;
+        sB[i] = i < lb ? Bv[b0 + i] : 0ull;
     }
-    const int i = lo;                                            // outputs before x that come from A
-    const bool takeA = i < la && (x - i >= lb || sA[i] > sB[x - i]);
-    if (exists) dst[(size_t)bh * Lc + o0 + x] = takeA ? sA[i] : sB[x - i];
-    const uint32_t bal = __ballot_sync(0xffffffffu, exists && !takeA);
-    if (lane == 0 && exists) lev_l[(size_t)bh * m * (Lc / 32) + (o0 + x) / 32] = make_uint2((uint32_t)(b0 + x - i), bal);
+    __syncthreads();
+    const int x = 4 * tid;
+    const bool exists = t0 + x < na + nb;
+    unsigned long long out[4];
+    uint32_t prov;
+    const int i0 = merge4(sA, la, sB, lb, x, out, prov);
+    if (exists) {
+        unsigned long long* d = dst + (size_t)bh * Lc + o0 + x;
+        *reinterpret_cast<ulonglong2*>(d) = make_ulonglong2(out[0], out[1]);
+        *reinterpret_cast<ulonglong2*>(d + 2) = make_ulonglong2(out[2], out[3]);
+    }
+    const uint32_t wv = gather_nibbles(exists ? prov : 0u, lane);
+    if ((lane & 7) == 0 && exists) lev_l[(size_t)bh * m * (Lc / 32) + ((o0 + x) >> 5)] = make_uint2((uint32_t)(b0 + x - i0), wv);
 }
 
 // One thread per rank r of a head: the key at rank r, the walk down the tree, expiry[j] = max(j, index found).
@@ -766,9 +763,22 @@ __global__ void __launch_bounds__(128) bitmap_kernel(const int32_t* __restrict__
         }
     }
     __syncthreads();
-    if (t == 0) {
-        int run = 0;
-        for (int q = 0; q < Tr; ++q) { run += diff[q]; diff[q] = run > 0; }
+    {   // running sum over the query tiles: each thread owns a contiguous segment, the segment totals are scanned by warp shuffles
+        __shared__ int wtot[4];
+        const int seg = (Tr + 127) / 128, q0 = t * seg, q1 = min(Tr, q0 + seg);
+        int tot = 0;
+        for (int q = q0; q < q1; ++q) tot += diff[q];
+        int incl = tot;
+        const int lane = t & 31, warp = t >> 5;
+        for (int o = 1; o < 32; o <<= 1) {
+            const int y = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += y;
+        }
+        if (lane == 31) wtot[warp] = incl;
+        __syncthreads();
+        int run = incl - tot;
+        for (int k = 0; k < warp; ++k) run += wtot[k];
+        for (int q = q0; q < q1; ++q) { run += diff[q]; diff[q] = run > 0; }
     }
     __syncthreads();
     for (int q = t; q < Tr; q += blockDim.x)
@@ -881,7 +891,7 @@ int launch_mask_build(const Prob& P, const void* V, const float* W, const float*
         }
         int l = m - 13;                                          // level of the nodes of 2 * kBlockKeys keys
         for (int R = kBlockKeys; R < Lc; R *= 2, --l, ++launches) {
-            tree_merge_kernel<<<dim3(Lc / kMergeThreads, BH), kMergeThreads, 0, st>>>(buf0, buf1, lev + (size_t)l * Wl, Lc, R, m);
+            tree_merge_kernel<<<dim3((Lc + kMergeOut - 1) / kMergeOut, BH), kMergeThreads, 0, st>>>(buf0, buf1, lev + (size_t)l * Wl, Lc, R, m);
             std::swap(buf0, buf1);
         }
         const dim3 grid((P.L + 255) / 256, BH);
