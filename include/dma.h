@@ -143,7 +143,7 @@ int dma_mask_build(const dma_problem_t* p, const void* V, const float* W_delta, 
  * at the point where the mask is built: an inference server that has handed all device memory to its own arena
  * and treats any later cudaMalloc as an error, or a plug-in that runs inside another framework's step and has no
  * allocator of its own to ask. This entry point allocates nothing and calls no allocating routine: its scratch is
- * a fixed 12 MiB array inside the library's device image, present on every GPU that loads the library until the
+ * a fixed 21 MiB array inside the library's device image, present on every GPU that loads the library until the
  * process exits.
  *   Limit: B * Hq * roundup(L, 256) <= 1,048,576 sort keys; beyond that it returns DMA_ERR_WORKSPACE and launches
  *   nothing (use dma_mask_build with a caller-provided workspace instead).

@@ -44,10 +44,8 @@ int launch_decode(const Prob& P, const void* q, const void* K, const void* V, co
                   int32_t* sel_idx, void* ws, cudaStream_t st);
 int launch_mask_bwd(const Prob& P, const void* V, const float* W, const float* A, const float* delta, const float* dM,
                     void* dV, float* dW, float* dA, void* ws, cudaStream_t st);
-// small_scratch: the workspace holds 12 bytes per padded key only (the entry point with static scratch)
 int launch_mask_build(const Prob& P, const void* V, const float* W, const float* A, float* bias, int32_t* expiry,
-                      uint32_t* bitmap, void* ws, cudaStream_t st, const int32_t* cu_seqlens = nullptr, int nseq = 0,
-                      bool small_scratch = false);
+                      uint32_t* bitmap, void* ws, cudaStream_t st, const int32_t* cu_seqlens = nullptr, int nseq = 0);
 
 size_t simt_bwd_ws_bytes(const Prob& P);
 int launch_simt_fwd(const Prob& P, const void* Q, const void* K, const void* V, const float* bias,

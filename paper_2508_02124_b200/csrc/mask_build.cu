@@ -5,12 +5,9 @@
 // Kernels
 //   delta_kernel        V read once (HBM-bound); z, softplus, exp in a fixed fp32 operation order
 //   chunk_sort_kernel   256-key chunks of (delta bits, ~index) keys sorted in shared memory
-//   tree_merge_kernel, expiry_tree_kernel
+//   tree_block_kernel, tree_merge_kernel, expiry_tree_kernel
 //                       selection as a rank tree: the merge passes that finish the sort leave one bit per key and level,
 //                       and a key's expiry (the w-th smallest index among the keys that beat it) is a walk of log2(L) steps
-//   rank_perm_kernel, expiry_kernel
-//                       the chunk-walking selection (packed sequences; the entry point with static scratch): per key, beaters
-//                       are counted chunk by chunk with a binary search in each sorted chunk
 //   bitmap_kernel       per key tile: union of the query-tile intervals its keys are kept in
 #include <mutex>
 #include <utility>
@@ -22,7 +19,6 @@ namespace dma {
 namespace {
 
 constexpr int kChunk = 256;   // keys per sorted chunk (= threads of the sort kernel)
-constexpr int kExpThreads = 256;
 
 // ---- fixed-order fp32 routines: every step is one correctly rounded IEEE operation -----------------------
 
@@ -304,16 +300,16 @@ __device__ __forceinline__ unsigned long long sort_key(float dl, int j) {
     return ((unsigned long long)__float_as_uint(dl) << 32) | (unsigned long long)(0xFFFFFFFFu - (unsigned)j);
 }
 
-// lev == nullptr: chunks written in ascending order (the chunk-walking expiry kernel). Otherwise (rank-tree selection,
-// see tree_merge_kernel): chunks written in DESCENDING order, padding keys carry their index, and the kernel also emits
-// the eight lowest levels of the tree (node sizes 256 ... 2) by splitting the sorted chunk on one index bit per level.
+// Chunks are written in DESCENDING order, padding keys (beyond L) carry their index and sort below every real key, and
+// the kernel also emits the eight lowest levels of the rank tree (node sizes 256 ... 2, see below) by splitting the sorted
+// chunk on one index bit per level.
 __global__ void __launch_bounds__(kChunk) chunk_sort_kernel(const float* __restrict__ delta,
                                                             unsigned long long* __restrict__ sorted, int L, int nchunk,
                                                             uint2* __restrict__ lev, int m) {
     __shared__ unsigned long long s[2][kChunk];
     const int bh = blockIdx.y, c = blockIdx.x, t = threadIdx.x, j = c * kChunk + t;
-    // padding sorts below every real key (delta > 0); in the rank-tree form it keeps its index in the low word
-    unsigned long long v = j < L ? sort_key(delta[(size_t)bh * L + j], j) : (lev ? (unsigned long long)(0xFFFFFFFFu - (unsigned)j) : 0ull);
+    // padding sorts below every real key (delta > 0) and keeps its index in the low word
+    unsigned long long v = j < L ? sort_key(delta[(size_t)bh * L + j], j) : (unsigned long long)(0xFFFFFFFFu - (unsigned)j);
     // bitonic network, ascending; thread t holds position t. Partners less than 32 apart exchange by shuffle, the six
     // wider exchanges go through shared memory (two buffers in turn: one barrier each).
     int nb = 0;
@@ -334,10 +330,6 @@ __global__ void __launch_bounds__(kChunk) chunk_sort_kernel(const float* __restr
             const bool want_min = ((t & mm) == 0) == up;
             v = want_min ? (v < o ? v : o) : (v > o ? v : o);
         }
-    }
-    if (!lev) {
-        sorted[((size_t)bh * nchunk + c) * kChunk + t] = v;      // ascending
-        return;
     }
     s[0][t] = v;
     __syncthreads();
@@ -516,228 +508,63 @@ __global__ void __launch_bounds__(kMergeThreads) tree_merge_kernel(const unsigne
 }
 
 // One thread per rank r of a head: the key at rank r, the walk down the tree, expiry[j] = max(j, index found).
-// kAllRows (non-causal): every row sees every key, so the key is kept by all rows iff fewer than w keys beat it.
-template <bool kAllRows>
+// kMode 2 (non-causal): every row sees every key, so the key is kept by all rows iff fewer than w keys beat it.
+// kMode 1: sequences packed along the key axis (sequence s owns the keys cu[s] <= j < cu[s+1]). A key competes only with
+// the keys of its own sequence [s0, s1): of the first r keys of the head, n0 have an index below s0 (a first walk, along
+// the path of s0, adds up the lower halves it leaves to its left), so the w-th beater inside the sequence is the
+// (n0 + w)-th smallest index overall, if that exists and lies below s1; otherwise the key lives to the end of its sequence.
+template <int kMode>
 __global__ void __launch_bounds__(256) expiry_tree_kernel(const unsigned long long* __restrict__ sorted, const uint2* __restrict__ lev,
-                                                          int32_t* __restrict__ expiry, int L, int Lc, int w, int m) {
+                                                          int32_t* __restrict__ expiry, int L, int Lc, int w, int m,
+                                                          const int32_t* __restrict__ cu, int nseq) {
     const int r = blockIdx.x * 256 + threadIdx.x, bh = blockIdx.y;
     if (r >= L) return;                                          // ranks from L on are padding
     const int j = (int)(0xFFFFFFFFu - (uint32_t)sorted[(size_t)bh * Lc + r]);
+    const size_t W = (size_t)Lc / 32;
+    const uint2* lv0 = lev + (size_t)bh * m * W;
+    // ones among the first c entries of the node that starts at position s of a level
+    auto ones_of = [](const uint2* lv, int s, int c) {
+        const int q = s + c - 1;                                 // last entry of the prefix (c >= 1)
+        const uint2 wd = lv[q >> 5];
+        const uint32_t upto = (2u << (q & 31)) - 1u, from = ~((1u << (s & 31)) - 1u);         // a node smaller than a word starts inside it
+        return (int)wd.x + __popc(wd.y & upto & from);
+    };
+    int s0 = 0, s1 = L, k = w;
+    if (kMode == 1) {
+        int lo = 0, hi = nseq;                                   // largest s with cu[s] <= j
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (cu[mid] <= j) lo = mid; else hi = mid;
+        }
+        s0 = max(cu[lo], 0);
+        s1 = min(cu[lo + 1], L);
+        if (r >= w && s0 > 0) {
+            const uint2* lv = lv0;
+            int c = r, s = 0, n0 = 0;
+            for (int l = 0; l < m && c > 0; ++l, lv += W) {
+                const int half = 1 << (m - 1 - l);
+                const int ones = ones_of(lv, s, c);
+                if (s0 & half) { n0 += c - ones; c = ones; s += half; } else { c -= ones; }
+            }
+            k = w + n0;
+        }
+    }
     int e;
-    if (r < w) {
-        e = L;                                                   // fewer than w keys beat it: never dropped
-    } else if (kAllRows) {
+    if (r < k) {
+        e = s1;                                                  // fewer than w keys beat it (inside its sequence): never dropped
+    } else if (kMode == 2) {
         e = 0;
     } else {
-        const size_t W = (size_t)Lc / 32;
-        const uint2* lv = lev + (size_t)bh * m * W;
-        int k = w, c = r, s = 0;                                 // k-th smallest among the first c entries of the node starting at s
+        const uint2* lv = lv0;
+        int c = r, s = 0;                                        // k-th smallest among the first c entries of the node starting at s
         for (int l = 0; l < m; ++l, lv += W) {
             const int half = 1 << (m - 1 - l);
-            const int q = s + c - 1;                             // last entry of the prefix (c >= k >= 1)
-            const uint2 wd = lv[q >> 5];
-            const uint32_t upto = (2u << (q & 31)) - 1u, from = ~((1u << (s & 31)) - 1u);     // a node smaller than a word starts inside it
-            const int ones = (int)wd.x + __popc(wd.y & upto & from);
-            const int zeros = c - ones;
+            const int ones = ones_of(lv, s, c), zeros = c - ones;
             if (k <= zeros) c = zeros; else { k -= zeros; c = ones; s += half; }
         }
-        e = max(j, s);
+        e = (kMode == 1 && s >= s1) ? s1 : max(j, s);
     }
     expiry[(size_t)bh * L + j] = e;
-}
-
-// Work assignment of the expiry kernel. A key's walk over the sorted chunks ends once w keys have beaten it, after
-// about w / q keys if a fraction q of the head beats it: weak keys stop early, and the keys that fewer than w keys
-// beat at all walk the whole row to learn that their expiry is L. Threads of a CTA walk together, so the keys are
-// handed out in the order of a coarse rank (a counting sort on 12 bits of delta: exponent and top four mantissa bits),
-// which gives the keys of a CTA walks of similar length, and a key whose whole class ranks below w (or, in the
-// non-causal mode, at or above w) is tagged so that it does not walk at all.
-// perm[bh][pos] = key index | (tag << 30); tag 1: fewer than w keys beat it; tag 2: at least w keys beat it.
-constexpr int kRankBins = 4096;
-
-__global__ void __launch_bounds__(1024) rank_perm_kernel(const float* __restrict__ delta, uint32_t* __restrict__ perm, int L, int w) {
-    __shared__ int hist[kRankBins];      // counts, then the next free position of each class
-    __shared__ int wsum[32];
-    __shared__ uint8_t tag[kRankBins];
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const float* dl = delta + (size_t)blockIdx.x * L;
-    uint32_t* out = perm + (size_t)blockIdx.x * L;
-    auto bin = [](float v) { return (int)((__float_as_uint(v) >> 19) & (kRankBins - 1)); };   // delta > 0: bit 31 is clear
-    for (int i = tid; i < kRankBins; i += 1024) hist[i] = 0;
-    __syncthreads();
-    for (int j = tid; j < L; j += 1024) atomicAdd(&hist[bin(dl[j])], 1);
-    __syncthreads();
-    // classes in descending order of delta: thread t owns the four classes kRankBins - 1 - 4t - {0, 1, 2, 3}
-    int c[4], run = 0;
-#pragma unroll
-    for (int u = 0; u < 4; ++u) { c[u] = hist[kRankBins - 1 - 4 * tid - u]; run += c[u]; }
-    int incl = run;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const int t = __shfl_up_sync(0xffffffffu, incl, o);
-        if (lane >= o) incl += t;
-    }
-    if (lane == 31) wsum[warp] = incl;
-    __syncthreads();
-    if (warp == 0) {
-        int v = wsum[lane];
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const int t = __shfl_up_sync(0xffffffffu, v, o);
-            if (lane >= o) v += t;
-        }
-        wsum[lane] = v;
-    }
-    __syncthreads();
-    int start = incl - run + (warp ? wsum[warp - 1] : 0);      // keys in classes above this thread's
-#pragma unroll
-    for (int u = 0; u < 4; ++u) {
-        const int b = kRankBins - 1 - 4 * tid - u;
-        hist[b] = start;
-        tag[b] = start + c[u] <= w ? 1 : (start >= w ? 2 : 0);   // ranks of the class: [start, start + count)
-        start += c[u];
-    }
-    __syncthreads();
-    for (int j = tid; j < L; j += 1024) {
-        const int b = bin(dl[j]);
-        out[atomicAdd(&hist[b], 1)] = (uint32_t)j | ((uint32_t)tag[b] << 30);
-    }
-}
-
-// expiry[j] = max(j, index of the w-th key in index order that beats j), or L if fewer than w keys beat it.
-// Phase 1: the CTA walks the sorted chunks together (each staged once in shared memory as separate high / low
-// words, the next one already in flight) and every thread counts its beaters chunk by chunk with a binary search
-// until the count reaches w. Phase 2: each thread locates the remaining need-th beater inside its final chunk, in index
-// order, 32 keys at a time.
-// kVarlen: sequences packed along the key axis (sequence s owns the keys cu[s] <= j < cu[s+1]). A key competes only
-// with the keys of its own sequence [s0, s1): chunks before s0 count nothing, a chunk that straddles s0 or s1 is
-// counted entry by entry with the index test, the walk ends at s1, and L is replaced by s1.
-// kMode 2 (non-causal): every row sees every key, so a key is kept by all rows (expiry L) iff fewer than w keys of the
-// whole head beat it, and by none (expiry 0) otherwise: phase 1 alone, over all chunks.
-template <int kMode>
-__global__ void __launch_bounds__(kExpThreads) expiry_kernel(const float* __restrict__ delta,
-                                                             const unsigned long long* __restrict__ sorted,
-                                                             int32_t* __restrict__ expiry, int L, int w, int nchunk,
-                                                             const int32_t* __restrict__ cu, int nseq,
-                                                             const uint32_t* __restrict__ perm) {
-    constexpr int kPer = kChunk / kExpThreads;
-    constexpr bool kVarlen = kMode == 1, kAllRows = kMode == 2;
-    static_assert(kChunk == 256 && kPer == 1, "the level-order layout below is written for 256-key chunks");
-    // sbf: the high words once more, in level order of the implicit search tree over the first 255 sorted entries (root at
-    // index 1, children of k at 2k and 2k + 1; the largest entry sits in slot 0). The probes of one search level are
-    // then neighbours in memory, so the first five levels of a warp's 32 searches cost one shared-memory access each;
-    // probing the sorted array itself puts every early level into a single bank (addresses 128 apart, 64 apart, ...).
-    __shared__ uint32_t shi[2][kChunk], slo[2][kChunk], sbf[2][kChunk];
-    __shared__ int c_first;
-    const int bh = blockIdx.y, t = threadIdx.x, slot = blockIdx.x * kExpThreads + t;
-    const float* dl = delta + (size_t)bh * L;
-    const unsigned long long* srt = sorted + (size_t)bh * nchunk * kChunk;
-    const bool valid = slot < L;
-    // packed sequences keep the index order (perm == nullptr): a CTA's keys then share their documents' boundary chunks
-    const uint32_t entry = valid ? (perm ? perm[(size_t)bh * L + slot] : (uint32_t)slot) : 0u;
-    const int j = (int)(entry & 0x3FFFFFFFu), tag = (int)(entry >> 30);     // rank order: see rank_perm_kernel
-    const unsigned long long key = valid ? sort_key(dl[j], j) : ~0ull;
-    const uint32_t khi = (uint32_t)(key >> 32), klo = (uint32_t)key;
-    int s0 = 0, s1 = L;
-    if (kVarlen) {
-        if (valid) {
-            int lo = 0, hi = nseq;                         // largest s with cu[s] <= j
-            while (hi - lo > 1) {
-                const int mid = (lo + hi) >> 1;
-                if (cu[mid] <= j) lo = mid; else hi = mid;
-            }
-            s0 = max(cu[lo], 0);
-            s1 = min(cu[lo + 1], L);
-        }
-        if (t == 0) c_first = nchunk;
-        __syncthreads();
-        if (valid && tag != 1) atomicMin(&c_first, s0 / kChunk);   // the walk starts at the earliest sequence of the CTA's keys
-        __syncthreads();
-    }
-    const int c_begin = kVarlen ? c_first : 0;
-    int cnt = 0, fin = -1, need = 0;
-    // tag 1: fewer than w keys of the whole head beat the key, so it is never dropped; tag 2 (used in the non-causal
-    // mode only): at least w beat it
-    const bool dropped = kAllRows && tag == 2;
-    bool done = !valid || tag == 1 || dropped;
-    unsigned long long nxt[kPer];
-#pragma unroll
-    for (int u = 0; u < kPer; ++u) nxt[u] = c_begin < nchunk ? srt[(size_t)c_begin * kChunk + u * kExpThreads + t] : 0ull;
-    bool all_done = __syncthreads_and(done);               // a CTA of keys that need no walk (see rank_perm_kernel)
-    for (int c = c_begin; c < nchunk && !all_done; ++c) {
-        uint32_t* hi = shi[c & 1];
-        uint32_t* lo = slo[c & 1];
-        uint32_t* bf = sbf[c & 1];
-        {
-            hi[t] = (uint32_t)(nxt[0] >> 32);
-            lo[t] = (uint32_t)nxt[0];
-            const int p1 = t + 1, z = __ffs(p1) - 1;                       // in-order position (1-based) and its level from the leaves
-            bf[t == kChunk - 1 ? 0 : (1 << (7 - z)) + (p1 >> (z + 1))] = (uint32_t)(nxt[0] >> 32);
-        }
-        if (c + 1 < nchunk) {
-#pragma unroll
-            for (int u = 0; u < kPer; ++u) nxt[u] = srt[(size_t)(c + 1) * kChunk + u * kExpThreads + t];
-        }
-        __syncthreads();
-        if (kVarlen && !done && c * kChunk >= s1) done = true;          // past the end of the sequence: expiry = s1
-        if (!done) {
-            int n;
-            if (!kVarlen || (c * kChunk >= s0 && (c + 1) * kChunk <= s1)) {
-                // a = first position whose 64-bit key is greater than ours: fixed-depth, branch-free lower bound on
-                // the high words (delta bits), then the (normally empty) run of equal high words is resolved by the
-                // low words
-                int a = 0, k = 1;
-#pragma unroll
-                for (int s = kChunk / 2; s > 0; s >>= 1) {     // node k is the sorted entry a + s - 1
-                    const int right = bf[k] < khi ? 1 : 0;
-                    a += right ? s : 0;
-                    k = 2 * k + right;
-                }
-                a += (a == kChunk - 1 && bf[0] < khi) ? 1 : 0;   // a = number of entries with hi < khi (0 .. kChunk)
-                while (a < kChunk && hi[a] == khi && lo[a] <= klo) ++a;
-                n = kChunk - a;
-            } else if ((c + 1) * kChunk <= s0) {
-                n = 0;
-            } else {
-                n = 0;
-                for (int a = 0; a < kChunk; ++a) {
-                    const int idx = (int)(0xFFFFFFFFu - lo[a]);
-                    const bool beats = hi[a] > khi || (hi[a] == khi && lo[a] > klo);
-                    n += (beats && idx >= s0 && idx < s1) ? 1 : 0;
-                }
-            }
-            if (cnt + n >= w) { need = w - cnt; fin = c; done = true; }
-            cnt += n;
-        }
-        all_done = __syncthreads_and(done);
-    }
-    // phase 2: each thread scans its final chunk in index order, 32 keys at a time (32 independent loads), until the
-    // remaining need-th beater is found
-    int e = s1;
-    if (!kAllRows && fin >= 0) {
-        const int base = fin * kChunk;
-        int nd = need, found = s1;
-        for (int g = 0; g < kChunk; g += 32) {
-            uint32_t m = 0u;
-#pragma unroll
-            for (int u = 0; u < 32; ++u) {
-                const int k = base + g + u;
-                const bool in = k >= s0 && k < s1;
-                const float v = in ? __ldg(dl + k) : 0.0f;
-                m |= (in && sort_key(v, k) > key) ? 1u << u : 0u;
-            }
-            const int pc = __popc(m);
-            if (nd <= pc) {
-                for (int r = 1; r < nd; ++r) m &= m - 1;          // drop the nd-1 lowest beaters
-                found = base + g + __ffs(m) - 1;
-                break;
-            }
-            nd -= pc;
-        }
-        e = max(j, found);
-    }
-    if (kAllRows) e = (fin >= 0 || dropped) ? 0 : L;
-    if (valid) expiry[(size_t)bh * L + j] = e;
 }
 
 __global__ void fill_i32_kernel(int32_t* p, size_t n, int32_t v) {
@@ -797,8 +624,7 @@ static int tree_levels(int Lc) {
 }
 
 // workspace: header | two buffers of sort keys (8 bytes per padded key each: the merge passes alternate between them) |
-// the rank tree (m levels of 8 bytes per 32 padded keys). The chunk-walking selection (packed sequences, and the
-// entry point with static scratch) uses the first 12 bytes per padded key of the same region: sorted chunks | rank permutation.
+// the rank tree (m levels of 8 bytes per 32 padded keys)
 size_t mask_ws_bytes(const Prob& P) {
     const size_t nchunk = (P.L + kChunk - 1) / kChunk, keys = (size_t)P.B * P.Hq * nchunk * kChunk;
     return kWsHeaderBytes + keys * 2 * sizeof(unsigned long long) + keys / 32 * tree_levels((int)(nchunk * kChunk)) * sizeof(uint2);
@@ -857,9 +683,11 @@ static int mask_build_limits(const Prob& P) {
 }
 
 int launch_mask_build(const Prob& P, const void* V, const float* W, const float* A, float* bias, int32_t* expiry,
-                      uint32_t* bitmap, void* ws, cudaStream_t st, const int32_t* cu, int nseq, bool small_scratch) {
+                      uint32_t* bitmap, void* ws, cudaStream_t st, const int32_t* cu, int nseq) {
     int rc;
     if ((rc = mask_build_limits(P))) return rc;          // an error return means that no kernel has been launched
+    constexpr size_t kBlockSmem = 2 * (size_t)kBlockKeys * sizeof(unsigned long long);
+    if (cudaFuncSetAttribute(tree_block_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kBlockSmem) != cudaSuccess) return DMA_ERR_CUDA;
     if (P.dtype == DMA_BF16)
         rc = P.d == 128 ? launch_delta<__nv_bfloat16, 128>(P, V, W, A, bias, st)
                         : launch_delta<__nv_bfloat16, 64>(P, V, W, A, bias, st);
@@ -873,7 +701,7 @@ int launch_mask_build(const Prob& P, const void* V, const float* W, const float*
         size_t n = (size_t)BH * P.L;
         fill_i32_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(expiry, n, P.L);
         count_launch();
-    } else if (!cu && !small_scratch) {
+    } else {
         // rank tree: sorted chunks and the low levels, one merge pass per further level, then one walk per key
         const int Lc = nchunk * kChunk, m = tree_levels(Lc);
         const size_t keys = (size_t)BH * Lc, Wl = (size_t)Lc / 32;
@@ -883,9 +711,7 @@ int launch_mask_build(const Prob& P, const void* V, const float* W, const float*
         chunk_sort_kernel<<<dim3(nchunk, BH), kChunk, 0, st>>>(bias, buf0, P.L, nchunk, lev, m);
         int launches = 2;
         if (Lc > kChunk) {
-            const size_t smem = 2 * (size_t)kBlockKeys * sizeof(unsigned long long);
-            if (cudaFuncSetAttribute(tree_block_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return DMA_ERR_CUDA;
-            tree_block_kernel<<<dim3((Lc + kBlockKeys - 1) / kBlockKeys, BH), kBlockThreads, smem, st>>>(buf0, buf1, lev, Lc, m);
+            tree_block_kernel<<<dim3((Lc + kBlockKeys - 1) / kBlockKeys, BH), kBlockThreads, kBlockSmem, st>>>(buf0, buf1, lev, Lc, m);
             std::swap(buf0, buf1);
             ++launches;
         }
@@ -895,19 +721,10 @@ int launch_mask_build(const Prob& P, const void* V, const float* W, const float*
             std::swap(buf0, buf1);
         }
         const dim3 grid((P.L + 255) / 256, BH);
-        if (P.causal) expiry_tree_kernel<false><<<grid, 256, 0, st>>>(buf0, lev, expiry, P.L, Lc, P.w, m);
-        else expiry_tree_kernel<true><<<grid, 256, 0, st>>>(buf0, lev, expiry, P.L, Lc, P.w, m);
+        if (cu) expiry_tree_kernel<1><<<grid, 256, 0, st>>>(buf0, lev, expiry, P.L, Lc, P.w, m, cu, nseq);
+        else if (P.causal) expiry_tree_kernel<0><<<grid, 256, 0, st>>>(buf0, lev, expiry, P.L, Lc, P.w, m, nullptr, 0);
+        else expiry_tree_kernel<2><<<grid, 256, 0, st>>>(buf0, lev, expiry, P.L, Lc, P.w, m, nullptr, 0);
         count_launch(launches);
-    } else {
-        auto* sorted = reinterpret_cast<unsigned long long*>((char*)ws + kWsHeaderBytes);
-        uint32_t* perm = reinterpret_cast<uint32_t*>(sorted + (size_t)BH * nchunk * kChunk);
-        chunk_sort_kernel<<<dim3(nchunk, BH), kChunk, 0, st>>>(bias, sorted, P.L, nchunk, nullptr, 0);
-        if (!cu) rank_perm_kernel<<<BH, 1024, 0, st>>>(bias, perm, P.L, P.w);
-        const dim3 grid((P.L + kExpThreads - 1) / kExpThreads, BH);
-        if (cu) expiry_kernel<1><<<grid, kExpThreads, 0, st>>>(bias, sorted, expiry, P.L, P.w, nchunk, cu, nseq, nullptr);
-        else if (!P.causal) expiry_kernel<2><<<grid, kExpThreads, 0, st>>>(bias, sorted, expiry, P.L, P.w, nchunk, nullptr, 0, perm);
-        else expiry_kernel<0><<<grid, kExpThreads, 0, st>>>(bias, sorted, expiry, P.L, P.w, nchunk, nullptr, 0, perm);
-        count_launch(cu ? 2 : 3);
     }
     if ((rc = check_launch())) return rc;
 
@@ -923,13 +740,15 @@ int launch_mask_build(const Prob& P, const void* V, const float* W, const float*
 
 // ---------------------------------------------------------------------------------------------------------------
 // dma_mask_build_static: mask generation for callers that cannot hand over a workspace.
-// The sorted-chunk scratch lives in this file-scope device array, which every GPU that loads the library keeps
+// The selection's scratch (sort keys and rank tree) lives in this file-scope device array, which every GPU that loads the library keeps
 // until the process exits. In host code the array's name is only a stand-in; its device address is looked up
 // once per device with cudaGetSymbolAddress and that pointer is what the kernels receive.
 // ---------------------------------------------------------------------------------------------------------------
 namespace {
-constexpr size_t kStaticKeys = 1u << 20;   // 1 Mi sort keys (8 MiB) and their rank permutation (4 MiB): B * Hq * roundup(L, 256) must not exceed this
-static __device__ __align__(256) unsigned long long g_static_scratch[dma::kWsHeaderBytes / 8 + kStaticKeys + kStaticKeys / 2];
+// 1 Mi padded keys: two buffers of sort keys (8 MiB each) and a rank tree of at most 20 levels (8 bytes per 32 keys and
+// level: 5 MiB). B * Hq * roundup(L, 256) must not exceed this.
+constexpr size_t kStaticKeys = 1u << 20;
+static __device__ __align__(256) unsigned long long g_static_scratch[dma::kWsHeaderBytes / 8 + 2 * kStaticKeys + kStaticKeys / 32 * 20];
 constexpr int kMaxDevices = 64;
 void* g_static_ptr[kMaxDevices];            // per-device address of g_static_scratch (0 = not looked up yet)
 std::mutex g_static_mutex;
@@ -958,5 +777,5 @@ extern "C" int dma_mask_build_static(const dma_problem_t* p, const void* V, cons
         }
         scratch = g_static_ptr[dev];
     }
-    return dma::launch_mask_build(P, V, W_delta, A, bias, expiry, bitmap, scratch, (cudaStream_t)cuda_stream, nullptr, 0, true);
+    return dma::launch_mask_build(P, V, W_delta, A, bias, expiry, bitmap, scratch, (cudaStream_t)cuda_stream);
 }

@@ -51,6 +51,18 @@ def test_mask_heavy_ties():
     assert (e[..., :200] == case.L).all() and (e[..., 200:] == np.arange(200, case.L)).all()
 
 
+@pytest.mark.parametrize("L,w", [(300_001, 5000), (4097, 64), (8192 + 256, 300), (131_072, 131_071)])
+def test_mask_long_heads_with_ragged_run_counts(L, w):
+    """The selection merges sorted runs level by level; a length that is not a power of two leaves a trailing run without
+    a partner on some levels (300 001 keys: 1172 chunks, 19 levels). Every expiry and the bitmap against the oracle."""
+    case = wl.small(C2, B=1, Hq=2, Hkv=1, L=L, w=w, d=64, name="long")
+    g = torch.Generator().manual_seed(L)
+    inp = {"V": torch.randn(case.B, case.L, case.Hkv, case.d, generator=g).to(case.torch_dtype),
+           "W_delta": torch.randn(case.Hq, case.d, generator=g) / 8.0, "A": torch.rand(case.Hq, generator=g) * 1.5 + 0.5}
+    inp["V"][:, L // 3: L // 3 + 700] = inp["V"][:, :1]                 # a run of exactly equal delta across chunk boundaries
+    check_mask(case, inp)
+
+
 def test_mask_other_tile_sizes():
     case = wl.small(C2, B=1, Hq=2, Hkv=1, L=900, w=64, name="tiles")
     inp = wl.make_inputs(case)

@@ -43,11 +43,13 @@ def test_static_scratch_matches_workspace_version_on_consecutive_calls():
         build_both(case, inp, out, full=True)                     # go through the same scratch
 
 
-def test_static_scratch_at_exactly_its_limit():
-    # 32 heads x 32768 keys = 1,048,576 sort keys: the rank permutation ends on the array's last byte. V is the
-    # recipe's noise; the check is bit-equality with the workspace version, twice in a row.
+@pytest.mark.parametrize("Hq,Hkv,L", [(32, 8, 32768), (1, 1, 1 << 20)])
+def test_static_scratch_at_exactly_its_limit(Hq, Hkv, L):
+    # 1,048,576 sort keys in all, as 32 heads of 32768 keys or as one head of 2^20 keys: the one head needs all 20 levels of
+    # the rank tree the array has room for, so its last level ends on the array's last byte. V is the recipe's noise; the
+    # check is bit-equality with the workspace version, twice in a row.
     dev = torch.device("cuda:0")
-    case = wl.small(wl.CONFIGS["3"], B=1, Hq=32, Hkv=8, L=32768, d=64, w=1000, name="static-limit")
+    case = wl.small(wl.CONFIGS["3"], B=1, Hq=Hq, Hkv=Hkv, L=L, d=64, w=1000, name="static-limit")
     g = torch.Generator().manual_seed(77)
     inp = {"V": torch.randn(case.B, case.L, case.Hkv, case.d, generator=g).to(case.torch_dtype),
            "W_delta": torch.randn(case.Hq, case.d, generator=g) / 8.0, "A": torch.rand(case.Hq, generator=g) * 1.5 + 0.5}
