@@ -20,10 +20,12 @@
 // warps 13 and 14 MMA issuers (S^T, dP^T | dV, dK, dQ^T; whole warps with warp-uniform values, one elected lane
 // issues), warp 15 stages the ninth k-step operand of each step's query rows.
 // TMEM columns: dK [0,128) dV [128,256) S^T [256,320) dP^T [320,384) P^T [384,416) dS^T [416,448) dQ^T [448,512).
-// kD = 64 (its own instantiations): K, V, Q and dO tiles are one swizzled half tile each (the second half of every buffer
-// stays unused), S^T and dP^T have four k-steps and the ninth, dK and dV take 64 columns. dQ^T = K^T dS^T keeps M = 128:
-// its upper 64 lanes multiply whatever the unused half of the K buffer holds and are never read (rows of an MMA do not
-// mix), so drain warps 2 and 3 only follow the barriers.
+// kD = 64 (its own instantiations): K, V, Q and dO tiles are one swizzled half tile each, S^T and dP^T have four k-steps
+// and the ninth, dK and dV take 64 columns. What that frees is spent on the two chains that bound a step at d = 128:
+//   - P^T and dS^T are double-buffered (tensor-memory columns [64,128) and the unused half of the V buffer for the
+//     shared-memory copy of dS^T), so the compute warps store step n+1 while the MMAs of step n still read step n's;
+//   - dQ^T = K^T dS^T keeps M = 128 with the K tile loaded a second time into the unused half of its buffer: lanes
+//     64-127 repeat lanes 0-63, so all four drain warps work, two per 32 channels, each on half of the step's rows.
 #include <cstdlib>
 
 #include "common.cuh"
@@ -40,6 +42,7 @@ constexpr int kThreads = 512;
 constexpr uint32_t kKVBytes = 128 * 128 * 2;   // K or V tile: two 16 KB halves (channels 0-63 | 64-127)
 constexpr uint32_t kQBytes = 64 * 128 * 2;     // Q or dO step tile (64 rows): two 8 KB halves
 constexpr int cDK = 0, cDV = 128, cS = 256, cDP = 320, cP = 384, cDS = 416, cDQ = 448;
+constexpr int cP1 = 64, cDS1 = 96;             // second P^T / dS^T buffer (d = 64 only: beside the 64 columns of dK)
 
 struct SharedStorage {
     alignas(1024) uint8_t k[kKVBytes];
@@ -57,7 +60,7 @@ struct SharedStorage {
     alignas(128) uint8_t qext[kStages][2048];
     uint16_t sched[kMaxSteps];                       // head-in-group << 11 | query tile << 1 | half
     uint64_t kv_full, qd_full[kStages], qd_empty[kStages];
-    uint64_t sdp_full, sdp_free, pds_ready, pds_free, dq_full, dq_free;
+    uint64_t sdp_full, sdp_free, pds_ready[2], pds_free[2], dq_full, dq_free;
     uint32_t tmem_base;
     int n_steps;
     int abort_flag;
@@ -113,6 +116,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
            const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmG, const BwdParams P) {
     static_assert(kD == 128 || kD == 64, "head dimensions of the tensor-core kernels");
     constexpr int kHalves = kD / 64;                 // 64-channel (128-byte) swizzled half tiles per operand tile
+    constexpr bool kDouble = kD == 64;               // P^T / dS^T in two buffers used in turn (see the file header)
     extern __shared__ uint8_t smem_raw[];
     SharedStorage& S = *reinterpret_cast<SharedStorage*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const int tid = threadIdx.x, lane = tid & 31;
@@ -143,8 +147,10 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
         }
         mbar_init(&S.sdp_full, 1);
         mbar_init(&S.sdp_free, 8);        // one arrival per compute warp (256 serialised arrivals would cost hundreds of cycles)
-        mbar_init(&S.pds_ready, 8);
-        mbar_init(&S.pds_free, 1);
+        for (int u = 0; u < 2; ++u) {
+            mbar_init(&S.pds_ready[u], 8);
+            mbar_init(&S.pds_free[u], 1);
+        }
         mbar_init(&S.dq_full, 1);
         mbar_init(&S.dq_free, 4);         // one arrival per drain warp
         S.abort_flag = 0;
@@ -301,14 +307,17 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                     dd[(c >> 1) + 1] = pack_bf16(d1.x, d1.y);
                 }
             }
-            // the previous step's dV / dK / dQ GEMMs must have finished reading P^T, dS^T (TMEM) and dS^T (smem)
-            if (n > 0) ok = mbar_wait_warp(&S.pds_free, (n - 1) & 1, abort_flag);
+            // the dV / dK / dQ GEMMs that last used this P^T / dS^T buffer (TMEM and smem) must have finished reading it:
+            // those of the previous step, or with two buffers those of the step before it
+            const int pb = kDouble ? (n & 1) : 0;
+            if (kDouble) { if (n > 1) ok = mbar_wait_warp(&S.pds_free[pb], ((n >> 1) - 1) & 1, abort_flag); }
+            else if (n > 0) ok = mbar_wait_warp(&S.pds_free[0], (n - 1) & 1, abort_flag);
             if (!ok) break;
             tc_fence_after();
-            tmem_st16(tmem + lane_base + cP + hsel * 16, pp);
-            tmem_st16(tmem + lane_base + cDS + hsel * 16, dd);
+            tmem_st16(tmem + lane_base + (pb ? cP1 : cP) + hsel * 16, pp);
+            tmem_st16(tmem + lane_base + (pb ? cDS1 : cDS) + hsel * 16, dd);
             {   // dS^T row r -> shared memory: 16-byte chunk q of the row sits at q XOR (row % 8) (128-byte swizzle)
-                uint8_t* row = S.ds + r * 128;
+                uint8_t* row = (pb ? S.v + kKVBytes / 2 : S.ds) + r * 128;
 #pragma unroll
                 for (int q = 0; q < 4; ++q)
                     *reinterpret_cast<uint4*>(row + (((hsel * 4 + q) ^ (r & 7)) << 4)) = make_uint4(dd[4 * q], dd[4 * q + 1], dd[4 * q + 2], dd[4 * q + 3]);
@@ -317,11 +326,13 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             tc_wait_st();
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(&S.pds_ready);
+            if (lane == 0) mbar_arrive(&S.pds_ready[pb]);
         }
         if (cur_g >= 0 && j < P.L) atomicAdd(&P.dM[(size_t)(b * P.Hq + hk * P.G + cur_g) * P.L + j], dm2.x + dm2.y);
         // epilogue: dK (scaled) and dV rows to global memory; warps w and w+4 each write one half of the channels
-        if (ok && n_steps > 0) ok = mbar_wait_warp(&S.pds_free, (n_steps - 1) & 1, abort_flag);
+        if (ok && n_steps > 0)
+            ok = kDouble ? mbar_wait_warp(&S.pds_free[(n_steps - 1) & 1], ((n_steps - 1) >> 1) & 1, abort_flag)
+                         : mbar_wait_warp(&S.pds_free[0], (n_steps - 1) & 1, abort_flag);
         if (ok) {
             tc_fence_after();
             __nv_bfloat16* dk = P.dK + b * P.ks_b + (int64_t)j * P.ks_l + hk * P.ks_h;
@@ -378,7 +389,11 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
         // Each warp owns 32 channels and its own pair of staging buffers (16 query rows each, used in turn), so the
         // warps never wait for each other: a buffer is rewritten once the reduce-add issued from it two groups ago has
         // finished reading it.
+        // d = 64: lanes 64-127 of dQ^T repeat lanes 0-63 (the K tile sits in both halves of its buffer), so warps 2 and 3
+        // own the same channels as warps 0 and 1 and take the second half of the step's rows.
         const int dw = warp & 3;
+        constexpr int kQuarters = kD == 64 ? 2 : 4;                     // quarter steps per warp
+        const int ch = kD == 64 ? (dw & 1) : dw, qr0 = kD == 64 ? (dw >> 1) * 2 : 0;
         const uint32_t lane_base = (uint32_t)(dw * 32) << 16;
         bool ok = true;
         for (int n = 0; n < n_steps && ok; ++n) {
@@ -387,26 +402,25 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             ok = mbar_wait_warp(&S.dq_full, n & 1, abort_flag);
             if (!ok) break;
             tc_fence_after();
-            uint32_t v[64];
-            if (dw * 32 < kD) {
-                tmem_ld32(tmem + lane_base + cDQ, *reinterpret_cast<uint32_t(*)[32]>(&v[0]));
-                tmem_ld32(tmem + lane_base + cDQ + 32, *reinterpret_cast<uint32_t(*)[32]>(&v[32]));
-                tc_wait_ld();
-            }
+            uint32_t v[kQuarters * 16];
+#pragma unroll
+            for (int c = 0; c < kQuarters / 2; ++c)
+                tmem_ld32(tmem + lane_base + cDQ + qr0 * 16 + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&v[c * 32]));
+            tc_wait_ld();
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&S.dq_free);
-            if (dw * 32 >= kD) continue;               // (no channels of this warp)
 #pragma unroll
-            for (int qr = 0; qr < 4; ++qr) {           // quarter steps of 16 query rows, two staging buffers in turn
+            for (int q = 0; q < kQuarters; ++q) {      // quarter steps of 16 query rows, two staging buffers in turn
+                const int qr = qr0 + q;
                 if (lane == 0) bulk_wait_read_1(); __syncwarp();
 #pragma unroll
-                for (int u = 0; u < 16; ++u) S.dq_stage[dw][qr & 1][u][lane] = __uint_as_float(v[qr * 16 + u]);
+                for (int u = 0; u < 16; ++u) S.dq_stage[dw][q & 1][u][lane] = __uint_as_float(v[q * 16 + u]);
                 fence_proxy_async();
                 __syncwarp();
                 if (lane == 0 && i0 + qr * 16 < P.L) {       // (rows beyond L inside the block land in the accumulator's padding)
-                    float* blk = P.dQacc + ((((size_t)(b * P.Hq + hk * P.G + g) * P.Lblk + (i0 >> 4) + qr) * (kD / 32) + dw) << 9);
-                    bulk_reduce_add_f32(blk, &S.dq_stage[dw][qr & 1][0][0], 2048);
+                    float* blk = P.dQacc + ((((size_t)(b * P.Hq + hk * P.G + g) * P.Lblk + (i0 >> 4) + qr) * (kD / 32) + ch) << 9);
+                    bulk_reduce_add_f32(blk, &S.dq_stage[dw][q & 1][0][0], 2048);
                 }
                 if (lane == 0) bulk_commit();
             }
@@ -428,7 +442,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                     const uint32_t off = r * 128 + ((c ^ (r & 7)) << 4);
                     const int nb = j < P.L ? 16 : 0;
                     cp_async16(S.k + off, P.Kg + krow, nb);
-                    if constexpr (kD == 128) cp_async16(S.k + off + kKVBytes / 2, P.Kg + krow + 64, nb);
+                    cp_async16(S.k + off + kKVBytes / 2, P.Kg + krow + (kD == 128 ? 64 : 0), nb);     // d = 64: the same 64 channels once more
                     cp_async16(S.v + off, P.Vg + vrow, nb);
                     if constexpr (kD == 128) cp_async16(S.v + off + kKVBytes / 2, P.Vg + vrow + 64, nb);
                 }
@@ -438,10 +452,10 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&S.kv_full);
             } else if (lane == 0) {
-                mbar_arrive_expect_tx(&S.kv_full, kHalves * kKVBytes);
-                for (int hf = 0; hf < kHalves; ++hf) {
-                    tma_load_4d(&S.k[hf * (kKVBytes / 2)], &tmK, &S.kv_full, hf * 64, j0, hk, b);
-                    tma_load_4d(&S.v[hf * (kKVBytes / 2)], &tmV, &S.kv_full, hf * 64, j0, hk, b);
+                mbar_arrive_expect_tx(&S.kv_full, (kD == 128 ? 4 : 3) * (kKVBytes / 2));
+                for (int hf = 0; hf < 2; ++hf) {           // d = 64: both halves of the K buffer hold the same 64 channels
+                    tma_load_4d(&S.k[hf * (kKVBytes / 2)], &tmK, &S.kv_full, kD == 128 ? hf * 64 : 0, j0, hk, b);
+                    if (hf < kHalves) tma_load_4d(&S.v[hf * (kKVBytes / 2)], &tmV, &S.kv_full, hf * 64, j0, hk, b);
                 }
             }
             bool ok = true;
@@ -537,31 +551,35 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             // ============================ MMA issuer 2: dV += P^T dO, dK += dS^T Q, dQ^T = K^T dS^T ============================
             constexpr uint32_t id_dkv = idesc_bf16(128, kD, 0, 1);     // P^T|dS^T (TMEM) x dO|Q (MN-major)    -> 128 x d
             constexpr uint32_t id_dq = idesc_bf16(128, 64, 1, 1);      // K^T (MN-major) x dS^T (MN-major)     -> 128 x 64
-            const uint64_t dKt = smem_desc_sw128(smem_u32(S.k), kKVBytes / 2, 1024), dDs = smem_desc_sw128(smem_u32(S.ds), 16, 1024);
+            const uint64_t dKt = smem_desc_sw128(smem_u32(S.k), kKVBytes / 2, 1024), dDs0 = smem_desc_sw128(smem_u32(S.ds), 16, 1024);
+            const uint64_t dDs1 = smem_desc_sw128(smem_u32(S.v + kKVBytes / 2), 16, 1024);      // second dS^T buffer (d = 64)
             const uint64_t dGm0 = smem_desc_sw128(smem_u32(S.g[0]), kQBytes / 2, 1024), dQm0 = smem_desc_sw128(smem_u32(S.q[0]), kQBytes / 2, 1024);
             const uint32_t tmem_u = __shfl_sync(0xffffffffu, tmem, 0);
             const int n_steps_u = __shfl_sync(0xffffffffu, n_steps, 0);
             bool ok = true;
             for (int n = 0; n < n_steps_u && ok; ++n) {
                 const int st = n % kStages;
-                ok = mbar_wait_warp(&S.pds_ready, n & 1, abort_flag);
+                const int pb = kDouble ? (n & 1) : 0;
+                ok = mbar_wait_warp(&S.pds_ready[pb], (kDouble ? (n >> 1) : n) & 1, abort_flag);
                 if (ok && n > 0) ok = mbar_wait_warp(&S.dq_free, (n - 1) & 1, abort_flag);
                 if (!ok) break;
                 tc_fence_after();
+                const uint32_t tP = tmem_u + (pb ? cP1 : cP), tDS = tmem_u + (pb ? cDS1 : cDS);
+                const uint64_t dDs = pb ? dDs1 : dDs0;
                 const uint64_t dGm = dGm0 + (uint64_t)(st * (kQBytes >> 4)), dQm = dQm0 + (uint64_t)(st * (kQBytes >> 4));
                 const uint32_t acc0 = n > 0 ? 1u : 0u;
                 if (elect_one()) {
 #pragma unroll
                     for (int kk = 0; kk < 4; ++kk)         // 64 query rows = 4 k-steps of 16
-                        mma_ts(tmem_u + cDV, tmem_u + cP + kk * 8, dGm + (uint64_t)((kk * 2048) >> 4), id_dkv, kk > 0 ? 1u : acc0);
+                        mma_ts(tmem_u + cDV, tP + kk * 8, dGm + (uint64_t)((kk * 2048) >> 4), id_dkv, kk > 0 ? 1u : acc0);
 #pragma unroll
                     for (int kk = 0; kk < 4; ++kk)
-                        mma_ts(tmem_u + cDK, tmem_u + cDS + kk * 8, dQm + (uint64_t)((kk * 2048) >> 4), id_dkv, kk > 0 ? 1u : acc0);
+                        mma_ts(tmem_u + cDK, tDS + kk * 8, dQm + (uint64_t)((kk * 2048) >> 4), id_dkv, kk > 0 ? 1u : acc0);
                     tc_commit(&S.qd_empty[st]);            // the dQ GEMM reads K and dS^T only: Q / dO of this stage are free here
 #pragma unroll
                     for (int kk = 0; kk < 8; ++kk)         // 128 keys = 8 k-steps of 16
                         mma_ss(tmem_u + cDQ, dKt + (uint64_t)((kk * 2048) >> 4), dDs + (uint64_t)((kk * 2048) >> 4), id_dq, kk > 0);
-                    tc_commit(&S.pds_free);
+                    tc_commit(&S.pds_free[pb]);
                     tc_commit(&S.dq_full);
                 }
                 __syncwarp();
