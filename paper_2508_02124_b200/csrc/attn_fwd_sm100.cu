@@ -32,6 +32,9 @@ using namespace ptx;
 constexpr int kStages = 2;
 constexpr int kMaxSched = 1024;               // key tiles per CTA schedule (L <= 131072)
 constexpr int kThreads = 384;
+constexpr int kLaunchRegs = 168;             // registers per thread the kernel must be compiled to: its setmaxnreg requests
+                                            // (8 warps up by 40, 4 warps down by 80) balance only for this count, and an
+                                            // unbalanced request waits forever
 constexpr uint32_t kTileBytes = 128 * 128 * 2;   // one 128 x 128 bf16 tile = two 16 KB swizzled half tiles
 constexpr int kMaskSlots = 13;                 // keys expiring inside a tile's rows that the ninth k-step can mask
 constexpr float kSmallStab = 1048576.0f;        // 2^20: below it the stabiliser is fl(m_ref c), see the softmax groups
@@ -897,6 +900,15 @@ int launch_tc_fwd(const Prob& P, const void* Q, const void* K, const void* V, co
                   const int32_t* expiry, const uint32_t* bitmap, void* O, float* lse, void* ws, cudaStream_t st) {
     const bool compact = (P.flags & DMA_FLAG_COMPACT_KV) != 0;
     if (P.Tc > kMaxSched) return DMA_ERR_UNSUPPORTED;
+    const bool block_skip = (P.flags & DMA_FLAG_BLOCK_SKIP) != 0;
+    auto kern = P.d == 128 ? (compact ? (block_skip ? fwd_kernel<true, true, 128> : fwd_kernel<true, false, 128>)
+                                      : (block_skip ? fwd_kernel<false, true, 128> : fwd_kernel<false, false, 128>))
+                           : (compact ? (block_skip ? fwd_kernel<true, true, 64> : fwd_kernel<true, false, 64>)
+                                      : (block_skip ? fwd_kernel<false, true, 64> : fwd_kernel<false, false, 64>));
+    {
+        cudaFuncAttributes fa;       // (before anything is enqueued)
+        if (cudaFuncGetAttributes(&fa, kern) != cudaSuccess || fa.numRegs != kLaunchRegs) return DMA_ERR_CUDA;
+    }
     CUtensorMap tmQ, tmK, tmV;
     int rc;
     const int Trq = (P.Lq + 127) / 128, npairs = (Trq + 1) / 2;
@@ -930,11 +942,6 @@ int launch_tc_fwd(const Prob& P, const void* Q, const void* K, const void* V, co
     const size_t smem = sizeof(SharedStorage) + 1024;
     dim3 grid(P.B * P.Hq, npairs);
     timing_mark(0, false, st);
-    const bool block_skip = (P.flags & DMA_FLAG_BLOCK_SKIP) != 0;
-    auto kern = P.d == 128 ? (compact ? (block_skip ? fwd_kernel<true, true, 128> : fwd_kernel<true, false, 128>)
-                                      : (block_skip ? fwd_kernel<false, true, 128> : fwd_kernel<false, false, 128>))
-                           : (compact ? (block_skip ? fwd_kernel<true, true, 64> : fwd_kernel<true, false, 64>)
-                                      : (block_skip ? fwd_kernel<false, true, 64> : fwd_kernel<false, false, 64>));
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return DMA_ERR_CUDA;
     kern<<<grid, kThreads, smem, st>>>(tmQ, tmK, tmV, fp);
     timing_mark(0, true, st);
