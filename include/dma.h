@@ -103,7 +103,7 @@ typedef struct {
     int32_t causal;              /* 1: key j is visible to row i iff j <= i. 0 (non-causal, the App. A listing with an
                                     all-zero causal mask): every row sees every key, so all rows of a head keep the same
                                     min(w, L) keys; expiry[j] is then L for a kept key and 0 otherwise, key j is kept by the
-                                    rows 0 <= i < expiry[j], and every bitmap row of a head is the same. bf16 with d = 128
+                                    rows 0 <= i < expiry[j], and every bitmap row of a head is the same. bf16 (tensor-core kernels)
                                     always runs token-compacted in this mode (DMA_FLAG_COMPACT_KV is implied: the larger
                                     workspaces); dma_mask_build_varlen needs causal = 1              */
     int32_t dtype;               /* DMA_BF16 | DMA_FP32                                                         */
@@ -174,8 +174,8 @@ int dma_mask_build_varlen(const dma_problem_t* p, const void* V, const float* W_
  *   s_j = q_i . k_j * scale + bias[j]   over keys with j <= i < expiry[j];   p = softmax(s);   O_i = sum p_j v_j
  *   lse_i = log sum_j exp(s_j)   (natural log; replaces Alg. 1's (l, m) pair)
  * Key tiles whose bitmap bit is 0 are neither loaded nor computed. Any self-consistent (bias, expiry, bitmap)
- * triple is accepted. bf16: tcgen05/TMA kernel for d = 128; d = 64 runs the same kernel on zero-padded 128-channel copies
- * held in the workspace (forward and backward; dma_query_workspace reports the larger sizes); fp32: CUDA-core kernel. */
+ * triple is accepted. bf16: tcgen05/TMA kernels, one instantiation for d = 128 and one for d = 64 (forward and backward);
+ * fp32: CUDA-core kernel. */
 int dma_attn_fwd(const dma_problem_t* p, const void* Q, const void* K, const void* V,
                  const float* bias, const int32_t* expiry, const uint32_t* bitmap,
                  void* O, float* lse, void* ws, size_t ws_bytes, void* cuda_stream);
@@ -184,7 +184,7 @@ int dma_attn_fwd(const dma_problem_t* p, const void* Q, const void* K, const voi
  * to the rows q_begin <= i < q_begin + q_len of the sequence of p->L keys, bottom-right aligned when q_begin + q_len = L):
  * Q and O are [B, q_len, Hq, d] (q_stride / o_stride, all 0 = packed with q_len rows), lse is [B, Hq, q_len]; K, V, bias
  * and expiry are those of the whole sequence (the mask built over all p->L keys). q_begin and q_len need no alignment.
- * bf16 with d = 128 runs the token-compacted kernel (its workspace size: dma_query_workspace with DMA_FLAG_COMPACT_KV set);
+ * bf16 (d = 128 or 64) runs the token-compacted kernel (its workspace size: dma_query_workspace with DMA_FLAG_COMPACT_KV set);
  * the other cases run the CUDA-core kernel. No bitmap is needed. */
 int dma_attn_fwd_chunk(const dma_problem_t* p, int32_t q_begin, int32_t q_len, const void* Q, const void* K, const void* V,
                        const float* bias, const int32_t* expiry, void* O, float* lse, void* ws, size_t ws_bytes,
