@@ -308,9 +308,13 @@ def host(T):
         inp = wl.make_inputs(case)
         try:
             got, dev = TH.host_step(case, inp), gpu_run(case, inp, backward=bwd)
-            bad = [k for k in ("O", "lse") + (("dK", "dV") if bwd else ()) if not torch.equal(got[k], dev[k].cpu())]
+            # where the library picks the token-compacted kernels (L >= 2048, 4 w <= L) and a KV head serves several query
+            # heads, dK and dV are summed over the group with floating-point atomics: equal up to the order of the adds
+            atomic = case.dtype == "bf16" and L >= 2048 and 4 * min(w, L) <= L and G > 1
+            exact = ("O", "lse") + (("dK", "dV") if bwd and not atomic else ())
+            bad = [k for k in exact if not torch.equal(got[k], dev[k].cpu())]
             if bwd:
-                bad += [k for k in ("dQ", "dM") if not close(got[k], dev[k].cpu(), 2e-2)]
+                bad += [k for k in ("dQ", "dM") + (("dK", "dV") if atomic else ()) if not close(got[k], dev[k].cpu(), 2e-2)]
             if bad:
                 T.fail(case, bad)
         except dma.DmaError as ex:
