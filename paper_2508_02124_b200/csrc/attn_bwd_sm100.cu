@@ -73,7 +73,10 @@ struct BwdParams {
     const int32_t* expiry;
     const uint32_t* bitmap;
     int sched_group;            // (batch, head) entries per scheduling group, a divisor of gridDim.x
-    float* dQacc;               // fp32, zeroed, blocked: [B, Hq, Lblk, d / 32][16 rows][32 channels]
+    float* dQacc;               // fp32, zeroed, blocked: [B, Hq, Lblk, d / 32] blocks of 16 rows x 32 channels = 2 KB, each laid out
+                                // as the drain warps stage it: channel c owns 64 bytes (its 16 rows), and the 16-byte chunk of
+                                // rows 4q .. 4q + 3 sits at chunk q ^ ((c >> 1) & 3) (a thread = a channel then stores four
+                                // 16-byte chunks without bank conflicts, instead of 16 scalars)
     int Lblk;                   // 16-row blocks per head: 8 * Tr (rows padded to whole 128-row tiles)
     __nv_bfloat16* dK;
     __nv_bfloat16* dV;
@@ -414,8 +417,13 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             for (int q = 0; q < kQuarters; ++q) {      // quarter steps of 16 query rows, two staging buffers in turn
                 const int qr = qr0 + q;
                 if (lane == 0) bulk_wait_read_1(); __syncwarp();
+                {   // this thread's channel, 16 rows: four 16-byte stores (see BwdParams::dQacc for the block's layout)
+                    uint8_t* line = reinterpret_cast<uint8_t*>(&S.dq_stage[dw][q & 1][0][0]) + lane * 64;
 #pragma unroll
-                for (int u = 0; u < 16; ++u) S.dq_stage[dw][q & 1][u][lane] = __uint_as_float(v[q * 16 + u]);
+                    for (int qq = 0; qq < 4; ++qq)
+                        *reinterpret_cast<uint4*>(line + ((qq ^ ((lane >> 1) & 3)) << 4)) =
+                            make_uint4(v[q * 16 + 4 * qq], v[q * 16 + 4 * qq + 1], v[q * 16 + 4 * qq + 2], v[q * 16 + 4 * qq + 3]);
+                }
                 fence_proxy_async();
                 __syncwarp();
                 if (lane == 0 && i0 + qr * 16 < P.L) {       // (rows beyond L inside the block land in the accumulator's padding)
@@ -637,19 +645,24 @@ __global__ void dq_convert_bf16_kernel(const float* __restrict__ acc, __nv_bfloa
     *reinterpret_cast<uint4*>(dQ + b * qs_b + (int64_t)i * qs_l + h * qs_h + c) = o;
 }
 
-// blocked fp32 dQ accumulator (see BwdParams::dQacc) -> softmax scale applied -> bf16 dQ in the caller's layout; 8 elements per thread
-__global__ void dq_unblock_bf16_kernel(const float* __restrict__ acc, __nv_bfloat16* __restrict__ dQ, size_t n8, int L, int Hq, int Lblk,
-                                       int64_t qs_b, int64_t qs_l, int64_t qs_h, float scale, int d) {
-    const size_t t = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (t >= n8) return;
-    const size_t e = t * 8;                       // element of the packed [B, L, Hq, d] order
-    const int c = e % d, h = (e / d) % Hq, i = (e / ((size_t)d * Hq)) % L, b = e / ((size_t)d * Hq * L);
-    const float* src = acc + (((((size_t)(b * Hq + h) * Lblk + (i >> 4)) * (d >> 5) + (c >> 5)) * 16 + (i & 15)) << 5) + (c & 31);
-    const float4 a = *reinterpret_cast<const float4*>(src), bb = *reinterpret_cast<const float4*>(src + 4);
-    uint4 o;
-    o.x = ptx::pack_bf16(a.x * scale, a.y * scale); o.y = ptx::pack_bf16(a.z * scale, a.w * scale);
-    o.z = ptx::pack_bf16(bb.x * scale, bb.y * scale); o.w = ptx::pack_bf16(bb.z * scale, bb.w * scale);
-    *reinterpret_cast<uint4*>(dQ + b * qs_b + (int64_t)i * qs_l + h * qs_h + c) = o;
+// blocked fp32 dQ accumulator (see BwdParams::dQacc) -> softmax scale applied -> bf16 dQ in the caller's layout. One CTA per
+// (batch, head, 16-row block); a thread takes two neighbouring channels (they share their chunk position) and four rows:
+// two 16-byte loads, four 4-byte stores that the lanes of a warp, consecutive channel pairs, make whole 128-byte lines of.
+__global__ void __launch_bounds__(256) dq_unblock_bf16_kernel(const float* __restrict__ acc, __nv_bfloat16* __restrict__ dQ, int L, int Hq,
+                                                              int Lblk, int64_t qs_b, int64_t qs_l, int64_t qs_h, float scale, int d) {
+    const int t = threadIdx.x, rb = blockIdx.x % Lblk, bh = blockIdx.x / Lblk, h = bh % Hq, b = bh / Hq;
+    const int pairs = d >> 1, p = t % pairs, q = t / pairs;            // channel pair, quad of rows
+    if (q >= 4) return;
+    const int c = 2 * p, cc = c & 31;
+    const float* src = acc + ((size_t)bh * Lblk + rb) * (size_t)d * 16 + (c >> 5) * 512 + cc * 16 + ((q ^ ((cc >> 1) & 3)) << 2);
+    const float4 x = *reinterpret_cast<const float4*>(src), y = *reinterpret_cast<const float4*>(src + 16);
+    const float xs[4] = {x.x, x.y, x.z, x.w}, ys[4] = {y.x, y.y, y.z, y.w};
+    __nv_bfloat16* out = dQ + b * qs_b + h * qs_h + c;
+#pragma unroll
+    for (int rr = 0; rr < 4; ++rr) {
+        const int i = rb * 16 + 4 * q + rr;
+        if (i < L) *reinterpret_cast<uint32_t*>(out + (int64_t)i * qs_l) = ptx::pack_bf16(xs[rr] * scale, ys[rr] * scale);
+    }
 }
 
 }  // namespace
@@ -781,7 +794,7 @@ int launch_tc_bwd(const Prob& P, const void* Q, const void* K, const void* V, co
         kern<<<dim3(P.B * P.Hkv, P.Tc), kThreads, smem, st>>>(tmQ, tmK, tmV, tmG, bp);
         timing_mark(1, true, st);
     }
-    dq_unblock_bf16_kernel<<<(unsigned)((nq / 8 + 255) / 256), 256, 0, st>>>(acc, (__nv_bfloat16*)dQ, nq / 8, P.L, P.Hq, P.Tr * 8, P.qs[0], P.qs[1], P.qs[2], P.scale, P.d);
+    dq_unblock_bf16_kernel<<<(unsigned)((size_t)P.B * P.Hq * P.Tr * 8), 256, 0, st>>>(acc, (__nv_bfloat16*)dQ, P.L, P.Hq, P.Tr * 8, P.qs[0], P.qs[1], P.qs[2], P.scale, P.d);
     count_launch(3);
     return check_launch();
 }
