@@ -672,10 +672,13 @@ __global__ void __launch_bounds__(256) dq_unblock_bf16_kernel(const float* __res
 // keys stay in index order, so 128 consecutive entries start at nearby rows and expire within one band of each other:
 // on i.i.d. importance at L = 16384, w = 2048 the walk covers 1.4 x the (row, key) pairs actually kept, against 4.3 x
 // for tiles of consecutive keys. Padded with L up to Tc * 128.
-// One CTA of 1024 threads per (batch, head); the warps take turns per 1024-key chunk so that the order is kept.
+// One CTA of 1024 threads per (batch, head). Per 1024-key chunk every warp ranks its 32 keys within their class
+// (match_any), the per-warp class counts are turned into start positions by 64 threads (one per class, a running sum over
+// the 32 warps and over the chunks), and every key is written to its place: stable in key order, three barriers per chunk.
 __global__ void __launch_bounds__(1024) lifetime_perm_kernel(const int32_t* __restrict__ expiry, int* __restrict__ perm, int L, int Tc, int causal) {
     __shared__ int hist[64];
-    __shared__ int offs[64];
+    __shared__ int offs[64];                 // next free position of each class
+    __shared__ int cnt[32][64];              // per warp and class: keys in this chunk, then their start position
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int32_t* e = expiry + (size_t)blockIdx.x * L;
     int* out = perm + (size_t)blockIdx.x * Tc * 128;
@@ -693,17 +696,25 @@ __global__ void __launch_bounds__(1024) lifetime_perm_kernel(const int32_t* __re
     for (int base = 0; base < L; base += 1024) {
         const int j = base + tid;
         const int c = j < L ? cls(j) : -1;
-        for (int wq = 0; wq < 32; ++wq) {
-            if (warp == wq && base + wq * 32 < L) {
-                const uint32_t same = __match_any_sync(0xffffffffu, c);
-                const int leader = __ffs(same) - 1, rank = __popc(same & ((1u << lane) - 1));
-                int start = 0;
-                if (lane == leader && c >= 0) { start = offs[c]; offs[c] = start + __popc(same); }
-                start = __shfl_sync(0xffffffffu, start, leader);
-                if (c >= 0) out[start + rank] = j;
+        const uint32_t same = __match_any_sync(0xffffffffu, c);
+        const int leader = __ffs(same) - 1, rank = __popc(same & ((1u << lane) - 1));
+        cnt[warp][lane] = 0;
+        cnt[warp][lane + 32] = 0;
+        __syncwarp();
+        if (lane == leader && c >= 0) cnt[warp][c] = __popc(same);
+        __syncthreads();
+        if (tid < 64) {
+            int run = offs[tid];
+            for (int w = 0; w < 32; ++w) {
+                const int n = cnt[w][tid];
+                cnt[w][tid] = run;
+                run += n;
             }
-            __syncthreads();
+            offs[tid] = run;
         }
+        __syncthreads();
+        if (c >= 0) out[cnt[warp][c] + rank] = j;
+        __syncthreads();
     }
     for (int t = L + tid; t < Tc * 128; t += 1024) out[t] = L;
 }
