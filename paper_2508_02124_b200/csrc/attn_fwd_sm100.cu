@@ -851,34 +851,38 @@ int make_tmap_bf16(CUtensorMap* m, const void* base, int B, int L, int H, int d,
 
 // Token-compacted mode, per (batch, head, pair of query tiles): the ascending list of keys j that some row i of the
 // pair's 256 rows keeps, i.e. j <= i < expiry[j] for some i in [i0, i0 + 255]  <=>  j <= i0 + 255 and expiry[j] > max(i0, j).
-// At most w + 256 keys qualify. One CTA of 256 threads per list: 256 keys per pass, ballots and per-warp counts keep the
-// order; the list is padded with -1 to the next multiple of 128.
+// At most w + 256 keys qualify. One CTA of 256 threads per list; every warp owns a contiguous eighth of the candidate keys,
+// counts its kept keys in a first pass and writes them from its start position (the sum of the earlier warps' counts) in a
+// second one: ascending order, one barrier. The list is padded with -1 to the next multiple of 128.
 __global__ void __launch_bounds__(256) compact_lists_kernel(const int32_t* __restrict__ expiry, int* __restrict__ cidx,
                                                             int* __restrict__ ccnt, int L, int npairs, int cap, int causal,
                                                             int q_off, int32_t* __restrict__ status) {
-    __shared__ int wsum[2][8];
+    __shared__ int wcount[8];
     const int list = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int bh = list / npairs, pair = list % npairs, i0 = q_off + pair * 256;
     const int32_t* e = expiry + (size_t)bh * L;
     int* out = cidx + (size_t)list * cap;
     const int jend = causal ? min(L, i0 + 256) : L;     // non-causal: key j is kept by the rows i < expiry[j], whatever j
-    int n = 0, buf = 0;
-    for (int base = 0; base < jend; base += 256, buf ^= 1) {
-        const int j = base + tid;
-        const bool keep = j < jend && e[j] > (causal ? max(i0, j) : i0);
-        const uint32_t bal = __ballot_sync(0xffffffffu, keep);
-        if (lane == 0) wsum[buf][warp] = __popc(bal);
-        __syncthreads();                                   // (the other buffer is free to be rewritten next pass)
-        int before = 0, total = 0;
+    const int seg = (((jend + 7) / 8 + 31) / 32) * 32, j0 = warp * seg, j1 = min(jend, j0 + seg);
+    auto kept = [&](int j) { return j < j1 && e[j] > (causal ? max(i0, j) : i0); };
+    int cnt = 0;
+    for (int base = j0; base < j1; base += 32) cnt += __popc(__ballot_sync(0xffffffffu, kept(base + lane)));
+    if (lane == 0) wcount[warp] = cnt;
+    __syncthreads();
+    int pos = 0, n = 0;
 #pragma unroll
-        for (int wq = 0; wq < 8; ++wq) {
-            const int c = wsum[buf][wq];
-            before += wq < warp ? c : 0;
-            total += c;
-        }
-        const int pos = n + before + __popc(bal & ((1u << lane) - 1));
-        if (keep && pos < cap) out[pos] = j;
-        n += total;
+    for (int wq = 0; wq < 8; ++wq) {
+        const int c = wcount[wq];
+        pos += wq < warp ? c : 0;
+        n += c;
+    }
+    for (int base = j0; base < j1; base += 32) {
+        const int j = base + lane;
+        const bool keep = kept(j);
+        const uint32_t bal = __ballot_sync(0xffffffffu, keep);
+        const int at = pos + __popc(bal & ((1u << lane) - 1));
+        if (keep && at < cap) out[at] = j;
+        pos += __popc(bal);
     }
     // more kept keys than the list holds (a mask that keeps more than w keys in some row): reported, not truncated silently
     if (n > cap && tid == 0) atomicExch(status, (int32_t)DMA_ERR_MASK_OVERFLOW);
