@@ -75,8 +75,8 @@ struct FwdParams {
     float scale_log2;                          // softmax scale * log2(e)
     float inv_scale;                           // 1 / softmax scale
     float rescale_gap;                         // growth of a row max (score units) beyond which O is rescaled
-    // token-compacted mode: per (batch, head, pair of query tiles) the ascending list of keys that some row of the
-    // pair keeps, padded with -1 to a multiple of 128 (ccap entries per list), and its length
+    // token-compacted mode: per (batch, head, pair of query tiles) the list of keys that some row of the
+    // pair keeps (see compact_lists_kernel), padded with -1 to a multiple of 128 (ccap entries per list), and its length
     const int* cidx;
     const int* ccnt;
     const __nv_bfloat16* Kg;                   // K and V base pointers for the row gathers (strides below)
@@ -849,41 +849,59 @@ int make_tmap_bf16(CUtensorMap* m, const void* base, int B, int L, int H, int d,
     return r == CUDA_SUCCESS ? DMA_OK : DMA_ERR_CUDA;
 }
 
-// Token-compacted mode, per (batch, head, pair of query tiles): the ascending list of keys j that some row i of the
+// Token-compacted mode, per (batch, head, pair of query tiles): the list of keys j that some row i of the
 // pair's 256 rows keeps, i.e. j <= i < expiry[j] for some i in [i0, i0 + 255]  <=>  j <= i0 + 255 and expiry[j] > max(i0, j).
-// At most w + 256 keys qualify. One CTA of 256 threads per list; every warp owns a contiguous eighth of the candidate keys,
-// counts its kept keys in a first pass and writes them from its start position (the sum of the earlier warps' counts) in a
-// second one: ascending order, one barrier. The list is padded with -1 to the next multiple of 128.
+// At most w + 256 keys qualify. The list is in two parts, each ascending: first the keys that ALL 256 rows keep
+// (j <= i0 and expiry[j] >= i0 + 256), then the keys that enter or expire inside the pair's rows. The forward kernel
+// needs no order among the columns, and this one leaves the keys that need the per-element test (a few hundred per pair)
+// in the last slices instead of a few in every slice. One CTA of 256 threads per list; every warp owns a contiguous
+// eighth of the candidate keys, counts its keys of either part in a first pass and writes them from its start positions
+// (the sums of the earlier warps' counts) in a second one: one barrier. Padded with -1 to the next multiple of 128.
 __global__ void __launch_bounds__(256) compact_lists_kernel(const int32_t* __restrict__ expiry, int* __restrict__ cidx,
                                                             int* __restrict__ ccnt, int L, int npairs, int cap, int causal,
                                                             int q_off, int32_t* __restrict__ status) {
-    __shared__ int wcount[8];
+    __shared__ int wcount[2][8];
     const int list = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int bh = list / npairs, pair = list % npairs, i0 = q_off + pair * 256;
     const int32_t* e = expiry + (size_t)bh * L;
     int* out = cidx + (size_t)list * cap;
     const int jend = causal ? min(L, i0 + 256) : L;     // non-causal: key j is kept by the rows i < expiry[j], whatever j
     const int seg = (((jend + 7) / 8 + 31) / 32) * 32, j0 = warp * seg, j1 = min(jend, j0 + seg);
-    auto kept = [&](int j) { return j < j1 && e[j] > (causal ? max(i0, j) : i0); };
-    int cnt = 0;
-    for (int base = j0; base < j1; base += 32) cnt += __popc(__ballot_sync(0xffffffffu, kept(base + lane)));
-    if (lane == 0) wcount[warp] = cnt;
+    // 0: not in the list, 1: kept by every row of the pair, 2: kept by some
+    auto kind = [&](int j) {
+        if (j >= j1) return 0;
+        const int ej = e[j], first = causal ? j : 0;
+        if (ej <= max(i0, first)) return 0;
+        return (first <= i0 && ej >= i0 + 256) ? 1 : 2;
+    };
+    int c1 = 0, c2 = 0;
+    for (int base = j0; base < j1; base += 32) {
+        const int k = kind(base + lane);
+        c1 += __popc(__ballot_sync(0xffffffffu, k == 1));
+        c2 += __popc(__ballot_sync(0xffffffffu, k == 2));
+    }
+    if (lane == 0) { wcount[0][warp] = c1; wcount[1][warp] = c2; }
     __syncthreads();
-    int pos = 0, n = 0;
+    int p1 = 0, p2 = 0, n1 = 0, n2 = 0;
 #pragma unroll
     for (int wq = 0; wq < 8; ++wq) {
-        const int c = wcount[wq];
-        pos += wq < warp ? c : 0;
-        n += c;
+        const int a = wcount[0][wq], bq = wcount[1][wq];
+        p1 += wq < warp ? a : 0;
+        p2 += wq < warp ? bq : 0;
+        n1 += a;
+        n2 += bq;
     }
+    p2 += n1;                                            // the second part starts behind the first
     for (int base = j0; base < j1; base += 32) {
-        const int j = base + lane;
-        const bool keep = kept(j);
-        const uint32_t bal = __ballot_sync(0xffffffffu, keep);
-        const int at = pos + __popc(bal & ((1u << lane) - 1));
-        if (keep && at < cap) out[at] = j;
-        pos += __popc(bal);
+        const int j = base + lane, k = kind(j);
+        const uint32_t b1 = __ballot_sync(0xffffffffu, k == 1), b2 = __ballot_sync(0xffffffffu, k == 2);
+        const uint32_t below = (1u << lane) - 1;
+        const int at = k == 1 ? p1 + __popc(b1 & below) : p2 + __popc(b2 & below);
+        if (k != 0 && at < cap) out[at] = j;
+        p1 += __popc(b1);
+        p2 += __popc(b2);
     }
+    int n = n1 + n2;
     // more kept keys than the list holds (a mask that keeps more than w keys in some row): reported, not truncated silently
     if (n > cap && tid == 0) atomicExch(status, (int32_t)DMA_ERR_MASK_OVERFLOW);
     n = min(n, cap);
