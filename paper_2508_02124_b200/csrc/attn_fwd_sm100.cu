@@ -119,6 +119,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
     const int pair = npairs - 1 - (int)blockIdx.y;          // heaviest query tiles first
     const int qt0 = 2 * pair, qt1 = 2 * pair + 1;           // query tiles inside the chunk (the whole sequence unless P.q_off / P.Lq say otherwise)
     const bool has1 = qt1 < P.Trq;
+    const int lpair = (kCompact && !P.causal) ? 0 : pair;   // non-causal: all rows of a head keep the same keys, one list serves every pair
     volatile int* abort_flag = &S.abort_flag;
 
     if (tid == 0) {
@@ -149,7 +150,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
         int n = 0;
         if constexpr (kCompact) {
             // every 128-key slice of the gathered list, used by both query tiles
-            n = min((P.ccnt[(size_t)bh * npairs + pair] + 127) / 128, kMaxSched);
+            n = min((P.ccnt[(size_t)bh * npairs + lpair] + 127) / 128, kMaxSched);
             for (int t = lane; t < n; t += 32) S.sched[t] = (uint32_t)t | (1u << 30) | (has1 ? (1u << 31) : 0u);
         } else {
             const int kt_last = min(has1 ? qt1 : qt0, P.Tc - 1);
@@ -384,7 +385,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                     for (int hf = 0; hf < kHalves; ++hf)
                         tma_load_4d(&S.q[w][hf * (kTileBytes / 2)], &tmQ, &S.q_full, hf * 64, (qt0 + w) * 128, h, b);
             }
-            const int* list = P.cidx + ((size_t)bh * npairs + pair) * P.ccap;
+            const int* list = P.cidx + ((size_t)bh * npairs + lpair) * P.ccap;
             const int64_t row_stride = isK ? P.ks_l : P.vs_l;
             const __nv_bfloat16* src = (isK ? P.Kg + b * P.ks_b + hk * P.ks_h : P.Vg + b * P.vs_b + hk * P.vs_h) + (lane & 7) * 8;
             const int rsub = lane >> 3;
@@ -434,7 +435,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                     *reinterpret_cast<uint4*>(S.bext[w] + (r >> 3) * 256 + (r & 7) * 16 + 128) = make_uint4(0u, 0u, 0u, 0u);
                 }
             }
-            const int* list = P.cidx + ((size_t)bh * npairs + pair) * P.ccap;
+            const int* list = P.cidx + ((size_t)bh * npairs + lpair) * P.ccap;
             auto vals = [&](const int (&jv)[4], float (&bv)[4], int (&ev)[4]) {
 #pragma unroll
                 for (int t = 0; t < 4; ++t) {
@@ -863,6 +864,7 @@ __global__ void __launch_bounds__(256) compact_lists_kernel(const int32_t* __res
     __shared__ int wcount[2][8];
     const int list = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int bh = list / npairs, pair = list % npairs, i0 = q_off + pair * 256;
+    if (!causal && pair != 0) return;                    // non-causal: the head's one list is that of its first pair
     const int32_t* e = expiry + (size_t)bh * L;
     int* out = cidx + (size_t)list * cap;
     const int jend = causal ? min(L, i0 + 256) : L;     // non-causal: key j is kept by the rows i < expiry[j], whatever j
