@@ -182,14 +182,22 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                 emax = max(emax, __shfl_xor_sync(0xffffffffu, emax, o));
             }
             if (emax > 0) {
+                // The walk goes BACKWARDS, from the last row that keeps one of the keys to the first key's row: the CTAs
+                // of neighbouring entries of the permutation share their expiry band, i.e. the END of their walks, and start
+                // about together, so walking down from there they pass the same query rows (the Q / dO tiles they load, the
+                // dQ accumulator rows they add to) at about the same time, while those are in L2; walking up, each from its
+                // own first key, they passed a row at times spread over the life of the whole group.
                 const int g = hq_c % P.G, q0 = jmin / 128, q1 = (emax - 1) / 128;
-                for (int qt = q0 + lane; qt <= q1; qt += 32) {
-                    const int pos = 2 * (qt - q0);
-                    if (pos < kMaxSteps) S.sched[pos] = (uint16_t)((g << 11) | (qt << 1));
-                    if (pos + 1 < kMaxSteps) S.sched[pos + 1] = (uint16_t)((g << 11) | (qt << 1) | 1);
-                }
                 n = 2 * (q1 - q0 + 1);
                 if (q1 * 128 + 64 >= P.L) n -= 1;       // the last tile has one 64-row step only
+                n = min(n, kMaxSteps);
+                for (int qt = q0 + lane; qt <= q1; qt += 32) {
+#pragma unroll
+                    for (int hf = 0; hf < 2; ++hf) {
+                        const int pos = n - 1 - (2 * (qt - q0) + hf);
+                        if (pos >= 0) S.sched[pos] = (uint16_t)((g << 11) | (qt << 1) | hf);
+                    }
+                }
             }
         } else {
         for (int g = 0; g < P.G; ++g) {
