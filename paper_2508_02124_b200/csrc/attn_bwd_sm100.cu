@@ -786,10 +786,9 @@ int launch_tc_bwd(const Prob& P, const void* Q, const void* K, const void* V, co
         int sg = gx;
         {
             const double per_entry = (double)(compact ? 1 : P.G) * P.L * P.d * 8;     // token-compacted mode: an entry is one query head
-            // (token-compacted mode with long sequences, a head's rows above 12 MB: half of that was the best of 40, 80, 160
-            //  and 320 MB, 1.77 against 1.88 ms at L = 16384 with 32 heads; the CTAs of a head walk rows far apart and also add
-            //  into the fp32 dK / dV accumulators. At L = 8192 the larger group is the better one by 2 to 4 %.)
-            int want = (int)((compact && per_entry >= 12e6 ? 80.0 : 160.0) * 1024 * 1024 / per_entry);
+            // (token-compacted mode, eight heads at L = 16384: 1.69 ms against 1.74 with four and 1.82 with sixteen, once the
+            //  CTAs walk backwards; with the forward walk four at a time was the best, 1.77 against 1.88)
+            int want = (int)(160.0 * 1024 * 1024 / per_entry);
             want = want < 1 ? 1 : want;
             for (sg = want < gx ? want : gx; gx % sg; --sg) {}
         }
